@@ -1,0 +1,178 @@
+"""Declarative descriptions of fused operator chains and their seeded synthetic inputs.
+
+A ``Chain`` is data only (producer kind, sizes, ordered epilogue ops, reduction); the CPU oracle
+and the CUDA binding each interpret it with their own code.  ``make_inputs`` draws the tensors.
+
+The five benchmark workloads C1..C5 stand in for composed-operator problems of the kind the paper
+evaluates (Level-2 style chains: a contraction or a memory-bound pass, an elementwise epilogue and
+an optional row / channel reduction); the paper prints no shapes, so the shapes are the fixed
+synthetic configurations of this repository.  Dense random data; no sparsity or structure.
+
+Reading of "N(0, s)": ``s`` is the standard deviation (primary).  ``variant="var"`` re-reads it as a
+variance, which makes GEMM outputs O(1) so that clamps fire and softmax rows are far from uniform.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field, replace
+from typing import List, Tuple
+
+import numpy as np
+
+from . import rng
+
+
+@dataclass(frozen=True)
+class Chain:
+    name: str
+    producer: str                 # "elementwise" | "gemm_nt" | "conv2d_nhwc"
+    in_dtype: str                 # "f32" | "bf16"  storage of inputs[0] (and inputs[1] for contractions)
+    out_dtype: str                # storage of the main output (reductions other than softmax are f32)
+    M: int = 0                    # elementwise: rows; gemm: rows of A
+    N: int = 0                    # elementwise: cols; gemm: rows of B
+    K: int = 0
+    batch: int = 0                # conv only from here
+    H: int = 0
+    W: int = 0
+    Cin: int = 0
+    Cout: int = 0
+    R: int = 3
+    S: int = 3
+    stride: int = 1
+    pad: int = 1
+    # ops: ("bias_n", i) ("affine_n", i, j) ("relu",) ("gelu_tanh",) ("scale", f) ("clamp", lo, hi)
+    #      ("add_tensor", i)   -- i, j index the input list
+    ops: Tuple[tuple, ...] = ()
+    reduce: str = "none"          # "none" | "row_logsumexp" | "row_softmax" | "global_avgpool"
+    store_main: bool = True
+    # (tag, dtype, shape, dist, p0, p1) per input, in input order
+    input_recipe: Tuple[tuple, ...] = field(default=(), compare=False)
+
+    @property
+    def OH(self) -> int:
+        return (self.H + 2 * self.pad - self.R) // self.stride + 1
+
+    @property
+    def OW(self) -> int:
+        return (self.W + 2 * self.pad - self.S) // self.stride + 1
+
+    def flops(self) -> float:
+        if self.producer == "gemm_nt":
+            return 2.0 * self.M * self.N * self.K
+        if self.producer == "conv2d_nhwc":
+            return 2.0 * self.batch * self.OH * self.OW * self.Cout * self.R * self.S * self.Cin
+        return 0.0
+
+
+def _size(dtype: str) -> int:
+    return 4 if dtype == "f32" else 2
+
+
+def gemm_bias_relu_f32(M=256, N=256, K=256, variant="std") -> Chain:
+    s = 1.0 / K if variant == "std" else (1.0 / K) ** 0.5
+    return Chain("gemm_f32_bias_relu", "gemm_nt", "f32", "f32", M=M, N=N, K=K,
+                 ops=(("bias_n", 2), ("relu",)),
+                 input_recipe=(("X", "f32", (M, K), "normal", 0.0, s),
+                               ("W", "f32", (N, K), "normal", 0.0, s),
+                               ("b", "f32", (N,), "uniform", -0.1, 0.1)))
+
+
+def affine_gelu_residual_lse(M=16384, N=4096) -> Chain:
+    return Chain("ew_affine_gelu_add_lse", "elementwise", "bf16", "bf16", M=M, N=N,
+                 ops=(("affine_n", 1, 2), ("gelu_tanh",), ("add_tensor", 3)),
+                 reduce="row_logsumexp", store_main=True,
+                 input_recipe=(("x", "bf16", (M, N), "normal", 0.0, 1.0),
+                               ("gamma", "bf16", (N,), "normal", 1.0, 0.1),
+                               ("beta", "bf16", (N,), "normal", 0.0, 0.1),
+                               ("r", "bf16", (M, N), "normal", 0.0, 1.0)))
+
+
+def gemm_bias_gelu_scale_clamp(M=8192, N=8192, K=4096, variant="std") -> Chain:
+    s = K ** -0.5 if variant == "std" else K ** -0.25
+    return Chain("gemm_bf16_bias_gelu_scale_clamp", "gemm_nt", "bf16", "bf16", M=M, N=N, K=K,
+                 ops=(("bias_n", 2), ("gelu_tanh",), ("scale", 0.5), ("clamp", -1.0, 1.0)),
+                 input_recipe=(("A", "bf16", (M, K), "normal", 0.0, s),
+                               ("B", "bf16", (N, K), "normal", 0.0, s),
+                               ("bias", "bf16", (N,), "uniform", -0.1, 0.1)))
+
+
+def gemm_softmax(M=4096, N=4096, K=4096, variant="std") -> Chain:
+    s = K ** -0.5 if variant == "std" else K ** -0.25
+    return Chain("gemm_bf16_row_softmax", "gemm_nt", "bf16", "bf16", M=M, N=N, K=K,
+                 ops=(), reduce="row_softmax", store_main=False,
+                 input_recipe=(("A", "bf16", (M, K), "normal", 0.0, s),
+                               ("B", "bf16", (N, K), "normal", 0.0, s)))
+
+
+def conv_bias_relu_avgpool(batch=32, H=56, W=56, Cin=256, Cout=256, R=3, S=3, stride=1, pad=1) -> Chain:
+    s = (R * S * Cin) ** -0.5
+    return Chain("conv_bf16_bias_relu_avgpool", "conv2d_nhwc", "bf16", "f32",
+                 batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, stride=stride, pad=pad,
+                 ops=(("bias_n", 2), ("relu",)), reduce="global_avgpool", store_main=False,
+                 input_recipe=(("in", "bf16", (batch, H, W, Cin), "normal", 0.0, 1.0),
+                               ("Wt", "bf16", (Cout, R, S, Cin), "normal", 0.0, s),
+                               ("bias", "bf16", (Cout,), "uniform", -0.1, 0.1)))
+
+
+#: The five benchmark configurations, in the order the benchmark numbers them.
+CONFIGS = {
+    "C1": gemm_bias_relu_f32,
+    "C2": affine_gelu_residual_lse,
+    "C3": gemm_bias_gelu_scale_clamp,
+    "C4": gemm_softmax,
+    "C5": conv_bias_relu_avgpool,
+}
+
+
+def make_inputs(chain: Chain, seed: int = 0) -> List[np.ndarray]:
+    """Draw every input of ``chain`` (float32 arrays, or uint16 bf16 bit patterns)."""
+    out = []
+    for tag, dtype, shape, dist, p0, p1 in chain.input_recipe:
+        key = f"{chain.name}/{tag}"
+        if dist == "normal":
+            a = rng.normal_f32(seed, key, shape, p0, p1)
+        elif dist == "uniform":
+            a = rng.uniform_f32(seed, key, shape, p0, p1)
+        elif dist == "int":
+            a = rng.integers_f32(seed, key, shape, int(p0), int(p1))
+        else:
+            raise ValueError(dist)
+        out.append(rng.store(a, dtype))
+    return out
+
+
+def with_integer_inputs(chain: Chain, lo: int = -4, hi: int = 4) -> Chain:
+    """Same chain with the two contraction operands drawn as small integers (exact in bf16 and in
+    fp32 accumulation), which makes every correct contraction agree bit for bit."""
+    rec = list(chain.input_recipe)
+    for i in range(min(2, len(rec))):
+        tag, dtype, shape, _, _, _ = rec[i]
+        rec[i] = (tag, dtype, shape, "int", lo, hi)
+    return replace(chain, input_recipe=tuple(rec))
+
+
+def input_bytes(chain: Chain) -> int:
+    return sum(int(np.prod(shape)) * _size(dtype) for _, dtype, shape, *_ in chain.input_recipe)
+
+
+def output_shapes(chain: Chain):
+    """[(role, dtype, shape)] of the outputs, in output order: main first (if stored), then the reduction."""
+    outs = []
+    if chain.producer == "conv2d_nhwc":
+        main_shape = (chain.batch, chain.OH, chain.OW, chain.Cout)
+    else:
+        main_shape = (chain.M, chain.N)
+    if chain.reduce == "row_softmax":
+        outs.append(("reduce", chain.out_dtype, main_shape))
+        return outs
+    if chain.store_main:
+        outs.append(("main", chain.out_dtype, main_shape))
+    if chain.reduce == "row_logsumexp":
+        outs.append(("reduce", "f32", (chain.M,)))
+    elif chain.reduce == "global_avgpool":
+        outs.append(("reduce", "f32", (chain.batch, chain.Cout)))
+    return outs
+
+
+def algorithmic_bytes(chain: Chain) -> int:
+    """Each input read once plus each output written once."""
+    return input_bytes(chain) + sum(int(np.prod(s)) * _size(d) for _, d, s in output_shapes(chain))

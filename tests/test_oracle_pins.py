@@ -1,0 +1,279 @@
+"""Pins for the CPU oracle: closed forms, invariants, library routines on special cases, exact
+brute force on tiny shapes.  CPU only.  A plausible mistake in the oracle (dropped term, wrong
+sign or index, transposed operand, swapped op order) fails at least one test here."""
+import math
+import os
+from dataclasses import replace
+
+import mpmath as mp
+import numpy as np
+import pytest
+import torch
+
+from fc_inputs import rng, workloads as wl
+from tests import brute
+
+mp.mp.dps = 50
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand(shape, seed, lo=-1.0, hi=1.0):
+    return np.random.default_rng(seed).uniform(lo, hi, size=shape)
+
+
+# ----------------------------------------------------------------------------- widening
+def test_widen_bf16_all_patterns(orc):
+    bits = np.arange(65536, dtype=np.uint16)
+    got = orc.widen(bits)
+    want = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    ok = (got == want) | (np.isnan(got) & np.isnan(want))
+    assert ok.all()
+
+
+def test_widen_f32_exact(orc):
+    a = np.array([0.1, -3.5, 1e-40, 3e38, -0.0], dtype=np.float32)
+    assert np.array_equal(orc.widen(a), a.astype(np.float64))
+
+
+# ----------------------------------------------------------------------------- GEMM NT
+def test_gemm_identity_weight_returns_x(orc):
+    X = _rand((7, 5), 1)
+    assert np.array_equal(orc.gemm_nt(X, np.eye(5)), X)
+
+
+def test_gemm_zero_weight_gives_bias_chain(orc):
+    ch = wl.gemm_bias_relu_f32(6, 9, 5)
+    X, W, b = wl.make_inputs(ch, 3)
+    out = orc.run_chain(ch, [X, np.zeros_like(W), b])["main"]
+    want = np.maximum(b.astype(np.float64), 0.0)
+    assert np.array_equal(out, np.broadcast_to(want, (6, 9)))
+
+
+def test_gemm_rank_one(orc):
+    a = np.arange(1, 8, dtype=np.float64)          # M=7
+    b = np.arange(-2, 3, dtype=np.float64)         # N=5
+    K = 11
+    A = np.repeat(a[:, None], K, 1)
+    B = np.repeat(b[:, None], K, 1)
+    assert np.array_equal(orc.gemm_nt(A, B), K * np.outer(a, b))
+
+
+def test_gemm_one_hot_selects_entry(orc):
+    # non-square everywhere: a transposed operand or swapped M/N index cannot pass
+    M, N, K = 4, 6, 9
+    A = np.zeros((M, K)); B = _rand((N, K), 2)
+    A[2, 7] = 1.0
+    V = orc.gemm_nt(A, B)
+    assert np.array_equal(V[2], B[:, 7]) and np.count_nonzero(V[[0, 1, 3]]) == 0
+
+
+def test_gemm_small_integers_exact(orc):
+    r = np.random.default_rng(5)
+    A = r.integers(-8, 9, size=(33, 70)).astype(np.float64)
+    B = r.integers(-8, 9, size=(19, 70)).astype(np.float64)
+    want = A.astype(np.int64) @ B.astype(np.int64).T
+    assert np.array_equal(orc.gemm_nt(A, B), want.astype(np.float64))
+
+
+def test_gemm_matches_library_matmul(orc):
+    A = _rand((37, 129), 6); B = _rand((23, 129), 7)
+    np.testing.assert_allclose(orc.gemm_nt(A, B), A @ B.T, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (3, 5, 2), (7, 5, 9)])
+def test_gemm_chain_vs_exact_brute_force(orc, M, N, K):
+    ch = wl.gemm_bias_gelu_scale_clamp(M, N, K, variant="var")
+    ins = wl.make_inputs(ch, 11)
+    got = orc.run_chain(ch, ins)["main"]
+    want = brute.run_chain(ch, ins)["main"]
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- conv
+def _delta_weight(C, r, s):
+    w = np.zeros((C, 3, 3, C))
+    for c in range(C):
+        w[c, r, s, c] = 1.0
+    return w
+
+
+def test_conv_centre_delta_is_identity(orc):
+    x = _rand((2, 5, 7, 3), 8)
+    assert np.array_equal(orc.conv2d_nhwc(x, _delta_weight(3, 1, 1), 1, 1), x)
+
+
+def test_conv_shifted_delta_pins_direction_and_padding(orc):
+    x = _rand((1, 5, 7, 2), 9)
+    y = orc.conv2d_nhwc(x, _delta_weight(2, 0, 0), 1, 1)     # out[h][w] = in[h-1][w-1]
+    assert np.array_equal(y[:, 1:, 1:, :], x[:, :-1, :-1, :])
+    assert np.count_nonzero(y[:, 0, :, :]) == 0 and np.count_nonzero(y[:, :, 0, :]) == 0
+    y2 = orc.conv2d_nhwc(x, _delta_weight(2, 2, 1), 1, 1)    # out[h][w] = in[h+1][w]
+    assert np.array_equal(y2[:, :-1, :, :], x[:, 1:, :, :]) and np.count_nonzero(y2[:, -1]) == 0
+
+
+def test_conv_all_ones_counts_valid_taps(orc):
+    Cin, H, W = 4, 6, 5
+    y = orc.conv2d_nhwc(np.ones((1, H, W, Cin)), np.ones((2, 3, 3, Cin)), 1, 1)
+    assert y[0, 2, 2, 0] == 9 * Cin and y[0, 0, 2, 1] == 6 * Cin and y[0, 0, 0, 0] == 4 * Cin
+    assert y[0, H - 1, W - 1, 1] == 4 * Cin
+    pooled = orc.global_avgpool(y)
+    want = Cin * (3 * H - 2) * (3 * W - 2) / (H * W)
+    np.testing.assert_allclose(pooled, want, rtol=1e-15)
+
+
+def test_pool_closed_form_at_benchmark_shape(orc):
+    # all-ones 56x56x256 image and weights: mean over pixels of Cin * (#valid taps)
+    H = W = 56
+    taps = np.full((H, W), 9.0); taps[0, :] = taps[-1, :] = 6; taps[:, 0] = taps[:, -1] = 6
+    taps[0, 0] = taps[0, -1] = taps[-1, 0] = taps[-1, -1] = 4
+    V = (256.0 * taps)[None, :, :, None].repeat(3, axis=3)
+    got = orc.global_avgpool(np.ascontiguousarray(V))
+    assert got.shape == (1, 3)
+    np.testing.assert_allclose(got, 256.0 * (3 * H - 2) * (3 * W - 2) / (H * W), rtol=1e-15)
+    np.testing.assert_allclose(got, 2249.469387755102, rtol=1e-15)
+
+
+@pytest.mark.parametrize("stride,pad,H,W", [(1, 1, 6, 5), (2, 1, 7, 8), (1, 0, 5, 5), (2, 0, 6, 9)])
+def test_conv_matches_library_conv(orc, stride, pad, H, W):
+    x = _rand((2, H, W, 3), 10); w = _rand((4, 3, 3, 3), 11)
+    got = orc.conv2d_nhwc(x, w, stride, pad)
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2),
+                                     torch.from_numpy(w).permute(0, 3, 1, 2), stride=stride, padding=pad)
+    np.testing.assert_allclose(got, ref.permute(0, 2, 3, 1).numpy(), rtol=0, atol=1e-13)
+
+
+def test_conv_1x1_image_reduces_to_gemm(orc):
+    x = _rand((5, 1, 1, 6), 12); w = _rand((4, 3, 3, 6), 13)
+    got = orc.conv2d_nhwc(x, w, 1, 1).reshape(5, 4)
+    want = orc.gemm_nt(np.ascontiguousarray(x.reshape(5, 6)), np.ascontiguousarray(w[:, 1, 1, :]))
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-15)
+
+
+def test_conv_chain_vs_exact_brute_force(orc):
+    ch = wl.conv_bias_relu_avgpool(batch=2, H=4, W=3, Cin=3, Cout=2)
+    ins = wl.make_inputs(ch, 4)
+    got = orc.run_chain(ch, ins)
+    want = brute.run_chain(ch, ins)
+    np.testing.assert_allclose(got["main"], want["main"], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(got["reduce"], want["reduce"], rtol=0, atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- elementwise ops
+def test_relu_scale_clamp_exhaustive_bf16(orc):
+    bits = np.arange(65536, dtype=np.uint16)
+    v = orc.widen(bits)
+    v = v[np.isfinite(v)]
+    a = v.copy(); orc.apply_op(a, ("relu",), [])
+    assert np.array_equal(a, np.where(v < 0, 0.0, v))
+    a = v.copy(); orc.apply_op(a, ("scale", 0.5), [])
+    assert np.array_equal(a, v * 0.5)
+    a = v.copy(); orc.apply_op(a, ("clamp", -1.0, 1.0), [])
+    assert np.array_equal(a, np.clip(v, -1.0, 1.0))
+    assert a.max() == 1.0 and a.min() == -1.0
+
+
+def test_bias_affine_add_broadcast_axis(orc):
+    V = _rand((3, 4), 14); g = np.array([1., 2., 3., 4.]); b = np.array([10., 20., 30., 40.])
+    a = V.copy(); orc.apply_op(a, ("bias_n", 0), [b]); assert np.array_equal(a, V + b[None, :])
+    a = V.copy(); orc.apply_op(a, ("affine_n", 0, 1), [g, b]); assert np.array_equal(a, V * g[None, :] + b[None, :])
+    T = _rand((3, 4), 15)
+    a = V.copy(); orc.apply_op(a, ("add_tensor", 0), [T]); assert np.array_equal(a, V + T)
+
+
+def test_gelu_tanh_values_and_identities(orc):
+    pts = np.array([-6.0, -3.0, -2.0, -1.0, -0.5, -1e-3, 0.0, 1e-3, 0.5, 1.0, 2.0, 3.0, 6.0, 11.0])
+    g = pts.copy(); orc.apply_op(g, ("gelu_tanh",), [])
+    want = np.array([float(brute.gelu_tanh(mp.mpf(float(v)))) for v in pts])
+    # 1 + tanh(.) cancels near v = -6 in fp64: absolute error there is ~1e-17 * |v|
+    np.testing.assert_allclose(g, want, rtol=1e-14, atol=1e-15)
+    assert g[6] == 0.0
+    # G(v) - G(-v) = v because tanh is odd
+    sym = np.array([0.3, 1.0, 2.5, 4.0]); gp = sym.copy(); gm = -sym
+    orc.apply_op(gp, ("gelu_tanh",), []); orc.apply_op(gm, ("gelu_tanh",), [])
+    np.testing.assert_allclose(gp - gm, sym, rtol=1e-14)
+    # limits and a library routine
+    assert abs(g[-1] - 11.0) < 1e-12 and abs(g[0]) < 1e-9
+    v = _rand((1000,), 16, -5, 5)
+    a = v.copy(); orc.apply_op(a, ("gelu_tanh",), [])
+    ref = torch.nn.functional.gelu(torch.from_numpy(v), approximate="tanh").numpy()
+    np.testing.assert_allclose(a, ref, rtol=0, atol=1e-14)
+
+
+def test_op_order_is_respected(orc):
+    # clamp(scale(v)) differs from scale(clamp(v)); relu(bias) differs from bias(relu)
+    v = np.array([[3.0, -3.0]])
+    a = v.copy(); orc.apply_op(a, ("scale", 0.5), []); orc.apply_op(a, ("clamp", -1.0, 1.0), [])
+    assert np.array_equal(a, [[1.0, -1.0]])
+    ch = replace(wl.gemm_bias_relu_f32(1, 2, 1), ops=(("relu",), ("bias_n", 2)))
+    out = orc.run_chain(ch, [np.array([[1.0]], np.float32), np.array([[-2.0], [2.0]], np.float32),
+                             np.array([-1.0, -1.0], np.float32)])["main"]
+    assert np.array_equal(out, [[-1.0, 1.0]])
+
+
+# ----------------------------------------------------------------------------- reductions
+def test_lse_size_one_is_identity_golden(orc):
+    vals = [float(l) for l in open(os.path.join(GOLDEN, "lse_size_one.txt")) if l.strip() and not l.startswith("#")]
+    V = np.array(vals).reshape(-1, 1)
+    assert np.array_equal(orc.row_logsumexp(V), np.array(vals))
+
+
+def test_lse_closed_forms(orc):
+    N = 4096
+    out = orc.row_logsumexp(np.full((2, N), 2.5))
+    np.testing.assert_allclose(out, 2.5 + 8.317766166719343, rtol=1e-15)
+    v = _rand((5, 300), 17, -4, 4)
+    base = orc.row_logsumexp(v)
+    for c in (1e4, -1e4, 3.0):
+        np.testing.assert_allclose(orc.row_logsumexp(v + c), base + c, rtol=1e-13)
+    assert np.all(base >= v.max(1)) and np.all(base <= v.max(1) + math.log(300))
+    dom = np.full((1, 50), -800.0); dom[0, 17] = 42.0
+    assert orc.row_logsumexp(dom)[0] == 42.0
+    want = [float(mp.log(mp.fsum([mp.exp(mp.mpf(float(x))) for x in row]))) for row in v]
+    np.testing.assert_allclose(base, want, rtol=1e-14)
+    np.testing.assert_allclose(base, torch.logsumexp(torch.from_numpy(v), 1).numpy(), rtol=1e-14)
+
+
+def test_softmax_properties(orc):
+    v = _rand((6, 257), 18, -6, 6)
+    P = orc.row_softmax(v)
+    assert np.abs(P.sum(1) - 1).max() <= 1e-12
+    np.testing.assert_allclose(orc.row_softmax(v + 1234.5), P, rtol=1e-11)
+    np.testing.assert_allclose(orc.row_softmax(np.full((1, 64), -3.0)), 1 / 64, rtol=1e-15)
+    np.testing.assert_allclose(np.log(P), v - orc.row_logsumexp(v)[:, None], rtol=0, atol=1e-12)
+    order = np.argsort(v[0]); assert np.all(np.diff(P[0][order]) >= 0)
+    np.testing.assert_allclose(P, torch.softmax(torch.from_numpy(v), 1).numpy(), rtol=1e-13)
+
+
+def test_avgpool_properties(orc):
+    V = _rand((2, 3, 4, 5), 19); U = _rand((2, 3, 4, 5), 20)
+    np.testing.assert_allclose(orc.global_avgpool(np.full((2, 3, 4, 5), 7.25)), 7.25, rtol=1e-15)
+    np.testing.assert_allclose(orc.global_avgpool(2 * V + U), 2 * orc.global_avgpool(V) + orc.global_avgpool(U), atol=1e-15)
+    np.testing.assert_allclose(orc.global_avgpool(V), V.mean(axis=(1, 2)), atol=1e-15)
+    # pixel/channel index not swapped: one hot pixel in one channel
+    Z = np.zeros((1, 3, 4, 5)); Z[0, 2, 1, 3] = 12.0
+    want = np.zeros((1, 5)); want[0, 3] = 1.0
+    assert np.array_equal(orc.global_avgpool(Z), want)
+
+
+# ----------------------------------------------------------------------------- whole chains
+def test_all_five_patterns_vs_brute_force(orc):
+    chains = [wl.gemm_bias_relu_f32(3, 5, 7, variant="var"),
+              wl.affine_gelu_residual_lse(3, 9),
+              wl.gemm_bias_gelu_scale_clamp(5, 3, 4, variant="var"),
+              wl.gemm_softmax(3, 7, 5, variant="var"),
+              wl.conv_bias_relu_avgpool(batch=1, H=3, W=3, Cin=2, Cout=3)]
+    for ch in chains:
+        ins = wl.make_inputs(ch, 21)
+        got, want = orc.run_chain(ch, ins), brute.run_chain(ch, ins)
+        for k in want:
+            np.testing.assert_allclose(got[k], want[k], rtol=1e-13, atol=1e-14, err_msg=f"{ch.name}:{k}")
+
+
+def test_elementwise_chain_matches_library_sequence(orc):
+    ch = wl.affine_gelu_residual_lse(17, 130)
+    ins = wl.make_inputs(ch, 22)
+    x, g, b, r = [torch.from_numpy(rng.bf16_bits_to_f32(a)).double() for a in ins]
+    y = torch.nn.functional.gelu(x * g + b, approximate="tanh") + r
+    got = orc.run_chain(ch, ins)
+    np.testing.assert_allclose(got["main"], y.numpy(), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(got["reduce"], torch.logsumexp(y, 1).numpy(), rtol=1e-13)
