@@ -1,0 +1,175 @@
+/*
+ * fc.h -- C ABI of the fused-chain library for NVIDIA B200 (sm_100a).
+ *
+ * A "chain" is what the paper's agent produces when it fuses a PyTorch operator sequence into
+ * one CUDA kernel (composed-operator problems, "Level 2"; the paper's fusion rationale is to
+ * remove global-memory round trips and extra launches between a producer and its epilogue):
+ *
+ *     producer  ->  ordered elementwise epilogue ops  ->  optional row / channel reduction
+ *
+ *   producer   ELEMENTWISE  v[m][n] = x[m][n]
+ *              GEMM_NT      v[m][n] = sum_k A[m][k] * B[n][k]          (B stored [N x K] row-major,
+ *                           the "weight is [out_features x in_features]" convention of the paper's
+ *                           appendix GEMM / linear-layer kernels), fp32 accumulation
+ *              CONV2D_NHWC  v[b][oh][ow][co] = sum_{r,s,ci} in[b][oh*stride-pad+r][ow*stride-pad+s][ci]
+ *                           * W[co][r][s][ci]   (cross-correlation, zero padding, floor output size,
+ *                           as in the paper's appendix convolution kernel; layout restated for NHWC)
+ *   ops        bias over the last index, per-column affine, ReLU, tanh-GELU, scalar scale, clamp,
+ *              add a tensor of the output's shape (bias -> ReLU -> scale is the paper's appendix
+ *              epilogue; the others are named by this repository's benchmark configurations)
+ *   reduction  row logsumexp (its size-one case is the identity the paper's Q18 analysis uses),
+ *              row softmax, global average pool over (oh, ow)
+ *
+ * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
+ * allocates device memory and never synchronises; it enqueues at most two memsets and one or two
+ * kernels on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
+ *
+ * Pointers.  Unless a function says "host", every fc_tensor.ptr is a DEVICE pointer.
+ *
+ * Layout.  Row-major contiguous only (stride[] must describe exactly that, in elements).
+ *   GEMM_NT: inputs[0] = A [M,K], inputs[1] = B [N,K].  CONV2D_NHWC: inputs[0] = image
+ *   [batch,H,W,Cin], inputs[1] = weights [Cout,R,S,Cin].  ELEMENTWISE: inputs[0] = x [M,N].
+ *   Further inputs are the vectors ([N] or [Cout]) and tensors that fc_op.in0 / in1 index.
+ *   Outputs, in order: the main output (if store_main, or if reduce == ROW_SOFTMAX, whose
+ *   probabilities take the main output's place), then the reduction (LOGSUMEXP: f32 [M];
+ *   GLOBAL_AVGPOOL: f32 [batch,Cout]).
+ *
+ * Alignment.  Base pointers of bf16 operands of GEMM / CONV must be 16-byte aligned and K (GEMM)
+ * or Cin (CONV) a multiple of 8; violations return FC_ERR_ALIGNMENT.  Other tensors need only the
+ * natural alignment of their element type (vector access is used when 16-byte alignment holds).
+ *
+ * Errors.  Return code only: nothing is thrown or printed, the process is never aborted.  Chains
+ * outside the supported patterns return FC_ERR_UNSUPPORTED; there is no CPU fallback and no other
+ * backend.  A device that is not compute capability 10.x returns FC_ERR_ARCH.  Device-side waits
+ * are bounded; if one expires the kernel records FC_ERR_TIMEOUT in a device status word, skips its
+ * remaining stores and exits; fc_get_async_status reports it.
+ *
+ * Threading.  fc_run may be called from several host threads.  The workspace set by
+ * fc_set_workspace is shared by all calls: launches that use it (ROW_SOFTMAX on a GEMM) must not
+ * overlap on the device.
+ */
+#ifndef FC_H_
+#define FC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FC_VERSION 1
+#define FC_MAX_OPS 8
+
+typedef enum {
+    FC_OK = 0,
+    FC_ERR_NULL = 1,          /* a required pointer is null                                   */
+    FC_ERR_INVALID_SPEC = 2,  /* struct_size / version / enum value / op operand index wrong  */
+    FC_ERR_UNSUPPORTED = 3,   /* well-formed chain that no kernel here implements             */
+    FC_ERR_SHAPE = 4,         /* a dimension < 1, or a tensor's shape does not fit the spec   */
+    FC_ERR_ALIGNMENT = 5,
+    FC_ERR_WORKSPACE = 6,     /* chain needs a workspace and none (or too small) was set      */
+    FC_ERR_ARCH = 7,
+    FC_ERR_CUDA = 8,          /* a CUDA runtime / driver call failed; see fc_last_error       */
+    FC_ERR_TIMEOUT = 9        /* a bounded device-side wait expired                           */
+} fc_status;
+
+typedef enum { FC_F32 = 0, FC_BF16 = 1 } fc_dtype;
+
+typedef enum { FC_PROD_ELEMENTWISE = 0, FC_PROD_GEMM_NT = 1, FC_PROD_CONV2D_NHWC = 2 } fc_producer;
+
+typedef enum {
+    FC_OP_BIAS_N = 0,     /* v += vec[in0][n]                      n = last (column / channel) index */
+    FC_OP_AFFINE_N = 1,   /* v  = v * vec[in0][n] + vec[in1][n]                                      */
+    FC_OP_RELU = 2,       /* v  = v < 0 ? 0 : v                                                      */
+    FC_OP_GELU_TANH = 3,  /* v  = 0.5 v (1 + tanh(sqrt(2/pi) (v + 0.044715 v^3)))                    */
+    FC_OP_SCALE = 4,      /* v *= f0                                                                 */
+    FC_OP_CLAMP = 5,      /* v  = min(max(v, f0), f1)                                                */
+    FC_OP_ADD_TENSOR = 6  /* v += tensor[in0][m][n]              same shape as the main output       */
+} fc_op_kind;
+
+typedef enum {
+    FC_RED_NONE = 0,
+    FC_RED_ROW_LOGSUMEXP = 1,   /* out[m] = max_n v + log sum_n exp(v - max)          */
+    FC_RED_ROW_SOFTMAX = 2,     /* p[m][n] = exp(v - max) / sum_n exp(v - max)         */
+    FC_RED_GLOBAL_AVGPOOL = 3   /* out[b][c] = mean over (oh, ow) of v[b][oh][ow][c]   */
+} fc_reduce;
+
+typedef struct {
+    int32_t kind;      /* fc_op_kind                       */
+    int32_t in0, in1;  /* indices into inputs[] (unused: 0) */
+    float f0, f1;
+} fc_op;
+
+typedef struct {
+    uint32_t struct_size;   /* sizeof(fc_chain_spec) */
+    uint32_t version;       /* FC_VERSION            */
+    int32_t producer;       /* fc_producer           */
+    int32_t in_dtype;       /* storage of inputs[0] (and inputs[1] for GEMM / CONV) */
+    int32_t acc_dtype;      /* FC_F32                */
+    int32_t out_dtype;      /* storage of the main output / softmax probabilities   */
+    int64_t M, N, K;        /* ELEMENTWISE: M rows x N cols; GEMM: M x N x K        */
+    int64_t batch, H, W, Cin, Cout, R, S, stride, pad;   /* CONV only              */
+    int32_t n_ops;
+    fc_op ops[FC_MAX_OPS];  /* applied in order      */
+    int32_t reduce;         /* fc_reduce             */
+    int32_t store_main;     /* also write the main output when a reduction exists   */
+} fc_chain_spec;
+
+typedef struct {
+    void* ptr;
+    int32_t dtype;          /* fc_dtype */
+    int32_t rank;
+    int64_t shape[4];
+    int64_t stride[4];      /* in elements; must be the contiguous row-major strides */
+} fc_tensor;
+
+/*
+ * Run one fused chain: the whole operator sequence described by `spec` in one pass over the data
+ * (the paper's fused-kernel launch, with raw pointers plus sizes as in its harness convention).
+ * All tensor pointers are device pointers on the current device; `cuda_stream` is a cudaStream_t
+ * (NULL = the legacy default stream).  Asynchronous.  Returns FC_OK once the work is enqueued.
+ */
+fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_inputs,
+                 fc_tensor* outputs, int n_outputs, void* cuda_stream);
+
+/*
+ * Same chain with HOST buffers: every inputs[i].ptr / outputs[i].ptr is a host pointer (pinned
+ * memory makes the copies asynchronous).  `staging` is a caller-owned DEVICE buffer of at least
+ * fc_staging_size() bytes into which inputs are copied (cudaMemcpyAsync on the stream), the chain
+ * runs there, and outputs are copied back.  Enqueues only; the caller synchronises the stream
+ * before reading the outputs.
+ */
+fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, int n_inputs,
+                      fc_tensor* host_outputs, int n_outputs, void* staging, size_t staging_bytes,
+                      void* cuda_stream);
+fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, int n_inputs,
+                          const fc_tensor* outputs, int n_outputs, size_t* bytes);
+
+/*
+ * Scratch memory.  Only GEMM_NT + ROW_SOFTMAX needs any (per-tile row maxima and sums plus
+ * per-panel arrival counters for the cross-tile online max/sum merge).  fc_workspace_size reports
+ * the bytes a spec needs (0 for the other chains); fc_set_workspace registers a caller-owned DEVICE
+ * buffer (256-byte aligned) for the current device, used by later fc_run calls until replaced.
+ */
+fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes);
+fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
+
+/*
+ * Synchronises `cuda_stream`, then reads and clears the device status word of the current
+ * device.  Returns FC_OK, FC_ERR_TIMEOUT (a bounded device-side wait expired in some launch since
+ * the last call) or FC_ERR_CUDA.
+ */
+fc_status fc_get_async_status(void* cuda_stream);
+
+/* Number of kernels this library has launched in this process (all devices, all threads). */
+uint64_t fc_launch_count(void);
+
+const char* fc_status_string(fc_status s);
+const char* fc_last_error(void);   /* thread-local text of the last failure in this thread */
+int fc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FC_H_ */

@@ -1,0 +1,263 @@
+"""ctypes binding with the same names as the C ABI (include/fc.h).
+
+Argument marshalling only: every step of a chain runs inside the CUDA library.  torch is used for
+device memory and streams.  There is no fallback: if the built library is missing, importing this
+module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(PKG, "libfc.so")
+
+FC_F32, FC_BF16 = 0, 1
+_PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2}
+_OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6}
+_REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3}
+_DTYPE = {"f32": FC_F32, "bf16": FC_BF16}
+FC_MAX_OPS = 8
+
+
+class fc_op(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("in0", ctypes.c_int32), ("in1", ctypes.c_int32),
+                ("f0", ctypes.c_float), ("f1", ctypes.c_float)]
+
+
+class fc_chain_spec(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("version", ctypes.c_uint32),
+                ("producer", ctypes.c_int32), ("in_dtype", ctypes.c_int32),
+                ("acc_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+                ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("batch", ctypes.c_int64), ("H", ctypes.c_int64), ("W", ctypes.c_int64),
+                ("Cin", ctypes.c_int64), ("Cout", ctypes.c_int64), ("R", ctypes.c_int64),
+                ("S", ctypes.c_int64), ("stride", ctypes.c_int64), ("pad", ctypes.c_int64),
+                ("n_ops", ctypes.c_int32), ("ops", fc_op * FC_MAX_OPS),
+                ("reduce", ctypes.c_int32), ("store_main", ctypes.c_int32)]
+
+
+class fc_tensor(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("rank", ctypes.c_int32),
+                ("shape", ctypes.c_int64 * 4), ("stride", ctypes.c_int64 * 4)]
+
+
+class FcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = lib().fc_status_string(status).decode()
+        super().__init__(f"{where}: {name}: {fc_last_error()}")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_14293_b200.build` "
+                              "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        pt, ps = ctypes.POINTER(fc_tensor), ctypes.POINTER(fc_chain_spec)
+        L.fc_run.argtypes = [ps, pt, ctypes.c_int, pt, ctypes.c_int, ctypes.c_void_p]
+        L.fc_run.restype = ctypes.c_int
+        L.fc_run_host.argtypes = [ps, pt, ctypes.c_int, pt, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.fc_run_host.restype = ctypes.c_int
+        L.fc_staging_size.argtypes = [ps, pt, ctypes.c_int, pt, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
+        L.fc_staging_size.restype = ctypes.c_int
+        L.fc_workspace_size.argtypes = [ps, ctypes.POINTER(ctypes.c_size_t)]
+        L.fc_workspace_size.restype = ctypes.c_int
+        L.fc_set_workspace.argtypes = [ctypes.c_void_p, ctypes.c_size_t]
+        L.fc_set_workspace.restype = ctypes.c_int
+        L.fc_get_async_status.argtypes = [ctypes.c_void_p]
+        L.fc_get_async_status.restype = ctypes.c_int
+        L.fc_launch_count.restype = ctypes.c_uint64
+        L.fc_status_string.argtypes = [ctypes.c_int]
+        L.fc_status_string.restype = ctypes.c_char_p
+        L.fc_last_error.restype = ctypes.c_char_p
+        L.fc_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def fc_last_error() -> str:
+    return lib().fc_last_error().decode()
+
+
+def fc_version() -> int:
+    return int(lib().fc_version())
+
+
+def fc_launch_count() -> int:
+    return int(lib().fc_launch_count())
+
+
+def make_spec(chain) -> fc_chain_spec:
+    """Build an fc_chain_spec from a declarative chain description (any object with the fields
+    producer, in_dtype, out_dtype, M, N, K, batch, H, W, Cin, Cout, R, S, stride, pad, ops, reduce,
+    store_main; ops are tuples such as ("bias_n", 2) or ("clamp", -1.0, 1.0))."""
+    s = fc_chain_spec()
+    s.struct_size = ctypes.sizeof(fc_chain_spec)
+    s.version = 1
+    s.producer = _PRODUCER[chain.producer]
+    s.in_dtype = _DTYPE[chain.in_dtype]
+    s.acc_dtype = FC_F32
+    s.out_dtype = _DTYPE[chain.out_dtype]
+    for f in ("M", "N", "K", "batch", "H", "W", "Cin", "Cout", "R", "S", "stride", "pad"):
+        setattr(s, f, int(getattr(chain, f)))
+    s.n_ops = len(chain.ops)
+    for i, op in enumerate(chain.ops):
+        o = s.ops[i]
+        o.kind = _OPKIND[op[0]]
+        if op[0] in ("bias_n", "add_tensor"):
+            o.in0 = int(op[1])
+        elif op[0] == "affine_n":
+            o.in0, o.in1 = int(op[1]), int(op[2])
+        elif op[0] == "scale":
+            o.f0 = float(op[1])
+        elif op[0] == "clamp":
+            o.f0, o.f1 = float(op[1]), float(op[2])
+    s.reduce = _REDUCE[chain.reduce]
+    s.store_main = 1 if chain.store_main else 0
+    return s
+
+
+def _tensor_struct(t: torch.Tensor) -> fc_tensor:
+    ft = fc_tensor()
+    ft.ptr = t.data_ptr()
+    if t.dtype == torch.float32:
+        ft.dtype = FC_F32
+    elif t.dtype == torch.bfloat16:
+        ft.dtype = FC_BF16
+    else:
+        raise TypeError(f"unsupported dtype {t.dtype}")
+    if t.dim() > 4:
+        raise ValueError("rank > 4")
+    ft.rank = t.dim()
+    for i in range(t.dim()):
+        ft.shape[i] = t.shape[i]
+        ft.stride[i] = t.stride(i)
+    return ft
+
+
+def _tensor_array(ts: Sequence[torch.Tensor]):
+    arr = (fc_tensor * max(1, len(ts)))()
+    for i, t in enumerate(ts):
+        arr[i] = _tensor_struct(t)
+    return arr
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise FcError(status, where)
+
+
+def fc_run(spec: fc_chain_spec, inputs: Sequence[torch.Tensor], outputs: Sequence[torch.Tensor], stream=None) -> None:
+    """fc_run of the C ABI: device tensors in, device tensors out, enqueued on `stream`."""
+    _check(lib().fc_run(ctypes.byref(spec), _tensor_array(inputs), len(inputs), _tensor_array(outputs), len(outputs),
+                        _stream_handle(stream)), "fc_run")
+
+
+def fc_staging_size(spec, inputs, outputs) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().fc_staging_size(ctypes.byref(spec), _tensor_array(inputs), len(inputs), _tensor_array(outputs),
+                                 len(outputs), ctypes.byref(n)), "fc_staging_size")
+    return int(n.value)
+
+
+def fc_run_host(spec, host_inputs: Sequence[torch.Tensor], host_outputs: Sequence[torch.Tensor],
+                staging: torch.Tensor, stream=None) -> None:
+    """fc_run_host of the C ABI: host (ideally pinned) tensors in and out, `staging` a device byte buffer."""
+    _check(lib().fc_run_host(ctypes.byref(spec), _tensor_array(host_inputs), len(host_inputs),
+                             _tensor_array(host_outputs), len(host_outputs), ctypes.c_void_p(staging.data_ptr()),
+                             staging.numel() * staging.element_size(), _stream_handle(stream)), "fc_run_host")
+
+
+def fc_workspace_size(spec) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().fc_workspace_size(ctypes.byref(spec), ctypes.byref(n)), "fc_workspace_size")
+    return int(n.value)
+
+
+def fc_set_workspace(buf: Optional[torch.Tensor]) -> None:
+    if buf is None:
+        _check(lib().fc_set_workspace(None, 0), "fc_set_workspace")
+    else:
+        _check(lib().fc_set_workspace(ctypes.c_void_p(buf.data_ptr()), buf.numel() * buf.element_size()), "fc_set_workspace")
+
+
+def fc_get_async_status(stream=None) -> None:
+    _check(lib().fc_get_async_status(_stream_handle(stream)), "fc_get_async_status")
+
+
+# --------------------------------------------------------------------------- conveniences
+_TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+_workspace = {}
+
+
+def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
+    """Stored numpy tensor (float32, or uint16 bf16 bit patterns) -> torch tensor on `device`."""
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(device)
+    return torch.from_numpy(a).to(device)
+
+
+def output_tensors(chain, device="cuda", pinned=False) -> List[torch.Tensor]:
+    """Allocate (uninitialised) output tensors for `chain`, in the ABI's output order."""
+    if chain.producer == "conv2d_nhwc":
+        OH = (chain.H + 2 * chain.pad - chain.R) // chain.stride + 1
+        OW = (chain.W + 2 * chain.pad - chain.S) // chain.stride + 1
+        main_shape = (chain.batch, OH, OW, chain.Cout)
+    else:
+        main_shape = (chain.M, chain.N)
+    kw = dict(device=device, pin_memory=pinned) if device == "cpu" else dict(device=device)
+    outs = []
+    if chain.reduce == "row_softmax" or chain.store_main:
+        outs.append(torch.empty(main_shape, dtype=_TORCH_DT[chain.out_dtype], **kw))
+    if chain.reduce == "row_logsumexp":
+        outs.append(torch.empty((chain.M,), dtype=torch.float32, **kw))
+    elif chain.reduce == "global_avgpool":
+        outs.append(torch.empty((chain.batch, chain.Cout), dtype=torch.float32, **kw))
+    return outs
+
+
+def ensure_workspace(spec) -> None:
+    """Register a torch-owned workspace large enough for `spec` on the current device."""
+    need = fc_workspace_size(spec)
+    if need == 0:
+        return
+    dev = torch.cuda.current_device()
+    cur = _workspace.get(dev)
+    if cur is None or cur.numel() < need:
+        cur = torch.empty(need, dtype=torch.uint8, device=f"cuda:{dev}")
+        _workspace[dev] = cur
+        fc_set_workspace(cur)
+
+
+def run_chain(chain, inputs: Sequence[torch.Tensor], outputs: Optional[Sequence[torch.Tensor]] = None, stream=None):
+    """Run `chain` on device tensors; allocates the outputs (torch) unless given.  Returns them."""
+    spec = make_spec(chain)
+    if outputs is None:
+        outputs = output_tensors(chain, device=inputs[0].device)
+    ensure_workspace(spec)
+    fc_run(spec, inputs, outputs, stream)
+    return list(outputs)
+
+
+def run_chain_host(chain, host_inputs, host_outputs, staging, stream=None):
+    spec = make_spec(chain)
+    ensure_workspace(spec)
+    fc_run_host(spec, host_inputs, host_outputs, staging, stream)
+    return list(host_outputs)

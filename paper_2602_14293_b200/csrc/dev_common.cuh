@@ -1,0 +1,126 @@
+// Device helpers shared by the kernels: bf16 packing, tanh-GELU, the epilogue op interpreter and
+// (max, sum) pair algebra for online logsumexp / softmax.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "fc_internal.h"
+
+namespace fc {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// two floats -> packed bf16x2 (lo in bits 0..15), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ float tanh_fast(float x) {
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float exp2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// GELU, tanh form.  tanh.approx has ~2^-11 relative error, which is below bf16 resolution; chains
+// whose result feeds an fp32 output use the exp-based form (error ~1e-6) instead.
+template <bool kPrecise>
+__device__ __forceinline__ float gelu_tanh(float v) {
+    const float z = 0.7978845608028654f * v * fmaf(0.044715f, v * v, 1.0f);
+    if (kPrecise) {
+        // 0.5 v (1 + tanh z) = v / (1 + exp(-2 z))
+        const float e = exp2_fast(-2.0f * kLog2e * z);
+        return __fdividef(v, 1.0f + e);
+    } else {
+        const float hv = 0.5f * v;
+        return fmaf(hv, tanh_fast(z), hv);
+    }
+}
+
+__device__ __forceinline__ float load_scalar(const void* p, int dt, long long i) {
+    if (dt == FC_BF16) return __uint_as_float(((uint32_t) __ldg((const unsigned short*) p + i)) << 16);
+    return __ldg((const float*) p + i);
+}
+
+// Apply the op list to kN consecutive columns n0.. of row m (values in registers).
+// `ld` is the row pitch (elements) of ADD_TENSOR operands; columns >= n_limit are not touched
+// in memory (their register values are garbage-in, garbage-out and must not be stored).
+template <int kN, bool kPreciseGelu>
+__device__ __forceinline__ void apply_ops(float (&v)[kN], const DevOps& ops, long long m, long long n0,
+                                          long long n_limit, long long ld) {
+#pragma unroll 1
+    for (int i = 0; i < ops.n; ++i) {
+        const DevOp& op = ops.op[i];
+        switch (op.kind) {
+            case FC_OP_BIAS_N:
+#pragma unroll
+                for (int j = 0; j < kN; ++j)
+                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, n0 + j);
+                break;
+            case FC_OP_AFFINE_N:
+#pragma unroll
+                for (int j = 0; j < kN; ++j)
+                    if (n0 + j < n_limit)
+                        v[j] = fmaf(v[j], load_scalar(op.p0, op.dt0, n0 + j), load_scalar(op.p1, op.dt1, n0 + j));
+                break;
+            case FC_OP_RELU:
+#pragma unroll
+                for (int j = 0; j < kN; ++j) v[j] = v[j] < 0.0f ? 0.0f : v[j];
+                break;
+            case FC_OP_GELU_TANH:
+#pragma unroll
+                for (int j = 0; j < kN; ++j) v[j] = gelu_tanh<kPreciseGelu>(v[j]);
+                break;
+            case FC_OP_SCALE:
+#pragma unroll
+                for (int j = 0; j < kN; ++j) v[j] *= op.f0;
+                break;
+            case FC_OP_CLAMP:
+#pragma unroll
+                for (int j = 0; j < kN; ++j) v[j] = fminf(fmaxf(v[j], op.f0), op.f1);
+                break;
+            case FC_OP_ADD_TENSOR:
+#pragma unroll
+                for (int j = 0; j < kN; ++j)
+                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, m * ld + n0 + j);
+                break;
+            default:
+                break;
+        }
+    }
+}
+
+// (max, sum of exp(v - max)) pairs.  Merge is associative and commutative.
+struct MaxSum {
+    float m, s;
+};
+__device__ __forceinline__ MaxSum ms_identity() { return MaxSum{-CUDART_INF_F, 0.0f}; }
+__device__ __forceinline__ MaxSum ms_merge(MaxSum a, MaxSum b) {
+    const float m = fmaxf(a.m, b.m);
+    if (m == -CUDART_INF_F) return MaxSum{m, 0.0f};
+    return MaxSum{m, a.s * exp2_fast((a.m - m) * kLog2e) + b.s * exp2_fast((b.m - m) * kLog2e)};
+}
+__device__ __forceinline__ MaxSum ms_warp_reduce(MaxSum a) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        MaxSum b;
+        b.m = __shfl_xor_sync(0xffffffffu, a.m, o);
+        b.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+        a = ms_merge(a, b);
+    }
+    return a;
+}
+
+}  // namespace fc

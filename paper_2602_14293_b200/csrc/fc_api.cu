@@ -1,0 +1,526 @@
+// Host side of the C ABI: spec validation, kernel selection, TMA descriptor encoding, launch.
+// Nothing here allocates device memory or synchronises (fc_get_async_status excepted).
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "fc_internal.h"
+
+namespace fc {
+
+__device__ int g_status_word;  // written by kernels when a bounded wait expires
+
+namespace {
+
+thread_local char t_err[512] = "";
+std::atomic<uint64_t> g_launches{0};
+
+fc_status fail(fc_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_err, sizeof(t_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+    bool ready = false;
+    int cc_major = 0, num_sms = 0;
+    int* status = nullptr;
+    void* workspace = nullptr;
+    size_t workspace_bytes = 0;
+};
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_mu;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+
+fc_status get_device(DeviceInfo** out, int* dev_out = nullptr) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(FC_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return fail(FC_ERR_CUDA, "device ordinal %d out of range", dev);
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceInfo& d = g_dev[dev];
+    if (!d.ready) {
+        if ((e = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return fail(FC_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+        if (d.cc_major != 10) return fail(FC_ERR_ARCH, "device %d has compute capability %d.x; sm_100a is required", dev, d.cc_major);
+        if ((e = cudaGetSymbolAddress((void**) &d.status, g_status_word)) != cudaSuccess)
+            return fail(FC_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        if (!g_encode_tiled) {
+            cudaDriverEntryPointQueryResult q;
+            void* fn = nullptr;
+            e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+            if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn)
+                return fail(FC_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
+            g_encode_tiled = (EncodeTiledFn) fn;
+            fn = nullptr;
+            e = cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &q);
+            if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn)
+                return fail(FC_ERR_CUDA, "cuTensorMapEncodeIm2col entry point not available");
+            g_encode_im2col = (EncodeIm2colFn) fn;
+        }
+        d.ready = true;
+    }
+    *out = &d;
+    if (dev_out) *dev_out = dev;
+    return FC_OK;
+}
+
+size_t dt_size(int dt) { return dt == FC_BF16 ? 2 : 4; }
+
+// ------------------------------------------------------------------------------- validation
+struct Plan {
+    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_CONV } kind;
+    long long out_rows, out_cols;  // main output viewed as [rows][cols]
+    int n_prod_inputs;
+    int n_outputs;
+    int main_index, red_index;     // indices into outputs[], -1 if absent
+};
+
+bool contiguous(const fc_tensor& t) {
+    long long s = 1;
+    for (int i = t.rank - 1; i >= 0; --i) {
+        if (t.shape[i] != 1 && t.stride[i] != s) return false;
+        s *= t.shape[i];
+    }
+    return true;
+}
+
+fc_status check_tensor(const fc_tensor& t, const char* what, int dtype_or_any, int rank, const long long* shape) {
+    if (!t.ptr) return fail(FC_ERR_NULL, "%s: null pointer", what);
+    if (t.dtype != FC_F32 && t.dtype != FC_BF16) return fail(FC_ERR_INVALID_SPEC, "%s: unknown dtype %d", what, t.dtype);
+    if (dtype_or_any >= 0 && t.dtype != dtype_or_any) return fail(FC_ERR_INVALID_SPEC, "%s: dtype %d, expected %d", what, t.dtype, dtype_or_any);
+    if (t.rank != rank) return fail(FC_ERR_SHAPE, "%s: rank %d, expected %d", what, t.rank, rank);
+    for (int i = 0; i < rank; ++i)
+        if (t.shape[i] != shape[i]) return fail(FC_ERR_SHAPE, "%s: shape[%d] = %lld, expected %lld", what, i, (long long) t.shape[i], shape[i]);
+    if (!contiguous(t)) return fail(FC_ERR_UNSUPPORTED, "%s: only contiguous row-major tensors are supported", what);
+    if (reinterpret_cast<uintptr_t>(t.ptr) % dt_size(t.dtype)) return fail(FC_ERR_ALIGNMENT, "%s: pointer not aligned to its element size", what);
+    return FC_OK;
+}
+
+fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
+    if (!s) return fail(FC_ERR_NULL, "spec is null");
+    if (s->struct_size != sizeof(fc_chain_spec)) return fail(FC_ERR_INVALID_SPEC, "struct_size %u, expected %zu", s->struct_size, sizeof(fc_chain_spec));
+    if (s->version != FC_VERSION) return fail(FC_ERR_INVALID_SPEC, "version %u, expected %d", s->version, FC_VERSION);
+    if (s->producer < 0 || s->producer > FC_PROD_CONV2D_NHWC) return fail(FC_ERR_INVALID_SPEC, "unknown producer %d", s->producer);
+    if ((s->in_dtype != FC_F32 && s->in_dtype != FC_BF16) || (s->out_dtype != FC_F32 && s->out_dtype != FC_BF16))
+        return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
+    if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
+    if (s->reduce < 0 || s->reduce > FC_RED_GLOBAL_AVGPOOL) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
+    if (s->n_ops < 0 || s->n_ops > FC_MAX_OPS) return fail(FC_ERR_INVALID_SPEC, "n_ops %d out of range", s->n_ops);
+    for (int i = 0; i < s->n_ops; ++i)
+        if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_ADD_TENSOR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
+
+    plan->n_prod_inputs = s->producer == FC_PROD_ELEMENTWISE ? 1 : 2;
+    if (s->producer == FC_PROD_CONV2D_NHWC) {
+        if (s->batch < 1 || s->H < 1 || s->W < 1 || s->Cin < 1 || s->Cout < 1 || s->R < 1 || s->S < 1 || s->stride < 1 || s->pad < 0)
+            return fail(FC_ERR_SHAPE, "conv dimensions must be positive (pad >= 0)");
+        const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
+        if (s->H + 2 * s->pad < s->R || s->W + 2 * s->pad < s->S) return fail(FC_ERR_SHAPE, "filter larger than the padded image");
+        plan->out_rows = s->batch * OH * OW;
+        plan->out_cols = s->Cout;
+        if (plan->out_rows > 0x7fffffffLL || s->R * s->S * s->Cin > 0x7fffffffLL) return fail(FC_ERR_SHAPE, "conv too large");
+    } else {
+        if (s->M < 1 || s->N < 1 || (s->producer == FC_PROD_GEMM_NT && s->K < 1)) return fail(FC_ERR_SHAPE, "M, N, K must be >= 1");
+        if (s->producer == FC_PROD_GEMM_NT && (s->M > 0x7fffffffLL || s->N > 0x7fffffffLL || s->K > 0x7fffffffLL))
+            return fail(FC_ERR_SHAPE, "GEMM dimension exceeds 2^31-1");
+        plan->out_rows = s->M;
+        plan->out_cols = s->N;
+    }
+
+    // supported patterns
+    if (s->reduce == FC_RED_NONE && !s->store_main) return fail(FC_ERR_INVALID_SPEC, "chain has no output (no reduction and store_main = 0)");
+    plan->main_index = plan->red_index = -1;
+    switch (s->producer) {
+        case FC_PROD_ELEMENTWISE:
+            if (s->reduce != FC_RED_NONE && s->reduce != FC_RED_ROW_LOGSUMEXP)
+                return fail(FC_ERR_UNSUPPORTED, "elementwise producer supports reduce NONE or ROW_LOGSUMEXP");
+            plan->kind = Plan::EW;
+            break;
+        case FC_PROD_GEMM_NT:
+            if (s->in_dtype == FC_F32) {
+                if (s->reduce != FC_RED_NONE || s->out_dtype != FC_F32)
+                    return fail(FC_ERR_UNSUPPORTED, "fp32 GEMM supports fp32 output without reduction");
+                plan->kind = Plan::GEMM_F32;
+            } else if (s->reduce == FC_RED_NONE) {
+                plan->kind = Plan::TC_PLAIN;
+            } else if (s->reduce == FC_RED_ROW_SOFTMAX) {
+                plan->kind = Plan::TC_SOFTMAX;
+            } else {
+                return fail(FC_ERR_UNSUPPORTED, "bf16 GEMM supports reduce NONE or ROW_SOFTMAX");
+            }
+            break;
+        default:
+            if (s->in_dtype != FC_BF16 || s->reduce != FC_RED_GLOBAL_AVGPOOL || s->store_main)
+                return fail(FC_ERR_UNSUPPORTED, "conv supports bf16 input with GLOBAL_AVGPOOL and store_main = 0");
+            if (s->stride != 1) return fail(FC_ERR_UNSUPPORTED, "conv supports stride 1");
+            if (s->pad >= s->R || s->pad >= s->S || s->R > 16 || s->S > 16) return fail(FC_ERR_UNSUPPORTED, "conv supports pad < R,S <= 16");
+            plan->kind = Plan::TC_CONV;
+            break;
+    }
+    int n = 0;
+    if (s->reduce == FC_RED_ROW_SOFTMAX) {
+        plan->main_index = n++;
+    } else {
+        if (s->store_main) plan->main_index = n++;
+        if (s->reduce != FC_RED_NONE) plan->red_index = n++;
+    }
+    plan->n_outputs = n;
+    return FC_OK;
+}
+
+fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_tensor* in, int n_in, const fc_tensor* out, int n_out) {
+    if (!in || !out) return fail(FC_ERR_NULL, "inputs / outputs array is null");
+    if (n_in < plan.n_prod_inputs) return fail(FC_ERR_INVALID_SPEC, "producer needs %d inputs, got %d", plan.n_prod_inputs, n_in);
+    if (n_out != plan.n_outputs) return fail(FC_ERR_INVALID_SPEC, "chain has %d outputs, got %d", plan.n_outputs, n_out);
+    fc_status st;
+    if (s->producer == FC_PROD_ELEMENTWISE) {
+        const long long sh[2] = {s->M, s->N};
+        if ((st = check_tensor(in[0], "inputs[0]", s->in_dtype, 2, sh))) return st;
+    } else if (s->producer == FC_PROD_GEMM_NT) {
+        const long long sa[2] = {s->M, s->K}, sb[2] = {s->N, s->K};
+        if ((st = check_tensor(in[0], "inputs[0] (A)", s->in_dtype, 2, sa))) return st;
+        if ((st = check_tensor(in[1], "inputs[1] (B)", s->in_dtype, 2, sb))) return st;
+        if (s->in_dtype == FC_BF16) {
+            if (s->K % 8) return fail(FC_ERR_ALIGNMENT, "bf16 GEMM needs K %% 8 == 0 (K = %lld)", (long long) s->K);
+            if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr)) & 15)
+                return fail(FC_ERR_ALIGNMENT, "bf16 GEMM operands must be 16-byte aligned");
+        }
+    } else {
+        const long long si[4] = {s->batch, s->H, s->W, s->Cin}, sw[4] = {s->Cout, s->R, s->S, s->Cin};
+        if ((st = check_tensor(in[0], "inputs[0] (image)", s->in_dtype, 4, si))) return st;
+        if ((st = check_tensor(in[1], "inputs[1] (weights)", s->in_dtype, 4, sw))) return st;
+        if (s->Cin % 8) return fail(FC_ERR_ALIGNMENT, "conv needs Cin %% 8 == 0 (Cin = %lld)", (long long) s->Cin);
+        if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr)) & 15)
+            return fail(FC_ERR_ALIGNMENT, "conv operands must be 16-byte aligned");
+    }
+    for (int i = 0; i < s->n_ops; ++i) {
+        const fc_op& op = s->ops[i];
+        char what[64];
+        const long long vec[1] = {plan.out_cols};
+        if (op.kind == FC_OP_BIAS_N || op.kind == FC_OP_AFFINE_N) {
+            const int idx[2] = {op.in0, op.in1};
+            for (int k = 0; k < (op.kind == FC_OP_AFFINE_N ? 2 : 1); ++k) {
+                if (idx[k] < plan.n_prod_inputs || idx[k] >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, idx[k]);
+                snprintf(what, sizeof(what), "inputs[%d] (op %d vector)", idx[k], i);
+                if ((st = check_tensor(in[idx[k]], what, -1, 1, vec))) return st;
+            }
+        } else if (op.kind == FC_OP_ADD_TENSOR) {
+            if (op.in0 < plan.n_prod_inputs || op.in0 >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, op.in0);
+            snprintf(what, sizeof(what), "inputs[%d] (op %d tensor)", op.in0, i);
+            if (s->producer == FC_PROD_CONV2D_NHWC) {
+                const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
+                const long long sh[4] = {s->batch, OH, OW, s->Cout};
+                if ((st = check_tensor(in[op.in0], what, -1, 4, sh))) return st;
+            } else {
+                const long long sh[2] = {s->M, s->N};
+                if ((st = check_tensor(in[op.in0], what, -1, 2, sh))) return st;
+            }
+        } else if (op.kind == FC_OP_CLAMP && !(op.f0 <= op.f1)) {
+            return fail(FC_ERR_INVALID_SPEC, "op %d: clamp bounds lo > hi", i);
+        }
+    }
+    if (plan.main_index >= 0) {
+        if (s->producer == FC_PROD_CONV2D_NHWC) {
+            const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
+            const long long sh[4] = {s->batch, OH, OW, s->Cout};
+            if ((st = check_tensor(out[plan.main_index], "main output", s->out_dtype, 4, sh))) return st;
+        } else {
+            const long long sh[2] = {s->M, s->N};
+            if ((st = check_tensor(out[plan.main_index], "main output", s->out_dtype, 2, sh))) return st;
+        }
+    }
+    if (plan.red_index >= 0) {
+        if (s->reduce == FC_RED_ROW_LOGSUMEXP) {
+            const long long sh[1] = {s->M};
+            if ((st = check_tensor(out[plan.red_index], "logsumexp output", FC_F32, 1, sh))) return st;
+        } else {
+            const long long sh[2] = {s->batch, s->Cout};
+            if ((st = check_tensor(out[plan.red_index], "pooled output", FC_F32, 2, sh))) return st;
+        }
+    }
+    return FC_OK;
+}
+
+void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
+    d->n = s->n_ops;
+    for (int i = 0; i < s->n_ops; ++i) {
+        const fc_op& op = s->ops[i];
+        DevOp& o = d->op[i];
+        o.kind = op.kind;
+        o.f0 = op.f0;
+        o.f1 = op.f1;
+        o.p0 = o.p1 = nullptr;
+        o.dt0 = o.dt1 = FC_F32;
+        if (op.kind == FC_OP_BIAS_N || op.kind == FC_OP_AFFINE_N || op.kind == FC_OP_ADD_TENSOR) {
+            o.p0 = in[op.in0].ptr;
+            o.dt0 = in[op.in0].dtype;
+        }
+        if (op.kind == FC_OP_AFFINE_N) {
+            o.p1 = in[op.in1].ptr;
+            o.dt1 = in[op.in1].dtype;
+        }
+    }
+}
+
+constexpr int kSoftmaxBN = 256;
+
+size_t softmax_workspace_bytes(long long M, long long N) {
+    const long long tiles_n = (N + kSoftmaxBN - 1) / kSoftmaxBN, panels = (M + 127) / 128;
+    size_t counters = (size_t) panels * 4;
+    counters = (counters + 255) / 256 * 256;
+    return counters + (size_t) M * tiles_n * sizeof(float2);
+}
+
+fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long cols, int box_rows) {
+    const cuuint64_t dims[2] = {(cuuint64_t) cols, (cuuint64_t) rows};
+    const cuuint64_t strides[1] = {(cuuint64_t) cols * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t) box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d (rows %lld cols %lld)", (int) r, rows, cols);
+    return FC_OK;
+}
+
+fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr) {
+    const cuuint64_t dims[4] = {(cuuint64_t) s->Cin, (cuuint64_t) s->W, (cuuint64_t) s->H, (cuuint64_t) s->batch};
+    const cuuint64_t strides[3] = {(cuuint64_t) s->Cin * 2, (cuuint64_t) s->W * s->Cin * 2, (cuuint64_t) s->H * s->W * s->Cin * 2};
+    // base pixels run over the output grid shifted by -pad; a filter tap adds (s, r) to every base pixel
+    const int lower[2] = {(int) -s->pad, (int) -s->pad};
+    const int upper[2] = {(int) (s->pad - (s->S - 1)), (int) (s->pad - (s->R - 1))};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = g_encode_im2col(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper,
+                                 64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeIm2col failed with CUresult %d", (int) r);
+    return FC_OK;
+}
+
+fc_status cuda_fail(cudaError_t e, const char* what) { return fail(FC_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e)); }
+
+}  // namespace
+}  // namespace fc
+
+using namespace fc;
+
+extern "C" {
+
+fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_inputs, fc_tensor* outputs, int n_outputs,
+                 void* cuda_stream) {
+    Plan plan;
+    fc_status st;
+    if ((st = validate_spec(spec, &plan))) return st;
+    if ((st = validate_tensors(spec, plan, inputs, n_inputs, outputs, n_outputs))) return st;
+    DeviceInfo* dev;
+    if ((st = get_device(&dev))) return st;
+    cudaStream_t stream = (cudaStream_t) cuda_stream;
+    int launches = 0;
+    cudaError_t e = cudaSuccess;
+
+    switch (plan.kind) {
+        case Plan::EW: {
+            EwParams p;
+            p.x = inputs[0].ptr; p.x_dt = spec->in_dtype;
+            p.y = plan.main_index >= 0 ? outputs[plan.main_index].ptr : nullptr;
+            p.y_dt = spec->out_dtype;
+            p.red = plan.red_index >= 0 ? (float*) outputs[plan.red_index].ptr : nullptr;
+            p.M = spec->M; p.N = spec->N; p.reduce = spec->reduce;
+            build_ops(spec, inputs, &p.ops);
+            e = launch_ew_rowreduce(p, dev->num_sms, stream, &launches);
+            break;
+        }
+        case Plan::GEMM_F32: {
+            GemmF32Params p;
+            p.A = (const float*) inputs[0].ptr; p.B = (const float*) inputs[1].ptr;
+            p.C = (float*) outputs[plan.main_index].ptr;
+            p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+            build_ops(spec, inputs, &p.ops);
+            e = launch_gemm_f32(p, stream, &launches);
+            break;
+        }
+        case Plan::TC_PLAIN:
+        case Plan::TC_SOFTMAX: {
+            TcParams p;
+            memset(&p, 0, sizeof(p));
+            p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : 0;
+            p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+            p.out = outputs[plan.main_index].ptr; p.out_dt = spec->out_dtype;
+            p.status = dev->status;
+            build_ops(spec, inputs, &p.ops);
+            const int bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
+            if (p.mode == 1) {
+                const size_t need = softmax_workspace_bytes(spec->M, spec->N);
+                const long long panels = (spec->M + 127) / 128;
+                if (!dev->workspace || dev->workspace_bytes < need)
+                    return fail(FC_ERR_WORKSPACE, "row softmax needs a %zu-byte workspace (fc_set_workspace); have %zu", need, dev->workspace_bytes);
+                size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
+                p.counters = (unsigned int*) dev->workspace;
+                p.stats = (float2*) ((char*) dev->workspace + counters);
+                if ((e = cudaMemsetAsync(p.counters, 0, counters, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+            }
+            CUtensorMap tmA, tmB;
+            if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn))) return st;
+            e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
+            break;
+        }
+        case Plan::TC_CONV: {
+            TcParams p;
+            memset(&p, 0, sizeof(p));
+            p.mode = 2;
+            p.batch = (int) spec->batch; p.H = (int) spec->H; p.W = (int) spec->W; p.Cin = (int) spec->Cin; p.Cout = (int) spec->Cout;
+            p.R = (int) spec->R; p.S = (int) spec->S; p.stride = (int) spec->stride; p.pad = (int) spec->pad;
+            p.OH = (int) ((spec->H + 2 * spec->pad - spec->R) / spec->stride + 1);
+            p.OW = (int) ((spec->W + 2 * spec->pad - spec->S) / spec->stride + 1);
+            p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
+            p.inv_hw = 1.0f / (float) (p.OH * p.OW);
+            p.out = outputs[plan.red_index].ptr; p.out_dt = FC_F32;
+            p.status = dev->status;
+            build_ops(spec, inputs, &p.ops);
+            const int bn = spec->Cout <= 128 ? 128 : 256;
+            if ((e = cudaMemsetAsync(p.out, 0, (size_t) spec->batch * spec->Cout * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+            CUtensorMap tmA, tmB;
+            if ((st = encode_im2col(&tmA, spec, inputs[0].ptr))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn))) return st;
+            e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
+            break;
+        }
+    }
+    g_launches.fetch_add((uint64_t) launches);
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    return FC_OK;
+}
+
+fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, int n_inputs, const fc_tensor* outputs,
+                          int n_outputs, size_t* bytes) {
+    if (!bytes || !inputs || !outputs) return fail(FC_ERR_NULL, "null argument");
+    (void) spec;
+    size_t total = 0;
+    auto add = [&](const fc_tensor& t) {
+        size_t n = dt_size(t.dtype);
+        for (int i = 0; i < t.rank; ++i) n *= (size_t) t.shape[i];
+        total += (n + 255) / 256 * 256;
+    };
+    for (int i = 0; i < n_inputs; ++i) add(inputs[i]);
+    for (int i = 0; i < n_outputs; ++i) add(outputs[i]);
+    *bytes = total;
+    return FC_OK;
+}
+
+fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, int n_inputs, fc_tensor* host_outputs,
+                      int n_outputs, void* staging, size_t staging_bytes, void* cuda_stream) {
+    Plan plan;
+    fc_status st;
+    if ((st = validate_spec(spec, &plan))) return st;
+    if (!host_inputs || !host_outputs || !staging) return fail(FC_ERR_NULL, "null argument");
+    if (n_inputs < 0 || n_inputs > 16 || n_outputs < 0 || n_outputs > 4) return fail(FC_ERR_INVALID_SPEC, "too many tensors");
+    size_t need = 0;
+    if ((st = fc_staging_size(spec, host_inputs, n_inputs, host_outputs, n_outputs, &need))) return st;
+    if (staging_bytes < need) return fail(FC_ERR_WORKSPACE, "staging buffer has %zu bytes, %zu needed", staging_bytes, need);
+    if (reinterpret_cast<uintptr_t>(staging) & 255) return fail(FC_ERR_ALIGNMENT, "staging buffer must be 256-byte aligned");
+    cudaStream_t stream = (cudaStream_t) cuda_stream;
+    fc_tensor din[16], dout[4];
+    size_t nbytes_out[4];
+    char* cur = (char*) staging;
+    for (int i = 0; i < n_inputs; ++i) {
+        if (!host_inputs[i].ptr) return fail(FC_ERR_NULL, "host_inputs[%d]: null pointer", i);
+        size_t n = dt_size(host_inputs[i].dtype);
+        for (int k = 0; k < host_inputs[i].rank; ++k) n *= (size_t) host_inputs[i].shape[k];
+        din[i] = host_inputs[i];
+        din[i].ptr = cur;
+        cudaError_t e = cudaMemcpyAsync(cur, host_inputs[i].ptr, n, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync H2D");
+        cur += (n + 255) / 256 * 256;
+    }
+    for (int i = 0; i < n_outputs; ++i) {
+        if (!host_outputs[i].ptr) return fail(FC_ERR_NULL, "host_outputs[%d]: null pointer", i);
+        size_t n = dt_size(host_outputs[i].dtype);
+        for (int k = 0; k < host_outputs[i].rank; ++k) n *= (size_t) host_outputs[i].shape[k];
+        nbytes_out[i] = n;
+        dout[i] = host_outputs[i];
+        dout[i].ptr = cur;
+        cur += (n + 255) / 256 * 256;
+    }
+    if ((st = fc_run(spec, din, n_inputs, dout, n_outputs, cuda_stream))) return st;
+    for (int i = 0; i < n_outputs; ++i) {
+        cudaError_t e = cudaMemcpyAsync(host_outputs[i].ptr, dout[i].ptr, nbytes_out[i], cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync D2H");
+    }
+    return FC_OK;
+}
+
+fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
+    Plan plan;
+    fc_status st;
+    if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
+    if ((st = validate_spec(spec, &plan))) return st;
+    *bytes = plan.kind == Plan::TC_SOFTMAX ? softmax_workspace_bytes(spec->M, spec->N) : 0;
+    return FC_OK;
+}
+
+fc_status fc_set_workspace(void* dev_ptr, size_t bytes) {
+    if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255)) return fail(FC_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+    DeviceInfo* dev;
+    fc_status st;
+    if ((st = get_device(&dev))) return st;
+    std::lock_guard<std::mutex> lk(g_mu);
+    dev->workspace = dev_ptr;
+    dev->workspace_bytes = dev_ptr ? bytes : 0;
+    return FC_OK;
+}
+
+fc_status fc_get_async_status(void* cuda_stream) {
+    DeviceInfo* dev;
+    fc_status st;
+    if ((st = get_device(&dev))) return st;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t) cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    int word = 0;
+    if ((e = cudaMemcpy(&word, dev->status, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy status");
+    if (word != 0) {
+        const int zero = 0;
+        if ((e = cudaMemcpy(dev->status, &zero, sizeof(int), cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy status");
+        return fail((fc_status) word, "a bounded device-side wait expired");
+    }
+    return FC_OK;
+}
+
+uint64_t fc_launch_count(void) { return g_launches.load(); }
+
+const char* fc_status_string(fc_status s) {
+    switch (s) {
+        case FC_OK: return "FC_OK";
+        case FC_ERR_NULL: return "FC_ERR_NULL";
+        case FC_ERR_INVALID_SPEC: return "FC_ERR_INVALID_SPEC";
+        case FC_ERR_UNSUPPORTED: return "FC_ERR_UNSUPPORTED";
+        case FC_ERR_SHAPE: return "FC_ERR_SHAPE";
+        case FC_ERR_ALIGNMENT: return "FC_ERR_ALIGNMENT";
+        case FC_ERR_WORKSPACE: return "FC_ERR_WORKSPACE";
+        case FC_ERR_ARCH: return "FC_ERR_ARCH";
+        case FC_ERR_CUDA: return "FC_ERR_CUDA";
+        case FC_ERR_TIMEOUT: return "FC_ERR_TIMEOUT";
+    }
+    return "FC_ERR_?";
+}
+
+const char* fc_last_error(void) { return t_err; }
+
+int fc_version(void) { return FC_VERSION; }
+
+}  // extern "C"

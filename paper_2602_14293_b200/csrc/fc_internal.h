@@ -1,0 +1,68 @@
+// Internal declarations shared by the host planner and the kernels of the fused-chain library.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fc.h"
+
+namespace fc {
+
+// ---- epilogue op list as the kernels see it (passed by value in kernel parameters) ----
+struct DevOp {
+    int kind;          // fc_op_kind
+    int dt0, dt1;      // fc_dtype of p0 / p1
+    float f0, f1;
+    const void* p0;    // vector [N] or tensor [M,N]
+    const void* p1;    // second vector (AFFINE_N)
+};
+
+struct DevOps {
+    int n;
+    DevOp op[FC_MAX_OPS];
+};
+
+// Device status word values (also fc_status values).
+constexpr int kStatusTimeout = FC_ERR_TIMEOUT;
+
+// Every bounded device-side wait gives up after this many nanoseconds of %globaltimer.
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ---- launchers (defined one per .cu file); all enqueue on `stream` and return a cudaError_t ----
+struct EwParams {
+    const void* x; int x_dt;
+    void* y; int y_dt;          // may be null when !store_main
+    float* red;                 // row logsumexp out, or null
+    long long M, N;
+    int reduce;                 // FC_RED_NONE or FC_RED_ROW_LOGSUMEXP
+    DevOps ops;
+};
+cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t stream, int* launches);
+
+struct GemmF32Params {
+    const float* A; const float* B; float* C;
+    int M, N, K;
+    DevOps ops;
+};
+cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* launches);
+
+// tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
+struct TcParams {
+    int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool
+    int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
+    void* out; int out_dt;      // mode 0/1: [M,N] bf16 or f32.  mode 2: f32 [batch,Cout] (pre-zeroed)
+    DevOps ops;
+    // mode 1
+    float2* stats;              // [M][tiles_n] (max, sum) per tile
+    unsigned int* counters;     // [panels], zeroed before launch
+    // mode 2
+    int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
+    float inv_hw;
+    int* status;                // device status word
+};
+cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                           int bn, int num_sms, cudaStream_t stream, int* launches);
+size_t gemm_tc_smem_bytes(int bn);
+
+}  // namespace fc

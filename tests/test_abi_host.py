@@ -1,0 +1,135 @@
+"""Host-side checks that need no GPU: the library loads, exports every symbol the header declares,
+and rejects malformed chains before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from fc_inputs import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def fc():
+    entry.build()
+    import paper_2602_14293_b200 as fc
+    return fc
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            src = open(os.path.join(ROOT, "include", fn)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names |= set(re.findall(r"\b(fc_[a-z_0-9]+)\s*\(", src))
+    return names
+
+
+def test_library_exports_every_declared_symbol(fc):
+    L = fc.lib()
+    names = _declared_symbols()
+    assert {"fc_run", "fc_run_host", "fc_workspace_size", "fc_set_workspace", "fc_get_async_status"} <= names
+    for n in names:
+        assert hasattr(L, n), n
+    assert fc.fc_version() == 1
+
+
+def test_spec_struct_matches_header_size(fc):
+    # 4 + 4 + 4*4 + 12*8 + 4 (+4 pad?) ... the library checks struct_size itself; a mismatch is INVALID_SPEC
+    spec = fc.make_spec(wl.CONFIGS["C3"]())
+    n = ctypes.c_size_t(0)
+    assert fc.lib().fc_workspace_size(ctypes.byref(spec), ctypes.byref(n)) == 0 and n.value == 0
+
+
+def test_workspace_size_softmax(fc):
+    spec = fc.make_spec(wl.CONFIGS["C4"]())
+    # 32 panel counters (padded to 256 B) + 4096 rows x 16 tiles x (max, sum) fp32
+    assert fc.fc_workspace_size(spec) == 256 + 4096 * 16 * 8
+
+
+def _status(fc, spec, ins=None, outs=None):
+    pi = ctypes.cast(ins, ctypes.POINTER(type(ins[0]))) if ins is not None else None
+    po = ctypes.cast(outs, ctypes.POINTER(type(outs[0]))) if outs is not None else None
+    return fc.lib().fc_run(ctypes.byref(spec) if spec is not None else None, pi, len(ins) if ins is not None else 0,
+                           po, len(outs) if outs is not None else 0, None)
+
+
+def _fake_tensor(fc, shape, dtype, ptr=0x1000):
+    from paper_2602_14293_b200.binding import fc_tensor
+    t = fc_tensor()
+    t.ptr = ptr
+    t.dtype = dtype
+    t.rank = len(shape)
+    st = 1
+    for i in reversed(range(len(shape))):
+        t.shape[i] = shape[i]
+        t.stride[i] = st
+        st *= shape[i]
+    return t
+
+
+def _arr(fc, ts):
+    from paper_2602_14293_b200.binding import fc_tensor
+    a = (fc_tensor * len(ts))()
+    for i, t in enumerate(ts):
+        a[i] = t
+    return a
+
+
+def test_rejections_happen_before_any_device_access(fc):
+    L = fc.lib()
+    launches_before = fc.fc_launch_count()
+    ch = wl.gemm_bias_gelu_scale_clamp(256, 256, 64)
+    good_in = _arr(fc, [_fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (256,), 1)])
+    good_out = _arr(fc, [_fake_tensor(fc, (256, 256), 1)])
+    FC_ERR_NULL, INVALID, UNSUP, SHAPE, ALIGN = 1, 2, 3, 4, 5
+
+    assert L.fc_run(None, None, 0, None, 0, None) == FC_ERR_NULL
+    s = fc.make_spec(ch); s.struct_size = 8
+    assert _status(fc, s, good_in, good_out) == INVALID
+    s = fc.make_spec(ch); s.version = 99
+    assert _status(fc, s, good_in, good_out) == INVALID
+    s = fc.make_spec(ch); s.producer = 7
+    assert _status(fc, s, good_in, good_out) == INVALID
+    s = fc.make_spec(ch); s.ops[0].kind = 42
+    assert _status(fc, s, good_in, good_out) == INVALID
+    s = fc.make_spec(ch); s.ops[0].in0 = 9          # operand index out of range
+    assert _status(fc, s, good_in, good_out) == INVALID
+    s = fc.make_spec(ch); s.ops[3].f0, s.ops[3].f1 = 1.0, -1.0   # clamp lo > hi
+    assert _status(fc, s, good_in, good_out) == INVALID
+    s = fc.make_spec(ch); s.K = 0
+    assert _status(fc, s, good_in, good_out) == SHAPE
+    s = fc.make_spec(ch)
+    bad_in = _arr(fc, [_fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (128, 64), 1), _fake_tensor(fc, (256,), 1)])
+    assert _status(fc, s, bad_in, good_out) == SHAPE
+    null_in = _arr(fc, [_fake_tensor(fc, (256, 64), 1, ptr=0), _fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (256,), 1)])
+    assert _status(fc, s, null_in, good_out) == FC_ERR_NULL
+    mis_in = _arr(fc, [_fake_tensor(fc, (256, 64), 1, ptr=0x1008), _fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (256,), 1)])
+    assert _status(fc, s, mis_in, good_out) == ALIGN
+    ch_k = wl.gemm_bias_gelu_scale_clamp(256, 256, 60)     # K % 8 != 0
+    k_in = _arr(fc, [_fake_tensor(fc, (256, 60), 1), _fake_tensor(fc, (256, 60), 1), _fake_tensor(fc, (256,), 1)])
+    assert _status(fc, fc.make_spec(ch_k), k_in, good_out) == ALIGN
+    # well-formed but not implemented: logsumexp after a GEMM, strided conv, softmax on an elementwise producer
+    s = fc.make_spec(ch); s.reduce = 1
+    assert _status(fc, s, good_in, good_out) == UNSUP
+    s = fc.make_spec(wl.conv_bias_relu_avgpool(stride=2))
+    assert _status(fc, s, good_in, good_out) == UNSUP
+    s = fc.make_spec(wl.affine_gelu_residual_lse(8, 8)); s.reduce = 2
+    assert _status(fc, s, good_in, good_out) == UNSUP
+    assert "FC_ERR_UNSUPPORTED" == L.fc_status_string(UNSUP).decode()
+    assert len(fc.fc_last_error()) > 0
+    # nothing above reached a launch
+    assert fc.fc_launch_count() == launches_before
+
+
+def test_non_contiguous_tensor_is_rejected(fc):
+    ch = wl.affine_gelu_residual_lse(8, 16)
+    s = fc.make_spec(ch)
+    x = _fake_tensor(fc, (8, 16), 1); x.stride[0] = 32
+    ins = _arr(fc, [x, _fake_tensor(fc, (16,), 1), _fake_tensor(fc, (16,), 1), _fake_tensor(fc, (8, 16), 1)])
+    outs = _arr(fc, [_fake_tensor(fc, (8, 16), 1), _fake_tensor(fc, (8,), 0)])
+    assert _status(fc, s, ins, outs) == 3

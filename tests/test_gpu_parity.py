@@ -1,0 +1,270 @@
+"""Parity of the CUDA path with the CPU oracle, element by element, through the C ABI.
+
+Tolerances (written here, as the benchmark states them): fp32 outputs |err| <= 1e-4 (1 + |ref|)
+for every element; bf16 outputs max relative error <= 2e-2 and mean absolute error <= 2e-3.
+Integer-valued contractions must agree bit for bit.  Outputs are NaN-poisoned before every run.
+"""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from fc_inputs import rng, workloads as wl
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fc():
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2602_14293_b200 as fc
+    assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
+    torch.cuda.set_device(0)
+    return fc
+
+
+def run_and_check(fc, orc, ch, seed=0, ins=None, tag=""):
+    if ins is None:
+        ins = wl.make_inputs(ch, seed)
+    ref = orc.run_chain(ch, ins)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    before = fc.fc_launch_count()
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    assert fc.fc_launch_count() > before, "no kernel of the library was launched"
+    names = [r for r, _, _ in wl.output_shapes(ch)]
+    res = {}
+    for name, t in zip(names, outs):
+        res[name] = util.check(t, ref[name], f"{ch.name}{tag} seed {seed}: {name}")
+    return outs, ref, res
+
+
+# ------------------------------------------------------------------ C1: strict fp32 GEMM + bias + ReLU
+@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("variant", ["std", "var"])
+def test_c1_gemm_f32(fc, orc, seed, variant):
+    run_and_check(fc, orc, wl.gemm_bias_relu_f32(256, 256, 256, variant), seed)
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (33, 65, 70), (100, 37, 129), (257, 31, 32)])
+def test_gemm_f32_ragged(fc, orc, M, N, K):
+    run_and_check(fc, orc, wl.gemm_bias_relu_f32(M, N, K, "var"), 3)
+
+
+# ------------------------------------------------------------------ kernel (a): elementwise + logsumexp
+@pytest.mark.parametrize("M,N", [(1, 1), (3, 8), (5, 1000), (7, 4097), (33, 2048), (64, 4096), (9, 12345)])
+def test_elementwise_lse_shapes(fc, orc, M, N):
+    run_and_check(fc, orc, wl.affine_gelu_residual_lse(M, N), 1)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_c2_reduced_rows(fc, orc, seed):
+    run_and_check(fc, orc, wl.affine_gelu_residual_lse(1024, 4096), seed)
+
+
+def test_elementwise_f32_and_other_op_lists(fc, orc):
+    base = wl.affine_gelu_residual_lse(37, 515)
+    rec32 = tuple((t, "f32", s, d, a, b) for t, _, s, d, a, b in base.input_recipe)
+    # fp32 storage in and out, no reduction
+    run_and_check(fc, orc, replace(base, in_dtype="f32", out_dtype="f32", reduce="none", input_recipe=rec32), 2)
+    # logsumexp only (main output not stored)
+    run_and_check(fc, orc, replace(base, store_main=False), 2)
+    # bias -> relu -> scale -> clamp on bf16, no reduction
+    ch = replace(base, ops=(("bias_n", 1), ("relu",), ("scale", 0.5), ("clamp", -0.25, 0.75), ("add_tensor", 3)), reduce="none")
+    run_and_check(fc, orc, ch, 2)
+    # no ops at all: a copy with logsumexp
+    run_and_check(fc, orc, replace(base, ops=()), 2)
+
+
+def test_lse_shift_overflow_safety(fc, orc):
+    ch = replace(wl.affine_gelu_residual_lse(4, 512), ops=(), in_dtype="f32", out_dtype="f32",
+                 input_recipe=(("x", "f32", (4, 512), "normal", 0.0, 1.0),))
+    x = wl.make_inputs(ch, 0)[0]
+    x[1] += 1.0e4
+    x[2] -= 1.0e4
+    x[3, :] = -3.0
+    x[3, 17] = 60.0
+    run_and_check(fc, orc, ch, ins=[x])
+
+
+def test_c2_full_size_sampled_rows(fc, orc):
+    """The benchmark workload itself, in the launch configuration the benchmark times: rows sampled
+    for the oracle (each row is an independent problem: elementwise ops and a per-row reduction)."""
+    ch = wl.CONFIGS["C2"]()
+    ins = wl.make_inputs(ch, 0)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    rows = np.unique(np.concatenate([np.arange(0, 16384, 331), [0, 1, 16382, 16383]]))
+    sub = replace(ch, M=len(rows))
+    ref = orc.run_chain(sub, [ins[0][rows], ins[1], ins[2], ins[3][rows]])
+    util.check(outs[0][torch.from_numpy(rows).cuda()], ref["main"], "C2 y (sampled rows)")
+    util.check(outs[1][torch.from_numpy(rows).cuda()], ref["reduce"], "C2 logsumexp (sampled rows)")
+    assert torch.isfinite(outs[0].float()).all() and torch.isfinite(outs[1]).all()
+
+
+# ------------------------------------------------------------------ kernel (b): tcgen05 GEMM + epilogue
+def _plain_gemm(M, N, K, out_dtype="f32"):
+    return replace(wl.gemm_bias_gelu_scale_clamp(M, N, K), ops=(), out_dtype=out_dtype,
+                   input_recipe=wl.gemm_bias_gelu_scale_clamp(M, N, K).input_recipe[:2])
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 512), (256, 512, 128), (384, 768, 4096),
+                                   (200, 264, 72), (1, 8, 8), (130, 40, 200), (128, 128, 64), (77, 100, 136)])
+def test_gemm_tc_small_integers_bit_exact(fc, orc, M, N, K):
+    """Integer operands (exact in bf16, partial sums < 2^24): any correct contraction gives the same
+    bits, so the tensor-core path must equal the fp64 oracle exactly; exposes any layout permutation."""
+    ch = wl.with_integer_inputs(_plain_gemm(M, N, K), -4, 4)
+    ins = wl.make_inputs(ch, 5)
+    ref = orc.run_chain(ch, ins)["main"]
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    got = util.to_f64(outs[0])
+    assert np.array_equal(got, ref), f"{np.count_nonzero(got != ref)} of {got.size} elements differ"
+
+
+def test_gemm_tc_one_hot_rows(fc, orc):
+    M, N, K = 256, 512, 192
+    ch = _plain_gemm(M, N, K)
+    A = np.zeros((M, K), np.float32)
+    A[np.arange(M), (np.arange(M) * 7) % K] = 1.0       # row m selects column (7m mod K) of B^T
+    B = rng.integers_f32(0, "onehot/B", (N, K), -100, 100)
+    ins = [rng.store(A, "bf16"), rng.store(B, "bf16")]
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    want = B[:, (np.arange(M) * 7) % K].T.astype(np.float64)
+    assert np.array_equal(util.to_f64(outs[0]), want)
+
+
+@pytest.mark.parametrize("variant", ["std", "var"])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_c3_chain_reduced(fc, orc, seed, variant):
+    run_and_check(fc, orc, wl.gemm_bias_gelu_scale_clamp(512, 1024, 512, variant), seed)
+
+
+@pytest.mark.parametrize("M,N,K", [(200, 264, 72), (129, 8, 8), (1000, 1000, 200)])
+def test_c3_chain_ragged(fc, orc, M, N, K):
+    run_and_check(fc, orc, wl.gemm_bias_gelu_scale_clamp(M, N, K, "var"), 4)
+    run_and_check(fc, orc, replace(wl.gemm_bias_gelu_scale_clamp(M, N, K, "var"), out_dtype="f32"), 4)
+
+
+def test_c3_full_size_sampled_rows(fc, orc):
+    ch = wl.CONFIGS["C3"]()
+    ins = wl.make_inputs(ch, 0)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    rows = np.unique(np.concatenate([np.arange(0, 8192, 397), [0, 127, 128, 8191]]))
+    sub = replace(ch, M=len(rows))
+    ref = orc.run_chain(sub, [ins[0][rows], ins[1], ins[2]])
+    util.check(outs[0][torch.from_numpy(rows).cuda()], ref["main"], "C3 (sampled rows)")
+    assert torch.isfinite(outs[0].float()).all()
+
+
+# ------------------------------------------------------------------ kernel (c): GEMM + cross-tile row softmax
+def _check_softmax_rows(t):
+    s = t.float().sum(1)
+    assert float((s - 1).abs().max()) <= 4e-3, "softmax rows must sum to 1 within bf16 rounding"
+
+
+@pytest.mark.parametrize("variant", ["std", "var"])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 1024, 256), (300, 1000, 136), (512, 4096, 128), (130, 264, 72)])
+def test_c4_softmax_reduced(fc, orc, M, N, K, variant):
+    outs, _, _ = run_and_check(fc, orc, wl.gemm_softmax(M, N, K, variant), 1)
+    _check_softmax_rows(outs[0])
+
+
+def test_c4_softmax_dominant_logits(fc, orc):
+    """A few logits per row far above the rest, in different column tiles: stresses the max merge."""
+    ch = wl.gemm_softmax(256, 2048, 64, "var")
+    A, B = wl.make_inputs(ch, 2)
+    Af = rng.bf16_bits_to_f32(A).copy()
+    Bf = rng.bf16_bits_to_f32(B).copy()
+    Af[:, 0] = 8.0
+    Bf[:, 0] = 0.0
+    Bf[[5, 300, 900, 2047], 0] = [6.0, 6.25, 3.0, 6.25]     # +48..50 on columns in tiles 0, 1, 3, 7
+    ins = [rng.store(Af, "bf16"), rng.store(Bf, "bf16")]
+    outs, _, _ = run_and_check(fc, orc, ch, ins=ins)
+    _check_softmax_rows(outs[0])
+
+
+def test_c4_full_size_sampled_rows(fc, orc):
+    ch = wl.CONFIGS["C4"]()
+    for variant in ("std", "var"):
+        ch = wl.gemm_softmax(variant=variant)
+        ins = wl.make_inputs(ch, 0)
+        outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+        fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+        fc.fc_get_async_status()
+        rows = np.unique(np.concatenate([np.arange(0, 4096, 211), [0, 127, 128, 4095]]))
+        sub = replace(ch, M=len(rows))
+        ref = orc.run_chain(sub, [ins[0][rows], ins[1]])
+        util.check(outs[0][torch.from_numpy(rows).cuda()], ref["reduce"], f"C4 {variant} (sampled rows)")
+        _check_softmax_rows(outs[0])
+
+
+# ------------------------------------------------------------------ kernel (d): implicit-GEMM conv + ReLU + avg-pool
+def _delta_weights(C, r, s):
+    w = np.zeros((C, 3, 3, C), np.float32)
+    w[np.arange(C), r, s, np.arange(C)] = 1.0
+    return rng.store(w, "bf16")
+
+
+@pytest.mark.parametrize("r,s", [(1, 1), (0, 0), (2, 1), (0, 2)])
+def test_conv_delta_kernels_pool_shifted_image(fc, orc, r, s):
+    """A one-hot 3x3 kernel copies a shifted image, so the pooled output is the mean of ReLU(image)
+    minus the row / column that falls off the edge: pins tap direction and zero padding."""
+    ch = replace(wl.conv_bias_relu_avgpool(batch=3, H=10, W=12, Cin=64, Cout=64), ops=(("relu",),))
+    x = wl.make_inputs(ch, 6)[0]
+    run_and_check(fc, orc, ch, ins=[x, _delta_weights(64, r, s)])
+
+
+@pytest.mark.parametrize("batch,H,W,Cin,Cout", [(1, 8, 16, 64, 64), (2, 14, 14, 64, 128), (3, 7, 9, 128, 256),
+                                                (2, 56, 56, 64, 64), (5, 5, 5, 72, 40), (1, 1, 1, 8, 8)])
+@pytest.mark.parametrize("seed", [0, 1])
+def test_conv_chain_reduced(fc, orc, batch, H, W, Cin, Cout, seed):
+    run_and_check(fc, orc, wl.conv_bias_relu_avgpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout), seed)
+
+
+def test_conv_all_ones_closed_form(fc, orc):
+    ch = replace(wl.conv_bias_relu_avgpool(batch=2, H=56, W=56, Cin=256, Cout=256), ops=())
+    x = rng.store(np.ones((2, 56, 56, 256), np.float32), "bf16")
+    w = rng.store(np.ones((256, 3, 3, 256), np.float32), "bf16")
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(x), fc.to_device(w)], outs)
+    fc.fc_get_async_status()
+    np.testing.assert_allclose(util.to_f64(outs[0]), 2249.469387755102, rtol=1e-5)
+
+
+def test_c5_full_size_sampled_images(fc, orc):
+    ch = wl.CONFIGS["C5"]()
+    ins = wl.make_inputs(ch, 0)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    imgs = np.array([0, 13, 31])
+    sub = replace(ch, batch=len(imgs))
+    ref = orc.run_chain(sub, [ins[0][imgs], ins[1], ins[2]])
+    util.check(outs[0][torch.from_numpy(imgs).cuda()], ref["reduce"], "C5 (sampled images)")
+    assert torch.isfinite(outs[0]).all()
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+def test_run_host_matches_device_path(fc, orc):
+    ch = wl.gemm_bias_gelu_scale_clamp(256, 512, 128, "var")
+    ins = wl.make_inputs(ch, 3)
+    host_in = [fc.to_device(a, "cpu").pin_memory() for a in ins]
+    host_out = util.poison_(fc.binding.output_tensors(ch, "cpu", pinned=True))
+    spec = fc.make_spec(ch)
+    staging = torch.empty(fc.fc_staging_size(spec, host_in, host_out), dtype=torch.uint8, device="cuda")
+    fc.run_chain_host(ch, host_in, host_out, staging)
+    fc.fc_get_async_status()
+    dev_out = fc.run_chain(ch, [t.cuda() for t in host_in])
+    torch.cuda.synchronize()
+    assert torch.equal(dev_out[0].cpu(), host_out[0])
+    util.check(host_out[0], orc.run_chain(ch, ins)["main"], "fc_run_host")
