@@ -1,0 +1,468 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-chain hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl reference]
+
+A step is one fc_run of the workload's whole chain (producer -> epilogue -> reduction) over one
+batch of seeded synthetic input.  The headline workload is C2 (the memory-bound chain the metric is
+quoted on); `--workload C1|C3|C4|C5` selects another.  Rank 0 prints ONE JSON line.  With N > 1
+(launched by torch.distributed.run) every rank runs its own batch (the chains' rows / images are
+independent problems: weak scaling, no data-path collective); the time is the max over ranks.
+
+`value` times fc_run with inputs resident in HBM (CUDA events on the launch stream); `e2e` times
+fc_run_host with pinned HOST buffers, copies inside the timed region.  `roofline` relates the
+kernel's algorithmic bytes or FLOPs per launch to the measured peak of this machine's B200s.
+`cpu_baseline` is the CPU oracle, as it stands, on a bounded sample of the same workload.
+`--impl reference` times that oracle as the reference arm.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from fc_inputs import workloads as wl  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                p = json.load(f)
+            return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured (MEASURED_PEAKS.json)"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback (earlier measurement on this pool)"
+
+
+def load_traffic(workload: str):
+    """DRAM bytes per launch from the committed ncu capture of this workload's kernel, if any."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                return json.load(f).get(workload)
+        except Exception:
+            return None
+    return None
+
+
+# ------------------------------------------------------------------------------ units per workload
+def units(ch):
+    """(metric name, unit, algorithmic units per step, roofline bound)."""
+    if ch.producer == "elementwise":
+        return "fused_chain_throughput", "GB/s", wl.algorithmic_bytes(ch) / 1e9, "hbm"
+    return "fused_chain_throughput", "TFLOP/s", ch.flops() / 1e12, "tensor" if ch.in_dtype == "bf16" else "alu"
+
+
+def dtype_of(ch):
+    return "bf16" if ch.in_dtype == "bf16" else "f32"
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) in a background thread."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.samples = []
+        self._stop = threading.Event()
+        self._period = period_s
+        self._thread = None
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                self.samples.append((time.perf_counter(), int(mhz), int(reasons)))
+            except Exception:
+                pass
+            time.sleep(self._period)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float, note: str):
+        if self._nv is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML not available"}
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        sel = [s for s in self.samples if t0 <= s[0] <= t1]
+        if not sel:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "note": note}
+        bits = 0
+        for s in sel:
+            bits |= s[2]
+        reasons = sorted(n for b, n in names.items() if bits & b)
+        return {"sm_mhz": statistics.median(s[1] for s in sel), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(sel), "note": note}
+
+
+# ------------------------------------------------------------------------------ eager context
+def eager_fn(ch, t):
+    """The unfused PyTorch eager sequence of the chain (context only; never a parity reference)."""
+    import torch
+    import torch.nn.functional as F
+    name = ch.name
+    if name == "gemm_f32_bias_relu":
+        return lambda: torch.relu(F.linear(t[0], t[1], t[2]))
+    if name == "ew_affine_gelu_add_lse":
+        def f():
+            y = F.gelu(t[0] * t[1] + t[2], approximate="tanh") + t[3]
+            return y, torch.logsumexp(y.float(), 1)
+        return f
+    if name == "gemm_bf16_bias_gelu_scale_clamp":
+        return lambda: torch.clamp(F.gelu(F.linear(t[0], t[1], t[2]), approximate="tanh") * 0.5, -1.0, 1.0)
+    if name == "gemm_bf16_row_softmax":
+        return lambda: torch.softmax(t[0] @ t[1].t(), dim=1)
+    if name == "conv_bf16_bias_relu_avgpool":
+        x = t[0].permute(0, 3, 1, 2)            # NHWC storage viewed as NCHW = channels_last
+        w = t[1].permute(0, 3, 1, 2)
+        return lambda: F.adaptive_avg_pool2d(torch.relu(F.conv2d(x, w, t[2], padding=ch.pad)), 1).float()
+    return None
+
+
+def time_loop(fn, steps, warmup, flush=None):
+    """CUDA-event timing on the current stream.  Without `flush`: one event pair around `steps`
+    back-to-back calls.  With `flush`: an L2-evicting write before every call, one pair per call."""
+    import torch
+    for _ in range(warmup):
+        if flush is not None:
+            flush()
+        fn()
+    torch.cuda.synchronize()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+    total = 0.0
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        flush()
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    for a, b in evs:
+        total += a.elapsed_time(b)
+    return total / steps
+
+
+# ------------------------------------------------------------------------------ CPU oracle legs
+def oracle_sample(ch, ins, target_s=15.0):
+    """A bounded sample of the workload for the CPU oracle: leading rows (or images) sized so that the
+    oracle runs for roughly `target_s` seconds.  Returns (sub-chain, sub-inputs, description)."""
+    import oracle
+    threads = oracle.num_threads()
+    # rough oracle speed on these host cores: ~0.5 GFLOP/s/thread for the naive contraction,
+    # ~15 M elements/s/thread for the transcendental elementwise chain
+    if ch.producer == "elementwise":
+        rows = int(min(ch.M, max(1, target_s * 15e6 * threads / ch.N)))
+        sub = replace(ch, M=rows)
+        sub_ins = [a[:rows] if a.ndim == 2 else a for a in ins]
+        return sub, sub_ins, f"first {rows} of {ch.M} rows"
+    if ch.producer == "gemm_nt":
+        rows = int(min(ch.M, max(1, target_s * 0.5e9 * threads / (2.0 * ch.N * ch.K))))
+        sub = replace(ch, M=rows)
+        sub_ins = [ins[0][:rows]] + list(ins[1:])
+        return sub, sub_ins, f"first {rows} of {ch.M} rows of A (all of B)"
+    per_img = 2.0 * ch.OH * ch.OW * ch.Cout * ch.R * ch.S * ch.Cin
+    n = int(min(ch.batch, max(1, target_s * 0.5e9 * threads / per_img)))
+    sub = replace(ch, batch=n)
+    return sub, [ins[0][:n]] + list(ins[1:]), f"first {n} of {ch.batch} images"
+
+
+def sample_units(sub):
+    _, _, u, _ = units(sub)
+    return u
+
+
+def cpu_baseline_leg(ch, ins, gpu_outputs=None, target_s=15.0):
+    """Times the oracle on the sample and (when GPU outputs are given) compares them on the sample."""
+    import oracle
+    oracle.build()
+    sub, sub_ins, desc = oracle_sample(ch, ins, target_s)
+    t0 = time.perf_counter()
+    ref = oracle.run_chain(sub, sub_ins)
+    dt = time.perf_counter() - t0
+    _, unit, _, _ = units(ch)
+    out = {"value": sample_units(sub) / dt, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": desc, "seconds": round(dt, 3)}
+    if gpu_outputs is not None:
+        from tests import util
+        names = [r for r, _, _ in wl.output_shapes(ch)]
+        n = sub.batch if ch.producer == "conv2d_nhwc" else sub.M
+        worst = {}
+        for name, t in zip(names, gpu_outputs):
+            got = util.to_f64(t[:n])
+            r = ref[name]
+            worst[name] = float(np.abs(got - r).max())
+            util.check(t[:n], r, f"bench {ch.name}:{name}")
+        out["parity_on_sample"] = {"ok": True, "max_abs_err": worst}
+    return out
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    oracle.build()
+    ch = wl.CONFIGS[args.workload]()
+    ins = wl.make_inputs(ch, 0)
+    metric, unit, _, _ = units(ch)
+    sub, sub_ins, desc = oracle_sample(ch, ins, target_s=5.0)
+    for _ in range(min(args.warmup, 1)):
+        oracle.run_chain(sub, sub_ins)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.run_chain(sub, sub_ins)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sample_units(sub) / dt
+    line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: {ch.name}", "step": f"CPU oracle on a sample: {desc}"},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------ main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="C2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-eager", action="store_true")
+    ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (context)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import paper_2602_14293_b200 as fc
+    from paper_2602_14293_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peaks, peaks_src = load_peaks()
+    ch = wl.CONFIGS[args.workload]()
+    metric, unit, units_per_step, bound = units(ch)
+    ins = wl.make_inputs(ch, seed=rank)              # every rank draws its own batch
+    dev_in = [fc.to_device(a) for a in ins]
+    outs = binding.output_tensors(ch, "cuda")
+    spec = fc.make_spec(ch)
+    binding.ensure_workspace(spec)
+    in_bytes = wl.input_bytes(ch)
+    flush_buf = None
+    flush = None
+    if in_bytes <= L2_BYTES:
+        flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+        flush = lambda: flush_buf.zero_()  # noqa: E731
+
+    def step():
+        fc.fc_run(spec, dev_in, outs)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = fc.fc_launch_count()
+    for _ in range(args.warmup):
+        if flush:
+            flush()
+        step()
+    barrier()
+    launches1 = fc.fc_launch_count()
+    t_wall0 = time.perf_counter()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        ms_total = e0.elapsed_time(e1)
+    else:
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in evs:
+            flush()
+            a.record()
+            step()
+            b.record()
+        barrier()
+        ms_total = sum(a.elapsed_time(b) for a, b in evs)
+    t_wall1 = time.perf_counter()
+    launches = fc.fc_launch_count() - launches1
+    fc.fc_get_async_status()
+    ms_total = max_over_ranks(ms_total)
+    ms_per_step = ms_total / args.steps
+    value = world * units_per_step / (ms_per_step * 1e-3)
+
+    clocks = sampler.summary(t_wall0, t_wall1, "sampled during the timed region")
+    if clocks.get("samples", 0) < 3:
+        # the timed region was shorter than a few sampling periods: sample a longer loop of the same kernel
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < 0.4:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize()
+        clocks = sampler.summary(t0, time.perf_counter(), "timed region too short to sample; taken over a 0.4 s loop of the same kernel right after it")
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) ----
+    host_in = [t.cpu().pin_memory() for t in dev_in]
+    host_out = binding.output_tensors(ch, "cpu", pinned=True)
+    staging = torch.empty(fc.fc_staging_size(spec, host_in, host_out), dtype=torch.uint8, device="cuda")
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        fc.fc_run_host(spec, host_in, host_out, staging)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        fc.fc_run_host(spec, host_in, host_out, staging)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+    e2e = {"value": world * units_per_step / (e2e_ms * 1e-3), "unit": unit, "ms_per_step": e2e_ms, "steps": e2e_steps,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- roofline of the (single) kernel of this workload ----
+    if bound == "hbm":
+        peak, peak_unit = peaks["hbm_gbs"], "GB/s"
+        peak_note = f"HBM copy bandwidth, {peaks_src}"
+    elif bound == "tensor":
+        long_region = ms_total > 1000.0
+        peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
+        peak_unit = "TFLOP/s"
+        peak_note = f"cuBLAS bf16 {'sustained' if long_region else 'burst'}, {peaks_src}"
+    else:
+        peak, peak_unit = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
+        peak_note = "fp32 FMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived)"
+    achieved = units_per_step / (ms_per_step * 1e-3)
+    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": peak_unit, "frac": achieved / peak,
+                "traffic": load_traffic(args.workload), "peak_source": peak_note,
+                "algorithmic_units_per_launch": units_per_step, "kernel_ms": ms_per_step}
+
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": dtype_of(ch), "data": "synthetic",
+            "config": {"workload": f"{args.workload}: {ch.name}", "shape": {k: getattr(ch, k) for k in ("M", "N", "K", "batch", "H", "W", "Cin", "Cout") if getattr(ch, k)},
+                       "ops": [o[0] for o in ch.ops], "reduce": ch.reduce,
+                       "l2": "inputs larger than L2, no flush" if flush is None else "L2 flushed (252 MiB write) before every timed step",
+                       "parallelism": f"independent batches per GPU x{world}"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
+
+    if rank == 0 and not args.no_eager:
+        fn = eager_fn(ch, dev_in)
+        if fn is not None:
+            torch.backends.cuda.matmul.allow_tf32 = False
+            torch.backends.cudnn.allow_tf32 = False
+            ems = time_loop(fn, max(5, min(args.steps, 50)), 3, flush)
+            line["eager"] = {"ms_per_step": ems, "value": units_per_step / (ems * 1e-3), "unit": unit,
+                             "note": "unfused PyTorch eager sequence on the same GPU and tensors (context)"}
+
+    if rank == 0 and args.all_configs:
+        per = {}
+        for key in sorted(wl.CONFIGS):
+            if key == args.workload:
+                continue
+            c2 = wl.CONFIGS[key]()
+            i2 = [fc.to_device(a) for a in wl.make_inputs(c2, 0)]
+            o2 = binding.output_tensors(c2, "cuda")
+            s2 = fc.make_spec(c2)
+            binding.ensure_workspace(s2)
+            if flush_buf is None:
+                flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+            fl = (lambda: flush_buf.zero_()) if wl.input_bytes(c2) <= L2_BYTES else None
+            ms = time_loop(lambda: fc.fc_run(s2, i2, o2), 50, 5, fl)
+            _, u2, n2, b2 = units(c2)
+            ent = {"ms": ms, "value": n2 / (ms * 1e-3), "unit": u2, "bound": b2}
+            if b2 == "tensor":
+                ent["frac_of_burst_peak"] = ent["value"] / peaks["bf16_tflops"]
+            f2 = eager_fn(c2, i2)
+            if f2 is not None and not args.no_eager:
+                ent["eager_ms"] = time_loop(f2, 20, 3, fl)
+            per[key] = ent
+            del i2, o2
+        line["per_config"] = per
+
+    sampler.stop()
+    if rank == 0 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline_leg(ch, ins, outs)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -36,7 +36,10 @@ def check_bf16(got: np.ndarray, ref: np.ndarray, what=""):
     rel = err / np.maximum(np.abs(ref), max(floor, 1e-30))
     mx, mean_abs = float(rel.max()), float(err.mean())
     assert mx <= 2e-2, f"{what}: max rel err {mx:.4g} at {np.unravel_index(rel.argmax(), rel.shape)}"
-    assert mean_abs <= 2e-3, f"{what}: mean abs err {mean_abs:.4g}"
+    # a mean over a handful of elements is just one element's bf16 rounding (up to 2^-9 |ref|):
+    # below 256 elements the bound scales with the largest magnitude present
+    mean_bound = 2e-3 if ref.size >= 256 else 2e-3 * max(1.0, float(np.abs(ref).max()))
+    assert mean_abs <= mean_bound, f"{what}: mean abs err {mean_abs:.4g}"
     return mx, mean_abs
 
 
