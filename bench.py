@@ -281,6 +281,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-eager", action="store_true")
     ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (context)")
+    ap.add_argument("--rows", type=int, default=0, help="override M (or the conv batch): a smaller case of the same kernel for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -313,6 +314,8 @@ def main():
 
     peaks, peaks_src = load_peaks()
     ch = wl.CONFIGS[args.workload]()
+    if args.rows > 0:
+        ch = wl.CONFIGS[args.workload](batch=args.rows) if ch.producer == "conv2d_nhwc" else wl.CONFIGS[args.workload](M=args.rows)
     metric, unit, units_per_step, bound = units(ch)
     ins = wl.make_inputs(ch, seed=rank)              # every rank draws its own batch
     dev_in = [fc.to_device(a) for a in ins]

@@ -108,18 +108,231 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
     }
 }
 
+
+// ------------------------------------------------------------------------------------ fast path
+// bf16 rows, N a multiple of 8, 16-byte aligned: [bias | affine]? -> [relu | gelu]? -> [+ tensor]?
+// -> [row logsumexp]?.  One WARP owns a whole row, so the row reduction is a per-lane online
+// (max, sum) plus a single warp shuffle merge: no block-level synchronisation in the row loop.
+// Lane l handles the 16-byte chunks l, l+32, ... (every warp-wide access covers 512 contiguous
+// bytes), four chunks of the input and of the residual tensor in flight per lane.  The per-column
+// vectors are converted to fp32 once per CTA and kept in shared memory.
+struct EwFastParams {
+    const uint4* x;         // [M][N/8]
+    const uint4* res;       // [M][N/8] or null
+    uint4* y;               // [M][N/8] or null
+    float* lse;             // [M] or null
+    const void* vec0; int vec0_dt;   // bias / gamma
+    const void* vec1; int vec1_dt;   // beta
+    long long M;
+    int N;
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+constexpr int kPreNone = 0, kPreBias = 1, kPreAffine = 2;
+constexpr int kActNone = 0, kActRelu = 1, kActGeluPrecise = 2, kActGeluFast = 3;
+constexpr int kGroup = 4;   // chunks in flight per lane and tensor
+
+template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
+__global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams p) {
+    extern __shared__ float svec[];   // PRE != none: vec0 as fp32 [N], then vec1 [N]
+    const int N = p.N;
+    if (PRE != kPreNone) {
+        for (int i = threadIdx.x; i < N; i += kThreads) {
+            svec[i] = load_scalar(p.vec0, p.vec0_dt, i);
+            if (PRE == kPreAffine) svec[N + i] = load_scalar(p.vec1, p.vec1_dt, i);
+        }
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chunks = N >> 3;
+    const long long row_step = (long long) gridDim.x * kWarps;
+
+    for (long long row = (long long) blockIdx.x * kWarps + warp; row < p.M; row += row_step) {
+        const uint4* xr = p.x + row * chunks;
+        const uint4* rr = RES ? p.res + row * chunks : nullptr;
+        uint4* yr = STORE ? p.y + row * chunks : nullptr;
+        float run_m = -CUDART_INF_F, run_s = 0.0f;   // log2 domain: sum of 2^(y*log2e - run_m)
+
+        for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
+            uint4 xv[kGroup], rv[kGroup];
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) {
+                const int c = c0 + 32 * g;
+                if (c < chunks) {
+                    xv[g] = ld_stream(xr + c);
+                    if (RES) rv[g] = ld_stream(rr + c);
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) {
+                const int c = c0 + 32 * g;
+                if (c >= chunks) break;
+                float v[8];
+                v[0] = bf16_lo(xv[g].x); v[1] = bf16_hi(xv[g].x); v[2] = bf16_lo(xv[g].y); v[3] = bf16_hi(xv[g].y);
+                v[4] = bf16_lo(xv[g].z); v[5] = bf16_hi(xv[g].z); v[6] = bf16_lo(xv[g].w); v[7] = bf16_hi(xv[g].w);
+                if (PRE != kPreNone) {
+                    const float4 a0 = *reinterpret_cast<const float4*>(svec + c * 8);
+                    const float4 a1 = *reinterpret_cast<const float4*>(svec + c * 8 + 4);
+                    const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    if (PRE == kPreAffine) {
+                        const float4 b0 = *reinterpret_cast<const float4*>(svec + N + c * 8);
+                        const float4 b1 = *reinterpret_cast<const float4*>(svec + N + c * 8 + 4);
+                        const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) v[j] = fmaf(v[j], a[j], b[j]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) v[j] += a[j];
+                    }
+                }
+                float r[8];
+                if (RES) {
+                    r[0] = bf16_lo(rv[g].x); r[1] = bf16_hi(rv[g].x); r[2] = bf16_lo(rv[g].y); r[3] = bf16_hi(rv[g].y);
+                    r[4] = bf16_lo(rv[g].z); r[5] = bf16_hi(rv[g].z); r[6] = bf16_lo(rv[g].w); r[7] = bf16_hi(rv[g].w);
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float t = v[j];
+                    if (ACT == kActRelu) t = t < 0.0f ? 0.0f : t;
+                    if (ACT == kActGeluPrecise || ACT == kActGeluFast) {
+                        // z = sqrt(2/pi) (t + 0.044715 t^3); gelu = t / (1 + exp(-2 z))
+                        const float t2 = t * t;
+                        if (ACT == kActGeluPrecise) {
+                            const float w = t * fmaf(t2, -2.0f * kLog2e * 0.7978845608028654f * 0.044715f,
+                                                     -2.0f * kLog2e * 0.7978845608028654f);
+                            const float d = 1.0f + exp2_fast(w);
+                            float inv;
+                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(d));
+                            t = RES ? fmaf(t, inv, r[j]) : t * inv;
+                        } else {
+                            const float z = t * fmaf(t2, 0.7978845608028654f * 0.044715f, 0.7978845608028654f);
+                            const float hv = 0.5f * t;
+                            t = fmaf(hv, tanh_fast(z), RES ? hv + r[j] : hv);
+                        }
+                    } else if (RES) {
+                        t += r[j];
+                    }
+                    v[j] = t;
+                }
+                if (STORE) {
+                    uint4 q;
+                    q.x = pack_bf16x2(v[0], v[1]); q.y = pack_bf16x2(v[2], v[3]);
+                    q.z = pack_bf16x2(v[4], v[5]); q.w = pack_bf16x2(v[6], v[7]);
+                    st_stream(yr + c, q);
+                }
+                if (LSE) {
+                    float cm = fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
+                    const float nm = fmaxf(run_m, cm * kLog2e);
+                    float cs = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) cs += exp2_fast(fmaf(v[j], kLog2e, -nm));
+                    run_s = fmaf(run_s, exp2_fast(run_m - nm), cs);
+                    run_m = nm;
+                }
+            }
+        }
+        if (LSE) {
+            // merge the 32 per-lane pairs (log2 domain)
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, run_m, o);
+                const float os = __shfl_xor_sync(0xffffffffu, run_s, o);
+                const float nm = fmaxf(run_m, om);
+                const float sa = run_m == -CUDART_INF_F ? 0.0f : run_s * exp2_fast(run_m - nm);
+                const float sb = om == -CUDART_INF_F ? 0.0f : os * exp2_fast(om - nm);
+                run_s = sa + sb;
+                run_m = nm;
+            }
+            if (lane == 0) p.lse[row] = (run_m + log2f(run_s)) * kLn2;
+        }
+    }
+}
+
 }  // namespace
 
+// Recognise [bias | affine]? -> [relu | gelu]? -> [add tensor]? and fill the fast-path parameters.
+static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, bool* res) {
+    if (p.x_dt != FC_BF16 || (p.y && p.y_dt != FC_BF16)) return false;
+    if (p.N % 8 != 0 || p.N > 24576) return false;
+    if ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y)) & 15) return false;
+    int i = 0;
+    *pre = kPreNone; *act = kActNone; *res = false;
+    f->vec0 = f->vec1 = nullptr; f->vec0_dt = f->vec1_dt = FC_F32; f->res = nullptr;
+    if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_BIAS_N || p.ops.op[i].kind == FC_OP_AFFINE_N)) {
+        *pre = p.ops.op[i].kind == FC_OP_BIAS_N ? kPreBias : kPreAffine;
+        f->vec0 = p.ops.op[i].p0; f->vec0_dt = p.ops.op[i].dt0;
+        f->vec1 = p.ops.op[i].p1; f->vec1_dt = p.ops.op[i].dt1;
+        ++i;
+    }
+    if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_RELU || p.ops.op[i].kind == FC_OP_GELU_TANH)) {
+        *act = p.ops.op[i].kind == FC_OP_RELU ? kActRelu : kActGeluPrecise;
+        ++i;
+    }
+    if (i < p.ops.n && p.ops.op[i].kind == FC_OP_ADD_TENSOR) {
+        if (p.ops.op[i].dt0 != FC_BF16 || (reinterpret_cast<uintptr_t>(p.ops.op[i].p0) & 15)) return false;
+        *res = true;
+        f->res = (const uint4*) p.ops.op[i].p0;
+        ++i;
+    }
+    if (i != p.ops.n) return false;
+    f->x = (const uint4*) p.x; f->y = (uint4*) p.y; f->lse = p.red; f->M = p.M; f->N = (int) p.N;
+    return true;
+}
+
+template <int PRE, int ACT, bool RES>
+static cudaError_t launch_fast(const EwFastParams& f, bool lse, bool store, int num_sms, cudaStream_t stream) {
+    const size_t smem = PRE == kPreNone ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
+    long long ctas = (f.M + kWarps - 1) / kWarps;
+    int per_sm = smem > 0 ? (int) ((200 * 1024) / smem) : 4;
+    per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);
+    if (ctas > (long long) num_sms * per_sm) ctas = (long long) num_sms * per_sm;
+    auto go = [&](auto kernel) -> cudaError_t {
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int) smem);
+            if (e != cudaSuccess) return e;
+        }
+        kernel<<<(unsigned) ctas, kThreads, smem, stream>>>(f);
+        return cudaGetLastError();
+    };
+    if (lse && store) return go(ew_rows_kernel<PRE, ACT, RES, true, true>);
+    if (lse) return go(ew_rows_kernel<PRE, ACT, RES, true, false>);
+    return go(ew_rows_kernel<PRE, ACT, RES, false, true>);
+}
+
 cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t stream, int* launches) {
+    *launches += 1;
+    EwFastParams f;
+    int pre, act;
+    bool res;
+    const bool lse = p.reduce == FC_RED_ROW_LOGSUMEXP;
+    if (match_fast(p, &f, &pre, &act, &res) && (lse || p.y)) {
+        const bool store = p.y != nullptr;
+#define FC_EW_CASE(PRE_, ACT_)                                                                       \
+    if (pre == PRE_ && act == ACT_)                                                                  \
+        return res ? launch_fast<PRE_, ACT_, true>(f, lse, store, num_sms, stream)                  \
+                   : launch_fast<PRE_, ACT_, false>(f, lse, store, num_sms, stream);
+        FC_EW_CASE(kPreNone, kActNone) FC_EW_CASE(kPreNone, kActRelu) FC_EW_CASE(kPreNone, kActGeluPrecise)
+        FC_EW_CASE(kPreBias, kActNone) FC_EW_CASE(kPreBias, kActRelu) FC_EW_CASE(kPreBias, kActGeluPrecise)
+        FC_EW_CASE(kPreAffine, kActNone) FC_EW_CASE(kPreAffine, kActRelu) FC_EW_CASE(kPreAffine, kActGeluPrecise)
+#undef FC_EW_CASE
+    }
     // precise GELU whenever an fp32 result (the logsumexp, or an fp32 main output) depends on it
-    const bool precise = p.reduce == FC_RED_ROW_LOGSUMEXP || p.y_dt == FC_F32;
+    const bool precise = lse || p.y_dt == FC_F32;
     long long grid = p.M < (long long) num_sms * 8 ? p.M : (long long) num_sms * 8;
     if (grid < 1) grid = 1;
     if (precise)
         ew_generic_kernel<true><<<(unsigned) grid, kThreads, 0, stream>>>(p);
     else
         ew_generic_kernel<false><<<(unsigned) grid, kThreads, 0, stream>>>(p);
-    *launches += 1;
     return cudaGetLastError();
 }
 
