@@ -172,6 +172,11 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             plan->kind = Plan::TC_CONV;
             break;
     }
+    if (plan->kind == Plan::TC_PLAIN || plan->kind == Plan::TC_SOFTMAX || plan->kind == Plan::TC_CONV) {
+        int vecs = 0;
+        for (int i = 0; i < s->n_ops; ++i) vecs += s->ops[i].kind == FC_OP_BIAS_N ? 1 : (s->ops[i].kind == FC_OP_AFFINE_N ? 2 : 0);
+        if (vecs > 3) return fail(FC_ERR_UNSUPPORTED, "tensor-core chains support at most 3 per-column vector operands");
+    }
     int n = 0;
     if (s->reduce == FC_RED_ROW_SOFTMAX) {
         plan->main_index = n++;
@@ -376,7 +381,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             }
             CUtensorMap tmA, tmB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128))) return st;
-            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2))) return st;   // each CTA of a pair loads half
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }
@@ -397,7 +402,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             if ((e = cudaMemsetAsync(p.out, 0, (size_t) spec->batch * spec->Cout * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;
             if ((st = encode_im2col(&tmA, spec, inputs[0].ptr))) return st;
-            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn / 2))) return st;
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }

@@ -10,33 +10,42 @@
 //           epilogue applies ops (bias, ReLU) and sums each channel over the tile's pixels, adding
 //           the scaled partial sums into out[image][channel]
 //
-// One persistent CTA per SM, 192 threads: warp 0 = TMA producer (one lane), warp 1 = MMA issuer
-// (one lane) and owner of the tensor-memory allocation, warps 2..5 = epilogue (warp w reads TMEM
-// lanes 32*(w%4)..).  A ring of kStages shared-memory stages (A 128x64, B BNx64, 128-byte swizzle)
-// is handed over with full/empty mbarriers; two accumulator buffers in tensor memory let the
-// epilogue of tile i overlap the main loop of tile i+1.  Every wait is bounded: on expiry the CTA
-// records FC_ERR_TIMEOUT in the status word, stops storing and drains.
+// Work unit: a 256 x BN output tile owned by a PAIR of CTAs on neighbouring SMs (cluster of 2,
+// tcgen05 cta_group::2).  Each CTA loads its own 128 rows of A and HALF of the B tile, so a k-block
+// costs each SM 16 KB + BN/2 * 128 B of L2 traffic instead of 16 KB + BN * 128 B; the leader CTA's
+// MMA thread issues one 256 x BN x 16 MMA for both, and each CTA keeps the accumulator rows of its
+// own 128 rows in its own tensor memory.  No TMA multicast is used anywhere.
+//
+// Per CTA, 192 threads: warp 0 = TMA producer (one lane), warp 1 = tensor-memory owner and, in the
+// leader, MMA issuer (one lane), warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4)..).
+// Shared-memory stages (A 128x64, B BN/2 x 64, 128-byte swizzle) are handed over with mbarriers:
+// both producers signal the leader's "full" barrier, the leader's commit releases the stage in both
+// CTAs.  Two accumulator buffers in tensor memory let the epilogue of tile i overlap the main loop
+// of tile i+1.  Every wait is bounded: on expiry the CTA records FC_ERR_TIMEOUT in the status word,
+// stops storing and drains.
 #include "dev_common.cuh"
 #include "ptx.cuh"
 
 namespace fc {
 namespace {
 
-constexpr int BM = 128;
+constexpr int BM = 128;          // rows per CTA; the pair covers 2 * BM
 constexpr int BK = 64;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr int kGroupM = 8;  // mode-0 raster: kGroupM row panels share each sweep over the columns
+constexpr int kGroupM = 4;       // mode-0 raster: kGroupM pair-panels share each sweep over the columns
+constexpr int kMaxVecSlots = 3;  // per-column vectors staged in shared memory per tile
 
 template <int BN>
 struct Cfg {
     static constexpr int kABytes = BM * BK * 2;
-    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kBBytes = (BN / 2) * BK * 2;   // this CTA's half of the B tile
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = BN == 256 ? 4 : 6;
+    static constexpr int kStages = BN == 256 ? 6 : 8;
     static constexpr int kTmemCols = 2 * BN;
+    static constexpr int kVecBytes = 2 * kMaxVecSlots * BN * 4;   // double-buffered per-tile vector slices
     static constexpr int kCtrlBytes = 256;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kCtrlBytes + 1024;  // 1024: alignment slack
+    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024;  // 1024: alignment slack
 };
 
 struct Ctrl {
@@ -68,6 +77,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return true;
 }
 
+// pair-tile index -> (pair-panel index, column-tile index)
 __device__ __forceinline__ void tile_coords(int mode, int t, int tiles_m, int tiles_n, int& mb, int& nb) {
     if (mode == 0) {
         const int group = kGroupM * tiles_n;
@@ -98,29 +108,129 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
     return v[0];
 }
 
+// The op list applied to 16 consecutive columns (col0.. within the tile) of one row.  Per-column
+// vectors come from the shared-memory slices staged for this tile (slot order = order of the
+// vector operands in the op list); ADD_TENSOR reads global memory.
+template <bool kPreciseGelu>
+__device__ __forceinline__ void apply_ops16(float (&v)[16], const DevOps& ops, const float* svec, int bn, int col0,
+                                            long long m, long long n0, long long n_limit, long long ld) {
+    int slot = 0;
+#pragma unroll 1
+    for (int i = 0; i < ops.n; ++i) {
+        const DevOp& op = ops.op[i];
+        switch (op.kind) {
+            case FC_OP_BIAS_N: {
+                const float4* b = reinterpret_cast<const float4*>(svec + slot * bn + col0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 t = b[q];
+                    v[4 * q] += t.x; v[4 * q + 1] += t.y; v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
+                }
+                ++slot;
+                break;
+            }
+            case FC_OP_AFFINE_N: {
+                const float4* g = reinterpret_cast<const float4*>(svec + slot * bn + col0);
+                const float4* b = reinterpret_cast<const float4*>(svec + (slot + 1) * bn + col0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 s = g[q], t = b[q];
+                    v[4 * q] = fmaf(v[4 * q], s.x, t.x); v[4 * q + 1] = fmaf(v[4 * q + 1], s.y, t.y);
+                    v[4 * q + 2] = fmaf(v[4 * q + 2], s.z, t.z); v[4 * q + 3] = fmaf(v[4 * q + 3], s.w, t.w);
+                }
+                slot += 2;
+                break;
+            }
+            case FC_OP_RELU:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = v[j] < 0.0f ? 0.0f : v[j];
+                break;
+            case FC_OP_GELU_TANH:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = gelu_tanh<kPreciseGelu>(v[j]);
+                break;
+            case FC_OP_SCALE:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] *= op.f0;
+                break;
+            case FC_OP_CLAMP:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = fminf(fmaxf(v[j], op.f0), op.f1);
+                break;
+            case FC_OP_ADD_TENSOR:
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, m * ld + n0 + j);
+                break;
+            default:
+                break;
+        }
+    }
+}
+
+// 16 fp32 values of one row -> global memory as bf16 or fp32 (vector stores when aligned and in range)
+__device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, const float (&v)[16], long long m,
+                                        long long n0, long long N) {
+    if (out_dt == FC_BF16) {
+        unsigned short* o = (unsigned short*) out + m * N + n0;
+        if (vec_ok && n0 + 16 <= N) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint4 w;
+                w.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
+                w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+                w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+                w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+                reinterpret_cast<uint4*>(o)[q] = w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (n0 + j < N) o[j] = (unsigned short) (pack_bf16x2(v[j], 0.0f) & 0xffffu);
+        }
+    } else {
+        float* o = (float*) out + m * N + n0;
+        if (vec_ok && n0 + 16 <= N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                reinterpret_cast<float4*>(o)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (n0 + j < N) o[j] = v[j];
+        }
+    }
+}
+
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
+    // the same offset in both CTAs of the pair: the MMA addresses the peer's tiles by this CTA's descriptors
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + C::kStages * C::kStageBytes);
+    float* svec_all = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + C::kStages * C::kStageBytes + C::kVecBytes);
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const uint32_t cta_rank = ptx::cluster_ctarank();
+    const bool leader = cta_rank == 0;
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+    const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM);   // pair-panels of 256 rows
+    const int tiles_n = (p.N + BN - 1) / BN;
     const int total_tiles = tiles_m * tiles_n;
-    const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 0;
+    const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
     const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&ctrl->full[s]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->empty[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->full[s]), 1);    // the leader's arrive.expect_tx for both CTAs' bytes
+            ptx::mbar_init(ptx::smem_u32(&ctrl->empty[s]), 1);   // the leader's commit
         }
         for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(ptx::smem_u32(&ctrl->tfull[b]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->tempty[b]), 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->tfull[b]), 1);   // the leader's commit
+            ptx::mbar_init(ptx::smem_u32(&ctrl->tempty[b]), 8);  // 4 epilogue warps of each CTA
         }
         ctrl->abort = 0;
         ptx::fence_mbar_init();
@@ -133,50 +243,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     ptx::tc_fence_before();
     __syncthreads();
+    ptx::cluster_sync();   // the peer's barriers exist before anything is signalled on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                int mb, nb;
-                tile_coords(MODE == 0 ? 0 : 1, t, tiles_m, tiles_n, mb, nb);
+            for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
+                int mb2, nb;
+                tile_coords(MODE == 0 ? 0 : 1, t, tiles_m, tiles_n, mb2, nb);
+                const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
+                const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
                 if constexpr (MODE == 2) {
-                    const int pix = mb * BM, hw = p.OH * p.OW;
-                    img = pix / hw;
-                    const int rem = pix - img * hw;
+                    const int hw = p.OH * p.OW;
+                    img = row0 / hw;
+                    const int rem = row0 - img * hw;
                     oh = rem / p.OW;
                     ow = rem - oh * p.OW;
                 }
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                     if (!(ok = wait_bar(ptx::smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, p.status))) break;
-                    const uint32_t full = ptx::smem_u32(&ctrl->full[s]);
+                    const uint32_t full = ptx::mapa(ptx::smem_u32(&ctrl->full[s]), 0);   // the leader's barrier
                     const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
-                    ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+                    // the leader expects the bytes of both CTAs; the peer's copies signal the same barrier.  A
+                    // peer copy may land before the expectation is posted: the phase cannot complete before
+                    // the leader's arrival, and the peer starts the next phase only after the leader's MMAs
+                    // of this one (the commit that frees the stage) are done.
+                    if (leader) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->full[s]), 2 * C::kStageBytes);
                     if constexpr (MODE == 2) {
                         const int tap = kb / kb_per_tap, c0 = (kb - tap * kb_per_tap) * BK;
                         const int r = tap / p.S, sx = tap - r * p.S;
-                        ptx::tma_load_im2col_4d(sa, &tmA, c0, ow - p.pad, oh - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
-                        ptx::tma_load_2d(sa + C::kABytes, &tmB, tap * p.Cin + c0, nb * BN, full);
+                        ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow - p.pad, oh - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
+                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap * p.Cin + c0, bcol0, full);
                     } else {
-                        ptx::tma_load_2d(sa, &tmA, kb * BK, mb * BM, full);
-                        ptx::tma_load_2d(sa + C::kABytes, &tmB, kb * BK, nb * BN, full);
+                        ptx::tma_load_2d_pair(sa, &tmA, kb * BK, row0, full);
+                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * BK, bcol0, full);
                     }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, BN);
             uint32_t it = 0, tile_iter = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_iter) {
+            for (int t = cluster_id; t < total_tiles && ok; t += num_clusters, ++tile_iter) {
                 const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
                 if (!(ok = wait_bar(ptx::smem_u32(&ctrl->tempty[buf]), aph ^ 1u, abort_flag, p.status))) break;
                 ptx::tc_fence_after();
@@ -187,99 +304,114 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tc_fence_after();
                     const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
                     const uint64_t da = ptx::smem_desc_k128(sa), db = ptx::smem_desc_k128(sa + C::kABytes);
+#ifndef FC_DBG_SKIP_MMA
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
-                        ptx::tc_mma_f16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-                    ptx::tc_commit(ptx::smem_u32(&ctrl->empty[s]));
+                        ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+#endif
+                    ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);     // frees the stage in both CTAs
                 }
-                if (ok) ptx::tc_commit(ptx::smem_u32(&ctrl->tfull[buf]));
+                if (ok) ptx::tc_commit_pair(ptx::smem_u32(&ctrl->tfull[buf]), 3);   // accumulators ready in both CTAs
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue warps
+        // ------------------------------------------------------------------ epilogue warps (both CTAs)
         const int lane_grp = warp & 3;
         const int row = lane_grp * 32 + lane;
+        const int et = threadIdx.x - 64;   // 0..127
         const uint32_t lane_addr = (uint32_t) (lane_grp * 32) << 16;
         const bool precise = p.out_dt == FC_F32;
         const bool out_vec = (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 && (p.N & 7) == 0;
+        const uint32_t tempty_leader = ptx::mapa(ptx::smem_u32(&ctrl->tempty[0]), 0);
         uint32_t tile_iter = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++tile_iter) {
-            int mb, nb;
-            tile_coords(MODE == 0 ? 0 : 1, t, tiles_m, tiles_n, mb, nb);
+        for (int t = cluster_id; t < total_tiles; t += num_clusters, ++tile_iter) {
+            int mb2, nb;
+            tile_coords(MODE == 0 ? 0 : 1, t, tiles_m, tiles_n, mb2, nb);
+            const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+            const int n_tile = nb * BN;
+            float* svec = svec_all + buf * (kMaxVecSlots * BN);
+            // stage this tile's slices of the per-column vectors (fp32) before the accumulator wait
+            {
+                int slot = 0;
+                for (int i = 0; i < p.ops.n && slot < kMaxVecSlots; ++i) {
+                    const DevOp& op = p.ops.op[i];
+                    const int nvec = op.kind == FC_OP_BIAS_N ? 1 : (op.kind == FC_OP_AFFINE_N ? 2 : 0);
+                    for (int k = 0; k < nvec && slot < kMaxVecSlots; ++k, ++slot)
+                        for (int c = et; c < BN; c += kEpiThreads)
+                            svec[slot * BN + c] = n_tile + c < p.N ? load_scalar(k ? op.p1 : op.p0, k ? op.dt1 : op.dt0, n_tile + c) : 0.0f;
+                }
+            }
             // one thread waits for the accumulator; its verdict reaches all four warps through shared
             // memory and a named barrier, so that they leave the loop together or not at all
-            if (threadIdx.x == 64) ctrl->epi_ok[buf] = wait_bar(ptx::smem_u32(&ctrl->tfull[buf]), aph, abort_flag, p.status);
+            if (et == 0) ctrl->epi_ok[buf] = wait_bar(ptx::smem_u32(&ctrl->tfull[buf]), aph, abort_flag, p.status);
             ptx::bar_sync(2, kEpiThreads);
             if (!*(volatile int*) &ctrl->epi_ok[buf]) break;
             ptx::tc_fence_after();
+#ifdef FC_DBG_SKIP_EPI
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
+            continue;
+#endif
             const uint32_t tacc = tmem_base + buf * BN + lane_addr;
             const long long m = (long long) mb * BM + row;
-            const int n_tile = nb * BN;
+            constexpr int kChunks = BN / 16;
 
             if constexpr (MODE == 0) {
+                uint32_t ra[16], rb[16];
+                ptx::tmem_ld_32x16_async(tacc, ra);
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(tacc + c * 32, r);
-                    const int n0 = n_tile + c * 32;
-                    if (m < p.M && n0 < p.N) {
-                        float v[32];
+                for (int c = 0; c < kChunks; c += 2) {
+                    // chunk c is in flight in ra; prefetch c+1 into rb while c is processed, then swap roles
+                    ptx::tmem_wait_ld(ra);
+                    ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
+                    {
+                        const int n0 = n_tile + c * 16;
+                        if (m < p.M && n0 < p.N) {
+                            float v[16];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                        if (precise) apply_ops<32, true>(v, p.ops, m, n0, p.N, p.N);
-                        else apply_ops<32, false>(v, p.ops, m, n0, p.N, p.N);
-                        if (p.out_dt == FC_BF16) {
-                            unsigned short* o = (unsigned short*) p.out + m * p.N + n0;
-                            if (out_vec && n0 + 32 <= p.N) {
+                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
+                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
+                            else apply_ops16<false>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
+                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                        }
+                    }
+                    ptx::tmem_wait_ld(rb);
+                    if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
+                    {
+                        const int n0 = n_tile + (c + 1) * 16;
+                        if (m < p.M && n0 < p.N) {
+                            float v[16];
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    uint4 w;
-                                    w.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
-                                    w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
-                                    w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
-                                    w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
-                                    reinterpret_cast<uint4*>(o)[q] = w;
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (n0 + j < p.N) o[j] = (unsigned short) (pack_bf16x2(v[j], 0.0f) & 0xffffu);
-                            }
-                        } else {
-                            float* o = (float*) p.out + m * p.N + n0;
-                            if (out_vec && n0 + 32 <= p.N) {
-#pragma unroll
-                                for (int q = 0; q < 8; ++q)
-                                    reinterpret_cast<float4*>(o)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (n0 + j < p.N) o[j] = v[j];
-                            }
+                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
+                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, (c + 1) * 16, m, n0, p.N, p.N);
+                            else apply_ops16<false>(v, p.ops, svec, BN, (c + 1) * 16, m, n0, p.N, p.N);
+                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                         }
                     }
                 }
             } else if constexpr (MODE == 1) {
-                // pass 1: (max, sum) of this tile's slice of the row, online over 32-column chunks
+                // pass 1: (max, sum) of this tile's slice of the row, online over 16-column chunks
                 float mx = -CUDART_INF_F, sm = 0.0f;
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(tacc + c * 32, r);
-                    const int n0 = n_tile + c * 32;
+                for (int c = 0; c < kChunks; ++c) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+                    ptx::tmem_wait_ld(r);
+                    const int n0 = n_tile + c * 16;
                     if (m < p.M && n0 < p.N) {
-                        float v[32];
+                        float v[16];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                        apply_ops<32, false>(v, p.ops, m, n0, p.N, p.N);
+                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                        apply_ops16<false>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
                         float cm = -CUDART_INF_F;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
+                        for (int j = 0; j < 16; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
                         const float nm = fmaxf(mx, cm);
                         float cs = 0.0f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) cs += n0 + j < p.N ? exp2_fast((v[j] - nm) * kLog2e) : 0.0f;
+                        for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast((v[j] - nm) * kLog2e) : 0.0f;
                         sm = sm * exp2_fast((mx - nm) * kLog2e) + cs;
                         mx = nm;
                     }
@@ -288,7 +420,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
                 // one thread announces the tile and waits (bounded) for the panel's other tiles
-                if (warp == 2 && lane == 0) {
+                if (et == 0) {
                     ptx::red_release_gpu_add(&p.counters[mb], 1u);
                     const unsigned long long t0 = ptx::globaltimer();
                     unsigned spins = 0;
@@ -319,40 +451,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const float inv = 1.0f / row_s, off = -row_m * kLog2e;
                 // pass 2: normalise straight from tensor memory and store once
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(tacc + c * 32, r);
-                    const int n0 = n_tile + c * 32;
+                for (int c = 0; c < kChunks; ++c) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+                    ptx::tmem_wait_ld(r);
+                    const int n0 = n_tile + c * 16;
                     if (m < p.M && n0 < p.N && store) {
-                        float v[32];
+                        float v[16];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                        apply_ops<32, false>(v, p.ops, m, n0, p.N, p.N);
+                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                        apply_ops16<false>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = exp2_fast(fmaf(v[j], kLog2e, off)) * inv;
-                        if (p.out_dt == FC_BF16) {
-                            unsigned short* o = (unsigned short*) p.out + m * p.N + n0;
-                            if (out_vec && n0 + 32 <= p.N) {
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    uint4 w;
-                                    w.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
-                                    w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
-                                    w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
-                                    w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
-                                    reinterpret_cast<uint4*>(o)[q] = w;
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (n0 + j < p.N) o[j] = (unsigned short) (pack_bf16x2(v[j], 0.0f) & 0xffffu);
-                            }
-                        } else {
-                            float* o = (float*) p.out + m * p.N + n0;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + j < p.N) o[j] = v[j];
-                        }
+                        for (int j = 0; j < 16; ++j) v[j] = exp2_fast(fmaf(v[j], kLog2e, off)) * inv;
+                        store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                     }
                 }
             } else {
@@ -364,28 +475,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int img_last = pix_last >= pix_first ? (int) (pix_last / hw) : img_first - 1;
                 const int my_img = m < p.M ? (int) (m / hw) : -1;
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(tacc + c * 32, r);
-                    const int n0 = n_tile + c * 32;
+                for (int c = 0; c < kChunks; c += 2) {
+                    uint32_t ra[16], rb[16];
+                    ptx::tmem_ld_32x16_async(tacc + c * 16, ra);
+                    ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
+                    ptx::tmem_wait_ld(ra);
+                    ptx::tmem_wait_ld(rb);
+                    const int n0 = n_tile + c * 16;
                     if (n0 >= p.N) continue;
-                    float v[32];
+                    float va[16], vb[16];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                    if (m < p.M) apply_ops<32, true>(v, p.ops, m, n0, p.N, p.N);
+                    for (int j = 0; j < 16; ++j) { va[j] = __uint_as_float(ra[j]); vb[j] = __uint_as_float(rb[j]); }
+                    if (m < p.M) {
+                        apply_ops16<true>(va, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
+                        apply_ops16<true>(vb, p.ops, svec, BN, (c + 1) * 16, m, n0 + 16, p.N, p.N);
+                    }
                     for (int img = img_first; img <= img_last; ++img) {
                         float w[32];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) w[j] = my_img == img ? v[j] : 0.0f;
+                        for (int j = 0; j < 16; ++j) { w[j] = my_img == img ? va[j] : 0.0f; w[16 + j] = my_img == img ? vb[j] : 0.0f; }
                         const float s = warp_transpose_sum(w, lane);
                         if (n0 + lane < p.N) atomicAdd((float*) p.out + (long long) img * p.N + n0 + lane, s * p.inv_hw);
                     }
                 }
             }
-            // hand the accumulator buffer back to the MMA warp
+            // hand the accumulator buffer back to the leader's MMA thread
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tempty[buf]));
+            if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
         }
     }
 
@@ -396,36 +513,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // a wait expired: give copies and MMAs still in flight time to land before releasing memory
         const unsigned long long t0 = ptx::globaltimer();
         while (ptx::globaltimer() - t0 < 2000000ull) __nanosleep(1000);
-        __syncthreads();
     }
+    ptx::cluster_sync();   // neither CTA leaves while the other may still read its tiles or signal its barriers
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, C::kTmemCols);
     }
 }
 
-template <int BN>
-cudaError_t launch_bn(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int grid, cudaStream_t stream) {
+template <int BN, int MODE>
+cudaError_t launch_one(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int num_sms, cudaStream_t stream) {
+    static int max_clusters[64] = {0};   // per device, filled on first use
     const int smem = Cfg<BN>::kSmemBytes;
-    cudaError_t e = cudaSuccess;
-    switch (p.mode) {
-        case 0:
-            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            gemm_tc_kernel<BN, 0><<<grid, kThreads, smem, stream>>>(tmA, tmB, p);
-            break;
-        case 1:
-            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            gemm_tc_kernel<BN, 1><<<grid, kThreads, smem, stream>>>(tmA, tmB, p);
-            break;
-        default:
-            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            gemm_tc_kernel<BN, 2><<<grid, kThreads, smem, stream>>>(tmA, tmB, p);
-            break;
+    auto kernel = gemm_tc_kernel<BN, MODE>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && max_clusters[dev] == 0) {
+        cfg.gridDim = dim3(num_sms & ~1);
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+        if (e != cudaSuccess) return e;
+        max_clusters[dev] = n > 0 ? n : 1;
     }
-    return cudaGetLastError();
+    const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * ((p.N + BN - 1) / BN);
+    int clusters = dev >= 0 && dev < 64 ? max_clusters[dev] : num_sms / 2;
+    if (clusters > num_sms / 2) clusters = num_sms / 2;
+    if (clusters > tiles) clusters = tiles;
+    cfg.gridDim = dim3(2 * clusters);
+    return cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+}
+
+template <int BN>
+cudaError_t launch_bn(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int num_sms, cudaStream_t stream) {
+    switch (p.mode) {
+        case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream);
+        case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream);
+        default: return launch_one<BN, 2>(p, tmA, tmB, num_sms, stream);
+    }
 }
 
 }  // namespace
@@ -434,10 +571,8 @@ size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : Cf
 
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int num_sms,
                            cudaStream_t stream, int* launches) {
-    const int tiles = ((p.M + BM - 1) / BM) * ((p.N + bn - 1) / bn);
-    const int grid = tiles < num_sms ? tiles : num_sms;
     *launches += 1;
-    return bn == 256 ? launch_bn<256>(p, tmA, tmB, grid, stream) : launch_bn<128>(p, tmA, tmB, grid, stream);
+    return bn == 256 ? launch_bn<256>(p, tmA, tmB, num_sms, stream) : launch_bn<128>(p, tmA, tmB, num_sms, stream);
 }
 
 }  // namespace fc
