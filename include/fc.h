@@ -156,6 +156,31 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes);
 fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
 
 /*
+ * GEMM_NT + ROW_SOFTMAX for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)
+ *
+ * Some callers have no allocator to hand: a plug-in that is given tensors but no memory pool, a
+ * latency-critical loop or callback where cudaMalloc (which may synchronise the whole device) is
+ * off limits, or a process whose device memory was reserved up front by another component.  They
+ * cannot provide the workspace that fc_set_workspace wants.  This entry point runs the same kernel as fc_run, but takes its scratch
+ * (per-tile row maxima and sums, per-panel arrival counters) from a fixed array that is part of
+ * the library image: FC_STATIC_SCRATCH_BYTES bytes of device memory, resident on every GPU that
+ * loads the library until the process exits.  The caller passes inputs and outputs exactly as to
+ * fc_run (device pointers); nothing is allocated or freed, here or in any library this calls.
+ *
+ * Limits and rules.  Only GEMM_NT with reduce == FC_RED_ROW_SOFTMAX; other chains return
+ * FC_ERR_UNSUPPORTED.  A spec whose fc_workspace_size exceeds FC_STATIC_SCRATCH_BYTES returns
+ * FC_ERR_WORKSPACE ("needs N bytes, the built-in scratch holds M").  The first call on each device
+ * looks up the array's device address (with that device current); make that first call outside
+ * any stream capture.  All calls on a device share the one array, which keeps whatever the last
+ * call left in it: the counters are cleared on the stream before each launch, and two calls that
+ * overlap on the GPU (different streams, no dependency) race on it and give wrong results.
+ */
+#define FC_STATIC_SCRATCH_BYTES (1u << 20)
+fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, const fc_tensor* inputs, int n_inputs,
+                                        fc_tensor* outputs, int n_outputs, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then reads and clears the device status word of the current
  * device.  Returns FC_OK, FC_ERR_TIMEOUT (a bounded device-side wait expired in some launch since
  * the last call) or FC_ERR_CUDA.

@@ -71,6 +71,8 @@ def lib():
         L.fc_run_host.restype = ctypes.c_int
         L.fc_staging_size.argtypes = [ps, pt, ctypes.c_int, pt, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
         L.fc_staging_size.restype = ctypes.c_int
+        L.fc_run_softmax_static_scratch.argtypes = [ps, pt, ctypes.c_int, pt, ctypes.c_int, ctypes.c_void_p]
+        L.fc_run_softmax_static_scratch.restype = ctypes.c_int
         L.fc_workspace_size.argtypes = [ps, ctypes.POINTER(ctypes.c_size_t)]
         L.fc_workspace_size.restype = ctypes.c_int
         L.fc_set_workspace.argtypes = [ctypes.c_void_p, ctypes.c_size_t]
@@ -168,6 +170,16 @@ def fc_run(spec: fc_chain_spec, inputs: Sequence[torch.Tensor], outputs: Sequenc
     """fc_run of the C ABI: device tensors in, device tensors out, enqueued on `stream`."""
     _check(lib().fc_run(ctypes.byref(spec), _tensor_array(inputs), len(inputs), _tensor_array(outputs), len(outputs),
                         _stream_handle(stream)), "fc_run")
+
+
+def fc_run_softmax_static_scratch(spec: fc_chain_spec, inputs: Sequence[torch.Tensor], outputs: Sequence[torch.Tensor],
+                                  stream=None) -> None:
+    """GEMM + row softmax for callers that cannot allocate: same arguments as fc_run, scratch taken from
+    the fixed array built into the library (no workspace to register, nothing allocated).  Calls that
+    overlap on the GPU share that array and race; see include/fc.h for the size limit."""
+    _check(lib().fc_run_softmax_static_scratch(ctypes.byref(spec), _tensor_array(inputs), len(inputs),
+                                               _tensor_array(outputs), len(outputs), _stream_handle(stream)),
+           "fc_run_softmax_static_scratch")
 
 
 def fc_staging_size(spec, inputs, outputs) -> int:

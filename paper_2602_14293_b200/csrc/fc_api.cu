@@ -529,3 +529,62 @@ const char* fc_last_error(void) { return t_err; }
 int fc_version(void) { return FC_VERSION; }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ built-in scratch (no allocation)
+// Scratch of fc_run_softmax_static_scratch.  Lives in the library image on every device that loads
+// it.  In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[FC_STATIC_SCRATCH_BYTES];
+
+namespace {
+void* g_static_scratch_ptr[fc::kMaxDevices] = {nullptr};   // device address per device, looked up once
+}
+
+extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, const fc_tensor* inputs, int n_inputs,
+                                                   fc_tensor* outputs, int n_outputs, void* cuda_stream) {
+    Plan plan;
+    fc_status st;
+    if ((st = validate_spec(spec, &plan))) return st;
+    if (plan.kind != Plan::TC_SOFTMAX) return fail(FC_ERR_UNSUPPORTED, "the built-in scratch serves GEMM_NT + ROW_SOFTMAX chains only");
+    if ((st = validate_tensors(spec, plan, inputs, n_inputs, outputs, n_outputs))) return st;
+    const size_t need = softmax_workspace_bytes(spec->M, spec->N);
+    if (need > FC_STATIC_SCRATCH_BYTES)
+        return fail(FC_ERR_WORKSPACE, "this chain needs %zu bytes of scratch, the built-in scratch holds %u", need, (unsigned) FC_STATIC_SCRATCH_BYTES);
+    DeviceInfo* dev;
+    int ordinal = 0;
+    if ((st = get_device(&dev, &ordinal))) return st;
+    void* scratch = nullptr;
+    {
+        // set-up, once per device, with that device current: the array's address on THIS device
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!g_static_scratch_ptr[ordinal]) {
+            void* ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            if (e != cudaSuccess || !ptr) return fail(FC_ERR_CUDA, "cudaGetSymbolAddress(built-in scratch): %s", cudaGetErrorString(e));
+            g_static_scratch_ptr[ordinal] = ptr;
+        }
+        scratch = g_static_scratch_ptr[ordinal];
+    }
+    cudaStream_t stream = (cudaStream_t) cuda_stream;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.mode = 1;
+    p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+    p.out = outputs[plan.main_index].ptr; p.out_dt = spec->out_dtype;
+    p.status = dev->status;
+    build_ops(spec, inputs, &p.ops);
+    const long long panels = (spec->M + 127) / 128;
+    const size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
+    p.counters = (unsigned int*) scratch;
+    p.stats = (float2*) ((char*) scratch + counters);
+    // the array keeps the previous call's contents: the arrival counters must start at zero
+    cudaError_t e = cudaMemsetAsync(p.counters, 0, counters, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    CUtensorMap tmA, tmB;
+    if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128))) return st;
+    if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, kSoftmaxBN / 2))) return st;
+    int launches = 0;
+    e = launch_gemm_tc(p, tmA, tmB, kSoftmaxBN, dev->num_sms, stream, &launches);
+    g_launches.fetch_add((uint64_t) launches);
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    return FC_OK;
+}
