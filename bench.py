@@ -291,33 +291,18 @@ def main():
     import paper_2602_14293_b200 as fc
     from paper_2602_14293_b200 import binding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    from paper_2602_14293_b200.ranks import Ranks
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    rk = Ranks("nccl")
+    rank, world, local_rank = rk.rank, rk.world, rk.local_rank
+    barrier, max_over_ranks = rk.barrier, rk.max_over_ranks
 
     peaks, peaks_src = load_peaks()
     ch = wl.CONFIGS[args.workload]()
     if args.rows > 0:
         ch = wl.CONFIGS[args.workload](batch=args.rows) if ch.producer == "conv2d_nhwc" else wl.CONFIGS[args.workload](M=args.rows)
     metric, unit, units_per_step, bound = units(ch)
-    ins = wl.make_inputs(ch, seed=rank)              # every rank draws its own batch
+    ins = wl.make_inputs(ch, seed=rk.batch_seed(0))   # every rank draws its own batch
     dev_in = [fc.to_device(a) for a in ins]
     outs = binding.output_tensors(ch, "cuda")
     spec = fc.make_spec(ch)
@@ -364,7 +349,7 @@ def main():
     fc.fc_get_async_status()
     ms_total = max_over_ranks(ms_total)
     ms_per_step = ms_total / args.steps
-    value = world * units_per_step / (ms_per_step * 1e-3)
+    value = rk.aggregate(units_per_step, ms_per_step)
 
     clocks = sampler.summary(t_wall0, t_wall1, "sampled during the timed region")
     if clocks.get("samples", 0) < 3:
@@ -393,7 +378,7 @@ def main():
     e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
     h2d = sum(t.numel() * t.element_size() for t in host_in)
     d2h = sum(t.numel() * t.element_size() for t in host_out)
-    e2e = {"value": world * units_per_step / (e2e_ms * 1e-3), "unit": unit, "ms_per_step": e2e_ms, "steps": e2e_steps,
+    e2e = {"value": rk.aggregate(units_per_step, e2e_ms), "unit": unit, "ms_per_step": e2e_ms, "steps": e2e_steps,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # ---- roofline of the (single) kernel of this workload ----
@@ -461,9 +446,7 @@ def main():
         line["cpu_baseline"] = cpu_baseline_leg(ch, ins, outs)
     if rank == 0:
         print(json.dumps(line))
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    rk.finish()
     return 0
 
 
