@@ -16,13 +16,16 @@
 // MMA thread issues one 256 x BN x 16 MMA for both, and each CTA keeps the accumulator rows of its
 // own 128 rows in its own tensor memory.  No TMA multicast is used anywhere.
 //
-// Per CTA, 192 threads: warp 0 = TMA producer (one lane), warp 1 = tensor-memory owner and, in the
-// leader, MMA issuer (one lane), warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4)..).
+// Per CTA, 320 threads: warp 0 = TMA producer (one lane), warp 1 = tensor-memory owner and, in the
+// leader, MMA issuer (one lane), warps 2..9 = epilogue: warp w reads TMEM lanes 32*(w%4).. and the
+// column half (w-2)/4 of the tile, so two warps per scheduler interleave their dependent chains.
 // Shared-memory stages (A 128x64, B BN/2 x 64, 128-byte swizzle) are handed over with mbarriers:
 // both producers signal the leader's "full" barrier, the leader's commit releases the stage in both
 // CTAs.  Two accumulator buffers in tensor memory let the epilogue of tile i overlap the main loop
 // of tile i+1.  Every wait is bounded: on expiry the CTA records FC_ERR_TIMEOUT in the status word,
 // stops storing and drains.
+#include <cstdio>
+
 #include "dev_common.cuh"
 #include "ptx.cuh"
 
@@ -31,8 +34,8 @@ namespace {
 
 constexpr int BM = 128;          // rows per CTA; the pair covers 2 * BM
 constexpr int BK = 64;
-constexpr int kThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kThreads = 320;
+constexpr int kEpiThreads = 256;
 constexpr int kGroupM = 4;       // mode-0 raster: kGroupM pair-panels share each sweep over the columns
 constexpr int kMaxVecSlots = 3;  // per-column vectors staged in shared memory per tile
 
@@ -45,7 +48,7 @@ struct Cfg {
     static constexpr int kTmemCols = 2 * BN;
     static constexpr int kVecBytes = 2 * kMaxVecSlots * BN * 4;   // double-buffered per-tile vector slices
     static constexpr int kCtrlBytes = 256;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024;  // 1024: alignment slack
+    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024 + 1024;  // exchange + alignment slack
 };
 
 struct Ctrl {
@@ -211,9 +214,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float* svec_all = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes);
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + C::kStages * C::kStageBytes + C::kVecBytes);
+    float2* xchg = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes + C::kVecBytes + C::kCtrlBytes);
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef FC_DBG_CLOCK
+    const long long dbg_c0 = clock64();
+    const unsigned long long dbg_t0 = ptx::globaltimer();
+#endif
     const uint32_t cta_rank = ptx::cluster_ctarank();
     const bool leader = cta_rank == 0;
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
@@ -230,7 +238,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tfull[b]), 1);   // the leader's commit
-            ptx::mbar_init(ptx::smem_u32(&ctrl->tempty[b]), 8);  // 4 epilogue warps of each CTA
+            ptx::mbar_init(ptx::smem_u32(&ctrl->tempty[b]), 16); // 8 epilogue warps of each CTA
         }
         ctrl->abort = 0;
         ptx::fence_mbar_init();
@@ -317,8 +325,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         // ------------------------------------------------------------------ epilogue warps (both CTAs)
         const int lane_grp = warp & 3;
+        const int half = (warp - 2) >> 2;  // which half of the tile's columns this warp handles
         const int row = lane_grp * 32 + lane;
-        const int et = threadIdx.x - 64;   // 0..127
+        const int et = threadIdx.x - 64;   // 0..255
         const uint32_t lane_addr = (uint32_t) (lane_grp * 32) << 16;
         const bool precise = p.out_dt == FC_F32;
         const bool out_vec = (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 && (p.N & 7) == 0;
@@ -354,9 +363,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
             continue;
 #endif
-            const uint32_t tacc = tmem_base + buf * BN + lane_addr;
+            constexpr int kChunks = BN / 32;           // 16-column chunks per thread (half a tile row)
+            const int col_half = half * (BN / 2);
+            const uint32_t tacc = tmem_base + buf * BN + col_half + lane_addr;
             const long long m = (long long) mb * BM + row;
-            constexpr int kChunks = BN / 16;
+            const int n_half = n_tile + col_half;
 
             if constexpr (MODE == 0) {
                 uint32_t ra[16], rb[16];
@@ -367,27 +378,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_wait_ld(ra);
                     ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
                     {
-                        const int n0 = n_tile + c * 16;
+                        const int n0 = n_half + c * 16;
                         if (m < p.M && n0 < p.N) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
-                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
-                            else apply_ops16<false>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
+#ifndef FC_DBG_NO_MATH
+                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                            else apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+#endif
+#ifndef FC_DBG_NO_STORE
                             store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+#else
+                            if (v[3] == 1.2345f) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+#endif
                         }
                     }
+#ifdef FC_DBG_SLEEP
+                    __nanosleep(FC_DBG_SLEEP);
+#endif
                     ptx::tmem_wait_ld(rb);
                     if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
                     {
-                        const int n0 = n_tile + (c + 1) * 16;
+                        const int n0 = n_half + (c + 1) * 16;
                         if (m < p.M && n0 < p.N) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
-                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, (c + 1) * 16, m, n0, p.N, p.N);
-                            else apply_ops16<false>(v, p.ops, svec, BN, (c + 1) * 16, m, n0, p.N, p.N);
+#ifndef FC_DBG_NO_MATH
+                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
+                            else apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
+#endif
+#ifndef FC_DBG_NO_STORE
                             store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+#else
+                            if (v[3] == 1.2345f) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+#endif
                         }
                     }
                 }
@@ -399,12 +425,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     uint32_t r[16];
                     ptx::tmem_ld_32x16_async(tacc + c * 16, r);
                     ptx::tmem_wait_ld(r);
-                    const int n0 = n_tile + c * 16;
+                    const int n0 = n_half + c * 16;
                     if (m < p.M && n0 < p.N) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                        apply_ops16<false>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
+                        apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                         float cm = -CUDART_INF_F;
 #pragma unroll
                         for (int j = 0; j < 16; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
@@ -416,7 +442,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         mx = nm;
                     }
                 }
-                if (m < p.M) __stcg(&p.stats[m * tiles_n + nb], make_float2(mx, sm));
+                // the two column halves of a row meet in shared memory; the lower half publishes the tile's pair
+                if (half == 1) xchg[row] = make_float2(mx, sm);
+                ptx::bar_sync(1, kEpiThreads);
+                if (half == 0 && m < p.M) {
+                    const float2 o = xchg[row];
+                    const MaxSum a = ms_merge(MaxSum{mx, sm}, MaxSum{o.x, o.y});
+                    __stcg(&p.stats[m * tiles_n + nb], make_float2(a.m, a.s));
+                }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
                 // one thread announces the tile and waits (bounded) for the panel's other tiles
@@ -455,12 +488,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     uint32_t r[16];
                     ptx::tmem_ld_32x16_async(tacc + c * 16, r);
                     ptx::tmem_wait_ld(r);
-                    const int n0 = n_tile + c * 16;
+                    const int n0 = n_half + c * 16;
                     if (m < p.M && n0 < p.N && store) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                        apply_ops16<false>(v, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
+                        apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = exp2_fast(fmaf(v[j], kLog2e, off)) * inv;
                         store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
@@ -481,14 +514,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
                     ptx::tmem_wait_ld(ra);
                     ptx::tmem_wait_ld(rb);
-                    const int n0 = n_tile + c * 16;
+                    const int n0 = n_half + c * 16;
                     if (n0 >= p.N) continue;
                     float va[16], vb[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) { va[j] = __uint_as_float(ra[j]); vb[j] = __uint_as_float(rb[j]); }
                     if (m < p.M) {
-                        apply_ops16<true>(va, p.ops, svec, BN, c * 16, m, n0, p.N, p.N);
-                        apply_ops16<true>(vb, p.ops, svec, BN, (c + 1) * 16, m, n0 + 16, p.N, p.N);
+                        apply_ops16<true>(va, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                        apply_ops16<true>(vb, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0 + 16, p.N, p.N);
                     }
                     for (int img = img_first; img <= img_last; ++img) {
                         float w[32];
@@ -509,6 +542,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------------------------------------------------------------- teardown
     ptx::tc_fence_before();
     __syncthreads();
+#ifdef FC_DBG_CLOCK
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const long long dc = clock64() - dbg_c0;
+        const unsigned long long dt = ptx::globaltimer() - dbg_t0;
+        printf("kernel: %lld cycles in %llu ns -> %.0f MHz\n", dc, dt, 1e3 * (double) dc / (double) dt);
+    }
+#endif
     if (*abort_flag) {
         // a wait expired: give copies and MMAs still in flight time to land before releasing memory
         const unsigned long long t0 = ptx::globaltimer();
