@@ -49,6 +49,7 @@ __device__ __forceinline__ float gelu_tanh(float v) {
     }
 }
 
+
 __device__ __forceinline__ float load_scalar(const void* p, int dt, long long i) {
     if (dt == FC_BF16) return __uint_as_float(((uint32_t) __ldg((const unsigned short*) p + i)) << 16);
     return __ldg((const float*) p + i);

@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
 // -> [row logsumexp]?.  One WARP owns a whole row, so the row reduction is a per-lane online
 // (max, sum) plus a single warp shuffle merge: no block-level synchronisation in the row loop.
 // Lane l handles the 16-byte chunks l, l+32, ... (every warp-wide access covers 512 contiguous
-// bytes), four chunks of the input and of the residual tensor in flight per lane.  The per-column
+// bytes).  The per-column
 // vectors are converted to fp32 once per CTA and kept in shared memory.
 struct EwFastParams {
     const uint4* x;         // [M][N/8]
@@ -141,6 +141,86 @@ constexpr int kPreNone = 0, kPreBias = 1, kPreAffine = 2;
 constexpr int kActNone = 0, kActRelu = 1, kActGeluPrecise = 2, kActGeluFast = 3;
 constexpr int kGroup = 4;   // chunks in flight per lane and tensor
 
+// One chunk (8 columns starting at column 8*c) of one row: ops in packed fp32x2, one 16-byte store,
+// and the chunk's contribution to the running (max, sum) of the row (log2 domain).
+template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
+__device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
+                                         float& run_m, float& run_s) {
+    float2 v[4];
+    v[0] = make_float2(bf16_lo(xq.x), bf16_hi(xq.x));
+    v[1] = make_float2(bf16_lo(xq.y), bf16_hi(xq.y));
+    v[2] = make_float2(bf16_lo(xq.z), bf16_hi(xq.z));
+    v[3] = make_float2(bf16_lo(xq.w), bf16_hi(xq.w));
+    if (PRE != kPreNone) {
+        const float4 a0 = *reinterpret_cast<const float4*>(svec + c * 8);
+        const float4 a1 = *reinterpret_cast<const float4*>(svec + c * 8 + 4);
+        const float2 a[4] = {make_float2(a0.x, a0.y), make_float2(a0.z, a0.w), make_float2(a1.x, a1.y), make_float2(a1.z, a1.w)};
+        if (PRE == kPreAffine) {
+            const float4 b0 = *reinterpret_cast<const float4*>(svec + N + c * 8);
+            const float4 b1 = *reinterpret_cast<const float4*>(svec + N + c * 8 + 4);
+            const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = __ffma2_rn(v[j], a[j], b[j]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = __fadd2_rn(v[j], a[j]);
+        }
+    }
+    float2 r[4];
+    if (RES) {
+        r[0] = make_float2(bf16_lo(rq.x), bf16_hi(rq.x));
+        r[1] = make_float2(bf16_lo(rq.y), bf16_hi(rq.y));
+        r[2] = make_float2(bf16_lo(rq.z), bf16_hi(rq.z));
+        r[3] = make_float2(bf16_lo(rq.w), bf16_hi(rq.w));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float2 t = v[j];
+        if (ACT == kActRelu) t = make_float2(t.x < 0.0f ? 0.0f : t.x, t.y < 0.0f ? 0.0f : t.y);
+        if (ACT == kActGeluPrecise) {
+            // z = sqrt(2/pi) (t + 0.044715 t^3); gelu = t / (1 + exp(-2 z)); w = -2 z log2(e)
+            constexpr float k0 = -2.0f * kLog2e * 0.7978845608028654f, k1 = k0 * 0.044715f;
+            const float2 t2 = __fmul2_rn(t, t);
+            const float2 w = __fmul2_rn(t, __ffma2_rn(t2, make_float2(k1, k1), make_float2(k0, k0)));
+            const float2 d = __fadd2_rn(make_float2(exp2_fast(w.x), exp2_fast(w.y)), make_float2(1.0f, 1.0f));
+            float2 inv;
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.x) : "f"(d.x));
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.y) : "f"(d.y));
+            t = RES ? __ffma2_rn(t, inv, r[j]) : __fmul2_rn(t, inv);
+        } else if (ACT == kActGeluFast) {
+            constexpr float k0 = 0.7978845608028654f, k1 = k0 * 0.044715f;
+            const float2 t2 = __fmul2_rn(t, t);
+            const float2 z = __fmul2_rn(t, __ffma2_rn(t2, make_float2(k1, k1), make_float2(k0, k0)));
+            const float2 hv = __fmul2_rn(t, make_float2(0.5f, 0.5f));
+            const float2 th = make_float2(tanh_fast(z.x), tanh_fast(z.y));
+            t = __ffma2_rn(hv, th, RES ? __fadd2_rn(hv, r[j]) : hv);
+        } else if (RES) {
+            t = __fadd2_rn(t, r[j]);
+        }
+        v[j] = t;
+    }
+    if (STORE) {
+        uint4 q;
+        q.x = pack_bf16x2(v[0].x, v[0].y); q.y = pack_bf16x2(v[1].x, v[1].y);
+        q.z = pack_bf16x2(v[2].x, v[2].y); q.w = pack_bf16x2(v[3].x, v[3].y);
+        st_stream(yr + c, q);
+    }
+    if (LSE) {
+        const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)),
+                               fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
+        const float nm = fmaxf(run_m, cm * kLog2e);
+        const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-nm, -nm);
+        float2 cs = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 e = __ffma2_rn(v[j], l2e, mnm);
+            cs = __fadd2_rn(cs, make_float2(exp2_fast(e.x), exp2_fast(e.y)));
+        }
+        run_s = fmaf(run_s, exp2_fast(run_m - nm), cs.x + cs.y);
+        run_m = nm;
+    }
+}
+
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
 __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams p) {
     extern __shared__ float svec[];   // PRE != none: vec0 as fp32 [N], then vec1 [N]
@@ -152,16 +232,19 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
         }
         __syncthreads();
     }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // Each warp walks whole rows, rows interleaved over all resident warps (measured: handing rows
+    // out through a global counter evens out the CTAs' finish times but not the kernel's duration,
+    // which is set by aggregate throughput).  Per row, a lane issues the loads of kGroup chunks of
+    // the input and of the residual tensor (8 x 16 bytes in flight), then does their arithmetic.
+    const int lane = threadIdx.x & 31;
     const int chunks = N >> 3;
+    const int warp = threadIdx.x >> 5;
     const long long row_step = (long long) gridDim.x * kWarps;
-
     for (long long row = (long long) blockIdx.x * kWarps + warp; row < p.M; row += row_step) {
         const uint4* xr = p.x + row * chunks;
         const uint4* rr = RES ? p.res + row * chunks : nullptr;
         uint4* yr = STORE ? p.y + row * chunks : nullptr;
         float run_m = -CUDART_INF_F, run_s = 0.0f;   // log2 domain: sum of 2^(y*log2e - run_m)
-
         for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
             uint4 xv[kGroup], rv[kGroup];
 #pragma unroll
@@ -175,69 +258,7 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
 #pragma unroll
             for (int g = 0; g < kGroup; ++g) {
                 const int c = c0 + 32 * g;
-                if (c >= chunks) break;
-                float v[8];
-                v[0] = bf16_lo(xv[g].x); v[1] = bf16_hi(xv[g].x); v[2] = bf16_lo(xv[g].y); v[3] = bf16_hi(xv[g].y);
-                v[4] = bf16_lo(xv[g].z); v[5] = bf16_hi(xv[g].z); v[6] = bf16_lo(xv[g].w); v[7] = bf16_hi(xv[g].w);
-                if (PRE != kPreNone) {
-                    const float4 a0 = *reinterpret_cast<const float4*>(svec + c * 8);
-                    const float4 a1 = *reinterpret_cast<const float4*>(svec + c * 8 + 4);
-                    const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-                    if (PRE == kPreAffine) {
-                        const float4 b0 = *reinterpret_cast<const float4*>(svec + N + c * 8);
-                        const float4 b1 = *reinterpret_cast<const float4*>(svec + N + c * 8 + 4);
-                        const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) v[j] = fmaf(v[j], a[j], b[j]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) v[j] += a[j];
-                    }
-                }
-                float r[8];
-                if (RES) {
-                    r[0] = bf16_lo(rv[g].x); r[1] = bf16_hi(rv[g].x); r[2] = bf16_lo(rv[g].y); r[3] = bf16_hi(rv[g].y);
-                    r[4] = bf16_lo(rv[g].z); r[5] = bf16_hi(rv[g].z); r[6] = bf16_lo(rv[g].w); r[7] = bf16_hi(rv[g].w);
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float t = v[j];
-                    if (ACT == kActRelu) t = t < 0.0f ? 0.0f : t;
-                    if (ACT == kActGeluPrecise || ACT == kActGeluFast) {
-                        // z = sqrt(2/pi) (t + 0.044715 t^3); gelu = t / (1 + exp(-2 z))
-                        const float t2 = t * t;
-                        if (ACT == kActGeluPrecise) {
-                            const float w = t * fmaf(t2, -2.0f * kLog2e * 0.7978845608028654f * 0.044715f,
-                                                     -2.0f * kLog2e * 0.7978845608028654f);
-                            const float d = 1.0f + exp2_fast(w);
-                            float inv;
-                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(d));
-                            t = RES ? fmaf(t, inv, r[j]) : t * inv;
-                        } else {
-                            const float z = t * fmaf(t2, 0.7978845608028654f * 0.044715f, 0.7978845608028654f);
-                            const float hv = 0.5f * t;
-                            t = fmaf(hv, tanh_fast(z), RES ? hv + r[j] : hv);
-                        }
-                    } else if (RES) {
-                        t += r[j];
-                    }
-                    v[j] = t;
-                }
-                if (STORE) {
-                    uint4 q;
-                    q.x = pack_bf16x2(v[0], v[1]); q.y = pack_bf16x2(v[2], v[3]);
-                    q.z = pack_bf16x2(v[4], v[5]); q.w = pack_bf16x2(v[6], v[7]);
-                    st_stream(yr + c, q);
-                }
-                if (LSE) {
-                    float cm = fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
-                    const float nm = fmaxf(run_m, cm * kLog2e);
-                    float cs = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) cs += exp2_fast(fmaf(v[j], kLog2e, -nm));
-                    run_s = fmaf(run_s, exp2_fast(run_m - nm), cs);
-                    run_m = nm;
-                }
+                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, run_m, run_s);
             }
         }
         if (LSE) {
@@ -262,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
 // Recognise [bias | affine]? -> [relu | gelu]? -> [add tensor]? and fill the fast-path parameters.
 static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, bool* res) {
     if (p.x_dt != FC_BF16 || (p.y && p.y_dt != FC_BF16)) return false;
-    if (p.N % 8 != 0 || p.N > 24576) return false;
+    if (p.N % 8 != 0 || p.N > 24576 || p.M >= 0x7fffffffLL) return false;
     if ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y)) & 15) return false;
     int i = 0;
     *pre = kPreNone; *act = kActNone; *res = false;
@@ -274,7 +295,8 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
         ++i;
     }
     if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_RELU || p.ops.op[i].kind == FC_OP_GELU_TANH)) {
-        *act = p.ops.op[i].kind == FC_OP_RELU ? kActRelu : kActGeluPrecise;
+        // tanh.approx (2^-11) is below bf16 resolution; an fp32 logsumexp of the result needs the exact form
+        *act = p.ops.op[i].kind == FC_OP_RELU ? kActRelu : (p.reduce == FC_RED_ROW_LOGSUMEXP ? kActGeluPrecise : kActGeluFast);
         ++i;
     }
     if (i < p.ops.n && p.ops.op[i].kind == FC_OP_ADD_TENSOR) {
@@ -323,6 +345,7 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
         FC_EW_CASE(kPreNone, kActNone) FC_EW_CASE(kPreNone, kActRelu) FC_EW_CASE(kPreNone, kActGeluPrecise)
         FC_EW_CASE(kPreBias, kActNone) FC_EW_CASE(kPreBias, kActRelu) FC_EW_CASE(kPreBias, kActGeluPrecise)
         FC_EW_CASE(kPreAffine, kActNone) FC_EW_CASE(kPreAffine, kActRelu) FC_EW_CASE(kPreAffine, kActGeluPrecise)
+        FC_EW_CASE(kPreNone, kActGeluFast) FC_EW_CASE(kPreBias, kActGeluFast) FC_EW_CASE(kPreAffine, kActGeluFast)
 #undef FC_EW_CASE
     }
     // precise GELU whenever an fp32 result (the logsumexp, or an fp32 main output) depends on it

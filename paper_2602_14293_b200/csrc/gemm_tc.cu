@@ -24,8 +24,6 @@
 // CTAs.  Two accumulator buffers in tensor memory let the epilogue of tile i overlap the main loop
 // of tile i+1.  Every wait is bounded: on expiry the CTA records FC_ERR_TIMEOUT in the status word,
 // stops storing and drains.
-#include <cstdio>
-
 #include "dev_common.cuh"
 #include "ptx.cuh"
 
@@ -218,10 +216,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef FC_DBG_CLOCK
-    const long long dbg_c0 = clock64();
-    const unsigned long long dbg_t0 = ptx::globaltimer();
-#endif
     const uint32_t cta_rank = ptx::cluster_ctarank();
     const bool leader = cta_rank == 0;
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
@@ -312,11 +306,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tc_fence_after();
                     const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
                     const uint64_t da = ptx::smem_desc_k128(sa), db = ptx::smem_desc_k128(sa + C::kABytes);
-#ifndef FC_DBG_SKIP_MMA
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
                         ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-#endif
                     ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);     // frees the stage in both CTAs
                 }
                 if (ok) ptx::tc_commit_pair(ptx::smem_u32(&ctrl->tfull[buf]), 3);   // accumulators ready in both CTAs
@@ -357,12 +349,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ptx::bar_sync(2, kEpiThreads);
             if (!*(volatile int*) &ctrl->epi_ok[buf]) break;
             ptx::tc_fence_after();
-#ifdef FC_DBG_SKIP_EPI
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
-            continue;
-#endif
             constexpr int kChunks = BN / 32;           // 16-column chunks per thread (half a tile row)
             const int col_half = half * (BN / 2);
             const uint32_t tacc = tmem_base + buf * BN + col_half + lane_addr;
@@ -383,20 +369,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
-#ifndef FC_DBG_NO_MATH
                             if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                             else apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-#endif
-#ifndef FC_DBG_NO_STORE
                             store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
-#else
-                            if (v[3] == 1.2345f) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
-#endif
                         }
                     }
-#ifdef FC_DBG_SLEEP
-                    __nanosleep(FC_DBG_SLEEP);
-#endif
                     ptx::tmem_wait_ld(rb);
                     if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
                     {
@@ -405,15 +382,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
-#ifndef FC_DBG_NO_MATH
                             if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
                             else apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
-#endif
-#ifndef FC_DBG_NO_STORE
                             store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
-#else
-                            if (v[3] == 1.2345f) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
-#endif
                         }
                     }
                 }
@@ -542,13 +513,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------------------------------------------------------------- teardown
     ptx::tc_fence_before();
     __syncthreads();
-#ifdef FC_DBG_CLOCK
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        const long long dc = clock64() - dbg_c0;
-        const unsigned long long dt = ptx::globaltimer() - dbg_t0;
-        printf("kernel: %lld cycles in %llu ns -> %.0f MHz\n", dc, dt, 1e3 * (double) dc / (double) dt);
-    }
-#endif
     if (*abort_flag) {
         // a wait expired: give copies and MMAs still in flight time to land before releasing memory
         const unsigned long long t0 = ptx::globaltimer();
