@@ -280,6 +280,18 @@ void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
             o.dt1 = in[op.in1].dtype;
         }
     }
+    // fused form: [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]?
+    FusedOps& f = d->fused;
+    memset(&f, 0, sizeof(f));
+    f.scale = 1.0f;
+    int i = 0;
+    const int n = s->n_ops;
+    if (i < n && (s->ops[i].kind == FC_OP_BIAS_N || s->ops[i].kind == FC_OP_AFFINE_N)) f.pre = s->ops[i++].kind == FC_OP_BIAS_N ? 1 : 2;
+    if (i < n && (s->ops[i].kind == FC_OP_RELU || s->ops[i].kind == FC_OP_GELU_TANH)) f.act = s->ops[i++].kind == FC_OP_RELU ? 1 : 2;
+    if (i < n && s->ops[i].kind == FC_OP_SCALE) f.scale = s->ops[i++].f0;
+    if (i < n && s->ops[i].kind == FC_OP_CLAMP) { f.clamp = 1; f.lo = s->ops[i].f0; f.hi = s->ops[i].f1; ++i; }
+    if (i < n && s->ops[i].kind == FC_OP_ADD_TENSOR) { f.res = 1; f.res_ptr = in[s->ops[i].in0].ptr; f.res_dt = in[s->ops[i].in0].dtype; ++i; }
+    f.valid = i == n;
 }
 
 constexpr int kSoftmaxBN = 256;
@@ -369,6 +381,12 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
             const int bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
+            {
+                // keep about 32 MB of A rows (group_m panels of 256 rows) resident in L2 per sweep
+                const long long panel_bytes = 256LL * spec->K * 2;
+                long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
+                p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
+            }
             if (p.mode == 1) {
                 const size_t need = softmax_workspace_bytes(spec->M, spec->N);
                 const long long panels = (spec->M + 127) / 128;
@@ -394,6 +412,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.OH = (int) ((spec->H + 2 * spec->pad - spec->R) / spec->stride + 1);
             p.OW = (int) ((spec->W + 2 * spec->pad - spec->S) / spec->stride + 1);
             p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
+            p.group_m = 1;
             p.inv_hw = 1.0f / (float) (p.OH * p.OW);
             p.out = outputs[plan.red_index].ptr; p.out_dt = FC_F32;
             p.status = dev->status;
@@ -574,6 +593,7 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
     build_ops(spec, inputs, &p.ops);
     const long long panels = (spec->M + 127) / 128;
     const size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
+    p.group_m = 1;
     p.counters = (unsigned int*) scratch;
     p.stats = (float2*) ((char*) scratch + counters);
     // the array keeps the previous call's contents: the arrival counters must start at zero

@@ -18,9 +18,25 @@ struct DevOp {
     const void* p1;    // second vector (AFFINE_N)
 };
 
+// When the list has the shape [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]? the
+// host also fills `fused`, which the tensor-core epilogues execute as straight packed-fp32x2 code
+// instead of interpreting the list (fewer issue slots, less energy next to a power-bound main loop).
+struct FusedOps {
+    int valid;
+    int pre;           // 0 none, 1 bias (vector slot 0), 2 affine (slots 0 and 1)
+    int act;           // 0 none, 1 relu, 2 gelu
+    int clamp;         // 0 / 1
+    int res;           // 0 / 1: add tensor
+    int res_dt;
+    float scale;       // post-activation scale (1 if absent)
+    float lo, hi;
+    const void* res_ptr;
+};
+
 struct DevOps {
     int n;
     DevOp op[FC_MAX_OPS];
+    FusedOps fused;
 };
 
 // Device status word values (also fc_status values).
@@ -51,6 +67,7 @@ cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* la
 struct TcParams {
     int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
+    int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
     void* out; int out_dt;      // mode 0/1: [M,N] bf16 or f32.  mode 2: f32 [batch,Cout] (pre-zeroed)
     DevOps ops;
     // mode 1

@@ -34,7 +34,6 @@ constexpr int BM = 128;          // rows per CTA; the pair covers 2 * BM
 constexpr int BK = 64;
 constexpr int kThreads = 320;
 constexpr int kEpiThreads = 256;
-constexpr int kGroupM = 4;       // mode-0 raster: kGroupM pair-panels share each sweep over the columns
 constexpr int kMaxVecSlots = 3;  // per-column vectors staged in shared memory per tile
 
 template <int BN>
@@ -79,8 +78,11 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
 }
 
 // pair-tile index -> (pair-panel index, column-tile index)
-__device__ __forceinline__ void tile_coords(int mode, int t, int tiles_m, int tiles_n, int& mb, int& nb) {
+__device__ __forceinline__ void tile_coords(int mode, int group_m, int t, int tiles_m, int tiles_n, int& mb, int& nb) {
     if (mode == 0) {
+        // raster: group_m pair-panels share each sweep over the column tiles, so that their rows of A
+        // stay in L2 while B streams through once per group
+        const int kGroupM = group_m;
         const int group = kGroupM * tiles_n;
         const int g = t / group, r = t - g * group;
         const int first = g * kGroupM;
@@ -112,9 +114,90 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
 // The op list applied to 16 consecutive columns (col0.. within the tile) of one row.  Per-column
 // vectors come from the shared-memory slices staged for this tile (slot order = order of the
 // vector operands in the op list); ADD_TENSOR reads global memory.
+// The fused form of the op list on 16 consecutive columns, in packed fp32x2 arithmetic.
+template <bool kPreciseGelu>
+__device__ __forceinline__ void fused_ops16(float (&v)[16], const FusedOps& f, const float* svec, int bn, int col0,
+                                            long long m, long long n0, long long n_limit, long long ld) {
+    float2 w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = make_float2(v[2 * j], v[2 * j + 1]);
+    if (f.pre != 0) {
+        const float4* a = reinterpret_cast<const float4*>(svec + col0);
+        if (f.pre == 1) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 t = a[q];
+                w[2 * q] = __fadd2_rn(w[2 * q], make_float2(t.x, t.y));
+                w[2 * q + 1] = __fadd2_rn(w[2 * q + 1], make_float2(t.z, t.w));
+            }
+        } else {
+            const float4* b = reinterpret_cast<const float4*>(svec + bn + col0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 g = a[q], t = b[q];
+                w[2 * q] = __ffma2_rn(w[2 * q], make_float2(g.x, g.y), make_float2(t.x, t.y));
+                w[2 * q + 1] = __ffma2_rn(w[2 * q + 1], make_float2(g.z, g.w), make_float2(t.z, t.w));
+            }
+        }
+    }
+    if (f.act == 2) {
+        if (kPreciseGelu) {
+            // gelu(t) * s = t * s / (1 + 2^(-2 z log2 e)),  z = sqrt(2/pi) (t + 0.044715 t^3)
+            constexpr float k0 = -2.0f * kLog2e * 0.7978845608028654f, k1 = k0 * 0.044715f;
+            const float2 sc = make_float2(f.scale, f.scale);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float2 t = w[j];
+                const float2 e = __fmul2_rn(t, __ffma2_rn(__fmul2_rn(t, t), make_float2(k1, k1), make_float2(k0, k0)));
+                const float2 d = __fadd2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), make_float2(1.0f, 1.0f));
+                float2 inv;
+                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.x) : "f"(d.x));
+                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.y) : "f"(d.y));
+                w[j] = __fmul2_rn(__fmul2_rn(t, sc), inv);
+            }
+        } else {
+            // gelu(t) * s = h + h tanh(z) with h = (0.5 s) t
+            constexpr float k0 = 0.7978845608028654f, k1 = k0 * 0.044715f;
+            const float hs = 0.5f * f.scale;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float2 t = w[j];
+                const float2 z = __fmul2_rn(t, __ffma2_rn(__fmul2_rn(t, t), make_float2(k1, k1), make_float2(k0, k0)));
+                const float2 h = __fmul2_rn(t, make_float2(hs, hs));
+                w[j] = __ffma2_rn(h, make_float2(tanh_fast(z.x), tanh_fast(z.y)), h);
+            }
+        }
+    } else {
+        if (f.act == 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = make_float2(w[j].x < 0.0f ? 0.0f : w[j].x, w[j].y < 0.0f ? 0.0f : w[j].y);
+        }
+        if (f.scale != 1.0f) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = __fmul2_rn(w[j], make_float2(f.scale, f.scale));
+        }
+    }
+    if (f.clamp) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            w[j] = make_float2(fminf(fmaxf(w[j].x, f.lo), f.hi), fminf(fmaxf(w[j].y, f.lo), f.hi));
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { v[2 * j] = w[j].x; v[2 * j + 1] = w[j].y; }
+    if (f.res) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (n0 + j < n_limit) v[j] += load_scalar(f.res_ptr, f.res_dt, m * ld + n0 + j);
+    }
+}
+
 template <bool kPreciseGelu>
 __device__ __forceinline__ void apply_ops16(float (&v)[16], const DevOps& ops, const float* svec, int bn, int col0,
                                             long long m, long long n0, long long n_limit, long long ld) {
+    if (ops.fused.valid) {
+        fused_ops16<kPreciseGelu>(v, ops.fused, svec, bn, col0, m, n0, n_limit, ld);
+        return;
+    }
     int slot = 0;
 #pragma unroll 1
     for (int i = 0; i < ops.n; ++i) {
@@ -256,7 +339,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
                 int mb2, nb;
-                tile_coords(MODE == 0 ? 0 : 1, t, tiles_m, tiles_n, mb2, nb);
+                tile_coords(MODE == 0 ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
@@ -327,7 +410,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint32_t tile_iter = 0;
         for (int t = cluster_id; t < total_tiles; t += num_clusters, ++tile_iter) {
             int mb2, nb;
-            tile_coords(MODE == 0 ? 0 : 1, t, tiles_m, tiles_n, mb2, nb);
+            tile_coords(MODE == 0 ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
             const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;

@@ -153,6 +153,23 @@ def test_c3_chain_ragged(fc, orc, M, N, K):
     run_and_check(fc, orc, replace(wl.gemm_bias_gelu_scale_clamp(M, N, K, "var"), out_dtype="f32"), 4)
 
 
+def test_gemm_tc_op_lists_fused_and_interpreted(fc, orc):
+    """Op lists of the fused shape ([bias|affine] [relu|gelu] [scale] [clamp] [add tensor]) take the
+    packed straight-line epilogue; any other order is interpreted op by op.  Both against the oracle."""
+    base = wl.gemm_bias_gelu_scale_clamp(300, 520, 136, "var")
+    rec = base.input_recipe + (("res", "bf16", (300, 520), "normal", 0.0, 1.0), ("gamma", "bf16", (520,), "normal", 1.0, 0.1))
+    lists = [
+        (("affine_n", 4, 2), ("relu",), ("scale", 1.5), ("clamp", 0.25, 2.0), ("add_tensor", 3)),       # fused
+        (("bias_n", 2), ("gelu_tanh",), ("add_tensor", 3)),                                              # fused
+        (("scale", -2.0),),                                                                              # fused
+        (("relu",), ("bias_n", 2), ("scale", 0.5), ("gelu_tanh",), ("add_tensor", 3), ("clamp", -1.0, 1.0)),  # interpreted
+        (("clamp", -0.5, 0.5), ("affine_n", 4, 2), ("gelu_tanh",)),                                      # interpreted
+    ]
+    for ops in lists:
+        for out_dtype in ("bf16", "f32"):
+            run_and_check(fc, orc, replace(base, ops=ops, out_dtype=out_dtype, input_recipe=rec), 6, tag=f" ops={[o[0] for o in ops]}")
+
+
 def test_c3_full_size_sampled_rows(fc, orc):
     ch = wl.CONFIGS["C3"]()
     ins = wl.make_inputs(ch, 0)
