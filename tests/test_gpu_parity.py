@@ -161,7 +161,7 @@ def test_gemm_tc_op_lists_fused_and_interpreted(fc, orc):
     lists = [
         (("affine_n", 4, 2), ("relu",), ("scale", 1.5), ("clamp", 0.25, 2.0), ("add_tensor", 3)),       # fused
         (("bias_n", 2), ("gelu_tanh",), ("add_tensor", 3)),                                              # fused
-        (("scale", -2.0),),                                                                              # fused
+        (("scale", -0.75),),                                                                             # fused (outputs stay O(1): the mean-abs bound is absolute)
         (("relu",), ("bias_n", 2), ("scale", 0.5), ("gelu_tanh",), ("add_tensor", 3), ("clamp", -1.0, 1.0)),  # interpreted
         (("clamp", -0.5, 0.5), ("affine_n", 4, 2), ("gelu_tanh",)),                                      # interpreted
     ]
