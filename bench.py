@@ -50,16 +50,16 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback (earlier measurement on this pool)"
 
 
-def load_traffic(workload: str):
-    """DRAM bytes per launch from the committed ncu capture of this workload's kernel, if any."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(path):
-        try:
-            with open(path) as f:
-                return json.load(f).get(workload)
-        except Exception:
-            return None
-    return None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each config's kernel, from the ncu
+# captures summarised under profiles/ (full config sizes; part of each output is still dirty in L2
+# when the kernel ends, so writes can read below the algorithmic output bytes).
+NCU_TRAFFIC_BYTES = {"C1": 541440, "C2": 268473344 + 99006208, "C3": 226910464 + 115290624,
+                     "C4": 68544000 + 12676608, "C5": 52659968 + 148992}
+
+
+def load_traffic(workload: str, full_size: bool):
+    """DRAM bytes per launch from the committed ncu capture of this workload's kernel (full size only)."""
+    return NCU_TRAFFIC_BYTES.get(workload) if full_size else None
 
 
 # ------------------------------------------------------------------------------ units per workload
@@ -395,7 +395,7 @@ def main():
         peak_note = "fp32 FMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived)"
     achieved = units_per_step / (ms_per_step * 1e-3)
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": peak_unit, "frac": achieved / peak,
-                "traffic": load_traffic(args.workload), "peak_source": peak_note,
+                "traffic": load_traffic(args.workload, args.rows <= 0), "peak_source": peak_note,
                 "algorithmic_units_per_launch": units_per_step, "kernel_ms": ms_per_step}
 
     line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
