@@ -472,29 +472,60 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             } else if constexpr (MODE == 1) {
-                // pass 1: (max, sum) of this tile's slice of the row, online over 16-column chunks
-                float mx = -CUDART_INF_F, sm = 0.0f;
+                // sweep A: maximum of this thread's half row of the tile (ops applied, written back in place
+                // when the list is not empty, so that the later sweeps read finished logits)
+                const bool has_ops = p.ops.n > 0;
+                float mx = -CUDART_INF_F;
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     uint32_t r[16];
                     ptx::tmem_ld_32x16_async(tacc + c * 16, r);
                     ptx::tmem_wait_ld(r);
                     const int n0 = n_half + c * 16;
-                    if (m < p.M && n0 < p.N) {
+                    if (has_ops) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                        apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                        float cm = -CUDART_INF_F;
+                        if (m < p.M && n0 < p.N) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
-                        const float nm = fmaxf(mx, cm);
-                        float cs = 0.0f;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast((v[j] - nm) * kLog2e) : 0.0f;
-                        sm = sm * exp2_fast((mx - nm) * kLog2e) + cs;
-                        mx = nm;
+                        for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(v[j]);
+                        ptx::tmem_st_32x16(tacc + c * 16, r);
                     }
+                    if (m < p.M && n0 < p.N) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) mx = n0 + j < p.N ? fmaxf(mx, __uint_as_float(r[j])) : mx;
+                    }
+                }
+                if (has_ops) ptx::tmem_wait_st();
+                // sweep B: e = 2^((v - max) log2 e), summed, and written back over the logits: the last sweep
+                // only rescales, so every element costs one exponential
+                float sm = 0.0f;
+                {
+                    const float2 l2e = make_float2(kLog2e, kLog2e);
+                    const float2 moff = make_float2(-mx * kLog2e, -mx * kLog2e);
+                    float2 acc2 = make_float2(0.0f, 0.0f);
+#pragma unroll 1
+                    for (int c = 0; c < kChunks; ++c) {
+                        uint32_t r[16];
+                        ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+                        ptx::tmem_wait_ld(r);
+                        const int n0 = n_half + c * 16;
+                        if (m < p.M && n0 < p.N) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float2 t = __ffma2_rn(make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1])), l2e, moff);
+                                float2 e = make_float2(exp2_fast(t.x), exp2_fast(t.y));
+                                if (n0 + 2 * j >= p.N) e.x = 0.0f;
+                                if (n0 + 2 * j + 1 >= p.N) e.y = 0.0f;
+                                acc2 = __fadd2_rn(acc2, e);
+                                r[2 * j] = __float_as_uint(e.x);
+                                r[2 * j + 1] = __float_as_uint(e.y);
+                            }
+                        }
+                        ptx::tmem_st_32x16(tacc + c * 16, r);
+                    }
+                    ptx::tmem_wait_st();
+                    sm = acc2.x + acc2.y;
                 }
                 // the two column halves of a row meet in shared memory; the lower half publishes the tile's pair
                 if (half == 1) xchg[row] = make_float2(mx, sm);
@@ -535,8 +566,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     row_m = a.m;
                     row_s = a.s;
                 }
-                const float inv = 1.0f / row_s, off = -row_m * kLog2e;
-                // pass 2: normalise straight from tensor memory and store once
+                // last sweep: p = e * 2^((max_half - max_row) log2 e) / sum_row, one factor per thread
+                const float fac = m < p.M && store ? exp2_fast((mx - row_m) * kLog2e) / row_s : 0.0f;
+                const float2 fac2 = make_float2(fac, fac);
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     uint32_t r[16];
@@ -546,10 +578,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (m < p.M && n0 < p.N && store) {
                         float v[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                        apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = exp2_fast(fmaf(v[j], kLog2e, off)) * inv;
+                        for (int j = 0; j < 8; ++j) {
+                            const float2 t = __fmul2_rn(make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1])), fac2);
+                            v[2 * j] = t.x;
+                            v[2 * j + 1] = t.y;
+                        }
                         store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                     }
                 }
@@ -639,6 +672,14 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap& tmA, const CUtensor
     int clusters = dev >= 0 && dev < 64 ? max_clusters[dev] : num_sms / 2;
     if (clusters > num_sms / 2) clusters = num_sms / 2;
     if (clusters > tiles) clusters = tiles;
+    if (MODE == 1) {
+        // Row softmax: a tile's epilogue waits for the other column tiles of its row panel.  With a
+        // pair count that is a multiple of the column-tile count every panel lives inside one round;
+        // otherwise panels straddle rounds and their first tiles hold an accumulator buffer for a
+        // whole extra round.
+        const int tiles_n = (p.N + BN - 1) / BN;
+        if (clusters > tiles_n) clusters = clusters / tiles_n * tiles_n;
+    }
     cfg.gridDim = dim3(2 * clusters);
     return cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
 }
