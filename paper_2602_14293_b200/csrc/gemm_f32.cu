@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Params p) {
         if (m >= p.M) continue;
         float v[2] = {acc[i][0], acc[i][1]};
         const int n = n0 + tx * 2;
-        apply_ops<2, true>(v, p.ops, m, n, p.N, p.N);
+        apply_ops<2, false>(v, p.ops, m, n, p.N, p.N);
         if (n < p.N) p.C[(long long) m * p.N + n] = v[0];
         if (n + 1 < p.N) p.C[(long long) m * p.N + n + 1] = v[1];
     }

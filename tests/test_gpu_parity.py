@@ -79,6 +79,18 @@ def test_elementwise_f32_and_other_op_lists(fc, orc):
     run_and_check(fc, orc, replace(base, ops=()), 2)
 
 
+def test_gelu_accuracy_dense_grid_fp32(fc, orc):
+    """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
+    inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
+    within 2e-5 of the fp64 value, five times inside the fp32 output tolerance at |ref| = 0."""
+    n = 1 << 20
+    x = np.linspace(-14.0, 14.0, n, dtype=np.float32).reshape(256, n // 256)
+    ch = replace(wl.affine_gelu_residual_lse(256, n // 256), ops=(("gelu_tanh",),), reduce="none", in_dtype="f32", out_dtype="f32",
+                 input_recipe=(("x", "f32", x.shape, "normal", 0.0, 1.0),))
+    outs, ref, _ = run_and_check(fc, orc, ch, ins=[x])
+    assert float(np.abs(util.to_f64(outs[0]) - ref["main"]).max()) <= 2e-5
+
+
 def test_lse_shift_overflow_safety(fc, orc):
     ch = replace(wl.affine_gelu_residual_lse(4, 512), ops=(), in_dtype="f32", out_dtype="f32",
                  input_recipe=(("x", "f32", (4, 512), "normal", 0.0, 1.0),))
@@ -88,6 +100,19 @@ def test_lse_shift_overflow_safety(fc, orc):
     x[3, :] = -3.0
     x[3, 17] = 60.0
     run_and_check(fc, orc, ch, ins=[x])
+
+
+def test_lse_row_dominated_by_one_gelu_value(fc, orc):
+    """Adversarial for an approximate activation: one moderate GELU value dominates the row (every
+    other residual is -30), so the logsumexp equals that value and inherits its full error."""
+    ch = replace(wl.affine_gelu_residual_lse(64, 512), store_main=False)   # y itself is ~ -30: only the fp32 reduction is judged
+    x, g, b, r = wl.make_inputs(ch, 9)
+    rf = np.full((64, 512), -30.0, np.float32)
+    cols = (np.arange(64) * 7) % 512
+    rf[np.arange(64), cols] = 0.0
+    xf = rng.bf16_bits_to_f32(x).copy()
+    xf[np.arange(64), cols] = np.linspace(-3.0, 3.0, 64, dtype=np.float32)
+    run_and_check(fc, orc, ch, ins=[rng.store(xf, "bf16"), g, b, rng.store(rf, "bf16")])
 
 
 def test_c2_full_size_sampled_rows(fc, orc):
