@@ -252,7 +252,8 @@ def reference_arm(args):
     ch = wl.CONFIGS[args.workload]()
     ins = wl.make_inputs(ch, 0)
     metric, unit, _, _ = units(ch)
-    sub, sub_ins, desc = oracle_sample(ch, ins, target_s=5.0)
+    # each step is a bounded sample of the workload, sized so that the whole run ends within a few minutes
+    sub, sub_ins, desc = oracle_sample(ch, ins, target_s=max(0.05, min(5.0, 120.0 / max(1, args.steps + 1))))
     for _ in range(min(args.warmup, 1)):
         oracle.run_chain(sub, sub_ins)
     t0 = time.perf_counter()
@@ -274,8 +275,8 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="C2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
