@@ -150,6 +150,8 @@ def eager_fn(ch, t):
         return f
     if name == "gemm_bf16_bias_gelu_scale_clamp":
         return lambda: torch.clamp(F.gelu(F.linear(t[0], t[1], t[2]), approximate="tanh") * 0.5, -1.0, 1.0)
+    if name == "gemm_bf16_bias_scale_lse":
+        return lambda: torch.logsumexp((F.linear(t[0], t[1], t[2]) * 0.5).float(), dim=1)
     if name == "gemm_bf16_row_softmax":
         return lambda: torch.softmax(t[0] @ t[1].t(), dim=1)
     if name == "conv_bf16_bias_relu_avgpool":
@@ -249,7 +251,7 @@ def reference_arm(args):
         return 0
     import oracle
     oracle.build()
-    ch = wl.CONFIGS[args.workload]()
+    ch = wl.ALL[args.workload]()
     ins = wl.make_inputs(ch, 0)
     metric, unit, _, _ = units(ch)
     # each step is a bounded sample of the workload, sized so that the whole run ends within a few minutes
@@ -277,7 +279,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="C2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default="C2", choices=sorted(wl.ALL))
     ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-eager", action="store_true")
@@ -299,9 +301,9 @@ def main():
     barrier, max_over_ranks = rk.barrier, rk.max_over_ranks
 
     peaks, peaks_src = load_peaks()
-    ch = wl.CONFIGS[args.workload]()
+    ch = wl.ALL[args.workload]()
     if args.rows > 0:
-        ch = wl.CONFIGS[args.workload](batch=args.rows) if ch.producer == "conv2d_nhwc" else wl.CONFIGS[args.workload](M=args.rows)
+        ch = wl.ALL[args.workload](batch=args.rows) if ch.producer == "conv2d_nhwc" else wl.ALL[args.workload](M=args.rows)
     metric, unit, units_per_step, bound = units(ch)
     ins = wl.make_inputs(ch, seed=rk.batch_seed(0))   # every rank draws its own batch
     dev_in = [fc.to_device(a) for a in ins]

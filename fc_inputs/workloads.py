@@ -103,6 +103,17 @@ def gemm_softmax(M=4096, N=4096, K=4096, variant="std") -> Chain:
                                ("B", "bf16", (N, K), "normal", 0.0, s)))
 
 
+def gemm_bias_scale_lse(M=1024, N=4096, K=1024, variant="var", store_main=False) -> Chain:
+    """A linear layer followed by a row reduction to one value per row (the shape of the paper's
+    appendix example: linear -> reduction -> logsumexp), here: logsumexp_n((A B^T + bias) * 0.5)."""
+    s = K ** -0.5 if variant == "std" else K ** -0.25
+    return Chain("gemm_bf16_bias_scale_lse", "gemm_nt", "bf16", "bf16", M=M, N=N, K=K,
+                 ops=(("bias_n", 2), ("scale", 0.5)), reduce="row_logsumexp", store_main=store_main,
+                 input_recipe=(("A", "bf16", (M, K), "normal", 0.0, s),
+                               ("B", "bf16", (N, K), "normal", 0.0, s),
+                               ("bias", "bf16", (N,), "uniform", -0.1, 0.1)))
+
+
 def conv_bias_relu_avgpool(batch=32, H=56, W=56, Cin=256, Cout=256, R=3, S=3, stride=1, pad=1) -> Chain:
     s = (R * S * Cin) ** -0.5
     return Chain("conv_bf16_bias_relu_avgpool", "conv2d_nhwc", "bf16", "f32",
@@ -121,6 +132,12 @@ CONFIGS = {
     "C4": gemm_softmax,
     "C5": conv_bias_relu_avgpool,
 }
+
+#: Further measured workloads beyond the five configurations (rows marked "next" in the scope table).
+EXTRA = {
+    "F1": lambda **kw: gemm_bias_scale_lse(**{"M": 4096, "N": 8192, "K": 4096, **kw}),
+}
+ALL = {**CONFIGS, **EXTRA}
 
 
 def make_inputs(chain: Chain, seed: int = 0) -> List[np.ndarray]:

@@ -45,7 +45,7 @@
  * remaining stores and exits; fc_get_async_status reports it.
  *
  * Threading.  fc_run may be called from several host threads.  The workspace set by
- * fc_set_workspace is shared by all calls: launches that use it (ROW_SOFTMAX on a GEMM) must not
+ * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM) must not
  * overlap on the device.
  */
 #ifndef FC_H_
@@ -147,8 +147,8 @@ fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, in
                           const fc_tensor* outputs, int n_outputs, size_t* bytes);
 
 /*
- * Scratch memory.  Only GEMM_NT + ROW_SOFTMAX needs any (per-tile row maxima and sums plus
- * per-panel arrival counters for the cross-tile online max/sum merge).  fc_workspace_size reports
+ * Scratch memory.  Only GEMM_NT + ROW_SOFTMAX / ROW_LOGSUMEXP needs any (per-tile row maxima and sums
+ * plus per-panel arrival counters for the cross-tile online max/sum merge).  fc_workspace_size reports
  * the bytes a spec needs (0 for the other chains); fc_set_workspace registers a caller-owned DEVICE
  * buffer (256-byte aligned) for the current device, used by later fc_run calls until replaced.
  */

@@ -84,7 +84,7 @@ size_t dt_size(int dt) { return dt == FC_BF16 ? 2 : 4; }
 
 // ------------------------------------------------------------------------------- validation
 struct Plan {
-    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_CONV } kind;
+    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV } kind;
     long long out_rows, out_cols;  // main output viewed as [rows][cols]
     int n_prod_inputs;
     int n_outputs;
@@ -160,8 +160,10 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
                 plan->kind = Plan::TC_PLAIN;
             } else if (s->reduce == FC_RED_ROW_SOFTMAX) {
                 plan->kind = Plan::TC_SOFTMAX;
+            } else if (s->reduce == FC_RED_ROW_LOGSUMEXP) {
+                plan->kind = Plan::TC_LSE;
             } else {
-                return fail(FC_ERR_UNSUPPORTED, "bf16 GEMM supports reduce NONE or ROW_SOFTMAX");
+                return fail(FC_ERR_UNSUPPORTED, "bf16 GEMM supports reduce NONE, ROW_SOFTMAX or ROW_LOGSUMEXP");
             }
             break;
         default:
@@ -172,7 +174,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             plan->kind = Plan::TC_CONV;
             break;
     }
-    if (plan->kind == Plan::TC_PLAIN || plan->kind == Plan::TC_SOFTMAX || plan->kind == Plan::TC_CONV) {
+    if (plan->kind == Plan::TC_PLAIN || plan->kind == Plan::TC_SOFTMAX || plan->kind == Plan::TC_LSE || plan->kind == Plan::TC_CONV) {
         int vecs = 0;
         for (int i = 0; i < s->n_ops; ++i) vecs += s->ops[i].kind == FC_OP_BIAS_N ? 1 : (s->ops[i].kind == FC_OP_AFFINE_N ? 2 : 0);
         if (vecs > 3) return fail(FC_ERR_UNSUPPORTED, "tensor-core chains support at most 3 per-column vector operands");
@@ -372,12 +374,14 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             break;
         }
         case Plan::TC_PLAIN:
+        case Plan::TC_LSE:
         case Plan::TC_SOFTMAX: {
             TcParams p;
             memset(&p, 0, sizeof(p));
-            p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : 0;
+            p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
             p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
-            p.out = outputs[plan.main_index].ptr; p.out_dt = spec->out_dtype;
+            p.out = plan.main_index >= 0 ? outputs[plan.main_index].ptr : nullptr; p.out_dt = spec->out_dtype;
+            p.red = plan.red_index >= 0 ? (float*) outputs[plan.red_index].ptr : nullptr;
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
             const int bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
@@ -387,11 +391,11 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
                 p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
             }
-            if (p.mode == 1) {
+            if (p.mode == 1 || p.mode == 3) {
                 const size_t need = softmax_workspace_bytes(spec->M, spec->N);
                 const long long panels = (spec->M + 127) / 128;
                 if (!dev->workspace || dev->workspace_bytes < need)
-                    return fail(FC_ERR_WORKSPACE, "row softmax needs a %zu-byte workspace (fc_set_workspace); have %zu", need, dev->workspace_bytes);
+                    return fail(FC_ERR_WORKSPACE, "this row reduction needs a %zu-byte workspace (fc_set_workspace); have %zu", need, dev->workspace_bytes);
                 size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
                 p.counters = (unsigned int*) dev->workspace;
                 p.stats = (float2*) ((char*) dev->workspace + counters);
@@ -494,7 +498,7 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     fc_status st;
     if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
     if ((st = validate_spec(spec, &plan))) return st;
-    *bytes = plan.kind == Plan::TC_SOFTMAX ? softmax_workspace_bytes(spec->M, spec->N) : 0;
+    *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N) : 0;
     return FC_OK;
 }
 

@@ -65,10 +65,11 @@ cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* la
 
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
-    int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool
+    int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row logsumexp
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
     int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
-    void* out; int out_dt;      // mode 0/1: [M,N] bf16 or f32.  mode 2: f32 [batch,Cout] (pre-zeroed)
+    void* out; int out_dt;      // mode 0/1/3: [M,N] bf16 or f32 (mode 3: may be null).  mode 2: f32 [batch,Cout] (pre-zeroed)
+    float* red;                 // mode 3: row logsumexp [M]
     DevOps ops;
     // mode 1
     float2* stats;              // [M][tiles_n] (max, sum) per tile

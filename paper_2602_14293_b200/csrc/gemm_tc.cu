@@ -5,6 +5,8 @@
 //   mode 1  row softmax over N fused across tiles: every tile publishes per-row (max, sum) of its
 //           column slice, waits (bounded) until the row panel's tiles have all published, merges
 //           the pairs and writes normalised probabilities straight from tensor memory
+//   mode 3  row logsumexp over N: as mode 0 (the main output is optional) plus per-tile (max, sum) pairs;
+//           the tile that publishes last for a row panel merges them, so no tile waits
 //   mode 2  implicit-GEMM convolution: the A operand is gathered by im2col-mode TMA from the NHWC
 //           image (zero fill outside the image), B is the [Cout][R*S*Cin] weight matrix; the
 //           epilogue applies ops (bias, ReLU) and sums each channel over the tile's pixels, adding
@@ -56,6 +58,7 @@ struct Ctrl {
     uint32_t tmem_base;
     int abort;
     int epi_ok[2];  // outcome of the epilogue's accumulator wait, one slot per accumulator buffer
+    int last;       // mode 3: this tile was the last of its row panel to publish
 };
 static_assert(sizeof(Ctrl) <= 256, "control block");
 
@@ -339,7 +342,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
                 int mb2, nb;
-                tile_coords(MODE == 0 ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
+                tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
@@ -410,7 +413,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint32_t tile_iter = 0;
         for (int t = cluster_id; t < total_tiles; t += num_clusters, ++tile_iter) {
             int mb2, nb;
-            tile_coords(MODE == 0 ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
+            tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
             const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;
@@ -470,6 +473,62 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                         }
                     }
+                }
+            } else if constexpr (MODE == 3) {
+                // ops, optional store, and a running (max, sum) of the row slice in the log2 domain; the
+                // tile that publishes last for its row panel merges all slices into the logsumexp, so
+                // nobody waits for anybody
+                float run_m = -CUDART_INF_F, run_s = 0.0f;
+#pragma unroll 1
+                for (int c = 0; c < kChunks; ++c) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+                    ptx::tmem_wait_ld(r);
+                    const int n0 = n_half + c * 16;
+                    if (m < p.M && n0 < p.N) {
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                        apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                        if (p.out) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                        float cm = -CUDART_INF_F;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
+                        const float nm = fmaxf(run_m, cm * kLog2e);
+                        float cs = 0.0f;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast(fmaf(v[j], kLog2e, -nm)) : 0.0f;
+                        run_s = fmaf(run_s, exp2_fast(run_m - nm), cs);
+                        run_m = nm;
+                    }
+                }
+                if (half == 1) xchg[row] = make_float2(run_m, run_s);
+                ptx::bar_sync(1, kEpiThreads);
+                if (half == 0 && m < p.M) {
+                    const float2 o = xchg[row];
+                    const float nm = fmaxf(run_m, o.x);
+                    const float sa = run_m == -CUDART_INF_F ? 0.0f : run_s * exp2_fast(run_m - nm);
+                    const float sb = o.x == -CUDART_INF_F ? 0.0f : o.y * exp2_fast(o.x - nm);
+                    __stcg(&p.stats[m * tiles_n + nb], make_float2(nm, sa + sb));
+                }
+                __threadfence();
+                ptx::bar_sync(1, kEpiThreads);
+                if (et == 0) {
+                    ctrl->last = ptx::atom_acq_rel_gpu_add(&p.counters[mb], 1u) == (unsigned) tiles_n - 1u;
+                    __threadfence();
+                }
+                ptx::bar_sync(1, kEpiThreads);
+                if (*(volatile int*) &ctrl->last && half == 0 && m < p.M) {
+                    float am = -CUDART_INF_F, as = 0.0f;
+                    for (int j = 0; j < tiles_n; ++j) {
+                        const float2 st = __ldcg(&p.stats[m * tiles_n + j]);
+                        const float nm = fmaxf(am, st.x);
+                        const float sa = am == -CUDART_INF_F ? 0.0f : as * exp2_fast(am - nm);
+                        const float sb = st.x == -CUDART_INF_F ? 0.0f : st.y * exp2_fast(st.x - nm);
+                        as = sa + sb;
+                        am = nm;
+                    }
+                    p.red[m] = (am + log2f(as)) * kLn2;
                 }
             } else if constexpr (MODE == 1) {
                 // sweep A: maximum of this thread's half row of the tile (ops applied, written back in place
@@ -689,6 +748,7 @@ cudaError_t launch_bn(const TcParams& p, const CUtensorMap& tmA, const CUtensorM
     switch (p.mode) {
         case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream);
         case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream);
+        case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream);
         default: return launch_one<BN, 2>(p, tmA, tmB, num_sms, stream);
     }
 }

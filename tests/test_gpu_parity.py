@@ -250,6 +250,26 @@ def test_c4_full_size_sampled_rows(fc, orc):
         _check_softmax_rows(outs[0])
 
 
+# ------------------------------------------------------------------ GEMM + row logsumexp (last tile of a panel merges)
+@pytest.mark.parametrize("store_main", [False, True])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 1000, 136), (256, 4096, 256), (130, 40, 72), (1024, 8200, 64)])
+def test_gemm_row_logsumexp(fc, orc, M, N, K, store_main):
+    run_and_check(fc, orc, wl.gemm_bias_scale_lse(M, N, K, "var", store_main), 3)
+
+
+def test_gemm_row_logsumexp_dominant_and_repeat(fc, orc):
+    """Dominant logits in different column tiles, and the same call twice (the scratch counters are
+    re-zeroed per launch)."""
+    ch = replace(wl.gemm_bias_scale_lse(256, 2048, 64, "var"), ops=())
+    A, B, bias = wl.make_inputs(ch, 2)
+    Af = rng.bf16_bits_to_f32(A).copy(); Bf = rng.bf16_bits_to_f32(B).copy()
+    Af[:, 0] = 8.0; Bf[:, 0] = 0.0
+    Bf[[5, 300, 900, 2047], 0] = [6.0, 6.25, 3.0, 6.25]
+    ins = [rng.store(Af, "bf16"), rng.store(Bf, "bf16"), bias]
+    for _ in range(2):
+        run_and_check(fc, orc, ch, ins=ins)
+
+
 # ------------------------------------------------------------------ kernel (d): implicit-GEMM conv + ReLU + avg-pool
 def _delta_weights(C, r, s):
     w = np.zeros((C, 3, 3, C), np.float32)
