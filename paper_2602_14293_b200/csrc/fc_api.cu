@@ -169,7 +169,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
         default:
             if (s->in_dtype != FC_BF16 || s->reduce != FC_RED_GLOBAL_AVGPOOL || s->store_main)
                 return fail(FC_ERR_UNSUPPORTED, "conv supports bf16 input with GLOBAL_AVGPOOL and store_main = 0");
-            if (s->stride != 1) return fail(FC_ERR_UNSUPPORTED, "conv supports stride 1");
+            if (s->stride > 8) return fail(FC_ERR_UNSUPPORTED, "conv supports stride <= 8");
             if (s->pad >= s->R || s->pad >= s->S || s->R > 16 || s->S > 16) return fail(FC_ERR_UNSUPPORTED, "conv supports pad < R,S <= 16");
             plan->kind = Plan::TC_CONV;
             break;
@@ -323,7 +323,8 @@ fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr
     // base pixels run over the output grid shifted by -pad; a filter tap adds (s, r) to every base pixel
     const int lower[2] = {(int) -s->pad, (int) -s->pad};
     const int upper[2] = {(int) (s->pad - (s->S - 1)), (int) (s->pad - (s->R - 1))};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    // base pixels advance by the convolution stride along w and h
+    const cuuint32_t estr[4] = {1, (cuuint32_t) s->stride, (cuuint32_t) s->stride, 1};
     CUresult r = g_encode_im2col(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper,
                                  64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

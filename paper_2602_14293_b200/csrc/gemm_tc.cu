@@ -366,7 +366,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if constexpr (MODE == 2) {
                         const int tap = kb / kb_per_tap, c0 = (kb - tap * kb_per_tap) * BK;
                         const int r = tap / p.S, sx = tap - r * p.S;
-                        ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow - p.pad, oh - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
+                        ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap * p.Cin + c0, bcol0, full);
                     } else {
                         ptx::tma_load_2d_pair(sa, &tmA, kb * BK, row0, full);

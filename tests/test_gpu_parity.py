@@ -105,7 +105,7 @@ def test_lse_shift_overflow_safety(fc, orc):
 def test_lse_row_dominated_by_one_gelu_value(fc, orc):
     """Adversarial for an approximate activation: one moderate GELU value dominates the row (every
     other residual is -30), so the logsumexp equals that value and inherits its full error."""
-    ch = replace(wl.affine_gelu_residual_lse(64, 512), store_main=False)   # y itself is ~ -30: only the fp32 reduction is judged
+    ch = replace(wl.affine_gelu_residual_lse(64, 512), store_main=False)   # y itself is ~ -30: only the fp32 reduction is checked
     x, g, b, r = wl.make_inputs(ch, 9)
     rf = np.full((64, 512), -30.0, np.float32)
     cols = (np.arange(64) * 7) % 512
@@ -291,6 +291,18 @@ def test_conv_delta_kernels_pool_shifted_image(fc, orc, r, s):
 @pytest.mark.parametrize("seed", [0, 1])
 def test_conv_chain_reduced(fc, orc, batch, H, W, Cin, Cout, seed):
     run_and_check(fc, orc, wl.conv_bias_relu_avgpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout), seed)
+
+
+@pytest.mark.parametrize("R,S,pad", [(1, 1, 0), (3, 3, 0), (5, 5, 2), (3, 5, 1), (5, 3, 2), (1, 3, 0), (7, 7, 3)])
+def test_conv_filter_shapes(fc, orc, R, S, pad):
+    """Filter sizes other than 3x3, non-square filters (pins which bounding-box corner belongs to
+    which axis) and pad 0."""
+    run_and_check(fc, orc, wl.conv_bias_relu_avgpool(batch=2, H=12, W=20, Cin=64, Cout=64, R=R, S=S, pad=pad), 5)
+
+
+@pytest.mark.parametrize("H,W,R,S,pad,stride", [(12, 20, 3, 3, 1, 2), (13, 21, 3, 3, 1, 2), (16, 16, 1, 1, 0, 2), (15, 18, 5, 5, 2, 3), (14, 14, 3, 3, 0, 2)])
+def test_conv_strided(fc, orc, H, W, R, S, pad, stride):
+    run_and_check(fc, orc, wl.conv_bias_relu_avgpool(batch=3, H=H, W=W, Cin=64, Cout=64, R=R, S=S, pad=pad, stride=stride), 7)
 
 
 def test_conv_all_ones_closed_form(fc, orc):
