@@ -138,7 +138,11 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
  * memory makes the copies asynchronous).  `staging` is a caller-owned DEVICE buffer of at least
  * fc_staging_size() bytes into which inputs are copied (cudaMemcpyAsync on the stream), the chain
  * runs there, and outputs are copied back.  Enqueues only; the caller synchronises the stream
- * before reading the outputs.
+ * before reading the outputs.  Chains that move 32 MB or more are cut into up to 8 row (image)
+ * chunks whose copies run on two internal copy streams (created on the first such call on a
+ * device), so that copy-in, kernel and copy-out of neighbouring chunks overlap; the work is still
+ * ordered after everything enqueued on `cuda_stream` before the call, and `cuda_stream` waits for
+ * the last copy-out.
  */
 fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, int n_inputs,
                       fc_tensor* host_outputs, int n_outputs, void* staging, size_t staging_bytes,

@@ -36,6 +36,16 @@ struct DeviceInfo {
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_mu;
 
+// copy streams and events of fc_run_host's chunk pipeline, created on first use per device
+struct HostPipe {
+    static constexpr int kEvents = 2 + 2 * 8;
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev[kEvents] = {};
+    std::mutex mu;
+};
+HostPipe g_pipe[kMaxDevices];
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -465,17 +475,18 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
     if (reinterpret_cast<uintptr_t>(staging) & 255) return fail(FC_ERR_ALIGNMENT, "staging buffer must be 256-byte aligned");
     cudaStream_t stream = (cudaStream_t) cuda_stream;
     fc_tensor din[16], dout[4];
-    size_t nbytes_out[4];
+    size_t nbytes_in[16], nbytes_out[4];
     char* cur = (char*) staging;
+    size_t moved = 0;
     for (int i = 0; i < n_inputs; ++i) {
         if (!host_inputs[i].ptr) return fail(FC_ERR_NULL, "host_inputs[%d]: null pointer", i);
         size_t n = dt_size(host_inputs[i].dtype);
         for (int k = 0; k < host_inputs[i].rank; ++k) n *= (size_t) host_inputs[i].shape[k];
+        nbytes_in[i] = n;
         din[i] = host_inputs[i];
         din[i].ptr = cur;
-        cudaError_t e = cudaMemcpyAsync(cur, host_inputs[i].ptr, n, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync H2D");
         cur += (n + 255) / 256 * 256;
+        moved += n;
     }
     for (int i = 0; i < n_outputs; ++i) {
         if (!host_outputs[i].ptr) return fail(FC_ERR_NULL, "host_outputs[%d]: null pointer", i);
@@ -485,12 +496,97 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
         dout[i] = host_outputs[i];
         dout[i].ptr = cur;
         cur += (n + 255) / 256 * 256;
+        moved += n;
     }
-    if ((st = fc_run(spec, din, n_inputs, dout, n_outputs, cuda_stream))) return st;
-    for (int i = 0; i < n_outputs; ++i) {
-        cudaError_t e = cudaMemcpyAsync(host_outputs[i].ptr, dout[i].ptr, nbytes_out[i], cudaMemcpyDeviceToHost, stream);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync D2H");
+
+    // Rows (images) are independent problems: large chains are cut into row chunks so that the
+    // host-to-device copy of chunk i+1, the kernel of chunk i and the device-to-host copy of chunk
+    // i-1 overlap (two internal copy streams; the kernels stay on the caller's stream).
+    const bool conv = spec->producer == FC_PROD_CONV2D_NHWC;
+    const long long rows = conv ? spec->batch : spec->M;
+    const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE) ? 256 : 1;
+    long long chunks = 1;
+    if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
+        chunks = rows / gran < 8 ? rows / gran : 8;
+        if (chunks < 1) chunks = 1;
     }
+    if (chunks == 1) {
+        for (int i = 0; i < n_inputs; ++i) {
+            cudaError_t e = cudaMemcpyAsync(din[i].ptr, host_inputs[i].ptr, nbytes_in[i], cudaMemcpyHostToDevice, stream);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync H2D");
+        }
+        if ((st = fc_run(spec, din, n_inputs, dout, n_outputs, cuda_stream))) return st;
+        for (int i = 0; i < n_outputs; ++i) {
+            cudaError_t e = cudaMemcpyAsync(host_outputs[i].ptr, dout[i].ptr, nbytes_out[i], cudaMemcpyDeviceToHost, stream);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync D2H");
+        }
+        return FC_OK;
+    }
+
+    // whole-shape validation first: the chunks below are validated against sub-shapes only
+    if ((st = validate_tensors(spec, plan, din, n_inputs, dout, n_outputs))) return st;
+    int ordinal = 0;
+    DeviceInfo* dev;
+    if ((st = get_device(&dev, &ordinal))) return st;
+    HostPipe& hp = g_pipe[ordinal];
+    std::lock_guard<std::mutex> lk(hp.mu);
+    cudaError_t e;
+    if (!hp.ready) {
+        if ((e = cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking)) != cudaSuccess ||
+            (e = cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking)) != cudaSuccess)
+            return cuda_fail(e, "cudaStreamCreateWithFlags");
+        for (int i = 0; i < HostPipe::kEvents; ++i)
+            if ((e = cudaEventCreateWithFlags(&hp.ev[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e, "cudaEventCreateWithFlags");
+        hp.ready = true;
+    }
+    bool split[16];
+    for (int i = 0; i < n_inputs; ++i) split[i] = i == 0;
+    for (int i = 0; i < spec->n_ops; ++i)
+        if (spec->ops[i].kind == FC_OP_ADD_TENSOR) split[spec->ops[i].in0] = true;
+    cudaEvent_t ev_start = hp.ev[0], ev_done = hp.ev[1];
+#define FC_TRY(call, what) do { if ((e = (call)) != cudaSuccess) return cuda_fail(e, what); } while (0)
+    FC_TRY(cudaEventRecord(ev_start, stream), "cudaEventRecord");
+    FC_TRY(cudaStreamWaitEvent(hp.s_in, ev_start, 0), "cudaStreamWaitEvent");
+    FC_TRY(cudaStreamWaitEvent(hp.s_out, ev_start, 0), "cudaStreamWaitEvent");
+    for (int i = 0; i < n_inputs; ++i)
+        if (!split[i]) FC_TRY(cudaMemcpyAsync(din[i].ptr, host_inputs[i].ptr, nbytes_in[i], cudaMemcpyHostToDevice, hp.s_in), "cudaMemcpyAsync H2D");
+    const long long per = ((rows + chunks - 1) / chunks + gran - 1) / gran * gran;
+    int c = 0;
+    for (long long r0 = 0; r0 < rows; r0 += per, ++c) {
+        const long long r1 = r0 + per < rows ? r0 + per : rows;
+        fc_chain_spec sub = *spec;
+        if (conv) sub.batch = r1 - r0; else sub.M = r1 - r0;
+        fc_tensor sin[16], sout[4];
+        for (int i = 0; i < n_inputs; ++i) {
+            sin[i] = din[i];
+            if (!split[i]) continue;
+            const size_t row_bytes = nbytes_in[i] / (size_t) rows;
+            sin[i].ptr = (char*) din[i].ptr + (size_t) r0 * row_bytes;
+            sin[i].shape[0] = r1 - r0;
+            FC_TRY(cudaMemcpyAsync(sin[i].ptr, (const char*) host_inputs[i].ptr + (size_t) r0 * row_bytes, (size_t) (r1 - r0) * row_bytes,
+                                   cudaMemcpyHostToDevice, hp.s_in), "cudaMemcpyAsync H2D");
+        }
+        cudaEvent_t ev_in = hp.ev[2 + 2 * c], ev_k = hp.ev[3 + 2 * c];
+        FC_TRY(cudaEventRecord(ev_in, hp.s_in), "cudaEventRecord");
+        FC_TRY(cudaStreamWaitEvent(stream, ev_in, 0), "cudaStreamWaitEvent");
+        for (int i = 0; i < n_outputs; ++i) {
+            const size_t row_bytes = nbytes_out[i] / (size_t) rows;
+            sout[i] = dout[i];
+            sout[i].ptr = (char*) dout[i].ptr + (size_t) r0 * row_bytes;
+            sout[i].shape[0] = r1 - r0;
+        }
+        if ((st = fc_run(&sub, sin, n_inputs, sout, n_outputs, cuda_stream))) return st;
+        FC_TRY(cudaEventRecord(ev_k, stream), "cudaEventRecord");
+        FC_TRY(cudaStreamWaitEvent(hp.s_out, ev_k, 0), "cudaStreamWaitEvent");
+        for (int i = 0; i < n_outputs; ++i) {
+            const size_t row_bytes = nbytes_out[i] / (size_t) rows;
+            FC_TRY(cudaMemcpyAsync((char*) host_outputs[i].ptr + (size_t) r0 * row_bytes, sout[i].ptr, (size_t) (r1 - r0) * row_bytes,
+                                   cudaMemcpyDeviceToHost, hp.s_out), "cudaMemcpyAsync D2H");
+        }
+    }
+    FC_TRY(cudaEventRecord(ev_done, hp.s_out), "cudaEventRecord");
+    FC_TRY(cudaStreamWaitEvent(stream, ev_done, 0), "cudaStreamWaitEvent");
+#undef FC_TRY
     return FC_OK;
 }
 

@@ -342,3 +342,27 @@ def test_run_host_matches_device_path(fc, orc):
     torch.cuda.synchronize()
     assert torch.equal(dev_out[0].cpu(), host_out[0])
     util.check(host_out[0], orc.run_chain(ch, ins)["main"], "fc_run_host")
+
+
+def test_run_host_chunk_pipeline_matches_device_path(fc, orc):
+    """Chains that move >= 32 MB go through fc_run_host's chunk pipeline (copies on two internal
+    streams).  The results must equal those of the plain device path on the same inputs."""
+    cases = [wl.affine_gelu_residual_lse(4100, 4096), wl.gemm_softmax(4096, 4096, 512, "var"),
+             wl.gemm_bias_gelu_scale_clamp(4000, 4096, 512, "var"), wl.gemm_bias_scale_lse(4096, 4096, 512, "var", True),
+             wl.conv_bias_relu_avgpool(batch=20)]
+    for ch in cases:
+        ins = wl.make_inputs(ch, 1)
+        host_in = [fc.to_device(a, "cpu").pin_memory() for a in ins]
+        host_out = util.poison_(fc.binding.output_tensors(ch, "cpu", pinned=True))
+        spec = fc.make_spec(ch)
+        staging = torch.empty(fc.fc_staging_size(spec, host_in, host_out), dtype=torch.uint8, device="cuda")
+        for _ in range(2):
+            fc.run_chain_host(ch, host_in, host_out, staging)
+        fc.fc_get_async_status()
+        dev_out = fc.run_chain(ch, [t.cuda() for t in host_in])
+        torch.cuda.synchronize()
+        for a, b in zip(dev_out, host_out):
+            if ch.reduce == "global_avgpool":      # pooled sums are combined with atomics: order varies
+                assert torch.allclose(a.cpu(), b, rtol=1e-5, atol=1e-6)
+            else:
+                assert torch.equal(a.cpu(), b), ch.name
