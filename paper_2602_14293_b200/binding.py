@@ -172,6 +172,24 @@ def fc_run(spec: fc_chain_spec, inputs: Sequence[torch.Tensor], outputs: Sequenc
                         _stream_handle(stream)), "fc_run")
 
 
+class PreparedRun:
+    """The marshalled arguments of one fc_run call, built once: `run()` is then a single C call
+    (building the ctypes structures costs more than a small kernel's run time)."""
+
+    def __init__(self, spec: fc_chain_spec, inputs: Sequence[torch.Tensor], outputs: Sequence[torch.Tensor], stream=None):
+        self._keep = (spec, list(inputs), list(outputs))      # keeps the tensors alive
+        self._spec = ctypes.byref(spec)
+        self._in, self._n_in = _tensor_array(inputs), len(inputs)
+        self._out, self._n_out = _tensor_array(outputs), len(outputs)
+        self._stream = _stream_handle(stream)
+        self._fn = lib().fc_run
+
+    def run(self) -> None:
+        st = self._fn(self._spec, self._in, self._n_in, self._out, self._n_out, self._stream)
+        if st != 0:
+            raise FcError(st, "fc_run")
+
+
 def fc_run_softmax_static_scratch(spec: fc_chain_spec, inputs: Sequence[torch.Tensor], outputs: Sequence[torch.Tensor],
                                   stream=None) -> None:
     """GEMM + row softmax for callers that cannot allocate: same arguments as fc_run, scratch taken from
