@@ -42,7 +42,7 @@ class Chain:
     # ops: ("bias_n", i) ("affine_n", i, j) ("relu",) ("gelu_tanh",) ("scale", f) ("clamp", lo, hi)
     #      ("add_tensor", i)   -- i, j index the input list
     ops: Tuple[tuple, ...] = ()
-    reduce: str = "none"          # "none" | "row_logsumexp" | "row_softmax" | "global_avgpool"
+    reduce: str = "none"          # "none" | "row_logsumexp" | "row_softmax" | "global_avgpool" | "row_sum" | "row_max" | "row_mean"
     store_main: bool = True
     # (tag, dtype, shape, dist, p0, p1) per input, in input order
     input_recipe: Tuple[tuple, ...] = field(default=(), compare=False)
@@ -183,7 +183,7 @@ def output_shapes(chain: Chain):
         return outs
     if chain.store_main:
         outs.append(("main", chain.out_dtype, main_shape))
-    if chain.reduce == "row_logsumexp":
+    if chain.reduce in ("row_logsumexp", "row_sum", "row_max", "row_mean"):
         outs.append(("reduce", "f32", (chain.M,)))
     elif chain.reduce == "global_avgpool":
         outs.append(("reduce", "f32", (chain.batch, chain.Cout)))

@@ -31,7 +31,8 @@
  *   [batch,H,W,Cin], inputs[1] = weights [Cout,R,S,Cin].  ELEMENTWISE: inputs[0] = x [M,N].
  *   Further inputs are the vectors ([N] or [Cout]) and tensors that fc_op.in0 / in1 index.
  *   Outputs, in order: the main output (if store_main, or if reduce == ROW_SOFTMAX, whose
- *   probabilities take the main output's place), then the reduction (LOGSUMEXP: f32 [M];
+ *   probabilities take the main output's place), then the reduction (LOGSUMEXP / ROW_SUM / ROW_MAX /
+ *   ROW_MEAN: f32 [M];
  *   GLOBAL_AVGPOOL: f32 [batch,Cout]).
  *
  * Alignment.  Base pointers of bf16 operands of GEMM / CONV must be 16-byte aligned and K (GEMM)
@@ -92,7 +93,10 @@ typedef enum {
     FC_RED_NONE = 0,
     FC_RED_ROW_LOGSUMEXP = 1,   /* out[m] = max_n v + log sum_n exp(v - max)          */
     FC_RED_ROW_SOFTMAX = 2,     /* p[m][n] = exp(v - max) / sum_n exp(v - max)         */
-    FC_RED_GLOBAL_AVGPOOL = 3   /* out[b][c] = mean over (oh, ow) of v[b][oh][ow][c]   */
+    FC_RED_GLOBAL_AVGPOOL = 3,  /* out[b][c] = mean over (oh, ow) of v[b][oh][ow][c]   */
+    FC_RED_ROW_SUM = 4,         /* out[m] = sum_n v          (elementwise producer)     */
+    FC_RED_ROW_MAX = 5,         /* out[m] = max_n v          (elementwise producer)     */
+    FC_RED_ROW_MEAN = 6         /* out[m] = (sum_n v) / N    (elementwise producer)     */
 } fc_reduce;
 
 typedef struct {

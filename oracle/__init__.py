@@ -133,6 +133,20 @@ def row_softmax(V: np.ndarray) -> np.ndarray:
     return P
 
 
+def row_sum(V: np.ndarray) -> np.ndarray:
+    rows, N = V.shape
+    out = np.empty((rows,), dtype=np.float64)
+    lib().orc_row_sum(_p(V), _i64(rows), _i64(N), _p(out))
+    return out
+
+
+def row_max(V: np.ndarray) -> np.ndarray:
+    rows, N = V.shape
+    out = np.empty((rows,), dtype=np.float64)
+    lib().orc_row_max(_p(V), _i64(rows), _i64(N), _p(out))
+    return out
+
+
 def global_avgpool(V: np.ndarray) -> np.ndarray:
     NB, OH, OW, C = V.shape
     out = np.empty((NB, C), dtype=np.float64)
@@ -161,6 +175,12 @@ def run_chain(chain, inputs: List[np.ndarray]) -> Dict[str, np.ndarray]:
         out["reduce"] = row_softmax(V.reshape(-1, V.shape[-1]))
     elif chain.reduce == "global_avgpool":
         out["reduce"] = global_avgpool(V)
+    elif chain.reduce == "row_sum":
+        out["reduce"] = row_sum(V.reshape(-1, V.shape[-1]))
+    elif chain.reduce == "row_max":
+        out["reduce"] = row_max(V.reshape(-1, V.shape[-1]))
+    elif chain.reduce == "row_mean":
+        out["reduce"] = row_sum(V.reshape(-1, V.shape[-1])) / V.shape[-1]
     elif chain.reduce != "none":
         raise ValueError(chain.reduce)
     return out

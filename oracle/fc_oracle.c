@@ -20,7 +20,8 @@
  *                      multiply).
  *   orc_row_logsumexp  max + log(sum exp(v - max)); over a row of length one this is the identity,
  *                      the closed form the paper's appendix (Level-2 Q18 analysis) relies on.
- *   orc_gelu_tanh, orc_clamp, orc_affine_n, orc_add_tensor, orc_row_softmax, orc_global_avgpool
+ *   orc_gelu_tanh, orc_clamp, orc_affine_n, orc_add_tensor, orc_row_softmax, orc_global_avgpool,
+ *   orc_row_sum, orc_row_max (row mean = row sum / N)
  *                      textbook definitions; the paper does not print them, the benchmark
  *                      configurations of this repository name them.
  *
@@ -185,5 +186,25 @@ void orc_global_avgpool(const double* V, int64_t NB, int64_t HW, int64_t C, doub
             for (int64_t p = 0; p < HW; ++p) s += V[(b * HW + p) * C + c];
             out[b * C + c] = s / (double)HW;
         }
+    }
+}
+
+/* out[m] = sum_n V[m][n], n ascending, one accumulator */
+void orc_row_sum(const double* V, int64_t rows, int64_t N, double* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < rows; ++m) {
+        double s = 0.0;
+        for (int64_t n = 0; n < N; ++n) s += V[m * N + n];
+        out[m] = s;
+    }
+}
+
+/* out[m] = max_n V[m][n] */
+void orc_row_max(const double* V, int64_t rows, int64_t N, double* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < rows; ++m) {
+        double mx = V[m * N];
+        for (int64_t n = 1; n < N; ++n) mx = V[m * N + n] > mx ? V[m * N + n] : mx;
+        out[m] = mx;
     }
 }

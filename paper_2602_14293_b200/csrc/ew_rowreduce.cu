@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
 
     for (long long m = blockIdx.x; m < p.M; m += gridDim.x) {
         MaxSum acc = ms_identity();
+        float psum = 0.0f, pmax = -CUDART_INF_F;   // ROW_SUM / ROW_MEAN and ROW_MAX
         for (long long c = threadIdx.x; c < chunks; c += kThreads) {
             const long long n0 = c * kV;
             const bool full = n0 + kV <= N;
@@ -75,6 +76,14 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
                 for (int j = 0; j < kV; ++j) s += n0 + j < N ? exp2_fast((v[j] - mx) * kLog2e) : 0.0f;
                 acc = ms_merge(acc, MaxSum{mx, s});
             }
+            if (p.reduce >= FC_RED_ROW_SUM) {
+#pragma unroll
+                for (int j = 0; j < kV; ++j)
+                    if (n0 + j < N) {
+                        psum += v[j];
+                        pmax = fmaxf(pmax, v[j]);
+                    }
+            }
             if (p.y) {
                 if (p.y_dt == FC_BF16) {
                     unsigned short* yp = (unsigned short*) p.y + m * N + n0;
@@ -104,6 +113,25 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
         if (p.reduce == FC_RED_ROW_LOGSUMEXP) {
             const MaxSum t = block_merge(acc, red);
             if (threadIdx.x == 0) p.red[m] = t.m + logf(t.s);
+        } else if (p.reduce >= FC_RED_ROW_SUM) {
+            // the pair slots carry (max, plain sum) here
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                psum += __shfl_xor_sync(0xffffffffu, psum, o);
+                pmax = fmaxf(pmax, __shfl_xor_sync(0xffffffffu, pmax, o));
+            }
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            __syncthreads();
+            if (lane == 0) red[warp] = MaxSum{pmax, psum};
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                float ts = 0.0f, tm = -CUDART_INF_F;
+                for (int w = 0; w < kWarps; ++w) {
+                    ts += red[w].s;
+                    tm = fmaxf(tm, red[w].m);
+                }
+                p.red[m] = p.reduce == FC_RED_ROW_MAX ? tm : (p.reduce == FC_RED_ROW_MEAN ? ts / (float) N : ts);
+            }
         }
     }
 }
@@ -125,6 +153,7 @@ struct EwFastParams {
     const void* vec1; int vec1_dt;   // beta
     long long M;
     int N;
+    int red_kind;           // fc_reduce of the row reduction (when the kernel is built with one)
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -145,7 +174,7 @@ constexpr int kGroup = 4;   // chunks in flight per lane and tensor
 // and the chunk's contribution to the running (max, sum) of the row (log2 domain).
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
 __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
-                                         float& run_m, float& run_s) {
+                                         int red_kind, float& run_m, float& run_s) {
     float2 v[4];
     v[0] = make_float2(bf16_lo(xq.x), bf16_hi(xq.x));
     v[1] = make_float2(bf16_lo(xq.y), bf16_hi(xq.y));
@@ -205,7 +234,14 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
         q.z = pack_bf16x2(v[2].x, v[2].y); q.w = pack_bf16x2(v[3].x, v[3].y);
         st_stream(yr + c, q);
     }
-    if (LSE) {
+    if (LSE && red_kind != FC_RED_ROW_LOGSUMEXP) {
+        // ROW_SUM / ROW_MEAN / ROW_MAX: plain running sum and maximum
+        const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)),
+                               fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
+        const float2 t = __fadd2_rn(__fadd2_rn(v[0], v[1]), __fadd2_rn(v[2], v[3]));
+        run_m = fmaxf(run_m, cm);
+        run_s += t.x + t.y;
+    } else if (LSE) {
         const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)),
                                fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
         const float nm = fmaxf(run_m, cm * kLog2e);
@@ -258,10 +294,18 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
 #pragma unroll
             for (int g = 0; g < kGroup; ++g) {
                 const int c = c0 + 32 * g;
-                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, run_m, run_s);
+                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, p.red_kind, run_m, run_s);
             }
         }
-        if (LSE) {
+        if (LSE && p.red_kind != FC_RED_ROW_LOGSUMEXP) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                run_s += __shfl_xor_sync(0xffffffffu, run_s, o);
+                run_m = fmaxf(run_m, __shfl_xor_sync(0xffffffffu, run_m, o));
+            }
+            if (lane == 0)
+                p.lse[row] = p.red_kind == FC_RED_ROW_MAX ? run_m : (p.red_kind == FC_RED_ROW_MEAN ? run_s / (float) N : run_s);
+        } else if (LSE) {
             // merge the 32 per-lane pairs (log2 domain)
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -308,6 +352,7 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
     }
     if (i != p.ops.n) return false;
     f->x = (const uint4*) p.x; f->y = (uint4*) p.y; f->lse = p.red; f->M = p.M; f->N = (int) p.N;
+    f->red_kind = p.reduce;
     return true;
 }
 
@@ -336,7 +381,7 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
     EwFastParams f;
     int pre, act;
     bool res;
-    const bool lse = p.reduce == FC_RED_ROW_LOGSUMEXP;
+    const bool lse = p.reduce != FC_RED_NONE;   // any row reduction
     if (match_fast(p, &f, &pre, &act, &res) && (lse || p.y)) {
         const bool store = p.y != nullptr;
 #define FC_EW_CASE(PRE_, ACT_)                                                                       \

@@ -130,7 +130,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if ((s->in_dtype != FC_F32 && s->in_dtype != FC_BF16) || (s->out_dtype != FC_F32 && s->out_dtype != FC_BF16))
         return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
     if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
-    if (s->reduce < 0 || s->reduce > FC_RED_GLOBAL_AVGPOOL) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
+    if (s->reduce < 0 || s->reduce > FC_RED_ROW_MEAN) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
     if (s->n_ops < 0 || s->n_ops > FC_MAX_OPS) return fail(FC_ERR_INVALID_SPEC, "n_ops %d out of range", s->n_ops);
     for (int i = 0; i < s->n_ops; ++i)
         if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_ADD_TENSOR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
@@ -157,8 +157,8 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     plan->main_index = plan->red_index = -1;
     switch (s->producer) {
         case FC_PROD_ELEMENTWISE:
-            if (s->reduce != FC_RED_NONE && s->reduce != FC_RED_ROW_LOGSUMEXP)
-                return fail(FC_ERR_UNSUPPORTED, "elementwise producer supports reduce NONE or ROW_LOGSUMEXP");
+            if (s->reduce == FC_RED_ROW_SOFTMAX || s->reduce == FC_RED_GLOBAL_AVGPOOL)
+                return fail(FC_ERR_UNSUPPORTED, "elementwise producer supports reduce NONE, ROW_LOGSUMEXP, ROW_SUM, ROW_MAX or ROW_MEAN");
             plan->kind = Plan::EW;
             break;
         case FC_PROD_GEMM_NT:
@@ -262,9 +262,9 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         }
     }
     if (plan.red_index >= 0) {
-        if (s->reduce == FC_RED_ROW_LOGSUMEXP) {
+        if (s->reduce != FC_RED_GLOBAL_AVGPOOL) {
             const long long sh[1] = {s->M};
-            if ((st = check_tensor(out[plan.red_index], "logsumexp output", FC_F32, 1, sh))) return st;
+            if ((st = check_tensor(out[plan.red_index], "row reduction output", FC_F32, 1, sh))) return st;
         } else {
             const long long sh[2] = {s->batch, s->Cout};
             if ((st = check_tensor(out[plan.red_index], "pooled output", FC_F32, 2, sh))) return st;

@@ -114,6 +114,10 @@ def run_chain(chain, inputs):
             s = mp.fsum(e)
             P.append([float(x / s) for x in e])
         out["reduce"] = np.array(P).reshape(shape)
+    elif chain.reduce in ("row_sum", "row_mean"):
+        out["reduce"] = np.array([float(mp.fsum(list(row)) / (N if chain.reduce == "row_mean" else 1)) for row in V])
+    elif chain.reduce == "row_max":
+        out["reduce"] = np.array([float(max(row)) for row in V])
     elif chain.reduce == "global_avgpool":
         NB, OH, OW, C = shape
         V4 = V.reshape(NB, OH * OW, C)

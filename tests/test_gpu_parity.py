@@ -91,6 +91,15 @@ def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     assert float(np.abs(util.to_f64(outs[0]) - ref["main"]).max()) <= 2e-5
 
 
+@pytest.mark.parametrize("red", ["row_sum", "row_max", "row_mean"])
+@pytest.mark.parametrize("M,N,dt", [(33, 4096, "bf16"), (7, 1000, "bf16"), (5, 333, "bf16"), (9, 515, "f32"), (64, 8192, "bf16")])
+def test_elementwise_row_sum_max_mean(fc, orc, red, M, N, dt):
+    base = wl.affine_gelu_residual_lse(M, N)
+    rec = tuple((t, dt, s, d, a, b) for t, _, s, d, a, b in base.input_recipe)
+    run_and_check(fc, orc, replace(base, reduce=red, in_dtype=dt, out_dtype=dt, input_recipe=rec), 4)
+    run_and_check(fc, orc, replace(base, reduce=red, store_main=False, ops=(("relu",),), in_dtype=dt, out_dtype=dt, input_recipe=rec), 4)
+
+
 def test_lse_shift_overflow_safety(fc, orc):
     ch = replace(wl.affine_gelu_residual_lse(4, 512), ops=(), in_dtype="f32", out_dtype="f32",
                  input_recipe=(("x", "f32", (4, 512), "normal", 0.0, 1.0),))

@@ -244,6 +244,25 @@ def test_softmax_properties(orc):
     np.testing.assert_allclose(P, torch.softmax(torch.from_numpy(v), 1).numpy(), rtol=1e-13)
 
 
+def test_row_sum_max_mean(orc):
+    V = _rand((5, 37), 23, -3, 3)
+    np.testing.assert_allclose(orc.row_sum(V), V.sum(1), rtol=0, atol=1e-13)
+    assert np.array_equal(orc.row_max(V), V.max(1))
+    ints = np.arange(1.0, 101.0)[None, :].repeat(2, 0)
+    assert np.array_equal(orc.row_sum(np.ascontiguousarray(ints)), [5050.0, 5050.0])
+    one = np.full((1, 9), -7.5); one[0, 4] = 2.0
+    assert orc.row_max(one)[0] == 2.0 and orc.row_sum(one)[0] == -58.0
+    from dataclasses import replace as _r
+    for red in ("row_sum", "row_max", "row_mean"):
+        ch = _r(wl.affine_gelu_residual_lse(3, 9), reduce=red)
+        ins = wl.make_inputs(ch, 5)
+        got, want = orc.run_chain(ch, ins), brute.run_chain(ch, ins)
+        np.testing.assert_allclose(got["reduce"], want["reduce"], rtol=1e-13, atol=1e-14)
+    ch = _r(wl.affine_gelu_residual_lse(4, 16), reduce="row_mean", ops=())
+    x = wl.make_inputs(ch, 1)[0]
+    np.testing.assert_allclose(orc.run_chain(ch, [x])["reduce"], rng.bf16_bits_to_f32(x).astype(np.float64).mean(1), atol=1e-15)
+
+
 def test_avgpool_properties(orc):
     V = _rand((2, 3, 4, 5), 19); U = _rand((2, 3, 4, 5), 20)
     np.testing.assert_allclose(orc.global_avgpool(np.full((2, 3, 4, 5), 7.25)), 7.25, rtol=1e-15)
