@@ -131,9 +131,11 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 
 
 def store(a_f32: np.ndarray, dtype: str) -> np.ndarray:
-    """Round an fp32 array to the storage type: 'f32' -> float32, 'bf16' -> uint16 patterns."""
+    """Round an fp32 array to the storage type: 'f32' -> float32, 'bf16' -> uint16 patterns, 'f16' -> float16."""
     if dtype == "f32":
         return np.ascontiguousarray(a_f32, dtype=np.float32)
     if dtype == "bf16":
         return f32_to_bf16_bits(a_f32)
+    if dtype == "f16":
+        return np.ascontiguousarray(a_f32, dtype=np.float32).astype(np.float16)   # IEEE half, round to nearest even
     raise ValueError(dtype)

@@ -35,7 +35,7 @@
  *   ROW_MEAN: f32 [M];
  *   GLOBAL_AVGPOOL: f32 [batch,Cout]).
  *
- * Alignment.  Base pointers of bf16 operands of GEMM / CONV must be 16-byte aligned and K (GEMM)
+ * Alignment.  Base pointers of bf16 / fp16 operands of GEMM / CONV must be 16-byte aligned and K (GEMM)
  * or Cin (CONV) a multiple of 8; violations return FC_ERR_ALIGNMENT.  Other tensors need only the
  * natural alignment of their element type (vector access is used when 16-byte alignment holds).
  *
@@ -75,7 +75,7 @@ typedef enum {
     FC_ERR_TIMEOUT = 9        /* a bounded device-side wait expired                           */
 } fc_status;
 
-typedef enum { FC_F32 = 0, FC_BF16 = 1 } fc_dtype;
+typedef enum { FC_F32 = 0, FC_BF16 = 1, FC_F16 = 2 } fc_dtype;   /* FC_F16: IEEE binary16, the storage type of the paper's kernels */
 
 typedef enum { FC_PROD_ELEMENTWISE = 0, FC_PROD_GEMM_NT = 1, FC_PROD_CONV2D_NHWC = 2 } fc_producer;
 

@@ -54,11 +54,13 @@ def _p(a: np.ndarray):
 
 
 def widen(a: np.ndarray) -> np.ndarray:
-    """Stored tensor (float32, or uint16 bf16 patterns) -> float64, exactly."""
+    """Stored tensor (float32, float16, or uint16 bf16 patterns) -> float64, exactly."""
     a = np.ascontiguousarray(a)
     out = np.empty(a.shape, dtype=np.float64)
     if a.dtype == np.uint16:
         lib().orc_widen_bf16(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
+    elif a.dtype == np.float16:
+        lib().orc_widen_f16(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
     elif a.dtype == np.float32:
         lib().orc_widen_f32(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
     elif a.dtype == np.float64:

@@ -56,6 +56,19 @@ void orc_widen_bf16(const uint16_t* src, int64_t n, double* dst) {
     }
 }
 
+/* IEEE binary16 -> double, exactly (sign, 5-bit exponent, 10-bit fraction; subnormals, inf, nan) */
+void orc_widen_f16(const uint16_t* src, int64_t n, double* dst) {
+    for (int64_t i = 0; i < n; ++i) {
+        const uint16_t h = src[i];
+        const int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+        double v;
+        if (e == 0) v = ldexp((double)f, -24);
+        else if (e == 31) v = f ? NAN : INFINITY;
+        else v = ldexp((double)(1024 + f), e - 25);
+        dst[i] = sign ? -v : v;
+    }
+}
+
 void orc_widen_f32(const float* src, int64_t n, double* dst) {
     for (int64_t i = 0; i < n; ++i) dst[i] = (double)src[i];
 }

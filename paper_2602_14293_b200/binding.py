@@ -16,11 +16,11 @@ import torch
 PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(PKG, "libfc.so")
 
-FC_F32, FC_BF16 = 0, 1
+FC_F32, FC_BF16, FC_F16 = 0, 1, 2
 _PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2}
 _OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6}
 _REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3, "row_sum": 4, "row_max": 5, "row_mean": 6}
-_DTYPE = {"f32": FC_F32, "bf16": FC_BF16}
+_DTYPE = {"f32": FC_F32, "bf16": FC_BF16, "f16": FC_F16}
 FC_MAX_OPS = 8
 
 
@@ -137,6 +137,8 @@ def _tensor_struct(t: torch.Tensor) -> fc_tensor:
         ft.dtype = FC_F32
     elif t.dtype == torch.bfloat16:
         ft.dtype = FC_BF16
+    elif t.dtype == torch.float16:
+        ft.dtype = FC_F16
     else:
         raise TypeError(f"unsupported dtype {t.dtype}")
     if t.dim() > 4:
@@ -233,12 +235,12 @@ def fc_get_async_status(stream=None) -> None:
 
 
 # --------------------------------------------------------------------------- conveniences
-_TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+_TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
 _workspace = {}
 
 
 def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
-    """Stored numpy tensor (float32, or uint16 bf16 bit patterns) -> torch tensor on `device`."""
+    """Stored numpy tensor (float32, float16, or uint16 bf16 bit patterns) -> torch tensor on `device`."""
     if a.dtype == np.uint16:
         return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(device)
     return torch.from_numpy(a).to(device)

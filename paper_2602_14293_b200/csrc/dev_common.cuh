@@ -22,6 +22,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
+// 16-bit storage types: bf16 (FC_BF16) or IEEE half (FC_F16), two per 32-bit word
+__device__ __forceinline__ float2 unpack16x2(uint32_t w, bool f16) {
+    if (f16) {
+        float2 r;
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}" : "=f"(r.x), "=f"(r.y) : "r"(w));
+        return r;
+    }
+    return make_float2(bf16_lo(w), bf16_hi(w));
+}
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi, bool f16) {
+    uint32_t r;
+    if (f16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
 __device__ __forceinline__ float tanh_fast(float x) {
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -55,6 +71,7 @@ __device__ __forceinline__ float gelu_tanh(float v) {
 
 __device__ __forceinline__ float load_scalar(const void* p, int dt, long long i) {
     if (dt == FC_BF16) return __uint_as_float(((uint32_t) __ldg((const unsigned short*) p + i)) << 16);
+    if (dt == FC_F16) return unpack16x2((uint32_t) __ldg((const unsigned short*) p + i), true).x;
     return __ldg((const float*) p + i);
 }
 

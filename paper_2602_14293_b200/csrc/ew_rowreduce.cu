@@ -33,8 +33,9 @@ template <bool kPreciseGelu>
 __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) {
     __shared__ MaxSum red[kWarps];
     const long long N = p.N;
-    const int ebytes = p.x_dt == FC_BF16 ? 2 : 4;
-    const int ybytes = p.y_dt == FC_BF16 ? 2 : 4;
+    const int ebytes = p.x_dt == FC_F32 ? 4 : 2;
+    const int ybytes = p.y_dt == FC_F32 ? 4 : 2;
+    const bool x_f16 = p.x_dt == FC_F16, y_f16 = p.y_dt == FC_F16;
     constexpr int kV = 8;  // columns per chunk
     const bool x_vec = ((reinterpret_cast<uintptr_t>(p.x) | (uintptr_t)(N * ebytes)) & 15) == 0;
     const bool y_vec = p.y && ((reinterpret_cast<uintptr_t>(p.y) | (uintptr_t)(N * ybytes)) & 15) == 0;
@@ -47,14 +48,14 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
             const long long n0 = c * kV;
             const bool full = n0 + kV <= N;
             float v[kV];
-            if (p.x_dt == FC_BF16) {
+            if (p.x_dt != FC_F32) {
                 if (full && x_vec) {
                     const uint4 q = __ldg(reinterpret_cast<const uint4*>((const unsigned short*) p.x + m * N + n0));
-                    v[0] = bf16_lo(q.x); v[1] = bf16_hi(q.x); v[2] = bf16_lo(q.y); v[3] = bf16_hi(q.y);
-                    v[4] = bf16_lo(q.z); v[5] = bf16_hi(q.z); v[6] = bf16_lo(q.w); v[7] = bf16_hi(q.w);
+                    const float2 a = unpack16x2(q.x, x_f16), b = unpack16x2(q.y, x_f16), c2 = unpack16x2(q.z, x_f16), d = unpack16x2(q.w, x_f16);
+                    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y; v[4] = c2.x; v[5] = c2.y; v[6] = d.x; v[7] = d.y;
                 } else {
 #pragma unroll
-                    for (int j = 0; j < kV; ++j) v[j] = n0 + j < N ? load_scalar(p.x, FC_BF16, m * N + n0 + j) : 0.0f;
+                    for (int j = 0; j < kV; ++j) v[j] = n0 + j < N ? load_scalar(p.x, p.x_dt, m * N + n0 + j) : 0.0f;
                 }
             } else {
                 if (full && x_vec) {
@@ -85,17 +86,17 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
                     }
             }
             if (p.y) {
-                if (p.y_dt == FC_BF16) {
+                if (p.y_dt != FC_F32) {
                     unsigned short* yp = (unsigned short*) p.y + m * N + n0;
                     if (full && y_vec) {
                         uint4 q;
-                        q.x = pack_bf16x2(v[0], v[1]); q.y = pack_bf16x2(v[2], v[3]);
-                        q.z = pack_bf16x2(v[4], v[5]); q.w = pack_bf16x2(v[6], v[7]);
+                        q.x = pack16x2(v[0], v[1], y_f16); q.y = pack16x2(v[2], v[3], y_f16);
+                        q.z = pack16x2(v[4], v[5], y_f16); q.w = pack16x2(v[6], v[7], y_f16);
                         *reinterpret_cast<uint4*>(yp) = q;
                     } else {
 #pragma unroll
                         for (int j = 0; j < kV; ++j)
-                            if (n0 + j < N) yp[j] = (unsigned short) (pack_bf16x2(v[j], 0.0f) & 0xffffu);
+                            if (n0 + j < N) yp[j] = (unsigned short) (pack16x2(v[j], 0.0f, y_f16) & 0xffffu);
                     }
                 } else {
                     float* yp = (float*) p.y + m * N + n0;
@@ -154,6 +155,7 @@ struct EwFastParams {
     long long M;
     int N;
     int red_kind;           // fc_reduce of the row reduction (when the kernel is built with one)
+    int is_f16;             // x, residual and y are IEEE half instead of bf16
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -174,12 +176,12 @@ constexpr int kGroup = 4;   // chunks in flight per lane and tensor
 // and the chunk's contribution to the running (max, sum) of the row (log2 domain).
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
 __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
-                                         int red_kind, float& run_m, float& run_s) {
+                                         int red_kind, bool f16, float& run_m, float& run_s) {
     float2 v[4];
-    v[0] = make_float2(bf16_lo(xq.x), bf16_hi(xq.x));
-    v[1] = make_float2(bf16_lo(xq.y), bf16_hi(xq.y));
-    v[2] = make_float2(bf16_lo(xq.z), bf16_hi(xq.z));
-    v[3] = make_float2(bf16_lo(xq.w), bf16_hi(xq.w));
+    v[0] = unpack16x2(xq.x, f16);
+    v[1] = unpack16x2(xq.y, f16);
+    v[2] = unpack16x2(xq.z, f16);
+    v[3] = unpack16x2(xq.w, f16);
     if (PRE != kPreNone) {
         const float4 a0 = *reinterpret_cast<const float4*>(svec + c * 8);
         const float4 a1 = *reinterpret_cast<const float4*>(svec + c * 8 + 4);
@@ -197,10 +199,10 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
     }
     float2 r[4];
     if (RES) {
-        r[0] = make_float2(bf16_lo(rq.x), bf16_hi(rq.x));
-        r[1] = make_float2(bf16_lo(rq.y), bf16_hi(rq.y));
-        r[2] = make_float2(bf16_lo(rq.z), bf16_hi(rq.z));
-        r[3] = make_float2(bf16_lo(rq.w), bf16_hi(rq.w));
+        r[0] = unpack16x2(rq.x, f16);
+        r[1] = unpack16x2(rq.y, f16);
+        r[2] = unpack16x2(rq.z, f16);
+        r[3] = unpack16x2(rq.w, f16);
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -230,8 +232,8 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
     }
     if (STORE) {
         uint4 q;
-        q.x = pack_bf16x2(v[0].x, v[0].y); q.y = pack_bf16x2(v[1].x, v[1].y);
-        q.z = pack_bf16x2(v[2].x, v[2].y); q.w = pack_bf16x2(v[3].x, v[3].y);
+        q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
+        q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
         st_stream(yr + c, q);
     }
     if (LSE && red_kind != FC_RED_ROW_LOGSUMEXP) {
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
 #pragma unroll
             for (int g = 0; g < kGroup; ++g) {
                 const int c = c0 + 32 * g;
-                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, p.red_kind, run_m, run_s);
+                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, p.red_kind, p.is_f16 != 0, run_m, run_s);
             }
         }
         if (LSE && p.red_kind != FC_RED_ROW_LOGSUMEXP) {
@@ -326,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
 
 // Recognise [bias | affine]? -> [relu | gelu]? -> [add tensor]? and fill the fast-path parameters.
 static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, bool* res) {
-    if (p.x_dt != FC_BF16 || (p.y && p.y_dt != FC_BF16)) return false;
+    if (p.x_dt == FC_F32 || (p.y && p.y_dt != p.x_dt)) return false;
     if (p.N % 8 != 0 || p.N > 24576 || p.M >= 0x7fffffffLL) return false;
     if ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y)) & 15) return false;
     int i = 0;
@@ -345,7 +347,7 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
         ++i;
     }
     if (i < p.ops.n && p.ops.op[i].kind == FC_OP_ADD_TENSOR) {
-        if (p.ops.op[i].dt0 != FC_BF16 || (reinterpret_cast<uintptr_t>(p.ops.op[i].p0) & 15)) return false;
+        if (p.ops.op[i].dt0 != p.x_dt || (reinterpret_cast<uintptr_t>(p.ops.op[i].p0) & 15)) return false;
         *res = true;
         f->res = (const uint4*) p.ops.op[i].p0;
         ++i;
@@ -353,6 +355,7 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
     if (i != p.ops.n) return false;
     f->x = (const uint4*) p.x; f->y = (uint4*) p.y; f->lse = p.red; f->M = p.M; f->N = (int) p.N;
     f->red_kind = p.reduce;
+    f->is_f16 = p.x_dt == FC_F16;
     return true;
 }
 

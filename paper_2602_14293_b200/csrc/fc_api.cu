@@ -90,7 +90,8 @@ fc_status get_device(DeviceInfo** out, int* dev_out = nullptr) {
     return FC_OK;
 }
 
-size_t dt_size(int dt) { return dt == FC_BF16 ? 2 : 4; }
+size_t dt_size(int dt) { return dt == FC_F32 ? 4 : 2; }
+bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16; }
 
 // ------------------------------------------------------------------------------- validation
 struct Plan {
@@ -112,7 +113,7 @@ bool contiguous(const fc_tensor& t) {
 
 fc_status check_tensor(const fc_tensor& t, const char* what, int dtype_or_any, int rank, const long long* shape) {
     if (!t.ptr) return fail(FC_ERR_NULL, "%s: null pointer", what);
-    if (t.dtype != FC_F32 && t.dtype != FC_BF16) return fail(FC_ERR_INVALID_SPEC, "%s: unknown dtype %d", what, t.dtype);
+    if (!dt_valid(t.dtype)) return fail(FC_ERR_INVALID_SPEC, "%s: unknown dtype %d", what, t.dtype);
     if (dtype_or_any >= 0 && t.dtype != dtype_or_any) return fail(FC_ERR_INVALID_SPEC, "%s: dtype %d, expected %d", what, t.dtype, dtype_or_any);
     if (t.rank != rank) return fail(FC_ERR_SHAPE, "%s: rank %d, expected %d", what, t.rank, rank);
     for (int i = 0; i < rank; ++i)
@@ -127,7 +128,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (s->struct_size != sizeof(fc_chain_spec)) return fail(FC_ERR_INVALID_SPEC, "struct_size %u, expected %zu", s->struct_size, sizeof(fc_chain_spec));
     if (s->version != FC_VERSION) return fail(FC_ERR_INVALID_SPEC, "version %u, expected %d", s->version, FC_VERSION);
     if (s->producer < 0 || s->producer > FC_PROD_CONV2D_NHWC) return fail(FC_ERR_INVALID_SPEC, "unknown producer %d", s->producer);
-    if ((s->in_dtype != FC_F32 && s->in_dtype != FC_BF16) || (s->out_dtype != FC_F32 && s->out_dtype != FC_BF16))
+    if (!dt_valid(s->in_dtype) || !dt_valid(s->out_dtype))
         return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
     if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
     if (s->reduce < 0 || s->reduce > FC_RED_ROW_MEAN) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
@@ -177,8 +178,8 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             }
             break;
         default:
-            if (s->in_dtype != FC_BF16 || s->reduce != FC_RED_GLOBAL_AVGPOOL || s->store_main)
-                return fail(FC_ERR_UNSUPPORTED, "conv supports bf16 input with GLOBAL_AVGPOOL and store_main = 0");
+            if (s->in_dtype == FC_F32 || s->reduce != FC_RED_GLOBAL_AVGPOOL || s->store_main)
+                return fail(FC_ERR_UNSUPPORTED, "conv supports bf16 / fp16 input with GLOBAL_AVGPOOL and store_main = 0");
             if (s->stride > 8) return fail(FC_ERR_UNSUPPORTED, "conv supports stride <= 8");
             if (s->pad >= s->R || s->pad >= s->S || s->R > 16 || s->S > 16) return fail(FC_ERR_UNSUPPORTED, "conv supports pad < R,S <= 16");
             plan->kind = Plan::TC_CONV;
@@ -212,7 +213,7 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         const long long sa[2] = {s->M, s->K}, sb[2] = {s->N, s->K};
         if ((st = check_tensor(in[0], "inputs[0] (A)", s->in_dtype, 2, sa))) return st;
         if ((st = check_tensor(in[1], "inputs[1] (B)", s->in_dtype, 2, sb))) return st;
-        if (s->in_dtype == FC_BF16) {
+        if (s->in_dtype != FC_F32) {
             if (s->K % 8) return fail(FC_ERR_ALIGNMENT, "bf16 GEMM needs K %% 8 == 0 (K = %lld)", (long long) s->K);
             if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr)) & 15)
                 return fail(FC_ERR_ALIGNMENT, "bf16 GEMM operands must be 16-byte aligned");
@@ -315,12 +316,12 @@ size_t softmax_workspace_bytes(long long M, long long N) {
     return counters + (size_t) M * tiles_n * sizeof(float2);
 }
 
-fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long cols, int box_rows) {
+fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long cols, int box_rows, int dt = FC_BF16) {
     const cuuint64_t dims[2] = {(cuuint64_t) cols, (cuuint64_t) rows};
     const cuuint64_t strides[1] = {(cuuint64_t) cols * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t) box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+    CUresult r = g_encode_tiled(tm, dt == FC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d (rows %lld cols %lld)", (int) r, rows, cols);
@@ -335,7 +336,7 @@ fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr
     const int upper[2] = {(int) (s->pad - (s->S - 1)), (int) (s->pad - (s->R - 1))};
     // base pixels advance by the convolution stride along w and h
     const cuuint32_t estr[4] = {1, (cuuint32_t) s->stride, (cuuint32_t) s->stride, 1};
-    CUresult r = g_encode_im2col(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper,
+    CUresult r = g_encode_im2col(tm, s->in_dtype == FC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper,
                                  64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeIm2col failed with CUresult %d", (int) r);
@@ -391,6 +392,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             memset(&p, 0, sizeof(p));
             p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
             p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+            p.in_dt = spec->in_dtype;
             p.out = plan.main_index >= 0 ? outputs[plan.main_index].ptr : nullptr; p.out_dt = spec->out_dtype;
             p.red = plan.red_index >= 0 ? (float*) outputs[plan.red_index].ptr : nullptr;
             p.status = dev->status;
@@ -413,8 +415,8 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 if ((e = cudaMemsetAsync(p.counters, 0, counters, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             }
             CUtensorMap tmA, tmB;
-            if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128))) return st;
-            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2))) return st;   // each CTA of a pair loads half
+            if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }
@@ -428,6 +430,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.OW = (int) ((spec->W + 2 * spec->pad - spec->S) / spec->stride + 1);
             p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
             p.group_m = 1;
+            p.in_dt = spec->in_dtype;
             p.inv_hw = 1.0f / (float) (p.OH * p.OW);
             p.out = outputs[plan.red_index].ptr; p.out_dt = FC_F32;
             p.status = dev->status;
@@ -436,7 +439,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             if ((e = cudaMemsetAsync(p.out, 0, (size_t) spec->batch * spec->Cout * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;
             if ((st = encode_im2col(&tmA, spec, inputs[0].ptr))) return st;
-            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn / 2))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn / 2, spec->in_dtype))) return st;
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }
@@ -695,14 +698,15 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
     const long long panels = (spec->M + 127) / 128;
     const size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
     p.group_m = 1;
+    p.in_dt = spec->in_dtype;
     p.counters = (unsigned int*) scratch;
     p.stats = (float2*) ((char*) scratch + counters);
     // the array keeps the previous call's contents: the arrival counters must start at zero
     cudaError_t e = cudaMemsetAsync(p.counters, 0, counters, stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     CUtensorMap tmA, tmB;
-    if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128))) return st;
-    if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, kSoftmaxBN / 2))) return st;
+    if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
+    if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, kSoftmaxBN / 2, spec->in_dtype))) return st;
     int launches = 0;
     e = launch_gemm_tc(p, tmA, tmB, kSoftmaxBN, dev->num_sms, stream, &launches);
     g_launches.fetch_add((uint64_t) launches);

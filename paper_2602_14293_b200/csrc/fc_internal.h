@@ -68,6 +68,7 @@ struct TcParams {
     int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row logsumexp
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
     int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
+    int in_dt;                  // FC_BF16 or FC_F16: storage of both MMA operands
     void* out; int out_dt;      // mode 0/1/3: [M,N] bf16 or f32 (mode 3: may be null).  mode 2: f32 [batch,Cout] (pre-zeroed)
     float* red;                 // mode 3: row logsumexp [M]
     DevOps ops;

@@ -258,22 +258,23 @@ __device__ __forceinline__ void apply_ops16(float (&v)[16], const DevOps& ops, c
 // 16 fp32 values of one row -> global memory as bf16 or fp32 (vector stores when aligned and in range)
 __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, const float (&v)[16], long long m,
                                         long long n0, long long N) {
-    if (out_dt == FC_BF16) {
+    if (out_dt != FC_F32) {
+        const bool f16 = out_dt == FC_F16;
         unsigned short* o = (unsigned short*) out + m * N + n0;
         if (vec_ok && n0 + 16 <= N) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 uint4 w;
-                w.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
-                w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
-                w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
-                w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+                w.x = pack16x2(v[8 * q + 0], v[8 * q + 1], f16);
+                w.y = pack16x2(v[8 * q + 2], v[8 * q + 3], f16);
+                w.z = pack16x2(v[8 * q + 4], v[8 * q + 5], f16);
+                w.w = pack16x2(v[8 * q + 6], v[8 * q + 7], f16);
                 reinterpret_cast<uint4*>(o)[q] = w;
             }
         } else {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (n0 + j < N) o[j] = (unsigned short) (pack_bf16x2(v[j], 0.0f) & 0xffffu);
+                if (n0 + j < N) o[j] = (unsigned short) (pack16x2(v[j], 0.0f, f16) & 0xffffu);
         }
     } else {
         float* o = (float*) out + m * N + n0;
@@ -378,7 +379,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (leader && lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, BN);
+            const uint32_t idesc = ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_F16 ? 0u : 1u);
             uint32_t it = 0, tile_iter = 0;
             bool ok = true;
             for (int t = cluster_id; t < total_tiles && ok; t += num_clusters, ++tile_iter) {

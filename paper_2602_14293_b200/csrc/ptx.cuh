@@ -113,11 +113,12 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
     return d;
 }
 
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, both operands K-major, dense.
-__host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n) {
+// Instruction descriptor for kind::f16: bf16 x bf16 (ab_format 1) or fp16 x fp16 (ab_format 0) -> fp32,
+// both operands K-major, dense.
+__host__ __device__ constexpr uint32_t idesc_f16kind_f32(int m, int n, uint32_t ab_format) {
     return (1u << 4)                      // D format  = f32
-           | (1u << 7)                    // A format  = bf16
-           | (1u << 10)                   // B format  = bf16
+           | (ab_format << 7)             // A format
+           | (ab_format << 10)            // B format
            | ((uint32_t) (n >> 3) << 17)  // N / 8
            | ((uint32_t) (m >> 4) << 24); // M / 16
 }

@@ -375,3 +375,33 @@ def test_run_host_chunk_pipeline_matches_device_path(fc, orc):
                 assert torch.allclose(a.cpu(), b, rtol=1e-5, atol=1e-6)
             else:
                 assert torch.equal(a.cpu(), b), ch.name
+
+
+# ------------------------------------------------------------------ fp16 storage (the paper's kernels store fp16)
+def _as_f16(ch):
+    rec = tuple((t, "f16" if d == "bf16" else d, sh, dist, a, b) for t, d, sh, dist, a, b in ch.input_recipe)
+    return replace(ch, in_dtype="f16", out_dtype="f16" if ch.out_dtype == "bf16" else ch.out_dtype, input_recipe=rec)
+
+
+def test_fp16_gemm_small_integers_bit_exact(fc, orc):
+    for M, N, K in [(256, 512, 128), (200, 264, 72), (384, 768, 1024)]:
+        ch = _as_f16(wl.with_integer_inputs(_plain_gemm(M, N, K), -4, 4))
+        ins = wl.make_inputs(ch, 5)
+        ref = orc.run_chain(ch, ins)["main"]
+        outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+        fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+        fc.fc_get_async_status()
+        assert np.array_equal(util.to_f64(outs[0]), ref)
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_fp16_chains(fc, orc, seed):
+    run_and_check(fc, orc, _as_f16(wl.gemm_bias_gelu_scale_clamp(512, 1024, 512, "var")), seed)
+    run_and_check(fc, orc, _as_f16(wl.gemm_bias_gelu_scale_clamp(200, 264, 72, "var")), seed)
+    outs, _, _ = run_and_check(fc, orc, _as_f16(wl.gemm_softmax(300, 1000, 136, "var")), seed)
+    assert float((outs[0].float().sum(1) - 1).abs().max()) <= 1e-3
+    run_and_check(fc, orc, _as_f16(wl.gemm_bias_scale_lse(256, 2048, 256, "var", True)), seed)
+    run_and_check(fc, orc, _as_f16(wl.conv_bias_relu_avgpool(batch=3, H=14, W=14, Cin=64, Cout=128)), seed)
+    run_and_check(fc, orc, _as_f16(wl.affine_gelu_residual_lse(65, 4096)), seed)
+    run_and_check(fc, orc, _as_f16(wl.affine_gelu_residual_lse(9, 1001)), seed)
+    run_and_check(fc, orc, replace(_as_f16(wl.affine_gelu_residual_lse(33, 2048)), reduce="row_mean"), seed)

@@ -56,7 +56,7 @@ def _random_chain(r):
     kind = r.choice(["ew", "gemm", "gemm", "conv", "gemm_f32"])
     if kind == "ew":
         M, N = int(r.integers(1, 70)), int(r.choice([8, 24, 200, 1000, 1024, 4096, 333]))
-        dt = str(r.choice(["bf16", "f32"]))
+        dt = str(r.choice(["bf16", "f32", "f16"]))
         rec = (("x", dt, (M, N), "normal", 0.0, 1.0), ("v0", dt, (N,), "normal", 1.0, 0.1), ("v1", "bf16", (N,), "normal", 0.0, 0.1),
                ("t", dt, (M, N), "normal", 0.0, 1.0))
         red = str(r.choice(["none", "row_logsumexp"]))
@@ -100,9 +100,9 @@ def test_random_chain(fc, orc, seed):
     for (name, _, _), t in zip(wl.output_shapes(ch), outs):
         got, want = util.to_f64(t), ref[name]
         what = f"seed {seed}: {ch.producer} {[o[0] for o in ch.ops]} reduce={ch.reduce} {name}"
-        if t.dtype == torch.bfloat16:
+        if t.dtype in (torch.bfloat16, torch.float16):
             # magnitudes are not O(1) for every random op list: scale the absolute mean bound with the output's rms
             scale = max(1.0, float(np.sqrt(np.mean(want * want))))
-            util.check_bf16(got / scale, want / scale, what)
+            (util.check_bf16 if t.dtype == torch.bfloat16 else util.check_f16)(got / scale, want / scale, what)
         else:
             util.check_f32(got, want, what)

@@ -30,6 +30,15 @@ def test_widen_bf16_all_patterns(orc):
     assert ok.all()
 
 
+def test_widen_f16_all_patterns(orc):
+    bits = np.arange(65536, dtype=np.uint16)
+    got = orc.widen(bits.view(np.float16))
+    want = torch.from_numpy(bits.view(np.int16)).view(torch.float16).to(torch.float64).numpy()
+    ok = (got == want) | (np.isnan(got) & np.isnan(want))
+    assert ok.all()
+    assert orc.widen(np.array([1.0, -2.5, 65504.0, 2.0 ** -24], np.float16)).tolist() == [1.0, -2.5, 65504.0, 2.0 ** -24]
+
+
 def test_widen_f32_exact(orc):
     a = np.array([0.1, -3.5, 1e-40, 3e38, -0.0], dtype=np.float32)
     assert np.array_equal(orc.widen(a), a.astype(np.float64))

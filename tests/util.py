@@ -43,10 +43,28 @@ def check_bf16(got: np.ndarray, ref: np.ndarray, what=""):
     return mx, mean_abs
 
 
+def check_f16(got: np.ndarray, ref: np.ndarray, what=""):
+    """fp16 outputs (the benchmark states no tolerance for them): one round-to-nearest to an 11-bit
+    significand is 2^-11 = 4.9e-4 relative, so max relative error <= 2e-3 (same floor as for bf16)
+    and mean absolute error <= 2.5e-4, i.e. the bf16 bounds tightened by the 8x finer grid."""
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite values in the output"
+    err = np.abs(got - ref)
+    floor = 0.1 * float(np.sqrt(np.mean(ref * ref)))
+    rel = err / np.maximum(np.abs(ref), max(floor, 1e-30))
+    mx, mean_abs = float(rel.max()), float(err.mean())
+    assert mx <= 2e-3, f"{what}: max rel err {mx:.4g} at {np.unravel_index(rel.argmax(), rel.shape)}"
+    mean_bound = 2.5e-4 if ref.size >= 256 else 2.5e-4 * max(1.0, float(np.abs(ref).max()))
+    assert mean_abs <= mean_bound, f"{what}: mean abs err {mean_abs:.4g}"
+    return mx, mean_abs
+
+
 def check(got_t: torch.Tensor, ref: np.ndarray, what=""):
     got = to_f64(got_t)
     if got_t.dtype == torch.bfloat16:
         return check_bf16(got, ref, what)
+    if got_t.dtype == torch.float16:
+        return check_f16(got, ref, what)
     return check_f32(got, ref, what)
 
 
