@@ -45,6 +45,10 @@
  * are bounded; if one expires the kernel records FC_ERR_TIMEOUT in a device status word, skips its
  * remaining stores and exits; fc_get_async_status reports it.
  *
+ * Testing aid.  With the environment variable FC_INJECT_PANEL_STALL=1, GEMM_NT + ROW_SOFTMAX launches
+ * make their cross-tile wait expect an arrival that never comes: the bounded wait expires (about two
+ * seconds), nothing is stored, and fc_get_async_status returns FC_ERR_TIMEOUT; the device stays usable.
+ *
  * Threading.  fc_run may be called from several host threads.  The workspace set by
  * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM) must not
  * overlap on the device.

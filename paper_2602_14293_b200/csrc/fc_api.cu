@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -403,6 +404,12 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 const long long panel_bytes = 256LL * spec->K * 2;
                 long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
                 p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
+            }
+            if (p.mode == 1) {
+                // testing only: FC_INJECT_PANEL_STALL=1 makes every panel wait expect one arrival that never
+                // comes, so that the bounded wait expires and the call ends with FC_ERR_TIMEOUT
+                const char* inj = getenv("FC_INJECT_PANEL_STALL");
+                p.expect_extra = inj && inj[0] == '1' ? 1 : 0;
             }
             if (p.mode == 1 || p.mode == 3) {
                 const size_t need = softmax_workspace_bytes(spec->M, spec->N);

@@ -79,6 +79,7 @@ struct TcParams {
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
     int* status;                // device status word
+    int expect_extra;           // mode 1, testing only: arrivals the panel wait expects beyond those that will come
 };
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                            int bn, int num_sms, cudaStream_t stream, int* launches);

@@ -602,7 +602,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::red_release_gpu_add(&p.counters[mb], 1u);
                     const unsigned long long t0 = ptx::globaltimer();
                     unsigned spins = 0;
-                    while (ptx::ld_acquire_gpu(&p.counters[mb]) < (unsigned) tiles_n) {
+                    while (ptx::ld_acquire_gpu(&p.counters[mb]) < (unsigned) (tiles_n + p.expect_extra)) {
                         if ((++spins & 63u) == 0) {
                             if (*abort_flag) break;
                             if (ptx::globaltimer() - t0 > kWaitLimitNs) {
