@@ -168,6 +168,29 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes);
 fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
 
 /*
+ * Optional extra scratch.  A tensor-core chain (GEMM_NT or CONV2D_NHWC in bf16 / fp16) whose output
+ * tiles do not fill the last round of SM pairs -- few rows, the regime of the paper's batch-sized
+ * linear layers (appendix GEMM listing, which splits K and adds fp32 partials through a workspace), or
+ * a ragged last round -- runs faster when those tiles are cut along K: the slices park fp32 partial
+ * accumulators in scratch and the slice that finishes last adds them up in tensor memory and runs the
+ * epilogue.  fc_workspace_size_split reports the workspace size that allows this for `spec`
+ * (fc_workspace_size plus a fixed region of about 20 MB; 0 for chains that never split).  A smaller
+ * workspace, or none where none is required, is not an error: fc_run then never splits.  Results are
+ * the same up to fp32 summation order.
+ */
+fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
+
+/*
+ * Writes a one-line description of how fc_run would execute `spec` on the current device with the
+ * workspace registered now: "kernel=ew_rowreduce", "kernel=gemm_f32", or
+ * "kernel=gemm_tc mode=<0 store|1 softmax|2 conv+pool|3 logsumexp> bn=<tile width> tiles=<256 x bn tiles>
+ * pairs=<CTA pairs launched> split=<slices per split tile, 1 = none> split_tiles=<tiles that are split>
+ * split_kb=<64-wide k-blocks per parking slice>".  `text` is a caller-owned HOST buffer of `capacity`
+ * bytes (truncated if too small).  Launches nothing.  For logs and tests; the format may gain fields.
+ */
+fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacity);
+
+/*
  * GEMM_NT + ROW_SOFTMAX for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a deployment convenience of this library.)
  *

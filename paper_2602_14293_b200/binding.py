@@ -75,6 +75,10 @@ def lib():
         L.fc_run_softmax_static_scratch.restype = ctypes.c_int
         L.fc_workspace_size.argtypes = [ps, ctypes.POINTER(ctypes.c_size_t)]
         L.fc_workspace_size.restype = ctypes.c_int
+        L.fc_workspace_size_split.argtypes = [ps, ctypes.POINTER(ctypes.c_size_t)]
+        L.fc_workspace_size_split.restype = ctypes.c_int
+        L.fc_describe_plan.argtypes = [ps, ctypes.c_char_p, ctypes.c_size_t]
+        L.fc_describe_plan.restype = ctypes.c_int
         L.fc_set_workspace.argtypes = [ctypes.c_void_p, ctypes.c_size_t]
         L.fc_set_workspace.restype = ctypes.c_int
         L.fc_get_async_status.argtypes = [ctypes.c_void_p]
@@ -223,6 +227,23 @@ def fc_workspace_size(spec) -> int:
     return int(n.value)
 
 
+def fc_workspace_size_split(spec) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().fc_workspace_size_split(ctypes.byref(spec), ctypes.byref(n)), "fc_workspace_size_split")
+    return int(n.value)
+
+
+def fc_describe_plan(spec) -> dict:
+    """How fc_run would execute `spec` now, as a dict ({"kernel": ..., "split": ..., ...}; numbers as int)."""
+    buf = ctypes.create_string_buffer(256)
+    _check(lib().fc_describe_plan(ctypes.byref(spec), buf, len(buf)), "fc_describe_plan")
+    out = {}
+    for item in buf.value.decode().split():
+        k, v = item.split("=")
+        out[k] = int(v) if v.lstrip("-").isdigit() else v
+    return out
+
+
 def fc_set_workspace(buf: Optional[torch.Tensor]) -> None:
     if buf is None:
         _check(lib().fc_set_workspace(None, 0), "fc_set_workspace")
@@ -266,8 +287,8 @@ def output_tensors(chain, device="cuda", pinned=False) -> List[torch.Tensor]:
 
 
 def ensure_workspace(spec) -> None:
-    """Register a torch-owned workspace large enough for `spec` on the current device."""
-    need = fc_workspace_size(spec)
+    """Register a torch-owned workspace large enough for `spec` (split tiles included) on the current device."""
+    need = max(fc_workspace_size(spec), fc_workspace_size_split(spec))
     if need == 0:
         return
     dev = torch.cuda.current_device()

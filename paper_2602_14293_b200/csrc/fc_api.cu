@@ -33,6 +33,7 @@ struct DeviceInfo {
     int* status = nullptr;
     void* workspace = nullptr;
     size_t workspace_bytes = 0;
+    uint64_t counter_layout = 0;   // which counter layout the workspace was last left clean for (0: none)
 };
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_mu;
@@ -310,11 +311,42 @@ void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
 
 constexpr int kSoftmaxBN = 256;
 
+// arrival counters and departure counters, one of each per 128-row panel
+size_t panel_counter_bytes(long long M) {
+    const long long panels = (M + 127) / 128;
+    return ((size_t) panels * 4 + 255) / 256 * 256;
+}
+
 size_t softmax_workspace_bytes(long long M, long long N) {
-    const long long tiles_n = (N + kSoftmaxBN - 1) / kSoftmaxBN, panels = (M + 127) / 128;
-    size_t counters = (size_t) panels * 4;
-    counters = (counters + 255) / 256 * 256;
-    return counters + (size_t) M * tiles_n * sizeof(float2);
+    const long long tiles_n = (N + kSoftmaxBN - 1) / kSoftmaxBN;
+    return 2 * panel_counter_bytes(M) + (size_t) M * tiles_n * sizeof(float2);
+}
+
+// The part of the caller's workspace behind the row-reduction statistics serves split tiles; without it
+// (no workspace, or a smaller one) the tensor-core kernels simply never split.
+size_t split_workspace_offset(size_t reduction_bytes) { return (reduction_bytes + 255) / 256 * 256; }
+
+void attach_split_scratch(const DeviceInfo* dev, size_t reduction_bytes, TcParams* p) {
+    const size_t off = split_workspace_offset(reduction_bytes);
+    if (!dev->workspace || dev->workspace_bytes < off + kTcSplitBytes) return;
+    p->split_counters = (unsigned int*) ((char*) dev->workspace + off);
+    p->split_ws = (float4*) ((char*) dev->workspace + off + kTcSplitCounterBytes);
+}
+
+// The kernels hand every counter back at zero, so the counters are cleared on the stream only when
+// the workspace may hold something else where this launch keeps them: after fc_set_workspace, after a
+// launch with another layout (different panel count, different place of the split counters), and after
+// a launch that ended in a timeout.  `p` has its counter pointers set already.
+cudaError_t clear_counters_if_needed(DeviceInfo* dev, const TcParams& p, size_t panel_bytes, cudaStream_t stream) {
+    const uint64_t split_off = p.split_counters ? (uint64_t) ((char*) p.split_counters - (char*) dev->workspace) + 1 : 0;
+    const uint64_t key = ((uint64_t) panel_bytes << 32) ^ split_off ^ (1ull << 63);
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (dev->counter_layout == key) return cudaSuccess;
+    cudaError_t e = cudaSuccess;
+    if (panel_bytes && (e = cudaMemsetAsync(p.counters, 0, 2 * panel_bytes, stream)) != cudaSuccess) return e;
+    if (p.split_counters && (e = cudaMemsetAsync(p.split_counters, 0, kTcSplitCounterBytes, stream)) != cudaSuccess) return e;
+    dev->counter_layout = key;
+    return cudaSuccess;
 }
 
 fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long cols, int box_rows, int dt = FC_BF16) {
@@ -411,16 +443,18 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 const char* inj = getenv("FC_INJECT_PANEL_STALL");
                 p.expect_extra = inj && inj[0] == '1' ? 1 : 0;
             }
+            size_t panel_bytes = 0;
             if (p.mode == 1 || p.mode == 3) {
                 const size_t need = softmax_workspace_bytes(spec->M, spec->N);
-                const long long panels = (spec->M + 127) / 128;
                 if (!dev->workspace || dev->workspace_bytes < need)
                     return fail(FC_ERR_WORKSPACE, "this row reduction needs a %zu-byte workspace (fc_set_workspace); have %zu", need, dev->workspace_bytes);
-                size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
+                panel_bytes = panel_counter_bytes(spec->M);
                 p.counters = (unsigned int*) dev->workspace;
-                p.stats = (float2*) ((char*) dev->workspace + counters);
-                if ((e = cudaMemsetAsync(p.counters, 0, counters, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+                p.departed = (unsigned int*) ((char*) dev->workspace + panel_bytes);
+                p.stats = (float2*) ((char*) dev->workspace + 2 * panel_bytes);
             }
+            attach_split_scratch(dev, p.mode == 1 || p.mode == 3 ? softmax_workspace_bytes(spec->M, spec->N) : 0, &p);
+            if ((e = clear_counters_if_needed(dev, p, panel_bytes, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
@@ -444,6 +478,8 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             build_ops(spec, inputs, &p.ops);
             const int bn = spec->Cout <= 128 ? 128 : 256;
             if ((e = cudaMemsetAsync(p.out, 0, (size_t) spec->batch * spec->Cout * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+            attach_split_scratch(dev, 0, &p);
+            if ((e = clear_counters_if_needed(dev, p, 0, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;
             if ((st = encode_im2col(&tmA, spec, inputs[0].ptr))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn / 2, spec->in_dtype))) return st;
@@ -609,6 +645,50 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     return FC_OK;
 }
 
+fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes) {
+    Plan plan;
+    fc_status st;
+    if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
+    if ((st = validate_spec(spec, &plan))) return st;
+    const bool tc = plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_CONV;
+    const size_t red = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N) : 0;
+    *bytes = tc ? split_workspace_offset(red) + kTcSplitBytes : 0;
+    return FC_OK;
+}
+
+fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacity) {
+    Plan plan;
+    fc_status st;
+    if (!text || capacity == 0) return fail(FC_ERR_NULL, "text is null or has no room");
+    if ((st = validate_spec(spec, &plan))) return st;
+    if (plan.kind == Plan::EW) { snprintf(text, capacity, "kernel=ew_rowreduce"); return FC_OK; }
+    if (plan.kind == Plan::GEMM_F32) { snprintf(text, capacity, "kernel=gemm_f32"); return FC_OK; }
+    DeviceInfo* dev;
+    if ((st = get_device(&dev))) return st;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    int bn;
+    size_t red = 0;
+    if (plan.kind == Plan::TC_CONV) {
+        p.mode = 2;
+        p.Cin = (int) spec->Cin; p.R = (int) spec->R; p.S = (int) spec->S;
+        p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
+        bn = spec->Cout <= 128 ? 128 : 256;
+    } else {
+        p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
+        p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+        bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
+        if (p.mode == 1 || p.mode == 3) red = softmax_workspace_bytes(spec->M, spec->N);
+    }
+    attach_split_scratch(dev, red, &p);
+    TcPlan tp;
+    cudaError_t e = plan_gemm_tc(p, bn, dev->num_sms, &tp);
+    if (e != cudaSuccess) return cuda_fail(e, "planning");
+    snprintf(text, capacity, "kernel=gemm_tc mode=%d bn=%d tiles=%d pairs=%d split=%d split_tiles=%d split_kb=%d", p.mode, tp.bn,
+             tp.tiles, tp.pairs, tp.split, tp.split_tiles, tp.split_kb);
+    return FC_OK;
+}
+
 fc_status fc_set_workspace(void* dev_ptr, size_t bytes) {
     if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255)) return fail(FC_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
     DeviceInfo* dev;
@@ -617,6 +697,7 @@ fc_status fc_set_workspace(void* dev_ptr, size_t bytes) {
     std::lock_guard<std::mutex> lk(g_mu);
     dev->workspace = dev_ptr;
     dev->workspace_bytes = dev_ptr ? bytes : 0;
+    dev->counter_layout = 0;
     return FC_OK;
 }
 
@@ -629,6 +710,10 @@ fc_status fc_get_async_status(void* cuda_stream) {
     int word = 0;
     if ((e = cudaMemcpy(&word, dev->status, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy status");
     if (word != 0) {
+        {
+            std::lock_guard<std::mutex> lk(g_mu);
+            dev->counter_layout = 0;   // the launch that gave up may have left counters behind
+        }
         const int zero = 0;
         if ((e = cudaMemcpy(dev->status, &zero, sizeof(int), cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy status");
         return fail((fc_status) word, "a bounded device-side wait expired");
@@ -702,14 +787,14 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
     p.out = outputs[plan.main_index].ptr; p.out_dt = spec->out_dtype;
     p.status = dev->status;
     build_ops(spec, inputs, &p.ops);
-    const long long panels = (spec->M + 127) / 128;
-    const size_t counters = ((size_t) panels * 4 + 255) / 256 * 256;
+    const size_t counters = panel_counter_bytes(spec->M);
     p.group_m = 1;
     p.in_dt = spec->in_dtype;
     p.counters = (unsigned int*) scratch;
-    p.stats = (float2*) ((char*) scratch + counters);
-    // the array keeps the previous call's contents: the arrival counters must start at zero
-    cudaError_t e = cudaMemsetAsync(p.counters, 0, counters, stream);
+    p.departed = (unsigned int*) ((char*) scratch + counters);
+    p.stats = (float2*) ((char*) scratch + 2 * counters);
+    // the array keeps the previous call's contents: the arrival and departure counters must start at zero
+    cudaError_t e = cudaMemsetAsync(p.counters, 0, 2 * counters, stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     CUtensorMap tmA, tmB;
     if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;

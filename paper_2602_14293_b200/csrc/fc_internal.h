@@ -74,15 +74,32 @@ struct TcParams {
     DevOps ops;
     // mode 1
     float2* stats;              // [M][tiles_n] (max, sum) per tile
-    unsigned int* counters;     // [panels], zeroed before launch
+    unsigned int* counters;     // [panels] arrivals; zero at launch, left at zero by a launch that completes
+    unsigned int* departed;     // mode 1: [panels] tiles that have left the panel wait; same rule
     // mode 2
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
     int* status;                // device status word
     int expect_extra;           // mode 1, testing only: arrivals the panel wait expects beyond those that will come
+    // Split tiles (filled by the launcher when the scratch below is given and a split pays): tiles from
+    // split_from on are cut into `split` slices along K.
+    int split, split_from, split_kb;   // split_kb: k-blocks of each parking slice; the merging slice takes the rest
+    float4* split_ws;           // kTcSplitUnits slots of 2 x 128 x BN fp32, or null: never split
+    unsigned int* split_counters;   // kTcSplitUnits arrival counters (two per split tile); zero at launch, left at zero
 };
+// Scratch for split tiles: at most this many slice units per launch.
+constexpr int kTcSplitUnits = 80;
+constexpr size_t kTcSplitCounterBytes = 1024;
+constexpr size_t kTcSplitBytes = kTcSplitCounterBytes + (size_t) kTcSplitUnits * 2 * 128 * 256 * 4;
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                            int bn, int num_sms, cudaStream_t stream, int* launches);
 size_t gemm_tc_smem_bytes(int bn);
+
+// What launch_gemm_tc would do with `p` on the current device (no launch).
+struct TcPlan {
+    int bn, tiles, pairs;       // tile width, 256 x bn output tiles, CTA pairs launched
+    int split, split_tiles, split_kb;   // slices per split tile (1: none), tiles that are split, k-blocks per parking slice
+};
+cudaError_t plan_gemm_tc(const TcParams& p, int bn, int num_sms, TcPlan* plan);
 
 }  // namespace fc

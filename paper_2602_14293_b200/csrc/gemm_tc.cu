@@ -26,6 +26,17 @@
 // CTAs.  Two accumulator buffers in tensor memory let the epilogue of tile i overlap the main loop
 // of tile i+1.  Every wait is bounded: on expiry the CTA records FC_ERR_TIMEOUT in the status word,
 // stops storing and drains.
+//
+// Split tiles.  When the tiles do not fill the last round of pairs (or there are fewer tiles than pairs
+// at all: small-M GEMMs), the host cuts each tile of that round into `split` slices along K, one work
+// unit each, all in that one round.  Every slice but the last parks its fp32 accumulator rows in scratch
+// and bumps the tile's arrival counter; the last slice, which is given a few more k-blocks so that it
+// finishes when the parked rows are there, waits (bounded) for the counter, adds the parked rows into
+// its own accumulator in tensor memory and runs the epilogue as if it had done the whole tile.  The
+// slices that park never wait, and every pair's split unit is its last one, so the wait cannot cycle.
+//
+// Arrival counters (split tiles, row panels) are handed back at zero: whoever observes the final count
+// resets it, so a launch needs no memset as long as the previous one ran to completion.
 #include "dev_common.cuh"
 #include "ptx.cuh"
 
@@ -59,6 +70,7 @@ struct Ctrl {
     int abort;
     int epi_ok[2];  // outcome of the epilogue's accumulator wait, one slot per accumulator buffer
     int last;       // mode 3: this tile was the last of its row panel to publish
+    int merge_ok;   // split tiles: the merging slice saw every other slice arrive
 };
 static_assert(sizeof(Ctrl) <= 256, "control block");
 
@@ -96,6 +108,28 @@ __device__ __forceinline__ void tile_coords(int mode, int group_m, int t, int ti
         mb = t / tiles_n;  // panel-major: the tiles of one row panel are consecutive
         nb = t - mb * tiles_n;
     }
+}
+
+// Work unit -> (tile, range of k-blocks).  Units below split_from are whole tiles; above it every tile is
+// `split` consecutive units, one per slice of its k-blocks.
+struct Unit {
+    int tile, kb0, kb1, slice, nsl, v0;   // v0: index of the tile's first slice among the split units
+};
+__device__ __forceinline__ Unit unit_decode(int u, int split_from, int split, int split_kb, int num_kb) {
+    Unit w;
+    if (u < split_from || split <= 1) {
+        w.tile = u; w.kb0 = 0; w.kb1 = num_kb; w.slice = 0; w.nsl = 1; w.v0 = 0;
+    } else {
+        const int v = u - split_from;
+        const int ti = v / split;
+        w.tile = split_from + ti;
+        w.slice = v - ti * split;
+        w.nsl = split;
+        w.v0 = ti * split;
+        w.kb0 = w.slice * split_kb;                                   // split_kb k-blocks per parking slice,
+        w.kb1 = w.slice == split - 1 ? num_kb : w.kb0 + split_kb;     // the rest for the merging one
+    }
+    return w;
 }
 
 // Column sums over the 32 lanes of a warp for 32 columns held one per register: after the call
@@ -311,6 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int total_tiles = tiles_m * tiles_n;
     const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
     const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + BK - 1) / BK;
+    const int total_units = p.split > 1 ? p.split_from + (total_tiles - p.split_from) * p.split : total_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
@@ -341,9 +376,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
+            for (int u = cluster_id; u < total_units && ok; u += num_clusters) {
+                const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 int mb2, nb;
-                tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
+                tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
@@ -354,7 +390,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     oh = rem / p.OW;
                     ow = rem - oh * p.OW;
                 }
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                     if (!(ok = wait_bar(ptx::smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, p.status))) break;
                     const uint32_t full = ptx::mapa(ptx::smem_u32(&ctrl->full[s]), 0);   // the leader's barrier
@@ -382,12 +418,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t idesc = ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_F16 ? 0u : 1u);
             uint32_t it = 0, tile_iter = 0;
             bool ok = true;
-            for (int t = cluster_id; t < total_tiles && ok; t += num_clusters, ++tile_iter) {
+            for (int u = cluster_id; u < total_units && ok; u += num_clusters, ++tile_iter) {
+                const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
                 if (!(ok = wait_bar(ptx::smem_u32(&ctrl->tempty[buf]), aph ^ 1u, abort_flag, p.status))) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                     if (!(ok = wait_bar(ptx::smem_u32(&ctrl->full[s]), ph, abort_flag, p.status))) break;
                     ptx::tc_fence_after();
@@ -395,7 +432,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint64_t da = ptx::smem_desc_k128(sa), db = ptx::smem_desc_k128(sa + C::kABytes);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
-                        ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                        ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
                     ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);     // frees the stage in both CTAs
                 }
                 if (ok) ptx::tc_commit_pair(ptx::smem_u32(&ctrl->tfull[buf]), 3);   // accumulators ready in both CTAs
@@ -412,9 +449,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool out_vec = (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 && (p.N & 7) == 0;
         const uint32_t tempty_leader = ptx::mapa(ptx::smem_u32(&ctrl->tempty[0]), 0);
         uint32_t tile_iter = 0;
-        for (int t = cluster_id; t < total_tiles; t += num_clusters, ++tile_iter) {
+        for (int u = cluster_id; u < total_units; u += num_clusters, ++tile_iter) {
+            const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
             int mb2, nb;
-            tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, t, tiles_m, tiles_n, mb2, nb);
+            tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);
             const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;
@@ -441,6 +479,96 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t tacc = tmem_base + buf * BN + col_half + lane_addr;
             const long long m = (long long) mb * BM + row;
             const int n_half = n_tile + col_half;
+            // hands the accumulator buffer back to the leader's MMA thread
+            auto release_buf = [&]() {
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
+            };
+
+            if (w.nsl > 1) {
+                // Slice of a split tile.  Scratch layout per (slice, CTA): [warp 8][chunk][quad 4][lane 32] float4,
+                // so that every warp instruction moves 512 contiguous bytes.
+                constexpr size_t kSliceF4 = (size_t) BM * BN / 4;
+                const int ws = warp - 2;
+                unsigned int* cnt = &p.split_counters[(w.v0 / w.nsl) * 2 + (int) cta_rank];
+                if (w.slice != w.nsl - 1) {
+                    float4* mine = p.split_ws + ((size_t) (w.v0 + w.slice) * 2 + cta_rank) * kSliceF4 + (size_t) ws * kChunks * 128 + lane;
+#pragma unroll 1
+                    for (int c = 0; c < kChunks; c += 2) {
+                        uint32_t ra[16], rb[16];
+                        ptx::tmem_ld_32x16_async(tacc + c * 16, ra);
+                        ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
+                        ptx::tmem_wait_ld(ra);
+                        ptx::tmem_wait_ld(rb);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            __stcg(mine + (c * 4 + j) * 32, make_float4(__uint_as_float(ra[4 * j]), __uint_as_float(ra[4 * j + 1]), __uint_as_float(ra[4 * j + 2]), __uint_as_float(ra[4 * j + 3])));
+                            __stcg(mine + ((c + 1) * 4 + j) * 32, make_float4(__uint_as_float(rb[4 * j]), __uint_as_float(rb[4 * j + 1]), __uint_as_float(rb[4 * j + 2]), __uint_as_float(rb[4 * j + 3])));
+                        }
+                    }
+                    __threadfence();
+                    ptx::bar_sync(1, kEpiThreads);
+                    if (et == 0) ptx::red_release_gpu_add(cnt, 1u);
+                    release_buf();
+                    continue;
+                }
+                // the merging slice: wait (bounded) until the others have parked their rows
+                if (et == 0) {
+                    const unsigned long long t0 = ptx::globaltimer();
+                    unsigned spins = 0;
+                    bool ok = true;
+                    while (ptx::ld_acquire_gpu(cnt) < (unsigned) w.nsl - 1u) {
+                        if ((++spins & 63u) == 0) {
+                            if (*abort_flag) { ok = false; break; }
+                            if (ptx::globaltimer() - t0 > kWaitLimitNs) {
+                                *abort_flag = 1;
+                                atomicExch(p.status, kStatusTimeout);
+                                ok = false;
+                                break;
+                            }
+                        }
+                    }
+                    if (ok) *cnt = 0u;   // nobody else touches it in this launch: the next launch finds zero
+                    ctrl->merge_ok = ok;
+                    __threadfence();
+                }
+                ptx::bar_sync(1, kEpiThreads);
+                if (!*(volatile int*) &ctrl->merge_ok) break;
+                // add the other slices' rows into the accumulator, four chunks of loads in flight
+#pragma unroll 1
+                for (int c0 = 0; c0 < kChunks; c0 += 4) {
+                    float4 acc[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    for (int q = 0; q < w.nsl; ++q) {
+                        if (q == w.slice) continue;
+                        const float4* src = p.split_ws + ((size_t) (w.v0 + q) * 2 + cta_rank) * kSliceF4 + (size_t) ws * kChunks * 128 + lane + c0 * 128;
+                        float4 t[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) t[i] = __ldcg(src + i * 32);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            acc[i].x += t[i].x; acc[i].y += t[i].y; acc[i].z += t[i].z; acc[i].w += t[i].w;
+                        }
+                    }
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t r[16];
+                        ptx::tmem_ld_32x16_async(tacc + (c0 + cc) * 16, r);
+                        ptx::tmem_wait_ld(r);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + acc[cc * 4 + j].x);
+                            r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + acc[cc * 4 + j].y);
+                            r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + acc[cc * 4 + j].z);
+                            r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + acc[cc * 4 + j].w);
+                        }
+                        ptx::tmem_st_32x16(tacc + (c0 + cc) * 16, r);
+                    }
+                }
+                ptx::tmem_wait_st();
+            }
 
             if constexpr (MODE == 0) {
                 uint32_t ra[16], rb[16];
@@ -515,7 +643,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
                 if (et == 0) {
-                    ctrl->last = ptx::atom_acq_rel_gpu_add(&p.counters[mb], 1u) == (unsigned) tiles_n - 1u;
+                    const bool last = ptx::atom_acq_rel_gpu_add(&p.counters[mb], 1u) == (unsigned) tiles_n - 1u;
+                    if (last) p.counters[mb] = 0u;   // left at zero for the next launch
+                    ctrl->last = last;
                     __threadfence();
                 }
                 ptx::bar_sync(1, kEpiThreads);
@@ -613,6 +743,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                     __threadfence();
+                    // the tile that leaves the wait last puts both counters back to zero for the next launch
+                    if (*abort_flag == 0 && ptx::atom_acq_rel_gpu_add(&p.departed[mb], 1u) == (unsigned) tiles_n - 1u) {
+                        p.counters[mb] = 0u;
+                        p.departed[mb] = 0u;
+                    }
                 }
                 ptx::bar_sync(1, kEpiThreads);
                 const bool store = *abort_flag == 0;
@@ -679,10 +814,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
-            // hand the accumulator buffer back to the leader's MMA thread
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
+            release_buf();
         }
     }
 
@@ -702,7 +834,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 template <int BN, int MODE>
-cudaError_t launch_one(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int num_sms, cudaStream_t stream) {
+cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int num_sms, cudaStream_t stream,
+                       TcPlan* plan) {
     static int max_clusters[64] = {0};   // per device, filled on first use
     const int smem = Cfg<BN>::kSmemBytes;
     auto kernel = gemm_tc_kernel<BN, MODE>;
@@ -728,29 +861,72 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap& tmA, const CUtensor
         if (e != cudaSuccess) return e;
         max_clusters[dev] = n > 0 ? n : 1;
     }
-    const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * ((p.N + BN - 1) / BN);
-    int clusters = dev >= 0 && dev < 64 ? max_clusters[dev] : num_sms / 2;
-    if (clusters > num_sms / 2) clusters = num_sms / 2;
-    if (clusters > tiles) clusters = tiles;
+    const int tiles_n = (p.N + BN - 1) / BN;
+    const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * tiles_n;
+    int max_pairs = dev >= 0 && dev < 64 ? max_clusters[dev] : num_sms / 2;
+    if (max_pairs > num_sms / 2) max_pairs = num_sms / 2;
+    int clusters = max_pairs < tiles ? max_pairs : tiles;
     if (MODE == 1) {
         // Row softmax: a tile's epilogue waits for the other column tiles of its row panel.  With a
         // pair count that is a multiple of the column-tile count every panel lives inside one round;
         // otherwise panels straddle rounds and their first tiles hold an accumulator buffer for a
         // whole extra round.
-        const int tiles_n = (p.N + BN - 1) / BN;
         if (clusters > tiles_n) clusters = clusters / tiles_n * tiles_n;
     }
+    TcParams q = p;
+    q.split = 1;
+    q.split_from = tiles;
+    q.split_kb = 0;
+    if (p.split_ws) {
+        // Tiles left over after the full rounds (all of them, when there are fewer tiles than pairs) are cut
+        // along K so that the last round keeps every pair busy.
+        const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
+        const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + BK - 1) / BK;
+        const int full = tiles / max_pairs, tail = tiles - full * max_pairs;
+        // (row softmax: only when everything fits one round; cutting the last of several rounds would let
+        // row panels straddle rounds, which costs more than the split saves)
+        if (tail > 0 && !(MODE == 1 && full > 0)) {
+            int s = max_pairs / tail;
+            if (s > 8) s = 8;
+            if (s > num_kb / 4) s = num_kb / 4;
+            if (s * tail > kTcSplitUnits) s = kTcSplitUnits / tail;
+            // The merging slice gets kExtra k-blocks more than the others (about the time they need to park),
+            // so the critical path of the round is its main loop plus the merge.  Measured, parking and
+            // merging cost about as much as kMerge k-blocks of main loop: a split must save more than that.
+            constexpr int kExtra = 6, kMerge = 24;
+            const int park_kb = s >= 2 ? (num_kb - kExtra > s ? (num_kb - kExtra) / s : 1) : num_kb;
+            const int merge_kb = num_kb - park_kb * (s - 1);
+            const long long plain = (long long) ((tiles + clusters - 1) / clusters) * num_kb;
+            const long long cut = (long long) full * num_kb + merge_kb + kMerge;
+            if (s >= 2 && cut < plain) {
+                q.split = s;
+                q.split_from = full * max_pairs;
+                q.split_kb = park_kb;
+                clusters = full > 0 ? max_pairs : tail * s;
+            }
+        }
+    }
+    if (plan) {
+        plan->bn = BN;
+        plan->tiles = tiles;
+        plan->pairs = clusters;
+        plan->split = q.split;
+        plan->split_tiles = tiles - q.split_from;
+        plan->split_kb = q.split_kb;
+    }
+    if (!tmA) return cudaSuccess;   // planning only
     cfg.gridDim = dim3(2 * clusters);
-    return cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+    return cudaLaunchKernelEx(&cfg, kernel, *tmA, *tmB, q);
 }
 
 template <int BN>
-cudaError_t launch_bn(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int num_sms, cudaStream_t stream) {
+cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int num_sms, cudaStream_t stream,
+                      TcPlan* plan) {
     switch (p.mode) {
-        case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream);
-        case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream);
-        case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream);
-        default: return launch_one<BN, 2>(p, tmA, tmB, num_sms, stream);
+        case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream, plan);
+        case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream, plan);
+        case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream, plan);
+        default: return launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
     }
 }
 
@@ -761,7 +937,11 @@ size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : Cf
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int num_sms,
                            cudaStream_t stream, int* launches) {
     *launches += 1;
-    return bn == 256 ? launch_bn<256>(p, tmA, tmB, num_sms, stream) : launch_bn<128>(p, tmA, tmB, num_sms, stream);
+    return bn == 256 ? launch_bn<256>(p, &tmA, &tmB, num_sms, stream, nullptr) : launch_bn<128>(p, &tmA, &tmB, num_sms, stream, nullptr);
+}
+
+cudaError_t plan_gemm_tc(const TcParams& p, int bn, int num_sms, TcPlan* plan) {
+    return bn == 256 ? launch_bn<256>(p, nullptr, nullptr, num_sms, nullptr, plan) : launch_bn<128>(p, nullptr, nullptr, num_sms, nullptr, plan);
 }
 
 }  // namespace fc
