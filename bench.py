@@ -65,7 +65,7 @@ def load_traffic(workload: str, full_size: bool):
 # ------------------------------------------------------------------------------ units per workload
 def units(ch):
     """(metric name, unit, algorithmic units per step, roofline bound)."""
-    if ch.producer == "elementwise":
+    if ch.producer == "elementwise" or wl.collapses(ch):
         return "fused_chain_throughput", "GB/s", wl.algorithmic_bytes(ch) / 1e9, "hbm"
     return "fused_chain_throughput", "TFLOP/s", ch.flops() / 1e12, "tensor" if ch.in_dtype == "bf16" else "alu"
 
@@ -152,6 +152,11 @@ def eager_fn(ch, t):
         return lambda: torch.clamp(F.gelu(F.linear(t[0], t[1], t[2]), approximate="tanh") * 0.5, -1.0, 1.0)
     if name == "gemm_bf16_bias_scale_lse":
         return lambda: torch.logsumexp((F.linear(t[0], t[1], t[2]) * 0.5).float(), dim=1)
+    if name.startswith("linear_bf16_row_"):
+        red = {"row_sum": lambda y: y.float().sum(1), "row_mean": lambda y: y.float().mean(1), "row_max": lambda y: y.float().amax(1)}[ch.reduce]
+        if ch.ops == (("bias_n", 2),):
+            return lambda: red(F.linear(t[0], t[1], t[2]))
+        return None
     if name == "gemm_bf16_row_softmax":
         return lambda: torch.softmax(t[0] @ t[1].t(), dim=1)
     if name == "conv_bf16_bias_relu_avgpool":

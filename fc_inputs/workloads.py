@@ -114,6 +114,22 @@ def gemm_bias_scale_lse(M=1024, N=4096, K=1024, variant="var", store_main=False)
                                ("bias", "bf16", (N,), "uniform", -0.1, 0.1)))
 
 
+def linear_row_reduce(M=1024, N=8192, K=8192, reduce="row_sum", ops=None, variant="std", store_main=False) -> Chain:
+    """A linear layer reduced over its output features to one value per row (the first steps of the
+    paper's showcase chain: linear -> sum over features).  Default ops: bias only, which leaves the chain
+    linear; pass ops with a ("relu",) to keep the contraction."""
+    s = K ** -0.5 if variant == "std" else K ** -0.25
+    if ops is None:
+        ops = (("bias_n", 2),)
+    return Chain(f"linear_bf16_{reduce}", "gemm_nt", "bf16", "bf16", M=M, N=N, K=K,
+                 ops=tuple(ops), reduce=reduce, store_main=store_main,
+                 input_recipe=(("A", "bf16", (M, K), "normal", 0.0, s),
+                               ("B", "bf16", (N, K), "normal", 0.0, s),
+                               ("bias", "bf16", (N,), "uniform", -0.1, 0.1),
+                               ("gamma", "bf16", (N,), "normal", 1.0, 0.1),
+                               ("beta", "bf16", (N,), "normal", 0.0, 0.1)))
+
+
 def conv_bias_relu_avgpool(batch=32, H=56, W=56, Cin=256, Cout=256, R=3, S=3, stride=1, pad=1) -> Chain:
     s = (R * S * Cin) ** -0.5
     return Chain("conv_bf16_bias_relu_avgpool", "conv2d_nhwc", "bf16", "f32",
@@ -136,6 +152,7 @@ CONFIGS = {
 #: Further measured workloads beyond the five configurations (rows marked "next" in the scope table).
 EXTRA = {
     "F1": lambda **kw: gemm_bias_scale_lse(**{"M": 4096, "N": 8192, "K": 4096, **kw}),
+    "F2": lambda **kw: linear_row_reduce(**{"M": 1024, "N": 8192, "K": 8192, **kw}),
 }
 ALL = {**CONFIGS, **EXTRA}
 
@@ -165,6 +182,14 @@ def with_integer_inputs(chain: Chain, lo: int = -4, hi: int = 4) -> Chain:
         tag, dtype, shape, _, _, _ = rec[i]
         rec[i] = (tag, dtype, shape, "int", lo, hi)
     return replace(chain, input_recipe=tuple(rec))
+
+
+def collapses(chain: Chain) -> bool:
+    """True for a 16-bit linear layer whose ops are all linear in the accumulator and whose only output is
+    the row sum / mean: the reduction then commutes with the contraction and the chain is bound by reading
+    its operands once, not by the M x N x K flops."""
+    return (chain.producer == "gemm_nt" and chain.in_dtype != "f32" and chain.reduce in ("row_sum", "row_mean")
+            and not chain.store_main and all(op[0] in ("bias_n", "affine_n", "scale") for op in chain.ops))
 
 
 def input_bytes(chain: Chain) -> int:

@@ -98,9 +98,9 @@ typedef enum {
     FC_RED_ROW_LOGSUMEXP = 1,   /* out[m] = max_n v + log sum_n exp(v - max)          */
     FC_RED_ROW_SOFTMAX = 2,     /* p[m][n] = exp(v - max) / sum_n exp(v - max)         */
     FC_RED_GLOBAL_AVGPOOL = 3,  /* out[b][c] = mean over (oh, ow) of v[b][oh][ow][c]   */
-    FC_RED_ROW_SUM = 4,         /* out[m] = sum_n v          (elementwise producer)     */
-    FC_RED_ROW_MAX = 5,         /* out[m] = max_n v          (elementwise producer)     */
-    FC_RED_ROW_MEAN = 6         /* out[m] = (sum_n v) / N    (elementwise producer)     */
+    FC_RED_ROW_SUM = 4,         /* out[m] = sum_n v          (elementwise or GEMM producer) */
+    FC_RED_ROW_MAX = 5,         /* out[m] = max_n v          (elementwise or GEMM producer) */
+    FC_RED_ROW_MEAN = 6         /* out[m] = (sum_n v) / N    (elementwise or GEMM producer) */
 } fc_reduce;
 
 typedef struct {
@@ -159,13 +159,22 @@ fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, in
                           const fc_tensor* outputs, int n_outputs, size_t* bytes);
 
 /*
- * Scratch memory.  Only GEMM_NT + ROW_SOFTMAX / ROW_LOGSUMEXP needs any (per-tile row maxima and sums
- * plus per-panel arrival counters for the cross-tile online max/sum merge).  fc_workspace_size reports
+ * Scratch memory.  Only a 16-bit GEMM_NT with a row reduction needs any (per-tile partial results plus
+ * per-panel arrival counters for the cross-tile merge; K + 1 doubles for the collapsed form, below).
+ * fc_workspace_size reports
  * the bytes a spec needs (0 for the other chains); fc_set_workspace registers a caller-owned DEVICE
  * buffer (256-byte aligned) for the current device, used by later fc_run calls until replaced.
  */
 fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes);
 fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
+
+/*
+ * Collapsed form.  A 16-bit GEMM_NT whose ops are only BIAS_N, AFFINE_N and SCALE, reduced by ROW_SUM or
+ * ROW_MEAN with store_main == 0, is not run as a GEMM: the sum over the output features commutes with
+ * the contraction (the rewrite of the paper's showcase chain, linear layer -> sum over features),
+ * out[m] = sum_k A[m][k] (sum_n a[n] B[n][k]) + sum_n c[n] with v -> a[n] v + c[n] the ops' effect, so
+ * the weights and the activations are each read once.  Accumulated in fp64, rounded once to fp32.
+ */
 
 /*
  * Optional extra scratch.  A tensor-core chain (GEMM_NT or CONV2D_NHWC in bf16 / fp16) whose output
@@ -182,7 +191,7 @@ fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
 
 /*
  * Writes a one-line description of how fc_run would execute `spec` on the current device with the
- * workspace registered now: "kernel=ew_rowreduce", "kernel=gemm_f32", or
+ * workspace registered now: "kernel=ew_rowreduce", "kernel=gemm_f32", "kernel=collapse", or
  * "kernel=gemm_tc mode=<0 store|1 softmax|2 conv+pool|3 logsumexp> bn=<tile width> tiles=<256 x bn tiles>
  * pairs=<CTA pairs launched> split=<slices per split tile, 1 = none> split_tiles=<tiles that are split>
  * split_kb=<64-wide k-blocks per parking slice>".  `text` is a caller-owned HOST buffer of `capacity`

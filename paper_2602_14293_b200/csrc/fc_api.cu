@@ -97,7 +97,7 @@ bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16; }
 
 // ------------------------------------------------------------------------------- validation
 struct Plan {
-    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV } kind;
+    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV, GEMM_COLLAPSE } kind;
     long long out_rows, out_cols;  // main output viewed as [rows][cols]
     int n_prod_inputs;
     int n_outputs;
@@ -173,10 +173,16 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
                 plan->kind = Plan::TC_PLAIN;
             } else if (s->reduce == FC_RED_ROW_SOFTMAX) {
                 plan->kind = Plan::TC_SOFTMAX;
-            } else if (s->reduce == FC_RED_ROW_LOGSUMEXP) {
-                plan->kind = Plan::TC_LSE;
+            } else if (s->reduce == FC_RED_ROW_LOGSUMEXP || s->reduce == FC_RED_ROW_SUM || s->reduce == FC_RED_ROW_MAX || s->reduce == FC_RED_ROW_MEAN) {
+                plan->kind = Plan::TC_LSE;   // any reduction of a row to one value
+                // A sum or mean over the output features of a purely linear epilogue, with no main output,
+                // commutes with the contraction: out = A (sum_n a[n] B[n][:]) + sum_n c[n]  (collapse.cu)
+                bool linear = (s->reduce == FC_RED_ROW_SUM || s->reduce == FC_RED_ROW_MEAN) && !s->store_main;
+                for (int i = 0; i < s->n_ops && linear; ++i)
+                    linear = s->ops[i].kind == FC_OP_BIAS_N || s->ops[i].kind == FC_OP_AFFINE_N || s->ops[i].kind == FC_OP_SCALE;
+                if (linear) plan->kind = Plan::GEMM_COLLAPSE;
             } else {
-                return fail(FC_ERR_UNSUPPORTED, "bf16 GEMM supports reduce NONE, ROW_SOFTMAX or ROW_LOGSUMEXP");
+                return fail(FC_ERR_UNSUPPORTED, "16-bit GEMM supports reduce NONE, ROW_SOFTMAX, ROW_LOGSUMEXP, ROW_SUM, ROW_MAX or ROW_MEAN");
             }
             break;
         default:
@@ -428,6 +434,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.in_dt = spec->in_dtype;
             p.out = plan.main_index >= 0 ? outputs[plan.main_index].ptr : nullptr; p.out_dt = spec->out_dtype;
             p.red = plan.red_index >= 0 ? (float*) outputs[plan.red_index].ptr : nullptr;
+            p.red_kind = spec->reduce;
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
             const int bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
@@ -459,6 +466,23 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
+            break;
+        }
+        case Plan::GEMM_COLLAPSE: {
+            const size_t need = collapse_workspace_bytes(spec->N, spec->K);
+            if (!dev->workspace || dev->workspace_bytes < need)
+                return fail(FC_ERR_WORKSPACE, "this chain needs a %zu-byte workspace (fc_set_workspace); have %zu", need, dev->workspace_bytes);
+            {
+                std::lock_guard<std::mutex> lk(g_mu);
+                dev->counter_layout = 0;   // the collapsed weights overwrite where other chains keep counters
+            }
+            CollapseParams p;
+            p.A = inputs[0].ptr; p.B = inputs[1].ptr; p.in_dt = spec->in_dtype;
+            p.M = spec->M; p.N = spec->N; p.K = spec->K;
+            build_ops(spec, inputs, &p.ops);
+            p.out = (float*) outputs[plan.red_index].ptr;
+            p.post = spec->reduce == FC_RED_ROW_MEAN ? 1.0f / (float) spec->N : 1.0f;
+            e = launch_collapse(p, dev->workspace, stream, &launches);
             break;
         }
         case Plan::TC_CONV: {
@@ -552,7 +576,7 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
     const long long rows = conv ? spec->batch : spec->M;
     const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE) ? 256 : 1;
     long long chunks = 1;
-    if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
+    if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && plan.kind != Plan::GEMM_COLLAPSE && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
         chunks = rows / gran < 8 ? rows / gran : 8;
         if (chunks < 1) chunks = 1;
     }
@@ -641,7 +665,8 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     fc_status st;
     if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
     if ((st = validate_spec(spec, &plan))) return st;
-    *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N) : 0;
+    *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N)
+           : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K) : 0;
     return FC_OK;
 }
 
@@ -663,6 +688,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     if ((st = validate_spec(spec, &plan))) return st;
     if (plan.kind == Plan::EW) { snprintf(text, capacity, "kernel=ew_rowreduce"); return FC_OK; }
     if (plan.kind == Plan::GEMM_F32) { snprintf(text, capacity, "kernel=gemm_f32"); return FC_OK; }
+    if (plan.kind == Plan::GEMM_COLLAPSE) { snprintf(text, capacity, "kernel=collapse"); return FC_OK; }
     DeviceInfo* dev;
     if ((st = get_device(&dev))) return st;
     TcParams p;

@@ -63,14 +63,28 @@ struct GemmF32Params {
 };
 cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* launches);
 
+// GEMM + linear ops + row sum / mean without a main output, rewritten as out = A u + C (see collapse.cu)
+struct CollapseParams {
+    const void* A; const void* B; int in_dt;   // [M,K], [N,K], FC_BF16 or FC_F16
+    long long M, N, K;
+    DevOps ops;                 // BIAS_N, AFFINE_N and SCALE only
+    float* out;                 // [M]
+    float post;                 // 1 (sum) or 1/N (mean)
+    // carved out of the workspace by the launcher
+    double* partial; double* cpart; double* cterm; float* u;
+};
+cudaError_t launch_collapse(const CollapseParams& p, void* workspace, cudaStream_t stream, int* launches);
+size_t collapse_workspace_bytes(long long N, long long K);
+
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
-    int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row logsumexp
+    int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row reduction to one value
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
     int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
     int in_dt;                  // FC_BF16 or FC_F16: storage of both MMA operands
     void* out; int out_dt;      // mode 0/1/3: [M,N] bf16 or f32 (mode 3: may be null).  mode 2: f32 [batch,Cout] (pre-zeroed)
-    float* red;                 // mode 3: row logsumexp [M]
+    float* red;                 // mode 3: row reduction [M]
+    int red_kind;               // mode 3: FC_RED_ROW_LOGSUMEXP, _SUM, _MAX or _MEAN
     DevOps ops;
     // mode 1
     float2* stats;              // [M][tiles_n] (max, sum) per tile

@@ -5,8 +5,8 @@
 //   mode 1  row softmax over N fused across tiles: every tile publishes per-row (max, sum) of its
 //           column slice, waits (bounded) until the row panel's tiles have all published, merges
 //           the pairs and writes normalised probabilities straight from tensor memory
-//   mode 3  row logsumexp over N: as mode 0 (the main output is optional) plus per-tile (max, sum) pairs;
-//           the tile that publishes last for a row panel merges them, so no tile waits
+//   mode 3  row logsumexp / sum / max / mean over N: as mode 0 (the main output is optional) plus per-tile
+//           partial results; the tile that publishes last for a row panel merges them, so no tile waits
 //   mode 2  implicit-GEMM convolution: the A operand is gathered by im2col-mode TMA from the NHWC
 //           image (zero fill outside the image), B is the [Cout][R*S*Cin] weight matrix; the
 //           epilogue applies ops (bias, ReLU) and sums each channel over the tile's pixels, adding
@@ -604,9 +604,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             } else if constexpr (MODE == 3) {
-                // ops, optional store, and a running (max, sum) of the row slice in the log2 domain; the
-                // tile that publishes last for its row panel merges all slices into the logsumexp, so
-                // nobody waits for anybody
+                // ops, optional store, and a running reduction of the row slice: (max, sum of exponentials) in
+                // the log2 domain for logsumexp, a plain sum or maximum otherwise.  The tile that publishes
+                // last for its row panel merges all slices, so nobody waits for anybody.
+                const int rk = p.red_kind;
                 float run_m = -CUDART_INF_F, run_s = 0.0f;
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
@@ -620,25 +621,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
                         apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                         if (p.out) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
-                        float cm = -CUDART_INF_F;
+                        if (rk == FC_RED_ROW_LOGSUMEXP || rk == FC_RED_ROW_MAX) {
+                            float cm = -CUDART_INF_F;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
-                        const float nm = fmaxf(run_m, cm * kLog2e);
-                        float cs = 0.0f;
+                            for (int j = 0; j < 16; ++j) cm = n0 + j < p.N ? fmaxf(cm, v[j]) : cm;
+                            if (rk == FC_RED_ROW_MAX) {
+                                run_m = fmaxf(run_m, cm);
+                            } else {
+                                const float nm = fmaxf(run_m, cm * kLog2e);
+                                float cs = 0.0f;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast(fmaf(v[j], kLog2e, -nm)) : 0.0f;
-                        run_s = fmaf(run_s, exp2_fast(run_m - nm), cs);
-                        run_m = nm;
+                                for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast(fmaf(v[j], kLog2e, -nm)) : 0.0f;
+                                run_s = fmaf(run_s, exp2_fast(run_m - nm), cs);
+                                run_m = nm;
+                            }
+                        } else {
+                            float cs = 0.0f;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? v[j] : 0.0f;
+                            run_s += cs;
+                        }
                     }
                 }
+                // merge of two partial results of one row, by kind
+                auto merge = [rk](float am, float as, float bm, float bs) {
+                    if (rk == FC_RED_ROW_LOGSUMEXP) {
+                        const float nm = fmaxf(am, bm);
+                        const float sa = am == -CUDART_INF_F ? 0.0f : as * exp2_fast(am - nm);
+                        const float sb = bm == -CUDART_INF_F ? 0.0f : bs * exp2_fast(bm - nm);
+                        return make_float2(nm, sa + sb);
+                    }
+                    return make_float2(fmaxf(am, bm), as + bs);
+                };
                 if (half == 1) xchg[row] = make_float2(run_m, run_s);
                 ptx::bar_sync(1, kEpiThreads);
                 if (half == 0 && m < p.M) {
                     const float2 o = xchg[row];
-                    const float nm = fmaxf(run_m, o.x);
-                    const float sa = run_m == -CUDART_INF_F ? 0.0f : run_s * exp2_fast(run_m - nm);
-                    const float sb = o.x == -CUDART_INF_F ? 0.0f : o.y * exp2_fast(o.x - nm);
-                    __stcg(&p.stats[m * tiles_n + nb], make_float2(nm, sa + sb));
+                    __stcg(&p.stats[m * tiles_n + nb], merge(run_m, run_s, o.x, o.y));
                 }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
@@ -650,16 +669,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 ptx::bar_sync(1, kEpiThreads);
                 if (*(volatile int*) &ctrl->last && half == 0 && m < p.M) {
-                    float am = -CUDART_INF_F, as = 0.0f;
+                    float2 a = make_float2(-CUDART_INF_F, 0.0f);
                     for (int j = 0; j < tiles_n; ++j) {
                         const float2 st = __ldcg(&p.stats[m * tiles_n + j]);
-                        const float nm = fmaxf(am, st.x);
-                        const float sa = am == -CUDART_INF_F ? 0.0f : as * exp2_fast(am - nm);
-                        const float sb = st.x == -CUDART_INF_F ? 0.0f : st.y * exp2_fast(st.x - nm);
-                        as = sa + sb;
-                        am = nm;
+                        a = merge(a.x, a.y, st.x, st.y);
                     }
-                    p.red[m] = (am + log2f(as)) * kLn2;
+                    p.red[m] = rk == FC_RED_ROW_LOGSUMEXP ? (a.x + log2f(a.y)) * kLn2
+                             : rk == FC_RED_ROW_MAX ? a.x
+                             : rk == FC_RED_ROW_MEAN ? a.y / (float) p.N : a.y;
                 }
             } else if constexpr (MODE == 1) {
                 // sweep A: maximum of this thread's half row of the tile (ops applied, written back in place

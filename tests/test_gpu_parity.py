@@ -405,3 +405,43 @@ def test_fp16_chains(fc, orc, seed):
     run_and_check(fc, orc, _as_f16(wl.affine_gelu_residual_lse(65, 4096)), seed)
     run_and_check(fc, orc, _as_f16(wl.affine_gelu_residual_lse(9, 1001)), seed)
     run_and_check(fc, orc, replace(_as_f16(wl.affine_gelu_residual_lse(33, 2048)), reduce="row_mean"), seed)
+
+
+# ------------------------------------------------------------------ linear layer reduced over its output features
+@pytest.mark.parametrize("red", ["row_sum", "row_max", "row_mean"])
+@pytest.mark.parametrize("M,N,K,store_main", [(128, 256, 64, False), (300, 1000, 136, True), (256, 4096, 256, False), (130, 40, 72, True)])
+def test_gemm_row_sum_max_mean_through_the_contraction(fc, orc, red, M, N, K, store_main):
+    """A ReLU between the linear layer and the reduction keeps the GEMM: tensor-core kernel, per-tile
+    partial results, last tile of a panel merges."""
+    ch = wl.linear_row_reduce(M, N, K, red, ops=(("bias_n", 2), ("relu",), ("scale", 0.5)), variant="var", store_main=store_main)
+    assert fc.binding.fc_describe_plan(fc.make_spec(ch))["kernel"] == "gemm_tc"
+    run_and_check(fc, orc, ch, 8)
+
+
+@pytest.mark.parametrize("red", ["row_sum", "row_mean"])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 1000, 136), (77, 520, 4104), (1200, 264, 2048), (5000, 96, 512)])
+@pytest.mark.parametrize("ops", [(), (("bias_n", 2),), (("bias_n", 2), ("scale", -0.75)), (("affine_n", 3, 4), ("bias_n", 2)),
+                                 (("scale", 2.0), ("affine_n", 3, 4), ("scale", 0.5), ("bias_n", 2))])
+def test_linear_row_sum_collapsed(fc, orc, red, M, N, K, ops):
+    """Purely linear ops and no main output: the sum over the features is taken through the weights
+    (out = A u + C); the oracle still does the full contraction."""
+    ch = wl.linear_row_reduce(M, N, K, red, ops=ops, variant="var")
+    assert fc.binding.fc_describe_plan(fc.make_spec(ch))["kernel"] == "collapse"
+    run_and_check(fc, orc, ch, 9)
+
+
+def test_linear_row_sum_collapsed_integer_inputs_exact(fc, orc):
+    """Integer operands and no ops: every partial sum is an integer below 2^53, so the fp64 path gives
+    the exact row sums; the fp32 output holds them exactly while they stay below 2^24."""
+    ch = wl.with_integer_inputs(wl.linear_row_reduce(200, 512, 264, "row_sum", ops=()), -3, 3)
+    ins = wl.make_inputs(ch, 3)
+    outs, ref, _ = run_and_check(fc, orc, ch, ins=ins)
+    assert np.abs(ref["reduce"]).max() < 2 ** 24
+    np.testing.assert_array_equal(util.to_f64(outs[0]), ref["reduce"])
+
+
+def test_linear_row_sum_fp16_collapsed_and_not(fc, orc):
+    for ops in [(("bias_n", 2),), (("bias_n", 2), ("gelu_tanh",))]:
+        ch = replace(wl.linear_row_reduce(256, 512, 256, "row_sum", ops=ops, variant="var"), in_dtype="f16", out_dtype="f16")
+        ch = replace(ch, input_recipe=tuple((t, "f16", sh, d, a, b) for t, d0, sh, d, a, b in ch.input_recipe))
+        run_and_check(fc, orc, ch, 10)
