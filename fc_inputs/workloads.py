@@ -42,7 +42,7 @@ class Chain:
     # ops: ("bias_n", i) ("affine_n", i, j) ("relu",) ("gelu_tanh",) ("scale", f) ("clamp", lo, hi)
     #      ("add_tensor", i)   -- i, j index the input list
     ops: Tuple[tuple, ...] = ()
-    reduce: str = "none"          # "none" | "row_logsumexp" | "row_softmax" | "global_avgpool" | "row_sum" | "row_max" | "row_mean"
+    reduce: str = "none"          # "none" | "row_logsumexp" | "row_softmax" | "global_avgpool" | "row_sum" | "row_max" | "row_mean" | "maxpool_2x2"
     store_main: bool = True
     # (tag, dtype, shape, dist, p0, p1) per input, in input order
     input_recipe: Tuple[tuple, ...] = field(default=(), compare=False)
@@ -140,6 +140,13 @@ def conv_bias_relu_avgpool(batch=32, H=56, W=56, Cin=256, Cout=256, R=3, S=3, st
                                ("bias", "bf16", (Cout,), "uniform", -0.1, 0.1)))
 
 
+def conv_bias_relu_maxpool(batch=8, H=32, W=32, Cin=64, Cout=128, R=5, S=5, stride=1, pad=2) -> Chain:
+    """Convolution -> bias -> ReLU -> 2x2 max-pool (the conv / ReLU / max-pool stage of the paper's
+    Level-3 LeNet-shaped example, at tensor-core-sized channel counts)."""
+    base = conv_bias_relu_avgpool(batch, H, W, Cin, Cout, R, S, stride, pad)
+    return replace(base, name="conv_bf16_bias_relu_maxpool", reduce="maxpool_2x2")
+
+
 #: The five benchmark configurations, in the order the benchmark numbers them.
 CONFIGS = {
     "C1": gemm_bias_relu_f32,
@@ -212,6 +219,8 @@ def output_shapes(chain: Chain):
         outs.append(("reduce", "f32", (chain.M,)))
     elif chain.reduce == "global_avgpool":
         outs.append(("reduce", "f32", (chain.batch, chain.Cout)))
+    elif chain.reduce == "maxpool_2x2":
+        outs.append(("reduce", "f32", (chain.batch, chain.OH // 2, chain.OW // 2, chain.Cout)))
     return outs
 
 

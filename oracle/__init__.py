@@ -156,6 +156,13 @@ def global_avgpool(V: np.ndarray) -> np.ndarray:
     return out
 
 
+def maxpool_2x2(V: np.ndarray) -> np.ndarray:
+    NB, OH, OW, C = V.shape
+    out = np.empty((NB, OH // 2, OW // 2, C), dtype=np.float64)
+    lib().orc_maxpool_2x2(_p(V), _i64(NB), _i64(OH), _i64(OW), _i64(C), _p(out))
+    return out
+
+
 def run_chain(chain, inputs: List[np.ndarray]) -> Dict[str, np.ndarray]:
     """Evaluate ``chain`` on stored ``inputs``.  Returns {"main": f64 array, "reduce": f64 array}
     ("reduce" only when the chain has a reduction; "main" is always the pre-reduction tensor)."""
@@ -177,6 +184,8 @@ def run_chain(chain, inputs: List[np.ndarray]) -> Dict[str, np.ndarray]:
         out["reduce"] = row_softmax(V.reshape(-1, V.shape[-1]))
     elif chain.reduce == "global_avgpool":
         out["reduce"] = global_avgpool(V)
+    elif chain.reduce == "maxpool_2x2":
+        out["reduce"] = maxpool_2x2(V)
     elif chain.reduce == "row_sum":
         out["reduce"] = row_sum(V.reshape(-1, V.shape[-1]))
     elif chain.reduce == "row_max":

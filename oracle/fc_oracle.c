@@ -20,6 +20,9 @@
  *                      multiply).
  *   orc_row_logsumexp  max + log(sum exp(v - max)); over a row of length one this is the identity,
  *                      the closed form the paper's appendix (Level-2 Q18 analysis) relies on.
+ *   orc_maxpool_2x2    maximum over non-overlapping 2 x 2 windows, floor output size (the window
+ *                      arithmetic of the paper's appendix max-pool listing with kernel 2, stride 2,
+ *                      no padding, restated for NHWC).
  *   orc_gelu_tanh, orc_clamp, orc_affine_n, orc_add_tensor, orc_row_softmax, orc_global_avgpool,
  *   orc_row_sum, orc_row_max (row mean = row sum / N)
  *                      textbook definitions; the paper does not print them, the benchmark
@@ -28,7 +31,8 @@
  * Pins (tests, CPU only): identity / zero / rank-1 weights, exact small-integer contractions,
  * exact-rational brute force with a different loop order on tiny shapes, centre and shifted delta
  * kernels, all-ones tap counts, high-precision (mpmath) values of GELU / logsumexp / softmax,
- * shift invariance, constant rows, rows summing to one, pooling linearity.
+ * shift invariance, constant rows, rows summing to one, pooling linearity; max-pool against a
+ * reshape-and-max in numpy, a single planted maximum per window, and dropped odd edges.
  */
 #include <math.h>
 #include <stdint.h>
@@ -198,6 +202,28 @@ void orc_global_avgpool(const double* V, int64_t NB, int64_t HW, int64_t C, doub
             double s = 0.0;
             for (int64_t p = 0; p < HW; ++p) s += V[(b * HW + p) * C + c];
             out[b * C + c] = s / (double)HW;
+        }
+    }
+}
+
+/* out[b][i][j][c] = max over the 2 x 2 window (rows 2i, 2i+1; columns 2j, 2j+1) of V[b][.][.][c];
+ * output size floor(OH/2) x floor(OW/2): a last odd row or column belongs to no window */
+void orc_maxpool_2x2(const double* V, int64_t NB, int64_t OH, int64_t OW, int64_t C, double* out) {
+    const int64_t PH = OH / 2, PW = OW / 2;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t b = 0; b < NB; ++b) {
+        for (int64_t i = 0; i < PH; ++i) {
+            for (int64_t j = 0; j < PW; ++j) {
+                for (int64_t c = 0; c < C; ++c) {
+                    double mx = V[((b * OH + 2 * i) * OW + 2 * j) * C + c];
+                    for (int64_t di = 0; di < 2; ++di)
+                        for (int64_t dj = 0; dj < 2; ++dj) {
+                            const double v = V[((b * OH + 2 * i + di) * OW + 2 * j + dj) * C + c];
+                            mx = v > mx ? v : mx;
+                        }
+                    out[((b * PH + i) * PW + j) * C + c] = mx;
+                }
+            }
         }
     }
 }

@@ -133,3 +133,32 @@ def test_non_contiguous_tensor_is_rejected(fc):
     ins = _arr(fc, [x, _fake_tensor(fc, (16,), 1), _fake_tensor(fc, (16,), 1), _fake_tensor(fc, (8, 16), 1)])
     outs = _arr(fc, [_fake_tensor(fc, (8, 16), 1), _fake_tensor(fc, (8,), 0)])
     assert _status(fc, s, ins, outs) == 3
+
+
+def test_workspace_sizes_of_split_and_collapsed_chains(fc):
+    """Sizes are host arithmetic: the optional split scratch is a fixed region behind the required part,
+    and a collapsing chain needs its slabs of fp64 column sums plus the fp32 vector."""
+    b = fc.binding
+    plain = fc.make_spec(wl.gemm_bias_gelu_scale_clamp(256, 1024, 4096))
+    assert b.fc_workspace_size(plain) == 0
+    split_region = b.fc_workspace_size_split(plain)
+    assert split_region == 1024 + 80 * 2 * 128 * 256 * 4
+    soft = fc.make_spec(wl.CONFIGS["C4"]())
+    assert b.fc_workspace_size_split(soft) == b.fc_workspace_size(soft) + split_region
+    ew = fc.make_spec(wl.CONFIGS["C2"]())
+    assert b.fc_workspace_size_split(ew) == 0
+    # collapse: 640 target blocks / 32 column blocks = 20 slabs for K = 8192
+    col = fc.make_spec(wl.linear_row_reduce(1024, 8192, 8192))
+    slabs = 20
+    doubles = slabs * 8192 + slabs + 1
+    assert b.fc_workspace_size(col) == (doubles * 8 + 255) // 256 * 256 + 8192 * 4
+    assert b.fc_workspace_size_split(col) == 0
+
+
+def test_collapse_is_chosen_only_for_linear_epilogues_without_main_output():
+    assert wl.collapses(wl.linear_row_reduce(64, 64, 64))
+    assert wl.collapses(wl.linear_row_reduce(64, 64, 64, "row_mean", ops=(("affine_n", 3, 4), ("scale", 2.0))))
+    assert not wl.collapses(wl.linear_row_reduce(64, 64, 64, "row_max"))
+    assert not wl.collapses(wl.linear_row_reduce(64, 64, 64, ops=(("bias_n", 2), ("relu",))))
+    assert not wl.collapses(wl.linear_row_reduce(64, 64, 64, store_main=True))
+    assert not wl.collapses(wl.gemm_bias_scale_lse(64, 64, 64))

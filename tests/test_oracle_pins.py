@@ -305,3 +305,32 @@ def test_elementwise_chain_matches_library_sequence(orc):
     got = orc.run_chain(ch, ins)
     np.testing.assert_allclose(got["main"], y.numpy(), rtol=0, atol=1e-13)
     np.testing.assert_allclose(got["reduce"], torch.logsumexp(y, 1).numpy(), rtol=1e-13)
+
+
+def test_maxpool_2x2_against_reshape_and_planted_maxima(orc):
+    """Non-overlapping 2x2 windows: numpy's reshape-and-max on even sizes; one planted maximum per
+    window recovered at the right output position; an odd last row / column belongs to no window."""
+    r = np.random.default_rng(5)
+    V = r.standard_normal((3, 6, 8, 5))
+    want = V.reshape(3, 3, 2, 4, 2, 5).max(axis=(2, 4))
+    assert np.array_equal(orc.maxpool_2x2(V), want)
+    # planted: window (i, j) of image b, channel c holds the value 100 + its own index at a random corner
+    Z = -np.abs(r.standard_normal((2, 4, 6, 3)))
+    tag = np.zeros((2, 2, 3, 3))
+    for b in range(2):
+        for i in range(2):
+            for j in range(3):
+                for c in range(3):
+                    di, dj = r.integers(0, 2, 2)
+                    tag[b, i, j, c] = 100 + ((b * 2 + i) * 3 + j) * 3 + c
+                    Z[b, 2 * i + di, 2 * j + dj, c] = tag[b, i, j, c]
+    assert np.array_equal(orc.maxpool_2x2(Z), tag)
+    # odd sizes: the last row and column are dropped, so poisoning them changes nothing
+    W = r.standard_normal((1, 5, 7, 2))
+    base = orc.maxpool_2x2(W)
+    assert base.shape == (1, 2, 3, 2)
+    W2 = W.copy(); W2[:, 4, :, :] = 1e9; W2[:, :, 6, :] = 1e9
+    assert np.array_equal(orc.maxpool_2x2(W2), base)
+    assert np.array_equal(base, W[:, :4, :6].reshape(1, 2, 2, 3, 2, 2).max(axis=(2, 4)))
+    # max commutes with a monotone map: pooling ReLU(V) equals ReLU of pooled V
+    assert np.array_equal(orc.maxpool_2x2(np.maximum(V, 0)), np.maximum(orc.maxpool_2x2(V), 0))
