@@ -159,6 +159,10 @@ def eager_fn(ch, t):
         return None
     if name == "gemm_bf16_row_softmax":
         return lambda: torch.softmax(t[0] @ t[1].t(), dim=1)
+    if name == "conv_bf16_bias_relu_maxpool":
+        x = t[0].permute(0, 3, 1, 2)
+        w = t[1].permute(0, 3, 1, 2)
+        return lambda: F.max_pool2d(torch.relu(F.conv2d(x, w, t[2], padding=ch.pad, stride=ch.stride)), 2).float()
     if name == "conv_bf16_bias_relu_avgpool":
         x = t[0].permute(0, 3, 1, 2)            # NHWC storage viewed as NCHW = channels_last
         w = t[1].permute(0, 3, 1, 2)
@@ -288,7 +292,7 @@ def main():
     ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-eager", action="store_true")
-    ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (context)")
+    ap.add_argument("--all-configs", action="store_true", help="also time the other configurations and the extra workloads (context)")
     ap.add_argument("--rows", type=int, default=0, help="override M (or the conv batch): a smaller case of the same kernel for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -426,10 +430,10 @@ def main():
 
     if rank == 0 and args.all_configs:
         per = {}
-        for key in sorted(wl.CONFIGS):
+        for key in sorted(wl.ALL):
             if key == args.workload:
                 continue
-            c2 = wl.CONFIGS[key]()
+            c2 = wl.ALL[key]()
             i2 = [fc.to_device(a) for a in wl.make_inputs(c2, 0)]
             o2 = binding.output_tensors(c2, "cuda")
             s2 = fc.make_spec(c2)

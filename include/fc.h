@@ -100,7 +100,10 @@ typedef enum {
     FC_RED_GLOBAL_AVGPOOL = 3,  /* out[b][c] = mean over (oh, ow) of v[b][oh][ow][c]   */
     FC_RED_ROW_SUM = 4,         /* out[m] = sum_n v          (elementwise or GEMM producer) */
     FC_RED_ROW_MAX = 5,         /* out[m] = max_n v          (elementwise or GEMM producer) */
-    FC_RED_ROW_MEAN = 6         /* out[m] = (sum_n v) / N    (elementwise or GEMM producer) */
+    FC_RED_ROW_MEAN = 6,        /* out[m] = (sum_n v) / N    (elementwise or GEMM producer) */
+    FC_RED_MAXPOOL_2X2 = 7      /* out[b][i][j][c] = max of v[b][2i..2i+1][2j..2j+1][c], fp32 [batch][OH/2][OW/2][Cout];
+                                   CONV producer whose op list ends with RELU (the conv / ReLU / max-pool stage
+                                   of the paper's appendix network); a last odd row or column is dropped       */
 } fc_reduce;
 
 typedef struct {

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(PKG, "libfc.so")
 FC_F32, FC_BF16, FC_F16 = 0, 1, 2
 _PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2}
 _OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6}
-_REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3, "row_sum": 4, "row_max": 5, "row_mean": 6}
+_REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3, "row_sum": 4, "row_max": 5, "row_mean": 6, "maxpool_2x2": 7}
 _DTYPE = {"f32": FC_F32, "bf16": FC_BF16, "f16": FC_F16}
 FC_MAX_OPS = 8
 
@@ -283,6 +283,8 @@ def output_tensors(chain, device="cuda", pinned=False) -> List[torch.Tensor]:
         outs.append(torch.empty((chain.M,), dtype=torch.float32, **kw))
     elif chain.reduce == "global_avgpool":
         outs.append(torch.empty((chain.batch, chain.Cout), dtype=torch.float32, **kw))
+    elif chain.reduce == "maxpool_2x2":
+        outs.append(torch.empty((chain.batch, OH // 2, OW // 2, chain.Cout), dtype=torch.float32, **kw))
     return outs
 
 

@@ -133,7 +133,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (!dt_valid(s->in_dtype) || !dt_valid(s->out_dtype))
         return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
     if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
-    if (s->reduce < 0 || s->reduce > FC_RED_ROW_MEAN) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
+    if (s->reduce < 0 || s->reduce > FC_RED_MAXPOOL_2X2) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
     if (s->n_ops < 0 || s->n_ops > FC_MAX_OPS) return fail(FC_ERR_INVALID_SPEC, "n_ops %d out of range", s->n_ops);
     for (int i = 0; i < s->n_ops; ++i)
         if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_ADD_TENSOR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
@@ -160,7 +160,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     plan->main_index = plan->red_index = -1;
     switch (s->producer) {
         case FC_PROD_ELEMENTWISE:
-            if (s->reduce == FC_RED_ROW_SOFTMAX || s->reduce == FC_RED_GLOBAL_AVGPOOL)
+            if (s->reduce == FC_RED_ROW_SOFTMAX || s->reduce == FC_RED_GLOBAL_AVGPOOL || s->reduce == FC_RED_MAXPOOL_2X2)
                 return fail(FC_ERR_UNSUPPORTED, "elementwise producer supports reduce NONE, ROW_LOGSUMEXP, ROW_SUM, ROW_MAX or ROW_MEAN");
             plan->kind = Plan::EW;
             break;
@@ -186,8 +186,15 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             }
             break;
         default:
-            if (s->in_dtype == FC_F32 || s->reduce != FC_RED_GLOBAL_AVGPOOL || s->store_main)
-                return fail(FC_ERR_UNSUPPORTED, "conv supports bf16 / fp16 input with GLOBAL_AVGPOOL and store_main = 0");
+            if (s->in_dtype == FC_F32 || (s->reduce != FC_RED_GLOBAL_AVGPOOL && s->reduce != FC_RED_MAXPOOL_2X2) || s->store_main)
+                return fail(FC_ERR_UNSUPPORTED, "conv supports bf16 / fp16 input with GLOBAL_AVGPOOL or MAXPOOL_2X2 and store_main = 0");
+            if (s->reduce == FC_RED_MAXPOOL_2X2) {
+                // the pooled maximum is taken with unsigned atomics on fp32 bit patterns over a zeroed output
+                if (s->n_ops < 1 || s->ops[s->n_ops - 1].kind != FC_OP_RELU)
+                    return fail(FC_ERR_UNSUPPORTED, "MAXPOOL_2X2 needs an op list that ends with RELU");
+                const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
+                if (OH < 2 || OW < 2) return fail(FC_ERR_SHAPE, "MAXPOOL_2X2 needs a conv output of at least 2 x 2 (is %lld x %lld)", OH, OW);
+            }
             if (s->stride > 8) return fail(FC_ERR_UNSUPPORTED, "conv supports stride <= 8");
             if (s->pad >= s->R || s->pad >= s->S || s->R > 16 || s->S > 16) return fail(FC_ERR_UNSUPPORTED, "conv supports pad < R,S <= 16");
             plan->kind = Plan::TC_CONV;
@@ -271,7 +278,11 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         }
     }
     if (plan.red_index >= 0) {
-        if (s->reduce != FC_RED_GLOBAL_AVGPOOL) {
+        if (s->reduce == FC_RED_MAXPOOL_2X2) {
+            const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
+            const long long sh[4] = {s->batch, OH / 2, OW / 2, s->Cout};
+            if ((st = check_tensor(out[plan.red_index], "pooled output", FC_F32, 4, sh))) return st;
+        } else if (s->reduce != FC_RED_GLOBAL_AVGPOOL) {
             const long long sh[1] = {s->M};
             if ((st = check_tensor(out[plan.red_index], "row reduction output", FC_F32, 1, sh))) return st;
         } else {
@@ -501,7 +512,9 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
             const int bn = spec->Cout <= 128 ? 128 : 256;
-            if ((e = cudaMemsetAsync(p.out, 0, (size_t) spec->batch * spec->Cout * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+            p.pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? 1 : 0;
+            const size_t out_elems = p.pool ? (size_t) spec->batch * (p.OH / 2) * (p.OW / 2) * spec->Cout : (size_t) spec->batch * spec->Cout;
+            if ((e = cudaMemsetAsync(p.out, 0, out_elems * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             attach_split_scratch(dev, 0, &p);
             if ((e = clear_counters_if_needed(dev, p, 0, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;

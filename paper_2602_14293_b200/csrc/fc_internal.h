@@ -51,7 +51,7 @@ struct EwParams {
     void* y; int y_dt;          // may be null when !store_main
     float* red;                 // row logsumexp out, or null
     long long M, N;
-    int reduce;                 // FC_RED_NONE or FC_RED_ROW_LOGSUMEXP
+    int reduce;                 // FC_RED_NONE or a row reduction
     DevOps ops;
 };
 cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t stream, int* launches);
@@ -93,6 +93,7 @@ struct TcParams {
     // mode 2
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
+    int pool;                   // mode 2: 0 global average pool, 1 2x2 max-pool (out pre-zeroed, values >= 0)
     int* status;                // device status word
     int expect_extra;           // mode 1, testing only: arrivals the panel wait expects beyond those that will come
     // Split tiles (filled by the launcher when the scratch below is given and a split pays): tiles from

@@ -10,7 +10,8 @@
 //   mode 2  implicit-GEMM convolution: the A operand is gathered by im2col-mode TMA from the NHWC
 //           image (zero fill outside the image), B is the [Cout][R*S*Cin] weight matrix; the
 //           epilogue applies ops (bias, ReLU) and sums each channel over the tile's pixels, adding
-//           the scaled partial sums into out[image][channel]
+//           the scaled partial sums into out[image][channel]; or takes the maximum over 2x2 windows
+//           into out[image][oh/2][ow/2][channel]
 //
 // Work unit: a 256 x BN output tile owned by a PAIR of CTAs on neighbouring SMs (cluster of 2,
 // tcgen05 cta_group::2).  Each CTA loads its own 128 rows of A and HALF of the B tile, so a k-block
@@ -58,7 +59,8 @@ struct Cfg {
     static constexpr int kTmemCols = 2 * BN;
     static constexpr int kVecBytes = 2 * kMaxVecSlots * BN * 4;   // double-buffered per-tile vector slices
     static constexpr int kCtrlBytes = 256;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024 + 1024;  // exchange + alignment slack
+    static constexpr int kPoolBytes = 8 * 32 * 17 * 4;   // max-pool: 32 pixels x 16 channels (+1 pad) per epilogue warp
+    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024 + kPoolBytes + 1024;  // exchange, pool staging, alignment slack
 };
 
 struct Ctrl {
@@ -334,6 +336,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     float* svec_all = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes);
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + C::kStages * C::kStageBytes + C::kVecBytes);
     float2* xchg = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes + C::kVecBytes + C::kCtrlBytes);
+    float* pool_stage = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes + C::kVecBytes + C::kCtrlBytes + 1024);
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -797,6 +800,59 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                         store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                     }
+                }
+            } else if (p.pool == 1) {
+                // conv + 2x2 max-pool of non-negative values (the op list ends with ReLU, the output starts at
+                // zero): every pixel that lies in a window takes part in an unsigned atomic maximum on the fp32
+                // bit pattern.  Horizontal neighbours are merged by a shuffle first; the values then go through
+                // shared memory so that one instruction updates 16 consecutive channels of two windows.
+                const int hw = p.OH * p.OW, PH = p.OH >> 1, PW = p.OW >> 1;
+                long long dst = 0;
+                bool merge = false, emit = false;
+                if (m < p.M) {
+                    const int img = (int) (m / hw);
+                    const int rem = (int) (m - (long long) img * hw);
+                    const int oh = rem / p.OW, ow = rem - oh * p.OW;
+                    if ((oh >> 1) < PH && (ow >> 1) < PW) {
+                        dst = (((long long) img * PH + (oh >> 1)) * PW + (ow >> 1)) * p.N;
+                        const bool even = (ow & 1) == 0;
+                        merge = even && lane < 31;      // the right neighbour sits in the next lane
+                        emit = even || lane == 0;       // an odd pixel is covered by its left neighbour, if this warp has it
+                    }
+                }
+                const unsigned emit_mask = __ballot_sync(0xffffffffu, emit);
+                float* stage = pool_stage + (warp - 2) * (32 * 17);
+                unsigned int* out_u = (unsigned int*) p.out;
+#pragma unroll 1
+                for (int c = 0; c < kChunks; ++c) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+                    ptx::tmem_wait_ld(r);
+                    const int n0 = n_half + c * 16;
+                    if (n0 >= p.N) continue;
+                    float v[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                    if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float nxt = __shfl_down_sync(0xffffffffu, v[j], 1);
+                        stage[lane * 17 + j] = merge ? fmaxf(v[j], nxt) : v[j];
+                    }
+                    __syncwarp();
+                    unsigned mask = emit_mask;
+                    while (mask) {
+                        const int i0 = __ffs(mask) - 1;
+                        mask &= mask - 1;
+                        int i1 = -1;
+                        if (mask) { i1 = __ffs(mask) - 1; mask &= mask - 1; }
+                        const int src = lane < 16 ? i0 : i1;
+                        const long long d = __shfl_sync(0xffffffffu, dst, src < 0 ? 0 : src);
+                        const int ch = lane & 15;
+                        if (src >= 0 && n0 + ch < p.N)
+                            atomicMax(out_u + d + n0 + ch, __float_as_uint(stage[src * 17 + ch]) & 0x7fffffffu);
+                    }
+                    __syncwarp();
                 }
             } else {
                 // conv + global average pool: channel sums over this warp's 32 pixels

@@ -445,3 +445,32 @@ def test_linear_row_sum_fp16_collapsed_and_not(fc, orc):
         ch = replace(wl.linear_row_reduce(256, 512, 256, "row_sum", ops=ops, variant="var"), in_dtype="f16", out_dtype="f16")
         ch = replace(ch, input_recipe=tuple((t, "f16", sh, d, a, b) for t, d0, sh, d, a, b in ch.input_recipe))
         run_and_check(fc, orc, ch, 10)
+
+
+# ------------------------------------------------------------------ conv -> ReLU -> 2x2 max-pool
+@pytest.mark.parametrize("batch,H,W,Cin,Cout,R,S,pad,stride", [
+    (2, 8, 8, 64, 64, 3, 3, 1, 1), (3, 12, 20, 64, 128, 5, 5, 2, 1), (2, 9, 7, 64, 40, 3, 3, 1, 1), (1, 56, 56, 64, 256, 3, 3, 1, 1),
+    (4, 5, 5, 72, 64, 1, 1, 0, 1), (2, 28, 28, 128, 64, 5, 5, 0, 1), (3, 17, 19, 64, 64, 3, 3, 1, 2), (5, 3, 2, 8, 8, 3, 3, 1, 1)])
+def test_conv_relu_maxpool(fc, orc, batch, H, W, Cin, Cout, R, S, pad, stride):
+    """Odd output sizes (dropped edge), windows that straddle warps and tiles, several images per tile."""
+    ch = wl.conv_bias_relu_maxpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, pad=pad, stride=stride)
+    for seed in (0, 1):
+        run_and_check(fc, orc, ch, seed)
+
+
+def test_conv_relu_maxpool_delta_kernel_is_pooled_relu_of_image(fc, orc):
+    """Centre-delta weights copy the image, so the output is the 2x2 max-pool of ReLU(image): compared
+    with numpy on the stored bf16 values, exactly."""
+    ch = replace(wl.conv_bias_relu_maxpool(batch=2, H=10, W=14, Cin=64, Cout=64, R=3, S=3, pad=1), ops=(("relu",),))
+    x = wl.make_inputs(ch, 3)[0]
+    outs, ref, _ = run_and_check(fc, orc, ch, ins=[x, _delta_weights(64, 1, 1)])
+    img = np.maximum(rng.bf16_bits_to_f32(x).astype(np.float64), 0.0)
+    want = img.reshape(2, 5, 2, 7, 2, 64).max(axis=(2, 4))
+    np.testing.assert_array_equal(util.to_f64(outs[0]), want)
+
+
+def test_maxpool_needs_relu_last(fc):
+    import ctypes
+    ch = replace(wl.conv_bias_relu_maxpool(), ops=(("bias_n", 2),))
+    n = ctypes.c_size_t(0)
+    assert fc.lib().fc_workspace_size(ctypes.byref(fc.make_spec(ch)), ctypes.byref(n)) == 3   # FC_ERR_UNSUPPORTED
