@@ -53,8 +53,9 @@ def load_peaks():
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each config's kernel, from the ncu
 # captures summarised under profiles/ (full config sizes; part of each output is still dirty in L2
 # when the kernel ends, so writes can read below the algorithmic output bytes).
-NCU_TRAFFIC_BYTES = {"C1": 541440, "C2": 268473344 + 99006208, "C3": 226910464 + 115290624,
-                     "C4": 68544000 + 12676608, "C5": 52659968 + 148992}
+NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268477184 + 95953152, "C3": 230077440 + 115409408,
+                     "C4": 67290112 + 9656320, "C5": 52669952 + 186624, "F1": 101696256 + 5212160,
+                     "F2": 134259968 + 4772096}   # F2: the weight pass, the dominant kernel of that workload
 
 
 def load_traffic(workload: str, full_size: bool):
