@@ -183,12 +183,16 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
     v[2] = unpack16x2(xq.z, f16);
     v[3] = unpack16x2(xq.w, f16);
     if (PRE != kPreNone) {
-        const float4 a0 = *reinterpret_cast<const float4*>(svec + c * 8);
-        const float4 a1 = *reinterpret_cast<const float4*>(svec + c * 8 + 4);
+        // shared-memory layout: the first and the second four columns of every chunk in separate arrays, so
+        // that consecutive lanes (consecutive chunks) read consecutive float4s: no bank conflicts
+        const int chunks = N >> 3;
+        const float4* sv = reinterpret_cast<const float4*>(svec);
+        const float4 a0 = sv[c];
+        const float4 a1 = sv[chunks + c];
         const float2 a[4] = {make_float2(a0.x, a0.y), make_float2(a0.z, a0.w), make_float2(a1.x, a1.y), make_float2(a1.z, a1.w)};
         if (PRE == kPreAffine) {
-            const float4 b0 = *reinterpret_cast<const float4*>(svec + N + c * 8);
-            const float4 b1 = *reinterpret_cast<const float4*>(svec + N + c * 8 + 4);
+            const float4 b0 = sv[2 * chunks + c];
+            const float4 b1 = sv[3 * chunks + c];
             const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
 #pragma unroll
             for (int j = 0; j < 4; ++j) v[j] = __ffma2_rn(v[j], a[j], b[j]);
@@ -261,12 +265,49 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
 
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
 __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams p) {
-    extern __shared__ float svec[];   // PRE != none: vec0 as fp32 [N], then vec1 [N]
+    extern __shared__ float svec[];   // PRE != none: vec0 as fp32 [N] (chunk halves de-interleaved), then vec1 [N]
     const int N = p.N;
     if (PRE != kPreNone) {
-        for (int i = threadIdx.x; i < N; i += kThreads) {
-            svec[i] = load_scalar(p.vec0, p.vec0_dt, i);
-            if (PRE == kPreAffine) svec[N + i] = load_scalar(p.vec1, p.vec1_dt, i);
+        // Every CTA converts the vectors once.  This prologue is a fixed cost of the launch (it measured 8 us
+        // with one scalar load per column and thread): 16-bit vectors that are 16-byte aligned are read
+        // eight columns per load, all loads of a thread issued before the first conversion.
+        const int nchunks = N >> 3;
+        float4* sv = reinterpret_cast<float4*>(svec);
+        const bool fast0 = p.vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(p.vec0) & 15) == 0;
+        const bool fast1 = PRE != kPreAffine || (p.vec1_dt != FC_F32 && (reinterpret_cast<uintptr_t>(p.vec1) & 15) == 0);
+        if (fast0 && fast1 && nchunks <= 4 * kThreads) {
+            uint4 q0[4], q1[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int c = threadIdx.x + k * kThreads;
+                if (c < nchunks) {
+                    q0[k] = __ldg(reinterpret_cast<const uint4*>(p.vec0) + c);
+                    if (PRE == kPreAffine) q1[k] = __ldg(reinterpret_cast<const uint4*>(p.vec1) + c);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int c = threadIdx.x + k * kThreads;
+                if (c < nchunks) {
+                    const bool h0 = p.vec0_dt == FC_F16;
+                    const float2 a = unpack16x2(q0[k].x, h0), b = unpack16x2(q0[k].y, h0), cc = unpack16x2(q0[k].z, h0), d = unpack16x2(q0[k].w, h0);
+                    sv[c] = make_float4(a.x, a.y, b.x, b.y);
+                    sv[nchunks + c] = make_float4(cc.x, cc.y, d.x, d.y);
+                    if (PRE == kPreAffine) {
+                        const bool h1 = p.vec1_dt == FC_F16;
+                        const float2 e = unpack16x2(q1[k].x, h1), f = unpack16x2(q1[k].y, h1), g = unpack16x2(q1[k].z, h1), h = unpack16x2(q1[k].w, h1);
+                        sv[2 * nchunks + c] = make_float4(e.x, e.y, f.x, f.y);
+                        sv[3 * nchunks + c] = make_float4(g.x, g.y, h.x, h.y);
+                    }
+                }
+            }
+        } else {
+            for (int i = threadIdx.x; i < N; i += kThreads) {
+                // column i = chunk i/8, half (i%8)/4, element i%4  ->  float4 number half * chunks + chunk
+                const int pos = ((((i >> 2) & 1) * nchunks) + (i >> 3)) * 4 + (i & 3);
+                svec[pos] = load_scalar(p.vec0, p.vec0_dt, i);
+                if (PRE == kPreAffine) svec[N + pos] = load_scalar(p.vec1, p.vec1_dt, i);
+            }
         }
         __syncthreads();
     }
