@@ -53,7 +53,7 @@ def load_peaks():
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each config's kernel, from the ncu
 # captures summarised under profiles/ (full config sizes; part of each output is still dirty in L2
 # when the kernel ends, so writes can read below the algorithmic output bytes).
-NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268477184 + 95953152, "C3": 230077440 + 115409408,
+NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268533248 + 98800896, "C3": 230077440 + 115409408,
                      "C4": 67290112 + 9656320, "C5": 52669952 + 186624, "F1": 101696256 + 5212160,
                      "F2": 134259968 + 4772096}   # F2: the weight pass, the dominant kernel of that workload
 
