@@ -326,6 +326,23 @@ __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, cons
     }
 }
 
+// One pass over this thread's half row of the accumulator in 16-column chunks, the load of chunk c + 1 in
+// flight while chunk c is processed.  f(c, r) may change r and store it back.
+template <int kChunks, class F>
+__device__ __forceinline__ void tmem_sweep(uint32_t tacc, F&& f) {
+    uint32_t ra[16], rb[16];
+    ptx::tmem_ld_32x16_async(tacc, ra);
+#pragma unroll 1
+    for (int c = 0; c < kChunks; c += 2) {
+        ptx::tmem_wait_ld(ra);
+        ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
+        f(c, ra);
+        ptx::tmem_wait_ld(rb);
+        if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
+        f(c + 1, rb);
+    }
+}
+
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
@@ -686,11 +703,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // when the list is not empty, so that the later sweeps read finished logits)
                 const bool has_ops = p.ops.n > 0;
                 float mx = -CUDART_INF_F;
-#pragma unroll 1
-                for (int c = 0; c < kChunks; ++c) {
-                    uint32_t r[16];
-                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
-                    ptx::tmem_wait_ld(r);
+                tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
                     if (has_ops) {
                         float v[16];
@@ -705,7 +718,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 16; ++j) mx = n0 + j < p.N ? fmaxf(mx, __uint_as_float(r[j])) : mx;
                     }
-                }
+                });
                 if (has_ops) ptx::tmem_wait_st();
                 // sweep B: e = 2^((v - max) log2 e), summed, and written back over the logits: the last sweep
                 // only rescales, so every element costs one exponential
@@ -714,11 +727,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const float2 l2e = make_float2(kLog2e, kLog2e);
                     const float2 moff = make_float2(-mx * kLog2e, -mx * kLog2e);
                     float2 acc2 = make_float2(0.0f, 0.0f);
-#pragma unroll 1
-                    for (int c = 0; c < kChunks; ++c) {
-                        uint32_t r[16];
-                        ptx::tmem_ld_32x16_async(tacc + c * 16, r);
-                        ptx::tmem_wait_ld(r);
+                    tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                         const int n0 = n_half + c * 16;
                         if (m < p.M && n0 < p.N) {
 #pragma unroll
@@ -733,7 +742,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             }
                         }
                         ptx::tmem_st_32x16(tacc + c * 16, r);
-                    }
+                    });
                     ptx::tmem_wait_st();
                     sm = acc2.x + acc2.y;
                 }
@@ -784,11 +793,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // last sweep: p = e * 2^((max_half - max_row) log2 e) / sum_row, one factor per thread
                 const float fac = m < p.M && store ? exp2_fast((mx - row_m) * kLog2e) / row_s : 0.0f;
                 const float2 fac2 = make_float2(fac, fac);
-#pragma unroll 1
-                for (int c = 0; c < kChunks; ++c) {
-                    uint32_t r[16];
-                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
-                    ptx::tmem_wait_ld(r);
+                tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
                     if (m < p.M && n0 < p.N && store) {
                         float v[16];
@@ -800,7 +805,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                         store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                     }
-                }
+                });
             } else if (p.pool == 1) {
                 // conv + 2x2 max-pool of non-negative values (the op list ends with ReLU, the output starts at
                 // zero): every pixel that lies in a window takes part in an unsigned atomic maximum on the fp32
