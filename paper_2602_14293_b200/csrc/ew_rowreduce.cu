@@ -407,17 +407,22 @@ static cudaError_t launch_fast(const EwFastParams& f, bool lse, bool store, int 
     int per_sm = smem > 0 ? (int) ((200 * 1024) / smem) : 4;
     per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);
     if (ctas > (long long) num_sms * per_sm) ctas = (long long) num_sms * per_sm;
-    auto go = [&](auto kernel) -> cudaError_t {
-        if (smem > 48 * 1024) {
-            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int) smem);
+    // the dynamic shared-memory limit of each instantiation is raised once per device, to the maximum
+    static bool raised[3][64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    auto go = [&](auto kernel, int variant) -> cudaError_t {
+        if (smem > 48 * 1024 && (dev < 0 || dev >= 64 || !raised[variant][dev])) {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
             if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < 64) raised[variant][dev] = true;
         }
         kernel<<<(unsigned) ctas, kThreads, smem, stream>>>(f);
         return cudaGetLastError();
     };
-    if (lse && store) return go(ew_rows_kernel<PRE, ACT, RES, true, true>);
-    if (lse) return go(ew_rows_kernel<PRE, ACT, RES, true, false>);
-    return go(ew_rows_kernel<PRE, ACT, RES, false, true>);
+    if (lse && store) return go(ew_rows_kernel<PRE, ACT, RES, true, true>, 0);
+    if (lse) return go(ew_rows_kernel<PRE, ACT, RES, true, false>, 1);
+    return go(ew_rows_kernel<PRE, ACT, RES, false, true>, 2);
 }
 
 cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t stream, int* launches) {

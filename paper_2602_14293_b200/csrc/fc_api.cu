@@ -366,7 +366,39 @@ cudaError_t clear_counters_if_needed(DeviceInfo* dev, const TcParams& p, size_t 
     return cudaSuccess;
 }
 
+// Tensor maps depend only on (pointer, extents, box, dtype): a step that runs the same chain on the same
+// buffers again finds them here instead of encoding them anew (a few of the microseconds of every call).
+struct MapKey {
+    const void* ptr;
+    long long d[8];   // extents and the other parameters the encoding depends on
+    bool operator==(const MapKey& o) const { return ptr == o.ptr && memcmp(d, o.d, sizeof(d)) == 0; }
+};
+struct MapCache {
+    static constexpr int kSlots = 16;
+    MapKey key[kSlots];
+    CUtensorMap map[kSlots];
+    bool used[kSlots] = {};
+    int next = 0;
+    std::mutex mu;
+    bool find(const MapKey& k, CUtensorMap* out) {
+        std::lock_guard<std::mutex> lk(mu);
+        for (int i = 0; i < kSlots; ++i)
+            if (used[i] && key[i] == k) { *out = map[i]; return true; }
+        return false;
+    }
+    void put(const MapKey& k, const CUtensorMap& m) {
+        std::lock_guard<std::mutex> lk(mu);
+        key[next] = k; map[next] = m; used[next] = true;
+        next = (next + 1) % kSlots;
+    }
+};
+MapCache g_maps;
+
 fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long cols, int box_rows, int dt = FC_BF16) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const MapKey mk = {ptr, {2, rows, cols, box_rows, dt, dev, 0, 0}};
+    if (g_maps.find(mk, tm)) return FC_OK;
     const cuuint64_t dims[2] = {(cuuint64_t) cols, (cuuint64_t) rows};
     const cuuint64_t strides[1] = {(cuuint64_t) cols * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t) box_rows};
@@ -375,10 +407,15 @@ fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long 
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d (rows %lld cols %lld)", (int) r, rows, cols);
+    g_maps.put(mk, *tm);
     return FC_OK;
 }
 
 fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const MapKey mk = {ptr, {4, s->batch * 65536 + dev, s->H, s->W, s->Cin, s->R * 64 + s->S, s->stride * 64 + s->pad, s->in_dtype}};
+    if (g_maps.find(mk, tm)) return FC_OK;
     const cuuint64_t dims[4] = {(cuuint64_t) s->Cin, (cuuint64_t) s->W, (cuuint64_t) s->H, (cuuint64_t) s->batch};
     const cuuint64_t strides[3] = {(cuuint64_t) s->Cin * 2, (cuuint64_t) s->W * s->Cin * 2, (cuuint64_t) s->H * s->W * s->Cin * 2};
     // base pixels run over the output grid shifted by -pad; a filter tap adds (s, r) to every base pixel
@@ -390,6 +427,7 @@ fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr
                                  64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeIm2col failed with CUresult %d", (int) r);
+    g_maps.put(mk, *tm);
     return FC_OK;
 }
 

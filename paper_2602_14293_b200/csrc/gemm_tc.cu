@@ -915,10 +915,16 @@ template <int BN, int MODE>
 cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int num_sms, cudaStream_t stream,
                        TcPlan* plan) {
     static int max_clusters[64] = {0};   // per device, filled on first use
+    static bool attr_set[64] = {false};  // per device: the dynamic shared-memory limit of this instantiation
     const int smem = Cfg<BN>::kSmemBytes;
     auto kernel = gemm_tc_kernel<BN, MODE>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -930,8 +936,6 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int dev = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && max_clusters[dev] == 0) {
         cfg.gridDim = dim3(num_sms & ~1);
         int n = 0;
