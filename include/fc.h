@@ -48,6 +48,8 @@
  * Testing aid.  With the environment variable FC_INJECT_PANEL_STALL=1, GEMM_NT + ROW_SOFTMAX launches
  * make their cross-tile wait expect an arrival that never comes: the bounded wait expires (about two
  * seconds), nothing is stored, and fc_get_async_status returns FC_ERR_TIMEOUT; the device stays usable.
+ * FC_INJECT_SPLIT_STALL=1 does the same to the other bounded wait that crosses CTAs, the one of a split
+ * tile's merging slice (GEMM_NT without softmax, with the split scratch registered).
  *
  * Threading.  fc_run may be called from several host threads.  The workspace set by
  * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM) must not

@@ -498,6 +498,10 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 // comes, so that the bounded wait expires and the call ends with FC_ERR_TIMEOUT
                 const char* inj = getenv("FC_INJECT_PANEL_STALL");
                 p.expect_extra = inj && inj[0] == '1' ? 1 : 0;
+            } else {
+                // testing only: FC_INJECT_SPLIT_STALL=1 does the same to the wait of a split tile's merging slice
+                const char* inj = getenv("FC_INJECT_SPLIT_STALL");
+                p.expect_extra = inj && inj[0] == '1' ? 1 : 0;
             }
             size_t panel_bytes = 0;
             if (p.mode == 1 || p.mode == 3) {

@@ -95,7 +95,8 @@ struct TcParams {
     float inv_hw;
     int pool;                   // mode 2: 0 global average pool, 1 2x2 max-pool (out pre-zeroed, values >= 0)
     int* status;                // device status word
-    int expect_extra;           // mode 1, testing only: arrivals the panel wait expects beyond those that will come
+    int expect_extra;           // testing only: arrivals a wait expects beyond those that will come (mode 1: the panel
+                                // wait; other modes: the wait of a split tile's merging slice)
     // Split tiles (filled by the launcher when the scratch below is given and a split pays): tiles from
     // split_from on are cut into `split` slices along K.
     int split, split_from, split_kb;   // split_kb: k-blocks of each parking slice; the merging slice takes the rest

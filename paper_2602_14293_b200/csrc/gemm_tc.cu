@@ -538,7 +538,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const unsigned long long t0 = ptx::globaltimer();
                     unsigned spins = 0;
                     bool ok = true;
-                    while (ptx::ld_acquire_gpu(cnt) < (unsigned) w.nsl - 1u) {
+                    while (ptx::ld_acquire_gpu(cnt) < (unsigned) (w.nsl - 1 + (MODE == 1 ? 0 : p.expect_extra))) {
                         if ((++spins & 63u) == 0) {
                             if (*abort_flag) { ok = false; break; }
                             if (ptx::globaltimer() - t0 > kWaitLimitNs) {
