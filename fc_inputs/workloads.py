@@ -40,7 +40,7 @@ class Chain:
     stride: int = 1
     pad: int = 1
     # ops: ("bias_n", i) ("affine_n", i, j) ("relu",) ("gelu_tanh",) ("scale", f) ("clamp", lo, hi)
-    #      ("add_tensor", i)   -- i, j index the input list
+    #      ("add_tensor", i) ("linear", i)   -- i, j index the input list
     ops: Tuple[tuple, ...] = ()
     reduce: str = "none"          # "none" | "row_logsumexp" | "row_softmax" | "global_avgpool" | "row_sum" | "row_max" | "row_mean" | "maxpool_2x2"
     store_main: bool = True
@@ -55,9 +55,23 @@ class Chain:
     def OW(self) -> int:
         return (self.W + 2 * self.pad - self.S) // self.stride + 1
 
+    @property
+    def widths(self):
+        """Output width after the producer and after every ("linear", i) op (gemm / elementwise chains)."""
+        w = [self.N]
+        for op in self.ops:
+            if op[0] == "linear":
+                w.append(self.input_recipe[op[1]][2][0])
+        return w
+
+    @property
+    def N_out(self) -> int:
+        return self.widths[-1]
+
     def flops(self) -> float:
         if self.producer == "gemm_nt":
-            return 2.0 * self.M * self.N * self.K
+            w = self.widths
+            return 2.0 * self.M * (self.N * self.K + sum(a * b for a, b in zip(w[:-1], w[1:])))
         if self.producer == "conv2d_nhwc":
             return 2.0 * self.batch * self.OH * self.OW * self.Cout * self.R * self.S * self.Cin
         return 0.0
@@ -128,6 +142,28 @@ def linear_row_reduce(M=1024, N=8192, K=8192, reduce="row_sum", ops=None, varian
                                ("bias", "bf16", (N,), "uniform", -0.1, 0.1),
                                ("gamma", "bf16", (N,), "normal", 1.0, 0.1),
                                ("beta", "bf16", (N,), "normal", 0.0, 0.1)))
+
+
+def mlp(M=4096, dims=(1024, 256, 256, 64), variant="std", act="relu", out_dtype="bf16") -> Chain:
+    """Back-to-back linear layers, x -> act(x W1^T + b1) -> act(. W2^T + b2) -> ... -> . WL^T + bL, with every
+    hidden width at most 256 so that a block of rows stays on chip from the first layer to the last (the
+    cross-layer fusion of the paper's Level-3 discussion; its appendix network ends in three such layers)."""
+    assert len(dims) >= 3
+    rec = [("x", "bf16", (M, dims[0]), "normal", 0.0, 1.0)]
+    ops = []
+    s0 = dims[0] ** -0.5 if variant == "std" else dims[0] ** -0.25
+    rec.append(("W1", "bf16", (dims[1], dims[0]), "normal", 0.0, s0))
+    rec.append(("b1", "bf16", (dims[1],), "uniform", -0.1, 0.1))
+    ops.append(("bias_n", 2))
+    for l in range(2, len(dims)):
+        ops.append((act,))
+        sl = (2.0 / dims[l - 1]) ** 0.5
+        rec.append((f"W{l}", "bf16", (dims[l], dims[l - 1]), "normal", 0.0, sl))
+        rec.append((f"b{l}", "bf16", (dims[l],), "uniform", -0.1, 0.1))
+        ops.append(("linear", len(rec) - 2))
+        ops.append(("bias_n", len(rec) - 1))
+    return Chain("mlp_bf16", "gemm_nt", "bf16", out_dtype, M=M, N=dims[1], K=dims[0], ops=tuple(ops), reduce="none",
+                 store_main=True, input_recipe=tuple(rec))
 
 
 def conv_bias_relu_avgpool(batch=32, H=56, W=56, Cin=256, Cout=256, R=3, S=3, stride=1, pad=1) -> Chain:
@@ -210,7 +246,7 @@ def output_shapes(chain: Chain):
     if chain.producer == "conv2d_nhwc":
         main_shape = (chain.batch, chain.OH, chain.OW, chain.Cout)
     else:
-        main_shape = (chain.M, chain.N)
+        main_shape = (chain.M, chain.N_out)
     if chain.reduce == "row_softmax":
         outs.append(("reduce", chain.out_dtype, main_shape))
         return outs

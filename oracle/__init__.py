@@ -156,6 +156,18 @@ def global_avgpool(V: np.ndarray) -> np.ndarray:
     return out
 
 
+def round_to(V: np.ndarray, dtype: str) -> np.ndarray:
+    """A copy of V rounded (nearest, ties to even) onto the grid of the storage type ('f32': unchanged)."""
+    out = np.ascontiguousarray(V, dtype=np.float64).copy()
+    if dtype == "bf16":
+        lib().orc_round_bf16(_p(out), _i64(out.size))
+    elif dtype == "f16":
+        lib().orc_round_f16(_p(out), _i64(out.size))
+    elif dtype != "f32":
+        raise ValueError(dtype)
+    return out
+
+
 def maxpool_2x2(V: np.ndarray) -> np.ndarray:
     NB, OH, OW, C = V.shape
     out = np.empty((NB, OH // 2, OW // 2, C), dtype=np.float64)
@@ -176,7 +188,11 @@ def run_chain(chain, inputs: List[np.ndarray]) -> Dict[str, np.ndarray]:
     else:
         raise ValueError(chain.producer)
     for op in chain.ops:
-        apply_op(V, op, x64)
+        if op[0] == "linear":
+            # the next contraction takes the activation as stored in the chain's 16-bit type
+            V = gemm_nt(round_to(V, chain.in_dtype), x64[op[1]])
+        else:
+            apply_op(V, op, x64)
     out = {"main": V}
     if chain.reduce == "row_logsumexp":
         out["reduce"] = row_logsumexp(V.reshape(-1, V.shape[-1]))

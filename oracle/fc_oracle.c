@@ -20,6 +20,9 @@
  *                      multiply).
  *   orc_row_logsumexp  max + log(sum exp(v - max)); over a row of length one this is the identity,
  *                      the closed form the paper's appendix (Level-2 Q18 analysis) relies on.
+ *   orc_round_bf16, orc_round_f16   round to nearest even onto the 16-bit grid: what a chain of linear
+ *                      layers does to an activation that it hands to the next contraction (the paper's
+ *                      appendix network keeps activations in the tensor dtype between layers).
  *   orc_maxpool_2x2    maximum over non-overlapping 2 x 2 windows, floor output size (the window
  *                      arithmetic of the paper's appendix max-pool listing with kernel 2, stride 2,
  *                      no padding, restated for NHWC).
@@ -32,7 +35,8 @@
  * exact-rational brute force with a different loop order on tiny shapes, centre and shifted delta
  * kernels, all-ones tap counts, high-precision (mpmath) values of GELU / logsumexp / softmax,
  * shift invariance, constant rows, rows summing to one, pooling linearity; max-pool against a
- * reshape-and-max in numpy, a single planted maximum per window, and dropped odd edges.
+ * reshape-and-max in numpy, a single planted maximum per window, and dropped odd edges; the 16-bit
+ * rounding against every stored pattern (identity), exact ties, and numpy's own conversions.
  */
 #include <math.h>
 #include <stdint.h>
@@ -75,6 +79,34 @@ void orc_widen_f16(const uint16_t* src, int64_t n, double* dst) {
 
 void orc_widen_f32(const float* src, int64_t n, double* dst) {
     for (int64_t i = 0; i < n; ++i) dst[i] = (double)src[i];
+}
+
+/* Round to nearest, ties to even, onto the grid of a binary floating-point format with `sig` significant
+ * bits, minimum (subnormal) exponent `emin_ulp` for the unit in the last place, and largest finite value
+ * `maxv` (values that round beyond it become infinite).  Used where a chain feeds a contraction with
+ * the output of a previous one: the tensor-core operand is the value as stored in the 16-bit type. */
+static double round_to_grid(double v, int sig, int emin_ulp, double maxv) {
+    if (v == 0.0 || isnan(v) || isinf(v)) return v;
+    int e;
+    (void) frexp(v, &e);                  /* |v| = f * 2^e, f in [0.5, 1)  ->  leading bit has weight 2^(e-1) */
+    int ulp_e = e - sig;                  /* weight of the last kept bit */
+    if (ulp_e < emin_ulp) ulp_e = emin_ulp;
+    const double q = nearbyint(ldexp(v, -ulp_e));   /* default rounding mode: to nearest, ties to even */
+    const double r = ldexp(q, ulp_e);
+    if (fabs(r) > maxv) return v < 0 ? -INFINITY : INFINITY;
+    return r;
+}
+
+/* bfloat16: 8 significant bits, smallest subnormal 2^-133, largest finite (2 - 2^-7) * 2^127 */
+void orc_round_bf16(double* V, int64_t count) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < count; ++i) V[i] = round_to_grid(V[i], 8, -133, 3.3895313892515355e38);
+}
+
+/* IEEE binary16: 11 significant bits, smallest subnormal 2^-24, largest finite 65504 */
+void orc_round_f16(double* V, int64_t count) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < count; ++i) V[i] = round_to_grid(V[i], 11, -24, 65504.0);
 }
 
 /* V[m][n] = sum_{k ascending} A[m][k] * B[n][k] */

@@ -124,3 +124,24 @@ def run_chain(chain, inputs):
         out["reduce"] = np.array([[float(mp.fsum(list(V4[b, :, c])) / (OH * OW)) for c in range(C)]
                                   for b in range(NB)])
     return out
+
+
+def round_to_grid_fraction(v: Fraction, sig: int, emin_ulp: int) -> Fraction:
+    """Nearest value with `sig` significant bits (ties to even), computed in exact rational arithmetic:
+    an independent restatement of the 16-bit rounding (no floating point involved)."""
+    if v == 0:
+        return v
+    a = abs(v)
+    e = 0                       # find e with 2^(e-1) <= a < 2^e
+    while Fraction(2) ** e <= a:
+        e += 1
+    while Fraction(2) ** (e - 1) > a:
+        e -= 1
+    ulp_e = max(e - sig, emin_ulp)
+    scaled = a / Fraction(2) ** ulp_e
+    q = scaled.numerator // scaled.denominator
+    rem = scaled - q
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and q % 2 == 1):
+        q += 1
+    r = q * Fraction(2) ** ulp_e
+    return r if v > 0 else -r

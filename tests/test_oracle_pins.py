@@ -334,3 +334,65 @@ def test_maxpool_2x2_against_reshape_and_planted_maxima(orc):
     assert np.array_equal(base, W[:, :4, :6].reshape(1, 2, 2, 3, 2, 2).max(axis=(2, 4)))
     # max commutes with a monotone map: pooling ReLU(V) equals ReLU of pooled V
     assert np.array_equal(orc.maxpool_2x2(np.maximum(V, 0)), np.maximum(orc.maxpool_2x2(V), 0))
+
+
+# ----------------------------------------------------------------------------- 16-bit rounding and chained linear layers
+def test_round_to_16_bit_grids(orc):
+    """Rounding onto the bf16 / fp16 grids: every stored pattern is a fixed point; numpy's and the input
+    generator's own conversions agree on random values; exact ties go to the even neighbour; an exact
+    rational restatement agrees on values with long fractions."""
+    pats = np.arange(65536, dtype=np.uint16)
+    w = orc.widen(pats)
+    fin = np.isfinite(w)
+    assert np.array_equal(orc.round_to(w[fin], "bf16"), w[fin])
+    h = pats.view(np.float16).astype(np.float64)
+    finh = np.isfinite(h)
+    assert np.array_equal(orc.round_to(h[finh], "f16"), h[finh])
+    r = np.random.default_rng(11)
+    x = (r.standard_normal(200000) * np.exp(r.uniform(-30, 30, 200000))).astype(np.float32)
+    want_bf16 = rng.bf16_bits_to_f32(rng.f32_to_bf16_bits(x)).astype(np.float64)       # integer bit arithmetic
+    assert np.array_equal(orc.round_to(x.astype(np.float64), "bf16"), want_bf16)
+    xs = (r.standard_normal(200000) * np.exp(r.uniform(-12, 10, 200000))).astype(np.float32)
+    with np.errstate(over="ignore"):
+        want_f16 = xs.astype(np.float16).astype(np.float64)                              # numpy's conversion
+    assert np.array_equal(orc.round_to(xs.astype(np.float64), "f16"), want_f16)
+    # ties: 1 + 2^-8 lies halfway between bf16 neighbours 1 and 1 + 2^-7 -> 1 (even); 1 + 3*2^-8 -> 1 + 2^-6
+    assert orc.round_to(np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, -(1 + 2.0 ** -8)]), "bf16").tolist() == [1.0, 1 + 2.0 ** -6, -1.0]
+    assert orc.round_to(np.array([1 + 2.0 ** -11, 1 + 3 * 2.0 ** -11]), "f16").tolist() == [1.0, 1 + 2.0 ** -9]
+    # just above a tie rounds up (a double rounding through fp32 would get this wrong)
+    assert orc.round_to(np.array([1 + 2.0 ** -8 + 2.0 ** -40]), "bf16")[0] == 1 + 2.0 ** -7
+    # subnormal and overflow ends of the fp16 grid
+    assert orc.round_to(np.array([2.0 ** -25, 3 * 2.0 ** -25, 65519.9, 65520.0]), "f16").tolist() == [0.0, 2.0 ** -23, 65504.0, np.inf]
+    from fractions import Fraction
+    for v in [0.3, -7.123456789, 1e-3, 255.5, 3.0e5]:
+        assert Fraction(float(orc.round_to(np.array([v]), "bf16")[0])) == brute.round_to_grid_fraction(Fraction(v), 8, -133)
+        if abs(v) < 65504:
+            assert Fraction(float(orc.round_to(np.array([v]), "f16")[0])) == brute.round_to_grid_fraction(Fraction(v), 11, -24)
+
+
+def test_chained_linear_layers(orc):
+    """x -> relu(x W1^T + b1) -> round to bf16 -> . W2^T + b2: identity second layer returns the rounded
+    activations; exact-rational brute force (different loop order, rational rounding) agrees to 1e-12."""
+    ch = wl.mlp(5, (16, 8, 8))
+    ins = wl.make_inputs(ch, 2)
+    ins[3] = rng.store(np.eye(8, dtype=np.float32), "bf16")
+    ins[4] = rng.store(np.zeros(8, np.float32), "bf16")
+    x = [orc.widen(a) for a in ins]
+    h = np.maximum(orc.gemm_nt(x[0], x[1]) + x[2], 0.0)
+    assert np.array_equal(orc.run_chain(ch, ins)["main"], orc.round_to(h, "bf16"))
+    from fractions import Fraction
+    ch = wl.mlp(3, (8, 8, 16, 8))
+    ins = wl.make_inputs(ch, 4)
+    got = orc.run_chain(ch, ins)["main"]
+    f = [brute.to_fraction_array(a) for a in ins]
+    v = brute.gemm_nt(f[0], f[1])
+    for l, (wi, bi) in enumerate([(1, 2), (3, 4), (5, 6)]):
+        if l > 0:
+            v = np.vectorize(lambda t: brute.round_to_grid_fraction(t, 8, -133), otypes=[object])(v)
+            v = brute.gemm_nt(v, f[wi])
+        v = v + f[bi][None, :]
+        if l < 2:
+            v = np.vectorize(lambda t: t if t > 0 else Fraction(0), otypes=[object])(v)
+    want = np.array([[float(t) for t in row] for row in v])
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    assert got.shape == (3, 8)
