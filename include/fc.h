@@ -65,8 +65,8 @@
 extern "C" {
 #endif
 
-#define FC_VERSION 1
-#define FC_MAX_OPS 8
+#define FC_VERSION 2    /* 2: FC_MAX_OPS 8 -> 12 (a four-layer chain with bias and activation needs ten ops) */
+#define FC_MAX_OPS 12
 
 typedef enum {
     FC_OK = 0,
@@ -92,7 +92,13 @@ typedef enum {
     FC_OP_GELU_TANH = 3,  /* v  = 0.5 v (1 + tanh(sqrt(2/pi) (v + 0.044715 v^3)))                    */
     FC_OP_SCALE = 4,      /* v *= f0                                                                 */
     FC_OP_CLAMP = 5,      /* v  = min(max(v, f0), f1)                                                */
-    FC_OP_ADD_TENSOR = 6  /* v += tensor[in0][m][n]              same shape as the main output       */
+    FC_OP_ADD_TENSOR = 6, /* v += tensor[in0][m][n]              same shape as the main output       */
+    FC_OP_LINEAR = 7      /* v[m][:] = round16(v[m][:]) W^T, W = inputs[in0] of shape [N_next][N] in the chain's 16-bit
+                             type: another linear layer.  The row is rounded to that type first (it is the tensor-core
+                             operand, and what an unfused sequence would have stored); N becomes N_next for the ops
+                             that follow.  16-bit GEMM_NT producer only, reduce NONE, every width (N and each N_next)
+                             a multiple of 8 and <= 256 so that a block of rows stays on chip, at most three LINEAR
+                             ops, no ADD_TENSOR: consecutive layers of the paper's appendix network                 */
 } fc_op_kind;
 
 typedef enum {
@@ -196,7 +202,7 @@ fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
 
 /*
  * Writes a one-line description of how fc_run would execute `spec` on the current device with the
- * workspace registered now: "kernel=ew_rowreduce", "kernel=gemm_f32", "kernel=collapse", or
+ * workspace registered now: "kernel=ew_rowreduce", "kernel=gemm_f32", "kernel=collapse", "kernel=mlp_tc", or
  * "kernel=gemm_tc mode=<0 store|1 softmax|2 conv+pool|3 logsumexp> bn=<tile width> tiles=<256 x bn tiles>
  * pairs=<CTA pairs launched> split=<slices per split tile, 1 = none> split_tiles=<tiles that are split>
  * split_kb=<64-wide k-blocks per parking slice>".  `text` is a caller-owned HOST buffer of `capacity`

@@ -18,10 +18,11 @@ LIB_PATH = os.path.join(PKG, "libfc.so")
 
 FC_F32, FC_BF16, FC_F16 = 0, 1, 2
 _PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2}
-_OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6}
+_OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6, "linear": 7}
 _REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3, "row_sum": 4, "row_max": 5, "row_mean": 6, "maxpool_2x2": 7}
 _DTYPE = {"f32": FC_F32, "bf16": FC_BF16, "f16": FC_F16}
-FC_MAX_OPS = 8
+FC_MAX_OPS = 12
+FC_VERSION = 2
 
 
 class fc_op(ctypes.Structure):
@@ -110,7 +111,7 @@ def make_spec(chain) -> fc_chain_spec:
     store_main; ops are tuples such as ("bias_n", 2) or ("clamp", -1.0, 1.0))."""
     s = fc_chain_spec()
     s.struct_size = ctypes.sizeof(fc_chain_spec)
-    s.version = 1
+    s.version = FC_VERSION
     s.producer = _PRODUCER[chain.producer]
     s.in_dtype = _DTYPE[chain.in_dtype]
     s.acc_dtype = FC_F32
@@ -121,7 +122,7 @@ def make_spec(chain) -> fc_chain_spec:
     for i, op in enumerate(chain.ops):
         o = s.ops[i]
         o.kind = _OPKIND[op[0]]
-        if op[0] in ("bias_n", "add_tensor"):
+        if op[0] in ("bias_n", "add_tensor", "linear"):
             o.in0 = int(op[1])
         elif op[0] == "affine_n":
             o.in0, o.in1 = int(op[1]), int(op[2])
@@ -274,7 +275,7 @@ def output_tensors(chain, device="cuda", pinned=False) -> List[torch.Tensor]:
         OW = (chain.W + 2 * chain.pad - chain.S) // chain.stride + 1
         main_shape = (chain.batch, OH, OW, chain.Cout)
     else:
-        main_shape = (chain.M, chain.N)
+        main_shape = (chain.M, getattr(chain, "N_out", chain.N))
     kw = dict(device=device, pin_memory=pinned) if device == "cpu" else dict(device=device)
     outs = []
     if chain.reduce == "row_softmax" or chain.store_main:

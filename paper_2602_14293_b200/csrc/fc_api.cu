@@ -97,7 +97,7 @@ bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16; }
 
 // ------------------------------------------------------------------------------- validation
 struct Plan {
-    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV, GEMM_COLLAPSE } kind;
+    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV, GEMM_COLLAPSE, TC_MLP } kind;
     long long out_rows, out_cols;  // main output viewed as [rows][cols]
     int n_prod_inputs;
     int n_outputs;
@@ -136,7 +136,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (s->reduce < 0 || s->reduce > FC_RED_MAXPOOL_2X2) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
     if (s->n_ops < 0 || s->n_ops > FC_MAX_OPS) return fail(FC_ERR_INVALID_SPEC, "n_ops %d out of range", s->n_ops);
     for (int i = 0; i < s->n_ops; ++i)
-        if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_ADD_TENSOR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
+        if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_LINEAR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
 
     plan->n_prod_inputs = s->producer == FC_PROD_ELEMENTWISE ? 1 : 2;
     if (s->producer == FC_PROD_CONV2D_NHWC) {
@@ -200,6 +200,26 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             plan->kind = Plan::TC_CONV;
             break;
     }
+    {
+        int linears = 0;
+        for (int i = 0; i < s->n_ops; ++i) linears += s->ops[i].kind == FC_OP_LINEAR;
+        if (linears > 0) {
+            if (plan->kind != Plan::TC_PLAIN)
+                return fail(FC_ERR_UNSUPPORTED, "LINEAR ops need a 16-bit GEMM_NT producer with reduce NONE");
+            if (linears > 3) return fail(FC_ERR_UNSUPPORTED, "at most three LINEAR ops (four layers)");
+            // per-layer limits that do not depend on the tensors; widths are checked with the tensors
+            int vecs = 0;
+            for (int i = 0; i < s->n_ops; ++i) {
+                const int k = s->ops[i].kind;
+                if (k == FC_OP_ADD_TENSOR) return fail(FC_ERR_UNSUPPORTED, "ADD_TENSOR cannot be combined with LINEAR ops");
+                if (k == FC_OP_LINEAR) vecs = 0;
+                vecs += k == FC_OP_BIAS_N ? 1 : (k == FC_OP_AFFINE_N ? 2 : 0);
+                if (vecs > 3) return fail(FC_ERR_UNSUPPORTED, "at most 3 per-column vector operands per layer");
+            }
+            if (s->N > 256 || s->N % 8) return fail(FC_ERR_UNSUPPORTED, "with LINEAR ops every layer width must be a multiple of 8 and <= 256 (N = %lld)", (long long) s->N);
+            plan->kind = Plan::TC_MLP;
+        }
+    }
     if (plan->kind == Plan::TC_PLAIN || plan->kind == Plan::TC_SOFTMAX || plan->kind == Plan::TC_LSE || plan->kind == Plan::TC_CONV) {
         int vecs = 0;
         for (int i = 0; i < s->n_ops; ++i) vecs += s->ops[i].kind == FC_OP_BIAS_N ? 1 : (s->ops[i].kind == FC_OP_AFFINE_N ? 2 : 0);
@@ -241,10 +261,24 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr)) & 15)
             return fail(FC_ERR_ALIGNMENT, "conv operands must be 16-byte aligned");
     }
+    long long cur_cols = plan.out_cols;   // width of a row at this point of the op list (LINEAR ops change it)
     for (int i = 0; i < s->n_ops; ++i) {
         const fc_op& op = s->ops[i];
         char what[64];
-        const long long vec[1] = {plan.out_cols};
+        if (op.kind == FC_OP_LINEAR) {
+            if (op.in0 < plan.n_prod_inputs || op.in0 >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, op.in0);
+            const fc_tensor& w = in[op.in0];
+            snprintf(what, sizeof(what), "inputs[%d] (op %d weights)", op.in0, i);
+            if (w.rank != 2 || w.shape[1] != cur_cols) return fail(FC_ERR_SHAPE, "%s: expected [N_next, %lld]", what, cur_cols);
+            const long long sw[2] = {w.shape[0], cur_cols};
+            if ((st = check_tensor(w, what, s->in_dtype, 2, sw))) return st;
+            if (w.shape[0] < 1 || w.shape[0] > 256 || w.shape[0] % 8)
+                return fail(FC_ERR_UNSUPPORTED, "%s: layer width %lld must be a multiple of 8 and <= 256", what, (long long) w.shape[0]);
+            if (reinterpret_cast<uintptr_t>(w.ptr) & 15) return fail(FC_ERR_ALIGNMENT, "%s must be 16-byte aligned", what);
+            cur_cols = w.shape[0];
+            continue;
+        }
+        const long long vec[1] = {cur_cols};
         if (op.kind == FC_OP_BIAS_N || op.kind == FC_OP_AFFINE_N) {
             const int idx[2] = {op.in0, op.in1};
             for (int k = 0; k < (op.kind == FC_OP_AFFINE_N ? 2 : 1); ++k) {
@@ -273,7 +307,7 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
             const long long sh[4] = {s->batch, OH, OW, s->Cout};
             if ((st = check_tensor(out[plan.main_index], "main output", s->out_dtype, 4, sh))) return st;
         } else {
-            const long long sh[2] = {s->M, s->N};
+            const long long sh[2] = {s->M, cur_cols};
             if ((st = check_tensor(out[plan.main_index], "main output", s->out_dtype, 2, sh))) return st;
         }
     }
@@ -291,6 +325,20 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         }
     }
     return FC_OK;
+}
+
+// fused form of an op list: [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]?
+void fused_from(const fc_op* ops, int n, const fc_tensor* in, FusedOps* out) {
+    FusedOps& f = *out;
+    memset(&f, 0, sizeof(f));
+    f.scale = 1.0f;
+    int i = 0;
+    if (i < n && (ops[i].kind == FC_OP_BIAS_N || ops[i].kind == FC_OP_AFFINE_N)) f.pre = ops[i++].kind == FC_OP_BIAS_N ? 1 : 2;
+    if (i < n && (ops[i].kind == FC_OP_RELU || ops[i].kind == FC_OP_GELU_TANH)) f.act = ops[i++].kind == FC_OP_RELU ? 1 : 2;
+    if (i < n && ops[i].kind == FC_OP_SCALE) f.scale = ops[i++].f0;
+    if (i < n && ops[i].kind == FC_OP_CLAMP) { f.clamp = 1; f.lo = ops[i].f0; f.hi = ops[i].f1; ++i; }
+    if (i < n && ops[i].kind == FC_OP_ADD_TENSOR) { f.res = 1; f.res_ptr = in[ops[i].in0].ptr; f.res_dt = in[ops[i].in0].dtype; ++i; }
+    f.valid = i == n;
 }
 
 void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
@@ -312,18 +360,7 @@ void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
             o.dt1 = in[op.in1].dtype;
         }
     }
-    // fused form: [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]?
-    FusedOps& f = d->fused;
-    memset(&f, 0, sizeof(f));
-    f.scale = 1.0f;
-    int i = 0;
-    const int n = s->n_ops;
-    if (i < n && (s->ops[i].kind == FC_OP_BIAS_N || s->ops[i].kind == FC_OP_AFFINE_N)) f.pre = s->ops[i++].kind == FC_OP_BIAS_N ? 1 : 2;
-    if (i < n && (s->ops[i].kind == FC_OP_RELU || s->ops[i].kind == FC_OP_GELU_TANH)) f.act = s->ops[i++].kind == FC_OP_RELU ? 1 : 2;
-    if (i < n && s->ops[i].kind == FC_OP_SCALE) f.scale = s->ops[i++].f0;
-    if (i < n && s->ops[i].kind == FC_OP_CLAMP) { f.clamp = 1; f.lo = s->ops[i].f0; f.hi = s->ops[i].f1; ++i; }
-    if (i < n && s->ops[i].kind == FC_OP_ADD_TENSOR) { f.res = 1; f.res_ptr = in[s->ops[i].in0].ptr; f.res_dt = in[s->ops[i].in0].dtype; ++i; }
-    f.valid = i == n;
+    fused_from(s->ops, s->n_ops, in, &d->fused);
 }
 
 constexpr int kSoftmaxBN = 256;
@@ -521,6 +558,50 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }
+        case Plan::TC_MLP: {
+            MlpParams p;
+            memset(&p, 0, sizeof(p));
+            p.M = (int) spec->M; p.K0 = (int) spec->K;
+            p.in_dt = spec->in_dtype;
+            p.out = outputs[plan.main_index].ptr; p.out_dt = spec->out_dtype;
+            p.status = dev->status;
+            p.width[0] = (int) spec->N;
+            CUtensorMap tmX, tmW[4];
+            auto box_rows = [](long long w) { return (int) ((w + 15) / 16 * 16); };   // the MMA's N step
+            if ((st = encode_2d(&tmX, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
+            if ((st = encode_2d(&tmW[0], inputs[1].ptr, spec->N, spec->K, box_rows(spec->N), spec->in_dtype))) return st;
+            int l = 0;
+            for (int i = 0; i < spec->n_ops; ++i) {
+                const fc_op& op = spec->ops[i];
+                if (op.kind == FC_OP_LINEAR) {
+                    const fc_tensor& w = inputs[op.in0];
+                    ++l;
+                    p.width[l] = (int) w.shape[0];
+                    if ((st = encode_2d(&tmW[l], w.ptr, w.shape[0], w.shape[1], box_rows(w.shape[0]), spec->in_dtype))) return st;
+                    continue;
+                }
+                DevOps& d = p.seg[l];
+                DevOp& o = d.op[d.n++];
+                o.kind = op.kind; o.f0 = op.f0; o.f1 = op.f1;
+                o.p0 = o.p1 = nullptr; o.dt0 = o.dt1 = FC_F32;
+                if (op.kind == FC_OP_BIAS_N || op.kind == FC_OP_AFFINE_N) { o.p0 = inputs[op.in0].ptr; o.dt0 = inputs[op.in0].dtype; }
+                if (op.kind == FC_OP_AFFINE_N) { o.p1 = inputs[op.in1].ptr; o.dt1 = inputs[op.in1].dtype; }
+            }
+            p.layers = l + 1;
+            {
+                // the packed straight-line form of each layer's ops, where the list has the usual shape
+                int first = 0;
+                for (int seg = 0, i = 0; i <= spec->n_ops; ++i) {
+                    if (i == spec->n_ops || spec->ops[i].kind == FC_OP_LINEAR) {
+                        fused_from(spec->ops + first, i - first, inputs, &p.seg[seg].fused);
+                        first = i + 1;
+                        ++seg;
+                    }
+                }
+            }
+            e = launch_mlp_tc(p, tmX, tmW, dev->num_sms, stream, &launches);
+            break;
+        }
         case Plan::GEMM_COLLAPSE: {
             const size_t need = collapse_workspace_bytes(spec->N, spec->K);
             if (!dev->workspace || dev->workspace_bytes < need)
@@ -629,7 +710,7 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
     // i-1 overlap (two internal copy streams; the kernels stay on the caller's stream).
     const bool conv = spec->producer == FC_PROD_CONV2D_NHWC;
     const long long rows = conv ? spec->batch : spec->M;
-    const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE) ? 256 : 1;
+    const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE) ? 256 : (plan.kind == Plan::TC_MLP ? 128 : 1);
     long long chunks = 1;
     if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && plan.kind != Plan::GEMM_COLLAPSE && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
         chunks = rows / gran < 8 ? rows / gran : 8;
@@ -744,6 +825,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     if (plan.kind == Plan::EW) { snprintf(text, capacity, "kernel=ew_rowreduce"); return FC_OK; }
     if (plan.kind == Plan::GEMM_F32) { snprintf(text, capacity, "kernel=gemm_f32"); return FC_OK; }
     if (plan.kind == Plan::GEMM_COLLAPSE) { snprintf(text, capacity, "kernel=collapse"); return FC_OK; }
+    if (plan.kind == Plan::TC_MLP) { snprintf(text, capacity, "kernel=mlp_tc"); return FC_OK; }
     DeviceInfo* dev;
     if ((st = get_device(&dev))) return st;
     TcParams p;

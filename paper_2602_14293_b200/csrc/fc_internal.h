@@ -111,6 +111,18 @@ cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUte
                            int bn, int num_sms, cudaStream_t stream, int* launches);
 size_t gemm_tc_smem_bytes(int bn);
 
+// Back-to-back linear layers kept on chip (mlp_tc.cu): layer l maps width[l-1] (K0 for l = 0) to width[l]
+struct MlpParams {
+    int M, K0, layers;          // 2..4 layers
+    int width[4];               // every width <= 256 and a multiple of 8
+    int in_dt;                  // FC_BF16 or FC_F16: storage of x, of every weight matrix and of the activations between layers
+    void* out; int out_dt;      // [M, width[layers-1]]
+    DevOps seg[4];              // ops applied to the accumulator of layer l (no ADD_TENSOR)
+    int* status;
+};
+cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUtensorMap* tmW, int num_sms, cudaStream_t stream,
+                          int* launches);
+
 // What launch_gemm_tc would do with `p` on the current device (no launch).
 struct TcPlan {
     int bn, tiles, pairs;       // tile width, 256 x bn output tiles, CTA pairs launched

@@ -1,0 +1,204 @@
+// Device code shared by the tensor-core kernels: the bounded mbarrier wait and the epilogue's op list
+// on 16 consecutive columns of one accumulator row.
+#pragma once
+
+#include "dev_common.cuh"
+#include "ptx.cuh"
+
+namespace fc {
+
+// Bounded mbarrier wait.  Returns false if the CTA is aborting (this or another wait expired).
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = ptx::globaltimer();
+    unsigned spins = 0;
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (ptx::globaltimer() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, kStatusTimeout);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// The op list applied to 16 consecutive columns (col0.. within the tile) of one row.  Per-column
+// vectors come from the shared-memory slices staged for this tile (slot order = order of the
+// vector operands in the op list); ADD_TENSOR reads global memory.
+// The fused form of the op list on 16 consecutive columns, in packed fp32x2 arithmetic.
+template <bool kPreciseGelu>
+__device__ __forceinline__ void fused_ops16(float (&v)[16], const FusedOps& f, const float* svec, int bn, int col0,
+                                            long long m, long long n0, long long n_limit, long long ld) {
+    float2 w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = make_float2(v[2 * j], v[2 * j + 1]);
+    if (f.pre != 0) {
+        const float4* a = reinterpret_cast<const float4*>(svec + col0);
+        if (f.pre == 1) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 t = a[q];
+                w[2 * q] = __fadd2_rn(w[2 * q], make_float2(t.x, t.y));
+                w[2 * q + 1] = __fadd2_rn(w[2 * q + 1], make_float2(t.z, t.w));
+            }
+        } else {
+            const float4* b = reinterpret_cast<const float4*>(svec + bn + col0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 g = a[q], t = b[q];
+                w[2 * q] = __ffma2_rn(w[2 * q], make_float2(g.x, g.y), make_float2(t.x, t.y));
+                w[2 * q + 1] = __ffma2_rn(w[2 * q + 1], make_float2(g.z, g.w), make_float2(t.z, t.w));
+            }
+        }
+    }
+    if (f.act == 2) {
+        if (kPreciseGelu) {
+            // gelu(t) * s = t * s / (1 + 2^(-2 z log2 e)),  z = sqrt(2/pi) (t + 0.044715 t^3)
+            constexpr float k0 = -2.0f * kLog2e * 0.7978845608028654f, k1 = k0 * 0.044715f;
+            const float2 sc = make_float2(f.scale, f.scale);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float2 t = w[j];
+                const float2 e = __fmul2_rn(t, __ffma2_rn(__fmul2_rn(t, t), make_float2(k1, k1), make_float2(k0, k0)));
+                const float2 d = __fadd2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), make_float2(1.0f, 1.0f));
+                float2 inv;
+                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.x) : "f"(d.x));
+                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.y) : "f"(d.y));
+                w[j] = __fmul2_rn(__fmul2_rn(t, sc), inv);
+            }
+        } else {
+            // gelu(t) * s = h + h tanh(z) with h = (0.5 s) t
+            constexpr float k0 = 0.7978845608028654f, k1 = k0 * 0.044715f;
+            const float hs = 0.5f * f.scale;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float2 t = w[j];
+                const float2 z = __fmul2_rn(t, __ffma2_rn(__fmul2_rn(t, t), make_float2(k1, k1), make_float2(k0, k0)));
+                const float2 h = __fmul2_rn(t, make_float2(hs, hs));
+                w[j] = __ffma2_rn(h, make_float2(tanh_fast(z.x), tanh_fast(z.y)), h);
+            }
+        }
+    } else {
+        if (f.act == 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = make_float2(w[j].x < 0.0f ? 0.0f : w[j].x, w[j].y < 0.0f ? 0.0f : w[j].y);
+        }
+        if (f.scale != 1.0f) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = __fmul2_rn(w[j], make_float2(f.scale, f.scale));
+        }
+    }
+    if (f.clamp) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            w[j] = make_float2(fminf(fmaxf(w[j].x, f.lo), f.hi), fminf(fmaxf(w[j].y, f.lo), f.hi));
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { v[2 * j] = w[j].x; v[2 * j + 1] = w[j].y; }
+    if (f.res) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (n0 + j < n_limit) v[j] += load_scalar(f.res_ptr, f.res_dt, m * ld + n0 + j);
+    }
+}
+
+template <bool kPreciseGelu>
+__device__ __forceinline__ void apply_ops16(float (&v)[16], const DevOps& ops, const float* svec, int bn, int col0,
+                                            long long m, long long n0, long long n_limit, long long ld) {
+    if (ops.fused.valid) {
+        fused_ops16<kPreciseGelu>(v, ops.fused, svec, bn, col0, m, n0, n_limit, ld);
+        return;
+    }
+    int slot = 0;
+#pragma unroll 1
+    for (int i = 0; i < ops.n; ++i) {
+        const DevOp& op = ops.op[i];
+        switch (op.kind) {
+            case FC_OP_BIAS_N: {
+                const float4* b = reinterpret_cast<const float4*>(svec + slot * bn + col0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 t = b[q];
+                    v[4 * q] += t.x; v[4 * q + 1] += t.y; v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
+                }
+                ++slot;
+                break;
+            }
+            case FC_OP_AFFINE_N: {
+                const float4* g = reinterpret_cast<const float4*>(svec + slot * bn + col0);
+                const float4* b = reinterpret_cast<const float4*>(svec + (slot + 1) * bn + col0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 s = g[q], t = b[q];
+                    v[4 * q] = fmaf(v[4 * q], s.x, t.x); v[4 * q + 1] = fmaf(v[4 * q + 1], s.y, t.y);
+                    v[4 * q + 2] = fmaf(v[4 * q + 2], s.z, t.z); v[4 * q + 3] = fmaf(v[4 * q + 3], s.w, t.w);
+                }
+                slot += 2;
+                break;
+            }
+            case FC_OP_RELU:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = v[j] < 0.0f ? 0.0f : v[j];
+                break;
+            case FC_OP_GELU_TANH:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = gelu_tanh<kPreciseGelu>(v[j]);
+                break;
+            case FC_OP_SCALE:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] *= op.f0;
+                break;
+            case FC_OP_CLAMP:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = fminf(fmaxf(v[j], op.f0), op.f1);
+                break;
+            case FC_OP_ADD_TENSOR:
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, m * ld + n0 + j);
+                break;
+            default:
+                break;
+        }
+    }
+}
+
+// 16 fp32 values of one row -> global memory as bf16 or fp32 (vector stores when aligned and in range)
+__device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, const float (&v)[16], long long m,
+                                        long long n0, long long N) {
+    if (out_dt != FC_F32) {
+        const bool f16 = out_dt == FC_F16;
+        unsigned short* o = (unsigned short*) out + m * N + n0;
+        if (vec_ok && n0 + 16 <= N) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint4 w;
+                w.x = pack16x2(v[8 * q + 0], v[8 * q + 1], f16);
+                w.y = pack16x2(v[8 * q + 2], v[8 * q + 3], f16);
+                w.z = pack16x2(v[8 * q + 4], v[8 * q + 5], f16);
+                w.w = pack16x2(v[8 * q + 6], v[8 * q + 7], f16);
+                reinterpret_cast<uint4*>(o)[q] = w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (n0 + j < N) o[j] = (unsigned short) (pack16x2(v[j], 0.0f, f16) & 0xffffu);
+        }
+    } else {
+        float* o = (float*) out + m * N + n0;
+        if (vec_ok && n0 + 16 <= N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                reinterpret_cast<float4*>(o)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (n0 + j < N) o[j] = v[j];
+        }
+    }
+}
+
+}  // namespace fc

@@ -35,7 +35,7 @@ def test_library_exports_every_declared_symbol(fc):
     assert {"fc_run", "fc_run_host", "fc_workspace_size", "fc_set_workspace", "fc_get_async_status"} <= names
     for n in names:
         assert hasattr(L, n), n
-    assert fc.fc_version() == 1
+    assert fc.fc_version() == 2
 
 
 def test_spec_struct_matches_header_size(fc):

@@ -73,3 +73,30 @@ def poison_(ts):
     for t in ts:
         t.fill_(float("nan"))
     return ts
+
+
+def check_chained(got_t: torch.Tensor, ref: np.ndarray, allowance: np.ndarray, what=""):
+    """Outputs of chained linear layers.  Between layers an activation is rounded to the 16-bit grid; where
+    its fp32 value lies within accumulation error of a rounding boundary, the kernel and the fp64 oracle may
+    legitimately pick neighbouring grid points (so would an unfused sequence).  `allowance[m][n]` bounds what
+    two such picks per hidden layer can do to output (m, n).  Criteria: the usual per-element bound of the
+    output type, widened by the allowance; at most 0.5 % of the elements may need the allowance at all; and
+    the mean absolute error keeps its usual bound (a systematic error cannot hide behind rare flips)."""
+    got = to_f64(got_t)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite values in the output"
+    err = np.abs(got - ref)
+    floor = 0.1 * float(np.sqrt(np.mean(ref * ref)))
+    if got_t.dtype == torch.float32:
+        base, mean_bound = 1e-4 * (1.0 + np.abs(ref)), None
+    else:
+        f16 = got_t.dtype == torch.float16
+        base = (2e-3 if f16 else 2e-2) * np.maximum(np.abs(ref), max(floor, 1e-30))
+        mean_bound = (2.5e-4 if f16 else 2e-3) * (1.0 if ref.size >= 256 else max(1.0, float(np.abs(ref).max())))
+    over = err > base
+    assert over.mean() <= 5e-3, f"{what}: {over.mean():.4%} of the elements exceed the plain bound"
+    worst = float((err / (base + allowance)).max())
+    assert worst <= 1.0, f"{what}: |err| / (bound + flip allowance) = {worst:.3f} at {np.unravel_index((err / (base + allowance)).argmax(), err.shape)}"
+    if mean_bound is not None:
+        assert float(err.mean()) <= mean_bound, f"{what}: mean abs err {float(err.mean()):.4g}"
+    return float(over.mean()), worst
