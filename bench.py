@@ -158,6 +158,13 @@ def eager_fn(ch, t):
         if ch.ops == (("bias_n", 2),):
             return lambda: red(F.linear(t[0], t[1], t[2]))
         return None
+    if name == "mlp_bf16":
+        def f():
+            h = F.linear(t[0], t[1], t[2])
+            for l in range(1, len(ch.widths)):
+                h = F.linear(torch.relu(h), t[1 + 2 * l], t[2 + 2 * l])
+            return h
+        return f
     if name == "gemm_bf16_row_softmax":
         return lambda: torch.softmax(t[0] @ t[1].t(), dim=1)
     if name == "conv_bf16_bias_relu_maxpool":
@@ -250,7 +257,10 @@ def cpu_baseline_leg(ch, ins, gpu_outputs=None, target_s=15.0):
             got = util.to_f64(t[:n])
             r = ref[name]
             worst[name] = float(np.abs(got - r).max())
-            util.check(t[:n], r, f"bench {ch.name}:{name}")
+            if any(op[0] == "linear" for op in ch.ops):
+                util.check_chained(t[:n], r, util.flip_allowance(oracle, sub, sub_ins), f"bench {ch.name}:{name}")
+            else:
+                util.check(t[:n], r, f"bench {ch.name}:{name}")
         out["parity_on_sample"] = {"ok": True, "max_abs_err": worst}
     return out
 

@@ -196,6 +196,7 @@ CONFIGS = {
 EXTRA = {
     "F1": lambda **kw: gemm_bias_scale_lse(**{"M": 4096, "N": 8192, "K": 4096, **kw}),
     "F2": lambda **kw: linear_row_reduce(**{"M": 1024, "N": 8192, "K": 8192, **kw}),
+    "F4": lambda **kw: mlp(**{"M": 16384, "dims": (1024, 256, 256, 64), **kw}),
     "F3": lambda **kw: conv_bias_relu_maxpool(**{"batch": 32, "H": 56, "W": 56, "Cin": 256, "Cout": 256, "R": 3, "S": 3, "pad": 1, **kw}),
 }
 ALL = {**CONFIGS, **EXTRA}

@@ -567,7 +567,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.status = dev->status;
             p.width[0] = (int) spec->N;
             CUtensorMap tmX, tmW[4];
-            auto box_rows = [](long long w) { return (int) ((w + 15) / 16 * 16); };   // the MMA's N step
+            auto box_rows = [](long long w) { return (int) ((w + 15) / 16 * 8); };   // each CTA of a pair loads half of the width padded to the MMA's N step
             if ((st = encode_2d(&tmX, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmW[0], inputs[1].ptr, spec->N, spec->K, box_rows(spec->N), spec->in_dtype))) return st;
             int l = 0;
@@ -710,7 +710,7 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
     // i-1 overlap (two internal copy streams; the kernels stay on the caller's stream).
     const bool conv = spec->producer == FC_PROD_CONV2D_NHWC;
     const long long rows = conv ? spec->batch : spec->M;
-    const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE) ? 256 : (plan.kind == Plan::TC_MLP ? 128 : 1);
+    const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_MLP) ? 256 : 1;
     long long chunks = 1;
     if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && plan.kind != Plan::GEMM_COLLAPSE && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
         chunks = rows / gran < 8 ? rows / gran : 8;

@@ -25,33 +25,6 @@ def fc():
     return fc
 
 
-def _flip_allowance(orc, ch, ins):
-    """What two neighbouring-grid-point picks per hidden layer can do to each output: for hidden layer l with
-    activations h (before rounding) and the remaining layers' weights W_{l+1} .. W_L, a pick moves h[m][k] by
-    one grid step ulp(h[m][k]) and output (m, n) by at most (|W_L| ... |W_{l+1}|)[n][k] ulp(h[m][k]) times the
-    activations' Lipschitz constant (1 for ReLU, below 1.13 for tanh-GELU)."""
-    x = [orc.widen(a) for a in ins]
-    sig = 8 if ch.in_dtype == "bf16" else 11
-    V = orc.gemm_nt(x[0], x[1])
-    hidden, weights = [], []
-    for op in ch.ops:
-        if op[0] == "linear":
-            hidden.append(V.copy())
-            weights.append(x[op[1]])
-            V = orc.gemm_nt(orc.round_to(V, ch.in_dtype), x[op[1]])
-        else:
-            orc.apply_op(V, op, x)
-    allowance = np.zeros_like(V)
-    for l, h in enumerate(hidden):
-        J = np.abs(weights[-1])
-        for w in reversed(weights[l:-1]):
-            J = 1.13 * (J @ np.abs(w))                      # [N_out, width of layer l]
-        with np.errstate(divide="ignore"):
-            ulp = np.where(h != 0, np.exp2(np.floor(np.log2(np.abs(h) + 1e-300)) - (sig - 1)), 0.0)
-        allowance += 2.0 * 1.13 * np.max(ulp[:, None, :] * J[None, :, :], axis=2)
-    return allowance
-
-
 def _run(fc, orc, ch, seed=0, ins=None):
     if ins is None:
         ins = wl.make_inputs(ch, seed)
@@ -62,7 +35,7 @@ def _run(fc, orc, ch, seed=0, ins=None):
         fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
     fc.fc_get_async_status()
     assert tuple(outs[0].shape) == ref["main"].shape
-    util.check_chained(outs[0], ref["main"], _flip_allowance(orc, ch, ins), f"{ch.name} {ch.widths} seed {seed}")
+    util.check_chained(outs[0], ref["main"], util.flip_allowance(orc, ch, ins), f"{ch.name} {ch.widths} seed {seed}")
     return outs, ref
 
 
