@@ -55,7 +55,8 @@ def load_peaks():
 # when the kernel ends, so writes can read below the algorithmic output bytes).
 NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268533248 + 98800896, "C3": 230077440 + 115409408,
                      "C4": 67290112 + 9656320, "C5": 52669952 + 186624, "F1": 101696256 + 5212160,
-                     "F2": 134259968 + 4772096}   # F2: the weight pass, the dominant kernel of that workload
+                     "F2": 134259968 + 4772096,   # F2: the weight pass, the dominant kernel of that workload
+                     "F3": 78327808 + 1775104, "F4": 34310912}
 
 
 def load_traffic(workload: str, full_size: bool):
