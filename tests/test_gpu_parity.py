@@ -358,7 +358,8 @@ def test_run_host_chunk_pipeline_matches_device_path(fc, orc):
     streams).  The results must equal those of the plain device path on the same inputs."""
     cases = [wl.affine_gelu_residual_lse(4100, 4096), wl.gemm_softmax(4096, 4096, 512, "var"),
              wl.gemm_bias_gelu_scale_clamp(4000, 4096, 512, "var"), wl.gemm_bias_scale_lse(4096, 4096, 512, "var", True),
-             wl.conv_bias_relu_avgpool(batch=20)]
+             wl.conv_bias_relu_avgpool(batch=20), wl.conv_bias_relu_maxpool(batch=24, H=56, W=56, Cin=128, Cout=64, R=3, S=3, pad=1),
+             wl.mlp(33000, (512, 256, 64)), wl.linear_row_reduce(20000, 1024, 1024)]
     for ch in cases:
         ins = wl.make_inputs(ch, 1)
         host_in = [fc.to_device(a, "cpu").pin_memory() for a in ins]
@@ -474,3 +475,9 @@ def test_maxpool_needs_relu_last(fc):
     ch = replace(wl.conv_bias_relu_maxpool(), ops=(("bias_n", 2),))
     n = ctypes.c_size_t(0)
     assert fc.lib().fc_workspace_size(ctypes.byref(fc.make_spec(ch)), ctypes.byref(n)) == 3   # FC_ERR_UNSUPPORTED
+
+
+def test_conv_relu_maxpool_fp16(fc, orc):
+    ch = wl.conv_bias_relu_maxpool(batch=3, H=12, W=20, Cin=64, Cout=128, R=3, S=3, pad=1)
+    ch = replace(ch, in_dtype="f16", input_recipe=tuple((t, "f16", sh, d, a, b) for t, _, sh, d, a, b in ch.input_recipe))
+    run_and_check(fc, orc, ch, 4)

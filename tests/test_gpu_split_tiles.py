@@ -110,6 +110,12 @@ def test_softmax_of_several_rounds_is_not_split(fc, orc):
     fc.binding.fc_set_workspace(None)
 
 
+def test_split_fp16(fc, orc):
+    ch = wl.gemm_bias_gelu_scale_clamp(192, 520, 4096, "var")
+    ch = replace(ch, in_dtype="f16", out_dtype="f16", input_recipe=tuple((t, "f16", sh, d, a, b) for t, _, sh, d, a, b in ch.input_recipe))
+    _run_both(fc, orc, ch, 16)
+
+
 def test_split_conv_5x5(fc, orc):
     _run_both(fc, orc, wl.conv_bias_relu_avgpool(batch=1, H=16, W=16, Cin=128, Cout=64, R=5, S=5, pad=2), 15)
 
