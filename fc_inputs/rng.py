@@ -130,12 +130,36 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def _e4m3_table():
+    """Value of each of the 127 non-negative finite E4M3 patterns (finite-only variant), ascending."""
+    b = np.arange(127)
+    e, f = b >> 3, b & 7
+    return np.where(e == 0, f * 2.0 ** -9, (8 + f) * 2.0 ** (e.astype(np.float64) - 10))
+
+
+def f32_to_e4m3_bits(a: np.ndarray) -> np.ndarray:
+    """Round fp32 values to 8-bit E4M3 (nearest, ties to the even pattern, magnitudes beyond 448 saturate)
+    and return the uint8 patterns."""
+    a = np.ascontiguousarray(a, dtype=np.float32).astype(np.float64)
+    tab = _e4m3_table()
+    mag = np.minimum(np.abs(a), tab[-1])
+    hi = np.clip(np.searchsorted(tab, mag, side="left"), 1, 126)
+    lo = hi - 1
+    dlo, dhi = mag - tab[lo], tab[hi] - mag
+    pick_hi = (dhi < dlo) | ((dhi == dlo) & (hi % 2 == 0))
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return np.where(np.signbit(a), code | np.uint8(0x80), code).astype(np.uint8)
+
+
 def store(a_f32: np.ndarray, dtype: str) -> np.ndarray:
-    """Round an fp32 array to the storage type: 'f32' -> float32, 'bf16' -> uint16 patterns, 'f16' -> float16."""
+    """Round an fp32 array to the storage type: 'f32' -> float32, 'bf16' -> uint16 patterns, 'f16' -> float16,
+    'f8e4m3' -> uint8 patterns."""
     if dtype == "f32":
         return np.ascontiguousarray(a_f32, dtype=np.float32)
     if dtype == "bf16":
         return f32_to_bf16_bits(a_f32)
     if dtype == "f16":
         return np.ascontiguousarray(a_f32, dtype=np.float32).astype(np.float16)   # IEEE half, round to nearest even
+    if dtype == "f8e4m3":
+        return f32_to_e4m3_bits(a_f32)
     raise ValueError(dtype)

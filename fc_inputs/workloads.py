@@ -78,6 +78,8 @@ class Chain:
 
 
 def _size(dtype: str) -> int:
+    if dtype == "f8e4m3":
+        return 1
     return 4 if dtype == "f32" else 2
 
 
@@ -106,6 +108,16 @@ def gemm_bias_gelu_scale_clamp(M=8192, N=8192, K=4096, variant="std") -> Chain:
                  ops=(("bias_n", 2), ("gelu_tanh",), ("scale", 0.5), ("clamp", -1.0, 1.0)),
                  input_recipe=(("A", "bf16", (M, K), "normal", 0.0, s),
                                ("B", "bf16", (N, K), "normal", 0.0, s),
+                               ("bias", "bf16", (N,), "uniform", -0.1, 0.1)))
+
+
+def gemm_f8_bias_gelu_scale_clamp(M=8192, N=8192, K=4096, out_dtype="bf16") -> Chain:
+    """C3's chain with both GEMM operands stored as 8-bit E4M3 floats (per-tensor scaling is the caller's: a
+    SCALE op in the epilogue undoes it).  Operand magnitudes sit in the middle of the E4M3 range."""
+    return Chain("gemm_f8e4m3_bias_gelu_scale_clamp", "gemm_nt", "f8e4m3", out_dtype, M=M, N=N, K=K,
+                 ops=(("scale", 1.0 / K ** 0.5), ("bias_n", 2), ("gelu_tanh",), ("scale", 0.5), ("clamp", -1.0, 1.0)),
+                 input_recipe=(("A", "f8e4m3", (M, K), "normal", 0.0, 1.0),
+                               ("B", "f8e4m3", (N, K), "normal", 0.0, 1.0),
                                ("bias", "bf16", (N,), "uniform", -0.1, 0.1)))
 
 
@@ -196,6 +208,7 @@ CONFIGS = {
 EXTRA = {
     "F1": lambda **kw: gemm_bias_scale_lse(**{"M": 4096, "N": 8192, "K": 4096, **kw}),
     "F2": lambda **kw: linear_row_reduce(**{"M": 1024, "N": 8192, "K": 8192, **kw}),
+    "F5": lambda **kw: gemm_f8_bias_gelu_scale_clamp(**kw),
     "F4": lambda **kw: mlp(**{"M": 16384, "dims": (1024, 256, 256, 64), **kw}),
     "F3": lambda **kw: conv_bias_relu_maxpool(**{"batch": 32, "H": 56, "W": 56, "Cin": 256, "Cout": 256, "R": 3, "S": 3, "pad": 1, **kw}),
 }

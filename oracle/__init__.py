@@ -54,10 +54,12 @@ def _p(a: np.ndarray):
 
 
 def widen(a: np.ndarray) -> np.ndarray:
-    """Stored tensor (float32, float16, or uint16 bf16 patterns) -> float64, exactly."""
+    """Stored tensor (float32, float16, uint16 bf16 patterns, or uint8 E4M3 patterns) -> float64, exactly."""
     a = np.ascontiguousarray(a)
     out = np.empty(a.shape, dtype=np.float64)
-    if a.dtype == np.uint16:
+    if a.dtype == np.uint8:
+        lib().orc_widen_f8e4m3(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
+    elif a.dtype == np.uint16:
         lib().orc_widen_bf16(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
     elif a.dtype == np.float16:
         lib().orc_widen_f16(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))

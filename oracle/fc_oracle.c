@@ -77,6 +77,20 @@ void orc_widen_f16(const uint16_t* src, int64_t n, double* dst) {
     }
 }
 
+/* 8-bit float E4M3 (finite-only variant: 1 sign, 4 exponent bits with bias 7, 3 fraction bits; exponent 0 is
+ * subnormal; the all-ones pattern of each sign is NaN, there are no infinities) -> double, exactly */
+void orc_widen_f8e4m3(const uint8_t* src, int64_t n, double* dst) {
+    for (int64_t i = 0; i < n; ++i) {
+        const uint8_t b = src[i];
+        const int sign = b >> 7, e = (b >> 3) & 15, f = b & 7;
+        double v;
+        if (e == 15 && f == 7) v = NAN;
+        else if (e == 0) v = ldexp((double) f, -9);           /* f/8 * 2^-6 */
+        else v = ldexp((double) (8 + f), e - 10);              /* (1 + f/8) * 2^(e-7) */
+        dst[i] = sign ? -v : v;
+    }
+}
+
 void orc_widen_f32(const float* src, int64_t n, double* dst) {
     for (int64_t i = 0; i < n; ++i) dst[i] = (double)src[i];
 }

@@ -396,3 +396,31 @@ def test_chained_linear_layers(orc):
     want = np.array([[float(t) for t in row] for row in v])
     np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
     assert got.shape == (3, 8)
+
+
+def test_widen_f8e4m3_all_patterns_and_generator_rounding(orc):
+    """All 256 E4M3 patterns against the library's own conversion (torch float8_e4m3fn), the closed form of a
+    few patterns, and the input generator's rounding against the library's on random values."""
+    pats = np.arange(256, dtype=np.uint8)
+    got = orc.widen(pats)
+    want = torch.from_numpy(pats).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.isnan(got).sum() == 2
+    assert np.array_equal(got[~np.isnan(got)], want[~np.isnan(want)])
+    assert got[0x01] == 2.0 ** -9 and got[0x08] == 2.0 ** -6 and got[0x38] == 1.0 and got[0x7E] == 448.0 and got[0xB8] == -1.0
+    r = np.random.default_rng(3)
+    x = np.clip(r.standard_normal(50000) * np.exp(r.uniform(-8, 5, 50000)), -440, 440).astype(np.float32)
+    assert np.array_equal(rng.f32_to_e4m3_bits(x), torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy())
+    assert rng.f32_to_e4m3_bits(np.array([2.0 ** -10, 3 * 2.0 ** -10, 1e4, -1e4], np.float32)).tolist() == [0, 2, 0x7E, 0xFE]
+
+
+def test_f8_gemm_chain_small_integers_and_brute_force(orc):
+    ch = wl.gemm_f8_bias_gelu_scale_clamp(4, 5, 16, out_dtype="f32")
+    ins = wl.make_inputs(ch, 1)
+    got = orc.run_chain(replace(ch, ops=()), ins)["main"]
+    a, b = orc.widen(ins[0]), orc.widen(ins[1])
+    np.testing.assert_allclose(got, a @ b.T, rtol=0, atol=1e-12)      # library matmul on the widened operands
+    from fractions import Fraction
+    fa = np.array([[Fraction(float(v)) for v in row] for row in a], dtype=object)
+    fb = np.array([[Fraction(float(v)) for v in row] for row in b], dtype=object)
+    exact = brute.gemm_nt(fa, fb)
+    assert all(Fraction(float(got[i, j])) == exact[i, j] for i in range(4) for j in range(5))   # 4-bit significands: exact in fp64
