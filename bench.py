@@ -56,7 +56,7 @@ def load_peaks():
 NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268533248 + 98800896, "C3": 230077440 + 115409408,
                      "C4": 67290112 + 9656320, "C5": 52669952 + 186624, "F1": 101696256 + 5212160,
                      "F2": 134259968 + 4772096,   # F2: the weight pass, the dominant kernel of that workload
-                     "F3": 78327808 + 1775104, "F4": 34310912}
+                     "F3": 78327808 + 1775104, "F4": 34310912, "F5": 74555136 + 96400128}
 
 
 def load_traffic(workload: str, full_size: bool):
@@ -69,11 +69,11 @@ def units(ch):
     """(metric name, unit, algorithmic units per step, roofline bound)."""
     if ch.producer == "elementwise" or wl.collapses(ch):
         return "fused_chain_throughput", "GB/s", wl.algorithmic_bytes(ch) / 1e9, "hbm"
-    return "fused_chain_throughput", "TFLOP/s", ch.flops() / 1e12, "tensor" if ch.in_dtype == "bf16" else "alu"
+    return "fused_chain_throughput", "TFLOP/s", ch.flops() / 1e12, "tensor" if ch.in_dtype in ("bf16", "f16", "f8e4m3") else "alu"
 
 
 def dtype_of(ch):
-    return "bf16" if ch.in_dtype == "bf16" else "f32"
+    return ch.in_dtype
 
 
 # ------------------------------------------------------------------------------ clocks
@@ -159,6 +159,16 @@ def eager_fn(ch, t):
         if ch.ops == (("bias_n", 2),):
             return lambda: red(F.linear(t[0], t[1], t[2]))
         return None
+    if name == "gemm_f8e4m3_bias_gelu_scale_clamp":
+        one = torch.ones((), device=t[0].device, dtype=torch.float32)
+        def f():
+            y = torch._scaled_mm(t[0], t[1].t(), scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+            return torch.clamp(F.gelu(y * (1.0 / ch.K ** 0.5) + t[2], approximate="tanh") * 0.5, -1.0, 1.0)
+        try:
+            f()
+        except Exception:
+            return None
+        return f
     if name == "mlp_bf16":
         def f():
             h = F.linear(t[0], t[1], t[2])
@@ -414,6 +424,9 @@ def main():
         peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
         peak_unit = "TFLOP/s"
         peak_note = f"cuBLAS bf16 {'sustained' if long_region else 'burst'}, {peaks_src}"
+        if ch.in_dtype == "f8e4m3":
+            peak *= 2.0   # no fp8 measurement on this machine: the measured bf16 peak times the nominal fp8 : bf16 ratio
+            peak_note += " x 2 (nominal fp8 : bf16 ratio)"
     else:
         peak, peak_unit = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
         peak_note = "fp32 FMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived)"

@@ -81,7 +81,15 @@ typedef enum {
     FC_ERR_TIMEOUT = 9        /* a bounded device-side wait expired                           */
 } fc_status;
 
-typedef enum { FC_F32 = 0, FC_BF16 = 1, FC_F16 = 2 } fc_dtype;   /* FC_F16: IEEE binary16, the storage type of the paper's kernels */
+typedef enum {
+    FC_F32 = 0,
+    FC_BF16 = 1,
+    FC_F16 = 2,       /* IEEE binary16, the storage type of the paper's kernels */
+    FC_F8E4M3 = 3     /* 8-bit float, 4 exponent bits (bias 7), 3 fraction bits, finite only (no infinities, all-ones is NaN):
+                         storage of BOTH operands of a GEMM_NT producer (fp32 accumulation on the tensor cores, K a multiple
+                         of 16); per-tensor scaling is the caller's, undone by a SCALE op.  Not an output, vector or
+                         residual type, not for ELEMENTWISE / CONV producers or LINEAR ops. */
+} fc_dtype;
 
 typedef enum { FC_PROD_ELEMENTWISE = 0, FC_PROD_GEMM_NT = 1, FC_PROD_CONV2D_NHWC = 2 } fc_producer;
 

@@ -92,8 +92,8 @@ fc_status get_device(DeviceInfo** out, int* dev_out = nullptr) {
     return FC_OK;
 }
 
-size_t dt_size(int dt) { return dt == FC_F32 ? 4 : 2; }
-bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16; }
+size_t dt_size(int dt) { return dt == FC_F32 ? 4 : (dt == FC_F8E4M3 ? 1 : 2); }
+bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16 || dt == FC_F8E4M3; }
 
 // ------------------------------------------------------------------------------- validation
 struct Plan {
@@ -133,6 +133,8 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (!dt_valid(s->in_dtype) || !dt_valid(s->out_dtype))
         return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
     if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
+    if (s->out_dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "FC_F8E4M3 is an operand type only (outputs are fp32, bf16 or fp16)");
+    if (s->in_dtype == FC_F8E4M3 && s->producer != FC_PROD_GEMM_NT) return fail(FC_ERR_UNSUPPORTED, "FC_F8E4M3 operands need a GEMM_NT producer");
     if (s->reduce < 0 || s->reduce > FC_RED_MAXPOOL_2X2) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
     if (s->n_ops < 0 || s->n_ops > FC_MAX_OPS) return fail(FC_ERR_INVALID_SPEC, "n_ops %d out of range", s->n_ops);
     for (int i = 0; i < s->n_ops; ++i)
@@ -177,7 +179,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
                 plan->kind = Plan::TC_LSE;   // any reduction of a row to one value
                 // A sum or mean over the output features of a purely linear epilogue, with no main output,
                 // commutes with the contraction: out = A (sum_n a[n] B[n][:]) + sum_n c[n]  (collapse.cu)
-                bool linear = (s->reduce == FC_RED_ROW_SUM || s->reduce == FC_RED_ROW_MEAN) && !s->store_main;
+                bool linear = (s->reduce == FC_RED_ROW_SUM || s->reduce == FC_RED_ROW_MEAN) && !s->store_main && s->in_dtype != FC_F8E4M3;
                 for (int i = 0; i < s->n_ops && linear; ++i)
                     linear = s->ops[i].kind == FC_OP_BIAS_N || s->ops[i].kind == FC_OP_AFFINE_N || s->ops[i].kind == FC_OP_SCALE;
                 if (linear) plan->kind = Plan::GEMM_COLLAPSE;
@@ -207,6 +209,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             if (plan->kind != Plan::TC_PLAIN)
                 return fail(FC_ERR_UNSUPPORTED, "LINEAR ops need a 16-bit GEMM_NT producer with reduce NONE");
             if (linears > 3) return fail(FC_ERR_UNSUPPORTED, "at most three LINEAR ops (four layers)");
+            if (s->in_dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "LINEAR ops need bf16 or fp16 operands");
             // per-layer limits that do not depend on the tensors; widths are checked with the tensors
             int vecs = 0;
             for (int i = 0; i < s->n_ops; ++i) {
@@ -249,7 +252,8 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         if ((st = check_tensor(in[0], "inputs[0] (A)", s->in_dtype, 2, sa))) return st;
         if ((st = check_tensor(in[1], "inputs[1] (B)", s->in_dtype, 2, sb))) return st;
         if (s->in_dtype != FC_F32) {
-            if (s->K % 8) return fail(FC_ERR_ALIGNMENT, "bf16 GEMM needs K %% 8 == 0 (K = %lld)", (long long) s->K);
+            const int kq = s->in_dtype == FC_F8E4M3 ? 16 : 8;   // a row of K elements must be a multiple of 16 bytes
+            if (s->K % kq) return fail(FC_ERR_ALIGNMENT, "this GEMM needs K %% %d == 0 (K = %lld)", kq, (long long) s->K);
             if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr)) & 15)
                 return fail(FC_ERR_ALIGNMENT, "bf16 GEMM operands must be 16-byte aligned");
         }
@@ -285,10 +289,12 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
                 if (idx[k] < plan.n_prod_inputs || idx[k] >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, idx[k]);
                 snprintf(what, sizeof(what), "inputs[%d] (op %d vector)", idx[k], i);
                 if ((st = check_tensor(in[idx[k]], what, -1, 1, vec))) return st;
+                if (in[idx[k]].dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "%s: FC_F8E4M3 vectors are not supported", what);
             }
         } else if (op.kind == FC_OP_ADD_TENSOR) {
             if (op.in0 < plan.n_prod_inputs || op.in0 >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, op.in0);
             snprintf(what, sizeof(what), "inputs[%d] (op %d tensor)", op.in0, i);
+            if (in[op.in0].dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "%s: FC_F8E4M3 tensors are not supported", what);
             if (s->producer == FC_PROD_CONV2D_NHWC) {
                 const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
                 const long long sh[4] = {s->batch, OH, OW, s->Cout};
@@ -436,11 +442,14 @@ fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long 
     cudaGetDevice(&dev);
     const MapKey mk = {ptr, {2, rows, cols, box_rows, dt, dev, 0, 0}};
     if (g_maps.find(mk, tm)) return FC_OK;
+    const cuuint64_t esize = dt == FC_F8E4M3 ? 1 : 2;
     const cuuint64_t dims[2] = {(cuuint64_t) cols, (cuuint64_t) rows};
-    const cuuint64_t strides[1] = {(cuuint64_t) cols * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t) box_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t) cols * esize};
+    const cuuint32_t box[2] = {(cuuint32_t) (128 / esize), (cuuint32_t) box_rows};   // 128-byte rows
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode_tiled(tm, dt == FC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+    const CUtensorMapDataType tdt = dt == FC_F8E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                    : (dt == FC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    CUresult r = g_encode_tiled(tm, tdt, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d (rows %lld cols %lld)", (int) r, rows, cols);
@@ -526,7 +535,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             const int bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
             {
                 // keep about 32 MB of A rows (group_m panels of 256 rows) resident in L2 per sweep
-                const long long panel_bytes = 256LL * spec->K * 2;
+                const long long panel_bytes = 256LL * spec->K * (long long) dt_size(spec->in_dtype);
                 long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
                 p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
             }

@@ -169,7 +169,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int tiles_n = (p.N + BN - 1) / BN;
     const int total_tiles = tiles_m * tiles_n;
     const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
-    const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + BK - 1) / BK;
+    const bool f8 = MODE != 2 && p.in_dt == FC_F8E4M3;
+    const int bk = f8 ? 2 * BK : BK;   // K elements per k-block: 128 bytes of a row
+    const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + bk - 1) / bk;
     const int total_units = p.split > 1 ? p.split_from + (total_tiles - p.split_from) * p.split : total_tiles;
 
     if (threadIdx.x == 0) {
@@ -231,8 +233,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap * p.Cin + c0, bcol0, full);
                     } else {
-                        ptx::tma_load_2d_pair(sa, &tmA, kb * BK, row0, full);
-                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * BK, bcol0, full);
+                        ptx::tma_load_2d_pair(sa, &tmA, kb * bk, row0, full);
+                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * bk, bcol0, full);
                     }
                 }
             }
@@ -240,7 +242,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (leader && lane == 0) {
-            const uint32_t idesc = ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_F16 ? 0u : 1u);
+            // operand format code: bf16 = 1 and fp16 = 0 under kind::f16, E4M3 = 0 under kind::f8f6f4
+            const uint32_t idesc = ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_BF16 ? 1u : 0u);
             uint32_t it = 0, tile_iter = 0;
             bool ok = true;
             for (int u = cluster_id; u < total_units && ok; u += num_clusters, ++tile_iter) {
@@ -255,9 +258,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tc_fence_after();
                     const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
                     const uint64_t da = ptx::smem_desc_k128(sa), db = ptx::smem_desc_k128(sa + C::kABytes);
+                    if (f8) {
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
-                        ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
+                        for (int k = 0; k < 4; ++k)  // 32 E4M3 values = 32 bytes per MMA along K -> +2 in 16-byte units
+                            ptx::tc_mma_f8_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
+                            ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
+                    }
                     ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);     // frees the stage in both CTAs
                 }
                 if (ok) ptx::tc_commit_pair(ptx::smem_u32(&ctrl->tfull[buf]), 3);   // accumulators ready in both CTAs
@@ -768,7 +777,8 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
         // Tiles left over after the full rounds (all of them, when there are fewer tiles than pairs) are cut
         // along K so that the last round keeps every pair busy.
         const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
-        const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + BK - 1) / BK;
+        const int bk = MODE != 2 && p.in_dt == FC_F8E4M3 ? 2 * BK : BK;
+        const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + bk - 1) / bk;
         const int full = tiles / max_pairs, tail = tiles - full * max_pairs;
         // (row softmax: only when everything fits one round; cutting the last of several rounds would let
         // row panels straddle rounds, which costs more than the split saves)
