@@ -105,7 +105,7 @@ typedef enum {
                              type: another linear layer.  The row is rounded to that type first (it is the tensor-core
                              operand, and what an unfused sequence would have stored); N becomes N_next for the ops
                              that follow.  16-bit GEMM_NT producer only, reduce NONE, every width (N and each N_next)
-                             a multiple of 8 and <= 256 so that a block of rows stays on chip, at most three LINEAR
+                             <= 256 so that a block of rows stays on chip and, except the last, a multiple of 8; at most three LINEAR
                              ops, no ADD_TENSOR: consecutive layers of the paper's appendix network                 */
 } fc_op_kind;
 

@@ -276,8 +276,10 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
             if (w.rank != 2 || w.shape[1] != cur_cols) return fail(FC_ERR_SHAPE, "%s: expected [N_next, %lld]", what, cur_cols);
             const long long sw[2] = {w.shape[0], cur_cols};
             if ((st = check_tensor(w, what, s->in_dtype, 2, sw))) return st;
-            if (w.shape[0] < 1 || w.shape[0] > 256 || w.shape[0] % 8)
-                return fail(FC_ERR_UNSUPPORTED, "%s: layer width %lld must be a multiple of 8 and <= 256", what, (long long) w.shape[0]);
+            bool more = false;   // another LINEAR follows: this width is the next weight matrix's row length
+            for (int j = i + 1; j < s->n_ops; ++j) more = more || s->ops[j].kind == FC_OP_LINEAR;
+            if (w.shape[0] < 1 || w.shape[0] > 256 || (more && w.shape[0] % 8))
+                return fail(FC_ERR_UNSUPPORTED, "%s: layer width %lld must be <= 256 and, unless it is the last, a multiple of 8", what, (long long) w.shape[0]);
             if (reinterpret_cast<uintptr_t>(w.ptr) & 15) return fail(FC_ERR_ALIGNMENT, "%s must be 16-byte aligned", what);
             cur_cols = w.shape[0];
             continue;

@@ -40,7 +40,7 @@ def _run(fc, orc, ch, seed=0, ins=None):
 
 
 @pytest.mark.parametrize("M,dims", [(128, (64, 64, 64)), (300, (64, 64, 64)), (1, (64, 16, 8)), (4096, (1024, 256, 256, 64)),
-                                    (777, (400, 120, 88, 16)), (2048, (136, 256, 8)), (640, (72, 40, 200, 96, 24)), (20000, (256, 32, 16))])
+                                    (777, (400, 120, 88, 16)), (2048, (136, 256, 8)), (640, (72, 40, 200, 96, 24)), (20000, (256, 32, 16)), (1000, (400, 120, 88, 10)), (300, (64, 64, 3))])
 def test_mlp_shapes(fc, orc, M, dims):
     _run(fc, orc, wl.mlp(M, dims, "std"), 1)
 
