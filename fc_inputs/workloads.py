@@ -24,7 +24,7 @@ from . import rng
 @dataclass(frozen=True)
 class Chain:
     name: str
-    producer: str                 # "elementwise" | "gemm_nt" | "conv2d_nhwc"
+    producer: str                 # "elementwise" | "gemm_nt" | "conv2d_nhwc" | "conv2d_nchw"
     in_dtype: str                 # "f32" | "bf16"  storage of inputs[0] (and inputs[1] for contractions)
     out_dtype: str                # storage of the main output (reductions other than softmax are f32)
     M: int = 0                    # elementwise: rows; gemm: rows of A
@@ -65,6 +65,10 @@ class Chain:
         return w
 
     @property
+    def is_conv(self) -> bool:
+        return self.producer in ("conv2d_nhwc", "conv2d_nchw")
+
+    @property
     def N_out(self) -> int:
         return self.widths[-1]
 
@@ -72,7 +76,7 @@ class Chain:
         if self.producer == "gemm_nt":
             w = self.widths
             return 2.0 * self.M * (self.N * self.K + sum(a * b for a, b in zip(w[:-1], w[1:])))
-        if self.producer == "conv2d_nhwc":
+        if self.is_conv:
             return 2.0 * self.batch * self.OH * self.OW * self.Cout * self.R * self.S * self.Cin
         return 0.0
 
@@ -195,6 +199,14 @@ def conv_bias_relu_maxpool(batch=8, H=32, W=32, Cin=64, Cout=128, R=5, S=5, stri
     return replace(base, name="conv_bf16_bias_relu_maxpool", reduce="maxpool_2x2")
 
 
+def conv_nchw(base: Chain) -> Chain:
+    """The same convolution chain with the image stored [batch, Cin, H, W] and the weights [Cout, Cin, R, S]
+    (the layouts of the paper's appendix listings); outputs are unchanged."""
+    (n0, d0, (b, H, W, Ci), *r0), (n1, d1, (Co, R, S, _), *r1) = base.input_recipe[0], base.input_recipe[1]
+    rec = ((n0, d0, (b, Ci, H, W), *r0), (n1, d1, (Co, Ci, R, S), *r1)) + tuple(base.input_recipe[2:])
+    return replace(base, name=base.name + "_nchw", producer="conv2d_nchw", input_recipe=rec)
+
+
 #: The five benchmark configurations, in the order the benchmark numbers them.
 CONFIGS = {
     "C1": gemm_bias_relu_f32,
@@ -257,7 +269,7 @@ def input_bytes(chain: Chain) -> int:
 def output_shapes(chain: Chain):
     """[(role, dtype, shape)] of the outputs, in output order: main first (if stored), then the reduction."""
     outs = []
-    if chain.producer == "conv2d_nhwc":
+    if chain.is_conv:
         main_shape = (chain.batch, chain.OH, chain.OW, chain.Cout)
     else:
         main_shape = (chain.M, chain.N_out)

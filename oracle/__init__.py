@@ -93,6 +93,19 @@ def conv2d_nhwc(x: np.ndarray, w: np.ndarray, stride: int, pad: int) -> np.ndarr
     return V
 
 
+def conv2d_nchw(x: np.ndarray, w: np.ndarray, stride: int, pad: int) -> np.ndarray:
+    """Image [NB, Cin, H, W], weights [Cout, Cin, R, S]; returns V[NB, OH, OW, Cout] (channels last)."""
+    NB, Cin, H, W = x.shape
+    Cout, Cin2, R, S = w.shape
+    assert Cin == Cin2
+    OH = (H + 2 * pad - R) // stride + 1
+    OW = (W + 2 * pad - S) // stride + 1
+    V = np.empty((NB, OH, OW, Cout), dtype=np.float64)
+    lib().orc_conv2d_nchw(_p(x), _p(w), _i64(NB), _i64(H), _i64(W), _i64(Cin), _i64(Cout),
+                          _i64(R), _i64(S), _i64(stride), _i64(pad), _p(V))
+    return V
+
+
 def apply_op(V: np.ndarray, op: tuple, inputs64: Sequence[np.ndarray]) -> None:
     """Apply one epilogue op in place to V (viewed as [rows, N] with N the last axis)."""
     L = lib()
@@ -187,6 +200,8 @@ def run_chain(chain, inputs: List[np.ndarray]) -> Dict[str, np.ndarray]:
         V = gemm_nt(x64[0], x64[1])
     elif chain.producer == "conv2d_nhwc":
         V = conv2d_nhwc(x64[0], x64[1], chain.stride, chain.pad)
+    elif chain.producer == "conv2d_nchw":
+        V = conv2d_nchw(x64[0], x64[1], chain.stride, chain.pad)
     else:
         raise ValueError(chain.producer)
     for op in chain.ops:

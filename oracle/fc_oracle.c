@@ -15,6 +15,8 @@
  *                      OH = (H + 2*pad - R)/stride + 1, input row = oh*stride - pad + r, taps that
  *                      fall outside the image contribute nothing (the indexing convention of the
  *                      paper's appendix convolution listing, restated for NHWC / [Cout][R][S][Cin]).
+ *   orc_conv2d_nchw    the same operation on the listing's own layouts, image [NB][Cin][H][W] and
+ *                      weights [Cout][Cin][R][S]; the output keeps channels last.
  *   orc_bias_n, orc_relu, orc_scale   bias broadcast over the output-feature / channel index, ReLU
  *                      as "negative -> 0", scaling by a scalar (the appendix epilogue: bias, ReLU,
  *                      multiply).
@@ -33,7 +35,8 @@
  *
  * Pins (tests, CPU only): identity / zero / rank-1 weights, exact small-integer contractions,
  * exact-rational brute force with a different loop order on tiny shapes, centre and shifted delta
- * kernels, all-ones tap counts, high-precision (mpmath) values of GELU / logsumexp / softmax,
+ * kernels, all-ones tap counts (both layouts; the channel-first form also against the library's
+ * convolution and against the channel-last form on permuted arrays), high-precision (mpmath) values of GELU / logsumexp / softmax,
  * shift invariance, constant rows, rows summing to one, pooling linearity; max-pool against a
  * reshape-and-max in numpy, a single planted maximum per window, and dropped odd edges; the 16-bit
  * rounding against every stored pattern (identity), exact ties, and numpy's own conversions.
@@ -156,6 +159,38 @@ void orc_conv2d_nhwc(const double* in, const double* Wt, int64_t NB, int64_t H, 
                             const double* px = in + ((b * H + ih) * W + iw) * Cin;
                             const double* wt = Wt + ((co * R + r) * S + s) * Cin;
                             for (int64_t ci = 0; ci < Cin; ++ci) acc += px[ci] * wt[ci];
+                        }
+                    }
+                    V[((b * OH + oh) * OW + ow) * Cout + co] = acc;
+                }
+            }
+        }
+    }
+}
+
+/* The same cross-correlation on the layouts the paper's appendix listing itself uses: image
+ * [NB][Cin][H][W], weights [Cout][Cin][R][S].  The result keeps the channel index last,
+ * V[NB][OH][OW][Cout], so that the epilogue ops and the pooling that follow see one layout. */
+void orc_conv2d_nchw(const double* in, const double* Wt, int64_t NB, int64_t H, int64_t W,
+                     int64_t Cin, int64_t Cout, int64_t R, int64_t S, int64_t stride, int64_t pad,
+                     double* V) {
+    const int64_t OH = (H + 2 * pad - R) / stride + 1;
+    const int64_t OW = (W + 2 * pad - S) / stride + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t b = 0; b < NB; ++b) {
+        for (int64_t co = 0; co < Cout; ++co) {
+            for (int64_t oh = 0; oh < OH; ++oh) {
+                for (int64_t ow = 0; ow < OW; ++ow) {
+                    double acc = 0.0;
+                    for (int64_t ci = 0; ci < Cin; ++ci) {
+                        for (int64_t r = 0; r < R; ++r) {
+                            const int64_t ih = oh * stride - pad + r;
+                            if (ih < 0 || ih >= H) continue;
+                            for (int64_t s = 0; s < S; ++s) {
+                                const int64_t iw = ow * stride - pad + s;
+                                if (iw < 0 || iw >= W) continue;
+                                acc += in[((b * Cin + ci) * H + ih) * W + iw] * Wt[((co * Cin + ci) * R + r) * S + s];
+                            }
                         }
                     }
                     V[((b * OH + oh) * OW + ow) * Cout + co] = acc;

@@ -75,6 +75,9 @@ def run_chain(chain, inputs):
         V = fr[0].copy()
     elif chain.producer == "gemm_nt":
         V = gemm_nt(fr[0], fr[1])
+    elif chain.producer == "conv2d_nchw":
+        # channel-first storage is a relabelling of the same numbers: move the axes, then the channel-last sum
+        V = conv2d_nhwc(fr[0].transpose(0, 2, 3, 1), fr[1].transpose(0, 2, 3, 1), chain.stride, chain.pad)
     else:
         V = conv2d_nhwc(fr[0], fr[1], chain.stride, chain.pad)
     shape = V.shape

@@ -167,6 +167,49 @@ def test_conv_chain_vs_exact_brute_force(orc):
     np.testing.assert_allclose(got["reduce"], want["reduce"], rtol=0, atol=1e-14)
 
 
+@pytest.mark.parametrize("stride,pad,H,W", [(1, 1, 6, 5), (2, 1, 7, 8), (1, 0, 5, 5), (2, 2, 6, 9)])
+def test_conv_nchw_matches_library_conv(orc, stride, pad, H, W):
+    """Channel-first storage: the library's convolution takes exactly these layouts, no permutation of the
+    inputs; only the result is moved to channels-last."""
+    x = _rand((2, 3, H, W), 14); w = _rand((4, 3, 3, 2), 15)
+    got = orc.conv2d_nchw(x, w, stride, pad)
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x), torch.from_numpy(w), stride=stride, padding=pad)
+    np.testing.assert_allclose(got, ref.permute(0, 2, 3, 1).numpy(), rtol=0, atol=1e-13)
+
+
+def test_conv_nchw_deltas_and_tap_counts(orc):
+    """A delta at (r, s) = (0, 2) in channel c -> c + 1 (cyclic): out[h][w][c+1] = in[c][h-1][w+1], zeros where the
+    tap leaves the image: pins the order of all four weight axes and of the image axes.  All-ones: valid taps."""
+    C, H, W = 3, 5, 7
+    x = _rand((2, C, H, W), 16)
+    w = np.zeros((C, C, 3, 3))
+    for c in range(C):
+        w[(c + 1) % C, c, 0, 2] = 1.0
+    y = orc.conv2d_nchw(x, w, 1, 1)
+    for c in range(C):
+        assert np.array_equal(y[:, 1:, :-1, (c + 1) % C], x[:, c, :-1, 1:])
+    assert np.count_nonzero(y[:, 0, :, :]) == 0 and np.count_nonzero(y[:, :, -1, :]) == 0
+    ones = orc.conv2d_nchw(np.ones((1, 4, 6, 5)), np.ones((2, 4, 3, 3)), 1, 1)
+    assert ones[0, 2, 2, 0] == 36 and ones[0, 0, 2, 1] == 24 and ones[0, 0, 0, 0] == 16 and ones[0, 5, 4, 1] == 16
+
+
+def test_conv_nchw_equals_nhwc_on_permuted_arrays(orc):
+    x = _rand((2, 5, 6, 7), 17); w = _rand((3, 5, 2, 3), 18)       # non-square filter, stride 2
+    a = orc.conv2d_nchw(x, w, 2, 1)
+    b = orc.conv2d_nhwc(np.ascontiguousarray(x.transpose(0, 2, 3, 1)), np.ascontiguousarray(w.transpose(0, 2, 3, 1)), 2, 1)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-14)
+
+
+def test_conv_nchw_chain_vs_exact_brute_force(orc):
+    ch = wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=2, H=4, W=5, Cin=3, Cout=2, R=3, S=3, pad=1))
+    ins = wl.make_inputs(ch, 5)
+    assert ins[0].shape == (2, 3, 4, 5) and ins[1].shape == (2, 3, 3, 3)
+    got = orc.run_chain(ch, ins)
+    want = brute.run_chain(ch, ins)
+    np.testing.assert_allclose(got["main"], want["main"], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(got["reduce"], want["reduce"], rtol=0, atol=1e-14)
+
+
 # ----------------------------------------------------------------------------- elementwise ops
 def test_relu_scale_clamp_exhaustive_bf16(orc):
     bits = np.arange(65536, dtype=np.uint16)
