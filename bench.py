@@ -182,6 +182,8 @@ def eager_fn(ch, t):
         x = t[0].permute(0, 3, 1, 2)
         w = t[1].permute(0, 3, 1, 2)
         return lambda: F.max_pool2d(torch.relu(F.conv2d(x, w, t[2], padding=ch.pad, stride=ch.stride)), 2).float()
+    if name == "conv_bf16_bias_relu_avgpool_nchw":   # contiguous channel-first storage, as torch keeps it by default
+        return lambda: F.adaptive_avg_pool2d(torch.relu(F.conv2d(t[0], t[1], t[2], padding=ch.pad)), 1).float()
     if name == "conv_bf16_bias_relu_avgpool":
         x = t[0].permute(0, 3, 1, 2)            # NHWC storage viewed as NCHW = channels_last
         w = t[1].permute(0, 3, 1, 2)
@@ -262,7 +264,7 @@ def cpu_baseline_leg(ch, ins, gpu_outputs=None, target_s=15.0):
     if gpu_outputs is not None:
         from tests import util
         names = [r for r, _, _ in wl.output_shapes(ch)]
-        n = sub.batch if ch.producer == "conv2d_nhwc" else sub.M
+        n = sub.batch if ch.is_conv else sub.M
         worst = {}
         for name, t in zip(names, gpu_outputs):
             got = util.to_f64(t[:n])
@@ -334,7 +336,7 @@ def main():
     peaks, peaks_src = load_peaks()
     ch = wl.ALL[args.workload]()
     if args.rows > 0:
-        ch = wl.ALL[args.workload](batch=args.rows) if ch.producer == "conv2d_nhwc" else wl.ALL[args.workload](M=args.rows)
+        ch = wl.ALL[args.workload](batch=args.rows) if ch.is_conv else wl.ALL[args.workload](M=args.rows)
     metric, unit, units_per_step, bound = units(ch)
     ins = wl.make_inputs(ch, seed=rk.batch_seed(0))   # every rank draws its own batch
     dev_in = [fc.to_device(a) for a in ins]

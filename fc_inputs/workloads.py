@@ -223,6 +223,7 @@ EXTRA = {
     "F5": lambda **kw: gemm_f8_bias_gelu_scale_clamp(**kw),
     "F4": lambda **kw: mlp(**{"M": 16384, "dims": (1024, 256, 256, 64), **kw}),
     "F3": lambda **kw: conv_bias_relu_maxpool(**{"batch": 32, "H": 56, "W": 56, "Cin": 256, "Cout": 256, "R": 3, "S": 3, "pad": 1, **kw}),
+    "F6": lambda **kw: conv_nchw(conv_bias_relu_avgpool(**kw)),
 }
 ALL = {**CONFIGS, **EXTRA}
 

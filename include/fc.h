@@ -14,6 +14,8 @@
  *              CONV2D_NHWC  v[b][oh][ow][co] = sum_{r,s,ci} in[b][oh*stride-pad+r][ow*stride-pad+s][ci]
  *                           * W[co][r][s][ci]   (cross-correlation, zero padding, floor output size,
  *                           as in the paper's appendix convolution kernel; layout restated for NHWC)
+ *              CONV2D_NCHW  the same sum on the appendix kernel's own layouts, in[b][ci][h][w] and
+ *                           W[co][ci][r][s]; outputs are the pooled ones, unchanged
  *   ops        bias over the last index, per-column affine, ReLU, tanh-GELU, scalar scale, clamp,
  *              add a tensor of the output's shape (bias -> ReLU -> scale is the paper's appendix
  *              epilogue; the others are named by this repository's benchmark configurations)
@@ -21,14 +23,15 @@
  *              row softmax, global average pool over (oh, ow)
  *
  * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
- * allocates device memory and never synchronises; it enqueues at most two memsets and one or two
+ * allocates device memory and never synchronises; it enqueues at most two memsets and one to three
  * kernels on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
  *
  * Pointers.  Unless a function says "host", every fc_tensor.ptr is a DEVICE pointer.
  *
  * Layout.  Row-major contiguous only (stride[] must describe exactly that, in elements).
  *   GEMM_NT: inputs[0] = A [M,K], inputs[1] = B [N,K].  CONV2D_NHWC: inputs[0] = image
- *   [batch,H,W,Cin], inputs[1] = weights [Cout,R,S,Cin].  ELEMENTWISE: inputs[0] = x [M,N].
+ *   [batch,H,W,Cin], inputs[1] = weights [Cout,R,S,Cin].  CONV2D_NCHW: inputs[0] = image [batch,Cin,H,W],
+ *   inputs[1] = weights [Cout,Cin,R,S].  ELEMENTWISE: inputs[0] = x [M,N].
  *   Further inputs are the vectors ([N] or [Cout]) and tensors that fc_op.in0 / in1 index.
  *   Outputs, in order: the main output (if store_main, or if reduce == ROW_SOFTMAX, whose
  *   probabilities take the main output's place), then the reduction (LOGSUMEXP / ROW_SUM / ROW_MAX /
@@ -52,7 +55,7 @@
  * tile's merging slice (GEMM_NT without softmax, with the split scratch registered).
  *
  * Threading.  fc_run may be called from several host threads.  The workspace set by
- * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM) must not
+ * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM, CONV2D_NCHW) must not
  * overlap on the device.
  */
 #ifndef FC_H_
@@ -91,7 +94,14 @@ typedef enum {
                          residual type, not for ELEMENTWISE / CONV producers or LINEAR ops. */
 } fc_dtype;
 
-typedef enum { FC_PROD_ELEMENTWISE = 0, FC_PROD_GEMM_NT = 1, FC_PROD_CONV2D_NHWC = 2 } fc_producer;
+typedef enum {
+    FC_PROD_ELEMENTWISE = 0,
+    FC_PROD_GEMM_NT = 1,
+    FC_PROD_CONV2D_NHWC = 2,
+    FC_PROD_CONV2D_NCHW = 3   /* image [batch,Cin,H,W], weights [Cout,Cin,R,S]: both are first rewritten channels-last into
+                                 the workspace (two transposition launches, fc_workspace_size reports the bytes: one copy
+                                 of each), then the CONV2D_NHWC kernel runs on the copies.  Same limits as CONV2D_NHWC. */
+} fc_producer;
 
 typedef enum {
     FC_OP_BIAS_N = 0,     /* v += vec[in0][n]                      n = last (column / channel) index */
@@ -178,8 +188,9 @@ fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, in
                           const fc_tensor* outputs, int n_outputs, size_t* bytes);
 
 /*
- * Scratch memory.  Only a 16-bit GEMM_NT with a row reduction needs any (per-tile partial results plus
- * per-panel arrival counters for the cross-tile merge; K + 1 doubles for the collapsed form, below).
+ * Scratch memory.  A 16-bit GEMM_NT with a row reduction needs some (per-tile partial results plus
+ * per-panel arrival counters for the cross-tile merge; K + 1 doubles for the collapsed form, below), and so
+ * does CONV2D_NCHW (the channels-last copies of image and weights).
  * fc_workspace_size reports
  * the bytes a spec needs (0 for the other chains); fc_set_workspace registers a caller-owned DEVICE
  * buffer (256-byte aligned) for the current device, used by later fc_run calls until replaced.

@@ -17,7 +17,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(PKG, "libfc.so")
 
 FC_F32, FC_BF16, FC_F16, FC_F8E4M3 = 0, 1, 2, 3
-_PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2}
+_PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2, "conv2d_nchw": 3}
 _OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6, "linear": 7}
 _REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3, "row_sum": 4, "row_max": 5, "row_mean": 6, "maxpool_2x2": 7}
 _DTYPE = {"f32": FC_F32, "bf16": FC_BF16, "f16": FC_F16, "f8e4m3": FC_F8E4M3}
@@ -248,10 +248,13 @@ def fc_describe_plan(spec) -> dict:
 
 
 def fc_set_workspace(buf: Optional[torch.Tensor]) -> None:
+    """Register `buf` (a uint8 device tensor, kept alive here) as the current device's workspace; None removes it."""
     if buf is None:
         _check(lib().fc_set_workspace(None, 0), "fc_set_workspace")
+        _workspace.pop(torch.cuda.current_device(), None)
     else:
         _check(lib().fc_set_workspace(ctypes.c_void_p(buf.data_ptr()), buf.numel() * buf.element_size()), "fc_set_workspace")
+        _workspace[buf.device.index] = buf
 
 
 def fc_get_async_status(stream=None) -> None:
@@ -274,7 +277,7 @@ def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
 
 def output_tensors(chain, device="cuda", pinned=False) -> List[torch.Tensor]:
     """Allocate (uninitialised) output tensors for `chain`, in the ABI's output order."""
-    if chain.producer == "conv2d_nhwc":
+    if chain.producer in ("conv2d_nhwc", "conv2d_nchw"):
         OH = (chain.H + 2 * chain.pad - chain.R) // chain.stride + 1
         OW = (chain.W + 2 * chain.pad - chain.S) // chain.stride + 1
         main_shape = (chain.batch, OH, OW, chain.Cout)

@@ -125,11 +125,19 @@ fc_status check_tensor(const fc_tensor& t, const char* what, int dtype_or_any, i
     return FC_OK;
 }
 
+bool is_conv(const fc_chain_spec* s) { return s->producer == FC_PROD_CONV2D_NHWC || s->producer == FC_PROD_CONV2D_NCHW; }
+
+// CONV2D_NCHW: channels-last copies of the image and of the weights at the head of the workspace
+size_t nchw_image_bytes(const fc_chain_spec* s) { return ((size_t) s->batch * s->H * s->W * s->Cin * 2 + 255) / 256 * 256; }
+size_t nchw_workspace_bytes(const fc_chain_spec* s) {
+    return nchw_image_bytes(s) + ((size_t) s->Cout * s->R * s->S * s->Cin * 2 + 255) / 256 * 256;
+}
+
 fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (!s) return fail(FC_ERR_NULL, "spec is null");
     if (s->struct_size != sizeof(fc_chain_spec)) return fail(FC_ERR_INVALID_SPEC, "struct_size %u, expected %zu", s->struct_size, sizeof(fc_chain_spec));
     if (s->version != FC_VERSION) return fail(FC_ERR_INVALID_SPEC, "version %u, expected %d", s->version, FC_VERSION);
-    if (s->producer < 0 || s->producer > FC_PROD_CONV2D_NHWC) return fail(FC_ERR_INVALID_SPEC, "unknown producer %d", s->producer);
+    if (s->producer < 0 || s->producer > FC_PROD_CONV2D_NCHW) return fail(FC_ERR_INVALID_SPEC, "unknown producer %d", s->producer);
     if (!dt_valid(s->in_dtype) || !dt_valid(s->out_dtype))
         return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
     if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
@@ -141,7 +149,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
         if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_LINEAR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
 
     plan->n_prod_inputs = s->producer == FC_PROD_ELEMENTWISE ? 1 : 2;
-    if (s->producer == FC_PROD_CONV2D_NHWC) {
+    if (is_conv(s)) {
         if (s->batch < 1 || s->H < 1 || s->W < 1 || s->Cin < 1 || s->Cout < 1 || s->R < 1 || s->S < 1 || s->stride < 1 || s->pad < 0)
             return fail(FC_ERR_SHAPE, "conv dimensions must be positive (pad >= 0)");
         const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
@@ -258,7 +266,9 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
                 return fail(FC_ERR_ALIGNMENT, "bf16 GEMM operands must be 16-byte aligned");
         }
     } else {
-        const long long si[4] = {s->batch, s->H, s->W, s->Cin}, sw[4] = {s->Cout, s->R, s->S, s->Cin};
+        const bool cf = s->producer == FC_PROD_CONV2D_NCHW;
+        const long long si[4] = {s->batch, cf ? s->Cin : s->H, cf ? s->H : s->W, cf ? s->W : s->Cin};
+        const long long sw[4] = {s->Cout, cf ? s->Cin : s->R, cf ? s->R : s->S, cf ? s->S : s->Cin};
         if ((st = check_tensor(in[0], "inputs[0] (image)", s->in_dtype, 4, si))) return st;
         if ((st = check_tensor(in[1], "inputs[1] (weights)", s->in_dtype, 4, sw))) return st;
         if (s->Cin % 8) return fail(FC_ERR_ALIGNMENT, "conv needs Cin %% 8 == 0 (Cin = %lld)", (long long) s->Cin);
@@ -297,7 +307,7 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
             if (op.in0 < plan.n_prod_inputs || op.in0 >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, op.in0);
             snprintf(what, sizeof(what), "inputs[%d] (op %d tensor)", op.in0, i);
             if (in[op.in0].dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "%s: FC_F8E4M3 tensors are not supported", what);
-            if (s->producer == FC_PROD_CONV2D_NHWC) {
+            if (is_conv(s)) {
                 const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
                 const long long sh[4] = {s->batch, OH, OW, s->Cout};
                 if ((st = check_tensor(in[op.in0], what, -1, 4, sh))) return st;
@@ -310,7 +320,7 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         }
     }
     if (plan.main_index >= 0) {
-        if (s->producer == FC_PROD_CONV2D_NHWC) {
+        if (is_conv(s)) {
             const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
             const long long sh[4] = {s->batch, OH, OW, s->Cout};
             if ((st = check_tensor(out[plan.main_index], "main output", s->out_dtype, 4, sh))) return st;
@@ -649,11 +659,31 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? 1 : 0;
             const size_t out_elems = p.pool ? (size_t) spec->batch * (p.OH / 2) * (p.OW / 2) * spec->Cout : (size_t) spec->batch * spec->Cout;
             if ((e = cudaMemsetAsync(p.out, 0, out_elems * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-            attach_split_scratch(dev, 0, &p);
+            const void* image = inputs[0].ptr;
+            const void* weights = inputs[1].ptr;
+            size_t head = 0;   // workspace bytes in front of the split scratch
+            if (spec->producer == FC_PROD_CONV2D_NCHW) {
+                head = nchw_workspace_bytes(spec);
+                if (!dev->workspace || dev->workspace_bytes < head)
+                    return fail(FC_ERR_WORKSPACE, "CONV2D_NCHW needs a workspace of %zu bytes (fc_workspace_size)", head);
+                void* img_cl = dev->workspace;
+                void* w_cl = (char*) dev->workspace + nchw_image_bytes(spec);
+                {   // the copies overwrite whatever counters a previous layout kept here
+                    std::lock_guard<std::mutex> lk(g_mu);
+                    dev->counter_layout = 0;
+                }
+                if ((e = launch_cfirst_to_clast(image, img_cl, spec->batch, p.Cin, p.H * p.W, stream, &launches)) != cudaSuccess)
+                    return cuda_fail(e, "layout kernel launch");
+                if ((e = launch_cfirst_to_clast(weights, w_cl, spec->Cout, p.Cin, p.R * p.S, stream, &launches)) != cudaSuccess)
+                    return cuda_fail(e, "layout kernel launch");
+                image = img_cl;
+                weights = w_cl;
+            }
+            attach_split_scratch(dev, head, &p);
             if ((e = clear_counters_if_needed(dev, p, 0, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;
-            if ((st = encode_im2col(&tmA, spec, inputs[0].ptr))) return st;
-            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->Cout, p.K, bn / 2, spec->in_dtype))) return st;
+            if ((st = encode_im2col(&tmA, spec, image))) return st;
+            if ((st = encode_2d(&tmB, weights, spec->Cout, p.K, bn / 2, spec->in_dtype))) return st;
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }
@@ -719,7 +749,7 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
     // Rows (images) are independent problems: large chains are cut into row chunks so that the
     // host-to-device copy of chunk i+1, the kernel of chunk i and the device-to-host copy of chunk
     // i-1 overlap (two internal copy streams; the kernels stay on the caller's stream).
-    const bool conv = spec->producer == FC_PROD_CONV2D_NHWC;
+    const bool conv = is_conv(spec);
     const long long rows = conv ? spec->batch : spec->M;
     const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_MLP) ? 256 : 1;
     long long chunks = 1;
@@ -813,7 +843,8 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
     if ((st = validate_spec(spec, &plan))) return st;
     *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N)
-           : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K) : 0;
+           : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K)
+           : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     return FC_OK;
 }
 
@@ -823,7 +854,8 @@ fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes) {
     if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
     if ((st = validate_spec(spec, &plan))) return st;
     const bool tc = plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_CONV;
-    const size_t red = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N) : 0;
+    const size_t red = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N)
+                     : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     *bytes = tc ? split_workspace_offset(red) + kTcSplitBytes : 0;
     return FC_OK;
 }
@@ -848,6 +880,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
         p.Cin = (int) spec->Cin; p.R = (int) spec->R; p.S = (int) spec->S;
         p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
         bn = spec->Cout <= 128 ? 128 : 256;
+        if (spec->producer == FC_PROD_CONV2D_NCHW) red = nchw_workspace_bytes(spec);
     } else {
         p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
         p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;

@@ -76,6 +76,9 @@ struct CollapseParams {
 cudaError_t launch_collapse(const CollapseParams& p, void* workspace, cudaStream_t stream, int* launches);
 size_t collapse_workspace_bytes(long long N, long long K);
 
+// Stack of `mats` 16-bit matrices [C][P] -> [P][C] (layout.cu): the channels-last rewrite for CONV2D_NCHW.  C even.
+cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, cudaStream_t stream, int* launches);
+
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
     int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row reduction to one value

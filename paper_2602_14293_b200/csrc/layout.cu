@@ -1,0 +1,86 @@
+// Channel-first -> channels-last rewrite of 16-bit tensors, the pre-pass of the CONV2D_NCHW producer.
+//
+// Both operands of the convolution are, per outer index, a [C][P] matrix that the tensor-core kernel wants as
+// [P][C]: the image per batch entry (P = H*W pixels) and the weights per output channel (P = R*S taps).  One
+// kernel transposes a stack of such matrices through a 64 x 64 shared-memory tile: reads are contiguous along P
+// (four pixels per load where the rows allow it), writes are contiguous along C (two channels per 32-bit store,
+// 128 bytes per warp; C is a multiple of 8 for the convolution).
+// HBM-bound: every element is read once and written once.
+#include "fc_internal.h"
+
+#include <cstdint>
+
+namespace fc {
+namespace {
+
+constexpr int kTile = 64;
+constexpr int kPitch = kTile + 2;   // 33 words per row: the column reads of the store phase touch each bank at most twice
+
+// kVec = 4: rows of P elements start on 8-byte boundaries (P % 4 == 0), four pixels per load; kVec = 1: any P.
+// All loads of a thread are issued before the first shared-memory store, so that a block keeps its whole
+// tile in flight instead of paying the memory latency once per row.
+template <int kVec>
+__global__ void __launch_bounds__(256) cfirst_to_clast_kernel(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
+                                                              int C, int P, int tiles_p) {
+    __shared__ __align__(16) unsigned short tile[kTile][kPitch];   // [c][p]
+    const long long mat = blockIdx.x / tiles_p;
+    const int p0 = (int) (blockIdx.x % tiles_p) * kTile, c0 = blockIdx.y * kTile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned short* s = src + mat * (long long) C * P;
+    unsigned short* d = dst + mat * (long long) C * P;
+    if constexpr (kVec == 4) {
+        const int pv = 4 * (threadIdx.x & 15), cr = threadIdx.x >> 4;
+        uint2 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = cr + 16 * i;
+            v[i] = make_uint2(0u, 0u);
+            if (c0 + c < C && p0 + pv < P) v[i] = *reinterpret_cast<const uint2*>(s + (long long) (c0 + c) * P + p0 + pv);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            unsigned int* w = reinterpret_cast<unsigned int*>(&tile[cr + 16 * i][pv]);
+            w[0] = v[i].x;
+            w[1] = v[i].y;
+        }
+    } else {
+        unsigned short v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = warp + 8 * (i >> 1), p = lane + 32 * (i & 1);
+            v[i] = 0;
+            if (c0 + c < C && p0 + p < P) v[i] = s[(long long) (c0 + c) * P + p0 + p];
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) tile[warp + 8 * (i >> 1)][lane + 32 * (i & 1)] = v[i];
+    }
+    __syncthreads();
+    const int c = 2 * lane;   // C is even: a pair of channels is either inside or outside
+    if (c0 + c < C) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int p = warp + 8 * i;
+            if (p0 + p < P) {
+                const unsigned int v = (unsigned int) tile[c][p] | ((unsigned int) tile[c + 1][p] << 16);
+                *reinterpret_cast<unsigned int*>(d + (long long) (p0 + p) * C + c0 + c) = v;
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, cudaStream_t stream, int* launches) {
+    const int tiles_p = (P + kTile - 1) / kTile;
+    const long long gx = mats * tiles_p;
+    if (gx > 0x7fffffffLL || (C & 1)) return cudaErrorInvalidValue;
+    dim3 grid((unsigned) gx, (unsigned) ((C + kTile - 1) / kTile));
+    if (P % 4 == 0 && reinterpret_cast<uintptr_t>(src) % 8 == 0)
+        cfirst_to_clast_kernel<4><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
+    else
+        cfirst_to_clast_kernel<1><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace fc

@@ -155,6 +155,23 @@ def test_workspace_sizes_of_split_and_collapsed_chains(fc):
     assert b.fc_workspace_size_split(col) == 0
 
 
+def test_workspace_size_of_channel_first_convolution(fc):
+    """CONV2D_NCHW keeps a channels-last copy of the image and of the weights, each rounded up to 256 bytes;
+    the optional split scratch follows them."""
+    b = fc.binding
+    base = wl.conv_bias_relu_avgpool(batch=3, H=7, W=9, Cin=8, Cout=24)
+    ch = wl.conv_nchw(base)
+    assert [r[2] for r in ch.input_recipe[:2]] == [(3, 8, 7, 9), (24, 8, 3, 3)]
+    assert wl.output_shapes(ch) == wl.output_shapes(base)
+    img = (3 * 7 * 9 * 8 * 2 + 255) // 256 * 256
+    wts = (24 * 3 * 3 * 8 * 2 + 255) // 256 * 256
+    spec = fc.make_spec(ch)
+    assert b.fc_workspace_size(spec) == img + wts
+    assert b.fc_workspace_size_split(spec) == img + wts + b.fc_workspace_size_split(fc.make_spec(base))
+    assert b.fc_workspace_size(fc.make_spec(base)) == 0
+    assert b.fc_describe_plan is not None
+
+
 def test_collapse_is_chosen_only_for_linear_epilogues_without_main_output():
     assert wl.collapses(wl.linear_row_reduce(64, 64, 64))
     assert wl.collapses(wl.linear_row_reduce(64, 64, 64, "row_mean", ops=(("affine_n", 3, 4), ("scale", 2.0))))

@@ -470,6 +470,64 @@ def test_conv_relu_maxpool_delta_kernel_is_pooled_relu_of_image(fc, orc):
     np.testing.assert_array_equal(util.to_f64(outs[0]), want)
 
 
+# ------------------------------------------------------------------ channel-first storage (CONV2D_NCHW)
+@pytest.mark.parametrize("batch,H,W,Cin,Cout,R,S,pad,stride", [
+    (2, 14, 14, 64, 128, 3, 3, 1, 1),
+    (3, 9, 13, 72, 40, 3, 3, 1, 1),        # pixels and channels that are no multiple of the 64-wide transposition tile
+    (1, 7, 7, 8, 8, 1, 1, 0, 1),           # one tap, fewest channels
+    (2, 23, 17, 136, 264, 5, 3, 2, 2),     # Cout over one 256-wide tile, strided, non-square filter
+    (70, 8, 8, 64, 64, 3, 3, 1, 1),
+])
+@pytest.mark.parametrize("pool", ["avg", "max"])
+def test_conv_channel_first(fc, orc, batch, H, W, Cin, Cout, R, S, pad, stride, pool):
+    make = wl.conv_bias_relu_avgpool if pool == "avg" else wl.conv_bias_relu_maxpool
+    ch = wl.conv_nchw(make(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, pad=pad, stride=stride))
+    if pool == "max" and (ch.OH < 2 or ch.OW < 2):
+        pytest.skip("no 2 x 2 window")
+    run_and_check(fc, orc, ch, 21)
+
+
+def test_conv_channel_first_equals_channel_last_bitwise(fc):
+    """The transposition moves bits: the pooled output of the channel-first chain is identical to the one of
+    the channels-last chain on the permuted arrays (avg-pool accumulates with atomics, so compare the
+    order-free max-pool)."""
+    base = wl.conv_bias_relu_maxpool(batch=4, H=20, W=12, Cin=72, Cout=136, R=3, S=3, pad=1)
+    ch = wl.conv_nchw(base)
+    ins = wl.make_inputs(ch, 3)
+    ins_cl = [np.ascontiguousarray(ins[0].transpose(0, 2, 3, 1)), np.ascontiguousarray(ins[1].transpose(0, 2, 3, 1))] + ins[2:]
+    a = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    b = util.poison_(fc.binding.output_tensors(base, "cuda"))
+    fc.run_chain(ch, [fc.to_device(x) for x in ins], a)
+    fc.run_chain(base, [fc.to_device(x) for x in ins_cl], b)
+    fc.fc_get_async_status()
+    assert torch.equal(a[0], b[0])
+
+
+def test_conv_channel_first_f16_and_host_path(fc, orc):
+    ch = _as_f16(wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=5, H=12, W=10, Cin=64, Cout=64)))
+    run_and_check(fc, orc, ch, 2)
+    ins = wl.make_inputs(ch, 2)
+    ref = orc.run_chain(ch, ins)
+    host_in = [fc.to_device(a, "cpu").pin_memory() for a in ins]
+    outs = util.poison_(fc.binding.output_tensors(ch, "cpu", pinned=True))
+    staging = torch.empty(fc.fc_staging_size(fc.make_spec(ch), host_in, outs), dtype=torch.uint8, device="cuda")
+    fc.run_chain_host(ch, host_in, outs, staging)
+    fc.fc_get_async_status()
+    util.check(outs[0], ref["reduce"], "channel-first conv through host buffers")
+
+
+def test_conv_channel_first_needs_workspace(fc):
+    ch = wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=2, H=8, W=8, Cin=64, Cout=64))
+    ins = [fc.to_device(a) for a in wl.make_inputs(ch, 0)]
+    outs = fc.binding.output_tensors(ch, "cuda")
+    spec = fc.make_spec(ch)
+    tiny = torch.empty(256, dtype=torch.uint8, device="cuda")
+    fc.binding.fc_set_workspace(tiny)
+    with pytest.raises(fc.FcError) as e:
+        fc.binding.fc_run(spec, ins, outs)
+    assert e.value.status == 6                        # FC_ERR_WORKSPACE
+
+
 def test_maxpool_needs_relu_last(fc):
     import ctypes
     ch = replace(wl.conv_bias_relu_maxpool(), ops=(("bias_n", 2),))
