@@ -639,40 +639,51 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         emit = even || lane == 0;       // an odd pixel is covered by its left neighbour, if this warp has it
                     }
                 }
+                // Emission slots: in slot k lanes 0-15 serve the (2k)-th emitting pixel of this warp and lanes
+                // 16-31 the (2k+1)-th, one channel per lane.  Which pixel that is, whether its right neighbour is
+                // merged in, and the window it updates do not depend on the channel chunk: found once per tile.
                 const unsigned emit_mask = __ballot_sync(0xffffffffu, emit);
+                const unsigned merge_mask = __ballot_sync(0xffffffffu, merge);
+                constexpr int kSlots = 9;                  // at most 17 emitters: 16 even pixels and an odd one in lane 0
+                const int n_slots = (__popc(emit_mask) + 1) >> 1;
+                const int win = (int) (dst / p.N);         // window index, below 2^31 like the pixel index
+                int slot_win[kSlots];
+                unsigned long long slot_src = 0;           // 7 bits per slot: source lane, merge flag, valid flag
+#pragma unroll
+                for (int k = 0; k < kSlots; ++k) {
+                    const unsigned src = __fns(emit_mask, 0, 2 * k + (lane >> 4) + 1);   // 0xffffffff: no such pixel
+                    const bool ok = src < 32u;
+                    slot_win[k] = __shfl_sync(0xffffffffu, win, ok ? (int) src : 0);
+                    const unsigned code = ok ? (src | ((merge_mask >> src & 1u) << 5) | 64u) : 0u;
+                    slot_src |= (unsigned long long) code << (7 * k);
+                }
                 float* stage = pool_stage + (warp - 2) * (32 * 17);
                 unsigned int* out_u = (unsigned int*) p.out;
-#pragma unroll 1
-                for (int c = 0; c < kChunks; ++c) {
-                    uint32_t r[16];
-                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
-                    ptx::tmem_wait_ld(r);
+                const int ch = lane & 15;
+                tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
-                    if (n0 >= p.N) continue;
+                    if (n0 >= p.N) return;
                     float v[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
                     if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float nxt = __shfl_down_sync(0xffffffffu, v[j], 1);
-                        stage[lane * 17 + j] = merge ? fmaxf(v[j], nxt) : v[j];
+                    for (int j = 0; j < 16; ++j) stage[lane * 17 + j] = v[j];
+                    __syncwarp();
+#pragma unroll
+                    for (int k = 0; k < kSlots; ++k) {
+                        if (k < n_slots) {
+                            const unsigned code = (unsigned) (slot_src >> (7 * k)) & 127u;
+                            const int src = code & 31u;
+                            if ((code & 64u) && n0 + ch < p.N) {
+                                float x = stage[src * 17 + ch];
+                                if (code & 32u) x = fmaxf(x, stage[(src + 1) * 17 + ch]);
+                                atomicMax(out_u + (long long) slot_win[k] * p.N + n0 + ch, __float_as_uint(x) & 0x7fffffffu);
+                            }
+                        }
                     }
                     __syncwarp();
-                    unsigned mask = emit_mask;
-                    while (mask) {
-                        const int i0 = __ffs(mask) - 1;
-                        mask &= mask - 1;
-                        int i1 = -1;
-                        if (mask) { i1 = __ffs(mask) - 1; mask &= mask - 1; }
-                        const int src = lane < 16 ? i0 : i1;
-                        const long long d = __shfl_sync(0xffffffffu, dst, src < 0 ? 0 : src);
-                        const int ch = lane & 15;
-                        if (src >= 0 && n0 + ch < p.N)
-                            atomicMax(out_u + d + n0 + ch, __float_as_uint(stage[src * 17 + ch]) & 0x7fffffffu);
-                    }
-                    __syncwarp();
-                }
+                });
             } else {
                 // conv + global average pool: channel sums over this warp's 32 pixels
                 const int hw = p.OH * p.OW;
