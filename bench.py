@@ -56,7 +56,7 @@ def load_peaks():
 NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268533248 + 98800896, "C3": 230077440 + 115409408,
                      "C4": 67290112 + 9656320, "C5": 52669952 + 186624, "F1": 101696256 + 5212160,
                      "F2": 134259968 + 4772096,   # F2: the weight pass, the dominant kernel of that workload
-                     "F3": 78327808 + 1775104, "F4": 34310912, "F5": 74555136 + 96400128}
+                     "F3": 78334720 + 1789696, "F4": 34311424, "F5": 74555136 + 96400128}
 
 
 def load_traffic(workload: str, full_size: bool):

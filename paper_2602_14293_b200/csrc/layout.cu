@@ -16,7 +16,9 @@ namespace {
 constexpr int kTile = 64;
 constexpr int kPitch = kTile + 2;   // 33 words per row: the column reads of the store phase touch each bank at most twice
 
-// kVec = 4: rows of P elements start on 8-byte boundaries (P % 4 == 0), four pixels per load; kVec = 1: any P.
+// kVec = 4: rows of P elements start on 8-byte boundaries (P % 4 == 0), four pixels per load; kVec = 1: any P;
+// kVec = 0: P <= 64 (filter taps), where the 64 rows of a tile are one contiguous run of 64 P elements that is
+// copied linearly (pitch P in shared memory) instead of row by row with most lanes idle.
 // All loads of a thread are issued before the first shared-memory store, so that a block keeps its whole
 // tile in flight instead of paying the memory latency once per row.
 template <int kVec>
@@ -43,6 +45,19 @@ __global__ void __launch_bounds__(256) cfirst_to_clast_kernel(const unsigned sho
             w[0] = v[i].x;
             w[1] = v[i].y;
         }
+    } else if constexpr (kVec == 0) {
+        unsigned short* flat = &tile[0][0];
+        const int n = min(kTile, C - c0) * P;
+        const unsigned short* run = s + (long long) c0 * P;
+        unsigned short v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int idx = threadIdx.x + 256 * i;
+            v[i] = 0;
+            if (idx < n) v[i] = run[idx];
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) flat[threadIdx.x + 256 * i] = v[i];
     } else {
         unsigned short v[16];
 #pragma unroll
@@ -56,7 +71,14 @@ __global__ void __launch_bounds__(256) cfirst_to_clast_kernel(const unsigned sho
     }
     __syncthreads();
     const int c = 2 * lane;   // C is even: a pair of channels is either inside or outside
-    if (c0 + c < C) {
+    if constexpr (kVec == 0) {
+        const unsigned short* flat = &tile[0][0];
+        if (c0 + c < C)
+            for (int p = warp; p < P; p += 8) {
+                const unsigned int v = (unsigned int) flat[c * P + p] | ((unsigned int) flat[(c + 1) * P + p] << 16);
+                *reinterpret_cast<unsigned int*>(d + (long long) p * C + c0 + c) = v;
+            }
+    } else if (c0 + c < C) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int p = warp + 8 * i;
@@ -75,7 +97,9 @@ cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, i
     const long long gx = mats * tiles_p;
     if (gx > 0x7fffffffLL || (C & 1)) return cudaErrorInvalidValue;
     dim3 grid((unsigned) gx, (unsigned) ((C + kTile - 1) / kTile));
-    if (P % 4 == 0 && reinterpret_cast<uintptr_t>(src) % 8 == 0)
+    if (P <= kTile && P % 4 != 0)
+        cfirst_to_clast_kernel<0><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
+    else if (P % 4 == 0 && reinterpret_cast<uintptr_t>(src) % 8 == 0)
         cfirst_to_clast_kernel<4><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
     else
         cfirst_to_clast_kernel<1><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
