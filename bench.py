@@ -191,6 +191,48 @@ def eager_fn(ch, t):
     return None
 
 
+def network_entry(fc, binding, flush, with_eager, batch=4096):
+    """The LeNet-shaped network (conv -> ReLU -> max-pool twice, three linear layers) as five chains per step, every
+    stage reading the previous stage's output in place; the unfused eager network on the same tensors beside it."""
+    import torch
+    import torch.nn.functional as F
+    stages = wl.lenet_shaped(batch)
+    runs, tensors, prev = [], [], None
+    for k, ch in enumerate(stages):
+        ins = [fc.to_device(a) for a in wl.make_inputs(ch, k)]
+        if prev is not None:
+            ins[0] = prev.reshape(ch.input_recipe[0][2])
+        outs = binding.output_tensors(ch, "cuda")
+        spec = fc.make_spec(ch)
+        binding.ensure_workspace(spec)
+        runs.append((spec, ins, outs))
+        tensors.append(ins)
+        prev = outs[0]
+    prepared = [fc.PreparedRun(sp, i, o) for sp, i, o in runs]   # after the last ensure_workspace: the workspace is final
+
+    def step():
+        for pr in prepared:
+            pr.run()
+    ms = time_loop(step, 20, 3, flush)
+    flops = sum(ch.flops() for ch in stages)
+    ent = {"ms": ms, "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "bound": "tensor", "chains_per_step": len(stages),
+           "workload": f"LeNet-shaped network, batch {batch}: conv5x5 8->64 + ReLU + pool, conv5x5 64->128 + ReLU + pool, 3200->120->88->10"}
+    if with_eager:
+        c1, c2, fcs = tensors[0], tensors[2], tensors[4]
+        x = c1[0].permute(0, 3, 1, 2)
+        w1, w2 = c1[1].permute(0, 3, 1, 2), c2[1].permute(0, 3, 1, 2)
+
+        def eager():
+            h = F.max_pool2d(torch.relu(F.conv2d(x, w1, c1[2])), 2)
+            h = F.max_pool2d(torch.relu(F.conv2d(h, w2, c2[2])), 2)
+            h = h.permute(0, 2, 3, 1).reshape(batch, -1)
+            h = torch.relu(F.linear(h, fcs[1], fcs[2]))
+            h = torch.relu(F.linear(h, fcs[3], fcs[4]))
+            return F.linear(h, fcs[5], fcs[6])
+        ent["eager_ms"] = time_loop(eager, 10, 3, flush)
+    return ent
+
+
 def time_loop(fn, steps, warmup, flush=None):
     """CUDA-event timing on the current stream.  Without `flush`: one event pair around `steps`
     back-to-back calls.  With `flush`: an L2-evicting write before every call, one pair per call."""
@@ -478,6 +520,7 @@ def main():
                 ent["eager_ms"] = time_loop(f2, 20, 3, fl)
             per[key] = ent
             del i2, o2
+        per["N1"] = network_entry(fc, binding, lambda: flush_buf.zero_(), not args.no_eager)
         line["per_config"] = per
 
     sampler.stop()

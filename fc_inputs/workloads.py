@@ -199,6 +199,24 @@ def conv_bias_relu_maxpool(batch=8, H=32, W=32, Cin=64, Cout=128, R=5, S=5, stri
     return replace(base, name="conv_bf16_bias_relu_maxpool", reduce="maxpool_2x2")
 
 
+def cast(M: int, N: int, in_dtype="f32", out_dtype="bf16") -> Chain:
+    """Elementwise chain with an empty op list: re-store a tensor in another type (what joins a pooled fp32
+    output to the 16-bit operand of the next contraction)."""
+    return Chain(f"cast_{in_dtype}_{out_dtype}", "elementwise", in_dtype, out_dtype, M=M, N=N, ops=(), reduce="none",
+                 store_main=True, input_recipe=(("x", in_dtype, (M, N), "normal", 0.0, 1.0),))
+
+
+def lenet_shaped(batch=64, C0=8, C1=64, C2=128, widths=(120, 88, 10)):
+    """The shape of the paper's Level-3 example network (LeNet-5) as a sequence of chains, at tensor-core-sized channel counts:
+    conv 5x5 -> ReLU -> 2x2 max-pool, twice (32x32 -> 28 -> 14 -> 10 -> 5), then three linear layers kept on chip.
+    The first input of every stage after the first is the previous stage's output (same bytes, reshaped)."""
+    s1 = conv_bias_relu_maxpool(batch=batch, H=32, W=32, Cin=C0, Cout=C1, R=5, S=5, pad=0)
+    s2 = conv_bias_relu_maxpool(batch=batch, H=14, W=14, Cin=C1, Cout=C2, R=5, S=5, pad=0)
+    flat = 5 * 5 * C2
+    return [replace(s1, name="lenet_conv1"), cast(batch, 14 * 14 * C1), replace(s2, name="lenet_conv2"), cast(batch, flat),
+            replace(mlp(batch, (flat,) + tuple(widths)), name="lenet_fc")]
+
+
 def conv_nchw(base: Chain) -> Chain:
     """The same convolution chain with the image stored [batch, Cin, H, W] and the weights [Cout, Cin, R, S]
     (the layouts of the paper's appendix listings); outputs are unchanged."""

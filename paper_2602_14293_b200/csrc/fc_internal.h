@@ -97,6 +97,7 @@ struct TcParams {
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
     int pool;                   // mode 2: 0 global average pool, 1 2x2 max-pool (out pre-zeroed, values >= 0)
+    int a_packed;               // mode 2: 1 = a k-block of A is eight 8-channel chunks, one per filter tap (Cin == 8)
     int* status;                // device status word
     int expect_extra;           // testing only: arrivals a wait expects beyond those that will come (mode 1: the panel
                                 // wait; other modes: the wait of a split tile's merging slice)

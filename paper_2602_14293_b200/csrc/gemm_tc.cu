@@ -12,6 +12,9 @@
 //           epilogue applies ops (bias, ReLU) and sums each channel over the tile's pixels, adding
 //           the scaled partial sums into out[image][channel]; or takes the maximum over 2x2 windows
 //           into out[image][oh/2][ow/2][channel]
+//   (template mode 4 is mode 2 for images of eight channels: a k-block then holds eight filter taps, gathered
+//    as eight 8-channel copies into an unswizzled operand tile; a separate instantiation, so that the loops
+//    of mode 2 stay as they are)
 //
 // Work unit: a 256 x BN output tile owned by a PAIR of CTAs on neighbouring SMs (cluster of 2,
 // tcgen05 cta_group::2).  Each CTA loads its own 128 rows of A and HALF of the B tile, so a k-block
@@ -148,6 +151,16 @@ __device__ __forceinline__ void tmem_sweep(uint32_t tacc, F&& f) {
     }
 }
 
+// k-blocks of one tile.  Convolution: one block per (tap, 64-channel slice), or (a_packed, chosen by the caller for
+// very few channels) blocks of eight 8-channel chunks that run on across the taps (K = R*S*Cin in order).
+template <int MODE>
+__host__ __device__ __forceinline__ int count_kb(const TcParams& p) {
+    if (MODE == 4) return (p.R * p.S * p.Cin + BK - 1) / BK;
+    if (MODE == 2) return p.R * p.S * ((p.Cin + BK - 1) / BK);
+    const int bk = p.in_dt == FC_F8E4M3 ? 2 * BK : BK;
+    return (p.K + bk - 1) / bk;
+}
+
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
@@ -168,10 +181,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM);   // pair-panels of 256 rows
     const int tiles_n = (p.N + BN - 1) / BN;
     const int total_tiles = tiles_m * tiles_n;
-    const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
-    const bool f8 = MODE != 2 && p.in_dt == FC_F8E4M3;
+    constexpr bool kConv = MODE == 2 || MODE == 4;   // 4: the convolution with eight filter taps per k-block (TcParams::a_packed)
+    const int kb_per_tap = kConv ? (p.Cin + BK - 1) / BK : 1;
+    const bool f8 = !kConv && p.in_dt == FC_F8E4M3;
     const int bk = f8 ? 2 * BK : BK;   // K elements per k-block: 128 bytes of a row
-    const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + bk - 1) / bk;
+    const int num_kb = count_kb<MODE>(p);
     const int total_units = p.split > 1 ? p.split_from + (total_tiles - p.split_from) * p.split : total_tiles;
 
     if (threadIdx.x == 0) {
@@ -210,7 +224,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
-                if constexpr (MODE == 2) {
+                if constexpr (kConv) {
                     const int hw = p.OH * p.OW;
                     img = row0 / hw;
                     const int rem = row0 - img * hw;
@@ -227,7 +241,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // the leader's arrival, and the peer starts the next phase only after the leader's MMAs
                     // of this one (the commit that frees the stage) are done.
                     if (leader) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->full[s]), 2 * C::kStageBytes);
-                    if constexpr (MODE == 2) {
+                    if constexpr (MODE == 4) {
+                        // eight copies of 128 pixels x 8 channels, each one column of core matrices (2 KB)
+                        const int cpt = p.Cin >> 3, chunks = p.R * p.S * cpt;
+#pragma unroll 1
+                        for (int q = 0; q < 8; ++q) {
+                            const int chunk = kb * 8 + q;
+                            int c0 = p.Cin, r = 0, sx = 0;     // past the last tap: channels out of range, filled with zeros
+                            if (chunk < chunks) {
+                                const int tap = chunk / cpt;
+                                c0 = (chunk - tap * cpt) * 8;
+                                r = tap / p.S;
+                                sx = tap - r * p.S;
+                            }
+                            ptx::tma_load_im2col_4d_pair(sa + q * 2048, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
+                        }
+                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * BK, bcol0, full);
+                    } else if constexpr (MODE == 2) {
                         const int tap = kb / kb_per_tap, c0 = (kb - tap * kb_per_tap) * BK;
                         const int r = tap / p.S, sx = tap - r * p.S;
                         ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
@@ -257,7 +287,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!(ok = wait_bar(ptx::smem_u32(&ctrl->full[s]), ph, abort_flag, p.status))) break;
                     ptx::tc_fence_after();
                     const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
-                    const uint64_t da = ptx::smem_desc_k128(sa), db = ptx::smem_desc_k128(sa + C::kABytes);
+                    const uint64_t db = ptx::smem_desc_k128(sa + C::kABytes);
+                    if constexpr (MODE == 4) {
+                        // A without swizzle: 2 KB between the core matrices of neighbouring 8-channel chunks, 128
+                        // bytes between 8-pixel groups; one MMA takes two chunks
+                        const uint64_t da = ptx::smem_desc_k_plain(sa, 2048, 128);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::tc_mma_f16_pair(d_tmem, da + (uint64_t) (k * (4096 >> 4)), db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
+                        ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);
+                        continue;
+                    }
+                    const uint64_t da = ptx::smem_desc_k128(sa);
                     if (f8) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)  // 32 E4M3 values = 32 bytes per MMA along K -> +2 in 16-byte units
@@ -787,9 +828,7 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     if (p.split_ws) {
         // Tiles left over after the full rounds (all of them, when there are fewer tiles than pairs) are cut
         // along K so that the last round keeps every pair busy.
-        const int kb_per_tap = MODE == 2 ? (p.Cin + BK - 1) / BK : 1;
-        const int bk = MODE != 2 && p.in_dt == FC_F8E4M3 ? 2 * BK : BK;
-        const int num_kb = MODE == 2 ? p.R * p.S * kb_per_tap : (p.K + bk - 1) / bk;
+        const int num_kb = count_kb<MODE>(p);
         const int full = tiles / max_pairs, tail = tiles - full * max_pairs;
         // (row softmax: only when everything fits one round; cutting the last of several rounds would let
         // row panels straddle rounds, which costs more than the split saves)
@@ -834,7 +873,7 @@ cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorM
         case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream, plan);
         case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream, plan);
         case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream, plan);
-        default: return launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
+        default: return p.a_packed ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan) : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
     }
 }
 

@@ -113,6 +113,18 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
     return d;
 }
 
+// K-major operand tile without swizzle: core matrices of 8 rows x 16 bytes stored as 128 contiguous bytes,
+// `k_stride` bytes between core matrices that are neighbours along K, `row_group_stride` bytes between
+// 8-row groups.  Stepping along K is done by adding whole core-matrix strides to `addr`.
+__device__ __forceinline__ uint64_t smem_desc_k_plain(uint32_t addr, uint32_t k_stride, uint32_t row_group_stride) {
+    uint64_t d = 0;
+    d |= (uint64_t) ((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t) (k_stride >> 4) << 16;            // leading-dimension byte offset
+    d |= (uint64_t) (row_group_stride >> 4) << 32;    // stride-dimension byte offset
+    d |= (uint64_t) 1 << 46;                          // descriptor version for sm_100
+    return d;                                         // swizzle field 0: none
+}
+
 // Instruction descriptor for kind::f16: bf16 x bf16 (ab_format 1) or fp16 x fp16 (ab_format 0) -> fp32,
 // both operands K-major, dense.
 __host__ __device__ constexpr uint32_t idesc_f16kind_f32(int m, int n, uint32_t ab_format) {

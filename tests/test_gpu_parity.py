@@ -309,6 +309,41 @@ def test_conv_filter_shapes(fc, orc, R, S, pad):
     run_and_check(fc, orc, wl.conv_bias_relu_avgpool(batch=2, H=12, W=20, Cin=64, Cout=64, R=R, S=S, pad=pad), 5)
 
 
+@pytest.mark.parametrize("R,S,pad,stride", [(1, 1, 0, 1), (3, 3, 1, 1), (5, 5, 0, 1), (5, 5, 2, 2), (3, 5, 1, 1), (7, 7, 3, 2), (4, 4, 1, 1)])
+@pytest.mark.parametrize("pool", ["avg", "max"])
+def test_conv_eight_channels_packs_filter_taps(fc, orc, R, S, pad, stride, pool):
+    """Cin = 8 (an RGB image padded to 8 channels): a k-block holds eight filter taps, gathered as eight
+    8-channel copies into an unswizzled operand tile; K = 8 R S ends inside a k-block for every shape here
+    but 4 x 4, so the zero-filled tail chunks are exercised too.  Delta kernels pin the tap order."""
+    make = wl.conv_bias_relu_avgpool if pool == "avg" else wl.conv_bias_relu_maxpool
+    ch = make(batch=3, H=17, W=22, Cin=8, Cout=40, R=R, S=S, pad=pad, stride=stride)
+    if pool == "max" and (ch.OH < 2 or ch.OW < 2):
+        pytest.skip("no 2 x 2 window")
+    run_and_check(fc, orc, ch, 9)
+
+
+def test_conv_eight_channels_delta_taps_bit_exact(fc):
+    """One-hot filter (tap (r, s), channel c -> output channel): the max-pooled output is the pooled ReLU of a
+    shifted image channel, exactly; every tap of a 5 x 5 filter in turn lands in a different chunk of the
+    packed k-blocks."""
+    B, H, W, R, S, pad = 2, 12, 14, 5, 5, 2
+    ch = replace(wl.conv_bias_relu_maxpool(batch=B, H=H, W=W, Cin=8, Cout=32, R=R, S=S, pad=pad), ops=(("relu",),))
+    ins = wl.make_inputs(ch, 4)
+    x = rng.bf16_bits_to_f32(ins[0])
+    w = np.zeros((32, R, S, 8), dtype=np.float32)
+    taps = [(co % 25 // 5, co % 25 % 5, co % 8) for co in range(32)]
+    for co, (r, s, c) in enumerate(taps):
+        w[co, r, s, c] = 1.0
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(ins[0]), fc.to_device(rng.store(w, "bf16"))], outs)
+    fc.fc_get_async_status()
+    xp = np.zeros((B, H + 2 * pad, W + 2 * pad, 8), dtype=np.float32)
+    xp[:, pad:pad + H, pad:pad + W] = x
+    want = np.stack([np.maximum(xp[:, r:r + H, s:s + W, c], 0) for r, s, c in taps], axis=-1)
+    want = want.reshape(B, H // 2, 2, W // 2, 2, 32).max(axis=(2, 4))
+    assert np.array_equal(outs[0].cpu().numpy(), want)
+
+
 @pytest.mark.parametrize("H,W,R,S,pad,stride", [(12, 20, 3, 3, 1, 2), (13, 21, 3, 3, 1, 2), (16, 16, 1, 1, 0, 2), (15, 18, 5, 5, 2, 3), (14, 14, 3, 3, 0, 2)])
 def test_conv_strided(fc, orc, H, W, R, S, pad, stride):
     run_and_check(fc, orc, wl.conv_bias_relu_avgpool(batch=3, H=H, W=W, Cin=64, Cout=64, R=R, S=S, pad=pad, stride=stride), 7)
@@ -475,6 +510,7 @@ def test_conv_relu_maxpool_delta_kernel_is_pooled_relu_of_image(fc, orc):
     (2, 14, 14, 64, 128, 3, 3, 1, 1),
     (3, 9, 13, 72, 40, 3, 3, 1, 1),        # pixels and channels that are no multiple of the 64-wide transposition tile
     (1, 7, 7, 8, 8, 1, 1, 0, 1),           # one tap, fewest channels
+    (5, 19, 11, 8, 72, 3, 5, 1, 2),        # 8 channels: eight filter taps per k-block, 15 taps = two blocks, the second one ragged
     (2, 23, 17, 136, 264, 5, 3, 2, 2),     # Cout over one 256-wide tile, strided, non-square filter
     (70, 8, 8, 64, 64, 3, 3, 1, 1),
 ])
