@@ -41,10 +41,8 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
     const bool y_vec = p.y && ((reinterpret_cast<uintptr_t>(p.y) | (uintptr_t)(N * ybytes)) & 15) == 0;
     const long long chunks = (N + kV - 1) / kV;
 
-    for (long long m = blockIdx.x; m < p.M; m += gridDim.x) {
-        MaxSum acc = ms_identity();
-        float psum = 0.0f, pmax = -CUDART_INF_F;   // ROW_SUM / ROW_MEAN and ROW_MAX
-        for (long long c = threadIdx.x; c < chunks; c += kThreads) {
+    // one 8-column chunk of row m: load, ops, reduction partials, store
+    auto chunk = [&](long long m, long long c, MaxSum& acc, float& psum, float& pmax) {
             const long long n0 = c * kV;
             const bool full = n0 + kV <= N;
             float v[kV];
@@ -110,7 +108,30 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
                     }
                 }
             }
+    };
+
+    if (p.reduce == FC_RED_NONE) {
+        // No reduction: rows do not matter, so the threads of the whole grid walk the chunks of the whole
+        // tensor in order (a row of 64 columns would otherwise keep 8 of a CTA's 256 threads busy).
+        const long long stride = (long long) gridDim.x * kThreads;
+        const long long dm = stride / chunks, dc = stride - dm * chunks;
+        const long long g = (long long) blockIdx.x * kThreads + threadIdx.x;
+        long long m = g / chunks, c = g - m * chunks;
+        MaxSum acc = ms_identity();
+        float psum = 0.0f, pmax = 0.0f;
+        while (m < p.M) {
+            chunk(m, c, acc, psum, pmax);
+            m += dm;
+            c += dc;
+            if (c >= chunks) { c -= chunks; ++m; }
         }
+        return;
+    }
+
+    for (long long m = blockIdx.x; m < p.M; m += gridDim.x) {
+        MaxSum acc = ms_identity();
+        float psum = 0.0f, pmax = -CUDART_INF_F;   // ROW_SUM / ROW_MEAN and ROW_MAX
+        for (long long c = threadIdx.x; c < chunks; c += kThreads) chunk(m, c, acc, psum, pmax);
         if (p.reduce == FC_RED_ROW_LOGSUMEXP) {
             const MaxSum t = block_merge(acc, red);
             if (threadIdx.x == 0) p.red[m] = t.m + logf(t.s);
@@ -431,7 +452,9 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
     int pre, act;
     bool res;
     const bool lse = p.reduce != FC_RED_NONE;   // any row reduction
-    if (match_fast(p, &f, &pre, &act, &res) && (lse || p.y)) {
+    // the row kernels give a warp to a row: without a reduction, rows under 256 columns go to the flat walk instead
+    const bool narrow = !lse && p.N < 256;
+    if (!narrow && match_fast(p, &f, &pre, &act, &res) && (lse || p.y)) {
         const bool store = p.y != nullptr;
 #define FC_EW_CASE(PRE_, ACT_)                                                                       \
     if (pre == PRE_ && act == ACT_)                                                                  \
@@ -444,7 +467,9 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
 #undef FC_EW_CASE
     }
     const bool precise = false;   // tanh.approx is accurate to 6e-6 here (see gelu_tanh)
-    long long grid = p.M < (long long) num_sms * 8 ? p.M : (long long) num_sms * 8;
+    long long work = p.M;   // CTAs that can be kept busy: rows, or 256-chunk slabs of the whole tensor
+    if (!lse) work = (p.M * ((p.N + 7) / 8) + kThreads - 1) / kThreads;
+    long long grid = work < (long long) num_sms * 8 ? work : (long long) num_sms * 8;
     if (grid < 1) grid = 1;
     if (precise)
         ew_generic_kernel<true><<<(unsigned) grid, kThreads, 0, stream>>>(p);

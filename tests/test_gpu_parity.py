@@ -79,6 +79,20 @@ def test_elementwise_f32_and_other_op_lists(fc, orc):
     run_and_check(fc, orc, replace(base, ops=()), 2)
 
 
+@pytest.mark.parametrize("M,N", [(1, 1), (1000, 8), (777, 64), (301, 72), (123, 200), (50, 255), (3000, 13), (9, 256), (4, 3000)])
+@pytest.mark.parametrize("dt", ["bf16", "f32"])
+def test_elementwise_without_reduction_walks_the_tensor_flat(fc, orc, M, N, dt):
+    """No reduction: the grid walks the chunks of the whole tensor, whatever the row length (narrow rows would
+    otherwise idle most of a CTA); per-column vectors and the residual must still line up with the columns,
+    also when a row is no multiple of eight columns."""
+    base = wl.affine_gelu_residual_lse(M, N)
+    if dt == "f32":
+        base = replace(base, in_dtype="f32", out_dtype="f32", input_recipe=tuple((t, "f32", s, d, a, b) for t, _, s, d, a, b in base.input_recipe))
+    run_and_check(fc, orc, replace(base, reduce="none"), 6)
+    run_and_check(fc, orc, replace(base, reduce="none", ops=(("bias_n", 2), ("relu",), ("add_tensor", 3))), 6)
+    run_and_check(fc, orc, wl.cast(M, N, "f32", "bf16" if dt == "bf16" else "f16"), 6)
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
