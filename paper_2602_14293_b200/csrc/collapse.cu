@@ -57,6 +57,13 @@ __device__ __forceinline__ void widen8(const uint4 w, bool f16, float (&v)[8]) {
     }
 }
 
+// The two kernels behind the weight pass are launched with programmatic stream serialization: their CTAs are
+// scheduled while the kernel in front drains, and wait here until that kernel has completed and its writes are
+// visible (a no-op under an ordinary launch).
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// (Releasing the next kernel early, griddepcontrol.launch_dependents at the top of each kernel, measured slightly
+// slower than the implicit release at exit: 37.5 vs 37.3 us on 1024 x 8192 x 8192.)
+
 __global__ void __launch_bounds__(kWarps * 32)
 weight_colsum_kernel(const CollapseParams p, int rows_per_block) {
     __shared__ double part[kWarps][kColsPerBlock];
@@ -122,8 +129,23 @@ weight_colsum_kernel(const CollapseParams p, int rows_per_block) {
     }
 }
 
+template <class... Args>
+cudaError_t launch_after(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 __global__ void __launch_bounds__(256)
 colsum_finish_kernel(const CollapseParams p, int splits) {
+    wait_for_previous_kernel();
     const long long k = (long long) blockIdx.x * blockDim.x + threadIdx.x;
     if (k < p.K) {
         double s = 0.0;
@@ -154,6 +176,7 @@ row_dot_kernel(const CollapseParams p) {
     double acc[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r) acc[r] = 0.0;
+    wait_for_previous_kernel();   // u and the constant term come from the kernel in front
 #pragma unroll 1
     for (long long kc = (long long) threadIdx.x * 8; kc < p.K; kc += kDotChunk) {
         float uu[kDotLoads][8];
@@ -241,14 +264,13 @@ cudaError_t launch_collapse(const CollapseParams& p_in, void* workspace, cudaStr
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     *launches += 1;
-    colsum_finish_kernel<<<col_blocks, 256, 0, stream>>>(p, splits);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_after(colsum_finish_kernel, dim3(col_blocks), dim3(256), stream, p, splits)) != cudaSuccess) return e;
     *launches += 1;
-    if (p.M <= 2048) row_dot_kernel<1, 8><<<(unsigned) p.M, kDotThreads, 0, stream>>>(p);
-    else if (p.K <= 4096) row_dot_kernel<4, 4><<<(unsigned) ((p.M + 3) / 4), kDotThreads, 0, stream>>>(p);
-    else row_dot_kernel<4, 8><<<(unsigned) ((p.M + 3) / 4), kDotThreads, 0, stream>>>(p);
+    if (p.M <= 2048) e = launch_after(row_dot_kernel<1, 8>, dim3((unsigned) p.M), dim3(kDotThreads), stream, p);
+    else if (p.K <= 4096) e = launch_after(row_dot_kernel<4, 4>, dim3((unsigned) ((p.M + 3) / 4)), dim3(kDotThreads), stream, p);
+    else e = launch_after(row_dot_kernel<4, 8>, dim3((unsigned) ((p.M + 3) / 4)), dim3(kDotThreads), stream, p);
     *launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace fc

@@ -681,9 +681,9 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                     std::lock_guard<std::mutex> lk(g_mu);
                     dev->counter_layout = 0;
                 }
-                if ((e = launch_cfirst_to_clast(image, img_cl, spec->batch, p.Cin, p.H * p.W, stream, &launches)) != cudaSuccess)
+                if ((e = launch_cfirst_to_clast(weights, w_cl, spec->Cout, p.Cin, p.R * p.S, false, stream, &launches)) != cudaSuccess)
                     return cuda_fail(e, "layout kernel launch");
-                if ((e = launch_cfirst_to_clast(weights, w_cl, spec->Cout, p.Cin, p.R * p.S, stream, &launches)) != cudaSuccess)
+                if ((e = launch_cfirst_to_clast(image, img_cl, spec->batch, p.Cin, p.H * p.W, true, stream, &launches)) != cudaSuccess)
                     return cuda_fail(e, "layout kernel launch");
                 image = img_cl;
                 weights = w_cl;

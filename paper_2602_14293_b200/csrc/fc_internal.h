@@ -77,7 +77,9 @@ cudaError_t launch_collapse(const CollapseParams& p, void* workspace, cudaStream
 size_t collapse_workspace_bytes(long long N, long long K);
 
 // Stack of `mats` 16-bit matrices [C][P] -> [P][C] (layout.cu): the channels-last rewrite for CONV2D_NCHW.  C even.
-cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, cudaStream_t stream, int* launches);
+// `beside_previous`: the kernel in front of this one in the stream shares no memory with it, so the two may overlap.
+cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,
+                                   int* launches);
 
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {

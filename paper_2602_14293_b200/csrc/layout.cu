@@ -70,6 +70,9 @@ __global__ void __launch_bounds__(256) cfirst_to_clast_kernel(const unsigned sho
         for (int i = 0; i < 16; ++i) tile[warp + 8 * (i >> 1)][lane + 32 * (i & 1)] = v[i];
     }
     __syncthreads();
+    // Under a programmatic launch (see the launcher) this kernel ran beside the tail of the one in front, with
+    // which it shares nothing; it must not be seen as complete before that one is.  A no-op otherwise.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int c = 2 * lane;   // C is even: a pair of channels is either inside or outside
     if constexpr (kVec == 0) {
         const unsigned short* flat = &tile[0][0];
@@ -92,19 +95,28 @@ __global__ void __launch_bounds__(256) cfirst_to_clast_kernel(const unsigned sho
 
 }  // namespace
 
-cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, cudaStream_t stream, int* launches) {
+cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,
+                                   int* launches) {
     const int tiles_p = (P + kTile - 1) / kTile;
     const long long gx = mats * tiles_p;
     if (gx > 0x7fffffffLL || (C & 1)) return cudaErrorInvalidValue;
-    dim3 grid((unsigned) gx, (unsigned) ((C + kTile - 1) / kTile));
-    if (P <= kTile && P % 4 != 0)
-        cfirst_to_clast_kernel<0><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
-    else if (P % 4 == 0 && reinterpret_cast<uintptr_t>(src) % 8 == 0)
-        cfirst_to_clast_kernel<4><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
-    else
-        cfirst_to_clast_kernel<1><<<grid, 256, 0, stream>>>((const unsigned short*) src, (unsigned short*) dst, C, P, tiles_p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned) gx, (unsigned) ((C + kTile - 1) / kTile));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    // `beside_previous`: the kernel in front of this one in the stream touches none of this one's memory (the
+    // other operand's transposition), so this one's CTAs may start while that one drains
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = beside_previous ? 1 : 0;
+    const unsigned short* s16 = (const unsigned short*) src;
+    unsigned short* d16 = (unsigned short*) dst;
     ++*launches;
-    return cudaGetLastError();
+    if (P <= kTile && P % 4 != 0) return cudaLaunchKernelEx(&cfg, cfirst_to_clast_kernel<0>, s16, d16, C, P, tiles_p);
+    if (P % 4 == 0 && reinterpret_cast<uintptr_t>(src) % 8 == 0) return cudaLaunchKernelEx(&cfg, cfirst_to_clast_kernel<4>, s16, d16, C, P, tiles_p);
+    return cudaLaunchKernelEx(&cfg, cfirst_to_clast_kernel<1>, s16, d16, C, P, tiles_p);
 }
 
 }  // namespace fc
