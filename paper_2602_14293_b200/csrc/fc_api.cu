@@ -178,6 +178,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             if (s->in_dtype == FC_F32) {
                 if (s->reduce != FC_RED_NONE || s->out_dtype != FC_F32)
                     return fail(FC_ERR_UNSUPPORTED, "fp32 GEMM supports fp32 output without reduction");
+                if (s->N > 65535LL * 32) return fail(FC_ERR_SHAPE, "fp32 GEMM supports N <= %lld", 65535LL * 32);
                 plan->kind = Plan::GEMM_F32;
             } else if (s->reduce == FC_RED_NONE) {
                 plan->kind = Plan::TC_PLAIN;

@@ -1,18 +1,119 @@
 // Strict-fp32 GEMM NT (C = epilogue(A * B^T), A [M,K], B [N,K], all fp32) for small problems.
 //
 // fp32 FMA on the plain ALUs: a single-pass TF32 tensor-core product would miss the fp32 output
-// tolerance, and at the sizes this path serves (hundreds per side) the run time is launch latency.
-// 32x32 output tile per CTA, 256 threads x (2x2) outputs, K staged through shared memory in
-// slabs of 32 with register prefetch of the next slab.
+// tolerance, and at the sizes this path serves (hundreds per side) the run time is launch latency plus
+// memory latency.  So the kernel is built to pay the memory latency once: a CTA owns a 16 x 32 output tile
+// (256^3 gives 128 CTAs), and stages K through shared memory in slabs of 128 columns with cp.async, two
+// slabs in flight from the first instruction on -- for K <= 256 every byte the CTA needs is requested
+// before it computes anything.  128 threads x (2 x 2) outputs; a thread's rows are 8 apart and its columns
+// 16 apart, so that its 16-byte shared-memory reads along K fall into distinct banks and its stores
+// coalesce.  Rows are padded to 132 floats (33 x 16 bytes).
 #include "dev_common.cuh"
 
 namespace fc {
 namespace {
 
+constexpr int kTM = 16, kTN = 32;      // output tile
+constexpr int kKS = 128;               // K columns per slab
+constexpr int kPitch = kKS + 4;        // floats per shared-memory row
+constexpr int kStages = 2;
+constexpr int kGemmThreads = 128;
+constexpr int kRows = kTM + kTN;       // rows of A and of B per slab
+constexpr int kSmemBytes = kStages * kRows * kPitch * (int) sizeof(float);
+
+__device__ __forceinline__ void cp_async16(float* dst, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned) __cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
+
+__global__ void __launch_bounds__(kGemmThreads) gemm_f32_kernel(const GemmF32Params p) {
+    extern __shared__ __align__(16) float smem_f32[];
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;                   // columns tx, tx + 16; rows ty, ty + 8
+    const int m0 = blockIdx.x * kTM, n0 = blockIdx.y * kTN;
+    const bool vec = ((reinterpret_cast<uintptr_t>(p.A) | reinterpret_cast<uintptr_t>(p.B)) & 15) == 0 && (p.K & 3) == 0;
+    const int slabs = (p.K + kKS - 1) / kKS;
+
+    // rows 0..15 of a stage hold A's tile, rows 16..47 B's; 48 rows x 32 chunks of 4 floats = 12 per thread
+    auto fill = [&](int slab) {
+        float* stage = smem_f32 + (slab % kStages) * kRows * kPitch;
+        const int k0 = slab * kKS;
+#pragma unroll     // (not unrolled, the copies are issued more slowly: 256^3 12.5 instead of 11.1 us from a cold L2)
+        for (int i = 0; i < kRows * (kKS / 4) / kGemmThreads; ++i) {
+            const int c = tid + i * kGemmThreads;
+            const int row = c >> 5, k = k0 + (c & 31) * 4;
+            const bool is_a = row < kTM;
+            const int grow = is_a ? m0 + row : n0 + row - kTM;
+            const bool row_ok = grow < (is_a ? p.M : p.N);
+            const float* src = (is_a ? p.A : p.B) + (long long) grow * p.K + k;
+            float* dst = stage + row * kPitch + (c & 31) * 4;
+            if (row_ok && vec && k + 3 < p.K) {
+                cp_async16(dst, src);
+            } else {
+                float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row_ok) {
+                    if (k + 0 < p.K) z.x = __ldg(src + 0);
+                    if (k + 1 < p.K) z.y = __ldg(src + 1);
+                    if (k + 2 < p.K) z.z = __ldg(src + 2);
+                    if (k + 3 < p.K) z.w = __ldg(src + 3);
+                }
+                *reinterpret_cast<float4*>(dst) = z;
+            }
+        }
+        cp_async_commit();
+    };
+
+    fill(0);
+    if (slabs > 1) fill(1);
+    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    for (int s = 0; s < slabs; ++s) {
+        if (s + 1 < slabs) cp_async_wait<1>(); else cp_async_wait<0>();
+        __syncthreads();
+        const float* stage = smem_f32 + (s % kStages) * kRows * kPitch;
+        const float* a0p = stage + ty * kPitch;
+        const float* a1p = stage + (ty + 8) * kPitch;
+        const float* b0p = stage + (kTM + tx) * kPitch;
+        const float* b1p = stage + (kTM + tx + 16) * kPitch;
+#pragma unroll 8
+        for (int k = 0; k < kKS; k += 4) {
+            const float4 a0 = *reinterpret_cast<const float4*>(a0p + k), a1 = *reinterpret_cast<const float4*>(a1p + k);
+            const float4 b0 = *reinterpret_cast<const float4*>(b0p + k), b1 = *reinterpret_cast<const float4*>(b1p + k);
+            acc[0][0] = fmaf(a0.x, b0.x, acc[0][0]); acc[0][1] = fmaf(a0.x, b1.x, acc[0][1]);
+            acc[1][0] = fmaf(a1.x, b0.x, acc[1][0]); acc[1][1] = fmaf(a1.x, b1.x, acc[1][1]);
+            acc[0][0] = fmaf(a0.y, b0.y, acc[0][0]); acc[0][1] = fmaf(a0.y, b1.y, acc[0][1]);
+            acc[1][0] = fmaf(a1.y, b0.y, acc[1][0]); acc[1][1] = fmaf(a1.y, b1.y, acc[1][1]);
+            acc[0][0] = fmaf(a0.z, b0.z, acc[0][0]); acc[0][1] = fmaf(a0.z, b1.z, acc[0][1]);
+            acc[1][0] = fmaf(a1.z, b0.z, acc[1][0]); acc[1][1] = fmaf(a1.z, b1.z, acc[1][1]);
+            acc[0][0] = fmaf(a0.w, b0.w, acc[0][0]); acc[0][1] = fmaf(a0.w, b1.w, acc[0][1]);
+            acc[1][0] = fmaf(a1.w, b0.w, acc[1][0]); acc[1][1] = fmaf(a1.w, b1.w, acc[1][1]);
+        }
+        __syncthreads();                       // everyone is done with this stage before it is refilled
+        if (s + kStages < slabs) fill(s + kStages);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int m = m0 + ty + 8 * i;
+        if (m >= p.M) continue;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int n = n0 + tx + 16 * j;
+            if (n >= p.N) continue;
+            float v[1] = {acc[i][j]};
+            apply_ops<1, false>(v, p.ops, m, n, p.N, p.N);
+            p.C[(long long) m * p.N + n] = v[0];
+        }
+    }
+}
+
+// Larger problems (several waves of 32 x 32 tiles): 256 threads x (2 x 2) outputs, slabs of 32 columns through
+// shared memory with the next slab prefetched into registers; more reuse per byte of shared memory than the
+// latency-oriented kernel above, whose small tiles cost 13 % at 1024^3.
 constexpr int kTile = 32;
 constexpr int kSlab = 32;
 
-__global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Params p) {
+__global__ void __launch_bounds__(256) gemm_f32_wide_kernel(const GemmF32Params p) {
     __shared__ float As[kTile][kSlab + 1];
     __shared__ float Bs[kTile][kSlab + 1];
     const int tid = threadIdx.x;
@@ -75,8 +176,24 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Params p) {
 }  // namespace
 
 cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* launches) {
-    dim3 grid((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile);
-    gemm_f32_kernel<<<grid, 256, 0, stream>>>(p);
+    static bool raised[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !raised[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        raised[dev] = true;
+    }
+    const long long wide_tiles = (long long) ((p.M + kTile - 1) / kTile) * ((p.N + kTile - 1) / kTile);
+    if (wide_tiles >= 512 && (p.M + kTile - 1) / kTile <= 65535) {
+        dim3 wide((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile);
+        gemm_f32_wide_kernel<<<wide, 256, 0, stream>>>(p);
+        *launches += 1;
+        return cudaGetLastError();
+    }
+    dim3 grid((p.M + kTM - 1) / kTM, (p.N + kTN - 1) / kTN);   // M tiles in x (up to 2^31 - 1), N tiles in y (up to 65535)
+    // a problem of one slab (K <= 128) asks for one stage only
+    gemm_f32_kernel<<<grid, kGemmThreads, p.K <= kKS ? kSmemBytes / kStages : kSmemBytes, stream>>>(p);
     *launches += 1;
     return cudaGetLastError();
 }
