@@ -589,3 +589,32 @@ def test_conv_relu_maxpool_fp16(fc, orc):
     ch = wl.conv_bias_relu_maxpool(batch=3, H=12, W=20, Cin=64, Cout=128, R=3, S=3, pad=1)
     ch = replace(ch, in_dtype="f16", input_recipe=tuple((t, "f16", sh, d, a, b) for t, _, sh, d, a, b in ch.input_recipe))
     run_and_check(fc, orc, ch, 4)
+
+
+# ------------------------------------------------------------------ the further measured workloads at full size
+@pytest.mark.parametrize("key", ["F1", "F2", "F3", "F4", "F5", "F6"])
+def test_further_workloads_full_size_sampled(fc, orc, key):
+    """Each workload the benchmark times beyond the five configurations, at its full size and in the launch
+    configuration the benchmark uses; rows (images) are independent problems, so the oracle recomputes a sample
+    of them: first and last, tile boundaries, and a stride through the rest."""
+    ch = wl.ALL[key]()
+    ins = wl.make_inputs(ch, 0)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    if ch.is_conv:
+        pick = np.array([0, 17, ch.batch - 1])
+        sub = replace(ch, batch=len(pick))
+    else:
+        pick = np.unique(np.concatenate([np.arange(0, ch.M, max(1, ch.M // 13) + 1), [0, 127, 128, 255, 256, ch.M - 1]]))
+        sub = replace(ch, M=len(pick))
+    sub_ins = [ins[0][pick]] + list(ins[1:])
+    ref = orc.run_chain(sub, sub_ins)
+    sel = torch.from_numpy(pick).cuda()
+    names = [r for r, _, _ in wl.output_shapes(ch)]
+    for name, t in zip(names, outs):
+        assert torch.isfinite(t.float()).all(), f"{key}: non-finite values in {name}"
+        if any(op[0] == "linear" for op in ch.ops):
+            util.check_chained(t[sel], ref[name], util.flip_allowance(orc, sub, sub_ins), f"{key} {name} (sampled rows)")
+        else:
+            util.check(t[sel], ref[name], f"{key} {name} (sampled)")
