@@ -150,6 +150,9 @@ def eager_fn(ch, t):
             y = F.gelu(t[0] * t[1] + t[2], approximate="tanh") + t[3]
             return y, torch.logsumexp(y.float(), 1)
         return f
+    if name == "ew_scale_add_softmax":
+        scale = [o for o in ch.ops if o[0] == "scale"][0][1]
+        return lambda: torch.softmax(t[0] * scale + t[1], dim=1)
     if name == "gemm_bf16_bias_gelu_scale_clamp":
         return lambda: torch.clamp(F.gelu(F.linear(t[0], t[1], t[2]), approximate="tanh") * 0.5, -1.0, 1.0)
     if name == "gemm_bf16_bias_scale_lse":

@@ -106,6 +106,14 @@ def affine_gelu_residual_lse(M=16384, N=4096) -> Chain:
                                ("r", "bf16", (M, N), "normal", 0.0, 1.0)))
 
 
+def scale_add_softmax(M=16384, N=4096, scale=0.125, dtype="bf16") -> Chain:
+    """x * scale + t -> row softmax: the memory-bound softmax of a score matrix with an additive term."""
+    return Chain("ew_scale_add_softmax", "elementwise", dtype, dtype, M=M, N=N,
+                 ops=(("scale", scale), ("add_tensor", 1)), reduce="row_softmax", store_main=False,
+                 input_recipe=(("x", dtype, (M, N), "normal", 0.0, 4.0),
+                               ("t", dtype, (M, N), "normal", 0.0, 1.0)))
+
+
 def gemm_bias_gelu_scale_clamp(M=8192, N=8192, K=4096, variant="std") -> Chain:
     s = K ** -0.5 if variant == "std" else K ** -0.25
     return Chain("gemm_bf16_bias_gelu_scale_clamp", "gemm_nt", "bf16", "bf16", M=M, N=N, K=K,
@@ -242,6 +250,7 @@ EXTRA = {
     "F4": lambda **kw: mlp(**{"M": 16384, "dims": (1024, 256, 256, 64), **kw}),
     "F3": lambda **kw: conv_bias_relu_maxpool(**{"batch": 32, "H": 56, "W": 56, "Cin": 256, "Cout": 256, "R": 3, "S": 3, "pad": 1, **kw}),
     "F6": lambda **kw: conv_nchw(conv_bias_relu_avgpool(**kw)),
+    "F7": lambda **kw: scale_add_softmax(**kw),
 }
 ALL = {**CONFIGS, **EXTRA}
 

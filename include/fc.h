@@ -122,7 +122,7 @@ typedef enum {
 typedef enum {
     FC_RED_NONE = 0,
     FC_RED_ROW_LOGSUMEXP = 1,   /* out[m] = max_n v + log sum_n exp(v - max)          */
-    FC_RED_ROW_SOFTMAX = 2,     /* p[m][n] = exp(v - max) / sum_n exp(v - max)         */
+    FC_RED_ROW_SOFTMAX = 2,     /* p[m][n] = exp(v - max) / sum_n exp(v - max)         (elementwise or GEMM producer) */
     FC_RED_GLOBAL_AVGPOOL = 3,  /* out[b][c] = mean over (oh, ow) of v[b][oh][ow][c]   */
     FC_RED_ROW_SUM = 4,         /* out[m] = sum_n v          (elementwise or GEMM producer) */
     FC_RED_ROW_MAX = 5,         /* out[m] = max_n v          (elementwise or GEMM producer) */

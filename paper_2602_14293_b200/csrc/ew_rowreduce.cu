@@ -42,7 +42,10 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
     const long long chunks = (N + kV - 1) / kV;
 
     // one 8-column chunk of row m: load, ops, reduction partials, store
-    auto chunk = [&](long long m, long long c, MaxSum& acc, float& psum, float& pmax) {
+    // `phase`: 0 the whole chunk; row softmax takes two passes over a row: 1 accumulates (max, sum) without
+    // storing, 2 computes the values again (the row's inputs are still in L2), turns them into
+    // exp(v - row_max) * inv_sum and stores
+    auto chunk = [&](long long m, long long c, MaxSum& acc, float& psum, float& pmax, int phase, float row_max, float inv_sum) {
             const long long n0 = c * kV;
             const bool full = n0 + kV <= N;
             float v[kV];
@@ -66,7 +69,10 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
                 }
             }
             apply_ops<kV, kPreciseGelu>(v, p.ops, m, n0, N, N);
-            if (p.reduce == FC_RED_ROW_LOGSUMEXP) {
+            if (phase == 2) {
+#pragma unroll
+                for (int j = 0; j < kV; ++j) v[j] = exp2_fast((v[j] - row_max) * kLog2e) * inv_sum;
+            } else if (p.reduce == FC_RED_ROW_LOGSUMEXP || p.reduce == FC_RED_ROW_SOFTMAX) {
                 float mx = -CUDART_INF_F;
 #pragma unroll
                 for (int j = 0; j < kV; ++j) mx = n0 + j < N ? fmaxf(mx, v[j]) : mx;
@@ -83,7 +89,7 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
                         pmax = fmaxf(pmax, v[j]);
                     }
             }
-            if (p.y) {
+            if (p.y && phase != 1) {
                 if (p.y_dt != FC_F32) {
                     unsigned short* yp = (unsigned short*) p.y + m * N + n0;
                     if (full && y_vec) {
@@ -120,7 +126,7 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
         MaxSum acc = ms_identity();
         float psum = 0.0f, pmax = 0.0f;
         while (m < p.M) {
-            chunk(m, c, acc, psum, pmax);
+            chunk(m, c, acc, psum, pmax, 0, 0.0f, 0.0f);
             m += dm;
             c += dc;
             if (c >= chunks) { c -= chunks; ++m; }
@@ -131,8 +137,13 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
     for (long long m = blockIdx.x; m < p.M; m += gridDim.x) {
         MaxSum acc = ms_identity();
         float psum = 0.0f, pmax = -CUDART_INF_F;   // ROW_SUM / ROW_MEAN and ROW_MAX
-        for (long long c = threadIdx.x; c < chunks; c += kThreads) chunk(m, c, acc, psum, pmax);
-        if (p.reduce == FC_RED_ROW_LOGSUMEXP) {
+        const int phase = p.reduce == FC_RED_ROW_SOFTMAX ? 1 : 0;
+        for (long long c = threadIdx.x; c < chunks; c += kThreads) chunk(m, c, acc, psum, pmax, phase, 0.0f, 0.0f);
+        if (p.reduce == FC_RED_ROW_SOFTMAX) {
+            const MaxSum t = block_merge(acc, red);   // every thread gets the row's pair
+            const float inv = 1.0f / t.s;
+            for (long long c = threadIdx.x; c < chunks; c += kThreads) chunk(m, c, acc, psum, pmax, 2, t.m, inv);
+        } else if (p.reduce == FC_RED_ROW_LOGSUMEXP) {
             const MaxSum t = block_merge(acc, red);
             if (threadIdx.x == 0) p.red[m] = t.m + logf(t.s);
         } else if (p.reduce >= FC_RED_ROW_SUM) {
@@ -177,6 +188,9 @@ struct EwFastParams {
     int N;
     int red_kind;           // fc_reduce of the row reduction (when the kernel is built with one)
     int is_f16;             // x, residual and y are IEEE half instead of bf16
+    int stash;              // row softmax: the row's fp32 values wait in shared memory for the second pass
+    float pre_scale;        // a SCALE op in front of everything, folded into gamma (PRE is then always affine;
+                            // vec0 == null means gamma = 1, vec1 == null means beta = 0)
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -195,10 +209,9 @@ constexpr int kGroup = 4;   // chunks in flight per lane and tensor
 
 // One chunk (8 columns starting at column 8*c) of one row: ops in packed fp32x2, one 16-byte store,
 // and the chunk's contribution to the running (max, sum) of the row (log2 domain).
-template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
-__device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
-                                         int red_kind, bool f16, float& run_m, float& run_s) {
-    float2 v[4];
+// The values of one chunk (8 columns starting at column 8*c) after the ops, as four fp32 pairs.
+template <int PRE, int ACT, bool RES>
+__device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const float* svec, int N, int c, bool f16, float2 (&v)[4]) {
     v[0] = unpack16x2(xq.x, f16);
     v[1] = unpack16x2(xq.y, f16);
     v[2] = unpack16x2(xq.z, f16);
@@ -255,13 +268,24 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
         }
         v[j] = t;
     }
+}
+
+template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
+__device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
+                                         int red_kind, bool f16, float& run_m, float& run_s, float4* stash) {
+    float2 v[4];
+    ew_values<PRE, ACT, RES>(xq, rq, svec, N, c, f16, v);
+    if (stash) {   // same de-interleaved layout as the vectors: conflict-free 16-byte accesses
+        stash[c] = make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
+        stash[(N >> 3) + c] = make_float4(v[2].x, v[2].y, v[3].x, v[3].y);
+    }
     if (STORE) {
         uint4 q;
         q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
         q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
         st_stream(yr + c, q);
     }
-    if (LSE && red_kind != FC_RED_ROW_LOGSUMEXP) {
+    if (LSE && red_kind >= FC_RED_ROW_SUM) {
         // ROW_SUM / ROW_MEAN / ROW_MAX: plain running sum and maximum
         const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)),
                                fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
@@ -284,8 +308,10 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
     }
 }
 
-template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
-__global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams p) {
+// SOFTMAX (with LSE and without STORE): the row's values are turned into probabilities in a second pass.  Its own
+// instantiations, with twice the registers: the second pass does not fit the 64 of the others without spilling.
+template <int PRE, int ACT, bool RES, bool LSE, bool STORE, bool SOFTMAX = false>
+__global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(const EwFastParams p) {
     extern __shared__ float svec[];   // PRE != none: vec0 as fp32 [N] (chunk halves de-interleaved), then vec1 [N]
     const int N = p.N;
     if (PRE != kPreNone) {
@@ -294,9 +320,10 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
         // eight columns per load, all loads of a thread issued before the first conversion.
         const int nchunks = N >> 3;
         float4* sv = reinterpret_cast<float4*>(svec);
-        const bool fast0 = p.vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(p.vec0) & 15) == 0;
-        const bool fast1 = PRE != kPreAffine || (p.vec1_dt != FC_F32 && (reinterpret_cast<uintptr_t>(p.vec1) & 15) == 0);
-        if (fast0 && fast1 && nchunks <= 4 * kThreads) {
+        const bool fast0 = p.vec0 && p.vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(p.vec0) & 15) == 0;
+        const bool fast1 = PRE != kPreAffine || (p.vec1 && p.vec1_dt != FC_F32 && (reinterpret_cast<uintptr_t>(p.vec1) & 15) == 0);
+        const bool plain = PRE != kPreAffine || p.pre_scale == 1.0f;   // a folded SCALE takes the scalar loop
+        if (fast0 && fast1 && plain && nchunks <= 4 * kThreads) {
             uint4 q0[4], q1[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -326,8 +353,8 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
             for (int i = threadIdx.x; i < N; i += kThreads) {
                 // column i = chunk i/8, half (i%8)/4, element i%4  ->  float4 number half * chunks + chunk
                 const int pos = ((((i >> 2) & 1) * nchunks) + (i >> 3)) * 4 + (i & 3);
-                svec[pos] = load_scalar(p.vec0, p.vec0_dt, i);
-                if (PRE == kPreAffine) svec[N + pos] = load_scalar(p.vec1, p.vec1_dt, i);
+                svec[pos] = (p.vec0 ? load_scalar(p.vec0, p.vec0_dt, i) : 1.0f) * (PRE == kPreAffine ? p.pre_scale : 1.0f);
+                if (PRE == kPreAffine) svec[N + pos] = p.vec1 ? load_scalar(p.vec1, p.vec1_dt, i) : 0.0f;
             }
         }
         __syncthreads();
@@ -340,15 +367,20 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
     const int chunks = N >> 3;
     const int warp = threadIdx.x >> 5;
     const long long row_step = (long long) gridDim.x * kWarps;
+    float4* stash = nullptr;
+    if (SOFTMAX && p.stash) stash = reinterpret_cast<float4*>(svec + (PRE == kPreNone ? 0 : (PRE == kPreAffine ? 2 : 1) * N)) + warp * (N >> 2);
     for (long long row = (long long) blockIdx.x * kWarps + warp; row < p.M; row += row_step) {
         const uint4* xr = p.x + row * chunks;
         const uint4* rr = RES ? p.res + row * chunks : nullptr;
         uint4* yr = STORE ? p.y + row * chunks : nullptr;
         float run_m = -CUDART_INF_F, run_s = 0.0f;   // log2 domain: sum of 2^(y*log2e - run_m)
-        for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
-            uint4 xv[kGroup], rv[kGroup];
+        // (softmax at 4096 columns runs one CTA per SM, its rows waiting in shared memory; twice the loads in flight
+        // per lane there gained 6 % and lost 7 % at 1024 columns: left alone)
+        constexpr int kInFlight = kGroup;
+        for (int c0 = lane; c0 < chunks; c0 += 32 * kInFlight) {
+            uint4 xv[kInFlight], rv[kInFlight];
 #pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
+            for (int g = 0; g < kInFlight; ++g) {
                 const int c = c0 + 32 * g;
                 if (c < chunks) {
                     xv[g] = ld_stream(xr + c);
@@ -356,12 +388,14 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
                 }
             }
 #pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
+            for (int g = 0; g < kInFlight; ++g) {
                 const int c = c0 + 32 * g;
-                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, p.red_kind, p.is_f16 != 0, run_m, run_s);
+                if (c < chunks)
+                    ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind, p.is_f16 != 0, run_m, run_s,
+                                                        SOFTMAX ? stash : nullptr);
             }
         }
-        if (LSE && p.red_kind != FC_RED_ROW_LOGSUMEXP) {
+        if (LSE && !SOFTMAX && p.red_kind >= FC_RED_ROW_SUM) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 run_s += __shfl_xor_sync(0xffffffffu, run_s, o);
@@ -381,7 +415,51 @@ __global__ void __launch_bounds__(kThreads, 4) ew_rows_kernel(const EwFastParams
                 run_s = sa + sb;
                 run_m = nm;
             }
-            if (lane == 0) p.lse[row] = (run_m + log2f(run_s)) * kLn2;
+            if constexpr (SOFTMAX) {
+                // Second pass over the row: the values wait in shared memory (rows of up to a few thousand columns),
+                // else the inputs are read again, from L2 where they still are, and the values computed again;
+                // stored as 2^(v log2e - max) / sum.
+                float inv;
+                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(run_s));
+                const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-run_m, -run_m), inv2 = make_float2(inv, inv);
+                uint4* pr = p.y + row * chunks;
+                for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
+                    uint4 xv[kGroup], rv[kGroup];
+                    if (!stash) {
+#pragma unroll
+                        for (int g = 0; g < kGroup; ++g) {
+                            const int c = c0 + 32 * g;
+                            if (c < chunks) {
+                                xv[g] = __ldcg(xr + c);
+                                if (RES) rv[g] = __ldcg(rr + c);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int g = 0; g < kGroup; ++g) {
+                        const int c = c0 + 32 * g;
+                        if (c < chunks) {
+                            float2 v[4];
+                            if (stash) {
+                                const float4 a = stash[c], b = stash[chunks + c];
+                                v[0] = make_float2(a.x, a.y); v[1] = make_float2(a.z, a.w);
+                                v[2] = make_float2(b.x, b.y); v[3] = make_float2(b.z, b.w);
+                            } else {
+                                ew_values<PRE, ACT, RES>(xv[g], rv[g], svec, N, c, p.is_f16 != 0, v);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 e = __ffma2_rn(v[j], l2e, mnm);
+                                v[j] = __fmul2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), inv2);
+                            }
+                            uint4 q;
+                            q.x = pack16x2(v[0].x, v[0].y, p.is_f16 != 0); q.y = pack16x2(v[1].x, v[1].y, p.is_f16 != 0);
+                            q.z = pack16x2(v[2].x, v[2].y, p.is_f16 != 0); q.w = pack16x2(v[3].x, v[3].y, p.is_f16 != 0);
+                            st_stream(pr + c, q);
+                        }
+                    }
+                }
+            } else if (lane == 0) p.lse[row] = (run_m + log2f(run_s)) * kLn2;
         }
     }
 }
@@ -396,11 +474,19 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
     int i = 0;
     *pre = kPreNone; *act = kActNone; *res = false;
     f->vec0 = f->vec1 = nullptr; f->vec0_dt = f->vec1_dt = FC_F32; f->res = nullptr;
+    f->pre_scale = 1.0f;
+    const bool scaled = i < p.ops.n && p.ops.op[i].kind == FC_OP_SCALE;
+    if (scaled) f->pre_scale = p.ops.op[i++].f0;
     if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_BIAS_N || p.ops.op[i].kind == FC_OP_AFFINE_N)) {
         *pre = p.ops.op[i].kind == FC_OP_BIAS_N ? kPreBias : kPreAffine;
         f->vec0 = p.ops.op[i].p0; f->vec0_dt = p.ops.op[i].dt0;
         f->vec1 = p.ops.op[i].p1; f->vec1_dt = p.ops.op[i].dt1;
         ++i;
+    }
+    if (scaled) {
+        // x * s (+ b)  or  (x * s) * g + b: an affine step whose gamma carries the factor
+        if (*pre == kPreBias) { f->vec1 = f->vec0; f->vec1_dt = f->vec0_dt; f->vec0 = nullptr; f->vec0_dt = FC_F32; }
+        *pre = kPreAffine;
     }
     if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_RELU || p.ops.op[i].kind == FC_OP_GELU_TANH)) {
         // with a logsumexp behind it the exp-based form (ex2 + rcp) measures no slower than tanh.approx
@@ -422,14 +508,20 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
 }
 
 template <int PRE, int ACT, bool RES>
-static cudaError_t launch_fast(const EwFastParams& f, bool lse, bool store, int num_sms, cudaStream_t stream) {
-    const size_t smem = PRE == kPreNone ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
+static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, int num_sms, cudaStream_t stream) {
+    EwFastParams f = f_in;
+    size_t smem = PRE == kPreNone ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
+    f.stash = 0;
+    if (f.red_kind == FC_RED_ROW_SOFTMAX && smem + (size_t) kWarps * f.N * 4 <= 200 * 1024) {
+        f.stash = 1;
+        smem += (size_t) kWarps * f.N * 4;
+    }
     long long ctas = (f.M + kWarps - 1) / kWarps;
     int per_sm = smem > 0 ? (int) ((200 * 1024) / smem) : 4;
     per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);
     if (ctas > (long long) num_sms * per_sm) ctas = (long long) num_sms * per_sm;
     // the dynamic shared-memory limit of each instantiation is raised once per device, to the maximum
-    static bool raised[3][64] = {};
+    static bool raised[4][64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     auto go = [&](auto kernel, int variant) -> cudaError_t {
@@ -441,6 +533,7 @@ static cudaError_t launch_fast(const EwFastParams& f, bool lse, bool store, int 
         kernel<<<(unsigned) ctas, kThreads, smem, stream>>>(f);
         return cudaGetLastError();
     };
+    if (f.red_kind == FC_RED_ROW_SOFTMAX) return go(ew_rows_kernel<PRE, ACT, RES, true, false, true>, 3);
     if (lse && store) return go(ew_rows_kernel<PRE, ACT, RES, true, true>, 0);
     if (lse) return go(ew_rows_kernel<PRE, ACT, RES, true, false>, 1);
     return go(ew_rows_kernel<PRE, ACT, RES, false, true>, 2);
@@ -455,7 +548,7 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
     // the row kernels give a warp to a row: without a reduction, rows under 256 columns go to the flat walk instead
     const bool narrow = !lse && p.N < 256;
     if (!narrow && match_fast(p, &f, &pre, &act, &res) && (lse || p.y)) {
-        const bool store = p.y != nullptr;
+        const bool store = p.y != nullptr && p.reduce != FC_RED_ROW_SOFTMAX;   // softmax stores in its second pass
 #define FC_EW_CASE(PRE_, ACT_)                                                                       \
     if (pre == PRE_ && act == ACT_)                                                                  \
         return res ? launch_fast<PRE_, ACT_, true>(f, lse, store, num_sms, stream)                  \

@@ -170,8 +170,8 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     plan->main_index = plan->red_index = -1;
     switch (s->producer) {
         case FC_PROD_ELEMENTWISE:
-            if (s->reduce == FC_RED_ROW_SOFTMAX || s->reduce == FC_RED_GLOBAL_AVGPOOL || s->reduce == FC_RED_MAXPOOL_2X2)
-                return fail(FC_ERR_UNSUPPORTED, "elementwise producer supports reduce NONE, ROW_LOGSUMEXP, ROW_SUM, ROW_MAX or ROW_MEAN");
+            if (s->reduce == FC_RED_GLOBAL_AVGPOOL || s->reduce == FC_RED_MAXPOOL_2X2)
+                return fail(FC_ERR_UNSUPPORTED, "elementwise producer supports reduce NONE, ROW_LOGSUMEXP, ROW_SOFTMAX, ROW_SUM, ROW_MAX or ROW_MEAN");
             plan->kind = Plan::EW;
             break;
         case FC_PROD_GEMM_NT:

@@ -113,12 +113,12 @@ def test_rejections_happen_before_any_device_access(fc):
     ch_k = wl.gemm_bias_gelu_scale_clamp(256, 256, 60)     # K % 8 != 0
     k_in = _arr(fc, [_fake_tensor(fc, (256, 60), 1), _fake_tensor(fc, (256, 60), 1), _fake_tensor(fc, (256,), 1)])
     assert _status(fc, fc.make_spec(ch_k), k_in, good_out) == ALIGN
-    # well-formed but not implemented: average pool after a GEMM, conv stride > 8, softmax on an elementwise producer
+    # well-formed but not implemented: average pool after a GEMM, conv stride > 8, pooling on an elementwise producer
     s = fc.make_spec(ch); s.reduce = 3          # global average pool after a GEMM
     assert _status(fc, s, good_in, good_out) == UNSUP
     s = fc.make_spec(wl.conv_bias_relu_avgpool(stride=9))
     assert _status(fc, s, good_in, good_out) == UNSUP
-    s = fc.make_spec(wl.affine_gelu_residual_lse(8, 8)); s.reduce = 2
+    s = fc.make_spec(wl.affine_gelu_residual_lse(8, 8)); s.reduce = 3
     assert _status(fc, s, good_in, good_out) == UNSUP
     assert "FC_ERR_UNSUPPORTED" == L.fc_status_string(UNSUP).decode()
     assert len(fc.fc_last_error()) > 0

@@ -93,6 +93,30 @@ def test_elementwise_without_reduction_walks_the_tensor_flat(fc, orc, M, N, dt):
     run_and_check(fc, orc, wl.cast(M, N, "f32", "bf16" if dt == "bf16" else "f16"), 6)
 
 
+@pytest.mark.parametrize("M,N", [(1, 1), (3, 8), (5, 1000), (7, 4097), (33, 2048), (64, 4096), (9, 12345), (300, 64)])
+@pytest.mark.parametrize("dt", ["bf16", "f32", "f16"])
+def test_elementwise_row_softmax(fc, orc, M, N, dt):
+    ch = wl.scale_add_softmax(M, N, dtype=dt)
+    outs, ref, _ = run_and_check(fc, orc, ch, 8)
+    sums = util.to_f64(outs[0]).sum(axis=1)
+    np.testing.assert_allclose(sums, 1.0, atol=2e-2 if dt == "bf16" else 2e-3)
+
+
+def test_elementwise_row_softmax_other_op_lists_and_extremes(fc, orc):
+    base = wl.scale_add_softmax(40, 777)
+    # no ops; affine -> GELU in front; a dominant logit per row and rows shifted by +-1e4 (fp32 storage)
+    run_and_check(fc, orc, replace(base, ops=()), 1)
+    aff = wl.affine_gelu_residual_lse(40, 777)
+    run_and_check(fc, orc, replace(aff, reduce="row_softmax", store_main=False), 1)
+    ch32 = wl.scale_add_softmax(16, 515, scale=1.0, dtype="f32")
+    ins = wl.make_inputs(ch32, 2)
+    ins[0][np.arange(16), np.arange(16) * 3] += 60.0
+    ins[0][::2] += 1.0e4
+    ins[0][1::2] -= 1.0e4
+    outs, ref, _ = run_and_check(fc, orc, ch32, ins=ins)
+    assert (util.to_f64(outs[0]).argmax(1) == np.arange(16) * 3).all()
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
@@ -592,7 +616,7 @@ def test_conv_relu_maxpool_fp16(fc, orc):
 
 
 # ------------------------------------------------------------------ the further measured workloads at full size
-@pytest.mark.parametrize("key", ["F1", "F2", "F3", "F4", "F5", "F6"])
+@pytest.mark.parametrize("key", ["F1", "F2", "F3", "F4", "F5", "F6", "F7"])
 def test_further_workloads_full_size_sampled(fc, orc, key):
     """Each workload the benchmark times beyond the five configurations, at its full size and in the launch
     configuration the benchmark uses; rows (images) are independent problems, so the oracle recomputes a sample
@@ -608,7 +632,8 @@ def test_further_workloads_full_size_sampled(fc, orc, key):
     else:
         pick = np.unique(np.concatenate([np.arange(0, ch.M, max(1, ch.M // 13) + 1), [0, 127, 128, 255, 256, ch.M - 1]]))
         sub = replace(ch, M=len(pick))
-    sub_ins = [ins[0][pick]] + list(ins[1:])
+    per_row = {0} | {op[1] for op in ch.ops if op[0] == "add_tensor"}      # inputs with one row per problem
+    sub_ins = [a[pick] if i in per_row else a for i, a in enumerate(ins)]
     ref = orc.run_chain(sub, sub_ins)
     sel = torch.from_numpy(pick).cuda()
     names = [r for r, _, _ in wl.output_shapes(ch)]
