@@ -76,10 +76,12 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
                 float mx = -CUDART_INF_F;
 #pragma unroll
                 for (int j = 0; j < kV; ++j) mx = n0 + j < N ? fmaxf(mx, v[j]) : mx;
-                float s = 0.0f;
+                if (mx != -CUDART_INF_F) {   // a chunk of -inf only (a masked stretch of the row) adds nothing
+                    float s = 0.0f;
 #pragma unroll
-                for (int j = 0; j < kV; ++j) s += n0 + j < N ? exp2_fast((v[j] - mx) * kLog2e) : 0.0f;
-                acc = ms_merge(acc, MaxSum{mx, s});
+                    for (int j = 0; j < kV; ++j) s += n0 + j < N ? exp2_fast((v[j] - mx) * kLog2e) : 0.0f;
+                    acc = ms_merge(acc, MaxSum{mx, s});
+                }
             }
             if (p.reduce >= FC_RED_ROW_SUM) {
 #pragma unroll
@@ -296,14 +298,17 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
         const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)),
                                fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
         const float nm = fmaxf(run_m, cm * kLog2e);
-        const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-nm, -nm);
+        // while everything seen so far is -inf (a masked stretch at the start of the lane's columns) the
+        // exponents are taken against 0, so that -inf stays -inf instead of turning into -inf - -inf
+        const float base = nm == -CUDART_INF_F ? 0.0f : nm;
+        const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-base, -base);
         float2 cs = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float2 e = __ffma2_rn(v[j], l2e, mnm);
             cs = __fadd2_rn(cs, make_float2(exp2_fast(e.x), exp2_fast(e.y)));
         }
-        run_s = fmaf(run_s, exp2_fast(run_m - nm), cs.x + cs.y);
+        run_s = fmaf(run_s, exp2_fast(run_m - base), cs.x + cs.y);
         run_m = nm;
     }
 }

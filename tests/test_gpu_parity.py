@@ -117,6 +117,28 @@ def test_elementwise_row_softmax_other_op_lists_and_extremes(fc, orc):
     assert (util.to_f64(outs[0]).argmax(1) == np.arange(16) * 3).all()
 
 
+@pytest.mark.parametrize("N,dt", [(1000, "bf16"), (4096, "bf16"), (515, "f32"), (20000, "bf16")])
+@pytest.mark.parametrize("red", ["row_softmax", "row_logsumexp"])
+def test_elementwise_softmax_and_logsumexp_with_minus_infinity_masks(fc, orc, N, dt, red):
+    """An additive mask of 0 / -inf (causal: row i keeps columns <= 37 i + 5; plus a row that keeps a single
+    column in the middle and rows masked on the left): masked entries get probability exactly 0, whole
+    stretches of -inf at the start, in the middle or at the end of a lane's columns leave the rest intact."""
+    M = 24
+    ch = replace(wl.scale_add_softmax(M, N, dtype=dt), reduce=red, store_main=False)   # (a stored main output would hold the -inf itself)
+    ins = wl.make_inputs(ch, 12)
+    keep = np.arange(N)[None, :] <= (37 * np.arange(M)[:, None] + 5)
+    keep[3] = False; keep[3, N // 2] = True
+    keep[5] = np.arange(N) >= N - 9
+    keep[7] = (np.arange(N) // 64) % 2 == 1
+    mask = np.where(keep, 0.0, -np.inf).astype(np.float32)
+    ins[1] = rng.store(mask, dt)
+    outs, ref, _ = run_and_check(fc, orc, ch, ins=ins)
+    if red == "row_softmax":
+        got = util.to_f64(outs[0])
+        assert (got[~keep] == 0.0).all()
+        np.testing.assert_allclose(got.sum(1), 1.0, atol=2e-2 if dt == "bf16" else 1e-4)
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
