@@ -190,7 +190,7 @@ struct EwFastParams {
     int N;
     int red_kind;           // fc_reduce of the row reduction (when the kernel is built with one)
     int is_f16;             // x, residual and y are IEEE half instead of bf16
-    int stash;              // row softmax: the row's fp32 values wait in shared memory for the second pass
+    int stash;              // row softmax: the row's exponentials wait in shared memory for the second pass
     float pre_scale;        // a SCALE op in front of everything, folded into gamma (PRE is then always affine;
                             // vec0 == null means gamma = 1, vec1 == null means beta = 0)
 };
@@ -274,13 +274,9 @@ __device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const 
 
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
 __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
-                                         int red_kind, bool f16, float& run_m, float& run_s, float4* stash) {
+                                         int red_kind, bool f16, float& run_m, float& run_s, uint4* stash_e, float* stash_m) {
     float2 v[4];
     ew_values<PRE, ACT, RES>(xq, rq, svec, N, c, f16, v);
-    if (stash) {   // same de-interleaved layout as the vectors: conflict-free 16-byte accesses
-        stash[c] = make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
-        stash[(N >> 3) + c] = make_float4(v[2].x, v[2].y, v[3].x, v[3].y);
-    }
     if (STORE) {
         uint4 q;
         q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
@@ -303,13 +299,25 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
         const float base = nm == -CUDART_INF_F ? 0.0f : nm;
         const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-base, -base);
         float2 cs = make_float2(0.0f, 0.0f);
+        float2 ex[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float2 e = __ffma2_rn(v[j], l2e, mnm);
-            cs = __fadd2_rn(cs, make_float2(exp2_fast(e.x), exp2_fast(e.y)));
+            ex[j] = make_float2(exp2_fast(e.x), exp2_fast(e.y));
+            cs = __fadd2_rn(cs, ex[j]);
         }
         run_s = fmaf(run_s, exp2_fast(run_m - base), cs.x + cs.y);
         run_m = nm;
+        if (stash_e) {
+            // Row softmax: the exponentials (in (0, 1], taken against the running maximum at this chunk) wait in the
+            // output's 16-bit type, the running maximum beside them; the second pass rescales by
+            // 2^(this maximum - row maximum) / sum.  Two roundings of 2^-9 (bf16) relative at most.
+            uint4 q;
+            q.x = pack16x2(ex[0].x, ex[0].y, f16); q.y = pack16x2(ex[1].x, ex[1].y, f16);
+            q.z = pack16x2(ex[2].x, ex[2].y, f16); q.w = pack16x2(ex[3].x, ex[3].y, f16);
+            stash_e[c] = q;
+            stash_m[c] = nm;
+        }
     }
 }
 
@@ -372,8 +380,14 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
     const int chunks = N >> 3;
     const int warp = threadIdx.x >> 5;
     const long long row_step = (long long) gridDim.x * kWarps;
-    float4* stash = nullptr;
-    if (SOFTMAX && p.stash) stash = reinterpret_cast<float4*>(svec + (PRE == kPreNone ? 0 : (PRE == kPreAffine ? 2 : 1) * N)) + warp * (N >> 2);
+    // row softmax: per warp N/8 chunks of eight 16-bit exponentials (16 bytes each), then N/8 running maxima
+    uint4* stash_e = nullptr;
+    float* stash_m = nullptr;
+    if (SOFTMAX && p.stash) {
+        float* base = svec + (PRE == kPreNone ? 0 : (PRE == kPreAffine ? 2 : 1) * N);
+        stash_e = reinterpret_cast<uint4*>(base) + (size_t) warp * chunks;
+        stash_m = base + (size_t) kWarps * chunks * 4 + (size_t) warp * chunks;
+    }
     for (long long row = (long long) blockIdx.x * kWarps + warp; row < p.M; row += row_step) {
         const uint4* xr = p.x + row * chunks;
         const uint4* rr = RES ? p.res + row * chunks : nullptr;
@@ -397,7 +411,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                 const int c = c0 + 32 * g;
                 if (c < chunks)
                     ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind, p.is_f16 != 0, run_m, run_s,
-                                                        SOFTMAX ? stash : nullptr);
+                                                        SOFTMAX ? stash_e : nullptr, stash_m);
             }
         }
         if (LSE && !SOFTMAX && p.red_kind >= FC_RED_ROW_SUM) {
@@ -421,16 +435,31 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                 run_m = nm;
             }
             if constexpr (SOFTMAX) {
-                // Second pass over the row: the values wait in shared memory (rows of up to a few thousand columns),
-                // else the inputs are read again, from L2 where they still are, and the values computed again;
-                // stored as 2^(v log2e - max) / sum.
+                // Second pass over the row: the exponentials wait in shared memory (rows of up to some 8000 columns)
+                // and are rescaled; else the inputs are read again, from L2 where they still are, the values
+                // computed again and stored as 2^(v log2e - max) / sum.
                 float inv;
                 asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(run_s));
                 const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-run_m, -run_m), inv2 = make_float2(inv, inv);
                 uint4* pr = p.y + row * chunks;
-                for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
-                    uint4 xv[kGroup], rv[kGroup];
-                    if (!stash) {
+                if (stash_e) {
+                    for (int c = lane; c < chunks; c += 32) {
+                        const uint4 q = stash_e[c];
+                        const float cmx = stash_m[c];
+                        // everything up to this chunk was -inf: its exponentials are zeros, any finite factor will do
+                        const float f = cmx == -CUDART_INF_F ? 0.0f : exp2_fast(cmx - run_m) * inv;
+                        const float2 f2 = make_float2(f, f);
+                        const bool h = p.is_f16 != 0;
+                        const float2 a = __fmul2_rn(unpack16x2(q.x, h), f2), b = __fmul2_rn(unpack16x2(q.y, h), f2);
+                        const float2 cc = __fmul2_rn(unpack16x2(q.z, h), f2), d = __fmul2_rn(unpack16x2(q.w, h), f2);
+                        uint4 o;
+                        o.x = pack16x2(a.x, a.y, h); o.y = pack16x2(b.x, b.y, h);
+                        o.z = pack16x2(cc.x, cc.y, h); o.w = pack16x2(d.x, d.y, h);
+                        st_stream(pr + c, o);
+                    }
+                } else {
+                    for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
+                        uint4 xv[kGroup], rv[kGroup];
 #pragma unroll
                         for (int g = 0; g < kGroup; ++g) {
                             const int c = c0 + 32 * g;
@@ -439,28 +468,22 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                                 if (RES) rv[g] = __ldcg(rr + c);
                             }
                         }
-                    }
 #pragma unroll
-                    for (int g = 0; g < kGroup; ++g) {
-                        const int c = c0 + 32 * g;
-                        if (c < chunks) {
-                            float2 v[4];
-                            if (stash) {
-                                const float4 a = stash[c], b = stash[chunks + c];
-                                v[0] = make_float2(a.x, a.y); v[1] = make_float2(a.z, a.w);
-                                v[2] = make_float2(b.x, b.y); v[3] = make_float2(b.z, b.w);
-                            } else {
+                        for (int g = 0; g < kGroup; ++g) {
+                            const int c = c0 + 32 * g;
+                            if (c < chunks) {
+                                float2 v[4];
                                 ew_values<PRE, ACT, RES>(xv[g], rv[g], svec, N, c, p.is_f16 != 0, v);
-                            }
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float2 e = __ffma2_rn(v[j], l2e, mnm);
-                                v[j] = __fmul2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), inv2);
+                                for (int j = 0; j < 4; ++j) {
+                                    const float2 e = __ffma2_rn(v[j], l2e, mnm);
+                                    v[j] = __fmul2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), inv2);
+                                }
+                                uint4 q;
+                                q.x = pack16x2(v[0].x, v[0].y, p.is_f16 != 0); q.y = pack16x2(v[1].x, v[1].y, p.is_f16 != 0);
+                                q.z = pack16x2(v[2].x, v[2].y, p.is_f16 != 0); q.w = pack16x2(v[3].x, v[3].y, p.is_f16 != 0);
+                                st_stream(pr + c, q);
                             }
-                            uint4 q;
-                            q.x = pack16x2(v[0].x, v[0].y, p.is_f16 != 0); q.y = pack16x2(v[1].x, v[1].y, p.is_f16 != 0);
-                            q.z = pack16x2(v[2].x, v[2].y, p.is_f16 != 0); q.w = pack16x2(v[3].x, v[3].y, p.is_f16 != 0);
-                            st_stream(pr + c, q);
                         }
                     }
                 }
@@ -517,12 +540,13 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
     EwFastParams f = f_in;
     size_t smem = PRE == kPreNone ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
     f.stash = 0;
-    if (f.red_kind == FC_RED_ROW_SOFTMAX && smem + (size_t) kWarps * f.N * 4 <= 200 * 1024) {
+    const size_t stash_bytes = (size_t) kWarps * (f.N / 8) * (16 + 4);   // per chunk: eight 16-bit values and a maximum
+    if (f.red_kind == FC_RED_ROW_SOFTMAX && smem + stash_bytes <= 200 * 1024) {
         f.stash = 1;
-        smem += (size_t) kWarps * f.N * 4;
+        smem += stash_bytes;
     }
     long long ctas = (f.M + kWarps - 1) / kWarps;
-    int per_sm = smem > 0 ? (int) ((200 * 1024) / smem) : 4;
+    int per_sm = smem > 0 ? (int) ((227 * 1024) / (smem + 1024)) : 4;   // 228 KB per SM, 1 KB of it reserved per CTA
     per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);
     if (ctas > (long long) num_sms * per_sm) ctas = (long long) num_sms * per_sm;
     // the dynamic shared-memory limit of each instantiation is raised once per device, to the maximum
