@@ -110,7 +110,9 @@ typedef enum {
     FC_OP_GELU_TANH = 3,  /* v  = 0.5 v (1 + tanh(sqrt(2/pi) (v + 0.044715 v^3)))                    */
     FC_OP_SCALE = 4,      /* v *= f0                                                                 */
     FC_OP_CLAMP = 5,      /* v  = min(max(v, f0), f1)                                                */
-    FC_OP_ADD_TENSOR = 6, /* v += tensor[in0][m][n]              same shape as the main output       */
+    FC_OP_ADD_TENSOR = 6, /* v += tensor[in0][m][n]              same shape as the main output; may hold -inf (an additive
+                             mask): ROW_SOFTMAX gives such entries exactly 0 and ROW_LOGSUMEXP ignores them; a row of -inf
+                             only has no softmax (NaN, as the definition gives)                       */
     FC_OP_LINEAR = 7      /* v[m][:] = round16(v[m][:]) W^T, W = inputs[in0] of shape [N_next][N] in the chain's 16-bit
                              type: another linear layer.  The row is rounded to that type first (it is the tensor-core
                              operand, and what an unfused sequence would have stored); N becomes N_next for the ops

@@ -504,10 +504,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 run_m = fmaxf(run_m, cm);
                             } else {
                                 const float nm = fmaxf(run_m, cm * kLog2e);
+                                // only -inf so far (an additive mask): exponents against 0, so that they stay -inf
+                                const float base = nm == -CUDART_INF_F ? 0.0f : nm;
                                 float cs = 0.0f;
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast(fmaf(v[j], kLog2e, -nm)) : 0.0f;
-                                run_s = fmaf(run_s, exp2_fast(run_m - nm), cs);
+                                for (int j = 0; j < 16; ++j) cs += n0 + j < p.N ? exp2_fast(fmaf(v[j], kLog2e, -base)) : 0.0f;
+                                run_s = fmaf(run_s, exp2_fast(run_m - base), cs);
                                 run_m = nm;
                             }
                         } else {
@@ -580,7 +582,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float sm = 0.0f;
                 {
                     const float2 l2e = make_float2(kLog2e, kLog2e);
-                    const float2 moff = make_float2(-mx * kLog2e, -mx * kLog2e);
+                    // a half row of -inf only (an additive mask): exponents against 0, so that they stay -inf
+                    const float mbase = mx == -CUDART_INF_F ? 0.0f : mx;
+                    const float2 moff = make_float2(-mbase * kLog2e, -mbase * kLog2e);
                     float2 acc2 = make_float2(0.0f, 0.0f);
                     tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                         const int n0 = n_half + c * 16;

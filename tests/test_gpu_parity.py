@@ -139,6 +139,26 @@ def test_elementwise_softmax_and_logsumexp_with_minus_infinity_masks(fc, orc, N,
         np.testing.assert_allclose(got.sum(1), 1.0, atol=2e-2 if dt == "bf16" else 1e-4)
 
 
+@pytest.mark.parametrize("red", ["row_softmax", "row_logsumexp"])
+def test_gemm_softmax_and_logsumexp_with_minus_infinity_mask(fc, orc, red):
+    """Scores = A B^T * scale + mask with a causal 0 / -inf mask (the attention-score chain): whole tiles, half
+    rows of a tile and single columns of -inf; masked probabilities are exactly 0."""
+    M, N, K = 300, 1000, 136
+    base = wl.gemm_softmax(M, N, K, "var")
+    rec = base.input_recipe + (("mask", "bf16", (M, N), "normal", 0.0, 1.0),)
+    ch = replace(base, ops=(("scale", 0.5), ("add_tensor", 2)), reduce=red, store_main=False, input_recipe=rec)
+    ins = wl.make_inputs(ch, 4)
+    keep = np.arange(N)[None, :] <= (3 * np.arange(M)[:, None] + 2)
+    keep[7] = False; keep[7, 600] = True
+    keep[9] = np.arange(N) >= 900
+    ins[2] = rng.store(np.where(keep, 0.0, -np.inf).astype(np.float32), "bf16")
+    outs, ref, _ = run_and_check(fc, orc, ch, ins=ins)
+    if red == "row_softmax":
+        got = util.to_f64(outs[0])
+        assert (got[~keep] == 0.0).all()
+        np.testing.assert_allclose(got.sum(1), 1.0, atol=2e-2)
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
