@@ -75,6 +75,35 @@ __device__ __forceinline__ float load_scalar(const void* p, int dt, long long i)
     return __ldg((const float*) p + i);
 }
 
+// kN consecutive elements starting at element i of a tensor of type dt; elements from `valid` on are left at 0.
+// Eight whole elements on a 16-byte boundary are read with one (16-bit types) or two (fp32) vector loads.
+template <int kN>
+__device__ __forceinline__ void load_run(const void* p, int dt, long long i, long long valid, float (&out)[kN]) {
+    if (kN == 8 && valid >= 8) {
+        if (dt != FC_F32) {
+            const unsigned short* q = (const unsigned short*) p + i;
+            if ((reinterpret_cast<uintptr_t>(q) & 15) == 0) {
+                const uint4 w = __ldg(reinterpret_cast<const uint4*>(q));
+                const bool h = dt == FC_F16;
+                const float2 a = unpack16x2(w.x, h), b = unpack16x2(w.y, h), c = unpack16x2(w.z, h), d = unpack16x2(w.w, h);
+                out[0] = a.x; out[1] = a.y; out[2 % kN] = b.x; out[3 % kN] = b.y;
+                out[4 % kN] = c.x; out[5 % kN] = c.y; out[6 % kN] = d.x; out[7 % kN] = d.y;
+                return;
+            }
+        } else {
+            const float* q = (const float*) p + i;
+            if ((reinterpret_cast<uintptr_t>(q) & 15) == 0) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(q)), b = __ldg(reinterpret_cast<const float4*>(q) + 1);
+                out[0] = a.x; out[1 % kN] = a.y; out[2 % kN] = a.z; out[3 % kN] = a.w;
+                out[4 % kN] = b.x; out[5 % kN] = b.y; out[6 % kN] = b.z; out[7 % kN] = b.w;
+                return;
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kN; ++j) out[j] = j < valid ? load_scalar(p, dt, i + j) : 0.0f;
+}
+
 // Apply the op list to kN consecutive columns n0.. of row m (values in registers).
 // `ld` is the row pitch (elements) of ADD_TENSOR operands; columns >= n_limit are not touched
 // in memory (their register values are garbage-in, garbage-out and must not be stored).
@@ -85,17 +114,21 @@ __device__ __forceinline__ void apply_ops(float (&v)[kN], const DevOps& ops, lon
     for (int i = 0; i < ops.n; ++i) {
         const DevOp& op = ops.op[i];
         switch (op.kind) {
-            case FC_OP_BIAS_N:
+            case FC_OP_BIAS_N: {
+                float b[kN];
+                load_run<kN>(op.p0, op.dt0, n0, n_limit - n0, b);
 #pragma unroll
-                for (int j = 0; j < kN; ++j)
-                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, n0 + j);
+                for (int j = 0; j < kN; ++j) v[j] += b[j];
                 break;
-            case FC_OP_AFFINE_N:
+            }
+            case FC_OP_AFFINE_N: {
+                float g[kN], b[kN];
+                load_run<kN>(op.p0, op.dt0, n0, n_limit - n0, g);
+                load_run<kN>(op.p1, op.dt1, n0, n_limit - n0, b);
 #pragma unroll
-                for (int j = 0; j < kN; ++j)
-                    if (n0 + j < n_limit)
-                        v[j] = fmaf(v[j], load_scalar(op.p0, op.dt0, n0 + j), load_scalar(op.p1, op.dt1, n0 + j));
+                for (int j = 0; j < kN; ++j) v[j] = n0 + j < n_limit ? fmaf(v[j], g[j], b[j]) : v[j];
                 break;
+            }
             case FC_OP_RELU:
 #pragma unroll
                 for (int j = 0; j < kN; ++j) v[j] = v[j] < 0.0f ? 0.0f : v[j];
@@ -112,11 +145,13 @@ __device__ __forceinline__ void apply_ops(float (&v)[kN], const DevOps& ops, lon
 #pragma unroll
                 for (int j = 0; j < kN; ++j) v[j] = fminf(fmaxf(v[j], op.f0), op.f1);
                 break;
-            case FC_OP_ADD_TENSOR:
+            case FC_OP_ADD_TENSOR: {
+                float t[kN];
+                load_run<kN>(op.p0, op.dt0, m * ld + n0, n_limit - n0, t);
 #pragma unroll
-                for (int j = 0; j < kN; ++j)
-                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, m * ld + n0 + j);
+                for (int j = 0; j < kN; ++j) v[j] += t[j];
                 break;
+            }
             default:
                 break;
         }
