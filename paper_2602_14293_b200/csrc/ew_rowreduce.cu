@@ -190,6 +190,7 @@ struct EwFastParams {
     int N;
     int red_kind;           // fc_reduce of the row reduction (when the kernel is built with one)
     int is_f16;             // x, residual and y are IEEE half instead of bf16
+    float post_scale, post_lo, post_hi;   // ACT with kActPost: v = clamp(v * post_scale, lo, hi) after the activation
     int stash;              // row softmax: the row's exponentials wait in shared memory for the second pass
     float pre_scale;        // a SCALE op in front of everything, folded into gamma (PRE is then always affine;
                             // vec0 == null means gamma = 1, vec1 == null means beta = 0)
@@ -207,13 +208,18 @@ __device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
 
 constexpr int kPreNone = 0, kPreBias = 1, kPreAffine = 2;
 constexpr int kActNone = 0, kActRelu = 1, kActGeluPrecise = 2, kActGeluFast = 3;
+constexpr int kActPost = 4;   // flag on top of the activation: a scale and a clamp follow it (before the residual)
 constexpr int kGroup = 4;   // chunks in flight per lane and tensor
 
 // One chunk (8 columns starting at column 8*c) of one row: ops in packed fp32x2, one 16-byte store,
 // and the chunk's contribution to the running (max, sum) of the row (log2 domain).
 // The values of one chunk (8 columns starting at column 8*c) after the ops, as four fp32 pairs.
-template <int PRE, int ACT, bool RES>
-__device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const float* svec, int N, int c, bool f16, float2 (&v)[4]) {
+template <int PRE, int ACT_, bool RES_>
+__device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const float* svec, int N, int c, bool f16, float2 (&v)[4],
+                                          const EwFastParams& prm) {
+    constexpr int ACT = ACT_ & 3;
+    constexpr bool kPost = (ACT_ & kActPost) != 0;
+    constexpr bool RES = RES_ && !kPost;   // with post ops the residual is added behind them, not inside the activation
     v[0] = unpack16x2(xq.x, f16);
     v[1] = unpack16x2(xq.y, f16);
     v[2] = unpack16x2(xq.z, f16);
@@ -238,7 +244,7 @@ __device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const 
         }
     }
     float2 r[4];
-    if (RES) {
+    if (RES_) {
         r[0] = unpack16x2(rq.x, f16);
         r[1] = unpack16x2(rq.y, f16);
         r[2] = unpack16x2(rq.z, f16);
@@ -268,15 +274,21 @@ __device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const 
         } else if (RES) {
             t = __fadd2_rn(t, r[j]);
         }
+        if (kPost) {
+            t = __fmul2_rn(t, make_float2(prm.post_scale, prm.post_scale));
+            t = make_float2(fminf(fmaxf(t.x, prm.post_lo), prm.post_hi), fminf(fmaxf(t.y, prm.post_lo), prm.post_hi));
+            if (RES_) t = __fadd2_rn(t, r[j]);
+        }
         v[j] = t;
     }
 }
 
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
 __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
-                                         int red_kind, bool f16, float& run_m, float& run_s, uint4* stash_e, float* stash_m) {
+                                         int red_kind, bool f16, float& run_m, float& run_s, uint4* stash_e, float* stash_m,
+                                         const EwFastParams& prm) {
     float2 v[4];
-    ew_values<PRE, ACT, RES>(xq, rq, svec, N, c, f16, v);
+    ew_values<PRE, ACT, RES>(xq, rq, svec, N, c, f16, v, prm);
     if (STORE) {
         uint4 q;
         q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
@@ -411,7 +423,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                 const int c = c0 + 32 * g;
                 if (c < chunks)
                     ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind, p.is_f16 != 0, run_m, run_s,
-                                                        SOFTMAX ? stash_e : nullptr, stash_m);
+                                                        SOFTMAX ? stash_e : nullptr, stash_m, p);
             }
         }
         if (LSE && !SOFTMAX && p.red_kind >= FC_RED_ROW_SUM) {
@@ -473,7 +485,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                             const int c = c0 + 32 * g;
                             if (c < chunks) {
                                 float2 v[4];
-                                ew_values<PRE, ACT, RES>(xv[g], rv[g], svec, N, c, p.is_f16 != 0, v);
+                                ew_values<PRE, ACT, RES>(xv[g], rv[g], svec, N, c, p.is_f16 != 0, v, p);
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
                                     const float2 e = __ffma2_rn(v[j], l2e, mnm);
@@ -494,7 +506,8 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
 
 }  // namespace
 
-// Recognise [bias | affine]? -> [relu | gelu]? -> [add tensor]? and fill the fast-path parameters.
+// Recognise [scale]? -> [bias | affine]? -> [relu | gelu]? -> [scale]? -> [clamp]? -> [add tensor]? and fill the
+// fast-path parameters.
 static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, bool* res) {
     if (p.x_dt == FC_F32 || (p.y && p.y_dt != p.x_dt)) return false;
     if (p.N % 8 != 0 || p.N > 24576 || p.M >= 0x7fffffffLL) return false;
@@ -521,6 +534,15 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
         // in this kernel and is the more accurate one; without, tanh.approx saves a MUFU operation
         *act = p.ops.op[i].kind == FC_OP_RELU ? kActRelu : (p.reduce == FC_RED_ROW_LOGSUMEXP ? kActGeluPrecise : kActGeluFast);
         ++i;
+    }
+    // [scale]? [clamp]? behind the activation: one flag, with neutral values for the one that is absent.  Not
+    // instantiated for the softmax and reduction-only kernels.
+    f->post_scale = 1.0f; f->post_lo = -INFINITY; f->post_hi = INFINITY;
+    if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_SCALE || p.ops.op[i].kind == FC_OP_CLAMP)) {
+        if (p.reduce == FC_RED_ROW_SOFTMAX || (p.reduce != FC_RED_NONE && !p.y)) return false;
+        if (p.ops.op[i].kind == FC_OP_SCALE) f->post_scale = p.ops.op[i++].f0;
+        if (i < p.ops.n && p.ops.op[i].kind == FC_OP_CLAMP) { f->post_lo = p.ops.op[i].f0; f->post_hi = p.ops.op[i].f1; ++i; }
+        *act |= kActPost;
     }
     if (i < p.ops.n && p.ops.op[i].kind == FC_OP_ADD_TENSOR) {
         if (p.ops.op[i].dt0 != p.x_dt || (reinterpret_cast<uintptr_t>(p.ops.op[i].p0) & 15)) return false;
@@ -562,9 +584,11 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
         kernel<<<(unsigned) ctas, kThreads, smem, stream>>>(f);
         return cudaGetLastError();
     };
-    if (f.red_kind == FC_RED_ROW_SOFTMAX) return go(ew_rows_kernel<PRE, ACT, RES, true, false, true>, 3);
+    if constexpr ((ACT & kActPost) == 0) {
+        if (f.red_kind == FC_RED_ROW_SOFTMAX) return go(ew_rows_kernel<PRE, ACT, RES, true, false, true>, 3);
+        if (lse && !store) return go(ew_rows_kernel<PRE, ACT, RES, true, false>, 1);
+    }
     if (lse && store) return go(ew_rows_kernel<PRE, ACT, RES, true, true>, 0);
-    if (lse) return go(ew_rows_kernel<PRE, ACT, RES, true, false>, 1);
     return go(ew_rows_kernel<PRE, ACT, RES, false, true>, 2);
 }
 
@@ -579,13 +603,17 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
     if (!narrow && match_fast(p, &f, &pre, &act, &res) && (lse || p.y)) {
         const bool store = p.y != nullptr && p.reduce != FC_RED_ROW_SOFTMAX;   // softmax stores in its second pass
 #define FC_EW_CASE(PRE_, ACT_)                                                                       \
-    if (pre == PRE_ && act == ACT_)                                                                  \
-        return res ? launch_fast<PRE_, ACT_, true>(f, lse, store, num_sms, stream)                  \
-                   : launch_fast<PRE_, ACT_, false>(f, lse, store, num_sms, stream);
+    if (pre == (PRE_) && act == (ACT_))                                                              \
+        return res ? launch_fast<(PRE_), (ACT_), true>(f, lse, store, num_sms, stream)              \
+                   : launch_fast<(PRE_), (ACT_), false>(f, lse, store, num_sms, stream);
         FC_EW_CASE(kPreNone, kActNone) FC_EW_CASE(kPreNone, kActRelu) FC_EW_CASE(kPreNone, kActGeluPrecise)
         FC_EW_CASE(kPreBias, kActNone) FC_EW_CASE(kPreBias, kActRelu) FC_EW_CASE(kPreBias, kActGeluPrecise)
         FC_EW_CASE(kPreAffine, kActNone) FC_EW_CASE(kPreAffine, kActRelu) FC_EW_CASE(kPreAffine, kActGeluPrecise)
         FC_EW_CASE(kPreNone, kActGeluFast) FC_EW_CASE(kPreBias, kActGeluFast) FC_EW_CASE(kPreAffine, kActGeluFast)
+        FC_EW_CASE(kPreNone, kActNone | kActPost) FC_EW_CASE(kPreNone, kActRelu | kActPost) FC_EW_CASE(kPreNone, kActGeluPrecise | kActPost)
+        FC_EW_CASE(kPreBias, kActNone | kActPost) FC_EW_CASE(kPreBias, kActRelu | kActPost) FC_EW_CASE(kPreBias, kActGeluPrecise | kActPost)
+        FC_EW_CASE(kPreAffine, kActNone | kActPost) FC_EW_CASE(kPreAffine, kActRelu | kActPost) FC_EW_CASE(kPreAffine, kActGeluPrecise | kActPost)
+        FC_EW_CASE(kPreNone, kActGeluFast | kActPost) FC_EW_CASE(kPreBias, kActGeluFast | kActPost) FC_EW_CASE(kPreAffine, kActGeluFast | kActPost)
 #undef FC_EW_CASE
     }
     const bool precise = false;   // tanh.approx is accurate to 6e-6 here (see gelu_tanh)

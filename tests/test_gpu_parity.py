@@ -159,6 +159,24 @@ def test_gemm_softmax_and_logsumexp_with_minus_infinity_mask(fc, orc, red):
         np.testing.assert_allclose(got.sum(1), 1.0, atol=2e-2)
 
 
+@pytest.mark.parametrize("ops", [
+    (("bias_n", 2), ("relu",), ("scale", 0.5), ("clamp", -0.25, 0.75), ("add_tensor", 3)),
+    (("affine_n", 1, 2), ("gelu_tanh",), ("clamp", -0.5, 1.5)),
+    (("gelu_tanh",), ("scale", 3.0)),
+    (("scale", 0.5), ("bias_n", 1), ("scale", 2.0), ("clamp", -1.0, 1.0), ("add_tensor", 3)),
+    (("clamp", -0.3, 0.3),),
+])
+@pytest.mark.parametrize("red", ["none", "row_logsumexp", "row_sum"])
+@pytest.mark.parametrize("M,N,dt", [(37, 512, "bf16"), (64, 4096, "f16"), (5, 264, "bf16")])
+def test_elementwise_scale_and_clamp_behind_the_activation(fc, orc, ops, red, M, N, dt):
+    """Op lists [scale] [bias | affine] [relu | gelu] [scale] [clamp] [add tensor] take the row kernel (16-bit
+    storage, N a multiple of 8); the residual is then added behind the clamp, not inside the activation."""
+    base = wl.affine_gelu_residual_lse(M, N)
+    if dt == "f16":
+        base = _as_f16(base)
+    run_and_check(fc, orc, replace(base, ops=ops, reduce=red, store_main=True), 13)
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
