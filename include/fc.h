@@ -23,7 +23,7 @@
  *              row softmax, global average pool over (oh, ow)
  *
  * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
- * allocates device memory and never synchronises; it enqueues at most two memsets and one to three
+ * allocates device memory and never synchronises; it enqueues at most two memsets and one to four
  * kernels on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
  *
  * Pointers.  Unless a function says "host", every fc_tensor.ptr is a DEVICE pointer.

@@ -668,7 +668,6 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? 1 : 0;
             p.a_packed = packed_taps(spec);
             const size_t out_elems = p.pool ? (size_t) spec->batch * (p.OH / 2) * (p.OW / 2) * spec->Cout : (size_t) spec->batch * spec->Cout;
-            if ((e = cudaMemsetAsync(p.out, 0, out_elems * 4, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             const void* image = inputs[0].ptr;
             const void* weights = inputs[1].ptr;
             size_t head = 0;   // workspace bytes in front of the split scratch
@@ -694,6 +693,10 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             CUtensorMap tmA, tmB;
             if ((st = encode_im2col(&tmA, spec, image, p.a_packed != 0))) return st;
             if ((st = encode_2d(&tmB, weights, spec->Cout, p.K, bn / 2, spec->in_dtype))) return st;
+            // The pooled output is cleared by a kernel directly in front of the convolution, which is launched
+            // programmatically behind it: its loads and MMAs start at once, only its epilogue warps wait for the zeros.
+            if ((e = launch_zero_fill(p.out, out_elems * 4, dev->num_sms, stream, &launches)) != cudaSuccess) return cuda_fail(e, "zero-fill launch");
+            p.after_zero_fill = 1;
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }

@@ -81,6 +81,10 @@ size_t collapse_workspace_bytes(long long N, long long K);
 cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,
                                    int* launches);
 
+// Zeroes `bytes` bytes (a multiple of 4, 4-byte aligned) with a kernel that lets the next kernel in the stream be
+// scheduled at once: the pooled outputs of the convolution are cleared while its first tiles are in the main loop.
+cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches);
+
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
     int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row reduction to one value
@@ -99,6 +103,8 @@ struct TcParams {
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
     int pool;                   // mode 2: 0 global average pool, 1 2x2 max-pool (out pre-zeroed, values >= 0)
+    int after_zero_fill;        // mode 2: launched programmatically behind the kernel that zeroes `out`; the epilogue warps wait
+                                // for that kernel before their first update of `out`, everything else starts at once
     int a_packed;               // mode 2: 1 = a k-block of A is eight 8-channel chunks, one per filter tap (Cin == 8)
     int* status;                // device status word
     int expect_extra;           // testing only: arrivals a wait expects beyond those that will come (mode 1: the panel

@@ -323,6 +323,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool precise = false;   // tanh.approx GELU is accurate to 6e-6 on sm_100a (see gelu_tanh)
         const bool out_vec = (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 && (p.N & 7) == 0;
         const uint32_t tempty_leader = ptx::mapa(ptx::smem_u32(&ctrl->tempty[0]), 0);
+        if constexpr (kConv) {
+            // the pooled output is zeroed by the kernel in front, which this one was allowed to overtake: only
+            // these warps, the ones that update the output, wait for it (a no-op under an ordinary launch)
+            if (p.after_zero_fill) asm volatile("griddepcontrol.wait;" ::: "memory");
+        }
         uint32_t tile_iter = 0;
         for (int u = cluster_id; u < total_units; u += num_clusters, ++tile_iter) {
             const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
@@ -796,11 +801,13 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // used only behind the zero-fill kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -867,6 +874,7 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     }
     if (!tmA) return cudaSuccess;   // planning only
     cfg.gridDim = dim3(2 * clusters);
+    cfg.numAttrs = (MODE == 2 || MODE == 4) && p.after_zero_fill ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, *tmA, *tmB, q);
 }
 

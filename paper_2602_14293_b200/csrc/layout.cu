@@ -93,7 +93,32 @@ __global__ void __launch_bounds__(256) cfirst_to_clast_kernel(const unsigned sho
     }
 }
 
+__global__ void __launch_bounds__(256) zero_fill_kernel(uint32_t* ptr, size_t words) {
+    // the kernel behind this one may be scheduled now; it waits (griddepcontrol.wait) where it first needs the zeros
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const size_t stride = (size_t) gridDim.x * blockDim.x;
+    size_t i = (size_t) blockIdx.x * blockDim.x + threadIdx.x;
+    if ((reinterpret_cast<uintptr_t>(ptr) & 15) == 0) {
+        uint4* p4 = reinterpret_cast<uint4*>(ptr);
+        const size_t quads = words >> 2;
+        for (size_t q = i; q < quads; q += stride) p4[q] = make_uint4(0u, 0u, 0u, 0u);
+        for (size_t w = (quads << 2) + i; w < words; w += stride) ptr[w] = 0u;
+    } else {
+        for (; i < words; i += stride) ptr[i] = 0u;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches) {
+    const size_t words = bytes / 4;
+    size_t blocks = (words / 4 + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > (size_t) num_sms * 4) blocks = (size_t) num_sms * 4;
+    zero_fill_kernel<<<(unsigned) blocks, 256, 0, stream>>>((uint32_t*) ptr, words);
+    ++*launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,
                                    int* launches) {
