@@ -32,6 +32,7 @@ __device__ __forceinline__ MaxSum block_merge(MaxSum a, MaxSum* smem /* [kWarps]
 template <bool kPreciseGelu>
 __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) {
     __shared__ MaxSum red[kWarps];
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // programmatic launch: see ew_rows_kernel
     const long long N = p.N;
     const int ebytes = p.x_dt == FC_F32 ? 4 : 2;
     const int ybytes = p.y_dt == FC_F32 ? 4 : 2;
@@ -338,6 +339,9 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
 template <int PRE, int ACT, bool RES, bool LSE, bool STORE, bool SOFTMAX = false>
 __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(const EwFastParams p) {
     extern __shared__ float svec[];   // PRE != none: vec0 as fp32 [N] (chunk halves de-interleaved), then vec1 [N]
+    // Launched with programmatic stream serialization: the CTAs are scheduled while the kernel in front drains and
+    // wait here, before their first access to global memory, until it has completed and its writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int N = p.N;
     if (PRE != kPreNone) {
         // Every CTA converts the vectors once.  This prologue is a fixed cost of the launch (it measured 8 us
@@ -581,8 +585,17 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < 64) raised[variant][dev] = true;
         }
-        kernel<<<(unsigned) ctas, kThreads, smem, stream>>>(f);
-        return cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned) ctas);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, f);
     };
     if constexpr ((ACT & kActPost) == 0) {
         if (f.red_kind == FC_RED_ROW_SOFTMAX) return go(ew_rows_kernel<PRE, ACT, RES, true, false, true>, 3);
@@ -621,11 +634,16 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
     if (!lse) work = (p.M * ((p.N + 7) / 8) + kThreads - 1) / kThreads;
     long long grid = work < (long long) num_sms * 8 ? work : (long long) num_sms * 8;
     if (grid < 1) grid = 1;
-    if (precise)
-        ew_generic_kernel<true><<<(unsigned) grid, kThreads, 0, stream>>>(p);
-    else
-        ew_generic_kernel<false><<<(unsigned) grid, kThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned) grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return precise ? cudaLaunchKernelEx(&cfg, ew_generic_kernel<true>, p) : cudaLaunchKernelEx(&cfg, ew_generic_kernel<false>, p);
 }
 
 }  // namespace fc

@@ -30,6 +30,9 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 __global__ void __launch_bounds__(kGemmThreads) gemm_f32_kernel(const GemmF32Params p) {
     extern __shared__ __align__(16) float smem_f32[];
+    // launched with programmatic stream serialization: scheduled while the kernel in front drains, and held here,
+    // before the first access to global memory, until that kernel has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;                   // columns tx, tx + 16; rows ty, ty + 8
     const int m0 = blockIdx.x * kTM, n0 = blockIdx.y * kTN;
@@ -193,9 +196,18 @@ cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* la
     }
     dim3 grid((p.M + kTM - 1) / kTM, (p.N + kTN - 1) / kTN);   // M tiles in x (up to 2^31 - 1), N tiles in y (up to 65535)
     // a problem of one slab (K <= 128) asks for one stage only
-    gemm_f32_kernel<<<grid, kGemmThreads, p.K <= kKS ? kSmemBytes / kStages : kSmemBytes, stream>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = p.K <= kKS ? kSmemBytes / kStages : kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
     *launches += 1;
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, gemm_f32_kernel, p);
 }
 
 }  // namespace fc

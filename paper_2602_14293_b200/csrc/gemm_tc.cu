@@ -211,6 +211,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::cluster_sync();   // the peer's barriers exist before anything is signalled on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
+    // Launched with programmatic stream serialization: everything above ran while the kernel in front was draining;
+    // nothing below touches global memory before that kernel has completed.  (Behind the zero-fill kernel of the
+    // convolution only the epilogue warps wait: see there.)
+    if (!(kConv && p.after_zero_fill)) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -806,7 +810,7 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // used only behind the zero-fill kernel
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // added for the launch itself, not for the occupancy query
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
@@ -874,7 +878,7 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     }
     if (!tmA) return cudaSuccess;   // planning only
     cfg.gridDim = dim3(2 * clusters);
-    cfg.numAttrs = (MODE == 2 || MODE == 4) && p.after_zero_fill ? 2 : 1;
+    cfg.numAttrs = 2;   // cluster shape + programmatic stream serialization
     return cudaLaunchKernelEx(&cfg, kernel, *tmA, *tmB, q);
 }
 

@@ -98,6 +98,9 @@ mlp_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     ptx::cluster_sync();   // the peer's barriers exist before anything is signalled on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
+    // launched with programmatic stream serialization: nothing below touches global memory before the kernel in
+    // front has completed; everything above overlapped its tail
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // k-blocks of layer l: over K of x for the first layer, over the previous layer's width afterwards
     auto num_kb = [&](int l) { return l == 0 ? (p.K0 + kBK - 1) / kBK : (p.width[l - 1] + kBK - 1) / kBK; };
@@ -290,11 +293,13 @@ cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUte
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // added for the launch itself, not for the occupancy query
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(kMlpThreads);
     cfg.dynamicSmemBytes = kMlpSmem;
     cfg.stream = stream;
@@ -315,6 +320,7 @@ cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUte
     const CUtensorMap& w2 = tmW[p.layers > 2 ? 2 : 0];
     const CUtensorMap& w3 = tmW[p.layers > 3 ? 3 : 0];
     *launches += 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, mlp_tc_kernel, tmX, tmW[0], w1, w2, w3, p);
 }
 
