@@ -76,26 +76,34 @@ __device__ __forceinline__ float load_scalar(const void* p, int dt, long long i)
 }
 
 // kN consecutive elements starting at element i of a tensor of type dt; elements from `valid` on are left at 0.
-// Eight whole elements on a 16-byte boundary are read with one (16-bit types) or two (fp32) vector loads.
+// Whole groups of eight elements on a 16-byte boundary are read with one (16-bit types) or two (fp32) vector
+// loads per group (kN = 8 or 16).
 template <int kN>
 __device__ __forceinline__ void load_run(const void* p, int dt, long long i, long long valid, float (&out)[kN]) {
-    if (kN == 8 && valid >= 8) {
+    if (kN % 8 == 0 && valid >= kN) {
         if (dt != FC_F32) {
             const unsigned short* q = (const unsigned short*) p + i;
             if ((reinterpret_cast<uintptr_t>(q) & 15) == 0) {
-                const uint4 w = __ldg(reinterpret_cast<const uint4*>(q));
                 const bool h = dt == FC_F16;
-                const float2 a = unpack16x2(w.x, h), b = unpack16x2(w.y, h), c = unpack16x2(w.z, h), d = unpack16x2(w.w, h);
-                out[0] = a.x; out[1] = a.y; out[2 % kN] = b.x; out[3 % kN] = b.y;
-                out[4 % kN] = c.x; out[5 % kN] = c.y; out[6 % kN] = d.x; out[7 % kN] = d.y;
+#pragma unroll
+                for (int g = 0; g < kN / 8; ++g) {
+                    const uint4 w = __ldg(reinterpret_cast<const uint4*>(q) + g);
+                    const float2 a = unpack16x2(w.x, h), b = unpack16x2(w.y, h), c = unpack16x2(w.z, h), d = unpack16x2(w.w, h);
+                    const int o = 8 * g;
+                    out[(o + 0) % kN] = a.x; out[(o + 1) % kN] = a.y; out[(o + 2) % kN] = b.x; out[(o + 3) % kN] = b.y;
+                    out[(o + 4) % kN] = c.x; out[(o + 5) % kN] = c.y; out[(o + 6) % kN] = d.x; out[(o + 7) % kN] = d.y;
+                }
                 return;
             }
         } else {
             const float* q = (const float*) p + i;
             if ((reinterpret_cast<uintptr_t>(q) & 15) == 0) {
-                const float4 a = __ldg(reinterpret_cast<const float4*>(q)), b = __ldg(reinterpret_cast<const float4*>(q) + 1);
-                out[0] = a.x; out[1 % kN] = a.y; out[2 % kN] = a.z; out[3 % kN] = a.w;
-                out[4 % kN] = b.x; out[5 % kN] = b.y; out[6 % kN] = b.z; out[7 % kN] = b.w;
+#pragma unroll
+                for (int g = 0; g < kN / 4; ++g) {
+                    const float4 a = __ldg(reinterpret_cast<const float4*>(q) + g);
+                    const int o = 4 * g;
+                    out[(o + 0) % kN] = a.x; out[(o + 1) % kN] = a.y; out[(o + 2) % kN] = a.z; out[(o + 3) % kN] = a.w;
+                }
                 return;
             }
         }

@@ -99,9 +99,11 @@ __device__ __forceinline__ void fused_ops16(float (&v)[16], const FusedOps& f, c
 #pragma unroll
     for (int j = 0; j < 8; ++j) { v[2 * j] = w[j].x; v[2 * j + 1] = w[j].y; }
     if (f.res) {
+        // this row's 16 columns of the residual: two 16-byte loads (16-bit storage) where the row allows it
+        float t[16];
+        load_run<16>(f.res_ptr, f.res_dt, m * ld + n0, n_limit - n0, t);
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-            if (n0 + j < n_limit) v[j] += load_scalar(f.res_ptr, f.res_dt, m * ld + n0 + j);
+        for (int j = 0; j < 16; ++j) v[j] += t[j];
     }
 }
 
@@ -155,11 +157,13 @@ __device__ __forceinline__ void apply_ops16(float (&v)[16], const DevOps& ops, c
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = fminf(fmaxf(v[j], op.f0), op.f1);
                 break;
-            case FC_OP_ADD_TENSOR:
+            case FC_OP_ADD_TENSOR: {
+                float t[16];
+                load_run<16>(op.p0, op.dt0, m * ld + n0, n_limit - n0, t);
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (n0 + j < n_limit) v[j] += load_scalar(op.p0, op.dt0, m * ld + n0 + j);
+                for (int j = 0; j < 16; ++j) v[j] += t[j];
                 break;
+            }
             default:
                 break;
         }

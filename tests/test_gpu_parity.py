@@ -302,6 +302,17 @@ def test_gemm_tc_op_lists_fused_and_interpreted(fc, orc):
             run_and_check(fc, orc, replace(base, ops=ops, out_dtype=out_dtype, input_recipe=rec), 6, tag=f" ops={[o[0] for o in ops]}")
 
 
+@pytest.mark.parametrize("N,res_dt", [(512, "bf16"), (520, "bf16"), (264, "f32"), (250, "bf16"), (250, "f32")])
+def test_gemm_residual_rows_aligned_and_not(fc, orc, N, res_dt):
+    """x + linear(x)-shaped chains: the residual row is read 16 columns at a time with 16-byte loads where its
+    address allows (N a multiple of 8 for 16-bit storage, of 4 for fp32) and element by element otherwise
+    (N = 250: odd rows start off a 16-byte boundary); the last, ragged chunk always goes element by element."""
+    base = wl.gemm_bias_gelu_scale_clamp(300, N, 136, "var")
+    rec = base.input_recipe + (("res", res_dt, (300, N), "normal", 0.0, 1.0),)
+    for ops in [(("bias_n", 2), ("add_tensor", 3)), (("add_tensor", 3), ("relu",))]:
+        run_and_check(fc, orc, replace(base, ops=ops, input_recipe=rec), 3)
+
+
 def test_c3_full_size_sampled_rows(fc, orc):
     ch = wl.CONFIGS["C3"]()
     ins = wl.make_inputs(ch, 0)
