@@ -464,7 +464,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
                     {
                         const int n0 = n_half + c * 16;
-                        if (m < p.M && n0 < p.N) {
+                        if (!out_vec && n0 < p.N) {
+                            // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
+                            float v[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
+                            if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                        } else if (m < p.M && n0 < p.N) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
@@ -477,7 +484,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
                     {
                         const int n0 = n_half + (c + 1) * 16;
-                        if (m < p.M && n0 < p.N) {
+                        if (!out_vec && n0 < p.N) {
+                            // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
+                            float v[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
+                            if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
+                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                        } else if (m < p.M && n0 < p.N) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
@@ -499,12 +513,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_ld_32x16_async(tacc + c * 16, r);
                     ptx::tmem_wait_ld(r);
                     const int n0 = n_half + c * 16;
+                    if (p.out && !out_vec && n0 < p.N) {
+                        // rows off 16-byte boundaries: every lane takes part in the store of the warp's block
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                        if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                    }
                     if (m < p.M && n0 < p.N) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
                         apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                        if (p.out) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                        if (p.out && out_vec) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
                         if (rk == FC_RED_ROW_LOGSUMEXP || rk == FC_RED_ROW_MAX) {
                             float cm = -CUDART_INF_F;
 #pragma unroll
@@ -663,7 +685,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const float2 fac2 = make_float2(fac, fac);
                 tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
-                    if (m < p.M && n0 < p.N && store) {
+                    if (!out_vec && n0 < p.N && __all_sync(0xffffffffu, store)) {
+                        // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float2 t = __fmul2_rn(make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1])), fac2);
+                            v[2 * j] = t.x;
+                            v[2 * j + 1] = t.y;
+                        }
+                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                    } else if (m < p.M && n0 < p.N && store && out_vec) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {

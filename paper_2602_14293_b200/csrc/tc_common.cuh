@@ -205,4 +205,29 @@ __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, cons
     }
 }
 
+// Rows that do not start on 16-byte boundaries (N not a multiple of 8 for 16-bit outputs, of 4 for fp32): a thread
+// storing its own row element by element makes every store instruction touch 32 sectors.  Here the warp's 32 x 16
+// values go through shared memory (`stage`: 32 x 17 floats of this warp) and are written two rows per
+// instruction, 16 consecutive elements each.  Every lane of the warp must call (`row_ok`: this lane's row exists).
+__device__ __forceinline__ void store16_rows(void* out, int out_dt, float* stage, const float (&v)[16], long long m_lane0,
+                                             long long M, long long n0, long long N, int lane) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) stage[lane * 17 + j] = v[j];
+    __syncwarp();
+    const int c = lane & 15;
+    if (n0 + c < N) {
+#pragma unroll 4
+        for (int it = 0; it < 16; ++it) {
+            const int r = 2 * it + (lane >> 4);
+            const long long row = m_lane0 + r;
+            if (row < M) {
+                const float x = stage[r * 17 + c];
+                if (out_dt == FC_F32) ((float*) out)[row * N + n0 + c] = x;
+                else ((unsigned short*) out)[row * N + n0 + c] = (unsigned short) (pack16x2(x, 0.0f, out_dt == FC_F16) & 0xffffu);
+            }
+        }
+    }
+    __syncwarp();
+}
+
 }  // namespace fc

@@ -313,6 +313,17 @@ def test_gemm_residual_rows_aligned_and_not(fc, orc, N, res_dt):
         run_and_check(fc, orc, replace(base, ops=ops, input_recipe=rec), 3)
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 250, 136), (129, 517, 72), (40, 33, 64), (513, 1001, 264)])
+@pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
+def test_gemm_output_rows_off_16_byte_boundaries(fc, orc, M, N, K, out_dtype):
+    """N that is no multiple of 8 (a vocabulary of 50257, say): output rows start anywhere, so the warp stores
+    its block of rows together, 16 consecutive elements of two rows per instruction.  Plain store, softmax
+    probabilities, and a stored main output beside a row reduction."""
+    run_and_check(fc, orc, replace(wl.gemm_bias_gelu_scale_clamp(M, N, K, "var"), out_dtype=out_dtype), 2)
+    run_and_check(fc, orc, replace(wl.gemm_softmax(M, N, K, "var"), out_dtype=out_dtype), 2)
+    run_and_check(fc, orc, replace(wl.gemm_bias_scale_lse(M, N, K, store_main=True), out_dtype=out_dtype), 2)
+
+
 def test_c3_full_size_sampled_rows(fc, orc):
     ch = wl.CONFIGS["C3"]()
     ins = wl.make_inputs(ch, 0)
