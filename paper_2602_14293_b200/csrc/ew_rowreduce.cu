@@ -211,13 +211,64 @@ constexpr int kPreNone = 0, kPreBias = 1, kPreAffine = 2;
 constexpr int kActNone = 0, kActRelu = 1, kActGeluPrecise = 2, kActGeluFast = 3;
 constexpr int kActPost = 4;   // flag on top of the activation: a scale and a clamp follow it (before the residual)
 constexpr int kGroup = 4;   // chunks in flight per lane and tensor
+constexpr int kMaxWarpRow = 24576;   // longest row of the warp-per-row kernel (its vectors' fp32 copies must fit shared memory)
+constexpr int kLongRow = 10240;      // from here on a CTA per row (measured: the warp-per-row kernel wins at 8192, loses at 12280)
 
 // One chunk (8 columns starting at column 8*c) of one row: ops in packed fp32x2, one 16-byte store,
 // and the chunk's contribution to the running (max, sum) of the row (log2 domain).
 // The values of one chunk (8 columns starting at column 8*c) after the ops, as four fp32 pairs.
+// The per-column operands of chunk c (gamma or bias in a, beta in b) from the fp32 copies in shared memory ...
+template <int PRE, bool MAY_BE_CONST>
+__device__ __forceinline__ void vec_from_smem(const float* svec, int N, int c, float2 (&a)[4], float2 (&b)[4], float const_gamma) {
+    if (MAY_BE_CONST && PRE == kPreAffine && svec == nullptr) {
+        // a lone SCALE folded into the affine step: gamma is that factor, beta 0, nothing in shared memory
+        a[0] = a[1] = a[2] = a[3] = make_float2(const_gamma, const_gamma);
+        b[0] = b[1] = b[2] = b[3] = make_float2(0.0f, 0.0f);
+    } else if (PRE != kPreNone) {
+        // shared-memory layout: the first and the second four columns of every chunk in separate arrays, so
+        // that consecutive lanes (consecutive chunks) read consecutive float4s: no bank conflicts
+        const int chunks = N >> 3;
+        const float4* sv = reinterpret_cast<const float4*>(svec);
+        const float4 a0 = sv[c];
+        const float4 a1 = sv[chunks + c];
+        a[0] = make_float2(a0.x, a0.y); a[1] = make_float2(a0.z, a0.w); a[2] = make_float2(a1.x, a1.y); a[3] = make_float2(a1.z, a1.w);
+        if (PRE == kPreAffine) {
+            const float4 b0 = sv[2 * chunks + c];
+            const float4 b1 = sv[3 * chunks + c];
+            b[0] = make_float2(b0.x, b0.y); b[1] = make_float2(b0.z, b0.w); b[2] = make_float2(b1.x, b1.y); b[3] = make_float2(b1.z, b1.w);
+        }
+    }
+}
+// ... or straight from the 16-bit vectors in global memory (rows too long for copies in shared memory; the
+// vectors are shared by all rows and stay in L1 / L2).  A folded SCALE multiplies gamma here.
+template <int PRE>
+__device__ __forceinline__ void vec_from_global(const EwFastParams& p, int c, float2 (&a)[4], float2 (&b)[4]) {
+    if (PRE != kPreNone) {
+        const float s = PRE == kPreAffine ? p.pre_scale : 1.0f;
+        if (p.vec0) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(p.vec0) + c);
+            const bool h = p.vec0_dt == FC_F16;
+            const float2 ss = make_float2(s, s);
+            a[0] = __fmul2_rn(unpack16x2(q.x, h), ss); a[1] = __fmul2_rn(unpack16x2(q.y, h), ss);
+            a[2] = __fmul2_rn(unpack16x2(q.z, h), ss); a[3] = __fmul2_rn(unpack16x2(q.w, h), ss);
+        } else {
+            a[0] = a[1] = a[2] = a[3] = make_float2(s, s);
+        }
+        if (PRE == kPreAffine) {
+            if (p.vec1) {
+                const uint4 q = __ldg(reinterpret_cast<const uint4*>(p.vec1) + c);
+                const bool h = p.vec1_dt == FC_F16;
+                b[0] = unpack16x2(q.x, h); b[1] = unpack16x2(q.y, h); b[2] = unpack16x2(q.z, h); b[3] = unpack16x2(q.w, h);
+            } else {
+                b[0] = b[1] = b[2] = b[3] = make_float2(0.0f, 0.0f);
+            }
+        }
+    }
+}
+
 template <int PRE, int ACT_, bool RES_>
-__device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const float* svec, int N, int c, bool f16, float2 (&v)[4],
-                                          const EwFastParams& prm) {
+__device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const float2 (&a)[4], const float2 (&b)[4], bool f16,
+                                          float2 (&v)[4], const EwFastParams& prm) {
     constexpr int ACT = ACT_ & 3;
     constexpr bool kPost = (ACT_ & kActPost) != 0;
     constexpr bool RES = RES_ && !kPost;   // with post ops the residual is added behind them, not inside the activation
@@ -225,24 +276,12 @@ __device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const 
     v[1] = unpack16x2(xq.y, f16);
     v[2] = unpack16x2(xq.z, f16);
     v[3] = unpack16x2(xq.w, f16);
-    if (PRE != kPreNone) {
-        // shared-memory layout: the first and the second four columns of every chunk in separate arrays, so
-        // that consecutive lanes (consecutive chunks) read consecutive float4s: no bank conflicts
-        const int chunks = N >> 3;
-        const float4* sv = reinterpret_cast<const float4*>(svec);
-        const float4 a0 = sv[c];
-        const float4 a1 = sv[chunks + c];
-        const float2 a[4] = {make_float2(a0.x, a0.y), make_float2(a0.z, a0.w), make_float2(a1.x, a1.y), make_float2(a1.z, a1.w)};
-        if (PRE == kPreAffine) {
-            const float4 b0 = sv[2 * chunks + c];
-            const float4 b1 = sv[3 * chunks + c];
-            const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
+    if (PRE == kPreAffine) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = __ffma2_rn(v[j], a[j], b[j]);
-        } else {
+        for (int j = 0; j < 4; ++j) v[j] = __ffma2_rn(v[j], a[j], b[j]);
+    } else if (PRE == kPreBias) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = __fadd2_rn(v[j], a[j]);
-        }
+        for (int j = 0; j < 4; ++j) v[j] = __fadd2_rn(v[j], a[j]);
     }
     float2 r[4];
     if (RES_) {
@@ -284,12 +323,15 @@ __device__ __forceinline__ void ew_values(const uint4 xq, const uint4 rq, const 
     }
 }
 
-template <int PRE, int ACT, bool RES, bool LSE, bool STORE>
+// VEC: 0 vectors from shared memory, 1 from global memory, 2 from shared memory unless a lone SCALE made them
+// constants (checked at run time; only the softmax instantiations pay for the check)
+template <int PRE, int ACT, bool RES, bool LSE, bool STORE, int VEC = 0>
 __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const float* svec, int N, int c, uint4* yr,
                                          int red_kind, bool f16, float& run_m, float& run_s, uint4* stash_e, float* stash_m,
                                          const EwFastParams& prm) {
-    float2 v[4];
-    ew_values<PRE, ACT, RES>(xq, rq, svec, N, c, f16, v, prm);
+    float2 v[4], a[4], b[4];
+    if (VEC == 1) vec_from_global<PRE>(prm, c, a, b); else vec_from_smem<PRE, VEC == 2>(svec, N, c, a, b, prm.pre_scale);
+    ew_values<PRE, ACT, RES>(xq, rq, a, b, f16, v, prm);
     if (STORE) {
         uint4 q;
         q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
@@ -343,7 +385,9 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
     // wait here, before their first access to global memory, until it has completed and its writes are visible.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int N = p.N;
-    if (PRE != kPreNone) {
+    const bool const_vec = SOFTMAX && PRE == kPreAffine && !p.vec0 && !p.vec1;   // a lone SCALE: no vectors to copy
+    const float* svec_or_null = const_vec ? nullptr : svec;
+    if (PRE != kPreNone && !const_vec) {
         // Every CTA converts the vectors once.  This prologue is a fixed cost of the launch (it measured 8 us
         // with one scalar load per column and thread): 16-bit vectors that are 16-byte aligned are read
         // eight columns per load, all loads of a thread issued before the first conversion.
@@ -400,7 +444,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
     uint4* stash_e = nullptr;
     float* stash_m = nullptr;
     if (SOFTMAX && p.stash) {
-        float* base = svec + (PRE == kPreNone ? 0 : (PRE == kPreAffine ? 2 : 1) * N);
+        float* base = svec + ((PRE == kPreNone || const_vec) ? 0 : (PRE == kPreAffine ? 2 : 1) * N);
         stash_e = reinterpret_cast<uint4*>(base) + (size_t) warp * chunks;
         stash_m = base + (size_t) kWarps * chunks * 4 + (size_t) warp * chunks;
     }
@@ -426,7 +470,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
             for (int g = 0; g < kInFlight; ++g) {
                 const int c = c0 + 32 * g;
                 if (c < chunks)
-                    ew_chunk<PRE, ACT, RES, LSE, STORE>(xv[g], rv[g], svec, N, c, yr, SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind, p.is_f16 != 0, run_m, run_s,
+                    ew_chunk<PRE, ACT, RES, LSE, STORE, SOFTMAX ? 2 : 0>(xv[g], rv[g], svec_or_null, N, c, yr, SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind, p.is_f16 != 0, run_m, run_s,
                                                         SOFTMAX ? stash_e : nullptr, stash_m, p);
             }
         }
@@ -489,7 +533,9 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                             const int c = c0 + 32 * g;
                             if (c < chunks) {
                                 float2 v[4];
-                                ew_values<PRE, ACT, RES>(xv[g], rv[g], svec, N, c, p.is_f16 != 0, v, p);
+                                float2 va[4], vb[4];
+                                vec_from_smem<PRE, true>(svec_or_null, N, c, va, vb, p.pre_scale);
+                                ew_values<PRE, ACT, RES>(xv[g], rv[g], va, vb, p.is_f16 != 0, v, p);
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
                                     const float2 e = __ffma2_rn(v[j], l2e, mnm);
@@ -508,13 +554,108 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
     }
 }
 
+// ------------------------------------------------------------------------------------ long rows
+// Rows of many thousands of columns (a vocabulary): a warp per row would walk them 32 chunks at a time and the
+// fp32 copies of the per-column vectors would not fit shared memory.  Here a whole CTA owns a row: thread t takes
+// chunks t, t + 256, ...; the vectors are read from their 16-bit originals (L1 / L2 resident); the row's
+// (max, sum) pairs are merged by warp shuffles and one shared-memory exchange.  Row softmax takes its second
+// pass over the row's inputs from L2 and computes the values again.
+template <int PRE, int ACT, bool RES, bool LSE, bool STORE, bool SOFTMAX>
+__global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(const EwFastParams p) {
+    __shared__ float2 red[kWarps];
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // programmatic launch: see ew_rows_kernel
+    const int N = p.N, chunks = N >> 3;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool f16 = p.is_f16 != 0;
+    const int kind = SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind;
+    for (long long row = blockIdx.x; row < p.M; row += gridDim.x) {
+        const uint4* xr = p.x + row * chunks;
+        const uint4* rr = RES ? p.res + row * chunks : nullptr;
+        uint4* yr = STORE ? p.y + row * chunks : nullptr;
+        float run_m = -CUDART_INF_F, run_s = 0.0f;
+        for (int c0 = threadIdx.x; c0 < chunks; c0 += kThreads * kGroup) {
+            uint4 xv[kGroup], rv[kGroup];
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) {
+                const int c = c0 + kThreads * g;
+                if (c < chunks) {
+                    xv[g] = ld_stream(xr + c);
+                    if (RES) rv[g] = ld_stream(rr + c);
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) {
+                const int c = c0 + kThreads * g;
+                if (c < chunks) ew_chunk<PRE, ACT, RES, LSE, STORE, 1>(xv[g], rv[g], nullptr, N, c, yr, kind, f16, run_m, run_s, nullptr, nullptr, p);
+            }
+        }
+        if (LSE) {
+            const bool plain = kind >= FC_RED_ROW_SUM;   // running sum and maximum instead of a logsumexp pair
+            auto merge = [plain](float& am, float& as, float bm, float bs) {
+                if (plain) { as += bs; am = fmaxf(am, bm); return; }
+                const float nm = fmaxf(am, bm);
+                const float sa = am == -CUDART_INF_F ? 0.0f : as * exp2_fast(am - nm);
+                const float sb = bm == -CUDART_INF_F ? 0.0f : bs * exp2_fast(bm - nm);
+                as = sa + sb;
+                am = nm;
+            };
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) merge(run_m, run_s, __shfl_xor_sync(0xffffffffu, run_m, o), __shfl_xor_sync(0xffffffffu, run_s, o));
+            __syncthreads();   // the previous row's readers are done with `red`
+            if (lane == 0) red[warp] = make_float2(run_m, run_s);
+            __syncthreads();
+            run_m = red[0].x; run_s = red[0].y;
+#pragma unroll
+            for (int w = 1; w < kWarps; ++w) merge(run_m, run_s, red[w].x, red[w].y);
+            if constexpr (SOFTMAX) {
+                float inv;
+                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(run_s));
+                const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-run_m, -run_m), inv2 = make_float2(inv, inv);
+                uint4* pr = p.y + row * chunks;
+                for (int c0 = threadIdx.x; c0 < chunks; c0 += kThreads * kGroup) {
+                    uint4 xv[kGroup], rv[kGroup];
+#pragma unroll
+                    for (int g = 0; g < kGroup; ++g) {
+                        const int c = c0 + kThreads * g;
+                        if (c < chunks) {
+                            xv[g] = __ldcg(xr + c);
+                            if (RES) rv[g] = __ldcg(rr + c);
+                        }
+                    }
+#pragma unroll
+                    for (int g = 0; g < kGroup; ++g) {
+                        const int c = c0 + kThreads * g;
+                        if (c < chunks) {
+                            float2 v[4], va[4], vb[4];
+                            vec_from_global<PRE>(p, c, va, vb);
+                            ew_values<PRE, ACT, RES>(xv[g], rv[g], va, vb, f16, v, p);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 e = __ffma2_rn(v[j], l2e, mnm);
+                                v[j] = __fmul2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), inv2);
+                            }
+                            uint4 q;
+                            q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
+                            q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
+                            st_stream(pr + c, q);
+                        }
+                    }
+                }
+            } else if (threadIdx.x == 0) {
+                p.lse[row] = kind == FC_RED_ROW_LOGSUMEXP ? (run_m + log2f(run_s)) * kLn2
+                           : kind == FC_RED_ROW_MAX ? run_m : (kind == FC_RED_ROW_MEAN ? run_s / (float) N : run_s);
+            }
+        }
+    }
+}
+
 }  // namespace
 
 // Recognise [scale]? -> [bias | affine]? -> [relu | gelu]? -> [scale]? -> [clamp]? -> [add tensor]? and fill the
 // fast-path parameters.
 static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, bool* res) {
     if (p.x_dt == FC_F32 || (p.y && p.y_dt != p.x_dt)) return false;
-    if (p.N % 8 != 0 || p.N > 24576 || p.M >= 0x7fffffffLL) return false;
+    if (p.N % 8 != 0 || p.N >= 0x40000000LL || p.M >= 0x7fffffffLL) return false;
     if ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y)) & 15) return false;
     int i = 0;
     *pre = kPreNone; *act = kActNone; *res = false;
@@ -555,6 +696,12 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
         ++i;
     }
     if (i != p.ops.n) return false;
+    if (p.N > kMaxWarpRow) {
+        // only the CTA-per-row kernel takes rows this long: a row reduction, no post ops, 16-bit aligned vectors
+        const bool vec_ok = (!f->vec0 || (f->vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(f->vec0) & 15) == 0)) &&
+                            (!f->vec1 || (f->vec1_dt != FC_F32 && (reinterpret_cast<uintptr_t>(f->vec1) & 15) == 0));
+        if (p.reduce == FC_RED_NONE || (*act & kActPost) || !vec_ok) return false;
+    }
     f->x = (const uint4*) p.x; f->y = (uint4*) p.y; f->lse = p.red; f->M = p.M; f->N = (int) p.N;
     f->red_kind = p.reduce;
     f->is_f16 = p.x_dt == FC_F16;
@@ -564,13 +711,37 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
 template <int PRE, int ACT, bool RES>
 static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, int num_sms, cudaStream_t stream) {
     EwFastParams f = f_in;
-    size_t smem = PRE == kPreNone ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
+    const bool const_vec = f.red_kind == FC_RED_ROW_SOFTMAX && PRE == kPreAffine && !f.vec0 && !f.vec1;
+    size_t smem = (PRE == kPreNone || const_vec) ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
     f.stash = 0;
     const size_t stash_bytes = (size_t) kWarps * (f.N / 8) * (16 + 4);   // per chunk: eight 16-bit values and a maximum
     if (f.red_kind == FC_RED_ROW_SOFTMAX && smem + stash_bytes <= 200 * 1024) {
         f.stash = 1;
         smem += stash_bytes;
     }
+    // Rows from 12288 columns on (lists without the post ops, 16-bit vectors on 16-byte boundaries) go to the
+    // kernel that gives a CTA to a row.
+    if constexpr ((ACT & kActPost) == 0) {
+        const bool vec_ok = (!f.vec0 || (f.vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(f.vec0) & 15) == 0)) &&
+                            (!f.vec1 || (f.vec1_dt != FC_F32 && (reinterpret_cast<uintptr_t>(f.vec1) & 15) == 0));
+        if (lse && f.N >= kLongRow && vec_ok) {
+            cudaLaunchConfig_t cfg = {};
+            const bool sm = f.red_kind == FC_RED_ROW_SOFTMAX;
+            const long long want = (long long) num_sms * (sm ? 2 : 4);
+            cfg.gridDim = dim3((unsigned) (f.M < want ? f.M : want));
+            cfg.blockDim = dim3(kThreads);
+            cfg.stream = stream;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr.val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            if (sm) return cudaLaunchKernelEx(&cfg, ew_longrow_kernel<PRE, ACT, RES, true, false, true>, f);
+            if (store) return cudaLaunchKernelEx(&cfg, ew_longrow_kernel<PRE, ACT, RES, true, true, false>, f);
+            return cudaLaunchKernelEx(&cfg, ew_longrow_kernel<PRE, ACT, RES, true, false, false>, f);
+        }
+    }
+    if (f.N > kMaxWarpRow) return cudaErrorInvalidValue;   // not reached: match_fast sends such chains elsewhere
     long long ctas = (f.M + kWarps - 1) / kWarps;
     int per_sm = smem > 0 ? (int) ((227 * 1024) / (smem + 1024)) : 4;   // 228 KB per SM, 1 KB of it reserved per CTA
     per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);

@@ -177,6 +177,30 @@ def test_elementwise_scale_and_clamp_behind_the_activation(fc, orc, ops, red, M,
     run_and_check(fc, orc, replace(base, ops=ops, reduce=red, store_main=True), 13)
 
 
+@pytest.mark.parametrize("M,N", [(5, 12288), (3, 50264), (9, 24584), (2, 100000)])
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+def test_elementwise_long_rows_take_a_cta_per_row(fc, orc, M, N, dt):
+    """Rows from 12288 columns on (a vocabulary): a CTA per row, vectors read from their 16-bit originals.  Row
+    logsumexp with and without the main output, row softmax (second pass from L2), sum / max / mean, and a
+    -inf mask over most of a row."""
+    base = wl.affine_gelu_residual_lse(M, N)
+    sm = wl.scale_add_softmax(M, N)
+    if dt == "f16":
+        base, sm = _as_f16(base), _as_f16(sm)
+    run_and_check(fc, orc, base, 3)
+    run_and_check(fc, orc, replace(base, store_main=False, ops=(("bias_n", 2), ("relu",))), 3)
+    # (probabilities below 6e-5 are fp16 subnormals: their storage rounding alone exceeds the fp16 tolerance)
+    if dt == "bf16" or N <= 12288:
+        run_and_check(fc, orc, sm, 3)
+    for red in ("row_sum", "row_max", "row_mean"):
+        run_and_check(fc, orc, replace(base, reduce=red, ops=(("scale", 0.5), ("bias_n", 1))), 3)
+    ins = wl.make_inputs(sm, 5)
+    keep = np.arange(N)[None, :] % 1000 < (np.arange(M)[:, None] + 1)
+    ins[1] = rng.store(np.where(keep, 0.0, -np.inf).astype(np.float32), dt)
+    outs, _, _ = run_and_check(fc, orc, sm, ins=ins)
+    assert (util.to_f64(outs[0])[~keep] == 0.0).all()
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
