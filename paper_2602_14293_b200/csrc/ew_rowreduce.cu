@@ -212,6 +212,7 @@ constexpr int kActNone = 0, kActRelu = 1, kActGeluPrecise = 2, kActGeluFast = 3;
 constexpr int kActPost = 4;   // flag on top of the activation: a scale and a clamp follow it (before the residual)
 constexpr int kGroup = 4;   // chunks in flight per lane and tensor
 constexpr int kMaxWarpRow = 24576;   // longest row of the warp-per-row kernel (its vectors' fp32 copies must fit shared memory)
+constexpr int kNarrowRow = 256;      // up to here (with a row reduction) a lane per chunk, several rows per warp
 constexpr int kLongRow = 10240;      // from here on a CTA per row (measured: the warp-per-row kernel wins at 8192, loses at 12280)
 
 // One chunk (8 columns starting at column 8*c) of one row: ops in packed fp32x2, one 16-byte store,
@@ -554,6 +555,115 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
     }
 }
 
+// ------------------------------------------------------------------------------------ narrow rows
+// Rows of at most 256 columns (at most 32 chunks) with a row reduction: a warp per row would leave most lanes
+// idle (64 columns: 8 of 32).  Here a lane owns one chunk and a warp covers 32 / cpr rows at a time, cpr = chunks
+// per row rounded up to a power of two; the row's (max, sum) pair is merged by xor shuffles inside its group of
+// cpr lanes.  The whole row sits in registers across the warp, so row softmax needs no second pass.  kGroup row
+// groups are in flight per warp.  Which reduction, and whether the main output is stored, is decided at run time:
+// this kernel is instantiated per op pattern only.
+template <int PRE, int ACT, bool RES>
+__global__ void __launch_bounds__(kThreads, 4) ew_narrow_kernel(const EwFastParams p, int cpr_log2) {
+    extern __shared__ float svec[];
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // programmatic launch: see ew_rows_kernel
+    const int N = p.N, chunks = N >> 3;
+    if (PRE != kPreNone) {
+        for (int i = threadIdx.x; i < N; i += kThreads) {
+            const int pos = ((((i >> 2) & 1) * chunks) + (i >> 3)) * 4 + (i & 3);   // de-interleaved, as in ew_rows_kernel
+            svec[pos] = (p.vec0 ? load_scalar(p.vec0, p.vec0_dt, i) : 1.0f) * (PRE == kPreAffine ? p.pre_scale : 1.0f);
+            if (PRE == kPreAffine) svec[N + pos] = p.vec1 ? load_scalar(p.vec1, p.vec1_dt, i) : 0.0f;
+        }
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int cpr = 1 << cpr_log2, rows_per_warp = 32 >> cpr_log2;
+    const int c = lane & (cpr - 1), sub = lane >> cpr_log2;
+    const bool f16 = p.is_f16 != 0;
+    const int kind = p.red_kind;
+    const bool softmax = kind == FC_RED_ROW_SOFTMAX, plain = kind >= FC_RED_ROW_SUM;
+    const bool store = p.y != nullptr && !softmax;
+    const long long step = (long long) gridDim.x * kWarps * rows_per_warp * kGroup;
+    for (long long base = ((long long) blockIdx.x * kWarps + warp) * rows_per_warp * kGroup; base < p.M; base += step) {
+        uint4 xv[kGroup], rv[kGroup];
+#pragma unroll
+        for (int g = 0; g < kGroup; ++g) {
+            const long long row = base + g * rows_per_warp + sub;
+            if (row < p.M && c < chunks) {
+                xv[g] = ld_stream(p.x + row * chunks + c);
+                if (RES) rv[g] = ld_stream(p.res + row * chunks + c);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < kGroup; ++g) {
+            const long long row = base + g * rows_per_warp + sub;
+            const bool valid = row < p.M && c < chunks;
+            float2 v[4], a[4], b[4];
+            float m = -CUDART_INF_F, sum = 0.0f;
+            if (valid) {
+                vec_from_smem<PRE, false>(svec, N, c, a, b, 1.0f);
+                ew_values<PRE, ACT, RES>(xv[g], rv[g], a, b, f16, v, p);
+                if (store) {
+                    uint4 q;
+                    q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
+                    q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
+                    st_stream(p.y + row * chunks + c, q);
+                }
+                const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)), fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
+                if (plain) {
+                    const float2 t = __fadd2_rn(__fadd2_rn(v[0], v[1]), __fadd2_rn(v[2], v[3]));
+                    m = cm;
+                    sum = t.x + t.y;
+                } else {
+                    // log2 domain; a chunk of -inf only takes its exponents against 0
+                    m = cm * kLog2e;
+                    const float base2 = m == -CUDART_INF_F ? 0.0f : m;
+                    const float2 l2e = make_float2(kLog2e, kLog2e), mb = make_float2(-base2, -base2);
+                    float2 cs = make_float2(0.0f, 0.0f);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 e = __ffma2_rn(v[j], l2e, mb);
+                        cs = __fadd2_rn(cs, make_float2(exp2_fast(e.x), exp2_fast(e.y)));
+                    }
+                    sum = cs.x + cs.y;
+                }
+            }
+            // merge inside the row's group of cpr lanes (lanes without a chunk hold the neutral pair)
+            for (int o = cpr >> 1; o > 0; o >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, sum, o);
+                if (plain) {
+                    sum += os;
+                    m = fmaxf(m, om);
+                } else {
+                    const float nm = fmaxf(m, om);
+                    const float sa = m == -CUDART_INF_F ? 0.0f : sum * exp2_fast(m - nm);
+                    const float sb = om == -CUDART_INF_F ? 0.0f : os * exp2_fast(om - nm);
+                    sum = sa + sb;
+                    m = nm;
+                }
+            }
+            if (softmax) {
+                if (valid) {
+                    float inv;
+                    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(sum));
+                    const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-m, -m), inv2 = make_float2(inv, inv);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 e = __ffma2_rn(v[j], l2e, mnm);
+                        v[j] = __fmul2_rn(make_float2(exp2_fast(e.x), exp2_fast(e.y)), inv2);
+                    }
+                    uint4 q;
+                    q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
+                    q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
+                    st_stream(p.y + row * chunks + c, q);
+                }
+            } else if (c == 0 && row < p.M) {
+                p.lse[row] = kind == FC_RED_ROW_LOGSUMEXP ? (m + log2f(sum)) * kLn2
+                           : kind == FC_RED_ROW_MAX ? m : (kind == FC_RED_ROW_MEAN ? sum / (float) N : sum);
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------ long rows
 // Rows of many thousands of columns (a vocabulary): a warp per row would walk them 32 chunks at a time and the
 // fp32 copies of the per-column vectors would not fit shared memory.  Here a whole CTA owns a row: thread t takes
@@ -684,7 +794,7 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
     // instantiated for the softmax and reduction-only kernels.
     f->post_scale = 1.0f; f->post_lo = -INFINITY; f->post_hi = INFINITY;
     if (i < p.ops.n && (p.ops.op[i].kind == FC_OP_SCALE || p.ops.op[i].kind == FC_OP_CLAMP)) {
-        if (p.reduce == FC_RED_ROW_SOFTMAX || (p.reduce != FC_RED_NONE && !p.y)) return false;
+        if (p.N > kNarrowRow && (p.reduce == FC_RED_ROW_SOFTMAX || (p.reduce != FC_RED_NONE && !p.y))) return false;
         if (p.ops.op[i].kind == FC_OP_SCALE) f->post_scale = p.ops.op[i++].f0;
         if (i < p.ops.n && p.ops.op[i].kind == FC_OP_CLAMP) { f->post_lo = p.ops.op[i].f0; f->post_hi = p.ops.op[i].f1; ++i; }
         *act |= kActPost;
@@ -719,7 +829,26 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
         f.stash = 1;
         smem += stash_bytes;
     }
-    // Rows from 12288 columns on (lists without the post ops, 16-bit vectors on 16-byte boundaries) go to the
+    // Rows of at most 256 columns with a row reduction: a lane per chunk, several rows per warp.
+    if (lse && f.N <= kNarrowRow) {
+        int cpr_log2 = 0;
+        while ((1 << cpr_log2) < f.N / 8) ++cpr_log2;
+        const int rows_per_cta = kWarps * (32 >> cpr_log2) * kGroup;
+        long long want = (f.M + rows_per_cta - 1) / rows_per_cta;
+        if (want > (long long) num_sms * 4) want = (long long) num_sms * 4;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned) want);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = PRE == kPreNone ? 0 : (size_t) f.N * 4 * (PRE == kPreAffine ? 2 : 1);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, ew_narrow_kernel<PRE, ACT, RES>, f, cpr_log2);
+    }
+    // Rows from kLongRow columns on (lists without the post ops, 16-bit vectors on 16-byte boundaries) go to the
     // kernel that gives a CTA to a row.
     if constexpr ((ACT & kActPost) == 0) {
         const bool vec_ok = (!f.vec0 || (f.vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(f.vec0) & 15) == 0)) &&

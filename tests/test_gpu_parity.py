@@ -201,6 +201,30 @@ def test_elementwise_long_rows_take_a_cta_per_row(fc, orc, M, N, dt):
     assert (util.to_f64(outs[0])[~keep] == 0.0).all()
 
 
+@pytest.mark.parametrize("M,N", [(1, 8), (1000, 8), (777, 24), (5, 64), (4001, 64), (333, 72), (129, 128), (77, 200), (1030, 256)])
+@pytest.mark.parametrize("red", ["row_logsumexp", "row_softmax", "row_sum", "row_max", "row_mean"])
+def test_elementwise_narrow_rows_share_a_warp(fc, orc, M, N, red):
+    """Rows of at most 256 columns: a lane per 8-column chunk, 32 / cpr rows per warp (cpr = chunks per row rounded
+    up to a power of two: 24 columns leave a lane of every four idle, 200 columns seven of 32), the row's pair
+    merged inside its lane group.  Every reduction, with and without the main output, bf16 and fp16, ragged
+    row counts, post ops, and -inf masks."""
+    base = wl.affine_gelu_residual_lse(M, N)
+    if red == "row_softmax":
+        run_and_check(fc, orc, replace(base, reduce=red, store_main=False), 4)
+        run_and_check(fc, orc, _as_f16(wl.scale_add_softmax(M, N)), 4)
+        sm = wl.scale_add_softmax(M, N)
+        ins = wl.make_inputs(sm, 6)
+        keep = (np.arange(N)[None, :] + np.arange(M)[:, None]) % 5 != 0
+        keep[:, 0] |= ~keep.any(axis=1)
+        ins[1] = rng.store(np.where(keep, 0.0, -np.inf).astype(np.float32), "bf16")
+        outs, _, _ = run_and_check(fc, orc, sm, ins=ins)
+        assert (util.to_f64(outs[0])[~keep] == 0.0).all()
+    else:
+        run_and_check(fc, orc, replace(base, reduce=red, store_main=True), 4)
+        run_and_check(fc, orc, replace(base, reduce=red, store_main=False, ops=(("bias_n", 2), ("relu",), ("scale", 0.5), ("clamp", -1.0, 1.0))), 4)
+        run_and_check(fc, orc, _as_f16(replace(base, reduce=red, store_main=False, ops=())), 4)
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
