@@ -55,11 +55,14 @@ def _random_ops(r, vec_idx, tensor_idx, max_vecs):
 def _random_chain(r):
     kind = r.choice(["ew", "gemm", "gemm", "conv", "gemm_f32"])
     if kind == "ew":
-        M, N = int(r.integers(1, 70)), int(r.choice([8, 24, 200, 1000, 1024, 4096, 333]))
+        M, N = int(r.integers(1, 70)), int(r.choice([8, 24, 64, 200, 256, 264, 1000, 1024, 4096, 333, 10240, 12296, 30000]))
         dt = str(r.choice(["bf16", "f32", "f16"]))
         rec = (("x", dt, (M, N), "normal", 0.0, 1.0), ("v0", dt, (N,), "normal", 1.0, 0.1), ("v1", "bf16", (N,), "normal", 0.0, 0.1),
                ("t", dt, (M, N), "normal", 0.0, 1.0))
-        red = str(r.choice(["none", "row_logsumexp"]))
+        red = str(r.choice(["none", "row_logsumexp", "row_softmax", "row_sum", "row_max", "row_mean"]))
+        if red == "row_softmax":
+            return wl.Chain("rand_ew", "elementwise", dt, dt, M=M, N=N, ops=_random_ops(r, [1, 2], 3, 8), reduce=red,
+                            store_main=False, input_recipe=rec)
         return wl.Chain("rand_ew", "elementwise", dt, dt, M=M, N=N, ops=_random_ops(r, [1, 2], 3, 8), reduce=red,
                         store_main=bool(red == "none" or r.random() < 0.7), input_recipe=rec)
     if kind == "gemm_f32":
@@ -88,7 +91,7 @@ def _random_chain(r):
     return replace(base, ops=ops, input_recipe=rec)
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(96))
 def test_random_chain(fc, orc, seed):
     r = np.random.default_rng(1000 + seed)
     ch = _random_chain(r)
