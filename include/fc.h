@@ -26,6 +26,10 @@
  * allocates device memory and never synchronises; it enqueues at most two memsets and one to four
  * kernels on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
  *
+ * Launches.  Kernels are launched with programmatic stream serialization and wait, before their first access to
+ * global memory, for everything in front of them in the stream: the order the caller sees is the stream's,
+ * only launch latency overlaps the tail of the work in front.  Calls may be captured into a CUDA graph.
+ *
  * Pointers.  Unless a function says "host", every fc_tensor.ptr is a DEVICE pointer.
  *
  * Layout.  Row-major contiguous only (stride[] must describe exactly that, in elements).
