@@ -24,7 +24,7 @@
  *
  * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
  * allocates device memory and never synchronises; it enqueues at most two memsets and one to four
- * kernels on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
+ * kernels (a GEMM + ROW_SOFTMAX over more than 16384 columns: the GEMM kernel and a rescaling pass) on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
  *
  * Launches.  Kernels are launched with programmatic stream serialization and wait, before their first access to
  * global memory, for everything in front of them in the stream: the order the caller sees is the stream's,

@@ -383,6 +383,7 @@ void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
 }
 
 constexpr int kSoftmaxBN = 256;
+constexpr int kSoftmaxOnePassTiles = 64;   // widest row (in tiles) that the single-pass softmax takes
 
 // arrival counters and departure counters, one of each per 128-row panel
 size_t panel_counter_bytes(long long M) {
@@ -585,7 +586,14 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             CUtensorMap tmA, tmB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
+            // Row softmax over more tiles per panel than the pairs' accumulator buffers can hold until the panel is
+            // complete (two per pair; with a margin: 64 tiles = 16384 columns): no waiting across tiles, and a second,
+            // memory-bound kernel finishes the rows.
+            const int tiles_n = (int) ((spec->N + bn - 1) / bn);
+            p.two_pass = p.mode == 1 && tiles_n > kSoftmaxOnePassTiles;
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
+            if (e == cudaSuccess && p.two_pass)
+                e = launch_softmax_rescale(p.out, p.out_dt, p.stats, spec->M, spec->N, tiles_n, bn, dev->num_sms, stream, &launches);
             break;
         }
         case Plan::TC_MLP: {
@@ -1000,6 +1008,8 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
         }
         scratch = g_static_scratch_ptr[ordinal];
     }
+    if ((spec->N + kSoftmaxBN - 1) / kSoftmaxBN > kSoftmaxOnePassTiles)
+        return fail(FC_ERR_UNSUPPORTED, "rows wider than %d columns take two kernels: use fc_run", kSoftmaxOnePassTiles * kSoftmaxBN);
     cudaStream_t stream = (cudaStream_t) cuda_stream;
     TcParams p;
     memset(&p, 0, sizeof(p));

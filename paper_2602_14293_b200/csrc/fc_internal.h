@@ -81,6 +81,11 @@ size_t collapse_workspace_bytes(long long N, long long K);
 cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,
                                    int* launches);
 
+// Second pass of a wide GEMM + row softmax: per row, merges the tiles' (max, sum) pairs and rescales the stored
+// exponentials of tile j by 2^((max_j - max_row) log2 e) / sum_row, in place.  `bn` = tile width in columns.
+cudaError_t launch_softmax_rescale(void* out, int out_dt, const float2* stats, long long M, long long N, int tiles_n, int bn,
+                                   int num_sms, cudaStream_t stream, int* launches);
+
 // Zeroes `bytes` bytes (a multiple of 4, 4-byte aligned) with a kernel that lets the next kernel in the stream be
 // scheduled at once: the pooled outputs of the convolution are cleared while its first tiles are in the main loop.
 cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches);
@@ -103,6 +108,9 @@ struct TcParams {
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
     int pool;                   // mode 2: 0 global average pool, 1 2x2 max-pool (out pre-zeroed, values >= 0)
+    int two_pass;               // mode 1: rows wider than the tiles the SM pairs can hold at once: no waiting across tiles; every
+                                // tile stores its exponentials against its own maximum and leaves (max, sum) in `stats`,
+                                // launch_softmax_rescale finishes the rows
     int after_zero_fill;        // mode 2: launched programmatically behind the kernel that zeroes `out`; the epilogue warps wait
                                 // for that kernel before their first update of `out`, everything else starts at once
     int a_packed;               // mode 2: 1 = a k-block of A is eight 8-channel chunks, one per filter tap (Cin == 8)

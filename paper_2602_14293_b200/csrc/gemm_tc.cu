@@ -644,10 +644,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const MaxSum a = ms_merge(MaxSum{mx, sm}, MaxSum{o.x, o.y});
                     __stcg(&p.stats[m * tiles_n + nb], make_float2(a.m, a.s));
                 }
+                float tile_m = mx;   // two-pass form: the maximum both halves of this tile rescale to
+                if (p.two_pass) {
+                    if (half == 0 && m < p.M) {
+                        const float2 o = xchg[row];
+                        tile_m = fmaxf(mx, o.x);
+                    }
+                    ptx::bar_sync(1, kEpiThreads);          // the upper half's pair has been read
+                    if (half == 0) xchg[row] = make_float2(tile_m, 0.0f);
+                }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
+                if (p.two_pass && half == 1) tile_m = xchg[row].x;
                 // one thread announces the tile and waits (bounded) for the panel's other tiles
-                if (et == 0) {
+                if (et == 0 && !p.two_pass) {
                     ptx::red_release_gpu_add(&p.counters[mb], 1u);
                     const unsigned long long t0 = ptx::globaltimer();
                     unsigned spins = 0;
@@ -671,7 +681,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::bar_sync(1, kEpiThreads);
                 const bool store = *abort_flag == 0;
                 float row_m = -CUDART_INF_F, row_s = 0.0f;
-                if (m < p.M && store) {
+                if (p.two_pass) {
+                    // no row results yet: the exponentials are stored against the tile's own maximum (in (0, 1]) and
+                    // the rescale kernel behind this one divides by the row's sum
+                    row_m = tile_m;
+                    row_s = 1.0f;
+                } else if (m < p.M && store) {
                     MaxSum a = ms_identity();
                     for (int j = 0; j < tiles_n; ++j) {
                         const float2 st = __ldcg(&p.stats[m * tiles_n + j]);
@@ -681,7 +696,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     row_s = a.s;
                 }
                 // last sweep: p = e * 2^((max_half - max_row) log2 e) / sum_row, one factor per thread
-                const float fac = m < p.M && store ? exp2_fast((mx - row_m) * kLog2e) / row_s : 0.0f;
+                const float fac = m < p.M && store && mx != -CUDART_INF_F ? exp2_fast((mx - row_m) * kLog2e) / row_s : 0.0f;   // (a half row of -inf only holds zeros)
                 const float2 fac2 = make_float2(fac, fac);
                 tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;

@@ -372,6 +372,23 @@ def test_gemm_output_rows_off_16_byte_boundaries(fc, orc, M, N, K, out_dtype):
     run_and_check(fc, orc, replace(wl.gemm_bias_scale_lse(M, N, K, store_main=True), out_dtype=out_dtype), 2)
 
 
+@pytest.mark.parametrize("M,N,K,out_dtype", [(300, 20000, 72, "bf16"), (129, 16640, 136, "bf16"), (260, 16401, 64, "bf16"), (70, 16648, 64, "f32")])
+def test_gemm_softmax_rows_wider_than_one_pass_allows(fc, orc, M, N, K, out_dtype):
+    """More than 64 tiles per row panel: the SM pairs cannot hold a whole panel in tensor memory until its last
+    tile arrives, so every tile stores its exponentials against its own maximum and a second kernel rescales
+    the rows.  With ops and an additive -inf mask in front, aligned and unaligned rows, bf16 and fp32."""
+    base = replace(wl.gemm_softmax(M, N, K, "var"), out_dtype=out_dtype)
+    outs, _, _ = run_and_check(fc, orc, base, 5)
+    np.testing.assert_allclose(util.to_f64(outs[0]).sum(1), 1.0, atol=3e-2 if out_dtype == "bf16" else 1e-4)
+    rec = base.input_recipe + (("mask", "bf16", (M, N), "normal", 0.0, 1.0),)
+    ch = replace(base, ops=(("scale", 0.5), ("add_tensor", 2)), input_recipe=rec)
+    ins = wl.make_inputs(ch, 6)
+    keep = np.arange(N)[None, :] <= (61 * np.arange(M)[:, None] + 3)
+    ins[2] = rng.store(np.where(keep, 0.0, -np.inf).astype(np.float32), "bf16")
+    outs, _, _ = run_and_check(fc, orc, ch, ins=ins)
+    assert (util.to_f64(outs[0])[~keep] == 0.0).all()
+
+
 def test_c3_full_size_sampled_rows(fc, orc):
     ch = wl.CONFIGS["C3"]()
     ins = wl.make_inputs(ch, 0)
