@@ -590,7 +590,12 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             // complete (two per pair; with a margin: 64 tiles = 16384 columns): no waiting across tiles, and a second,
             // memory-bound kernel finishes the rows.
             const int tiles_n = (int) ((spec->N + bn - 1) / bn);
-            p.two_pass = p.mode == 1 && tiles_n > kSoftmaxOnePassTiles;
+            if (p.mode == 1) {
+                // (never more tiles per panel than SM pairs take part, whatever the device offers)
+                TcPlan tp;
+                if ((e = plan_gemm_tc(p, bn, dev->num_sms, &tp)) != cudaSuccess) return cuda_fail(e, "planning");
+                p.two_pass = tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs;
+            }
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             if (e == cudaSuccess && p.two_pass)
                 e = launch_softmax_rescale(p.out, p.out_dt, p.stats, spec->M, spec->N, tiles_n, bn, dev->num_sms, stream, &launches);
