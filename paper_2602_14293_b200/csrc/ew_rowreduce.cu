@@ -192,6 +192,8 @@ struct EwFastParams {
     int red_kind;           // fc_reduce of the row reduction (when the kernel is built with one)
     int is_f16;             // x, residual and y are IEEE half instead of bf16
     float post_scale, post_lo, post_hi;   // ACT with kActPost: v = clamp(v * post_scale, lo, hi) after the activation
+    int ragged;             // long rows whose length is no multiple of 8 (no per-column vectors): rows start anywhere, the
+                            // aligned middle of each row goes in 16-byte chunks, up to 14 edge elements one by one
     int stash;              // row softmax: the row's exponentials wait in shared memory for the second pass
     float pre_scale;        // a SCALE op in front of everything, folded into gamma (PRE is then always affine;
                             // vec0 == null means gamma = 1, vec1 == null means beta = 0)
@@ -674,15 +676,40 @@ template <int PRE, int ACT, bool RES, bool LSE, bool STORE, bool SOFTMAX>
 __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(const EwFastParams p) {
     __shared__ float2 red[kWarps];
     asm volatile("griddepcontrol.wait;" ::: "memory");   // programmatic launch: see ew_rows_kernel
-    const int N = p.N, chunks = N >> 3;
+    const int N = p.N;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool f16 = p.is_f16 != 0;
     const int kind = SOFTMAX ? FC_RED_ROW_LOGSUMEXP : p.red_kind;
+    const bool plain_kind = kind >= FC_RED_ROW_SUM;
+    // one element of the row (ragged rows only): value after the ops, from 2-byte loads
+    auto edge_value = [&](long long e) -> float {
+        uint4 xq = make_uint4((uint32_t) __ldg((const unsigned short*) p.x + e), 0u, 0u, 0u), rq = make_uint4(0u, 0u, 0u, 0u);
+        if (RES) rq.x = (uint32_t) __ldg((const unsigned short*) p.res + e);
+        float2 v[4], a[4], b[4];
+        vec_from_global<PRE>(p, 0, a, b);   // no vectors on this path: constants
+        ew_values<PRE, ACT, RES>(xq, rq, a, b, f16, v, p);
+        return v[0].x;
+    };
     for (long long row = blockIdx.x; row < p.M; row += gridDim.x) {
-        const uint4* xr = p.x + row * chunks;
-        const uint4* rr = RES ? p.res + row * chunks : nullptr;
-        uint4* yr = STORE ? p.y + row * chunks : nullptr;
+        // rows of a ragged tensor start anywhere: `head` elements up to the next 16-byte boundary, then whole chunks,
+        // then `tail` elements (head = tail = 0 when N is a multiple of 8)
+        const long long e0 = row * N;
+        const int head = p.ragged ? (int) ((8 - (e0 & 7)) & 7) : 0;
+        const int chunks = (N - head) >> 3, tail = N - head - 8 * chunks;
+        const uint4* xr = reinterpret_cast<const uint4*>((const unsigned short*) p.x + e0 + head);
+        const uint4* rr = RES ? reinterpret_cast<const uint4*>((const unsigned short*) p.res + e0 + head) : nullptr;
+        uint4* yr = STORE ? reinterpret_cast<uint4*>((unsigned short*) p.y + e0 + head) : nullptr;
         float run_m = -CUDART_INF_F, run_s = 0.0f;
+        const bool edge = (int) threadIdx.x < head + tail;
+        const long long edge_e = e0 + ((int) threadIdx.x < head ? threadIdx.x : head + 8 * chunks + ((int) threadIdx.x - head));
+        if (edge) {
+            const float val = edge_value(edge_e);
+            if (STORE) ((unsigned short*) p.y)[edge_e] = (unsigned short) (pack16x2(val, 0.0f, f16) & 0xffffu);
+            if (LSE) {
+                if (plain_kind) { run_m = val; run_s = val; }
+                else if (val != -CUDART_INF_F) { run_m = val * kLog2e; run_s = 1.0f; }
+            }
+        }
         for (int c0 = threadIdx.x; c0 < chunks; c0 += kThreads * kGroup) {
             uint4 xv[kGroup], rv[kGroup];
 #pragma unroll
@@ -700,7 +727,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(c
             }
         }
         if (LSE) {
-            const bool plain = kind >= FC_RED_ROW_SUM;   // running sum and maximum instead of a logsumexp pair
+            const bool plain = plain_kind;   // running sum and maximum instead of a logsumexp pair
             auto merge = [plain](float& am, float& as, float bm, float bs) {
                 if (plain) { as += bs; am = fmaxf(am, bm); return; }
                 const float nm = fmaxf(am, bm);
@@ -721,7 +748,12 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(c
                 float inv;
                 asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(run_s));
                 const float2 l2e = make_float2(kLog2e, kLog2e), mnm = make_float2(-run_m, -run_m), inv2 = make_float2(inv, inv);
-                uint4* pr = p.y + row * chunks;
+                uint4* pr = reinterpret_cast<uint4*>((unsigned short*) p.y + e0 + head);
+                if (edge) {
+                    const float val = edge_value(edge_e);
+                    const float pe = exp2_fast(fmaf(val, kLog2e, -run_m)) * inv;
+                    ((unsigned short*) p.y)[edge_e] = (unsigned short) (pack16x2(pe, 0.0f, f16) & 0xffffu);
+                }
                 for (int c0 = threadIdx.x; c0 < chunks; c0 += kThreads * kGroup) {
                     uint4 xv[kGroup], rv[kGroup];
 #pragma unroll
@@ -765,7 +797,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(c
 // fast-path parameters.
 static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, bool* res) {
     if (p.x_dt == FC_F32 || (p.y && p.y_dt != p.x_dt)) return false;
-    if (p.N % 8 != 0 || p.N >= 0x40000000LL || p.M >= 0x7fffffffLL) return false;
+    if ((p.N % 8 != 0 && p.N < kLongRow) || p.N >= 0x40000000LL || p.M >= 0x7fffffffLL) return false;
     if ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.y)) & 15) return false;
     int i = 0;
     *pre = kPreNone; *act = kActNone; *res = false;
@@ -806,6 +838,8 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
         ++i;
     }
     if (i != p.ops.n) return false;
+    f->ragged = p.N % 8 != 0;
+    if (f->ragged && (f->vec0 || f->vec1 || p.reduce == FC_RED_NONE || (*act & kActPost))) return false;   // long-row kernel, no vectors
     if (p.N > kMaxWarpRow) {
         // only the CTA-per-row kernel takes rows this long: a row reduction, no post ops, 16-bit aligned vectors
         const bool vec_ok = (!f->vec0 || (f->vec0_dt != FC_F32 && (reinterpret_cast<uintptr_t>(f->vec0) & 15) == 0)) &&

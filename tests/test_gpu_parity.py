@@ -225,6 +225,28 @@ def test_elementwise_narrow_rows_share_a_warp(fc, orc, M, N, red):
         run_and_check(fc, orc, _as_f16(replace(base, reduce=red, store_main=False, ops=())), 4)
 
 
+@pytest.mark.parametrize("M,N", [(9, 50257), (17, 12289), (5, 10243), (3, 30001), (4, 20002)])
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+def test_elementwise_long_ragged_rows(fc, orc, M, N, dt):
+    """A vocabulary of 50257: rows whose length is no multiple of 8 start anywhere in memory.  Chains without
+    per-column vectors take the CTA-per-row kernel all the same: the aligned middle of every row in 16-byte chunks,
+    up to 14 edge elements one by one.  Softmax (with a -inf mask too), logsumexp with the main output stored,
+    sum / max / mean."""
+    sm = wl.scale_add_softmax(M, N, dtype=dt)
+    if dt == "bf16":
+        run_and_check(fc, orc, sm, 3)
+    ins = wl.make_inputs(sm, 5)
+    keep = (np.arange(N)[None, :] * 7 + np.arange(M)[:, None]) % 640 < 3
+    keep[:, [0, N - 1]] = True
+    ins[1] = rng.store(np.where(keep, 0.0, -np.inf).astype(np.float32), dt)
+    outs, _, _ = run_and_check(fc, orc, sm, ins=ins)
+    assert (util.to_f64(outs[0])[~keep] == 0.0).all()
+    base = replace(sm, ops=(("scale", 0.5), ("gelu_tanh",), ("add_tensor", 1)))
+    run_and_check(fc, orc, replace(base, reduce="row_logsumexp", store_main=True), 3)
+    for red in ("row_sum", "row_max", "row_mean"):
+        run_and_check(fc, orc, replace(base, reduce=red, store_main=False, ops=(("relu",),)), 3)
+
+
 def test_gelu_accuracy_dense_grid_fp32(fc, orc):
     """The kernels evaluate tanh-GELU with the hardware tanh approximation.  On a dense grid of
     inputs (fp32 in, fp32 out, so nothing but the activation's own error shows) the result must stay
