@@ -272,6 +272,9 @@ uint64_t fc_launch_count(void);
 
 const char* fc_status_string(fc_status s);
 const char* fc_last_error(void);   /* thread-local text of the last failure in this thread */
+/* Thread-local, space-separated names of the kernel variants that the last fc_run of this thread enqueued ("ew_rows",
+ * "ew_narrow", "gemm_tc_mode1_bn256_two_pass softmax_rescale", ...): which path a chain took, for logs and tests. */
+const char* fc_last_plan(void);
 int fc_version(void);
 
 #ifdef __cplusplus

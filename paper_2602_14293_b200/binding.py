@@ -88,6 +88,7 @@ def lib():
         L.fc_status_string.argtypes = [ctypes.c_int]
         L.fc_status_string.restype = ctypes.c_char_p
         L.fc_last_error.restype = ctypes.c_char_p
+        L.fc_last_plan.restype = ctypes.c_char_p
         L.fc_version.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -95,6 +96,11 @@ def lib():
 
 def fc_last_error() -> str:
     return lib().fc_last_error().decode()
+
+
+def fc_last_plan() -> str:
+    """Names of the kernel variants the last fc_run of this thread enqueued."""
+    return lib().fc_last_plan().decode()
 
 
 def fc_version() -> int:

@@ -260,6 +260,7 @@ cudaError_t launch_collapse(const CollapseParams& p_in, void* workspace, cudaStr
     p.cterm = p.cpart + full_splits;
     p.u = (float*) ((char*) workspace + ((full_splits * (size_t) p.K + full_splits + 1) * sizeof(double) + 255) / 256 * 256);
     const int col_blocks = (int) ((p.K + kColsPerBlock - 1) / kColsPerBlock);
+    note_kernel("weight_colsum colsum_finish row_dot");
     weight_colsum_kernel<<<dim3(col_blocks, splits), kWarps * 32, 0, stream>>>(p, rows_per_block);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

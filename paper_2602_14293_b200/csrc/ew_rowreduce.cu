@@ -880,6 +880,7 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
         attr.val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
+        note_kernel("ew_narrow");
         return cudaLaunchKernelEx(&cfg, ew_narrow_kernel<PRE, ACT, RES>, f, cpr_log2);
     }
     // Rows from kLongRow columns on (lists without the post ops, 16-bit vectors on 16-byte boundaries) go to the
@@ -899,6 +900,7 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
             attr.val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = &attr;
             cfg.numAttrs = 1;
+            note_kernel(f.ragged ? "ew_longrow_ragged" : "ew_longrow");
             if (sm) return cudaLaunchKernelEx(&cfg, ew_longrow_kernel<PRE, ACT, RES, true, false, true>, f);
             if (store) return cudaLaunchKernelEx(&cfg, ew_longrow_kernel<PRE, ACT, RES, true, true, false>, f);
             return cudaLaunchKernelEx(&cfg, ew_longrow_kernel<PRE, ACT, RES, true, false, false>, f);
@@ -931,6 +933,7 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, kernel, f);
     };
+    note_kernel(f.red_kind == FC_RED_ROW_SOFTMAX ? (f.stash ? "ew_rows_softmax_stash" : "ew_rows_softmax") : "ew_rows");
     if constexpr ((ACT & kActPost) == 0) {
         if (f.red_kind == FC_RED_ROW_SOFTMAX) return go(ew_rows_kernel<PRE, ACT, RES, true, false, true>, 3);
         if (lse && !store) return go(ew_rows_kernel<PRE, ACT, RES, true, false>, 1);
@@ -968,6 +971,7 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
     if (!lse) work = (p.M * ((p.N + 7) / 8) + kThreads - 1) / kThreads;
     long long grid = work < (long long) num_sms * 8 ? work : (long long) num_sms * 8;
     if (grid < 1) grid = 1;
+    note_kernel(lse ? "ew_interpreter_rows" : "ew_interpreter_flat");
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned) grid);
     cfg.blockDim = dim3(kThreads);

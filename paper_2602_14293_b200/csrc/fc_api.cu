@@ -16,6 +16,7 @@ __device__ int g_status_word;  // written by kernels when a bounded wait expires
 namespace {
 
 thread_local char t_err[512] = "";
+thread_local char t_plan[256] = "";
 std::atomic<uint64_t> g_launches{0};
 
 fc_status fail(fc_status s, const char* fmt, ...) {
@@ -132,6 +133,15 @@ size_t nchw_image_bytes(const fc_chain_spec* s) { return ((size_t) s->batch * s-
 size_t nchw_workspace_bytes(const fc_chain_spec* s) {
     return nchw_image_bytes(s) + ((size_t) s->Cout * s->R * s->S * s->Cin * 2 + 255) / 256 * 256;
 }
+
+}  // namespace
+
+void note_kernel(const char* name) {
+    const size_t have = strlen(t_plan);
+    snprintf(t_plan + have, sizeof(t_plan) - have, "%s%s", have ? " " : "", name);
+}
+
+namespace {
 
 fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (!s) return fail(FC_ERR_NULL, "spec is null");
@@ -512,6 +522,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                  void* cuda_stream) {
     Plan plan;
     fc_status st;
+    t_plan[0] = 0;
     if ((st = validate_spec(spec, &plan))) return st;
     if ((st = validate_tensors(spec, plan, inputs, n_inputs, outputs, n_outputs))) return st;
     DeviceInfo* dev;
@@ -974,6 +985,7 @@ const char* fc_status_string(fc_status s) {
 }
 
 const char* fc_last_error(void) { return t_err; }
+const char* fc_last_plan(void) { return t_plan; }
 
 int fc_version(void) { return FC_VERSION; }
 

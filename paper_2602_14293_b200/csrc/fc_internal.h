@@ -76,6 +76,9 @@ struct CollapseParams {
 cudaError_t launch_collapse(const CollapseParams& p, void* workspace, cudaStream_t stream, int* launches);
 size_t collapse_workspace_bytes(long long N, long long K);
 
+// Appends the name of a kernel variant to this thread's record of what the current fc_run enqueues (fc_last_plan).
+void note_kernel(const char* name);
+
 // Stack of `mats` 16-bit matrices [C][P] -> [P][C] (layout.cu): the channels-last rewrite for CONV2D_NCHW.  C even.
 // `beside_previous`: the kernel in front of this one in the stream shares no memory with it, so the two may overlap.
 cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,

@@ -190,6 +190,7 @@ cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* la
     const long long wide_tiles = (long long) ((p.M + kTile - 1) / kTile) * ((p.N + kTile - 1) / kTile);
     if (wide_tiles >= 512 && (p.M + kTile - 1) / kTile <= 65535) {
         dim3 wide((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile);
+        note_kernel("gemm_f32_wide");
         gemm_f32_wide_kernel<<<wide, 256, 0, stream>>>(p);
         *launches += 1;
         return cudaGetLastError();
@@ -207,6 +208,7 @@ cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* la
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     *launches += 1;
+    note_kernel("gemm_f32");
     return cudaLaunchKernelEx(&cfg, gemm_f32_kernel, p);
 }
 

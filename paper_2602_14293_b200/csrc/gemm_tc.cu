@@ -43,6 +43,8 @@
 // resets it, so a launch needs no memset as long as the previous one ran to completion.
 #include "tc_common.cuh"
 
+#include <cstdio>
+
 namespace fc {
 namespace {
 
@@ -926,6 +928,11 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     if (!tmA) return cudaSuccess;   // planning only
     cfg.gridDim = dim3(2 * clusters);
     cfg.numAttrs = 2;   // cluster shape + programmatic stream serialization
+    {
+        char name[64];
+        snprintf(name, sizeof(name), "gemm_tc_mode%d_bn%d%s%s", MODE, BN, q.split > 1 ? "_split" : "", MODE == 1 && p.two_pass ? "_two_pass" : "");
+        note_kernel(name);
+    }
     return cudaLaunchKernelEx(&cfg, kernel, *tmA, *tmB, q);
 }
 

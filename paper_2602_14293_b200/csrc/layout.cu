@@ -115,6 +115,7 @@ cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t 
     size_t blocks = (words / 4 + 255) / 256;
     if (blocks < 1) blocks = 1;
     if (blocks > (size_t) num_sms * 4) blocks = (size_t) num_sms * 4;
+    note_kernel("zero_fill");
     zero_fill_kernel<<<(unsigned) blocks, 256, 0, stream>>>((uint32_t*) ptr, words);
     ++*launches;
     return cudaGetLastError();
@@ -139,6 +140,7 @@ cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, i
     const unsigned short* s16 = (const unsigned short*) src;
     unsigned short* d16 = (unsigned short*) dst;
     ++*launches;
+    note_kernel("cfirst_to_clast");
     if (P <= kTile && P % 4 != 0) return cudaLaunchKernelEx(&cfg, cfirst_to_clast_kernel<0>, s16, d16, C, P, tiles_p);
     if (P % 4 == 0 && reinterpret_cast<uintptr_t>(src) % 8 == 0) return cudaLaunchKernelEx(&cfg, cfirst_to_clast_kernel<4>, s16, d16, C, P, tiles_p);
     return cudaLaunchKernelEx(&cfg, cfirst_to_clast_kernel<1>, s16, d16, C, P, tiles_p);

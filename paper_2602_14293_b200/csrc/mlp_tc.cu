@@ -321,6 +321,7 @@ cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUte
     const CUtensorMap& w3 = tmW[p.layers > 3 ? 3 : 0];
     *launches += 1;
     cfg.numAttrs = 2;
+    note_kernel("mlp_tc");
     return cudaLaunchKernelEx(&cfg, mlp_tc_kernel, tmX, tmW[0], w1, w2, w3, p);
 }
 

@@ -81,6 +81,7 @@ cudaError_t launch_softmax_rescale(void* out, int out_dt, const float2* stats, l
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     ++*launches;
+    note_kernel("softmax_rescale");
     return cudaLaunchKernelEx(&cfg, softmax_rescale_kernel, out, out_dt, stats, M, N, tiles_n, bn);
 }
 
