@@ -16,6 +16,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
+constexpr int kInterpreterWarpRowChunks = 1024;   // interpreter: rows up to 8192 columns get a warp, longer ones a CTA
 
 __device__ __forceinline__ MaxSum block_merge(MaxSum a, MaxSum* smem /* [kWarps] */) {
     a = ms_warp_reduce(a);
@@ -133,6 +134,35 @@ __global__ void __launch_bounds__(kThreads) ew_generic_kernel(const EwParams p) 
             m += dm;
             c += dc;
             if (c >= chunks) { c -= chunks; ++m; }
+        }
+        return;
+    }
+
+    if (chunks <= kInterpreterWarpRowChunks) {
+        // Rows of moderate length: a warp per row, the row's partial results merged by shuffles.  A CTA per row
+        // would pay two block barriers and a memory round trip per row with nothing else in flight (16384 rows
+        // of 4096 columns with an op list the row kernel does not take: 201 us against 182 us).
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        for (long long m = (long long) blockIdx.x * kWarps + warp; m < p.M; m += (long long) gridDim.x * kWarps) {
+            MaxSum acc = ms_identity();
+            float psum = 0.0f, pmax = -CUDART_INF_F;
+            const int phase = p.reduce == FC_RED_ROW_SOFTMAX ? 1 : 0;
+            for (long long c = lane; c < chunks; c += 32) chunk(m, c, acc, psum, pmax, phase, 0.0f, 0.0f);
+            if (p.reduce == FC_RED_ROW_SOFTMAX) {
+                const MaxSum t = ms_warp_reduce(acc);
+                const float inv = 1.0f / t.s;
+                for (long long c = lane; c < chunks; c += 32) chunk(m, c, acc, psum, pmax, 2, t.m, inv);
+            } else if (p.reduce == FC_RED_ROW_LOGSUMEXP) {
+                const MaxSum t = ms_warp_reduce(acc);
+                if (lane == 0) p.red[m] = t.m + logf(t.s);
+            } else {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    psum += __shfl_xor_sync(0xffffffffu, psum, o);
+                    pmax = fmaxf(pmax, __shfl_xor_sync(0xffffffffu, pmax, o));
+                }
+                if (lane == 0) p.red[m] = p.reduce == FC_RED_ROW_MAX ? pmax : (p.reduce == FC_RED_ROW_MEAN ? psum / (float) N : psum);
+            }
         }
         return;
     }
@@ -967,7 +997,8 @@ cudaError_t launch_ew_rowreduce(const EwParams& p, int num_sms, cudaStream_t str
 #undef FC_EW_CASE
     }
     const bool precise = false;   // tanh.approx is accurate to 6e-6 here (see gelu_tanh)
-    long long work = p.M;   // CTAs that can be kept busy: rows, or 256-chunk slabs of the whole tensor
+    long long work = p.M;   // CTAs that can be kept busy: rows (a warp each up to 8192 columns), or 256-chunk slabs of the whole tensor
+    if (lse && (p.N + 7) / 8 <= kInterpreterWarpRowChunks) work = (p.M + kWarps - 1) / kWarps;
     if (!lse) work = (p.M * ((p.N + 7) / 8) + kThreads - 1) / kThreads;
     long long grid = work < (long long) num_sms * 8 ? work : (long long) num_sms * 8;
     if (grid < 1) grid = 1;
