@@ -226,7 +226,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int u = cluster_id; u < total_units && ok; u += num_clusters) {
                 const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 int mb2, nb;
-                tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);
+                tile_coords((MODE == 0 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
@@ -338,7 +338,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int u = cluster_id; u < total_units; u += num_clusters, ++tile_iter) {
             const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
             int mb2, nb;
-            tile_coords((MODE == 0 || MODE == 3) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);
+            tile_coords((MODE == 0 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
             const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;
@@ -883,7 +883,7 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
         // pair count that is a multiple of the column-tile count every panel lives inside one round;
         // otherwise panels straddle rounds and their first tiles hold an accumulator buffer for a
         // whole extra round.
-        if (clusters > tiles_n) clusters = clusters / tiles_n * tiles_n;
+        if (clusters > tiles_n && !p.two_pass) clusters = clusters / tiles_n * tiles_n;
     }
     TcParams q = p;
     q.split = 1;
