@@ -393,7 +393,8 @@ void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
 }
 
 constexpr int kSoftmaxBN = 256;
-constexpr int kSoftmaxOnePassTiles = 64;   // widest row (in tiles) that the single-pass softmax takes
+constexpr int kSoftmaxOnePassTiles = 64;       // widest row (in tiles) that the single-pass softmax can take safely
+constexpr int kSoftmaxOnePassBestTiles = 16;   // widest row for which it is also the faster form (measured)
 
 // arrival counters and departure counters, one of each per 128-row panel
 size_t panel_counter_bytes(long long M) {
@@ -598,14 +599,18 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
             // Row softmax over more tiles per panel than the pairs' accumulator buffers can hold until the panel is
-            // complete (two per pair; with a margin: 64 tiles = 16384 columns): no waiting across tiles, and a second,
-            // memory-bound kernel finishes the rows.
+            // complete (two per pair; with a margin: 64 tiles = 16384 columns) cannot wait across tiles: a second,
+            // memory-bound kernel finishes the rows.  The same two-kernel form is also chosen where it is faster.
             const int tiles_n = (int) ((spec->N + bn - 1) / bn);
             if (p.mode == 1) {
                 // (never more tiles per panel than SM pairs take part, whatever the device offers)
                 TcPlan tp;
                 if ((e = plan_gemm_tc(p, bn, dev->num_sms, &tp)) != cudaSuccess) return cuda_fail(e, "planning");
-                p.two_pass = tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs;
+                // The single pass wins where it was built for (rows of up to 16 tiles and a long contraction: 4096^3 106
+                // against 118 us); its panel-by-panel order streams B once per panel and its epilogue waits for the
+                // panel, which loses from 8192 columns on and for short contractions (8192 x 16384 x 4096: 1208
+                // against 838 us; 16384 x 16384 x 1024: 2024 against 877 us).
+                p.two_pass = tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs || tiles_n > kSoftmaxOnePassBestTiles || spec->K < 4096;
             }
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             if (e == cudaSuccess && p.two_pass)

@@ -431,7 +431,8 @@ def _check_softmax_rows(t):
 
 
 @pytest.mark.parametrize("variant", ["std", "var"])
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 1024, 256), (300, 1000, 136), (512, 4096, 128), (130, 264, 72)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 1024, 256), (300, 1000, 136), (512, 4096, 128), (130, 264, 72),
+                                   (300, 1000, 4096), (129, 4096, 4104), (600, 264, 4096)])   # the last three: single-pass form (K >= 4096)
 def test_c4_softmax_reduced(fc, orc, M, N, K, variant):
     outs, _, _ = run_and_check(fc, orc, wl.gemm_softmax(M, N, K, variant), 1)
     _check_softmax_rows(outs[0])

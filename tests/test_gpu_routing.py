@@ -51,7 +51,10 @@ def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 512, 256)) == "gemm_tc_mode0_bn256"
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(128, 256, 4096)) == "gemm_tc_mode0_bn256_split"
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 128, 256)) == "gemm_tc_mode0_bn128"
-    assert _plan(fc, wl.gemm_softmax(256, 1024, 256)) == "gemm_tc_mode1_bn256"
+    assert _plan(fc, wl.gemm_softmax(256, 1024, 4096)) == "gemm_tc_mode1_bn256_split"      # 4 tiles: cut along K as well
+    assert _plan(fc, wl.gemm_softmax(4096, 4096, 4096)) == "gemm_tc_mode1_bn256"
+    assert _plan(fc, wl.gemm_softmax(256, 1024, 256)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"   # short contraction
+    assert _plan(fc, wl.gemm_softmax(256, 8192, 4096)) == "gemm_tc_mode1_bn256_split_two_pass softmax_rescale"  # 32 tiles per panel (and few enough to be cut along K)
     assert _plan(fc, wl.gemm_softmax(64, 20000, 64)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"
     assert _plan(fc, wl.gemm_bias_scale_lse(256, 1024, 256)) == "gemm_tc_mode3_bn256"
     assert _plan(fc, wl.linear_row_reduce(96, 512, 256)) == "weight_colsum colsum_finish row_dot"

@@ -21,7 +21,7 @@ def test_panel_wait_expires_with_status_and_device_stays_usable(orc):
     import paper_2602_14293_b200 as fc
     assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
     torch.cuda.set_device(0)
-    ch = wl.gemm_softmax(256, 512, 64, "var")
+    ch = wl.gemm_softmax(256, 512, 4096, "var")      # a long contraction: the single-pass form, whose tiles wait for their panel
     ins = wl.make_inputs(ch, 0)
     dev = [fc.to_device(a) for a in ins]
     outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
