@@ -402,10 +402,12 @@ size_t panel_counter_bytes(long long M) {
     return ((size_t) panels * 4 + 255) / 256 * 256;
 }
 
-size_t softmax_workspace_bytes(long long M, long long N) {
+size_t softmax_workspace_bytes(long long M, long long N, bool per_half = false) {
     const long long tiles_n = (N + kSoftmaxBN - 1) / kSoftmaxBN;
-    return 2 * panel_counter_bytes(M) + (size_t) M * tiles_n * sizeof(float2);
+    return 2 * panel_counter_bytes(M) + (size_t) M * tiles_n * sizeof(float2) * (per_half ? 2 : 1);
 }
+// fc_run's row softmax may take the two-kernel form, which keeps a pair per row, tile and column half
+size_t reduction_workspace_bytes(bool softmax, long long M, long long N) { return softmax_workspace_bytes(M, N, softmax); }
 
 // The part of the caller's workspace behind the row-reduction statistics serves split tiles; without it
 // (no workspace, or a smaller one) the tensor-core kernels simply never split.
@@ -585,7 +587,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             }
             size_t panel_bytes = 0;
             if (p.mode == 1 || p.mode == 3) {
-                const size_t need = softmax_workspace_bytes(spec->M, spec->N);
+                const size_t need = reduction_workspace_bytes(p.mode == 1, spec->M, spec->N);
                 if (!dev->workspace || dev->workspace_bytes < need)
                     return fail(FC_ERR_WORKSPACE, "this row reduction needs a %zu-byte workspace (fc_set_workspace); have %zu", need, dev->workspace_bytes);
                 panel_bytes = panel_counter_bytes(spec->M);
@@ -593,7 +595,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 p.departed = (unsigned int*) ((char*) dev->workspace + panel_bytes);
                 p.stats = (float2*) ((char*) dev->workspace + 2 * panel_bytes);
             }
-            attach_split_scratch(dev, p.mode == 1 || p.mode == 3 ? softmax_workspace_bytes(spec->M, spec->N) : 0, &p);
+            attach_split_scratch(dev, p.mode == 1 || p.mode == 3 ? reduction_workspace_bytes(p.mode == 1, spec->M, spec->N) : 0, &p);
             if ((e = clear_counters_if_needed(dev, p, panel_bytes, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
             CUtensorMap tmA, tmB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
@@ -884,7 +886,7 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     fc_status st;
     if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
     if ((st = validate_spec(spec, &plan))) return st;
-    *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N)
+    *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? reduction_workspace_bytes(plan.kind == Plan::TC_SOFTMAX, spec->M, spec->N)
            : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K)
            : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     return FC_OK;
@@ -896,7 +898,7 @@ fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes) {
     if (!bytes) return fail(FC_ERR_NULL, "bytes is null");
     if ((st = validate_spec(spec, &plan))) return st;
     const bool tc = plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_CONV;
-    const size_t red = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? softmax_workspace_bytes(spec->M, spec->N)
+    const size_t red = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? reduction_workspace_bytes(plan.kind == Plan::TC_SOFTMAX, spec->M, spec->N)
                      : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     *bytes = tc ? split_workspace_offset(red) + kTcSplitBytes : 0;
     return FC_OK;
@@ -928,7 +930,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
         p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
         p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
         bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
-        if (p.mode == 1 || p.mode == 3) red = softmax_workspace_bytes(spec->M, spec->N);
+        if (p.mode == 1 || p.mode == 3) red = reduction_workspace_bytes(p.mode == 1, spec->M, spec->N);
     }
     attach_split_scratch(dev, red, &p);
     TcPlan tp;

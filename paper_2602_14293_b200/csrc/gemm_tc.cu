@@ -610,6 +610,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 });
                 if (has_ops) ptx::tmem_wait_st();
+                if (p.two_pass) {
+                    // Two-kernel form: nobody waits for the panel.  One more sweep computes the exponentials against
+                    // this half row's own maximum (values in (0, 1]), sums them and stores them at once; the pair
+                    // (max, sum) of every (row, tile, half) goes to the workspace and the rescale kernel behind this
+                    // one finishes the rows.
+                    const float2 l2e = make_float2(kLog2e, kLog2e);
+                    const float mbase = mx == -CUDART_INF_F ? 0.0f : mx;   // a half row of -inf only: exponents against 0
+                    const float2 moff = make_float2(-mbase * kLog2e, -mbase * kLog2e);
+                    float2 acc2 = make_float2(0.0f, 0.0f);
+                    const bool ok = *abort_flag == 0;
+                    tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                        const int n0 = n_half + c * 16;
+                        if (n0 >= p.N) return;
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float2 t = __ffma2_rn(make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1])), l2e, moff);
+                            float2 e = make_float2(exp2_fast(t.x), exp2_fast(t.y));
+                            if (n0 + 2 * j >= p.N) e.x = 0.0f;
+                            if (n0 + 2 * j + 1 >= p.N) e.y = 0.0f;
+                            acc2 = __fadd2_rn(acc2, e);
+                            v[2 * j] = e.x;
+                            v[2 * j + 1] = e.y;
+                        }
+                        if (!out_vec) {
+                            if (__all_sync(0xffffffffu, ok)) store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                        } else if (m < p.M && ok) {
+                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                        }
+                    });
+                    if (m < p.M) __stcg(&p.stats[(m * tiles_n + nb) * 2 + half], make_float2(mx, acc2.x + acc2.y));
+                    release_buf();
+                    continue;
+                }
                 // sweep B: e = 2^((v - max) log2 e), summed, and written back over the logits: the last sweep
                 // only rescales, so every element costs one exponential
                 float sm = 0.0f;
@@ -646,20 +680,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const MaxSum a = ms_merge(MaxSum{mx, sm}, MaxSum{o.x, o.y});
                     __stcg(&p.stats[m * tiles_n + nb], make_float2(a.m, a.s));
                 }
-                float tile_m = mx;   // two-pass form: the maximum both halves of this tile rescale to
-                if (p.two_pass) {
-                    if (half == 0 && m < p.M) {
-                        const float2 o = xchg[row];
-                        tile_m = fmaxf(mx, o.x);
-                    }
-                    ptx::bar_sync(1, kEpiThreads);          // the upper half's pair has been read
-                    if (half == 0) xchg[row] = make_float2(tile_m, 0.0f);
-                }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
-                if (p.two_pass && half == 1) tile_m = xchg[row].x;
                 // one thread announces the tile and waits (bounded) for the panel's other tiles
-                if (et == 0 && !p.two_pass) {
+                if (et == 0) {
                     ptx::red_release_gpu_add(&p.counters[mb], 1u);
                     const unsigned long long t0 = ptx::globaltimer();
                     unsigned spins = 0;
@@ -683,12 +707,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::bar_sync(1, kEpiThreads);
                 const bool store = *abort_flag == 0;
                 float row_m = -CUDART_INF_F, row_s = 0.0f;
-                if (p.two_pass) {
-                    // no row results yet: the exponentials are stored against the tile's own maximum (in (0, 1]) and
-                    // the rescale kernel behind this one divides by the row's sum
-                    row_m = tile_m;
-                    row_s = 1.0f;
-                } else if (m < p.M && store) {
+                if (m < p.M && store) {
                     MaxSum a = ms_identity();
                     for (int j = 0; j < tiles_n; ++j) {
                         const float2 st = __ldcg(&p.stats[m * tiles_n + j]);

@@ -3,8 +3,9 @@
 // The single-pass kernel keeps every tile of a 256-row panel in tensor memory until the panel's last tile has
 // published its (max, sum); that needs no more tiles per panel than the pairs have accumulator buffers (two
 // each).  For wider rows (a vocabulary) the GEMM kernel does not wait: every tile stores its exponentials
-// against its own row maximum (values in (0, 1]) and leaves (max_j, sum_j) per row and tile in the workspace.
-// This kernel gives a CTA to a row: it merges the row's pairs and rescales the stored values of tile j by
+// against the maximum of its half row (values in (0, 1]) and leaves (max_j, sum_j) per row, tile and column half in the
+// workspace.
+// This kernel gives a CTA to a row: it merges the row's pairs and rescales the stored values of half tile j by
 // 2^((max_j - max_row) log2 e) / sum_row, in place.  HBM-bound: the probabilities are read and written once more.
 #include "dev_common.cuh"
 
@@ -20,9 +21,10 @@ __global__ void __launch_bounds__(kRescaleThreads) softmax_rescale_kernel(void* 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool f16 = out_dt == FC_F16;
     for (long long m = blockIdx.x; m < M; m += gridDim.x) {
-        const float2* st = stats + m * tiles_n;
+        const int halves = 2 * tiles_n, hw = bn >> 1;   // one pair per tile and column half
+        const float2* st = stats + m * halves;
         MaxSum a = ms_identity();
-        for (int j = threadIdx.x; j < tiles_n; j += kRescaleThreads) {
+        for (int j = threadIdx.x; j < halves; j += kRescaleThreads) {
             const float2 t = __ldcg(st + j);
             a = ms_merge(a, MaxSum{t.x, t.y});
         }
@@ -36,7 +38,7 @@ __global__ void __launch_bounds__(kRescaleThreads) softmax_rescale_kernel(void* 
         const float inv = 1.0f / a.s;
         if (out_dt != FC_F32 && (N & 7) == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0) {
             uint4* row = reinterpret_cast<uint4*>((unsigned short*) out + m * N);
-            const int chunks = (int) (N >> 3), per_tile = bn >> 3;
+            const int chunks = (int) (N >> 3), per_tile = hw >> 3;
             for (int c = threadIdx.x; c < chunks; c += kRescaleThreads) {
                 const float mj = __ldcg(st + c / per_tile).x;
                 const float f = mj == -CUDART_INF_F ? 0.0f : exp2_fast((mj - a.m) * kLog2e) * inv;
@@ -51,7 +53,7 @@ __global__ void __launch_bounds__(kRescaleThreads) softmax_rescale_kernel(void* 
             }
         } else {
             for (long long n = threadIdx.x; n < N; n += kRescaleThreads) {
-                const float mj = __ldcg(st + n / bn).x;
+                const float mj = __ldcg(st + n / hw).x;
                 const float f = mj == -CUDART_INF_F ? 0.0f : exp2_fast((mj - a.m) * kLog2e) * inv;
                 if (out_dt == FC_F32) {
                     float* o = (float*) out + m * N + n;
