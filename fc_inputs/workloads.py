@@ -251,6 +251,7 @@ EXTRA = {
     "F3": lambda **kw: conv_bias_relu_maxpool(**{"batch": 32, "H": 56, "W": 56, "Cin": 256, "Cout": 256, "R": 3, "S": 3, "pad": 1, **kw}),
     "F6": lambda **kw: conv_nchw(conv_bias_relu_avgpool(**kw)),
     "F7": lambda **kw: scale_add_softmax(**kw),
+    "F8": lambda **kw: gemm_softmax(**{"M": 2048, "N": 50264, "K": 4096, **kw}),   # a vocabulary-wide softmax: two kernels
 }
 ALL = {**CONFIGS, **EXTRA}
 
