@@ -369,7 +369,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             auto release_buf = [&]() {
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive_cluster(tempty_leader + buf * 8);
+                // relaxed: every lane's accumulator reads are complete (tcgen05.wait::ld) before the __syncwarp above,
+                // and a release here would hold the warp until its global stores of this tile have drained
+                if (lane == 0) ptx::mbar_arrive_cluster_relaxed(tempty_leader + buf * 8);
             };
 
             if (w.nsl > 1) {

@@ -177,6 +177,15 @@ __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, cons
         const bool f16 = out_dt == FC_F16;
         unsigned short* o = (unsigned short*) out + m * N + n0;
         if (vec_ok && n0 + 16 <= N) {
+            if ((reinterpret_cast<uintptr_t>(o) & 31) == 0) {
+                // one 256-bit store: a whole 32-byte sector per thread and instruction
+                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o), "r"(pack16x2(v[0], v[1], f16)),
+                             "r"(pack16x2(v[2], v[3], f16)), "r"(pack16x2(v[4], v[5], f16)), "r"(pack16x2(v[6], v[7], f16)),
+                             "r"(pack16x2(v[8], v[9], f16)), "r"(pack16x2(v[10], v[11], f16)), "r"(pack16x2(v[12], v[13], f16)),
+                             "r"(pack16x2(v[14], v[15], f16))
+                             : "memory");
+                return;
+            }
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 uint4 w;
@@ -194,6 +203,14 @@ __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, cons
     } else {
         float* o = (float*) out + m * N + n0;
         if (vec_ok && n0 + 16 <= N) {
+            if ((reinterpret_cast<uintptr_t>(o) & 31) == 0) {
+#pragma unroll
+                for (int q = 0; q < 2; ++q)
+                    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o + 8 * q), "f"(v[8 * q]), "f"(v[8 * q + 1]),
+                                 "f"(v[8 * q + 2]), "f"(v[8 * q + 3]), "f"(v[8 * q + 4]), "f"(v[8 * q + 5]), "f"(v[8 * q + 6]), "f"(v[8 * q + 7])
+                                 : "memory");
+                return;
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q)
                 reinterpret_cast<float4*>(o)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
