@@ -402,6 +402,27 @@ size_t panel_counter_bytes(long long M) {
     return ((size_t) panels * 4 + 255) / 256 * 256;
 }
 
+// Column-tile width of the GEMM kernels: 256, except that a small plain GEMM (mode 0, 256-wide tiles on at most
+// half of the SM pairs) takes 128-wide tiles where this cost model says so.  Such a call is one round of tiles,
+// so its time is the critical tile's: main loop (of the merging slice, when tiles are cut along K) + epilogue
+// + merge.  Measured, in microseconds: a k-block 0.33 (256 wide) / 0.30 (128 wide; 24 instead of 32 KB), the
+// epilogue 6 / 3, merging a split tile 8 / 4.4.  128 x 1024 x 1024: 13.7 -> 11.2; 256 x 4096 x 4096: 23.0 -> 20.1;
+// 16 x 8192 x 8192 stays at 256 (37 against 45).  `p` has its split scratch attached already.
+int gemm_tile_width(const TcParams& p, const fc_chain_spec* s, int num_sms) {
+    if (p.mode == 1) return kSoftmaxBN;
+    if (s->N <= 128) return 128;
+    const long long tiles = ((s->M + 255) / 256) * ((s->N + 255) / 256);
+    if (p.mode != 0 || 2 * tiles > num_sms / 2) return 256;
+    auto cost = [&](int bn) -> double {
+        TcPlan tp;
+        if (plan_gemm_tc(p, bn, num_sms, &tp) != cudaSuccess) return 1e30;
+        const bool cut = tp.split > 1;
+        const int kb = cut ? tp.num_kb - tp.split_kb * (tp.split - 1) : tp.num_kb;
+        return bn == 256 ? kb * 0.33 + 6.0 + (cut ? 8.0 : 0.0) : kb * 0.30 + 3.0 + (cut ? 4.4 : 0.0);
+    };
+    return cost(128) < cost(256) ? 128 : 256;
+}
+
 size_t softmax_workspace_bytes(long long M, long long N, bool per_half = false) {
     const long long tiles_n = (N + kSoftmaxBN - 1) / kSoftmaxBN;
     return 2 * panel_counter_bytes(M) + (size_t) M * tiles_n * sizeof(float2) * (per_half ? 2 : 1);
@@ -568,7 +589,6 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.red_kind = spec->reduce;
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
-            const int bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
             {
                 // keep about 32 MB of A rows (group_m panels of 256 rows) resident in L2 per sweep
                 const long long panel_bytes = 256LL * spec->K * (long long) dt_size(spec->in_dtype);
@@ -597,6 +617,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             }
             attach_split_scratch(dev, p.mode == 1 || p.mode == 3 ? reduction_workspace_bytes(p.mode == 1, spec->M, spec->N) : 0, &p);
             if ((e = clear_counters_if_needed(dev, p, panel_bytes, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+            const int bn = gemm_tile_width(p, spec, dev->num_sms);
             CUtensorMap tmA, tmB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
@@ -929,10 +950,11 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     } else {
         p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
         p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
-        bn = p.mode == 1 ? kSoftmaxBN : (spec->N <= 128 ? 128 : 256);
+        bn = 0;
         if (p.mode == 1 || p.mode == 3) red = reduction_workspace_bytes(p.mode == 1, spec->M, spec->N);
     }
     attach_split_scratch(dev, red, &p);
+    if (!bn) bn = gemm_tile_width(p, spec, dev->num_sms);
     TcPlan tp;
     cudaError_t e = plan_gemm_tc(p, bn, dev->num_sms, &tp);
     if (e != cudaSuccess) return cuda_fail(e, "planning");

@@ -150,6 +150,7 @@ cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUte
 struct TcPlan {
     int bn, tiles, pairs;       // tile width, 256 x bn output tiles, CTA pairs launched
     int split, split_tiles, split_kb;   // slices per split tile (1: none), tiles that are split, k-blocks per parking slice
+    int num_kb;                 // k-blocks of a whole tile
 };
 cudaError_t plan_gemm_tc(const TcParams& p, int bn, int num_sms, TcPlan* plan);
 

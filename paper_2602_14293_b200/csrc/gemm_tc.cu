@@ -380,10 +380,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 constexpr size_t kSliceF4 = (size_t) BM * BN / 4;
                 const int ws = warp - 2;
                 unsigned int* cnt = &p.split_counters[(w.v0 / w.nsl) * 2 + (int) cta_rank];
+                // a warp none of whose 32 rows exists (a short last panel: 16 rows of 256) parks and merges nothing
+                const bool live = m - lane < p.M;
                 if (w.slice != w.nsl - 1) {
                     float4* mine = p.split_ws + ((size_t) (w.v0 + w.slice) * 2 + cta_rank) * kSliceF4 + (size_t) ws * kChunks * 128 + lane;
 #pragma unroll 1
-                    for (int c = 0; c < kChunks; c += 2) {
+                    for (int c = 0; live && c < kChunks; c += 2) {
                         uint32_t ra[16], rb[16];
                         ptx::tmem_ld_32x16_async(tacc + c * 16, ra);
                         ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
@@ -425,7 +427,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (!*(volatile int*) &ctrl->merge_ok) break;
                 // add the other slices' rows into the accumulator, four chunks of loads in flight
 #pragma unroll 1
-                for (int c0 = 0; c0 < kChunks; c0 += 4) {
+                for (int c0 = 0; live && c0 < kChunks; c0 += 4) {
                     float4 acc[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) acc[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
@@ -945,6 +947,7 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
         plan->split = q.split;
         plan->split_tiles = tiles - q.split_from;
         plan->split_kb = q.split_kb;
+        plan->num_kb = count_kb<MODE>(p);
     }
     if (!tmA) return cudaSuccess;   // planning only
     cfg.gridDim = dim3(2 * clusters);

@@ -355,6 +355,17 @@ def test_c3_chain_ragged(fc, orc, M, N, K):
     run_and_check(fc, orc, replace(wl.gemm_bias_gelu_scale_clamp(M, N, K, "var"), out_dtype="f32"), 4)
 
 
+@pytest.mark.parametrize("M,N,K,plan", [(100, 1000, 4096, "bn128_split"), (2048, 1024, 1024, "bn128"), (250, 2304, 768, "bn128"),
+                                        (16, 8192, 4096, "bn128"), (16, 4096, 8192, "bn256_split"), (1024, 1024, 8192, "bn256_split")])
+def test_gemm_few_tiles_either_tile_width(fc, orc, M, N, K, plan):
+    """A GEMM of few tiles takes 128- or 256-column tiles, whole or cut along K, whichever a cost model makes
+    faster: every combination against the oracle, bf16 and fp32 output."""
+    ch = wl.gemm_bias_gelu_scale_clamp(M, N, K, "var")
+    run_and_check(fc, orc, ch, 9)
+    assert fc.fc_last_plan() == "gemm_tc_mode0_" + plan
+    run_and_check(fc, orc, replace(ch, out_dtype="f32"), 9)
+
+
 def test_gemm_tc_op_lists_fused_and_interpreted(fc, orc):
     """Op lists of the fused shape ([bias|affine] [relu|gelu] [scale] [clamp] [add tensor]) take the
     packed straight-line epilogue; any other order is interpreted op by op.  Both against the oracle."""

@@ -48,8 +48,12 @@ def test_elementwise_routing(fc):
 def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_bias_relu_f32(256, 256, 256)) == "gemm_f32"
     assert _plan(fc, wl.gemm_bias_relu_f32(1024, 1024, 64)) == "gemm_f32_wide"
-    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 512, 256)) == "gemm_tc_mode0_bn256"
-    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(128, 256, 4096)) == "gemm_tc_mode0_bn256_split"
+    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(4096, 4096, 256)) == "gemm_tc_mode0_bn256"
+    # few tiles: 128-wide ones where the cost model prefers twice the tiles with half the epilogue each ...
+    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 512, 256)) == "gemm_tc_mode0_bn128"
+    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(128, 256, 4096)) == "gemm_tc_mode0_bn128_split"
+    # ... and 256-wide ones cut along K where the main loop dominates
+    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(16, 8192, 8192)) == "gemm_tc_mode0_bn256_split"
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 128, 256)) == "gemm_tc_mode0_bn128"
     assert _plan(fc, wl.gemm_softmax(256, 1024, 4096)) == "gemm_tc_mode1_bn256_split"      # 4 tiles: cut along K as well
     assert _plan(fc, wl.gemm_softmax(4096, 4096, 4096)) == "gemm_tc_mode1_bn256"
