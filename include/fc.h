@@ -196,7 +196,9 @@ fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, in
 /*
  * Scratch memory.  A 16-bit GEMM_NT with a row reduction needs some (per-tile partial results plus
  * per-panel arrival counters for the cross-tile merge; K + 1 doubles for the collapsed form, below), and so
- * does CONV2D_NCHW (the channels-last copies of image and weights).
+ * does CONV2D_NCHW (the channels-last copies of image and weights).  The partial results are kept per row
+ * and output tile; tiles are 128 or 256 columns wide, whichever the launcher expects to be faster for the
+ * shape, so a row reduction's value depends on the row count of the call up to fp32 summation order.
  * fc_workspace_size reports
  * the bytes a spec needs (0 for the other chains); fc_set_workspace registers a caller-owned DEVICE
  * buffer (256-byte aligned) for the current device, used by later fc_run calls until replaced.

@@ -402,7 +402,7 @@ size_t panel_counter_bytes(long long M) {
     return ((size_t) panels * 4 + 255) / 256 * 256;
 }
 
-// Column-tile width of the GEMM kernels: 256, except that a small plain GEMM (mode 0, 256-wide tiles on at most
+// Column-tile width of the GEMM kernels: 256, except that a small GEMM (modes 0 and 3, 256-wide tiles on at most
 // half of the SM pairs) takes 128-wide tiles where this cost model says so.  Such a call is one round of tiles,
 // so its time is the critical tile's: main loop (of the merging slice, when tiles are cut along K) + epilogue
 // + merge.  Measured, in microseconds: a k-block 0.33 (256 wide) / 0.30 (128 wide; 24 instead of 32 KB), the
@@ -412,7 +412,7 @@ int gemm_tile_width(const TcParams& p, const fc_chain_spec* s, int num_sms) {
     if (p.mode == 1) return kSoftmaxBN;
     if (s->N <= 128) return 128;
     const long long tiles = ((s->M + 255) / 256) * ((s->N + 255) / 256);
-    if (p.mode != 0 || 2 * tiles > num_sms / 2) return 256;
+    if ((p.mode != 0 && p.mode != 3) || 2 * tiles > num_sms / 2) return 256;
     auto cost = [&](int bn) -> double {
         TcPlan tp;
         if (plan_gemm_tc(p, bn, num_sms, &tp) != cudaSuccess) return 1e30;
@@ -428,7 +428,8 @@ size_t softmax_workspace_bytes(long long M, long long N, bool per_half = false) 
     return 2 * panel_counter_bytes(M) + (size_t) M * tiles_n * sizeof(float2) * (per_half ? 2 : 1);
 }
 // fc_run's row softmax may take the two-kernel form, which keeps a pair per row, tile and column half
-size_t reduction_workspace_bytes(bool softmax, long long M, long long N) { return softmax_workspace_bytes(M, N, softmax); }
+// ... and the other row reductions may run with 128-column tiles (twice the tiles): the same room
+size_t reduction_workspace_bytes(bool /*softmax*/, long long M, long long N) { return softmax_workspace_bytes(M, N, true); }
 
 // The part of the caller's workspace behind the row-reduction statistics serves split tiles; without it
 // (no workspace, or a smaller one) the tensor-core kernels simply never split.

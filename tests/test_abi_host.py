@@ -49,6 +49,9 @@ def test_workspace_size_softmax(fc):
     spec = fc.make_spec(wl.CONFIGS["C4"]())
     # 32 arrival + 32 departure panel counters (each padded to 256 B) + 4096 rows x 16 tiles x (max, sum) fp32
     assert fc.fc_workspace_size(spec) == 2 * 256 + 4096 * 16 * 8 * 2      # a (max, sum) pair per row, tile and column half
+    # the other row reductions: the same room, for a pair per row and 128-column tile
+    lse = fc.make_spec(wl.gemm_bias_scale_lse(4096, 4096, 512))
+    assert fc.fc_workspace_size(lse) == 2 * 256 + 4096 * 32 * 8
 
 
 def _status(fc, spec, ins=None, outs=None):

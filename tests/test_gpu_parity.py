@@ -630,6 +630,11 @@ def test_run_host_chunk_pipeline_matches_device_path(fc, orc):
         for a, b in zip(dev_out, host_out):
             if ch.reduce == "global_avgpool":      # pooled sums are combined with atomics: order varies
                 assert torch.allclose(a.cpu(), b, rtol=1e-5, atol=1e-6)
+            elif ch.producer == "gemm_nt" and ch.reduce == "row_logsumexp" and a.dim() == 1:
+                # per-tile (max, sum) pairs are merged per row; the tile width depends on the row count of the
+                # launch (a chunk of rows may take 128-column tiles where the whole tensor takes 256): same
+                # terms, another grouping
+                assert torch.allclose(a.cpu(), b, rtol=2e-6, atol=2e-6), ch.name
             else:
                 assert torch.equal(a.cpu(), b), ch.name
 

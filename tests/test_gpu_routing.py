@@ -60,7 +60,8 @@ def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_softmax(256, 1024, 256)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"   # short contraction
     assert _plan(fc, wl.gemm_softmax(256, 8192, 4096)) == "gemm_tc_mode1_bn256_split_two_pass softmax_rescale"  # 32 tiles per panel (and few enough to be cut along K)
     assert _plan(fc, wl.gemm_softmax(64, 20000, 64)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"
-    assert _plan(fc, wl.gemm_bias_scale_lse(256, 1024, 256)) == "gemm_tc_mode3_bn256"
+    assert _plan(fc, wl.gemm_bias_scale_lse(256, 1024, 256)) == "gemm_tc_mode3_bn128"       # few tiles: as the plain GEMM
+    assert _plan(fc, wl.gemm_bias_scale_lse(2048, 4096, 256)) == "gemm_tc_mode3_bn256"
     assert _plan(fc, wl.linear_row_reduce(96, 512, 256)) == "weight_colsum colsum_finish row_dot"
     assert _plan(fc, wl.mlp(300, (64, 64, 32))) == "mlp_tc"
     conv = wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128)
