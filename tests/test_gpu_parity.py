@@ -366,6 +366,17 @@ def test_gemm_few_tiles_either_tile_width(fc, orc, M, N, K, plan):
     run_and_check(fc, orc, replace(ch, out_dtype="f32"), 9)
 
 
+@pytest.mark.parametrize("M,N,K,plan", [(100, 1000, 4096, "bn128_split"), (300, 1100, 512, "bn128"), (1024, 4096, 1024, "bn256"),
+                                        (64, 4096, 8192, "bn256_split")])
+@pytest.mark.parametrize("store_main", [False, True])
+def test_gemm_row_reduction_few_tiles_either_tile_width(fc, orc, M, N, K, plan, store_main):
+    """The same choice for a row reduction behind the GEMM: per-tile partial results of 128- or 256-column tiles,
+    whole or cut along K, merged per row."""
+    run_and_check(fc, orc, wl.gemm_bias_scale_lse(M, N, K, "var", store_main), 10)
+    assert fc.fc_last_plan() == "gemm_tc_mode3_" + plan
+    run_and_check(fc, orc, wl.linear_row_reduce(M, N, K, "row_max", ops=(("bias_n", 2), ("relu",)), store_main=store_main), 10)
+
+
 def test_gemm_tc_op_lists_fused_and_interpreted(fc, orc):
     """Op lists of the fused shape ([bias|affine] [relu|gelu] [scale] [clamp] [add tensor]) take the
     packed straight-line epilogue; any other order is interpreted op by op.  Both against the oracle."""
