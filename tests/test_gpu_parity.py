@@ -54,6 +54,14 @@ def test_gemm_f32_ragged(fc, orc, M, N, K):
     run_and_check(fc, orc, wl.gemm_bias_relu_f32(M, N, K, "var"), 3)
 
 
+@pytest.mark.parametrize("M,N,K", [(1500, 1100, 260), (1300, 1290, 131), (2048, 1024, 64), (900, 1800, 16), (1500, 1100, 7)])
+def test_gemm_f32_large_register_tiled(fc, orc, M, N, K):
+    """From 96 tiles of 128 x 128 on the strict-fp32 GEMM runs register-tiled (8 x 8 outputs per thread): ragged
+    edges in all three extents, K off the 16-byte grid (scalar loads), N off it (scalar stores)."""
+    run_and_check(fc, orc, wl.gemm_bias_relu_f32(M, N, K, "var"), 5)
+    assert fc.fc_last_plan() == "gemm_f32_big"
+
+
 # ------------------------------------------------------------------ kernel (a): elementwise + logsumexp
 @pytest.mark.parametrize("M,N", [(1, 1), (3, 8), (5, 1000), (7, 4097), (33, 2048), (64, 4096), (9, 12345)])
 def test_elementwise_lse_shapes(fc, orc, M, N):
