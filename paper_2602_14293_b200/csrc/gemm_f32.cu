@@ -110,86 +110,25 @@ __global__ void __launch_bounds__(kGemmThreads) gemm_f32_kernel(const GemmF32Par
     }
 }
 
-// Larger problems (several waves of 32 x 32 tiles): 256 threads x (2 x 2) outputs, slabs of 32 columns through
-// shared memory with the next slab prefetched into registers; more reuse per byte of shared memory than the
-// latency-oriented kernel above, whose small tiles cost 13 % at 1024^3.
-constexpr int kTile = 32;
-constexpr int kSlab = 32;
-
-__global__ void __launch_bounds__(256) gemm_f32_wide_kernel(const GemmF32Params p) {
-    __shared__ float As[kTile][kSlab + 1];
-    __shared__ float Bs[kTile][kSlab + 1];
-    const int tid = threadIdx.x;
-    const int tx = tid & 15, ty = tid >> 4;
-    const int m0 = blockIdx.y * kTile, n0 = blockIdx.x * kTile;
-    // loader mapping: each thread moves 4 consecutive k of one row for A and for B
-    const int lr = tid >> 3, lk = (tid & 7) * 4;
-    const bool vec = ((reinterpret_cast<uintptr_t>(p.A) | reinterpret_cast<uintptr_t>(p.B)) & 15) == 0 && (p.K & 3) == 0;
-
-    auto load4 = [&](const float* base, int row, int row_limit, int k) -> float4 {
-        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row < row_limit) {
-            const float* q = base + (long long) row * p.K + k;
-            if (vec && k + 3 < p.K) {
-                r = __ldg(reinterpret_cast<const float4*>(q));
-            } else {
-                if (k + 0 < p.K) r.x = __ldg(q + 0);
-                if (k + 1 < p.K) r.y = __ldg(q + 1);
-                if (k + 2 < p.K) r.z = __ldg(q + 2);
-                if (k + 3 < p.K) r.w = __ldg(q + 3);
-            }
-        }
-        return r;
-    };
-
-    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-    float4 ra = load4(p.A, m0 + lr, p.M, lk);
-    float4 rb = load4(p.B, n0 + lr, p.N, lk);
-    for (int k0 = 0; k0 < p.K; k0 += kSlab) {
-        As[lr][lk + 0] = ra.x; As[lr][lk + 1] = ra.y; As[lr][lk + 2] = ra.z; As[lr][lk + 3] = ra.w;
-        Bs[lr][lk + 0] = rb.x; Bs[lr][lk + 1] = rb.y; Bs[lr][lk + 2] = rb.z; Bs[lr][lk + 3] = rb.w;
-        __syncthreads();
-        if (k0 + kSlab < p.K) {
-            ra = load4(p.A, m0 + lr, p.M, k0 + kSlab + lk);
-            rb = load4(p.B, n0 + lr, p.N, k0 + kSlab + lk);
-        }
-#pragma unroll
-        for (int k = 0; k < kSlab; ++k) {
-            const float a0 = As[ty * 2][k], a1 = As[ty * 2 + 1][k];
-            const float b0 = Bs[tx * 2][k], b1 = Bs[tx * 2 + 1][k];
-            acc[0][0] = fmaf(a0, b0, acc[0][0]);
-            acc[0][1] = fmaf(a0, b1, acc[0][1]);
-            acc[1][0] = fmaf(a1, b0, acc[1][0]);
-            acc[1][1] = fmaf(a1, b1, acc[1][1]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int m = m0 + ty * 2 + i;
-        if (m >= p.M) continue;
-        float v[2] = {acc[i][0], acc[i][1]};
-        const int n = n0 + tx * 2;
-        apply_ops<2, false>(v, p.ops, m, n, p.N, p.N);
-        if (n < p.N) p.C[(long long) m * p.N + n] = v[0];
-        if (n + 1 < p.N) p.C[(long long) m * p.N + n + 1] = v[1];
-    }
-}
-
 // Large problems (at least 96 tiles of 128 x 128): the classic register-tiled form.  256 threads x (8 x 8) outputs,
 // as 2 x 2 blocks of 4 x 4 so that every shared-memory read is a 16-byte read without bank conflicts (64 FMAs per
 // four reads); K in slabs of 16 through double-buffered shared memory, stored transposed ([k][row]) because both
 // operands are K-major in global memory; the next slab is fetched into registers while this one is multiplied, one
 // block barrier per slab.  Each output is still one fp32 FMA chain over ascending k.
-constexpr int kBigTile = 128, kBigSlab = 16, kBigPitch = kBigTile + 4;
+constexpr int kBigTile = 128, kMidTile = 64, kBigSlab = 16;
 
-__global__ void __launch_bounds__(256, 2) gemm_f32_big_kernel(const GemmF32Params p) {
-    __shared__ __align__(16) float As[2][kBigSlab][kBigPitch];
-    __shared__ __align__(16) float Bs[2][kBigSlab][kBigPitch];
+// TILE = 128: as described; TILE = 64: one 4 x 4 block per thread (16 FMAs per two reads), for problems of fewer
+// large tiles than keep the SMs busy.
+template <int TILE>
+__global__ void __launch_bounds__(256, TILE == 128 ? 2 : 4) gemm_f32_big_kernel(const GemmF32Params p) {
+    constexpr int H = TILE / 64;            // 4 x 4 blocks per thread and dimension; rows lr + 64 h per loader thread
+    constexpr int kPitch = TILE + 4;
+    __shared__ __align__(16) float As[2][kBigSlab][kPitch];
+    __shared__ __align__(16) float Bs[2][kBigSlab][kPitch];
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
-    const int m0 = blockIdx.y * kBigTile, n0 = blockIdx.x * kBigTile;
-    // loader mapping: 4 consecutive k of rows lr and lr + 64, for A and for B
+    const int m0 = blockIdx.y * TILE, n0 = blockIdx.x * TILE;
+    // loader mapping: 4 consecutive k of rows lr (and lr + 64), for A and for B
     const int lr = tid >> 2, lk = (tid & 3) * 4;
     const bool vec = ((reinterpret_cast<uintptr_t>(p.A) | reinterpret_cast<uintptr_t>(p.B)) & 15) == 0 && (p.K & 3) == 0;
 
@@ -208,56 +147,71 @@ __global__ void __launch_bounds__(256, 2) gemm_f32_big_kernel(const GemmF32Param
         }
         return r;
     };
-    auto park = [&](float (*dst)[kBigPitch], int row, const float4& r) {
+    auto park = [&](float (*dst)[kPitch], int row, const float4& r) {
         dst[lk + 0][row] = r.x; dst[lk + 1][row] = r.y; dst[lk + 2][row] = r.z; dst[lk + 3][row] = r.w;
     };
 
-    float acc[8][8];
+    float acc[4 * H][4 * H];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 4 * H; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+        for (int j = 0; j < 4 * H; ++j) acc[i][j] = 0.0f;
 
-    float4 ra0 = load4(p.A, m0 + lr, p.M, lk), ra1 = load4(p.A, m0 + lr + 64, p.M, lk);
-    float4 rb0 = load4(p.B, n0 + lr, p.N, lk), rb1 = load4(p.B, n0 + lr + 64, p.N, lk);
-    park(As[0], lr, ra0); park(As[0], lr + 64, ra1);
-    park(Bs[0], lr, rb0); park(Bs[0], lr + 64, rb1);
+    float4 ra[H], rb[H];
+#pragma unroll
+    for (int h = 0; h < H; ++h) {
+        ra[h] = load4(p.A, m0 + lr + 64 * h, p.M, lk);
+        rb[h] = load4(p.B, n0 + lr + 64 * h, p.N, lk);
+    }
+#pragma unroll
+    for (int h = 0; h < H; ++h) {
+        park(As[0], lr + 64 * h, ra[h]);
+        park(Bs[0], lr + 64 * h, rb[h]);
+    }
     __syncthreads();
     int buf = 0;
     for (int k0 = 0; k0 < p.K; k0 += kBigSlab) {
         const bool more = k0 + kBigSlab < p.K;
         if (more) {
-            ra0 = load4(p.A, m0 + lr, p.M, k0 + kBigSlab + lk); ra1 = load4(p.A, m0 + lr + 64, p.M, k0 + kBigSlab + lk);
-            rb0 = load4(p.B, n0 + lr, p.N, k0 + kBigSlab + lk); rb1 = load4(p.B, n0 + lr + 64, p.N, k0 + kBigSlab + lk);
+#pragma unroll
+            for (int h = 0; h < H; ++h) {
+                ra[h] = load4(p.A, m0 + lr + 64 * h, p.M, k0 + kBigSlab + lk);
+                rb[h] = load4(p.B, n0 + lr + 64 * h, p.N, k0 + kBigSlab + lk);
+            }
         }
 #pragma unroll
         for (int k = 0; k < kBigSlab; ++k) {
-            const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
-            const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][k][64 + ty * 4]);
-            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
-            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][k][64 + tx * 4]);
-            const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-            const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+            float a[4 * H], b[4 * H];
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int h = 0; h < H; ++h) {
+                const float4 av = *reinterpret_cast<const float4*>(&As[buf][k][64 * h + ty * 4]);
+                const float4 bv = *reinterpret_cast<const float4*>(&Bs[buf][k][64 * h + tx * 4]);
+                a[4 * h] = av.x; a[4 * h + 1] = av.y; a[4 * h + 2] = av.z; a[4 * h + 3] = av.w;
+                b[4 * h] = bv.x; b[4 * h + 1] = bv.y; b[4 * h + 2] = bv.z; b[4 * h + 3] = bv.w;
+            }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            for (int i = 0; i < 4 * H; ++i)
+#pragma unroll
+                for (int j = 0; j < 4 * H; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
         if (more) {
             // the other buffer was last read one slab ago, before the barrier that ended that slab
-            park(As[buf ^ 1], lr, ra0); park(As[buf ^ 1], lr + 64, ra1);
-            park(Bs[buf ^ 1], lr, rb0); park(Bs[buf ^ 1], lr + 64, rb1);
+#pragma unroll
+            for (int h = 0; h < H; ++h) {
+                park(As[buf ^ 1], lr + 64 * h, ra[h]);
+                park(Bs[buf ^ 1], lr + 64 * h, rb[h]);
+            }
             __syncthreads();
             buf ^= 1;
         }
     }
     const bool c_vec = (reinterpret_cast<uintptr_t>(p.C) & 15) == 0 && (p.N & 3) == 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int m = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+    for (int i = 0; i < 4 * H; ++i) {
+        const int m = m0 + 64 * (i >> 2) + ty * 4 + (i & 3);
         if (m >= p.M) continue;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < H; ++h) {
             const int n = n0 + h * 64 + tx * 4;
             if (n >= p.N) continue;
             float v[4] = {acc[i][4 * h], acc[i][4 * h + 1], acc[i][4 * h + 2], acc[i][4 * h + 3]};
@@ -286,19 +240,22 @@ cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* la
         raised[dev] = true;
     }
     const long long big_tiles = (long long) ((p.M + kBigTile - 1) / kBigTile) * ((p.N + kBigTile - 1) / kBigTile);
-    // (1024^3, 64 tiles on 148 SMs: 137 us against 114 us with the 32 x 32 tiles; 4096 x 512 x 1024, 128 tiles: 137 against 219)
-    if (big_tiles >= 96 && (p.M + kBigTile - 1) / kBigTile <= 65535) {
+    // (1024^3 is 64 such tiles on 148 SMs: 137 us, against 77 us with 64 x 64 tiles)
+    // (and not where an extent of at most 64 would leave half of every such tile empty)
+    if (big_tiles >= 96 && p.M > kMidTile && p.N > kMidTile && (p.M + kBigTile - 1) / kBigTile <= 65535) {
         dim3 big((p.N + kBigTile - 1) / kBigTile, (p.M + kBigTile - 1) / kBigTile);
         note_kernel("gemm_f32_big");
-        gemm_f32_big_kernel<<<big, 256, 0, stream>>>(p);
+        gemm_f32_big_kernel<kBigTile><<<big, 256, 0, stream>>>(p);
         *launches += 1;
         return cudaGetLastError();
     }
-    const long long wide_tiles = (long long) ((p.M + kTile - 1) / kTile) * ((p.N + kTile - 1) / kTile);
-    if (wide_tiles >= 512 && (p.M + kTile - 1) / kTile <= 65535) {
-        dim3 wide((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile);
-        note_kernel("gemm_f32_wide");
-        gemm_f32_wide_kernel<<<wide, 256, 0, stream>>>(p);
+    // In between, from 512 tiles of 32 x 32 on, 64 x 64 tiles (768^3: 39 us, 1024^3: 77 us, 128 x 4096 x 4096: 191 us).
+    // Below that the latency-oriented kernel wins (512^3: 20 against 27 us; 128 x 1024 x 1024: 21 against 50).
+    const long long small_tiles = (long long) ((p.M + 31) / 32) * ((p.N + 31) / 32);
+    if (small_tiles >= 512 && (p.M + kMidTile - 1) / kMidTile <= 65535) {
+        dim3 mid((p.N + kMidTile - 1) / kMidTile, (p.M + kMidTile - 1) / kMidTile);
+        note_kernel("gemm_f32_mid");
+        gemm_f32_big_kernel<kMidTile><<<mid, 256, 0, stream>>>(p);
         *launches += 1;
         return cudaGetLastError();
     }

@@ -54,12 +54,15 @@ def test_gemm_f32_ragged(fc, orc, M, N, K):
     run_and_check(fc, orc, wl.gemm_bias_relu_f32(M, N, K, "var"), 3)
 
 
-@pytest.mark.parametrize("M,N,K", [(1500, 1100, 260), (1300, 1290, 131), (2048, 1024, 64), (900, 1800, 16), (1500, 1100, 7)])
-def test_gemm_f32_large_register_tiled(fc, orc, M, N, K):
-    """From 96 tiles of 128 x 128 on the strict-fp32 GEMM runs register-tiled (8 x 8 outputs per thread): ragged
-    edges in all three extents, K off the 16-byte grid (scalar loads), N off it (scalar stores)."""
+@pytest.mark.parametrize("M,N,K,plan", [(1500, 1100, 260, "big"), (1300, 1290, 131, "big"), (2048, 1024, 64, "big"), (900, 1800, 16, "big"),
+                                        (1500, 1100, 7, "big"), (700, 900, 260, "mid"), (1025, 600, 131, "mid"), (520, 1030, 7, "mid"),
+                                        (33, 16300, 72, "mid")])
+def test_gemm_f32_large_register_tiled(fc, orc, M, N, K, plan):
+    """Larger strict-fp32 GEMMs run register-tiled: 128 x 128 tiles (8 x 8 outputs per thread) from 96 such tiles
+    on, 64 x 64 tiles (4 x 4) below.  Ragged edges in all three extents, K off the 16-byte grid (scalar loads),
+    N off it (scalar stores)."""
     run_and_check(fc, orc, wl.gemm_bias_relu_f32(M, N, K, "var"), 5)
-    assert fc.fc_last_plan() == "gemm_f32_big"
+    assert fc.fc_last_plan() == "gemm_f32_" + plan
 
 
 # ------------------------------------------------------------------ kernel (a): elementwise + logsumexp

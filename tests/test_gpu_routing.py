@@ -47,7 +47,7 @@ def test_elementwise_routing(fc):
 
 def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_bias_relu_f32(256, 256, 256)) == "gemm_f32"
-    assert _plan(fc, wl.gemm_bias_relu_f32(1024, 1024, 64)) == "gemm_f32_wide"
+    assert _plan(fc, wl.gemm_bias_relu_f32(1024, 1024, 64)) == "gemm_f32_mid"
     assert _plan(fc, wl.gemm_bias_relu_f32(2048, 1024, 64)) == "gemm_f32_big"
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(4096, 4096, 256)) == "gemm_tc_mode0_bn256"
     # few tiles: 128-wide ones where the cost model prefers twice the tiles with half the epilogue each ...
