@@ -252,6 +252,7 @@ EXTRA = {
     "F6": lambda **kw: conv_nchw(conv_bias_relu_avgpool(**kw)),
     "F7": lambda **kw: scale_add_softmax(**kw),
     "F8": lambda **kw: gemm_softmax(**{"M": 2048, "N": 50264, "K": 4096, **kw}),   # a vocabulary-wide softmax: two kernels
+    "F9": lambda **kw: gemm_bias_relu_f32(**{"M": 2048, "N": 2048, "K": 2048, **kw}),   # C1's chain at a size the plain ALUs bound
 }
 ALL = {**CONFIGS, **EXTRA}
 
