@@ -9,11 +9,22 @@ quoted on); `--workload C1|C3|C4|C5` selects another.  Rank 0 prints ONE JSON li
 (launched by torch.distributed.run) every rank runs its own batch (the chains' rows / images are
 independent problems: weak scaling, no data-path collective); the time is the max over ranks.
 
-`value` times fc_run with inputs resident in HBM (CUDA events on the launch stream); `e2e` times
-fc_run_host with pinned HOST buffers, copies inside the timed region.  `roofline` relates the
-kernel's algorithmic bytes or FLOPs per launch to the measured peak of this machine's B200s.
-`cpu_baseline` is the CPU oracle, as it stands, on a bounded sample of the same workload.
-`--impl reference` times that oracle as the reference arm.
+`value` times fc_run with inputs resident in HBM (CUDA events on the launch stream): the timed region
+of exactly `--steps` steps is taken five times and the median is reported (`ms_per_step_repeats`,
+`ms_per_step_best` beside it).  `e2e` times fc_run_host with pinned HOST buffers, copies inside the
+timed region.  `roofline` relates the kernel's algorithmic bytes or FLOPs per launch to the measured
+peak of this machine's B200s (`frac`) and to the nominal peak the targets are stated against
+(`frac_nominal`: 8 TB/s, 2250 TFLOP/s dense bf16).  `cpu_baseline` is the CPU oracle, as it stands, on a
+bounded sample of the same workload.  `--impl reference` times that oracle as the reference arm.
+
+`per_config` (rank 0 of a one-GPU run; `--no-per-config` leaves it out) holds one entry for each of the
+five benchmark configurations C1..C5, each timed by the same protocol: fc_run enqueued back to back on one
+stream, the number of calls per timed region chosen so that the region lasts at least 20 ms, five such
+regions, median and best; configurations whose tensors fit in L2 (C1, C4, C5) are timed with an
+L2-evicting write before every call (one event pair per call) and, beside it, back to back (`warm`).
+Every entry has its own roofline fractions, its own clock sample over its own timed loop, the host cost
+of an fc_run call, the unfused eager sequence on the same tensors, and the oracle's verdict on a sample
+of its outputs.
 """
 from __future__ import annotations
 
@@ -50,18 +61,37 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback (earlier measurement on this pool)"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of each config's kernel, from the ncu
-# captures summarised under profiles/ (full config sizes; part of each output is still dirty in L2
-# when the kernel ends, so writes can read below the algorithmic output bytes).
-NCU_TRAFFIC_BYTES = {"C1": 543232, "C2": 268533248 + 98800896, "C3": 230077440 + 115409408,
-                     "C4": 67290112 + 9656320, "C5": 52669952 + 186624, "F1": 101696256 + 5212160,
-                     "F2": 134259968 + 4772096,   # F2: the weight pass, the dominant kernel of that workload
-                     "F3": 78334720 + 1789696, "F4": 34311424, "F5": 74555136 + 96400128}
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # what the targets are stated against (context for `frac`)
+TARGET_FRAC_NOMINAL = {"hbm": 0.80, "tensor": 0.60}          # memory-bound chain >= 80 % of HBM peak, GEMM / conv >= 60 % of bf16 peak
+
+
+def load_traffic_table():
+    """DRAM bytes per launch (read, write) of each profiled workload's dominant kernel, from the table in
+    profiles/dram_traffic.md, which the ncu summaries beside it are the sources of: a re-capture updates that
+    one file.  Rows: | workload | kernel | dram read bytes | dram write bytes | summary file |"""
+    table = {}
+    path = os.path.join(ROOT, "profiles", "dram_traffic.md")
+    try:
+        with open(path) as f:
+            for line in f:
+                cells = [c.strip() for c in line.strip().strip("|").split("|")]
+                if len(cells) >= 4 and cells[2].isdigit() and cells[3].isdigit():
+                    table[cells[0]] = int(cells[2]) + int(cells[3])
+    except OSError:
+        pass
+    return table
+
+
+_TRAFFIC = None
 
 
 def load_traffic(workload: str, full_size: bool):
-    """DRAM bytes per launch from the committed ncu capture of this workload's kernel (full size only)."""
-    return NCU_TRAFFIC_BYTES.get(workload) if full_size else None
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of this workload's
+    kernel (captures are of the full config sizes; None for a resized run or an unprofiled workload)."""
+    global _TRAFFIC
+    if _TRAFFIC is None:
+        _TRAFFIC = load_traffic_table()
+    return _TRAFFIC.get(workload) if full_size else None
 
 
 # ------------------------------------------------------------------------------ units per workload
@@ -351,6 +381,160 @@ def reference_arm(args):
     return 0
 
 
+# ------------------------------------------------------------------------------ timing protocol
+MIN_REGION_MS = 20.0
+REPEATS = 5
+
+
+def roofline_of(ch, workload, units_per_step, bound, ms, peaks, peaks_src, full_size, long_region=False):
+    """Roofline object of one launch: achieved units / s against the measured peak (`frac`) and against the nominal
+    peak the targets are stated against (`frac_nominal`)."""
+    frac_sustained = None
+    if bound == "hbm":
+        peak, peak_unit, nominal = peaks["hbm_gbs"], "GB/s", NOMINAL_PEAKS["hbm_gbs"]
+        peak_note = f"HBM copy bandwidth, {peaks_src}"
+    elif bound == "tensor":
+        mult = 2.0 if ch.in_dtype == "f8e4m3" else 1.0   # no fp8 measurement on this pool: the measured bf16 peak times the nominal fp8 : bf16 ratio
+        peak = mult * (peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"])
+        peak_unit, nominal = "TFLOP/s", mult * NOMINAL_PEAKS["bf16_tflops"]
+        peak_note = f"cuBLAS bf16 {'sustained' if long_region else 'burst'}, {peaks_src}" + (" x 2 (nominal fp8 : bf16 ratio)" if mult > 1 else "")
+        frac_sustained = units_per_step / (ms * 1e-3) / (mult * peaks["bf16_tflops_sustained"])
+    else:
+        peak, peak_unit = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
+        nominal = peak
+        peak_note = "fp32 FMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived)"
+    achieved = units_per_step / (ms * 1e-3)
+    r = {"bound": bound, "achieved": achieved, "peak": peak, "unit": peak_unit, "frac": achieved / peak,
+         "frac_measured": achieved / peak, "frac_nominal": achieved / nominal, "peak_nominal": nominal,
+         "traffic": load_traffic(workload, full_size), "peak_source": peak_note,
+         "algorithmic_units_per_launch": units_per_step, "kernel_ms": ms}
+    if frac_sustained is not None:
+        r["frac_of_sustained_peak"] = frac_sustained
+    if bound in TARGET_FRAC_NOMINAL:
+        r["target_frac_nominal"] = TARGET_FRAC_NOMINAL[bound]
+        r["target_met"] = bool(r["frac_nominal"] >= TARGET_FRAC_NOMINAL[bound])
+    return r
+
+
+def timed_regions(step, flush, n, repeats, barrier=None, max_over_ranks=None):
+    """`repeats` timed regions of `n` calls each, CUDA events on the current stream, a synchronize (and the ranks'
+    barrier) on both sides of every region.  Without `flush`: one event pair around the n back-to-back calls.
+    With `flush`: an L2-evicting write before every call and one event pair per call (the region's time is the
+    sum).  Returns the per-call milliseconds of every region (max over ranks)."""
+    import torch
+    sync = barrier if barrier is not None else torch.cuda.synchronize
+    out = []
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n if flush else 1)]
+    for _ in range(repeats):
+        sync()
+        if flush is None:
+            a, b = evs[0]
+            a.record()
+            for _ in range(n):
+                step()
+            b.record()
+            sync()
+            ms = a.elapsed_time(b)
+        else:
+            for a, b in evs:
+                flush()
+                a.record()
+                step()
+                b.record()
+            sync()
+            ms = sum(a.elapsed_time(b) for a, b in evs)
+        if max_over_ranks is not None:
+            ms = max_over_ranks(ms)
+        out.append(ms / n)
+    return out
+
+
+def calls_for_region(step, flush, min_ms=MIN_REGION_MS):
+    """Number of calls that make a timed region last at least `min_ms`, from a short trial."""
+    import math
+    trial = timed_regions(step, flush, 10, 1)[0]
+    return max(10, int(math.ceil(min_ms / max(trial, 1e-4))))
+
+
+def host_cost_us(step, kernel_ms, calls):
+    """Host time of one fc_run call: the host clock around batches of un-synchronised calls (batches small enough
+    that the launch queue never fills, the stream drained after each), divided by the number of calls."""
+    import torch
+    batch = 256
+    total, done = 0.0, 0
+    torch.cuda.synchronize()
+    while done < calls:
+        t0 = time.perf_counter()
+        for _ in range(batch):
+            step()
+        total += time.perf_counter() - t0
+        torch.cuda.synchronize()
+        done += batch
+    return total / done * 1e6, done
+
+
+def config_entry(fc, binding, key, ch, ins, sampler, flush_buf, peaks, peaks_src, with_eager, oracle_s):
+    """One per_config entry: the timing protocol, roofline, clocks, host cost, eager context, oracle parity."""
+    import torch
+    metric, unit, units_per_step, bound = units(ch)
+    dev_in = [fc.to_device(a) for a in ins]
+    outs = binding.output_tensors(ch, "cuda")
+    spec = fc.make_spec(ch)
+    binding.ensure_workspace(spec)
+    cold = wl.input_bytes(ch) <= L2_BYTES
+    flush = (lambda: flush_buf.zero_()) if cold else None
+    step = fc.PreparedRun(spec, dev_in, outs).run
+    for _ in range(3):
+        if flush:
+            flush()
+        step()
+    torch.cuda.synchronize()
+    n = calls_for_region(step, flush)
+    t0 = time.perf_counter()
+    reps = timed_regions(step, flush, n, REPEATS)
+    t1 = time.perf_counter()
+    fc.fc_get_async_status()
+    ms, best = statistics.median(reps), min(reps)
+    ent = {"workload": ch.name, "ms": ms, "ms_best": best, "ms_repeats": reps, "calls_per_region": n, "repeats": REPEATS,
+           "region_ms": ms * n, "value": units_per_step / (ms * 1e-3), "value_best": units_per_step / (best * 1e-3), "unit": unit,
+           "l2": "L2 flushed (252 MiB write) before every timed call, one event pair per call" if cold else "tensors larger than L2, calls back to back",
+           "roofline": roofline_of(ch, key, units_per_step, bound, ms, peaks, peaks_src, True),
+           "clocks": sampler.summary(t0, t1, "sampled during this config's timed regions")}
+    if cold:
+        nw = calls_for_region(step, None)
+        warm = timed_regions(step, None, nw, REPEATS)
+        ent["warm"] = {"ms": statistics.median(warm), "ms_best": min(warm), "calls_per_region": nw,
+                       "note": "same calls back to back, tensors resident in L2"}
+    us, calls = host_cost_us(step, ms, 10240 if ms < 0.05 else 2048)
+    ent["host_us_per_call"] = us
+    ent["host_calls"] = calls
+    # re-poisoned outputs, one more call, checked against the oracle on a sample
+    for t in outs:
+        t.fill_(float("nan"))
+    step()
+    fc.fc_get_async_status()
+    if with_eager:
+        fn = eager_fn(ch, dev_in)
+        if fn is not None:
+            torch.backends.cuda.matmul.allow_tf32 = False
+            torch.backends.cudnn.allow_tf32 = False
+            for _ in range(3):
+                if flush:
+                    flush()
+                fn()
+            ne = calls_for_region(fn, flush)
+            er = timed_regions(fn, flush, ne, 3)
+            ent["eager_ms"] = statistics.median(er)
+            ent["faster_than_eager"] = bool(ms < ent["eager_ms"])
+    if oracle_s > 0:
+        leg = cpu_baseline_leg(ch, ins, outs, target_s=oracle_s)
+        ent["parity_on_sample"] = dict(leg["parity_on_sample"], sample=leg["sample"], oracle_seconds=leg["seconds"])
+        ent["cpu_oracle"] = {"value": leg["value"], "unit": leg["unit"], "cores": leg["cores"]}
+    r = ent["roofline"]
+    ent["target_met"] = bool(r["target_met"] if "target_met" in r else ent.get("faster_than_eager", False))
+    return ent
+
+
 # ------------------------------------------------------------------------------ main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -361,7 +545,9 @@ def main():
     ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-eager", action="store_true")
-    ap.add_argument("--all-configs", action="store_true", help="also time the other configurations and the extra workloads (context)")
+    ap.add_argument("--no-per-config", action="store_true", help="leave out the per_config entries of C1..C5 (profiler captures)")
+    ap.add_argument("--single-region", action="store_true", help="time the --steps region once instead of five times (profiler captures)")
+    ap.add_argument("--all-configs", action="store_true", help="also time the extra workloads F1.. and the network N1 (context)")
     ap.add_argument("--rows", type=int, default=0, help="override M (or the conv batch): a smaller case of the same kernel for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -389,58 +575,38 @@ def main():
     spec = fc.make_spec(ch)
     binding.ensure_workspace(spec)
     in_bytes = wl.input_bytes(ch)
-    flush_buf = None
-    flush = None
-    if in_bytes <= L2_BYTES:
-        flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
-        flush = lambda: flush_buf.zero_()  # noqa: E731
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+    flush = (lambda: flush_buf.zero_()) if in_bytes <= L2_BYTES else None
 
     prepared = fc.PreparedRun(spec, dev_in, outs)     # arguments marshalled once; a step is one fc_run C call
     step = prepared.run
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    launches0 = fc.fc_launch_count()
     for _ in range(args.warmup):
         if flush:
             flush()
         step()
     barrier()
+    regions = 1 if args.single_region else REPEATS
     launches1 = fc.fc_launch_count()
     t_wall0 = time.perf_counter()
-    if flush is None:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            step()
-        e1.record()
-        barrier()
-        ms_total = e0.elapsed_time(e1)
-    else:
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-        for a, b in evs:
-            flush()
-            a.record()
-            step()
-            b.record()
-        barrier()
-        ms_total = sum(a.elapsed_time(b) for a, b in evs)
+    reps = timed_regions(step, flush, args.steps, regions, barrier, max_over_ranks)   # each region: EXACTLY --steps steps
     t_wall1 = time.perf_counter()
-    launches = fc.fc_launch_count() - launches1
+    launches = (fc.fc_launch_count() - launches1) // regions
     fc.fc_get_async_status()
-    ms_total = max_over_ranks(ms_total)
-    ms_per_step = ms_total / args.steps
+    ms_per_step = statistics.median(reps)
     value = rk.aggregate(units_per_step, ms_per_step)
 
-    clocks = sampler.summary(t_wall0, t_wall1, "sampled during the timed region")
+    clocks = sampler.summary(t_wall0, t_wall1, "sampled during the timed regions")
     if clocks.get("samples", 0) < 3:
-        # the timed region was shorter than a few sampling periods: sample a longer loop of the same kernel
+        # the timed regions were shorter than a few sampling periods: sample a longer loop of the same kernel
         t0 = time.perf_counter()
         while time.perf_counter() - t0 < 0.4:
             for _ in range(20):
                 step()
             torch.cuda.synchronize()
-        clocks = sampler.summary(t0, time.perf_counter(), "timed region too short to sample; taken over a 0.4 s loop of the same kernel right after it")
+        clocks = sampler.summary(t0, time.perf_counter(), "timed regions too short to sample; taken over a 0.4 s loop of the same kernel right after them")
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) ----
     host_in = [t.cpu().pin_memory() for t in dev_in]
@@ -461,33 +627,20 @@ def main():
     d2h = sum(t.numel() * t.element_size() for t in host_out)
     e2e = {"value": rk.aggregate(units_per_step, e2e_ms), "unit": unit, "ms_per_step": e2e_ms, "steps": e2e_steps,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    del host_in, host_out, staging
 
     # ---- roofline of the (single) kernel of this workload ----
-    if bound == "hbm":
-        peak, peak_unit = peaks["hbm_gbs"], "GB/s"
-        peak_note = f"HBM copy bandwidth, {peaks_src}"
-    elif bound == "tensor":
-        long_region = ms_total > 1000.0
-        peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
-        peak_unit = "TFLOP/s"
-        peak_note = f"cuBLAS bf16 {'sustained' if long_region else 'burst'}, {peaks_src}"
-        if ch.in_dtype == "f8e4m3":
-            peak *= 2.0   # no fp8 measurement on this machine: the measured bf16 peak times the nominal fp8 : bf16 ratio
-            peak_note += " x 2 (nominal fp8 : bf16 ratio)"
-    else:
-        peak, peak_unit = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
-        peak_note = "fp32 FMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived)"
-    achieved = units_per_step / (ms_per_step * 1e-3)
-    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": peak_unit, "frac": achieved / peak,
-                "traffic": load_traffic(args.workload, args.rows <= 0), "peak_source": peak_note,
-                "algorithmic_units_per_launch": units_per_step, "kernel_ms": ms_per_step}
+    roofline = roofline_of(ch, args.workload, units_per_step, bound, ms_per_step, peaks, peaks_src, args.rows <= 0,
+                           long_region=ms_per_step * args.steps > 1000.0)
 
     line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_per_step, "ms_per_step_best": min(reps), "ms_per_step_repeats": reps, "timed_regions": regions,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": dtype_of(ch), "data": "synthetic",
             "config": {"workload": f"{args.workload}: {ch.name}", "shape": {k: getattr(ch, k) for k in ("M", "N", "K", "batch", "H", "W", "Cin", "Cout") if getattr(ch, k)},
                        "ops": [o[0] for o in ch.ops], "reduce": ch.reduce,
                        "l2": "inputs larger than L2, no flush" if flush is None else "L2 flushed (252 MiB write) before every timed step",
+                       "timing": f"{regions} regions of exactly {args.steps} steps each, median reported",
                        "parallelism": f"independent batches per GPU x{world}"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
 
@@ -500,18 +653,31 @@ def main():
             line["eager"] = {"ms_per_step": ems, "value": units_per_step / (ems * 1e-3), "unit": unit,
                              "note": "unfused PyTorch eager sequence on the same GPU and tensors (context)"}
 
+    per = {}
+    if rank == 0 and world == 1 and not args.no_per_config:
+        # the five benchmark configurations, each by the same protocol (see the module docstring)
+        for key in sorted(wl.CONFIGS):
+            c2 = wl.CONFIGS[key]()
+            i2 = ins if (key == args.workload and args.rows <= 0) else wl.make_inputs(c2, 0)
+            per[key] = config_entry(fc, binding, key, c2, i2, sampler, flush_buf, peaks, peaks_src, not args.no_eager,
+                                    0.0 if args.no_cpu_baseline else 3.0)
+            del i2
+            torch.cuda.empty_cache()
+        line["targets"] = {"statement": "memory-bound chain >= 80 % of nominal HBM peak (8 TB/s); GEMM / conv chains >= 60 % of nominal dense "
+                                        "bf16 peak (2250 TFLOP/s); every config within the oracle's tolerances and faster than eager",
+                           "met": {k: v["target_met"] for k, v in per.items()},
+                           "faster_than_eager": {k: v.get("faster_than_eager") for k, v in per.items()},
+                           "parity": {k: v.get("parity_on_sample", {}).get("ok") for k, v in per.items()}}
+
     if rank == 0 and args.all_configs:
-        per = {}
         for key in sorted(wl.ALL):
-            if key == args.workload:
+            if key == args.workload or key in per:
                 continue
             c2 = wl.ALL[key]()
             i2 = [fc.to_device(a) for a in wl.make_inputs(c2, 0)]
             o2 = binding.output_tensors(c2, "cuda")
             s2 = fc.make_spec(c2)
             binding.ensure_workspace(s2)
-            if flush_buf is None:
-                flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
             fl = (lambda: flush_buf.zero_()) if wl.input_bytes(c2) <= L2_BYTES else None
             ms = time_loop(fc.PreparedRun(s2, i2, o2).run, 50, 5, fl)
             _, u2, n2, b2 = units(c2)
@@ -524,6 +690,7 @@ def main():
             per[key] = ent
             del i2, o2
         per["N1"] = network_entry(fc, binding, lambda: flush_buf.zero_(), not args.no_eager)
+    if per:
         line["per_config"] = per
 
     sampler.stop()

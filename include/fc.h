@@ -24,7 +24,10 @@
  *
  * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
  * allocates device memory and never synchronises; it enqueues at most two memsets and one to four
- * kernels (a GEMM + ROW_SOFTMAX over more than 16384 columns: the GEMM kernel and a rescaling pass) on the given stream and returns.  Inputs are read-only; outputs are fully overwritten.
+ * kernels on the given stream and returns (two kernels: a convolution behind the kernel that zeroes
+ * its pooled output, or a wide GEMM + ROW_SOFTMAX as the GEMM kernel and a rescaling pass; three: the
+ * collapsed linear layer; four: CONV2D_NCHW with its two layout kernels).  Inputs are read-only;
+ * outputs are fully overwritten.
  *
  * Launches.  Kernels are launched with programmatic stream serialization and wait, before their first access to
  * global memory, for everything in front of them in the stream: the order the caller sees is the stream's,
@@ -50,7 +53,10 @@
  * outside the supported patterns return FC_ERR_UNSUPPORTED; there is no CPU fallback and no other
  * backend.  A device that is not compute capability 10.x returns FC_ERR_ARCH.  Device-side waits
  * are bounded; if one expires the kernel records FC_ERR_TIMEOUT in a device status word, skips its
- * remaining stores and exits; fc_get_async_status reports it.
+ * remaining stores and exits; fc_get_async_status reports it.  A launch that gave up may leave its
+ * cross-tile counters (in the workspace) at a non-zero count, and only fc_get_async_status puts them
+ * back: after any fc_run that can have timed out, read the status before the next fc_run on that
+ * device, or the next chain that uses the workspace may skip its waits and store wrong values.
  *
  * Testing aid.  With the environment variable FC_INJECT_PANEL_STALL=1, GEMM_NT + ROW_SOFTMAX launches
  * make their cross-tile wait expect an arrival that never comes: the bounded wait expires (about two
@@ -251,8 +257,15 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
  * fc_run (device pointers); nothing is allocated or freed, here or in any library this calls.
  *
  * Limits and rules.  Only GEMM_NT with reduce == FC_RED_ROW_SOFTMAX; other chains return
- * FC_ERR_UNSUPPORTED.  A spec whose fc_workspace_size exceeds FC_STATIC_SCRATCH_BYTES returns
- * FC_ERR_WORKSPACE ("needs N bytes, the built-in scratch holds M").  The first call on each device
+ * FC_ERR_UNSUPPORTED.  The scratch a call needs is
+ *     2 * roundup(ceil(M / 128) * 4, 256)  +  M * ceil(N / 256) * 8   bytes
+ * (arrival and departure counters per 128-row panel, then one (max, sum) pair per row and 256-column
+ * tile).  That is about half of what fc_workspace_size reports for the same spec, because fc_run
+ * reserves room for its two-kernel form as well; a spec that needs more than FC_STATIC_SCRATCH_BYTES
+ * returns FC_ERR_WORKSPACE ("needs N bytes, the built-in scratch holds M").  Rows wider than 16384
+ * columns (64 tiles), or with more tiles than CTA pairs are resident on the device, would need that
+ * two-kernel form and return FC_ERR_UNSUPPORTED ("use fc_run").  All three checks come before the
+ * device is touched.  The first call on each device
  * looks up the array's device address (with that device current); make that first call outside
  * any stream capture.  All calls on a device share the one array, which keeps whatever the last
  * call left in it: the counters are cleared on the stream before each launch, and two calls that

@@ -1034,9 +1034,14 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
                                                    fc_tensor* outputs, int n_outputs, void* cuda_stream) {
     Plan plan;
     fc_status st;
+    t_plan[0] = 0;
     if ((st = validate_spec(spec, &plan))) return st;
     if (plan.kind != Plan::TC_SOFTMAX) return fail(FC_ERR_UNSUPPORTED, "the built-in scratch serves GEMM_NT + ROW_SOFTMAX chains only");
     if ((st = validate_tensors(spec, plan, inputs, n_inputs, outputs, n_outputs))) return st;
+    // size rules first, before anything touches the device
+    const int tiles_n = (int) ((spec->N + kSoftmaxBN - 1) / kSoftmaxBN);
+    if (tiles_n > kSoftmaxOnePassTiles)
+        return fail(FC_ERR_UNSUPPORTED, "rows wider than %d columns take two kernels: use fc_run", kSoftmaxOnePassTiles * kSoftmaxBN);
     const size_t need = softmax_workspace_bytes(spec->M, spec->N);
     if (need > FC_STATIC_SCRATCH_BYTES)
         return fail(FC_ERR_WORKSPACE, "this chain needs %zu bytes of scratch, the built-in scratch holds %u", need, (unsigned) FC_STATIC_SCRATCH_BYTES);
@@ -1055,8 +1060,6 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
         }
         scratch = g_static_scratch_ptr[ordinal];
     }
-    if ((spec->N + kSoftmaxBN - 1) / kSoftmaxBN > kSoftmaxOnePassTiles)
-        return fail(FC_ERR_UNSUPPORTED, "rows wider than %d columns take two kernels: use fc_run", kSoftmaxOnePassTiles * kSoftmaxBN);
     cudaStream_t stream = (cudaStream_t) cuda_stream;
     TcParams p;
     memset(&p, 0, sizeof(p));
@@ -1071,9 +1074,17 @@ extern "C" fc_status fc_run_softmax_static_scratch(const fc_chain_spec* spec, co
     p.counters = (unsigned int*) scratch;
     p.departed = (unsigned int*) ((char*) scratch + counters);
     p.stats = (float2*) ((char*) scratch + 2 * counters);
+    cudaError_t e;
+    {
+        // the same guard as fc_run: every tile of a row panel must be resident at once, so a panel may not have
+        // more tiles than CTA pairs take part on this device (fewer SMs, a partitioned context)
+        TcPlan tp;
+        if ((e = plan_gemm_tc(p, kSoftmaxBN, dev->num_sms, &tp)) != cudaSuccess) return cuda_fail(e, "planning");
+        if (tiles_n > tp.pairs)
+            return fail(FC_ERR_UNSUPPORTED, "a row panel has %d tiles but only %d CTA pairs are resident on this device: use fc_run", tiles_n, tp.pairs);
+    }
     // the array keeps the previous call's contents: the arrival and departure counters must start at zero
-    cudaError_t e = cudaMemsetAsync(p.counters, 0, 2 * counters, stream);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    if ((e = cudaMemsetAsync(p.counters, 0, 2 * counters, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     CUtensorMap tmA, tmB;
     if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
     if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, kSoftmaxBN / 2, spec->in_dtype))) return st;

@@ -4,9 +4,9 @@ fc_run_softmax_static_scratch exists for callers that are handed tensors but can
 workspace themselves (plug-ins without a memory pool, latency-critical loops where cudaMalloc is
 off limits, processes whose device memory is reserved up front): it runs the GEMM + row-softmax kernel with
 scratch from a fixed array inside the library.  Here it is called through the C ABI twice in a row,
-on different inputs, and each result is compared with what fc_run (caller-provided workspace)
-writes for the same inputs, within the bf16 tolerance of the parity tests.  The second call also
-shows that what the first call left in the shared array does no harm.  This file sorts last so that
+on different inputs, and each result is compared with the fp64 CPU oracle of the chain and with what
+fc_run (caller-provided workspace) writes for the same inputs, both within the bf16 tolerance of the
+parity tests.  The second call also shows that what the first call left in the shared array does no harm.  This file sorts last so that
 a run which stops at the first failure has already run every other test.
 """
 import numpy as np
@@ -27,10 +27,13 @@ def test_static_scratch_matches_fc_run_twice_in_a_row():
     assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
     torch.cuda.set_device(0)
 
+    import oracle
     cases = [(wl.gemm_softmax(384, 1024, 256, "var"), 7), (wl.gemm_softmax(300, 2000, 136, "var"), 8)]
     for ch, seed in cases:
         spec = fc.make_spec(ch)
-        ins = [fc.to_device(a) for a in wl.make_inputs(ch, seed)]
+        host_ins = wl.make_inputs(ch, seed)
+        ref = oracle.run_chain(ch, host_ins)["reduce"]       # the definition, in fp64 on the CPU
+        ins = [fc.to_device(a) for a in host_ins]
         want = fc.run_chain(ch, ins)[0]                      # existing entry point, torch-owned workspace
         fc.fc_get_async_status()
         got = util.poison_(binding.output_tensors(ch, "cuda"))
@@ -38,6 +41,9 @@ def test_static_scratch_matches_fc_run_twice_in_a_row():
         fc.fc_run_softmax_static_scratch(spec, ins, got)     # new entry point: nothing allocated
         fc.fc_get_async_status()
         assert fc.fc_launch_count() == launches + 1
+        # the record of what was enqueued names this call's one kernel only (the single-pass softmax), not fc_run's
+        assert fc.fc_last_plan() == "gemm_tc_mode1_bn256"
+        util.check(got[0], ref, f"static scratch vs oracle ({ch.M}x{ch.N}x{ch.K})")
         util.check_bf16(util.to_f64(got[0]), util.to_f64(want), f"static scratch vs fc_run ({ch.M}x{ch.N}x{ch.K})")
         rows = got[0].float().sum(1)
         assert float((rows - 1).abs().max()) <= 4e-3
