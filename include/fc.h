@@ -58,11 +58,10 @@
  * back: after any fc_run that can have timed out, read the status before the next fc_run on that
  * device, or the next chain that uses the workspace may skip its waits and store wrong values.
  *
- * Testing aid.  With the environment variable FC_INJECT_PANEL_STALL=1, GEMM_NT + ROW_SOFTMAX launches
- * make their cross-tile wait expect an arrival that never comes: the bounded wait expires (about two
- * seconds), nothing is stored, and fc_get_async_status returns FC_ERR_TIMEOUT; the device stays usable.
- * FC_INJECT_SPLIT_STALL=1 does the same to the other bounded wait that crosses CTAs, the one of a split
- * tile's merging slice (GEMM_NT without softmax, with the split scratch registered).
+ * Testing aid.  fc_testing_set (end of this file) flips switches that exist for the test suite only: one makes
+ * the cross-tile wait of GEMM_NT + ROW_SOFTMAX launches expect an arrival that never comes, so that the bounded
+ * wait expires (about two seconds), nothing is stored, and fc_get_async_status returns FC_ERR_TIMEOUT while the
+ * device stays usable; the other does the same to the wait of a split tile's merging slice.
  *
  * Threading.  fc_run may be called from several host threads.  The workspace set by
  * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM, CONV2D_NCHW) must not
@@ -291,6 +290,14 @@ const char* fc_last_error(void);   /* thread-local text of the last failure in t
  * "ew_narrow", "gemm_tc_mode1_bn256_two_pass softmax_rescale", ...): which path a chain took, for logs and tests. */
 const char* fc_last_plan(void);
 int fc_version(void);
+
+/*
+ * Testing switches (process-wide, default 0; the paper has no counterpart).  FC_TESTING_PANEL_STALL / _SPLIT_STALL:
+ * value 1 makes the named bounded wait expect one arrival too many (see "Testing aid" above).
+ */
+#define FC_TESTING_PANEL_STALL 0
+#define FC_TESTING_SPLIT_STALL 1
+void fc_testing_set(int which, int value);
 
 #ifdef __cplusplus
 }

@@ -90,6 +90,8 @@ def lib():
         L.fc_last_error.restype = ctypes.c_char_p
         L.fc_last_plan.restype = ctypes.c_char_p
         L.fc_version.restype = ctypes.c_int
+        L.fc_testing_set.argtypes = [ctypes.c_int, ctypes.c_int]
+        L.fc_testing_set.restype = None
         _lib = L
     return _lib
 
@@ -101,6 +103,14 @@ def fc_last_error() -> str:
 def fc_last_plan() -> str:
     """Names of the kernel variants the last fc_run of this thread enqueued."""
     return lib().fc_last_plan().decode()
+
+
+FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL = 0, 1
+
+
+def fc_testing_set(which: int, value: int) -> None:
+    """Testing switches of the library (see include/fc.h)."""
+    lib().fc_testing_set(int(which), int(value))
 
 
 def fc_version() -> int:

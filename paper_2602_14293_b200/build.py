@@ -36,6 +36,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
+    for d in os.environ.get("FC_DEFINES", "").split():   # development builds: e.g. FC_DEFINES="FC_PROF"
+        cmd.insert(1, "-D" + d)
     subprocess.run(cmd, check=True)
     return LIB
 

@@ -9,6 +9,7 @@
 // Two instantiations: a generic one (any op list, any N, any alignment) and a specialised one for
 // "affine -> tanh-GELU -> add tensor -> logsumexp" on bf16 with the per-column vectors held in
 // registers across rows.
+#include <atomic>
 #include "dev_common.cuh"
 
 namespace fc {
@@ -942,14 +943,14 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
     per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);
     if (ctas > (long long) num_sms * per_sm) ctas = (long long) num_sms * per_sm;
     // the dynamic shared-memory limit of each instantiation is raised once per device, to the maximum
-    static bool raised[4][64] = {};
+    static std::atomic<bool> raised[4][64];   // zero-initialised; set idempotently from any thread
     int dev = 0;
     cudaGetDevice(&dev);
     auto go = [&](auto kernel, int variant) -> cudaError_t {
-        if (smem > 48 * 1024 && (dev < 0 || dev >= 64 || !raised[variant][dev])) {
+        if (smem > 48 * 1024 && (dev < 0 || dev >= 64 || !raised[variant][dev].load(std::memory_order_acquire))) {
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
             if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < 64) raised[variant][dev] = true;
+            if (dev >= 0 && dev < 64) raised[variant][dev].store(true, std::memory_order_release);
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned) ctas);

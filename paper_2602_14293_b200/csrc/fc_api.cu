@@ -15,6 +15,9 @@ __device__ int g_status_word;  // written by kernels when a bounded wait expires
 
 namespace {
 
+// testing switches (fc_testing_set): read on every call, written by tests only
+std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0};
+
 thread_local char t_err[512] = "";
 thread_local char t_plan[256] = "";
 std::atomic<uint64_t> g_launches{0};
@@ -534,6 +537,23 @@ fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr
     return FC_OK;
 }
 
+// The convolution's launch parameters that depend on the spec alone (fc_run adds pointers and the workspace).
+int conv_params(const fc_chain_spec* spec, long long out_rows, TcParams* p) {
+    p->mode = 2;
+    p->batch = (int) spec->batch; p->H = (int) spec->H; p->W = (int) spec->W; p->Cin = (int) spec->Cin; p->Cout = (int) spec->Cout;
+    p->R = (int) spec->R; p->S = (int) spec->S; p->stride = (int) spec->stride; p->pad = (int) spec->pad;
+    p->OH = (int) ((spec->H + 2 * spec->pad - spec->R) / spec->stride + 1);
+    p->OW = (int) ((spec->W + 2 * spec->pad - spec->S) / spec->stride + 1);
+    p->M = (int) out_rows; p->N = (int) spec->Cout; p->K = (int) (spec->R * spec->S * spec->Cin);
+    p->group_m = 1;
+    p->in_dt = spec->in_dtype;
+    p->inv_hw = 1.0f / (float) (p->OH * p->OW);
+    p->pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? 1 : 0;
+    p->a_packed = packed_taps(spec);
+    const int bn = spec->Cout <= 128 ? 128 : 256;
+    return bn;
+}
+
 fc_status cuda_fail(cudaError_t e, const char* what) { return fail(FC_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e)); }
 
 }  // namespace
@@ -596,16 +616,9 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
                 long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
                 p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
             }
-            if (p.mode == 1) {
-                // testing only: FC_INJECT_PANEL_STALL=1 makes every panel wait expect one arrival that never
-                // comes, so that the bounded wait expires and the call ends with FC_ERR_TIMEOUT
-                const char* inj = getenv("FC_INJECT_PANEL_STALL");
-                p.expect_extra = inj && inj[0] == '1' ? 1 : 0;
-            } else {
-                // testing only: FC_INJECT_SPLIT_STALL=1 does the same to the wait of a split tile's merging slice
-                const char* inj = getenv("FC_INJECT_SPLIT_STALL");
-                p.expect_extra = inj && inj[0] == '1' ? 1 : 0;
-            }
+            // testing only (fc_testing_set): the panel wait, or the wait of a split tile's merging slice, expects one
+            // arrival that never comes, so that the bounded wait expires and the call ends with FC_ERR_TIMEOUT
+            p.expect_extra = (p.mode == 1 ? g_inject_panel_stall : g_inject_split_stall).load(std::memory_order_relaxed) ? 1 : 0;
             size_t panel_bytes = 0;
             if (p.mode == 1 || p.mode == 3) {
                 const size_t need = reduction_workspace_bytes(p.mode == 1, spec->M, spec->N);
@@ -705,21 +718,10 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
         case Plan::TC_CONV: {
             TcParams p;
             memset(&p, 0, sizeof(p));
-            p.mode = 2;
-            p.batch = (int) spec->batch; p.H = (int) spec->H; p.W = (int) spec->W; p.Cin = (int) spec->Cin; p.Cout = (int) spec->Cout;
-            p.R = (int) spec->R; p.S = (int) spec->S; p.stride = (int) spec->stride; p.pad = (int) spec->pad;
-            p.OH = (int) ((spec->H + 2 * spec->pad - spec->R) / spec->stride + 1);
-            p.OW = (int) ((spec->W + 2 * spec->pad - spec->S) / spec->stride + 1);
-            p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
-            p.group_m = 1;
-            p.in_dt = spec->in_dtype;
-            p.inv_hw = 1.0f / (float) (p.OH * p.OW);
+            const int bn = conv_params(spec, plan.out_rows, &p);
             p.out = outputs[plan.red_index].ptr; p.out_dt = FC_F32;
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
-            const int bn = spec->Cout <= 128 ? 128 : 256;
-            p.pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? 1 : 0;
-            p.a_packed = packed_taps(spec);
             const size_t out_elems = p.pool ? (size_t) spec->batch * (p.OH / 2) * (p.OW / 2) * spec->Cout : (size_t) spec->batch * spec->Cout;
             const void* image = inputs[0].ptr;
             const void* weights = inputs[1].ptr;
@@ -942,11 +944,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     int bn;
     size_t red = 0;
     if (plan.kind == Plan::TC_CONV) {
-        p.mode = 2;
-        p.Cin = (int) spec->Cin; p.R = (int) spec->R; p.S = (int) spec->S;
-        p.a_packed = packed_taps(spec);
-        p.M = (int) plan.out_rows; p.N = (int) spec->Cout; p.K = (int) (spec->R * spec->S * spec->Cin);
-        bn = spec->Cout <= 128 ? 128 : 256;
+        bn = conv_params(spec, plan.out_rows, &p);
         if (spec->producer == FC_PROD_CONV2D_NCHW) red = nchw_workspace_bytes(spec);
     } else {
         p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
@@ -1018,6 +1016,11 @@ const char* fc_last_error(void) { return t_err; }
 const char* fc_last_plan(void) { return t_plan; }
 
 int fc_version(void) { return FC_VERSION; }
+
+void fc_testing_set(int which, int value) {
+    if (which == FC_TESTING_PANEL_STALL) g_inject_panel_stall.store(value);
+    else if (which == FC_TESTING_SPLIT_STALL) g_inject_split_stall.store(value);
+}
 
 }  // extern "C"
 

@@ -95,7 +95,7 @@ cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t 
 
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
-    int mode;                   // 0 plain store, 1 row softmax, 2 conv + global average pool, 3 row reduction to one value
+    int mode;                   // 0 plain store, 1 row softmax, 2 conv + pooling, 3 row reduction to one value
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
     int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
     int in_dt;                  // FC_BF16 or FC_F16: storage of both MMA operands

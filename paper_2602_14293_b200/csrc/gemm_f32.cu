@@ -8,6 +8,7 @@
 // before it computes anything.  128 threads x (2 x 2) outputs; a thread's rows are 8 apart and its columns
 // 16 apart, so that its 16-byte shared-memory reads along K fall into distinct banks and its stores
 // coalesce.  Rows are padded to 132 floats (33 x 16 bytes).
+#include <atomic>
 #include "dev_common.cuh"
 
 namespace fc {
@@ -231,13 +232,13 @@ __global__ void __launch_bounds__(256, TILE == 128 ? 2 : 4) gemm_f32_big_kernel(
 }  // namespace
 
 cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* launches) {
-    static bool raised[64] = {};
+    static std::atomic<bool> raised[64];   // zero-initialised; set idempotently from any thread
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !raised[dev]) {
+    if (dev >= 0 && dev < 64 && !raised[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(gemm_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        raised[dev] = true;
+        raised[dev].store(true, std::memory_order_release);
     }
     const long long big_tiles = (long long) ((p.M + kBigTile - 1) / kBigTile) * ((p.N + kBigTile - 1) / kBigTile);
     // (1024^3 is 64 such tiles on 148 SMs: 137 us, against 77 us with 64 x 64 tiles)

@@ -43,9 +43,27 @@
 // resets it, so a launch needs no memset as long as the previous one ran to completion.
 #include "tc_common.cuh"
 
+#include <atomic>
 #include <cstdio>
 
 namespace fc {
+#ifdef FC_PROF
+// Development aid, compiled out by default (build with -DFC_PROF=1 or 2): cycle accounting of the two single-thread
+// roles of the leader CTA, per CTA pair.  Row = pair; columns: MMA thread total cycles, its waits for an accumulator
+// buffer, unused, its waits for operand stages, k-blocks issued, cycles in MMA issue + commit, producer total cycles,
+// producer waits for free stages, MMA thread total in nanoseconds (cycles / ns = the SM clock during the kernel).
+__device__ long long g_prof[160][10];
+#if FC_PROF >= 2   // per-wait accounting (itself costs about a hundred cycles per k-block)
+#define PROF_T0(q) q = clock64()
+#define PROF_ADD(acc, q) acc += clock64() - q
+#else             // totals only
+#define PROF_T0(q) (void) q
+#define PROF_ADD(acc, q) (void) acc
+#endif
+#else
+#define PROF_T0(q) (void) q
+#define PROF_ADD(acc, q) (void) acc
+#endif
 namespace {
 
 constexpr int BM = 128;          // rows per CTA; the pair covers 2 * BM
@@ -170,10 +188,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw[];
     // the same offset in both CTAs of the pair: the MMA addresses the peer's tiles by this CTA's descriptors
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float* svec_all = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes);
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + C::kStages * C::kStageBytes + C::kVecBytes);
-    float2* xchg = reinterpret_cast<float2*>(smem + C::kStages * C::kStageBytes + C::kVecBytes + C::kCtrlBytes);
-    float* pool_stage = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes + C::kVecBytes + C::kCtrlBytes + 1024);
+    constexpr int ring_bytes = C::kStages * C::kStageBytes;   // operand stages: A and B side by side per stage
+    float* svec_all = reinterpret_cast<float*>(smem + ring_bytes);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ring_bytes + C::kVecBytes);
+    float2* xchg = reinterpret_cast<float2*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes);
+    float* pool_stage = reinterpret_cast<float*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + 1024);
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -221,8 +240,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t hs = 0, hph = 0;   // stage and phase of the operand ring
             bool ok = true;
+            long long ppw = 0, ppq = 0, ppt0 = clock64();
             for (int u = cluster_id; u < total_units && ok; u += num_clusters) {
                 const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 int mb2, nb;
@@ -237,9 +257,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     oh = rem / p.OW;
                     ow = rem - oh * p.OW;
                 }
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
-                    const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                // (mode 2: filter tap and channel slice of the k-block, carried along instead of divided out per block)
+                int c0 = 0, tap_r = 0, tap_s = 0, tap_col = 0;
+                if constexpr (MODE == 2) {
+                    const int tap = w.kb0 / kb_per_tap;
+                    c0 = (w.kb0 - tap * kb_per_tap) * BK;
+                    tap_r = tap / p.S;
+                    tap_s = tap - tap_r * p.S;
+                    tap_col = tap * p.Cin;
+                }
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
+                    const uint32_t s = hs, ph = hph;
+                    if (++hs == (uint32_t) C::kStages) { hs = 0; hph ^= 1u; }
+                    PROF_T0(ppq);
                     if (!(ok = wait_bar(ptx::smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, p.status))) break;
+                    PROF_ADD(ppw, ppq);
                     const uint32_t full = ptx::mapa(ptx::smem_u32(&ctrl->full[s]), 0);   // the leader's barrier
                     const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
                     // the leader expects the bytes of both CTAs; the peer's copies signal the same barrier.  A
@@ -264,16 +296,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * BK, bcol0, full);
                     } else if constexpr (MODE == 2) {
-                        const int tap = kb / kb_per_tap, c0 = (kb - tap * kb_per_tap) * BK;
-                        const int r = tap / p.S, sx = tap - r * p.S;
-                        ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) sx, (uint16_t) r, full);
-                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap * p.Cin + c0, bcol0, full);
+                        ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) tap_s, (uint16_t) tap_r, full);
+                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap_col + c0, bcol0, full);
+                        c0 += BK;
+                        if (c0 >= kb_per_tap * BK) {
+                            c0 = 0;
+                            tap_col += p.Cin;
+                            if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
+                        }
                     } else {
                         ptx::tma_load_2d_pair(sa, &tmA, kb * bk, row0, full);
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * bk, bcol0, full);
                     }
                 }
             }
+#ifdef FC_PROF
+            if (leader && cluster_id < 160) { g_prof[cluster_id][6] = clock64() - ppt0; g_prof[cluster_id][7] = ppw; }
+#else
+            (void) ppw; (void) ppq; (void) ppt0;
+#endif
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
@@ -282,42 +323,88 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t idesc = ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_BF16 ? 1u : 0u);
             uint32_t it = 0, tile_iter = 0;
             bool ok = true;
+            long long pw_tempty = 0, pw_full = 0, pw_issue = 0, pt0 = clock64(), pq = 0;
+            const unsigned long long pns0 = ptx::globaltimer();
+            uint32_t hs = 0, hph = 0;   // stage and phase of the operand ring
+            const uint64_t desc0 = ptx::smem_desc_k128(ptx::smem_u32(smem));   // swizzled K-major tile at the first stage
+            const uint32_t desc_lo = (uint32_t) desc0, desc_hi = (uint32_t) (desc0 >> 32);
+            const uint32_t full0 = ptx::smem_u32(&ctrl->full[0]), empty0 = ptx::smem_u32(&ctrl->empty[0]);
             for (int u = cluster_id; u < total_units && ok; u += num_clusters, ++tile_iter) {
                 const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+                PROF_T0(pq);
                 if (!(ok = wait_bar(ptx::smem_u32(&ctrl->tempty[buf]), aph ^ 1u, abort_flag, p.status))) break;
+                PROF_ADD(pw_tempty, pq);
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
-                    const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                    if (!(ok = wait_bar(ptx::smem_u32(&ctrl->full[s]), ph, abort_flag, p.status))) break;
+                // This thread's own instruction stream sets the pace of the main loop: per k-block a wait, four MMA
+                // issues and a commit leave little of the 512 cycles the tensor pipe needs for them (measured: sixteen
+                // more dependent instructions per k-block cost forty cycles each time).  So whole rounds of the stage
+                // ring run unrolled, with barrier addresses and descriptor offsets as constants; the k-blocks in front
+                // of a round boundary and behind the last whole round take the same body with a run-time stage.
+                auto kblock = [&](uint32_t s, uint32_t ph, uint32_t acc0) -> bool {
+                    PROF_T0(pq);
+                    if (!wait_bar(full0 + 8u * s, ph, abort_flag, p.status)) return false;
+                    PROF_ADD(pw_full, pq);
                     ptx::tc_fence_after();
-                    const uint32_t sa = ptx::smem_u32(smem + s * C::kStageBytes);
-                    const uint64_t db = ptx::smem_desc_k128(sa + C::kABytes);
+                    PROF_T0(pq);
                     if constexpr (MODE == 4) {
                         // A without swizzle: 2 KB between the core matrices of neighbouring 8-channel chunks, 128
                         // bytes between 8-pixel groups; one MMA takes two chunks
-                        const uint64_t da = ptx::smem_desc_k_plain(sa, 2048, 128);
+                        const uint64_t dp = ptx::smem_desc_k_plain(ptx::smem_u32(smem) + s * C::kStageBytes, 2048, 128);
+                        const uint64_t db = desc0 + (uint64_t) (s * (C::kStageBytes >> 4) + (C::kABytes >> 4));
+                        ptx::tc_mma_f16_pair(d_tmem, dp, db, idesc, acc0);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            ptx::tc_mma_f16_pair(d_tmem, da + (uint64_t) (k * (4096 >> 4)), db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
-                        ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);
-                        continue;
-                    }
-                    const uint64_t da = ptx::smem_desc_k128(sa);
-                    if (f8) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)  // 32 E4M3 values = 32 bytes per MMA along K -> +2 in 16-byte units
-                            ptx::tc_mma_f8_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
+                        for (int k = 1; k < BK / 16; ++k)
+                            ptx::tc_mma_f16_pair(d_tmem, dp + (uint64_t) (k * (4096 >> 4)), db + 2 * k, idesc, 1u);
                     } else {
+                        const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);   // stage s, A tile; B follows kABytes further on
+                        const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
+                        if (f8) {
+                            ptx::tc_mma_f8_pair_lh(d_tmem, a_lo, b_lo, desc_hi, idesc, acc0);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
-                            ptx::tc_mma_f16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, ((kb - w.kb0) | k) != 0);
+                            for (int k = 1; k < 4; ++k)  // 32 E4M3 values = 32 bytes per MMA along K -> +2 in 16-byte units
+                                ptx::tc_mma_f8_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, idesc, 1u);
+                        } else {
+                            ptx::tc_mma_f16_pair_lh(d_tmem, a_lo, b_lo, desc_hi, idesc, acc0);
+#pragma unroll
+                            for (int k = 1; k < BK / 16; ++k)  // 16 bf16 = 32 bytes per MMA along K -> +2 in 16-byte units
+                                ptx::tc_mma_f16_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, idesc, 1u);
+                        }
                     }
-                    ptx::tc_commit_pair(ptx::smem_u32(&ctrl->empty[s]), 3);     // frees the stage in both CTAs
+                    ptx::tc_commit_pair(empty0 + 8u * s, 3);     // frees the stage in both CTAs
+                    PROF_ADD(pw_issue, pq);
+                    return true;
+                };
+                int kb = w.kb0;
+                uint32_t acc = 0;   // the unit's first MMA overwrites the accumulator
+                for (; ok && kb < w.kb1 && hs != 0; ++kb, ++it) {   // up to the next round boundary
+                    ok = kblock(hs, hph, acc);
+                    acc = 1;
+                    if (++hs == (uint32_t) C::kStages) { hs = 0; hph ^= 1u; }
+                }
+                for (; ok && kb + C::kStages <= w.kb1; kb += C::kStages, it += C::kStages) {   // whole rounds
+#pragma unroll
+                    for (int s = 0; s < C::kStages; ++s)
+                        if (ok) ok = kblock((uint32_t) s, hph, s == 0 ? acc : 1u);
+                    acc = 1;
+                    hph ^= 1u;
+                }
+                for (; ok && kb < w.kb1; ++kb, ++it) {   // the rest of the unit
+                    ok = kblock(hs, hph, acc);
+                    acc = 1;
+                    if (++hs == (uint32_t) C::kStages) { hs = 0; hph ^= 1u; }
                 }
                 if (ok) ptx::tc_commit_pair(ptx::smem_u32(&ctrl->tfull[buf]), 3);   // accumulators ready in both CTAs
             }
+#ifdef FC_PROF
+            if (cluster_id < 160) {
+                g_prof[cluster_id][0] = clock64() - pt0; g_prof[cluster_id][1] = pw_tempty; g_prof[cluster_id][2] = 0; g_prof[cluster_id][3] = pw_full;
+                g_prof[cluster_id][4] = it; g_prof[cluster_id][5] = pw_issue; g_prof[cluster_id][8] = (long long) (ptx::globaltimer() - pns0);
+            }
+#else
+            (void) pns0; (void) pt0; (void) pw_tempty; (void) pw_full; (void) pw_issue; (void) pq;
+#endif
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps (both CTAs)
@@ -862,19 +949,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
+// per device and instantiation: resident CTA pairs (0 = not asked yet) and whether the shared-memory limit is set
+struct LaunchState {
+    std::atomic<int> max_clusters[64];
+    std::atomic<bool> attr_set[64];
+};
+
 template <int BN, int MODE>
 cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int num_sms, cudaStream_t stream,
                        TcPlan* plan) {
-    static int max_clusters[64] = {0};   // per device, filled on first use
-    static bool attr_set[64] = {false};  // per device: the dynamic shared-memory limit of this instantiation
-    const int smem = Cfg<BN>::kSmemBytes;
+    static LaunchState state;   // zero-initialised; filled on first use, idempotently, from any thread
+    constexpr int kMaxSmem = 232448;   // 227 KB
+    constexpr int smem = Cfg<BN>::kSmemBytes;
+    static_assert(smem <= kMaxSmem, "shared memory per CTA");
     auto kernel = gemm_tc_kernel<BN, MODE>;
     cudaError_t e = cudaSuccess;
     int dev = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    const bool known = dev >= 0 && dev < 64;
+    if (!known || !state.attr_set[dev].load(std::memory_order_acquire)) {
         if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        if (known) state.attr_set[dev].store(true, std::memory_order_release);
     }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
@@ -889,16 +984,18 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (dev >= 0 && dev < 64 && max_clusters[dev] == 0) {
+    int resident = known ? state.max_clusters[dev].load(std::memory_order_acquire) : 0;
+    if (resident == 0) {
         cfg.gridDim = dim3(num_sms & ~1);
         int n = 0;
         e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
         if (e != cudaSuccess) return e;
-        max_clusters[dev] = n > 0 ? n : 1;
+        resident = n > 0 ? n : 1;
+        if (known) state.max_clusters[dev].store(resident, std::memory_order_release);
     }
     const int tiles_n = (p.N + BN - 1) / BN;
     const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * tiles_n;
-    int max_pairs = dev >= 0 && dev < 64 ? max_clusters[dev] : num_sms / 2;
+    int max_pairs = resident;
     if (max_pairs > num_sms / 2) max_pairs = num_sms / 2;
     int clusters = max_pairs < tiles ? max_pairs : tiles;
     if (MODE == 1) {
@@ -972,6 +1069,10 @@ cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorM
 }
 
 }  // namespace
+
+#ifdef FC_PROF
+extern "C" void fc_debug_prof(long long* out) { cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 160 * 10); }
+#endif
 
 size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : Cfg<128>::kSmemBytes; }
 

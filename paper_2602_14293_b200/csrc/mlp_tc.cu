@@ -21,6 +21,7 @@
 // written) live in the leader; the leader's commits release stages and announce accumulators in both.
 // Accumulators alternate between two 256-column buffers of tensor memory, so the last epilogue of one panel overlaps the first main loop of
 // the next.  Every wait is bounded, as in the other tensor-core kernels.
+#include <atomic>
 #include "tc_common.cuh"
 
 namespace fc {
@@ -283,14 +284,14 @@ mlp_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 
 cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUtensorMap* tmW, int num_sms, cudaStream_t stream,
                           int* launches) {
-    static bool attr_set[64] = {false};
-    static int max_clusters[64] = {0};
+    static std::atomic<bool> attr_set[64];     // zero-initialised; filled idempotently from any thread
+    static std::atomic<int> max_clusters[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
         if ((e = cudaFuncSetAttribute(mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMlpSmem)) != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
@@ -305,14 +306,14 @@ cudaError_t launch_mlp_tc(const MlpParams& p, const CUtensorMap& tmX, const CUte
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (dev >= 0 && dev < 64 && max_clusters[dev] == 0) {
+    if (dev >= 0 && dev < 64 && max_clusters[dev].load(std::memory_order_acquire) == 0) {
         cfg.gridDim = dim3(num_sms & ~1);
         int n = 0;
         if ((e = cudaOccupancyMaxActiveClusters(&n, mlp_tc_kernel, &cfg)) != cudaSuccess) return e;
-        max_clusters[dev] = n > 0 ? n : 1;
+        max_clusters[dev].store(n > 0 ? n : 1, std::memory_order_release);
     }
     const int panels = (p.M + 2 * kRows - 1) / (2 * kRows);
-    int pairs = dev >= 0 && dev < 64 ? max_clusters[dev] : num_sms / 2;
+    int pairs = dev >= 0 && dev < 64 ? max_clusters[dev].load(std::memory_order_acquire) : num_sms / 2;
     if (pairs > num_sms / 2) pairs = num_sms / 2;
     if (pairs > panels) pairs = panels;
     cfg.gridDim = dim3(2 * pairs);

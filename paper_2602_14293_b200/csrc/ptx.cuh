@@ -101,8 +101,10 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uin
 }
 
 // Shared-memory matrix descriptor, K-major operand tile written by TMA with 128-byte swizzle:
-// rows of 128 bytes, 8-row groups 1024 bytes apart.  `addr` must lie in a 1024-byte aligned tile;
-// stepping along K inside the 128-byte row is done by adding the byte offset to `addr`.
+// rows of 128 bytes, 8-row groups 1024 bytes apart.  Stepping along K inside the 128-byte row is done by adding
+// the byte offset to `addr`.  The tile may also start at any 128-byte row of a larger 1024-byte aligned buffer
+// (a row-shifted view of it): the swizzle is applied to the shared-memory address itself, and the descriptor's
+// base-offset field stays zero (measured: with the field set to the row phase the products are wrong).
 __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
     uint64_t d = 0;
     d |= (uint64_t) ((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
@@ -218,6 +220,36 @@ __device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t a_desc,
         "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t"
         "}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The same with both descriptors given as (low word, shared high word): swizzled K-major tiles differ only in the
+// start-address field of the low word, so stepping through stages and along K is one 32-bit add per operand.
+__device__ __forceinline__ void tc_mma_f16_pair_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                                   uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8_pair_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                                  uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // arrive on the mbarrier at this shared-memory offset in every CTA of `mask` once all MMAs issued so

@@ -2,7 +2,6 @@
 kernel's cross-tile wait expect an arrival that never comes.  The wait must give up after its time
 limit, the call must report FC_ERR_TIMEOUT through the status word instead of hanging, and the
 next launch on the same device must work and be correct."""
-import os
 import time
 
 import numpy as np
@@ -25,7 +24,7 @@ def test_panel_wait_expires_with_status_and_device_stays_usable(orc):
     ins = wl.make_inputs(ch, 0)
     dev = [fc.to_device(a) for a in ins]
     outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
-    os.environ["FC_INJECT_PANEL_STALL"] = "1"
+    fc.binding.fc_testing_set(fc.binding.FC_TESTING_PANEL_STALL, 1)
     try:
         t0 = time.perf_counter()
         fc.run_chain(ch, dev, outs)
@@ -33,7 +32,7 @@ def test_panel_wait_expires_with_status_and_device_stays_usable(orc):
             fc.fc_get_async_status()
         waited = time.perf_counter() - t0
     finally:
-        del os.environ["FC_INJECT_PANEL_STALL"]
+        fc.binding.fc_testing_set(fc.binding.FC_TESTING_PANEL_STALL, 0)
     assert err.value.status == 9                      # FC_ERR_TIMEOUT
     assert 1.5 <= waited <= 30.0, waited              # the limit is two seconds per wait
     assert torch.isnan(outs[0].float()).all()         # nothing was stored
@@ -58,7 +57,7 @@ def test_split_merge_wait_expires_with_status_and_device_stays_usable(orc):
     fc.binding.ensure_workspace(spec)
     assert fc.binding.fc_describe_plan(spec)["split"] > 1
     outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
-    os.environ["FC_INJECT_SPLIT_STALL"] = "1"
+    fc.binding.fc_testing_set(fc.binding.FC_TESTING_SPLIT_STALL, 1)
     try:
         t0 = time.perf_counter()
         fc.run_chain(ch, dev, outs)
@@ -66,7 +65,7 @@ def test_split_merge_wait_expires_with_status_and_device_stays_usable(orc):
             fc.fc_get_async_status()
         waited = time.perf_counter() - t0
     finally:
-        del os.environ["FC_INJECT_SPLIT_STALL"]
+        fc.binding.fc_testing_set(fc.binding.FC_TESTING_SPLIT_STALL, 0)
     assert err.value.status == 9                      # FC_ERR_TIMEOUT
     assert 1.5 <= waited <= 30.0, waited
     assert torch.isnan(outs[0].float()).all()         # the only tile was split: nothing was stored
