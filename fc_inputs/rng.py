@@ -153,7 +153,7 @@ def f32_to_e4m3_bits(a: np.ndarray) -> np.ndarray:
 
 def store(a_f32: np.ndarray, dtype: str) -> np.ndarray:
     """Round an fp32 array to the storage type: 'f32' -> float32, 'bf16' -> uint16 patterns, 'f16' -> float16,
-    'f8e4m3' -> uint8 patterns."""
+    'f8e4m3' -> uint8 patterns, 'e8m0' -> scale bytes (biased exponents) tagged int8."""
     if dtype == "f32":
         return np.ascontiguousarray(a_f32, dtype=np.float32)
     if dtype == "bf16":
@@ -162,4 +162,8 @@ def store(a_f32: np.ndarray, dtype: str) -> np.ndarray:
         return np.ascontiguousarray(a_f32, dtype=np.float32).astype(np.float16)   # IEEE half, round to nearest even
     if dtype == "f8e4m3":
         return f32_to_e4m3_bits(a_f32)
+    if dtype == "e8m0":
+        # the values are exponents x: the stored byte is x + 127 (scale 2^x), clipped to the finite patterns 0..254.
+        # The array is tagged int8 so that consumers can tell scale bytes from E4M3 elements (both are one byte).
+        return np.clip(np.rint(np.asarray(a_f32, dtype=np.float64)) + 127, 0, 254).astype(np.uint8).view(np.int8)
     raise ValueError(dtype)

@@ -82,7 +82,7 @@ class Chain:
 
 
 def _size(dtype: str) -> int:
-    if dtype == "f8e4m3":
+    if dtype in ("f8e4m3", "mxf8e4m3", "e8m0"):
         return 1
     return 4 if dtype == "f32" else 2
 
@@ -233,6 +233,21 @@ def conv_nchw(base: Chain) -> Chain:
     return replace(base, name=base.name + "_nchw", producer="conv2d_nchw", input_recipe=rec)
 
 
+def gemm_mxf8_bias_gelu_scale_clamp(M=8192, N=8192, K=4096, out_dtype="bf16", exp_lo=-2, exp_hi=2) -> Chain:
+    """C3's chain on block-scaled 8-bit operands (MXFP8): E4M3 elements, and per row and block of 32 elements along K
+    one power-of-two scale stored as an E8M0 byte (inputs 2 and 3, shapes [M, K/32] and [N, K/32]).  The block
+    exponents are uniform in [exp_lo, exp_hi]; the SCALE op brings the accumulator back to unit variance."""
+    span = np.arange(exp_lo, exp_hi + 1, dtype=np.float64)
+    var = K * float(np.mean(4.0 ** span)) ** 2         # unit-variance elements: variance of the scaled dot product
+    return Chain("gemm_mxf8e4m3_bias_gelu_scale_clamp", "gemm_nt", "mxf8e4m3", out_dtype, M=M, N=N, K=K,
+                 ops=(("scale", var ** -0.5), ("bias_n", 4), ("gelu_tanh",), ("scale", 0.5), ("clamp", -1.0, 1.0)),
+                 input_recipe=(("A", "f8e4m3", (M, K), "normal", 0.0, 1.0),
+                               ("B", "f8e4m3", (N, K), "normal", 0.0, 1.0),
+                               ("SA", "e8m0", (M, K // 32), "int", exp_lo, exp_hi),
+                               ("SB", "e8m0", (N, K // 32), "int", exp_lo, exp_hi),
+                               ("bias", "bf16", (N,), "uniform", -0.1, 0.1)))
+
+
 #: The five benchmark configurations, in the order the benchmark numbers them.
 CONFIGS = {
     "C1": gemm_bias_relu_f32,
@@ -253,6 +268,7 @@ EXTRA = {
     "F7": lambda **kw: scale_add_softmax(**kw),
     "F8": lambda **kw: gemm_softmax(**{"M": 2048, "N": 50264, "K": 4096, **kw}),   # a vocabulary-wide softmax: two kernels
     "F9": lambda **kw: gemm_bias_relu_f32(**{"M": 2048, "N": 2048, "K": 2048, **kw}),   # C1's chain at a size the plain ALUs bound
+    "F10": lambda **kw: gemm_mxf8_bias_gelu_scale_clamp(**kw),   # C3's chain on block-scaled 8-bit operands
 }
 ALL = {**CONFIGS, **EXTRA}
 
@@ -280,7 +296,7 @@ def with_integer_inputs(chain: Chain, lo: int = -4, hi: int = 4) -> Chain:
     rec = list(chain.input_recipe)
     for i in range(min(2, len(rec))):
         tag, dtype, shape, _, _, _ = rec[i]
-        rec[i] = (tag, dtype, shape, "int", lo, hi)
+        rec[i] = (tag, dtype, shape, "int", lo, hi)   # (block scales, inputs 2 and 3 of an MX chain, stay as they are)
     return replace(chain, input_recipe=tuple(rec))
 
 

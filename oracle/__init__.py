@@ -54,10 +54,13 @@ def _p(a: np.ndarray):
 
 
 def widen(a: np.ndarray) -> np.ndarray:
-    """Stored tensor (float32, float16, uint16 bf16 patterns, or uint8 E4M3 patterns) -> float64, exactly."""
+    """Stored tensor (float32, float16, uint16 bf16 patterns, uint8 E4M3 patterns, or int8-tagged E8M0 scale
+    bytes) -> float64, exactly."""
     a = np.ascontiguousarray(a)
     out = np.empty(a.shape, dtype=np.float64)
-    if a.dtype == np.uint8:
+    if a.dtype == np.int8:      # E8M0 scale bytes (the generator tags them with this dtype)
+        lib().orc_widen_e8m0(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
+    elif a.dtype == np.uint8:
         lib().orc_widen_f8e4m3(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
     elif a.dtype == np.uint16:
         lib().orc_widen_bf16(a.ctypes.data_as(ctypes.c_void_p), _i64(a.size), _p(out))
@@ -78,6 +81,16 @@ def gemm_nt(A: np.ndarray, B: np.ndarray) -> np.ndarray:
     assert K == K2
     V = np.empty((M, N), dtype=np.float64)
     lib().orc_gemm_nt(_p(A), _p(B), _i64(M), _i64(N), _i64(K), _p(V))
+    return V
+
+
+def gemm_nt_mx(A: np.ndarray, B: np.ndarray, SA: np.ndarray, SB: np.ndarray) -> np.ndarray:
+    """Block-scaled contraction: SA [M, K/32], SB [N, K/32] are the widened per-block scales."""
+    M, K = A.shape
+    N, K2 = B.shape
+    assert K == K2 and K % 32 == 0 and SA.shape == (M, K // 32) and SB.shape == (N, K // 32)
+    V = np.empty((M, N), dtype=np.float64)
+    lib().orc_gemm_nt_mx(_p(A), _p(B), _p(SA), _p(SB), _i64(M), _i64(N), _i64(K), _p(V))
     return V
 
 
@@ -196,6 +209,8 @@ def run_chain(chain, inputs: List[np.ndarray]) -> Dict[str, np.ndarray]:
     x64 = [widen(a) for a in inputs]
     if chain.producer == "elementwise":
         V = x64[0].copy()
+    elif chain.producer == "gemm_nt" and chain.in_dtype == "mxf8e4m3":
+        V = gemm_nt_mx(x64[0], x64[1], x64[2], x64[3])     # inputs 2, 3: the per-block scales of A and B
     elif chain.producer == "gemm_nt":
         V = gemm_nt(x64[0], x64[1])
     elif chain.producer == "conv2d_nhwc":

@@ -11,6 +11,12 @@
  *   orc_gemm_nt        Y = X * W^T with the weight stored [out_features x in_features] row-major,
  *                      i.e. both operands contiguous along the contracted index (the operand
  *                      convention of the paper's appendix GEMM and linear-layer listings).
+ *   orc_gemm_nt_mx     the same contraction with block-scaled ("microscaling", MX) operands: along the
+ *                      contracted index every 32 consecutive elements of a row share one power-of-two
+ *                      scale, stored as an 8-bit exponent (E8M0: 2^(e - 127), e = 255 is NaN), so
+ *                      Y[m][n] = sum_j 2^(sa[m][j] - 127) 2^(sb[n][j] - 127) sum_{k in block j} X[m][k] W[n][k].
+ *                      The paper only mentions 8-bit floats in passing; the format is the open
+ *                      microscaling one that the B200 tensor cores implement (MXFP8: E4M3 elements).
  *   orc_conv2d_nhwc    cross-correlation, zero padding, floor output size
  *                      OH = (H + 2*pad - R)/stride + 1, input row = oh*stride - pad + r, taps that
  *                      fall outside the image contribute nothing (the indexing convention of the
@@ -39,7 +45,10 @@
  * convolution and against the channel-last form on permuted arrays), high-precision (mpmath) values of GELU / logsumexp / softmax,
  * shift invariance, constant rows, rows summing to one, pooling linearity; max-pool against a
  * reshape-and-max in numpy, a single planted maximum per window, and dropped odd edges; the 16-bit
- * rounding against every stored pattern (identity), exact ties, and numpy's own conversions.
+ * rounding against every stored pattern (identity), exact ties, and numpy's own conversions; the scale
+ * bytes against the library's own E8M0 type over all 256 patterns, the block-scaled contraction against
+ * the plain one (unit scales), against diag(scales) products for a single block, on operands that are
+ * one-hot on either side of a block boundary, and against exact rationals.
  */
 #include <math.h>
 #include <stdint.h>
@@ -133,6 +142,30 @@ void orc_gemm_nt(const double* A, const double* B, int64_t M, int64_t N, int64_t
         for (int64_t n = 0; n < N; ++n) {
             double acc = 0.0;
             for (int64_t k = 0; k < K; ++k) acc += A[m * K + k] * B[n * K + k];
+            V[m * N + n] = acc;
+        }
+    }
+}
+
+/* E8M0 scale bytes -> double: 2^(e - 127); the pattern 255 is NaN (the format has no zero, sign or infinity) */
+void orc_widen_e8m0(const uint8_t* src, int64_t n, double* dst) {
+    for (int64_t i = 0; i < n; ++i) dst[i] = src[i] == 255 ? NAN : ldexp(1.0, (int) src[i] - 127);
+}
+
+/* Block-scaled contraction: V[m][n] = sum_{j ascending} SA[m][j] * SB[n][j] * (sum_{k = 32 j .. 32 j + 31} A[m][k] * B[n][k]),
+ * SA [M][K/32] and SB [N][K/32] the widened scales.  K must be a multiple of 32. */
+void orc_gemm_nt_mx(const double* A, const double* B, const double* SA, const double* SB, int64_t M, int64_t N,
+                    int64_t K, double* V) {
+    const int64_t blocks = K / 32;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t j = 0; j < blocks; ++j) {
+                double blk = 0.0;
+                for (int64_t k = 32 * j; k < 32 * j + 32; ++k) blk += A[m * K + k] * B[n * K + k];
+                acc += SA[m * blocks + j] * SB[n * blocks + j] * blk;
+            }
             V[m * N + n] = acc;
         }
     }

@@ -467,3 +467,70 @@ def test_f8_gemm_chain_small_integers_and_brute_force(orc):
     fb = np.array([[Fraction(float(v)) for v in row] for row in b], dtype=object)
     exact = brute.gemm_nt(fa, fb)
     assert all(Fraction(float(got[i, j])) == exact[i, j] for i in range(4) for j in range(5))   # 4-bit significands: exact in fp64
+
+
+# ------------------------------------------------------------------ block-scaled (MX) contraction
+def test_widen_e8m0_all_patterns(orc):
+    """All 256 scale bytes against the library's own E8M0 type and the format's corner values: 127 is one, 0 the
+    smallest scale 2^-127, 254 the largest 2^127, 255 not a number; neighbouring bytes differ by a factor of two."""
+    pats = np.arange(256, dtype=np.uint8)
+    got = orc.widen(pats.view(np.int8))
+    want = torch.from_numpy(pats).view(torch.float8_e8m0fnu).to(torch.float64).numpy()
+    assert np.array_equal(got[:255], want[:255]) and np.isnan(got[255]) and np.isnan(want[255])
+    assert got[127] == 1.0 and got[0] == 2.0 ** -127 and got[254] == 2.0 ** 127
+    assert np.array_equal(got[1:255] / got[0:254], np.full(254, 2.0))
+    # the generator stores exponent x as byte x + 127 and keeps to the finite patterns
+    assert rng.store(np.array([-3.0, 0.0, 5.0, 400.0, -400.0], np.float32), "e8m0").view(np.uint8).tolist() == [124, 127, 132, 254, 0]
+
+
+def _mx_case(M, N, K, seed, lo=-3, hi=3):
+    ch = replace(wl.gemm_mxf8_bias_gelu_scale_clamp(M, N, K, out_dtype="f32", exp_lo=lo, exp_hi=hi), ops=())
+    return ch, wl.make_inputs(ch, seed)[:4]
+
+
+def test_mx_gemm_unit_scales_is_the_plain_contraction(orc):
+    ch, ins = _mx_case(6, 5, 96, 3)
+    ones = [np.full(a.shape, 127, np.uint8).view(np.int8) for a in ins[2:4]]
+    got = orc.run_chain(ch, ins[:2] + ones)["main"]
+    assert np.array_equal(got, orc.gemm_nt(orc.widen(ins[0]), orc.widen(ins[1])))
+
+
+def test_mx_gemm_single_block_is_a_diagonally_scaled_product(orc):
+    """One block (K = 32): every row of A and of B has one scale, so V = diag(sa) (A B^T) diag(sb) exactly."""
+    ch, ins = _mx_case(7, 9, 32, 4, lo=-20, hi=20)
+    got = orc.run_chain(ch, ins)["main"]
+    a, b, sa, sb = (orc.widen(t) for t in ins)
+    assert np.array_equal(got, sa * (a @ b.T) * sb.T)       # powers of two: the scaling is exact in any order
+
+
+def test_mx_gemm_block_boundaries(orc):
+    """Operands that are one-hot at k = 31, 32 and 95: each product must pick up the scales of its own block
+    (0, 1 and 2), which pins the block length and the index of the scale arrays."""
+    M = N = 3
+    K = 96
+    a = np.zeros((M, K), np.float32)
+    b = np.zeros((N, K), np.float32)
+    ks = [31, 32, 95]
+    for i, k in enumerate(ks):
+        a[i, k] = 1.5
+        b[:, k] = 2.0
+    sa = np.array([[1, 2, 3], [4, 5, 6], [-1, -2, -3]], np.float32)
+    sb = np.array([[0, 1, 0], [2, 0, -2], [7, 8, 9]], np.float32)
+    got = orc.gemm_nt_mx(orc.widen(rng.store(a, "f8e4m3")), orc.widen(rng.store(b, "f8e4m3")),
+                         orc.widen(rng.store(sa, "e8m0")), orc.widen(rng.store(sb, "e8m0")))
+    want = np.array([[3.0 * 2.0 ** (sa[m, k // 32] + sb[n, k // 32]) for n in range(N)] for m, k in enumerate(ks)])
+    assert np.array_equal(got, want)
+
+
+def test_mx_gemm_brute_force_rationals(orc):
+    from fractions import Fraction
+    ch, ins = _mx_case(3, 4, 64, 5, lo=-6, hi=6)
+    got = orc.run_chain(ch, ins)["main"]
+    a, b, sa, sb = ([[Fraction(float(v)) for v in row] for row in orc.widen(t)] for t in ins)
+    for n in reversed(range(4)):                 # a different loop order: columns outermost, blocks and k descending
+        for m in range(3):
+            acc = Fraction(0)
+            for j in reversed(range(2)):
+                for k in reversed(range(32 * j, 32 * j + 32)):
+                    acc += sa[m][j] * sb[n][j] * a[m][k] * b[n][k]
+            assert Fraction(float(got[m, n])) == acc
