@@ -99,7 +99,7 @@ def units(ch):
     """(metric name, unit, algorithmic units per step, roofline bound)."""
     if ch.producer == "elementwise" or wl.collapses(ch):
         return "fused_chain_throughput", "GB/s", wl.algorithmic_bytes(ch) / 1e9, "hbm"
-    return "fused_chain_throughput", "TFLOP/s", ch.flops() / 1e12, "tensor" if ch.in_dtype in ("bf16", "f16", "f8e4m3") else "alu"
+    return "fused_chain_throughput", "TFLOP/s", ch.flops() / 1e12, "tensor" if ch.in_dtype in ("bf16", "f16", "f8e4m3", "mxf8e4m3") else "alu"
 
 
 def dtype_of(ch):
@@ -394,7 +394,7 @@ def roofline_of(ch, workload, units_per_step, bound, ms, peaks, peaks_src, full_
         peak, peak_unit, nominal = peaks["hbm_gbs"], "GB/s", NOMINAL_PEAKS["hbm_gbs"]
         peak_note = f"HBM copy bandwidth, {peaks_src}"
     elif bound == "tensor":
-        mult = 2.0 if ch.in_dtype == "f8e4m3" else 1.0   # no fp8 measurement on this machine: the measured bf16 peak times the nominal fp8 : bf16 ratio
+        mult = 2.0 if ch.in_dtype in ("f8e4m3", "mxf8e4m3") else 1.0   # no fp8 measurement on this machine: the measured bf16 peak times the nominal fp8 : bf16 ratio
         peak = mult * (peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"])
         peak_unit, nominal = "TFLOP/s", mult * NOMINAL_PEAKS["bf16_tflops"]
         peak_note = f"cuBLAS bf16 {'sustained' if long_region else 'burst'}, {peaks_src}" + (" x 2 (nominal fp8 : bf16 ratio)" if mult > 1 else "")

@@ -97,10 +97,20 @@ typedef enum {
     FC_F32 = 0,
     FC_BF16 = 1,
     FC_F16 = 2,       /* IEEE binary16, the storage type of the paper's kernels */
-    FC_F8E4M3 = 3     /* 8-bit float, 4 exponent bits (bias 7), 3 fraction bits, finite only (no infinities, all-ones is NaN):
+    FC_F8E4M3 = 3,    /* 8-bit float, 4 exponent bits (bias 7), 3 fraction bits, finite only (no infinities, all-ones is NaN):
                          storage of BOTH operands of a GEMM_NT producer (fp32 accumulation on the tensor cores, K a multiple
                          of 16); per-tensor scaling is the caller's, undone by a SCALE op.  Not an output, vector or
                          residual type, not for ELEMENTWISE / CONV producers or LINEAR ops. */
+    FC_MXF8E4M3 = 4,  /* spec.in_dtype only: block-scaled 8-bit operands (the open "microscaling" format MXFP8 that the B200
+                         tensor cores implement; the paper mentions 8-bit floats only in passing).  GEMM_NT with reduce NONE:
+                         inputs[0] = A [M,K] and inputs[1] = B [N,K] are FC_F8E4M3 tensors, inputs[2] = SA [M, K/32] and
+                         inputs[3] = SB [N, K/32] are FC_E8M0 tensors, and
+                           v[m][n] = sum_j 2^(SA[m][j] - 127) 2^(SB[n][j] - 127) sum_{k = 32 j .. 32 j + 31} A[m][k] B[n][k].
+                         K a multiple of 128, all four tensors 16-byte aligned.  The scales are first rewritten into the
+                         tensor cores' tile order in the workspace (two small launches; fc_workspace_size reports the bytes:
+                         (ceil(M/128) + ceil(N/128)) * K/128 * 512).  Ops and outputs as for the other 8-bit GEMM; vector and
+                         tensor operands of ops are inputs[4..]. */
+    FC_E8M0 = 5       /* a scale of FC_MXF8E4M3: one byte e meaning 2^(e - 127); 255 is NaN and must not occur */
 } fc_dtype;
 
 typedef enum {

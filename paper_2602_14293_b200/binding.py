@@ -16,11 +16,11 @@ import torch
 PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(PKG, "libfc.so")
 
-FC_F32, FC_BF16, FC_F16, FC_F8E4M3 = 0, 1, 2, 3
+FC_F32, FC_BF16, FC_F16, FC_F8E4M3, FC_MXF8E4M3, FC_E8M0 = 0, 1, 2, 3, 4, 5
 _PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2, "conv2d_nchw": 3}
 _OPKIND = {"bias_n": 0, "affine_n": 1, "relu": 2, "gelu_tanh": 3, "scale": 4, "clamp": 5, "add_tensor": 6, "linear": 7}
 _REDUCE = {"none": 0, "row_logsumexp": 1, "row_softmax": 2, "global_avgpool": 3, "row_sum": 4, "row_max": 5, "row_mean": 6, "maxpool_2x2": 7}
-_DTYPE = {"f32": FC_F32, "bf16": FC_BF16, "f16": FC_F16, "f8e4m3": FC_F8E4M3}
+_DTYPE = {"f32": FC_F32, "bf16": FC_BF16, "f16": FC_F16, "f8e4m3": FC_F8E4M3, "mxf8e4m3": FC_MXF8E4M3}
 FC_MAX_OPS = 12
 FC_VERSION = 2
 
@@ -162,6 +162,8 @@ def _tensor_struct(t: torch.Tensor) -> fc_tensor:
         ft.dtype = FC_F16
     elif t.dtype == torch.float8_e4m3fn:
         ft.dtype = FC_F8E4M3
+    elif t.dtype == torch.uint8:          # scale bytes of block-scaled operands
+        ft.dtype = FC_E8M0
     else:
         raise TypeError(f"unsupported dtype {t.dtype}")
     if t.dim() > 4:
@@ -283,11 +285,14 @@ _workspace = {}
 
 
 def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
-    """Stored numpy tensor (float32, float16, uint16 bf16 or uint8 E4M3 bit patterns) -> torch tensor on `device`."""
+    """Stored numpy tensor (float32, float16, uint16 bf16, uint8 E4M3 bit patterns or int8-tagged E8M0 scale bytes)
+    -> torch tensor on `device`."""
     if a.dtype == np.uint16:
         return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(device)
     if a.dtype == np.uint8:
         return torch.from_numpy(a).view(torch.float8_e4m3fn).to(device)
+    if a.dtype == np.int8:                # E8M0 scale bytes (the generator tags them int8): plain bytes on the device
+        return torch.from_numpy(a.view(np.uint8)).to(device)
     return torch.from_numpy(a).to(device)
 
 

@@ -96,12 +96,12 @@ fc_status get_device(DeviceInfo** out, int* dev_out = nullptr) {
     return FC_OK;
 }
 
-size_t dt_size(int dt) { return dt == FC_F32 ? 4 : (dt == FC_F8E4M3 ? 1 : 2); }
-bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16 || dt == FC_F8E4M3; }
+size_t dt_size(int dt) { return dt == FC_F32 ? 4 : (dt == FC_F8E4M3 || dt == FC_E8M0 || dt == FC_MXF8E4M3 ? 1 : 2); }
+bool dt_valid(int dt) { return dt == FC_F32 || dt == FC_BF16 || dt == FC_F16 || dt == FC_F8E4M3 || dt == FC_E8M0; }   // of a tensor (FC_MXF8E4M3 names a spec's operand format, not a tensor's)
 
 // ------------------------------------------------------------------------------- validation
 struct Plan {
-    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV, GEMM_COLLAPSE, TC_MLP } kind;
+    enum Kind { EW, GEMM_F32, TC_PLAIN, TC_SOFTMAX, TC_LSE, TC_CONV, GEMM_COLLAPSE, TC_MLP, TC_MX } kind;
     long long out_rows, out_cols;  // main output viewed as [rows][cols]
     int n_prod_inputs;
     int n_outputs;
@@ -151,17 +151,18 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
     if (s->struct_size != sizeof(fc_chain_spec)) return fail(FC_ERR_INVALID_SPEC, "struct_size %u, expected %zu", s->struct_size, sizeof(fc_chain_spec));
     if (s->version != FC_VERSION) return fail(FC_ERR_INVALID_SPEC, "version %u, expected %d", s->version, FC_VERSION);
     if (s->producer < 0 || s->producer > FC_PROD_CONV2D_NCHW) return fail(FC_ERR_INVALID_SPEC, "unknown producer %d", s->producer);
-    if (!dt_valid(s->in_dtype) || !dt_valid(s->out_dtype))
+    if ((!dt_valid(s->in_dtype) && s->in_dtype != FC_MXF8E4M3) || !dt_valid(s->out_dtype) || s->in_dtype == FC_E8M0)
         return fail(FC_ERR_INVALID_SPEC, "unknown in/out dtype");
     if (s->acc_dtype != FC_F32) return fail(FC_ERR_INVALID_SPEC, "acc_dtype must be FC_F32");
-    if (s->out_dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "FC_F8E4M3 is an operand type only (outputs are fp32, bf16 or fp16)");
-    if (s->in_dtype == FC_F8E4M3 && s->producer != FC_PROD_GEMM_NT) return fail(FC_ERR_UNSUPPORTED, "FC_F8E4M3 operands need a GEMM_NT producer");
+    if (s->out_dtype == FC_F8E4M3 || s->out_dtype == FC_E8M0) return fail(FC_ERR_UNSUPPORTED, "8-bit types are operand types only (outputs are fp32, bf16 or fp16)");
+    if ((s->in_dtype == FC_F8E4M3 || s->in_dtype == FC_MXF8E4M3) && s->producer != FC_PROD_GEMM_NT) return fail(FC_ERR_UNSUPPORTED, "8-bit operands need a GEMM_NT producer");
+    if (s->in_dtype == FC_MXF8E4M3 && s->reduce != FC_RED_NONE) return fail(FC_ERR_UNSUPPORTED, "block-scaled operands support reduce NONE");
     if (s->reduce < 0 || s->reduce > FC_RED_MAXPOOL_2X2) return fail(FC_ERR_INVALID_SPEC, "unknown reduce %d", s->reduce);
     if (s->n_ops < 0 || s->n_ops > FC_MAX_OPS) return fail(FC_ERR_INVALID_SPEC, "n_ops %d out of range", s->n_ops);
     for (int i = 0; i < s->n_ops; ++i)
         if (s->ops[i].kind < 0 || s->ops[i].kind > FC_OP_LINEAR) return fail(FC_ERR_INVALID_SPEC, "op %d: unknown kind %d", i, s->ops[i].kind);
 
-    plan->n_prod_inputs = s->producer == FC_PROD_ELEMENTWISE ? 1 : 2;
+    plan->n_prod_inputs = s->producer == FC_PROD_ELEMENTWISE ? 1 : (s->in_dtype == FC_MXF8E4M3 ? 4 : 2);
     if (is_conv(s)) {
         if (s->batch < 1 || s->H < 1 || s->W < 1 || s->Cin < 1 || s->Cout < 1 || s->R < 1 || s->S < 1 || s->stride < 1 || s->pad < 0)
             return fail(FC_ERR_SHAPE, "conv dimensions must be positive (pad >= 0)");
@@ -193,6 +194,8 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
                     return fail(FC_ERR_UNSUPPORTED, "fp32 GEMM supports fp32 output without reduction");
                 if (s->N > 65535LL * 32) return fail(FC_ERR_SHAPE, "fp32 GEMM supports N <= %lld", 65535LL * 32);
                 plan->kind = Plan::GEMM_F32;
+            } else if (s->in_dtype == FC_MXF8E4M3) {
+                plan->kind = Plan::TC_MX;
             } else if (s->reduce == FC_RED_NONE) {
                 plan->kind = Plan::TC_PLAIN;
             } else if (s->reduce == FC_RED_ROW_SOFTMAX) {
@@ -245,7 +248,7 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
             plan->kind = Plan::TC_MLP;
         }
     }
-    if (plan->kind == Plan::TC_PLAIN || plan->kind == Plan::TC_SOFTMAX || plan->kind == Plan::TC_LSE || plan->kind == Plan::TC_CONV) {
+    if (plan->kind == Plan::TC_PLAIN || plan->kind == Plan::TC_SOFTMAX || plan->kind == Plan::TC_LSE || plan->kind == Plan::TC_CONV || plan->kind == Plan::TC_MX) {
         int vecs = 0;
         for (int i = 0; i < s->n_ops; ++i) vecs += s->ops[i].kind == FC_OP_BIAS_N ? 1 : (s->ops[i].kind == FC_OP_AFFINE_N ? 2 : 0);
         if (vecs > 3) return fail(FC_ERR_UNSUPPORTED, "tensor-core chains support at most 3 per-column vector operands");
@@ -271,9 +274,18 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         if ((st = check_tensor(in[0], "inputs[0]", s->in_dtype, 2, sh))) return st;
     } else if (s->producer == FC_PROD_GEMM_NT) {
         const long long sa[2] = {s->M, s->K}, sb[2] = {s->N, s->K};
-        if ((st = check_tensor(in[0], "inputs[0] (A)", s->in_dtype, 2, sa))) return st;
-        if ((st = check_tensor(in[1], "inputs[1] (B)", s->in_dtype, 2, sb))) return st;
-        if (s->in_dtype != FC_F32) {
+        const int operand_dt = s->in_dtype == FC_MXF8E4M3 ? FC_F8E4M3 : s->in_dtype;
+        if ((st = check_tensor(in[0], "inputs[0] (A)", operand_dt, 2, sa))) return st;
+        if ((st = check_tensor(in[1], "inputs[1] (B)", operand_dt, 2, sb))) return st;
+        if (s->in_dtype == FC_MXF8E4M3) {
+            if (s->K % 128) return fail(FC_ERR_ALIGNMENT, "block-scaled operands need K %% 128 == 0 (K = %lld)", (long long) s->K);
+            const long long ssa[2] = {s->M, s->K / 32}, ssb[2] = {s->N, s->K / 32};
+            if ((st = check_tensor(in[2], "inputs[2] (scales of A)", FC_E8M0, 2, ssa))) return st;
+            if ((st = check_tensor(in[3], "inputs[3] (scales of B)", FC_E8M0, 2, ssb))) return st;
+            if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr) | reinterpret_cast<uintptr_t>(in[2].ptr) |
+                 reinterpret_cast<uintptr_t>(in[3].ptr)) & 15)
+                return fail(FC_ERR_ALIGNMENT, "block-scaled operands and their scales must be 16-byte aligned");
+        } else if (s->in_dtype != FC_F32) {
             const int kq = s->in_dtype == FC_F8E4M3 ? 16 : 8;   // a row of K elements must be a multiple of 16 bytes
             if (s->K % kq) return fail(FC_ERR_ALIGNMENT, "this GEMM needs K %% %d == 0 (K = %lld)", kq, (long long) s->K);
             if ((reinterpret_cast<uintptr_t>(in[0].ptr) | reinterpret_cast<uintptr_t>(in[1].ptr)) & 15)
@@ -315,12 +327,12 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
                 if (idx[k] < plan.n_prod_inputs || idx[k] >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, idx[k]);
                 snprintf(what, sizeof(what), "inputs[%d] (op %d vector)", idx[k], i);
                 if ((st = check_tensor(in[idx[k]], what, -1, 1, vec))) return st;
-                if (in[idx[k]].dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "%s: FC_F8E4M3 vectors are not supported", what);
+                if (in[idx[k]].dtype == FC_F8E4M3 || in[idx[k]].dtype == FC_E8M0) return fail(FC_ERR_UNSUPPORTED, "%s: 8-bit vectors are not supported", what);
             }
         } else if (op.kind == FC_OP_ADD_TENSOR) {
             if (op.in0 < plan.n_prod_inputs || op.in0 >= n_in) return fail(FC_ERR_INVALID_SPEC, "op %d: operand index %d out of range", i, op.in0);
             snprintf(what, sizeof(what), "inputs[%d] (op %d tensor)", op.in0, i);
-            if (in[op.in0].dtype == FC_F8E4M3) return fail(FC_ERR_UNSUPPORTED, "%s: FC_F8E4M3 tensors are not supported", what);
+            if (in[op.in0].dtype == FC_F8E4M3 || in[op.in0].dtype == FC_E8M0) return fail(FC_ERR_UNSUPPORTED, "%s: 8-bit tensors are not supported", what);
             if (is_conv(s)) {
                 const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
                 const long long sh[4] = {s->batch, OH, OW, s->Cout};
@@ -509,6 +521,23 @@ fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long 
     return FC_OK;
 }
 
+// Scale tiles of the block-scaled GEMM: rows of 128 words (512 bytes), one row per (128-row tile, k-block)
+fc_status encode_scale_tiles(CUtensorMap* tm, const void* ptr, long long tile_rows) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const MapKey mk = {ptr, {7, tile_rows, dev, 0, 0, 0, 0, 0}};
+    if (g_maps.find(mk, tm)) return FC_OK;
+    const cuuint64_t dims[2] = {128, (cuuint64_t) tile_rows};
+    const cuuint64_t strides[1] = {512};
+    const cuuint32_t box[2] = {128, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(FC_ERR_CUDA, "cuTensorMapEncodeTiled (scale tiles) failed with CUresult %d", (int) r);
+    g_maps.put(mk, *tm);
+    return FC_OK;
+}
+
 // Eight channels (a first layer: RGB padded to 8) leave 56 of a k-block's 64 channels empty; packing eight taps
 // into a k-block instead cuts a 5 x 5 filter from 25 k-blocks to 4.  The eight small copies of such a k-block
 // cost about 1.9 us against 0.35 - 0.65 us for one 64-channel copy (measured), so from 16 channels on the
@@ -652,6 +681,39 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             if (e == cudaSuccess && p.two_pass)
                 e = launch_softmax_rescale(p.out, p.out_dt, p.stats, spec->M, spec->N, tiles_n, bn, dev->num_sms, stream, &launches);
+            break;
+        }
+        case Plan::TC_MX: {
+            const size_t sa_bytes = (scale_tiles_bytes(spec->M, spec->K) + 255) / 256 * 256, sb_bytes = scale_tiles_bytes(spec->N, spec->K);
+            if (!dev->workspace || dev->workspace_bytes < sa_bytes + sb_bytes)
+                return fail(FC_ERR_WORKSPACE, "block-scaled operands need a %zu-byte workspace (fc_set_workspace); have %zu", sa_bytes + sb_bytes, dev->workspace_bytes);
+            {   // the scale tiles overwrite whatever counters a previous layout kept here
+                std::lock_guard<std::mutex> lk(g_mu);
+                dev->counter_layout = 0;
+            }
+            void* sa_tiles = dev->workspace;
+            void* sb_tiles = (char*) dev->workspace + sa_bytes;
+            if ((e = launch_scale_tiles(inputs[2].ptr, sa_tiles, spec->M, spec->K, false, stream, &launches)) != cudaSuccess) return cuda_fail(e, "scale-tile kernel launch");
+            if ((e = launch_scale_tiles(inputs[3].ptr, sb_tiles, spec->N, spec->K, true, stream, &launches)) != cudaSuccess) return cuda_fail(e, "scale-tile kernel launch");
+            TcParams p;
+            memset(&p, 0, sizeof(p));
+            p.mode = 6;
+            p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+            p.in_dt = FC_F8E4M3;   // the elements; the scales come through their own tensor maps
+            p.out = outputs[plan.main_index].ptr; p.out_dt = spec->out_dtype;
+            p.status = dev->status;
+            build_ops(spec, inputs, &p.ops);
+            {
+                const long long panel_bytes = 256LL * spec->K;
+                long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
+                p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
+            }
+            CUtensorMap tmA, tmB, tmSA, tmSB;
+            if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, FC_F8E4M3))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, 64, FC_F8E4M3))) return st;   // 256 x 128 tiles: each CTA of a pair loads 64 rows of B
+            if ((st = encode_scale_tiles(&tmSA, sa_tiles, (long long) ((spec->M + 127) / 128) * (spec->K / 128)))) return st;
+            if ((st = encode_scale_tiles(&tmSB, sb_tiles, (long long) ((spec->N + 127) / 128) * (spec->K / 128)))) return st;
+            e = launch_gemm_tc_mx(p, tmA, tmB, tmSA, tmSB, dev->num_sms, stream, &launches);
             break;
         }
         case Plan::TC_MLP: {
@@ -821,7 +883,7 @@ fc_status fc_run_host(const fc_chain_spec* spec, const fc_tensor* host_inputs, i
     const long long rows = conv ? spec->batch : spec->M;
     const long long gran = (plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_MLP) ? 256 : 1;
     long long chunks = 1;
-    if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && plan.kind != Plan::GEMM_COLLAPSE && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
+    if (moved >= ((size_t) 32 << 20) && plan.kind != Plan::GEMM_F32 && plan.kind != Plan::GEMM_COLLAPSE && plan.kind != Plan::TC_MX && n_inputs >= plan.n_prod_inputs && n_outputs == plan.n_outputs) {
         chunks = rows / gran < 8 ? rows / gran : 8;
         if (chunks < 1) chunks = 1;
     }
@@ -912,6 +974,7 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     if ((st = validate_spec(spec, &plan))) return st;
     *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? reduction_workspace_bytes(plan.kind == Plan::TC_SOFTMAX, spec->M, spec->N)
            : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K)
+           : plan.kind == Plan::TC_MX ? (spec->K % 128 ? 0 : (scale_tiles_bytes(spec->M, spec->K) + 255) / 256 * 256 + scale_tiles_bytes(spec->N, spec->K))
            : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     return FC_OK;
 }
@@ -937,6 +1000,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     if (plan.kind == Plan::GEMM_F32) { snprintf(text, capacity, "kernel=gemm_f32"); return FC_OK; }
     if (plan.kind == Plan::GEMM_COLLAPSE) { snprintf(text, capacity, "kernel=collapse"); return FC_OK; }
     if (plan.kind == Plan::TC_MLP) { snprintf(text, capacity, "kernel=mlp_tc"); return FC_OK; }
+    if (plan.kind == Plan::TC_MX) { snprintf(text, capacity, "kernel=gemm_tc mode=6 bn=128"); return FC_OK; }
     DeviceInfo* dev;
     if ((st = get_device(&dev))) return st;
     TcParams p;

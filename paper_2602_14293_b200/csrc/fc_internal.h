@@ -95,7 +95,8 @@ cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t 
 
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
-    int mode;                   // 0 plain store, 1 row softmax, 2 conv + pooling, 3 row reduction to one value
+    int mode;                   // 0 plain store, 1 row softmax, 2 conv + pooling, 3 row reduction to one value,
+                                // 6 plain store with block-scaled E4M3 operands (scale tiles through a third and fourth tensor map)
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
     int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
     int in_dt;                  // FC_BF16 or FC_F16: storage of both MMA operands
@@ -132,6 +133,16 @@ constexpr size_t kTcSplitCounterBytes = 1024;
 constexpr size_t kTcSplitBytes = kTcSplitCounterBytes + (size_t) kTcSplitUnits * 2 * 128 * 256 * 4;
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                            int bn, int num_sms, cudaStream_t stream, int* launches);
+// Mode 6: `tmSA` / `tmSB` map the scale tiles written by launch_scale_tiles (rows of 128 words, one row per
+// 128-row tile and 128-element k-block).
+cudaError_t launch_gemm_tc_mx(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
+                              const CUtensorMap& tmSB, int num_sms, cudaStream_t stream, int* launches);
+// E8M0 scales [rows][K/32] -> tiles of 512 bytes per (128 rows, 128 elements of K), in the order the tensor core's
+// scale columns want them: byte (r % 32) * 16 + (r / 32) * 4 + j holds the scale of row r of the tile and the j-th
+// block of 32 elements; rows past `rows` get the scale 1.  K a multiple of 128.  `beside_previous` as above.
+cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, long long K, bool beside_previous, cudaStream_t stream,
+                               int* launches);
+size_t scale_tiles_bytes(long long rows, long long K);
 size_t gemm_tc_smem_bytes(int bn);
 
 // Back-to-back linear layers kept on chip (mlp_tc.cu): layer l maps width[l-1] (K0 for l = 0) to width[l]

@@ -15,6 +15,14 @@
 //   (template mode 4 is mode 2 for images of eight channels: a k-block then holds eight filter taps, gathered
 //    as eight 8-channel copies into an unswizzled operand tile; a separate instantiation, so that the loops
 //    of mode 2 stay as they are)
+//   mode 6  mode 0 on block-scaled 8-bit operands (MXFP8: E4M3 elements, one E8M0 scale per row and 32 elements
+//           along K).  tcgen05.mma.kind::mxf8f6f4.block_scale takes the scales from tensor memory: per k-block of
+//           128 elements a 512-byte tile of A scales (this CTA's 128 rows x 4 blocks) and one of B scales (the
+//           tile's 128 columns x 4 blocks) arrive with the operands (two more TMA loads from scale tiles that a
+//           layout kernel has written, see launch_scale_tiles), tcgen05.cp moves them into four tensor-memory
+//           columns each in front of the k-block's four MMAs, and MMA j names byte j of those columns.  Measured
+//           layout: row r of the tile reads byte (r % 32) * 16 + (r / 32) * 4 + j of the 512.  Tiles are 256 x 128
+//           (two accumulator buffers and the scale columns must share the 512 columns of tensor memory).
 //
 // Work unit: a 256 x BN output tile owned by a PAIR of CTAs on neighbouring SMs (cluster of 2,
 // tcgen05 cta_group::2).  Each CTA loads its own 128 rows of A and HALF of the B tile, so a k-block
@@ -83,6 +91,7 @@ struct Cfg {
     static constexpr int kCtrlBytes = 256;
     static constexpr int kPoolBytes = 8 * 32 * 17 * 4;   // max-pool: 32 pixels x 16 channels (+1 pad) per epilogue warp
     static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024 + kPoolBytes + 1024;  // exchange, pool staging, alignment slack
+    static constexpr int kScaleBytes = kStages * 1024;   // mode 6: a tile of A scales and one of B scales per stage, behind everything else
 };
 
 struct Ctrl {
@@ -183,7 +192,8 @@ __host__ __device__ __forceinline__ int count_kb(const TcParams& p) {
 
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmSA,
+               const __grid_constant__ CUtensorMap tmSB, const TcParams p) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     // the same offset in both CTAs of the pair: the MMA addresses the peer's tiles by this CTA's descriptors
@@ -193,6 +203,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ring_bytes + C::kVecBytes);
     float2* xchg = reinterpret_cast<float2*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes);
     float* pool_stage = reinterpret_cast<float*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + 1024);
+    constexpr bool kMx = MODE == 6;
+    uint8_t* scale_ring = smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + 1024 + C::kPoolBytes;   // mode 6: [stage][A tile 512 B | B tile 512 B]
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -204,7 +216,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int total_tiles = tiles_m * tiles_n;
     constexpr bool kConv = MODE == 2 || MODE == 4;   // 4: the convolution with eight filter taps per k-block (TcParams::a_packed)
     const int kb_per_tap = kConv ? (p.Cin + BK - 1) / BK : 1;
-    const bool f8 = !kConv && p.in_dt == FC_F8E4M3;
+    const bool f8 = !kConv && (kMx || p.in_dt == FC_F8E4M3);
     const int bk = f8 ? 2 * BK : BK;   // K elements per k-block: 128 bytes of a row
     const int num_kb = count_kb<MODE>(p);
     const int total_units = p.split > 1 ? p.split_from + (total_tiles - p.split_from) * p.split : total_tiles;
@@ -222,9 +234,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmB);
+        if constexpr (kMx) {
+            ptx::prefetch_tensormap(&tmSA);
+            ptx::prefetch_tensormap(&tmSB);
+        }
     }
+    constexpr int kTmemAlloc = kMx ? 512 : C::kTmemCols;   // mode 6: eight more columns for the scales (a power of two must be asked for)
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), C::kTmemCols);
+        ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), kTmemAlloc);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
@@ -246,7 +263,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int u = cluster_id; u < total_units && ok; u += num_clusters) {
                 const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 int mb2, nb;
-                tile_coords((MODE == 0 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
+                tile_coords((MODE == 0 || MODE == 6 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
@@ -278,7 +295,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // peer copy may land before the expectation is posted: the phase cannot complete before
                     // the leader's arrival, and the peer starts the next phase only after the leader's MMAs
                     // of this one (the commit that frees the stage) are done.
-                    if (leader) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->full[s]), 2 * C::kStageBytes);
+                    if (leader) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->full[s]), 2 * (C::kStageBytes + (kMx ? 1024 : 0)));
+                    if constexpr (kMx) {
+                        // the scales of this k-block: this CTA's 128 rows of A, the tile's 128 columns of B
+                        const uint32_t sc = ptx::smem_u32(scale_ring) + s * 1024;
+                        ptx::tma_load_2d_pair(sc, &tmSA, 0, (mb2 * 2 + (int) cta_rank) * num_kb + kb, full);
+                        ptx::tma_load_2d_pair(sc + 512, &tmSB, 0, nb * num_kb + kb, full);
+                    }
                     if constexpr (MODE == 4) {
                         // eight copies of 128 pixels x 8 channels, each one column of core matrices (2 KB)
                         const int cpt = p.Cin >> 3, chunks = p.R * p.S * cpt;
@@ -357,6 +380,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int k = 1; k < BK / 16; ++k)
                             ptx::tc_mma_f16_pair(d_tmem, dp + (uint64_t) (k * (4096 >> 4)), db + 2 * k, idesc, 1u);
+                    } else if constexpr (kMx) {
+                        // scales into tensor memory (the copies and the MMAs run in the order they are issued), then four
+                        // MMAs of 32 elements along K, MMA j with byte j of the scale columns
+                        const uint32_t sc = ptx::smem_u32(scale_ring) + s * 1024;
+                        ptx::tc_cp_32x128b_pair(tmem_base + 2 * BN, ptx::smem_desc_k_plain(sc, 16, 128));
+                        ptx::tc_cp_32x128b_pair(tmem_base + 2 * BN + 4, ptx::smem_desc_k_plain(sc + 512, 16, 128));
+                        const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);
+                        const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
+                        ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo, b_lo, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, 0, 0), tmem_base + 2 * BN, tmem_base + 2 * BN + 4, acc0);
+#pragma unroll
+                        for (int k = 1; k < 4; ++k)
+                            ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, (uint32_t) k, (uint32_t) k), tmem_base + 2 * BN,
+                                                     tmem_base + 2 * BN + 4, 1u);
                     } else {
                         const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);   // stage s, A tile; B follows kABytes further on
                         const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
@@ -425,7 +461,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int u = cluster_id; u < total_units; u += num_clusters, ++tile_iter) {
             const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
             int mb2, nb;
-            tile_coords((MODE == 0 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
+            tile_coords((MODE == 0 || MODE == 6 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
             const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;
@@ -547,7 +583,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::tmem_wait_st();
             }
 
-            if constexpr (MODE == 0) {
+            if constexpr (MODE == 0 || MODE == 6) {
                 uint32_t ra[16], rb[16];
                 ptx::tmem_ld_32x16_async(tacc, ra);
 #pragma unroll 1
@@ -945,7 +981,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::cluster_sync();   // neither CTA leaves while the other may still read its tiles or signal its barriers
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+        ptx::tmem_dealloc(tmem_base, kTmemAlloc);
     }
 }
 
@@ -957,10 +993,10 @@ struct LaunchState {
 
 template <int BN, int MODE>
 cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int num_sms, cudaStream_t stream,
-                       TcPlan* plan) {
+                       TcPlan* plan, const CUtensorMap* tmSA = nullptr, const CUtensorMap* tmSB = nullptr) {
     static LaunchState state;   // zero-initialised; filled on first use, idempotently, from any thread
     constexpr int kMaxSmem = 232448;   // 227 KB
-    constexpr int smem = Cfg<BN>::kSmemBytes;
+    constexpr int smem = Cfg<BN>::kSmemBytes + (MODE == 6 ? Cfg<BN>::kScaleBytes : 0);
     static_assert(smem <= kMaxSmem, "shared memory per CTA");
     auto kernel = gemm_tc_kernel<BN, MODE>;
     cudaError_t e = cudaSuccess;
@@ -1054,7 +1090,8 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
         snprintf(name, sizeof(name), "gemm_tc_mode%d_bn%d%s%s", MODE, BN, q.split > 1 ? "_split" : "", MODE == 1 && p.two_pass ? "_two_pass" : "");
         note_kernel(name);
     }
-    return cudaLaunchKernelEx(&cfg, kernel, *tmA, *tmB, q);
+    // (the scale-tile maps are read in mode 6 only; the other modes get the operand maps again)
+    return cudaLaunchKernelEx(&cfg, kernel, *tmA, *tmB, tmSA ? *tmSA : *tmA, tmSB ? *tmSB : *tmB, q);
 }
 
 template <int BN>
@@ -1080,6 +1117,12 @@ cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUte
                            cudaStream_t stream, int* launches) {
     *launches += 1;
     return bn == 256 ? launch_bn<256>(p, &tmA, &tmB, num_sms, stream, nullptr) : launch_bn<128>(p, &tmA, &tmB, num_sms, stream, nullptr);
+}
+
+cudaError_t launch_gemm_tc_mx(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
+                              const CUtensorMap& tmSB, int num_sms, cudaStream_t stream, int* launches) {
+    *launches += 1;
+    return launch_one<128, 6>(p, &tmA, &tmB, num_sms, stream, nullptr, &tmSA, &tmSB);
 }
 
 cudaError_t plan_gemm_tc(const TcParams& p, int bn, int num_sms, TcPlan* plan) {

@@ -108,7 +108,57 @@ __global__ void __launch_bounds__(256) zero_fill_kernel(uint32_t* ptr, size_t wo
     }
 }
 
+// One thread per (row of a 128-row tile, four k-blocks): reads the row's 16 scale bytes of those k-blocks and writes
+// one word into each of their four tiles.
+__global__ void __launch_bounds__(256) scale_tiles_kernel(const uint8_t* __restrict__ scales, uint32_t* __restrict__ tiles, long long rows,
+                                                          int blocks32, int num_kb, long long padded_rows) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int groups = (num_kb + 3) >> 2;
+    const long long idx = (long long) blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= padded_rows * groups) return;
+    const long long r = idx / groups;
+    const int g = (int) (idx - r * groups);
+    uint32_t w[4] = {0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu};   // scale 1 for rows that do not exist
+    if (r < rows) {
+        const uint8_t* src = scales + r * blocks32 + 16 * g;
+        if (16 * g + 16 <= blocks32 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+            const uint4 q = *reinterpret_cast<const uint4*>(src);
+            w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
+        } else {
+            for (int i = 0; i < 4; ++i)
+                if (16 * g + 4 * i + 4 <= blocks32) w[i] = (uint32_t) src[4 * i] | (uint32_t) src[4 * i + 1] << 8 | (uint32_t) src[4 * i + 2] << 16 | (uint32_t) src[4 * i + 3] << 24;
+        }
+    }
+    const long long tile = r >> 7;
+    const int rr = (int) (r & 127), word = (rr & 31) * 4 + (rr >> 5);
+    for (int i = 0; i < 4; ++i) {
+        const int kb = 4 * g + i;
+        if (kb < num_kb) tiles[(tile * num_kb + kb) * 128 + word] = w[i];
+    }
+}
+
 }  // namespace
+
+size_t scale_tiles_bytes(long long rows, long long K) { return (size_t) ((rows + 127) / 128) * (size_t) (K / 128) * 512; }
+
+cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, long long K, bool beside_previous, cudaStream_t stream,
+                               int* launches) {
+    const int num_kb = (int) (K / 128), groups = (num_kb + 3) / 4;
+    const long long padded = (rows + 127) / 128 * 128, total = padded * groups;
+    if (K % 128 || total > 0x7fffffffLL * 256) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned) ((total + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = beside_previous ? 1 : 0;
+    note_kernel("scale_tiles");
+    ++*launches;
+    return cudaLaunchKernelEx(&cfg, scale_tiles_kernel, (const uint8_t*) scales, (uint32_t*) tiles, rows, (int) (K / 32), num_kb, padded);
+}
 
 cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches) {
     const size_t words = bytes / 4;

@@ -252,6 +252,36 @@ __device__ __forceinline__ void tc_mma_f8_pair_lh(uint32_t d_tmem, uint32_t a_lo
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Block-scaled 8-bit operands (kind::mxf8f6f4, one E8M0 scale per row and 32 elements along K = per MMA): the
+// instruction descriptor also names the scale format and which of the four scale bytes of a tensor-memory column
+// this MMA uses (measured layout, see gemm_tc.cu).
+__host__ __device__ constexpr uint32_t idesc_mxf8_e4m3(int m, int n, uint32_t a_sf_id, uint32_t b_sf_id) {
+    return (b_sf_id << 4)                 // byte of the B scale column
+           | (0u << 7) | (0u << 10)       // A, B format E4M3
+           | ((uint32_t) (n >> 3) << 17)  // N / 8
+           | (1u << 23)                   // scale format E8M0
+           | ((uint32_t) (m >> 4) << 24)  // M / 16
+           | (a_sf_id << 29);             // byte of the A scale column
+}
+__device__ __forceinline__ void tc_mma_mxf8_pair_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                                    uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %7, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], da, db, %4, [%5], [%6], p;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+        : "memory");
+}
+// 32 rows x 16 bytes of shared memory (rows 16 bytes apart) -> four tensor-memory columns, the same 32 x 16 bytes in
+// each of the four 32-lane quarters, in both CTAs of the pair (each from its own shared memory)
+__device__ __forceinline__ void tc_cp_32x128b_pair(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
 // arrive on the mbarrier at this shared-memory offset in every CTA of `mask` once all MMAs issued so
 // far have completed (a barrier multicast, not a data multicast)
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t mask) {
