@@ -63,6 +63,13 @@
  * wait expires (about two seconds), nothing is stored, and fc_get_async_status returns FC_ERR_TIMEOUT while the
  * device stays usable; the other does the same to the wait of a split tile's merging slice.
  *
+ * Debug build.  The same sources compiled with -DFC_DEBUG (paper_2602_14293_b200/build.py builds it as libfc_debug.so)
+ * check, in the kernels, every global-memory address that comes out of their own index arithmetic (output stores of
+ * the tensor-core epilogues, split-tile scratch, statistics, pooled atomics, the elementwise kernels' loads and
+ * stores) against the extent of the tensor it belongs to.  A failed check skips the access and records
+ * FC_ERR_BOUNDS with a site number in the device status word; nothing traps.  FC_TESTING_BOUNDS_TRIP makes such a
+ * build believe that the main output is one row shorter than it is, to show the mechanism at work.
+ *
  * Threading.  fc_run may be called from several host threads.  The workspace set by
  * fc_set_workspace is shared by all calls: launches that use it (row reductions on a GEMM, CONV2D_NCHW) must not
  * overlap on the device.
@@ -90,7 +97,10 @@ typedef enum {
     FC_ERR_WORKSPACE = 6,     /* chain needs a workspace and none (or too small) was set      */
     FC_ERR_ARCH = 7,
     FC_ERR_CUDA = 8,          /* a CUDA runtime / driver call failed; see fc_last_error       */
-    FC_ERR_TIMEOUT = 9        /* a bounded device-side wait expired                           */
+    FC_ERR_TIMEOUT = 9,       /* a bounded device-side wait expired                           */
+    FC_ERR_BOUNDS = 10        /* debug build (libfc_debug.so, compiled with -DFC_DEBUG) only: an address that a kernel
+                                 computed for one of its tensors lay outside that tensor; the access was skipped and
+                                 fc_get_async_status reports this code (fc_last_error names the site)              */
 } fc_status;
 
 typedef enum {
@@ -307,6 +317,7 @@ int fc_version(void);
  */
 #define FC_TESTING_PANEL_STALL 0
 #define FC_TESTING_SPLIT_STALL 1
+#define FC_TESTING_BOUNDS_TRIP 2   /* debug build only: value 1 shortens the checked extent of the main output by one row */
 void fc_testing_set(int which, int value);
 
 #ifdef __cplusplus

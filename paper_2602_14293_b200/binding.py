@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(PKG, "libfc.so")
+# FC_LIBRARY selects another build of the same library (the bounds-checked libfc_debug.so); the default is the product
+LIB_PATH = os.environ.get("FC_LIBRARY") or os.path.join(PKG, "libfc.so")
 
 FC_F32, FC_BF16, FC_F16, FC_F8E4M3, FC_MXF8E4M3, FC_E8M0 = 0, 1, 2, 3, 4, 5
 _PRODUCER = {"elementwise": 0, "gemm_nt": 1, "conv2d_nhwc": 2, "conv2d_nchw": 3}
@@ -105,7 +106,7 @@ def fc_last_plan() -> str:
     return lib().fc_last_plan().decode()
 
 
-FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL = 0, 1
+FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL, FC_TESTING_BOUNDS_TRIP = 0, 1, 2
 
 
 def fc_testing_set(which: int, value: int) -> None:

@@ -9,6 +9,23 @@
 
 namespace fc {
 
+// Debug build (-DFC_DEBUG): FC_DBG_IN(ptr, nbytes, base, bytes, status, site) is true when [ptr, ptr + nbytes) lies
+// inside the tensor [base, base + bytes); otherwise it records FC_ERR_BOUNDS and the site in the status word and is
+// false, and the caller skips the access.  In the ordinary build it is the constant true and costs nothing.
+enum DbgSite { kSiteStore16 = 1, kSiteStoreRows = 2, kSiteSplitPark = 3, kSiteSplitMerge = 4, kSiteStats = 5, kSiteRowResult = 6,
+               kSitePoolAvg = 7, kSitePoolMax = 8, kSitePoolStage = 9, kSiteEwLoad = 10, kSiteEwStore = 11, kSiteEwResult = 12 };
+#ifdef FC_DEBUG
+__device__ __forceinline__ bool dbg_in(const void* ptr, long long nbytes, const void* base, long long bytes, int* status, int site) {
+    const long long off = (const char*) ptr - (const char*) base;
+    const bool ok = base != nullptr && off >= 0 && off + nbytes <= bytes;
+    if (!ok && status) atomicCAS(status, 0, FC_ERR_BOUNDS | (site << 8));
+    return ok;
+}
+#define FC_DBG_IN(ptr, nbytes, base, bytes, status, site) ::fc::dbg_in((ptr), (nbytes), (base), (bytes), (status), (site))
+#else
+#define FC_DBG_IN(ptr, nbytes, base, bytes, status, site) true
+#endif
+
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 

@@ -226,6 +226,8 @@ struct EwFastParams {
     int ragged;             // long rows whose length is no multiple of 8 (no per-column vectors): rows start anywhere, the
                             // aligned middle of each row goes in 16-byte chunks, up to 14 edge elements one by one
     int stash;              // row softmax: the row's exponentials wait in shared memory for the second pass
+    int* status;            // device status word (debug build's address checks)
+    long long dbg_trim;     // debug build: bytes by which the checks believe y to be shorter (testing)
     float pre_scale;        // a SCALE op in front of everything, folded into gamma (PRE is then always affine;
                             // vec0 == null means gamma = 1, vec1 == null means beta = 0)
 };
@@ -239,6 +241,18 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
     asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+
+// Debug build: the row kernels' streaming accesses, checked against the extents of x / the residual (M * N 16-bit
+// elements) and of y (the same, less what a test trimmed off); see FC_DBG_IN.
+#ifdef FC_DEBUG
+#define LD_STREAM(ptr, base, prm) (FC_DBG_IN((ptr), 16, (base), (prm).M * (long long) (prm).N * 2, (prm).status, kSiteEwLoad) ? ld_stream(ptr) : make_uint4(0u, 0u, 0u, 0u))
+#define ST_STREAM(ptr, v, prm) do { if (FC_DBG_IN((ptr), 16, (prm).y, (prm).M * (long long) (prm).N * 2 - (prm).dbg_trim, (prm).status, kSiteEwStore)) st_stream((ptr), (v)); } while (0)
+#define ST_RESULT(prm, row, value) do { if (FC_DBG_IN(&(prm).lse[row], 4, (prm).lse, (prm).M * 4, (prm).status, kSiteEwResult)) (prm).lse[row] = (value); } while (0)
+#else
+#define LD_STREAM(ptr, base, prm) ld_stream(ptr)
+#define ST_STREAM(ptr, v, prm) st_stream((ptr), (v))
+#define ST_RESULT(prm, row, value) (prm).lse[row] = (value)
+#endif
 
 constexpr int kPreNone = 0, kPreBias = 1, kPreAffine = 2;
 constexpr int kActNone = 0, kActRelu = 1, kActGeluPrecise = 2, kActGeluFast = 3;
@@ -370,7 +384,7 @@ __device__ __forceinline__ void ew_chunk(const uint4 xq, const uint4 rq, const f
         uint4 q;
         q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
         q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
-        st_stream(yr + c, q);
+        ST_STREAM(yr + c, q, prm);
     }
     if (LSE && red_kind >= FC_RED_ROW_SUM) {
         // ROW_SUM / ROW_MEAN / ROW_MAX: plain running sum and maximum
@@ -496,8 +510,8 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
             for (int g = 0; g < kInFlight; ++g) {
                 const int c = c0 + 32 * g;
                 if (c < chunks) {
-                    xv[g] = ld_stream(xr + c);
-                    if (RES) rv[g] = ld_stream(rr + c);
+                    xv[g] = LD_STREAM(xr + c, p.x, p);
+                    if (RES) rv[g] = LD_STREAM(rr + c, p.res, p);
                 }
             }
 #pragma unroll
@@ -515,7 +529,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                 run_m = fmaxf(run_m, __shfl_xor_sync(0xffffffffu, run_m, o));
             }
             if (lane == 0)
-                p.lse[row] = p.red_kind == FC_RED_ROW_MAX ? run_m : (p.red_kind == FC_RED_ROW_MEAN ? run_s / (float) N : run_s);
+                ST_RESULT(p, row, p.red_kind == FC_RED_ROW_MAX ? run_m : (p.red_kind == FC_RED_ROW_MEAN ? run_s / (float) N : run_s));
         } else if (LSE) {
             // merge the 32 per-lane pairs (log2 domain)
 #pragma unroll
@@ -549,7 +563,7 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                         uint4 o;
                         o.x = pack16x2(a.x, a.y, h); o.y = pack16x2(b.x, b.y, h);
                         o.z = pack16x2(cc.x, cc.y, h); o.w = pack16x2(d.x, d.y, h);
-                        st_stream(pr + c, o);
+                        ST_STREAM(pr + c, o, p);
                     }
                 } else {
                     for (int c0 = lane; c0 < chunks; c0 += 32 * kGroup) {
@@ -578,12 +592,12 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
                                 uint4 q;
                                 q.x = pack16x2(v[0].x, v[0].y, p.is_f16 != 0); q.y = pack16x2(v[1].x, v[1].y, p.is_f16 != 0);
                                 q.z = pack16x2(v[2].x, v[2].y, p.is_f16 != 0); q.w = pack16x2(v[3].x, v[3].y, p.is_f16 != 0);
-                                st_stream(pr + c, q);
+                                ST_STREAM(pr + c, q, p);
                             }
                         }
                     }
                 }
-            } else if (lane == 0) p.lse[row] = (run_m + log2f(run_s)) * kLn2;
+            } else if (lane == 0) ST_RESULT(p, row, (run_m + log2f(run_s)) * kLn2);
         }
     }
 }
@@ -622,8 +636,8 @@ __global__ void __launch_bounds__(kThreads, 4) ew_narrow_kernel(const EwFastPara
         for (int g = 0; g < kGroup; ++g) {
             const long long row = base + g * rows_per_warp + sub;
             if (row < p.M && c < chunks) {
-                xv[g] = ld_stream(p.x + row * chunks + c);
-                if (RES) rv[g] = ld_stream(p.res + row * chunks + c);
+                xv[g] = LD_STREAM(p.x + row * chunks + c, p.x, p);
+                if (RES) rv[g] = LD_STREAM(p.res + row * chunks + c, p.res, p);
             }
         }
 #pragma unroll
@@ -639,7 +653,7 @@ __global__ void __launch_bounds__(kThreads, 4) ew_narrow_kernel(const EwFastPara
                     uint4 q;
                     q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
                     q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
-                    st_stream(p.y + row * chunks + c, q);
+                    ST_STREAM(p.y + row * chunks + c, q, p);
                 }
                 const float cm = fmaxf(fmaxf(fmaxf(v[0].x, v[0].y), fmaxf(v[1].x, v[1].y)), fmaxf(fmaxf(v[2].x, v[2].y), fmaxf(v[3].x, v[3].y)));
                 if (plain) {
@@ -687,11 +701,11 @@ __global__ void __launch_bounds__(kThreads, 4) ew_narrow_kernel(const EwFastPara
                     uint4 q;
                     q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
                     q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
-                    st_stream(p.y + row * chunks + c, q);
+                    ST_STREAM(p.y + row * chunks + c, q, p);
                 }
             } else if (c == 0 && row < p.M) {
-                p.lse[row] = kind == FC_RED_ROW_LOGSUMEXP ? (m + log2f(sum)) * kLn2
-                           : kind == FC_RED_ROW_MAX ? m : (kind == FC_RED_ROW_MEAN ? sum / (float) N : sum);
+                ST_RESULT(p, row, kind == FC_RED_ROW_LOGSUMEXP ? (m + log2f(sum)) * kLn2
+                           : kind == FC_RED_ROW_MAX ? m : (kind == FC_RED_ROW_MEAN ? sum / (float) N : sum));
             }
         }
     }
@@ -747,8 +761,8 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(c
             for (int g = 0; g < kGroup; ++g) {
                 const int c = c0 + kThreads * g;
                 if (c < chunks) {
-                    xv[g] = ld_stream(xr + c);
-                    if (RES) rv[g] = ld_stream(rr + c);
+                    xv[g] = LD_STREAM(xr + c, p.x, p);
+                    if (RES) rv[g] = LD_STREAM(rr + c, p.res, p);
                 }
             }
 #pragma unroll
@@ -810,13 +824,13 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_longrow_kernel(c
                             uint4 q;
                             q.x = pack16x2(v[0].x, v[0].y, f16); q.y = pack16x2(v[1].x, v[1].y, f16);
                             q.z = pack16x2(v[2].x, v[2].y, f16); q.w = pack16x2(v[3].x, v[3].y, f16);
-                            st_stream(pr + c, q);
+                            ST_STREAM(pr + c, q, p);
                         }
                     }
                 }
             } else if (threadIdx.x == 0) {
-                p.lse[row] = kind == FC_RED_ROW_LOGSUMEXP ? (run_m + log2f(run_s)) * kLn2
-                           : kind == FC_RED_ROW_MAX ? run_m : (kind == FC_RED_ROW_MEAN ? run_s / (float) N : run_s);
+                ST_RESULT(p, row, kind == FC_RED_ROW_LOGSUMEXP ? (run_m + log2f(run_s)) * kLn2
+                           : kind == FC_RED_ROW_MAX ? run_m : (kind == FC_RED_ROW_MEAN ? run_s / (float) N : run_s));
             }
         }
     }
@@ -878,6 +892,7 @@ static bool match_fast(const EwParams& p, EwFastParams* f, int* pre, int* act, b
         if (p.reduce == FC_RED_NONE || (*act & kActPost) || !vec_ok) return false;
     }
     f->x = (const uint4*) p.x; f->y = (uint4*) p.y; f->lse = p.red; f->M = p.M; f->N = (int) p.N;
+    f->status = p.status; f->dbg_trim = p.dbg_trim;
     f->red_kind = p.reduce;
     f->is_f16 = p.x_dt == FC_F16;
     return true;

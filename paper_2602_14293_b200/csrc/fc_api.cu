@@ -16,7 +16,7 @@ __device__ int g_status_word;  // written by kernels when a bounded wait expires
 namespace {
 
 // testing switches (fc_testing_set): read on every call, written by tests only
-std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0};
+std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0}, g_bounds_trip{0};
 
 thread_local char t_err[512] = "";
 thread_local char t_plan[256] = "";
@@ -608,6 +608,8 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
     switch (plan.kind) {
         case Plan::EW: {
             EwParams p;
+            p.status = dev->status;
+            p.dbg_trim = g_bounds_trip.load(std::memory_order_relaxed) ? spec->N * (long long) dt_size(spec->out_dtype) : 0;
             p.x = inputs[0].ptr; p.x_dt = spec->in_dtype;
             p.y = plan.main_index >= 0 ? outputs[plan.main_index].ptr : nullptr;
             p.y_dt = spec->out_dtype;
@@ -638,6 +640,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             p.red = plan.red_index >= 0 ? (float*) outputs[plan.red_index].ptr : nullptr;
             p.red_kind = spec->reduce;
             p.status = dev->status;
+            p.dbg_trim = g_bounds_trip.load(std::memory_order_relaxed) ? spec->N * (long long) dt_size(spec->out_dtype) : 0;
             build_ops(spec, inputs, &p.ops);
             {
                 // keep about 32 MB of A rows (group_m panels of 256 rows) resident in L2 per sweep
@@ -1053,6 +1056,8 @@ fc_status fc_get_async_status(void* cuda_stream) {
         }
         const int zero = 0;
         if ((e = cudaMemcpy(dev->status, &zero, sizeof(int), cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy status");
+        if ((word & 0xff) == FC_ERR_BOUNDS)   // debug build: the site of the first failed address check rides in the upper bits
+            return fail(FC_ERR_BOUNDS, "a kernel computed an address outside one of its tensors (check site %d); the access was skipped", word >> 8);
         return fail((fc_status) word, "a bounded device-side wait expired");
     }
     return FC_OK;
@@ -1072,6 +1077,7 @@ const char* fc_status_string(fc_status s) {
         case FC_ERR_ARCH: return "FC_ERR_ARCH";
         case FC_ERR_CUDA: return "FC_ERR_CUDA";
         case FC_ERR_TIMEOUT: return "FC_ERR_TIMEOUT";
+        case FC_ERR_BOUNDS: return "FC_ERR_BOUNDS";
     }
     return "FC_ERR_?";
 }
@@ -1084,6 +1090,7 @@ int fc_version(void) { return FC_VERSION; }
 void fc_testing_set(int which, int value) {
     if (which == FC_TESTING_PANEL_STALL) g_inject_panel_stall.store(value);
     else if (which == FC_TESTING_SPLIT_STALL) g_inject_split_stall.store(value);
+    else if (which == FC_TESTING_BOUNDS_TRIP) g_bounds_trip.store(value);
 }
 
 }  // extern "C"

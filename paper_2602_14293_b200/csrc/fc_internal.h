@@ -47,6 +47,8 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // ---- launchers (defined one per .cu file); all enqueue on `stream` and return a cudaError_t ----
 struct EwParams {
+    int* status;                // device status word (written by the debug build's address checks only)
+    long long dbg_trim;         // debug build: bytes by which the checks believe the main output to be shorter (testing)
     const void* x; int x_dt;
     void* y; int y_dt;          // may be null when !store_main
     float* red;                 // row logsumexp out, or null
@@ -119,6 +121,7 @@ struct TcParams {
                                 // for that kernel before their first update of `out`, everything else starts at once
     int a_packed;               // mode 2: 1 = a k-block of A is eight 8-channel chunks, one per filter tap (Cin == 8)
     int* status;                // device status word
+    long long dbg_trim;         // debug build: bytes by which the checks believe the main output to be shorter (testing)
     int expect_extra;           // testing only: arrivals a wait expects beyond those that will come (mode 1: the panel
                                 // wait; other modes: the wait of a split tile's merging slice)
     // Split tiles (filled by the launcher when the scratch below is given and a split pays): tiles from

@@ -452,6 +452,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool precise = false;   // tanh.approx GELU is accurate to 6e-6 on sm_100a (see gelu_tanh)
         const bool out_vec = (reinterpret_cast<uintptr_t>(p.out) & 15) == 0 && (p.N & 7) == 0;
         const uint32_t tempty_leader = ptx::mapa(ptx::smem_u32(&ctrl->tempty[0]), 0);
+        // debug build: the main output's extent for the address checks of the stores
+        const DbgOut dbg_out = {kConv ? 0 : (long long) p.M * p.N * (p.out_dt == FC_F32 ? 4 : 2) - p.dbg_trim, p.status};
+        const long long dbg_stats_bytes = (long long) p.M * tiles_n * 8 * (MODE == 1 && p.two_pass ? 2 : 1);
+        (void) dbg_stats_bytes;
         if constexpr (kConv) {
             // the pooled output is zeroed by the kernel in front, which this one was allowed to overtake: only
             // these warps, the ones that update the output, wait for it (a no-op under an ordinary launch)
@@ -514,6 +518,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
                         ptx::tmem_wait_ld(ra);
                         ptx::tmem_wait_ld(rb);
+                        if (!FC_DBG_IN(mine + c * 4 * 32, 2 * 4 * 32 * 16 - 31 * 16, p.split_ws, (long long) kTcSplitUnits * 2 * BM * 256 * 4, p.status, kSiteSplitPark)) continue;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             __stcg(mine + (c * 4 + j) * 32, make_float4(__uint_as_float(ra[4 * j]), __uint_as_float(ra[4 * j + 1]), __uint_as_float(ra[4 * j + 2]), __uint_as_float(ra[4 * j + 3])));
@@ -558,6 +563,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (q == w.slice) continue;
                         const float4* src = p.split_ws + ((size_t) (w.v0 + q) * 2 + cta_rank) * kSliceF4 + (size_t) ws * kChunks * 128 + lane + c0 * 128;
                         float4 t[16];
+                        if (!FC_DBG_IN(src, 15 * 32 * 16 + 16, p.split_ws, (long long) kTcSplitUnits * 2 * BM * 256 * 4, p.status, kSiteSplitMerge)) continue;
 #pragma unroll
                         for (int i = 0; i < 16; ++i) t[i] = __ldcg(src + i * 32);
 #pragma unroll
@@ -599,14 +605,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
                             if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
                         } else if (m < p.M && n0 < p.N) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
                             if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                             else apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                         }
                     }
                     ptx::tmem_wait_ld(rb);
@@ -619,14 +625,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
                             if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
-                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
                         } else if (m < p.M && n0 < p.N) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
                             if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
                             else apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
-                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                         }
                     }
                 }
@@ -648,14 +654,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
                         if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
                     }
                     if (m < p.M && n0 < p.N) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
                         apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                        if (p.out && out_vec) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                        if (p.out && out_vec) store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                         if (rk == FC_RED_ROW_LOGSUMEXP || rk == FC_RED_ROW_MAX) {
                             float cm = -CUDART_INF_F;
 #pragma unroll
@@ -694,7 +700,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::bar_sync(1, kEpiThreads);
                 if (half == 0 && m < p.M) {
                     const float2 o = xchg[row];
-                    __stcg(&p.stats[m * tiles_n + nb], merge(run_m, run_s, o.x, o.y));
+                    if (FC_DBG_IN(&p.stats[m * tiles_n + nb], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
+                        __stcg(&p.stats[m * tiles_n + nb], merge(run_m, run_s, o.x, o.y));
                 }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
@@ -711,6 +718,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const float2 st = __ldcg(&p.stats[m * tiles_n + j]);
                         a = merge(a.x, a.y, st.x, st.y);
                     }
+                    if (FC_DBG_IN(&p.red[m], 4, p.red, (long long) p.M * 4, p.status, kSiteRowResult))
                     p.red[m] = rk == FC_RED_ROW_LOGSUMEXP ? (a.x + log2f(a.y)) * kLn2
                              : rk == FC_RED_ROW_MAX ? a.x
                              : rk == FC_RED_ROW_MEAN ? a.y / (float) p.N : a.y;
@@ -762,12 +770,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             v[2 * j + 1] = e.y;
                         }
                         if (!out_vec) {
-                            if (__all_sync(0xffffffffu, ok)) store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                            if (__all_sync(0xffffffffu, ok)) store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
                         } else if (m < p.M && ok) {
-                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                         }
                     });
-                    if (m < p.M) __stcg(&p.stats[(m * tiles_n + nb) * 2 + half], make_float2(mx, acc2.x + acc2.y));
+                    if (m < p.M && FC_DBG_IN(&p.stats[(m * tiles_n + nb) * 2 + half], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
+                        __stcg(&p.stats[(m * tiles_n + nb) * 2 + half], make_float2(mx, acc2.x + acc2.y));
                     release_buf();
                     continue;
                 }
@@ -805,7 +814,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (half == 0 && m < p.M) {
                     const float2 o = xchg[row];
                     const MaxSum a = ms_merge(MaxSum{mx, sm}, MaxSum{o.x, o.y});
-                    __stcg(&p.stats[m * tiles_n + nb], make_float2(a.m, a.s));
+                    if (FC_DBG_IN(&p.stats[m * tiles_n + nb], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
+                        __stcg(&p.stats[m * tiles_n + nb], make_float2(a.m, a.s));
                 }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
@@ -857,7 +867,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             v[2 * j] = t.x;
                             v[2 * j + 1] = t.y;
                         }
-                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane);
+                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
                     } else if (m < p.M && n0 < p.N && store && out_vec) {
                         float v[16];
 #pragma unroll
@@ -866,7 +876,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             v[2 * j] = t.x;
                             v[2 * j + 1] = t.y;
                         }
-                        store16(p.out, p.out_dt, out_vec, v, m, n0, p.N);
+                        store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                     }
                 });
             } else if (p.pool == 1) {
@@ -917,7 +927,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
                     if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) stage[lane * 17 + j] = v[j];
+                    for (int j = 0; j < 16; ++j)
+                        if (FC_DBG_IN(&stage[lane * 17 + j], 4, pool_stage, (long long) C::kPoolBytes, p.status, kSitePoolStage)) stage[lane * 17 + j] = v[j];
                     __syncwarp();
 #pragma unroll
                     for (int k = 0; k < kSlots; ++k) {
@@ -927,7 +938,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if ((code & 64u) && n0 + ch < p.N) {
                                 float x = stage[src * 17 + ch];
                                 if (code & 32u) x = fmaxf(x, stage[(src + 1) * 17 + ch]);
-                                atomicMax(out_u + (long long) slot_win[k] * p.N + n0 + ch, __float_as_uint(x) & 0x7fffffffu);
+                                if (FC_DBG_IN(out_u + (long long) slot_win[k] * p.N + n0 + ch, 4, p.out, (long long) p.batch * PH * PW * p.N * 4, p.status, kSitePoolMax))
+                                    atomicMax(out_u + (long long) slot_win[k] * p.N + n0 + ch, __float_as_uint(x) & 0x7fffffffu);
                             }
                         }
                     }
@@ -962,7 +974,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 16; ++j) { w[j] = my_img == img ? va[j] : 0.0f; w[16 + j] = my_img == img ? vb[j] : 0.0f; }
                         const float s = warp_transpose_sum(w, lane);
-                        if (n0 + lane < p.N) atomicAdd((float*) p.out + (long long) img * p.N + n0 + lane, s * p.inv_hw);
+                        if (n0 + lane < p.N && FC_DBG_IN((float*) p.out + (long long) img * p.N + n0 + lane, 4, p.out, (long long) p.batch * p.N * 4 - p.dbg_trim, p.status, kSitePoolAvg))
+                            atomicAdd((float*) p.out + (long long) img * p.N + n0 + lane, s * p.inv_hw);
                     }
                 }
             }

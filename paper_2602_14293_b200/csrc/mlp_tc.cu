@@ -229,7 +229,7 @@ mlp_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
                             for (int j = 0; j < 16; ++j) v[j] = 0.0f;
                         }
                         if (last) {
-                            if (m < p.M) store16(p.out, p.out_dt, out_vec, v, m, c0, width);
+                            if (m < p.M) store16(p.out, p.out_dt, out_vec, v, m, c0, width, DbgOut{(long long) p.M * width * (p.out_dt == FC_F32 ? 4 : 2), p.status});
                         } else {
                             // A-operand layout: k-block c0/64, row `row` of 128 bytes, 16-byte chunk j stored at j ^ (row & 7)
                             uint8_t* kb_base = act + (c0 >> 6) * kABytes + row * 128;

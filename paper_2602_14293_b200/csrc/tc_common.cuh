@@ -171,8 +171,19 @@ __device__ __forceinline__ void apply_ops16(float (&v)[16], const DevOps& ops, c
 }
 
 // 16 fp32 values of one row -> global memory as bf16 or fp32 (vector stores when aligned and in range)
+// (debug build: `dbg` = the output's extent in bytes and the status word; a store that would leave it is skipped)
+struct DbgOut {
+    long long bytes;
+    int* status;
+};
 __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, const float (&v)[16], long long m,
-                                        long long n0, long long N) {
+                                        long long n0, long long N, const DbgOut& dbg) {
+#ifdef FC_DEBUG
+    {
+        const long long esz = out_dt != FC_F32 ? 2 : 4, cols = N - n0 < 16 ? N - n0 : 16;
+        if (!FC_DBG_IN((const char*) out + (m * N + n0) * esz, cols * esz, out, dbg.bytes, dbg.status, kSiteStore16)) return;
+    }
+#endif
     if (out_dt != FC_F32) {
         const bool f16 = out_dt == FC_F16;
         unsigned short* o = (unsigned short*) out + m * N + n0;
@@ -227,7 +238,7 @@ __device__ __forceinline__ void store16(void* out, int out_dt, bool vec_ok, cons
 // values go through shared memory (`stage`: 32 x 17 floats of this warp) and are written two rows per
 // instruction, 16 consecutive elements each.  Every lane of the warp must call (`row_ok`: this lane's row exists).
 __device__ __forceinline__ void store16_rows(void* out, int out_dt, float* stage, const float (&v)[16], long long m_lane0,
-                                             long long M, long long n0, long long N, int lane) {
+                                             long long M, long long n0, long long N, int lane, const DbgOut& dbg) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) stage[lane * 17 + j] = v[j];
     __syncwarp();
@@ -237,7 +248,8 @@ __device__ __forceinline__ void store16_rows(void* out, int out_dt, float* stage
         for (int it = 0; it < 16; ++it) {
             const int r = 2 * it + (lane >> 4);
             const long long row = m_lane0 + r;
-            if (row < M) {
+            if (row < M && FC_DBG_IN((const char*) out + (row * N + n0 + c) * (out_dt == FC_F32 ? 4 : 2), out_dt == FC_F32 ? 4 : 2, out, dbg.bytes,
+                                     dbg.status, kSiteStoreRows)) {
                 const float x = stage[r * 17 + c];
                 if (out_dt == FC_F32) ((float*) out)[row * N + n0 + c] = x;
                 else ((unsigned short*) out)[row * N + n0 + c] = (unsigned short) (pack16x2(x, 0.0f, out_dt == FC_F16) & 0xffffu);
