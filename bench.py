@@ -473,6 +473,20 @@ def host_cost_us(step, kernel_ms, calls):
     return total / done * 1e6, done
 
 
+def host_floor_us(fc, calls=20000):
+    """What a call costs before any work is done: a chain that validation rejects at once, through the same ctypes
+    path (the rest of host_us_per_call is validation, planning and the CUDA launch calls themselves)."""
+    import ctypes
+    ch = wl.CONFIGS["C1"]()
+    spec = fc.make_spec(ch)
+    spec.version = 0                          # rejected before anything else is looked at
+    fn, ref = fc.lib().fc_run, ctypes.byref(spec)
+    t0 = time.perf_counter()
+    for _ in range(calls):
+        fn(ref, None, 0, None, 0, None)
+    return (time.perf_counter() - t0) / calls * 1e6
+
+
 def config_entry(fc, binding, key, ch, ins, sampler, flush_buf, peaks, peaks_src, with_eager, oracle_s):
     """One per_config entry: the timing protocol, roofline, clocks, host cost, eager context, oracle parity."""
     import torch
@@ -663,6 +677,7 @@ def main():
                                     0.0 if args.no_cpu_baseline else 3.0)
             del i2
             torch.cuda.empty_cache()
+        line["host_floor_us_per_call"] = host_floor_us(fc)
         line["targets"] = {"statement": "memory-bound chain >= 80 % of nominal HBM peak (8 TB/s); GEMM / conv chains >= 60 % of nominal dense "
                                         "bf16 peak (2250 TFLOP/s); every config within the oracle's tolerances and faster than eager",
                            "met": {k: v["target_met"] for k, v in per.items()},

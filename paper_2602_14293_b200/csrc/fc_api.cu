@@ -18,6 +18,7 @@ namespace {
 // testing switches (fc_testing_set): read on every call, written by tests only
 std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0}, g_bounds_trip{0};
 
+thread_local int t_device = 0;   // ordinal of the current device, noted by get_device at the top of every entry point
 thread_local char t_err[512] = "";
 thread_local char t_plan[256] = "";
 std::atomic<uint64_t> g_launches{0};
@@ -32,7 +33,7 @@ fc_status fail(fc_status s, const char* fmt, ...) {
 
 constexpr int kMaxDevices = 64;
 struct DeviceInfo {
-    bool ready = false;
+    std::atomic<bool> ready{false};   // set last, with release: a reader that sees it sees the fields below
     int cc_major = 0, num_sms = 0;
     int* status = nullptr;
     void* workspace = nullptr;
@@ -67,9 +68,15 @@ fc_status get_device(DeviceInfo** out, int* dev_out = nullptr) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(FC_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (dev < 0 || dev >= kMaxDevices) return fail(FC_ERR_CUDA, "device ordinal %d out of range", dev);
-    std::lock_guard<std::mutex> lk(g_mu);
     DeviceInfo& d = g_dev[dev];
-    if (!d.ready) {
+    t_device = dev;
+    if (d.ready.load(std::memory_order_acquire)) {   // every call but the first on a device: no lock
+        *out = &d;
+        if (dev_out) *dev_out = dev;
+        return FC_OK;
+    }
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!d.ready.load(std::memory_order_relaxed)) {
         if ((e = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
             (e = cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
             return fail(FC_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
@@ -89,7 +96,7 @@ fc_status get_device(DeviceInfo** out, int* dev_out = nullptr) {
                 return fail(FC_ERR_CUDA, "cuTensorMapEncodeIm2col entry point not available");
             g_encode_im2col = (EncodeIm2colFn) fn;
         }
-        d.ready = true;
+        d.ready.store(true, std::memory_order_release);
     }
     *out = &d;
     if (dev_out) *dev_out = dev;
@@ -480,30 +487,26 @@ struct MapKey {
     long long d[8];   // extents and the other parameters the encoding depends on
     bool operator==(const MapKey& o) const { return ptr == o.ptr && memcmp(d, o.d, sizeof(d)) == 0; }
 };
-struct MapCache {
+struct MapCache {   // one per host thread: no lock on the per-call path
     static constexpr int kSlots = 16;
     MapKey key[kSlots];
     CUtensorMap map[kSlots];
     bool used[kSlots] = {};
     int next = 0;
-    std::mutex mu;
     bool find(const MapKey& k, CUtensorMap* out) {
-        std::lock_guard<std::mutex> lk(mu);
         for (int i = 0; i < kSlots; ++i)
             if (used[i] && key[i] == k) { *out = map[i]; return true; }
         return false;
     }
     void put(const MapKey& k, const CUtensorMap& m) {
-        std::lock_guard<std::mutex> lk(mu);
         key[next] = k; map[next] = m; used[next] = true;
         next = (next + 1) % kSlots;
     }
 };
-MapCache g_maps;
+thread_local MapCache g_maps;
 
 fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long cols, int box_rows, int dt = FC_BF16) {
-    int dev = 0;
-    cudaGetDevice(&dev);
+    const int dev = t_device;
     const MapKey mk = {ptr, {2, rows, cols, box_rows, dt, dev, 0, 0}};
     if (g_maps.find(mk, tm)) return FC_OK;
     const cuuint64_t esize = dt == FC_F8E4M3 ? 1 : 2;
@@ -523,8 +526,7 @@ fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long 
 
 // Scale tiles of the block-scaled GEMM: rows of 128 words (512 bytes), one row per (128-row tile, k-block)
 fc_status encode_scale_tiles(CUtensorMap* tm, const void* ptr, long long tile_rows) {
-    int dev = 0;
-    cudaGetDevice(&dev);
+    const int dev = t_device;
     const MapKey mk = {ptr, {7, tile_rows, dev, 0, 0, 0, 0, 0}};
     if (g_maps.find(mk, tm)) return FC_OK;
     const cuuint64_t dims[2] = {128, (cuuint64_t) tile_rows};
@@ -547,8 +549,7 @@ bool packed_taps(const fc_chain_spec* s) { return s->Cin == 8; }
 // `packed`: copies of 8 channels x 128 pixels without swizzle (one column of 8 x 16-byte core matrices each), for
 // channel counts that do not fill 64-channel k-blocks; otherwise 64 channels x 128 pixels with 128-byte swizzle.
 fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr, bool packed) {
-    int dev = 0;
-    cudaGetDevice(&dev);
+    const int dev = t_device;
     const MapKey mk = {ptr, {packed ? 5 : 4, s->batch * 65536 + dev, s->H, s->W, s->Cin, s->R * 64 + s->S, s->stride * 64 + s->pad, s->in_dtype}};
     if (g_maps.find(mk, tm)) return FC_OK;
     const cuuint64_t dims[4] = {(cuuint64_t) s->Cin, (cuuint64_t) s->W, (cuuint64_t) s->H, (cuuint64_t) s->batch};

@@ -204,3 +204,64 @@ def test_collapse_is_chosen_only_for_linear_epilogues_without_main_output():
     assert not wl.collapses(wl.linear_row_reduce(64, 64, 64, ops=(("bias_n", 2), ("relu",))))
     assert not wl.collapses(wl.linear_row_reduce(64, 64, 64, store_main=True))
     assert not wl.collapses(wl.gemm_bias_scale_lse(64, 64, 64))
+
+
+def test_two_host_threads_keep_their_own_errors(fc):
+    """fc_run may be called from several host threads: the error text and the plan record are per thread, and the
+    shared state (device table, launch counter, per-device launcher state) is atomic or lock-guarded.  Two threads
+    hammer the entry points with different rejected chains and each must always read back its own message."""
+    import threading
+    L = fc.lib()
+    ch = wl.gemm_bias_gelu_scale_clamp(256, 256, 64)
+    good_in = _arr(fc, [_fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (256, 64), 1), _fake_tensor(fc, (256,), 1)])
+    good_out = _arr(fc, [_fake_tensor(fc, (256, 256), 1)])
+    errors = []
+
+    def worker(kind):
+        s = fc.make_spec(ch)
+        if kind == 0:
+            s.version = 99
+            want_status, want_text = 2, "version 99"
+        else:
+            s.K = 0
+            want_status, want_text = 4, "M, N, K must be >= 1"
+        for _ in range(3000):
+            st = _status(fc, s, good_in, good_out)
+            msg = L.fc_last_error().decode()
+            if st != want_status or want_text not in msg:
+                errors.append((kind, st, msg))
+                return
+            n = ctypes.c_size_t(0)
+            if L.fc_workspace_size(ctypes.byref(fc.make_spec(wl.CONFIGS["C4"]())), ctypes.byref(n)) != 0 or n.value == 0:
+                errors.append((kind, "workspace", n.value))
+                return
+
+    threads = [threading.Thread(target=worker, args=(k,)) for k in (0, 1)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors[:3]
+
+
+def test_block_scaled_spec_is_validated_on_the_host(fc):
+    """FC_MXF8E4M3: four producer inputs (elements and scales), K a multiple of 128, reduce NONE, workspace for the
+    scale tiles."""
+    ch = wl.gemm_mxf8_bias_gelu_scale_clamp(256, 384, 512)
+    s = fc.make_spec(ch)
+    assert fc.fc_workspace_size(s) == (2 + 3) * 4 * 512
+    F8, E8 = 3, 5
+    ins = [_fake_tensor(fc, (256, 512), F8), _fake_tensor(fc, (384, 512), F8), _fake_tensor(fc, (256, 16), E8), _fake_tensor(fc, (384, 16), E8),
+           _fake_tensor(fc, (384,), 1)]
+    out = _arr(fc, [_fake_tensor(fc, (256, 384), 1)])
+    bad = list(ins); bad[2] = _fake_tensor(fc, (256, 16), F8)              # scales must be FC_E8M0
+    assert _status(fc, s, _arr(fc, bad), out) == 2
+    bad = list(ins); bad[3] = _fake_tensor(fc, (384, 8), E8)               # one scale per 32 elements
+    assert _status(fc, s, _arr(fc, bad), out) == 4
+    assert _status(fc, s, _arr(fc, ins[:3]), out) == 2                      # too few inputs
+    s2 = fc.make_spec(wl.gemm_mxf8_bias_gelu_scale_clamp(256, 384, 96))
+    ins96 = [_fake_tensor(fc, (256, 96), F8), _fake_tensor(fc, (384, 96), F8), _fake_tensor(fc, (256, 3), E8), _fake_tensor(fc, (384, 3), E8),
+             _fake_tensor(fc, (384,), 1)]
+    assert _status(fc, s2, _arr(fc, ins96), out) == 5                       # K % 128
+    s3 = fc.make_spec(ch); s3.reduce = 2
+    assert _status(fc, s3, _arr(fc, ins), out) == 3
