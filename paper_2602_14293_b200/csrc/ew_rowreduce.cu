@@ -956,7 +956,12 @@ static cudaError_t launch_fast(const EwFastParams& f_in, bool lse, bool store, i
     long long ctas = (f.M + kWarps - 1) / kWarps;
     int per_sm = smem > 0 ? (int) ((227 * 1024) / (smem + 1024)) : 4;   // 228 KB per SM, 1 KB of it reserved per CTA
     per_sm = per_sm > 4 ? 4 : (per_sm < 1 ? 1 : per_sm);
-    if (ctas > (long long) num_sms * per_sm) ctas = (long long) num_sms * per_sm;
+    // Two CTAs per resident slot, except for the softmax form: the second half of the grid starts as the first
+    // finishes, which evens out the tail.  Measured back to back in one process, 16384 x 4096: the logsumexp chain
+    // 69.9 us with one CTA per slot, 67.95 with two, 69.3 with three (a stand-alone copy of the kernel: 592 CTAs 68.8,
+    // 740 74.2, 888 76.1, 1184 67.1, 1776 67.8, a CTA per 8 rows 68.1); the softmax chain 74.2 / 75.0 / 76.0.
+    const int per_slot = f.red_kind == FC_RED_ROW_SOFTMAX ? 1 : 2;
+    if (ctas > (long long) num_sms * per_sm * per_slot) ctas = (long long) num_sms * per_sm * per_slot;
     // the dynamic shared-memory limit of each instantiation is raised once per device, to the maximum
     static std::atomic<bool> raised[4][64];   // zero-initialised; set idempotently from any thread
     int dev = 0;
