@@ -1,14 +1,17 @@
-// Kernel (a): memory-bound elementwise chain with an optional row logsumexp, one pass over the data.
+// Kernel (a): memory-bound elementwise chain with an optional row reduction (logsumexp, softmax, sum, max, mean),
+// one pass over the data.
 //
-// One CTA walks whole rows.  Each thread owns 16-byte chunks (8 bf16 or 4 fp32 values) at a fixed
-// column stride, issues all its loads for a row (input and residual tensors) before any arithmetic,
-// applies the op list in registers, stores the result once, and folds the fp32 values (before the
-// output rounding) into a running (max, sum) pair.  Pairs are merged with warp shuffles and one
-// shared-memory exchange per row.
+// The row kernels give a warp a whole row (a lane per 16-byte chunk and several rows per warp for rows of at most 256
+// columns; a CTA per row from 10240 columns on).  A lane owns 16-byte chunks (8 values of 16 bits) at a fixed column
+// stride, issues the loads of four chunks of the input and of the residual tensor before any arithmetic, applies the
+// op list in packed fp32x2 registers, stores the result once, and folds the fp32 values (before the output rounding)
+// into a running (max, sum) pair that one shuffle merge per row finishes: no block barrier in the row loop.  The
+// per-column vectors are converted to fp32 once per CTA and kept in shared memory, de-interleaved so that the lanes'
+// float4 reads hit distinct banks.
 //
-// Two instantiations: a generic one (any op list, any N, any alignment) and a specialised one for
-// "affine -> tanh-GELU -> add tensor -> logsumexp" on bf16 with the per-column vectors held in
-// registers across rows.
+// Instantiations: the row kernels for op lists of the shape [scale] [bias | affine] [relu | gelu] [scale] [clamp]
+// [add tensor] on 16-bit rows with 16-byte aligned tensors, and a generic interpreter (any op list, any N, any
+// alignment, fp32 storage) that also serves chains without a reduction whose rows are shorter than 256 columns.
 #include <atomic>
 #include "dev_common.cuh"
 
