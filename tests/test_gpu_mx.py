@@ -102,3 +102,34 @@ def test_mx_rejections(fc):
     with pytest.raises(fc.FcError) as err:
         fc.run_chain(ch, ins)
     assert err.value.status == 4
+
+
+def test_mx_host_path_and_graph_replay(fc, orc):
+    """The same chain through fc_run_host (host tensors, staging buffer: all four producer inputs travel, also at a
+    size that other chains would cut into row chunks) and, on the device, captured into a CUDA graph and replayed
+    (three launches: two scale-tile kernels and the GEMM)."""
+    for M, N, K in ((300, 264, 384), (6000, 2048, 2048)):
+        ch = wl.gemm_mxf8_bias_gelu_scale_clamp(M, N, K)
+        ins = wl.make_inputs(ch, 8)
+        ref = orc.run_chain(ch, ins)["main"]
+        host_in = [fc.to_device(a, "cpu").pin_memory() for a in ins]
+        host_out = util.poison_(fc.binding.output_tensors(ch, "cpu", pinned=True))
+        spec = fc.make_spec(ch)
+        staging = torch.empty(fc.fc_staging_size(spec, host_in, host_out), dtype=torch.uint8, device="cuda")
+        fc.run_chain_host(ch, host_in, host_out, staging)
+        fc.fc_get_async_status()
+        util.check(host_out[0], ref, f"mx fc_run_host {M}x{N}x{K}")
+    dev = [t.cuda() for t in host_in]
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, dev, outs)                       # first call: one-time set-up outside the capture
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        fc.fc_run(spec, dev, outs, torch.cuda.current_stream())
+    for _ in range(2):
+        util.poison_(outs)
+        graph.replay()
+        torch.cuda.synchronize()
+        util.check(outs[0], ref, "mx graph replay")
+    fc.fc_get_async_status()
