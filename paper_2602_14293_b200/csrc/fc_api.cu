@@ -378,12 +378,18 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
     return FC_OK;
 }
 
-// fused form of an op list: [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]?
+// fused form of an op list: [scale]? [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]?
 void fused_from(const fc_op* ops, int n, const fc_tensor* in, FusedOps* out) {
     FusedOps& f = *out;
     memset(&f, 0, sizeof(f));
     f.scale = 1.0f;
+    f.pre_scale = 1.0f;
     int i = 0;
+    // a leading SCALE counts as the front one only when something that it cannot be merged with follows (a vector
+    // or an activation); a lone SCALE, or one in front of a clamp or a residual, is the ordinary post-activation one
+    if (n >= 2 && ops[0].kind == FC_OP_SCALE &&
+        (ops[1].kind == FC_OP_BIAS_N || ops[1].kind == FC_OP_AFFINE_N || ops[1].kind == FC_OP_RELU || ops[1].kind == FC_OP_GELU_TANH))
+        f.pre_scale = ops[i++].f0;
     if (i < n && (ops[i].kind == FC_OP_BIAS_N || ops[i].kind == FC_OP_AFFINE_N)) f.pre = ops[i++].kind == FC_OP_BIAS_N ? 1 : 2;
     if (i < n && (ops[i].kind == FC_OP_RELU || ops[i].kind == FC_OP_GELU_TANH)) f.act = ops[i++].kind == FC_OP_RELU ? 1 : 2;
     if (i < n && ops[i].kind == FC_OP_SCALE) f.scale = ops[i++].f0;

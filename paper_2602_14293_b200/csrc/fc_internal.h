@@ -18,7 +18,7 @@ struct DevOp {
     const void* p1;    // second vector (AFFINE_N)
 };
 
-// When the list has the shape [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]? the
+// When the list has the shape [scale]? [bias | affine]? [relu | gelu]? [scale]? [clamp]? [add tensor]? the
 // host also fills `fused`, which the tensor-core epilogues execute as straight packed-fp32x2 code
 // instead of interpreting the list (fewer issue slots, less energy next to a power-bound main loop).
 struct FusedOps {
@@ -28,6 +28,7 @@ struct FusedOps {
     int clamp;         // 0 / 1
     int res;           // 0 / 1: add tensor
     int res_dt;
+    float pre_scale;   // a SCALE in front of everything (1 if absent): undoing the scaling of 8-bit operands, 1/sqrt(d) in front of a softmax
     float scale;       // post-activation scale (1 if absent)
     float lo, hi;
     const void* res_ptr;

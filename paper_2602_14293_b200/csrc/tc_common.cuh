@@ -35,14 +35,20 @@ __device__ __forceinline__ void fused_ops16(float (&v)[16], const FusedOps& f, c
     float2 w[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) w[j] = make_float2(v[2 * j], v[2 * j + 1]);
+    const float2 ps = make_float2(f.pre_scale, f.pre_scale);
+    if (f.pre != 1 && f.pre_scale != 1.0f) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) w[j] = __fmul2_rn(w[j], ps);
+    }
     if (f.pre != 0) {
         const float4* a = reinterpret_cast<const float4*>(svec + col0);
         if (f.pre == 1) {
+            // (a SCALE in front of the bias rides in the same instruction: v * s + b)
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const float4 t = a[q];
-                w[2 * q] = __fadd2_rn(w[2 * q], make_float2(t.x, t.y));
-                w[2 * q + 1] = __fadd2_rn(w[2 * q + 1], make_float2(t.z, t.w));
+                w[2 * q] = __ffma2_rn(w[2 * q], ps, make_float2(t.x, t.y));
+                w[2 * q + 1] = __ffma2_rn(w[2 * q + 1], ps, make_float2(t.z, t.w));
             }
         } else {
             const float4* b = reinterpret_cast<const float4*>(svec + bn + col0);
