@@ -118,7 +118,7 @@ typedef enum {
                            v[m][n] = sum_j 2^(SA[m][j] - 127) 2^(SB[n][j] - 127) sum_{k = 32 j .. 32 j + 31} A[m][k] B[n][k].
                          K a multiple of 128, all four tensors 16-byte aligned.  The scales are first rewritten into the
                          tensor cores' tile order in the workspace (two small launches; fc_workspace_size reports the bytes:
-                         (ceil(M/128) + ceil(N/128)) * K/128 * 512).  Ops and outputs as for the other 8-bit GEMM; vector and
+                         (ceil(M/128) + 2 ceil(N/240)) * K/128 * 512, for N <= 128: (ceil(M/128) + 1) * K/128 * 512).  Ops and outputs as for the other 8-bit GEMM; vector and
                          tensor operands of ops are inputs[4..]. */
     FC_E8M0 = 5       /* a scale of FC_MXF8E4M3: one byte e meaning 2^(e - 127); 255 is NaN and must not occur */
 } fc_dtype;

@@ -531,13 +531,13 @@ fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long 
 }
 
 // Scale tiles of the block-scaled GEMM: rows of 128 words (512 bytes), one row per (128-row tile, k-block)
-fc_status encode_scale_tiles(CUtensorMap* tm, const void* ptr, long long tile_rows) {
+fc_status encode_scale_tiles(CUtensorMap* tm, const void* ptr, long long tile_rows, int box_rows) {
     const int dev = t_device;
-    const MapKey mk = {ptr, {7, tile_rows, dev, 0, 0, 0, 0, 0}};
+    const MapKey mk = {ptr, {7, tile_rows, dev, box_rows, 0, 0, 0, 0}};
     if (g_maps.find(mk, tm)) return FC_OK;
     const cuuint64_t dims[2] = {128, (cuuint64_t) tile_rows};
     const cuuint64_t strides[1] = {512};
-    const cuuint32_t box[2] = {128, 1};
+    const cuuint32_t box[2] = {128, (cuuint32_t) box_rows};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -694,7 +694,8 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             break;
         }
         case Plan::TC_MX: {
-            const size_t sa_bytes = (scale_tiles_bytes(spec->M, spec->K) + 255) / 256 * 256, sb_bytes = scale_tiles_bytes(spec->N, spec->K);
+            const int bn = mx_tile_width(spec->N), parts = (bn + 127) / 128;
+            const size_t sa_bytes = (scale_tiles_bytes(spec->M, spec->K, 128) + 255) / 256 * 256, sb_bytes = scale_tiles_bytes(spec->N, spec->K, bn);
             if (!dev->workspace || dev->workspace_bytes < sa_bytes + sb_bytes)
                 return fail(FC_ERR_WORKSPACE, "block-scaled operands need a %zu-byte workspace (fc_set_workspace); have %zu", sa_bytes + sb_bytes, dev->workspace_bytes);
             {   // the scale tiles overwrite whatever counters a previous layout kept here
@@ -703,8 +704,8 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             }
             void* sa_tiles = dev->workspace;
             void* sb_tiles = (char*) dev->workspace + sa_bytes;
-            if ((e = launch_scale_tiles(inputs[2].ptr, sa_tiles, spec->M, spec->K, false, stream, &launches)) != cudaSuccess) return cuda_fail(e, "scale-tile kernel launch");
-            if ((e = launch_scale_tiles(inputs[3].ptr, sb_tiles, spec->N, spec->K, true, stream, &launches)) != cudaSuccess) return cuda_fail(e, "scale-tile kernel launch");
+            if ((e = launch_scale_tiles(inputs[2].ptr, sa_tiles, spec->M, spec->K, 128, false, stream, &launches)) != cudaSuccess) return cuda_fail(e, "scale-tile kernel launch");
+            if ((e = launch_scale_tiles(inputs[3].ptr, sb_tiles, spec->N, spec->K, bn, true, stream, &launches)) != cudaSuccess) return cuda_fail(e, "scale-tile kernel launch");
             TcParams p;
             memset(&p, 0, sizeof(p));
             p.mode = 6;
@@ -720,9 +721,9 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             }
             CUtensorMap tmA, tmB, tmSA, tmSB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, FC_F8E4M3))) return st;
-            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, 64, FC_F8E4M3))) return st;   // 256 x 128 tiles: each CTA of a pair loads 64 rows of B
-            if ((st = encode_scale_tiles(&tmSA, sa_tiles, (long long) ((spec->M + 127) / 128) * (spec->K / 128)))) return st;
-            if ((st = encode_scale_tiles(&tmSB, sb_tiles, (long long) ((spec->N + 127) / 128) * (spec->K / 128)))) return st;
+            if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, FC_F8E4M3))) return st;   // each CTA of a pair loads half of the tile's rows of B
+            if ((st = encode_scale_tiles(&tmSA, sa_tiles, (long long) ((spec->M + 127) / 128) * (spec->K / 128), 1))) return st;
+            if ((st = encode_scale_tiles(&tmSB, sb_tiles, (long long) ((spec->N + bn - 1) / bn) * (spec->K / 128) * parts, parts))) return st;
             e = launch_gemm_tc_mx(p, tmA, tmB, tmSA, tmSB, dev->num_sms, stream, &launches);
             break;
         }
@@ -984,7 +985,7 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     if ((st = validate_spec(spec, &plan))) return st;
     *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? reduction_workspace_bytes(plan.kind == Plan::TC_SOFTMAX, spec->M, spec->N)
            : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K)
-           : plan.kind == Plan::TC_MX ? (spec->K % 128 ? 0 : (scale_tiles_bytes(spec->M, spec->K) + 255) / 256 * 256 + scale_tiles_bytes(spec->N, spec->K))
+           : plan.kind == Plan::TC_MX ? (spec->K % 128 ? 0 : (scale_tiles_bytes(spec->M, spec->K, 128) + 255) / 256 * 256 + scale_tiles_bytes(spec->N, spec->K, mx_tile_width(spec->N)))
            : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     return FC_OK;
 }
@@ -1010,7 +1011,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     if (plan.kind == Plan::GEMM_F32) { snprintf(text, capacity, "kernel=gemm_f32"); return FC_OK; }
     if (plan.kind == Plan::GEMM_COLLAPSE) { snprintf(text, capacity, "kernel=collapse"); return FC_OK; }
     if (plan.kind == Plan::TC_MLP) { snprintf(text, capacity, "kernel=mlp_tc"); return FC_OK; }
-    if (plan.kind == Plan::TC_MX) { snprintf(text, capacity, "kernel=gemm_tc mode=6 bn=128"); return FC_OK; }
+    if (plan.kind == Plan::TC_MX) { snprintf(text, capacity, "kernel=gemm_tc mode=6 bn=%d", mx_tile_width(spec->N)); return FC_OK; }
     DeviceInfo* dev;
     if ((st = get_device(&dev))) return st;
     TcParams p;

@@ -137,16 +137,19 @@ constexpr size_t kTcSplitCounterBytes = 1024;
 constexpr size_t kTcSplitBytes = kTcSplitCounterBytes + (size_t) kTcSplitUnits * 2 * 128 * 256 * 4;
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                            int bn, int num_sms, cudaStream_t stream, int* launches);
-// Mode 6: `tmSA` / `tmSB` map the scale tiles written by launch_scale_tiles (rows of 128 words, one row per
-// 128-row tile and 128-element k-block).
+// Mode 6: `tmSA` / `tmSB` map the scale tiles written by launch_scale_tiles (rows of 128 words: one row per 128-row
+// tile of A and k-block; one or two rows per column tile of B and k-block).  Column tiles are mx_tile_width(N) wide.
 cudaError_t launch_gemm_tc_mx(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
                               const CUtensorMap& tmSB, int num_sms, cudaStream_t stream, int* launches);
 // E8M0 scales [rows][K/32] -> tiles of 512 bytes per (128 rows, 128 elements of K), in the order the tensor core's
 // scale columns want them: byte (r % 32) * 16 + (r / 32) * 4 + j holds the scale of row r of the tile and the j-th
-// block of 32 elements; rows past `rows` get the scale 1.  K a multiple of 128.  `beside_previous` as above.
-cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, long long K, bool beside_previous, cudaStream_t stream,
-                               int* launches);
-size_t scale_tiles_bytes(long long rows, long long K);
+// block of 32 elements.  Rows are grouped into row tiles of `tile_rows` (128 for A; the GEMM's column-tile width for B,
+// 240 or 128), each ceil(tile_rows / 128) consecutive 512-byte tiles per k-block; positions without a row get the
+// scale 1.  K a multiple of 128.  `beside_previous` as above.
+cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, long long K, int tile_rows, bool beside_previous,
+                               cudaStream_t stream, int* launches);
+size_t scale_tiles_bytes(long long rows, long long K, int tile_rows);
+inline int mx_tile_width(long long N) { return N <= 128 ? 128 : 240; }   // column-tile width of the block-scaled GEMM
 size_t gemm_tc_smem_bytes(int bn);
 
 // Back-to-back linear layers kept on chip (mlp_tc.cu): layer l maps width[l-1] (K0 for l = 0) to width[l]

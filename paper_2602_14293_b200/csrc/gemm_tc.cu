@@ -21,8 +21,10 @@
 //           tile's 128 columns x 4 blocks) arrive with the operands (two more TMA loads from scale tiles that a
 //           layout kernel has written, see launch_scale_tiles), tcgen05.cp moves them into four tensor-memory
 //           columns each in front of the k-block's four MMAs, and MMA j names byte j of those columns.  Measured
-//           layout: row r of the tile reads byte (r % 32) * 16 + (r / 32) * 4 + j of the 512.  Tiles are 256 x 128
-//           (two accumulator buffers and the scale columns must share the 512 columns of tensor memory).
+//           layout: row r of the tile reads byte (r % 32) * 16 + (r / 32) * 4 + j of the 512; a B tile wider than 128
+//           columns takes one such 512-byte tile (four more tensor-memory columns) per 128 columns.  Tiles are
+//           256 x 240: two accumulator buffers of 240 columns and 12 scale columns share the 512 columns of tensor
+//           memory (256 x 128 for N <= 128).  The epilogue's two warp groups take columns 0..127 and 128..239.
 //
 // Work unit: a 256 x BN output tile owned by a PAIR of CTAs on neighbouring SMs (cluster of 2,
 // tcgen05 cta_group::2).  Each CTA loads its own 128 rows of A and HALF of the B tile, so a k-block
@@ -85,13 +87,16 @@ struct Cfg {
     static constexpr int kABytes = BM * BK * 2;
     static constexpr int kBBytes = (BN / 2) * BK * 2;   // this CTA's half of the B tile
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = BN == 256 ? 6 : 8;
+    static constexpr int kStages = BN >= 240 ? 6 : 8;
     static constexpr int kTmemCols = 2 * BN;
     static constexpr int kVecBytes = 2 * kMaxVecSlots * BN * 4;   // double-buffered per-tile vector slices
     static constexpr int kCtrlBytes = 256;
     static constexpr int kPoolBytes = 8 * 32 * 17 * 4;   // max-pool: 32 pixels x 16 channels (+1 pad) per epilogue warp
     static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024 + kPoolBytes + 1024;  // exchange, pool staging, alignment slack
-    static constexpr int kScaleBytes = kStages * 1024;   // mode 6: a tile of A scales and one of B scales per stage, behind everything else
+    // mode 6: per stage a 512-byte tile of A scales (this CTA's 128 rows) and one of B scales per 128 columns of the tile
+    static constexpr int kScaleStage = 512 + 512 * ((BN + 127) / 128);
+    static constexpr int kScaleBytes = kStages * kScaleStage;   // behind everything else
+    static constexpr int kColHalf = BN == 240 ? 128 : BN / 2;   // columns of the first of the two epilogue warp groups
 };
 
 struct Ctrl {
@@ -295,12 +300,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // peer copy may land before the expectation is posted: the phase cannot complete before
                     // the leader's arrival, and the peer starts the next phase only after the leader's MMAs
                     // of this one (the commit that frees the stage) are done.
-                    if (leader) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->full[s]), 2 * (C::kStageBytes + (kMx ? 1024 : 0)));
+                    if (leader) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->full[s]), 2 * (C::kStageBytes + (kMx ? C::kScaleStage : 0)));
                     if constexpr (kMx) {
-                        // the scales of this k-block: this CTA's 128 rows of A, the tile's 128 columns of B
-                        const uint32_t sc = ptx::smem_u32(scale_ring) + s * 1024;
+                        // the scales of this k-block: this CTA's 128 rows of A, the tile's columns of B (one box of one or two tiles)
+                        const uint32_t sc = ptx::smem_u32(scale_ring) + s * C::kScaleStage;
                         ptx::tma_load_2d_pair(sc, &tmSA, 0, (mb2 * 2 + (int) cta_rank) * num_kb + kb, full);
-                        ptx::tma_load_2d_pair(sc + 512, &tmSB, 0, nb * num_kb + kb, full);
+                        ptx::tma_load_2d_pair(sc + 512, &tmSB, 0, (nb * num_kb + kb) * ((BN + 127) / 128), full);
                     }
                     if constexpr (MODE == 4) {
                         // eight copies of 128 pixels x 8 channels, each one column of core matrices (2 KB)
@@ -383,16 +388,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else if constexpr (kMx) {
                         // scales into tensor memory (the copies and the MMAs run in the order they are issued), then four
                         // MMAs of 32 elements along K, MMA j with byte j of the scale columns
-                        const uint32_t sc = ptx::smem_u32(scale_ring) + s * 1024;
-                        ptx::tc_cp_32x128b_pair(tmem_base + 2 * BN, ptx::smem_desc_k_plain(sc, 16, 128));
-                        ptx::tc_cp_32x128b_pair(tmem_base + 2 * BN + 4, ptx::smem_desc_k_plain(sc + 512, 16, 128));
+                        const uint32_t sc = ptx::smem_u32(scale_ring) + s * C::kScaleStage;
+                        const uint32_t t_sfa = tmem_base + 2 * BN, t_sfb = t_sfa + 4;
+                        ptx::tc_cp_32x128b_pair(t_sfa, ptx::smem_desc_k_plain(sc, 16, 128));
+#pragma unroll
+                        for (int t = 0; t < (BN + 127) / 128; ++t)
+                            ptx::tc_cp_32x128b_pair(t_sfb + 4 * t, ptx::smem_desc_k_plain(sc + 512 + 512 * t, 16, 128));
                         const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);
                         const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
-                        ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo, b_lo, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, 0, 0), tmem_base + 2 * BN, tmem_base + 2 * BN + 4, acc0);
+                        ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo, b_lo, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, 0, 0), t_sfa, t_sfb, acc0);
 #pragma unroll
                         for (int k = 1; k < 4; ++k)
-                            ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, (uint32_t) k, (uint32_t) k), tmem_base + 2 * BN,
-                                                     tmem_base + 2 * BN + 4, 1u);
+                            ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, (uint32_t) k, (uint32_t) k), t_sfa, t_sfb, 1u);
                     } else {
                         const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);   // stage s, A tile; B follows kABytes further on
                         const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
@@ -487,8 +494,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ptx::bar_sync(2, kEpiThreads);
             if (!*(volatile int*) &ctrl->epi_ok[buf]) break;
             ptx::tc_fence_after();
-            constexpr int kChunks = BN / 32;           // 16-column chunks per thread (half a tile row)
-            const int col_half = half * (BN / 2);
+            constexpr int kChunks = C::kColHalf / 16;  // 16-column chunks per thread (half a tile row; 240-column tiles: 8 and 7)
+            const int col_half = half * C::kColHalf;
+            const int n_lim = min(p.N, n_tile + BN);   // first column that is not this tile's
             const uint32_t tacc = tmem_base + buf * BN + col_half + lane_addr;
             const long long m = (long long) mb * BM + row;
             const int n_half = n_tile + col_half;
@@ -599,14 +607,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
                     {
                         const int n0 = n_half + c * 16;
-                        if (!out_vec && n0 < p.N) {
+                        if (!out_vec && n0 < n_lim) {
                             // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
                             if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                             store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
-                        } else if (m < p.M && n0 < p.N) {
+                        } else if (m < p.M && n0 < n_lim) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
@@ -619,14 +627,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
                     {
                         const int n0 = n_half + (c + 1) * 16;
-                        if (!out_vec && n0 < p.N) {
+                        if (!out_vec && n0 < n_lim) {
                             // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
                             if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
                             store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
-                        } else if (m < p.M && n0 < p.N) {
+                        } else if (m < p.M && n0 < n_lim) {
                             float v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
@@ -1135,7 +1143,8 @@ cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUte
 cudaError_t launch_gemm_tc_mx(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
                               const CUtensorMap& tmSB, int num_sms, cudaStream_t stream, int* launches) {
     *launches += 1;
-    return launch_one<128, 6>(p, &tmA, &tmB, num_sms, stream, nullptr, &tmSA, &tmSB);
+    return p.N <= 128 ? launch_one<128, 6>(p, &tmA, &tmB, num_sms, stream, nullptr, &tmSA, &tmSB)
+                      : launch_one<240, 6>(p, &tmA, &tmB, num_sms, stream, nullptr, &tmSA, &tmSB);
 }
 
 cudaError_t plan_gemm_tc(const TcParams& p, int bn, int num_sms, TcPlan* plan) {

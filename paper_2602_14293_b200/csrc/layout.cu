@@ -108,18 +108,24 @@ __global__ void __launch_bounds__(256) zero_fill_kernel(uint32_t* ptr, size_t wo
     }
 }
 
-// One thread per (row of a 128-row tile, four k-blocks): reads the row's 16 scale bytes of those k-blocks and writes
-// one word into each of their four tiles.
+// One thread per (position of a scale tile, four k-blocks): reads the 16 scale bytes of its row for those k-blocks and
+// writes one word into each of their four tiles.  A tile of `tile_rows` rows (128 for A, the GEMM's column-tile width for
+// B) is ceil(tile_rows / 128) consecutive 512-byte tiles; positions that stand for no row get the scale 1.
 __global__ void __launch_bounds__(256) scale_tiles_kernel(const uint8_t* __restrict__ scales, uint32_t* __restrict__ tiles, long long rows,
-                                                          int blocks32, int num_kb, long long padded_rows) {
+                                                          int blocks32, int num_kb, int tile_rows, long long positions) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int groups = (num_kb + 3) >> 2;
+    const int parts = (tile_rows + 127) >> 7;            // 512-byte tiles per row tile
     const long long idx = (long long) blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= padded_rows * groups) return;
-    const long long r = idx / groups;
-    const int g = (int) (idx - r * groups);
-    uint32_t w[4] = {0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu};   // scale 1 for rows that do not exist
-    if (r < rows) {
+    if (idx >= positions * groups) return;
+    const long long pos = idx / groups;                  // (row tile, part, row within the part)
+    const int g = (int) (idx - pos * groups);
+    const long long tile = pos / (parts * 128);
+    const int within = (int) (pos - tile * (parts * 128)), part = within >> 7, rr = within & 127;
+    const int in_tile = part * 128 + rr;
+    const long long r = tile * tile_rows + in_tile;
+    uint32_t w[4] = {0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu};   // scale 1 where there is no row
+    if (in_tile < tile_rows && r < rows) {
         const uint8_t* src = scales + r * blocks32 + 16 * g;
         if (16 * g + 16 <= blocks32 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
             const uint4 q = *reinterpret_cast<const uint4*>(src);
@@ -129,22 +135,23 @@ __global__ void __launch_bounds__(256) scale_tiles_kernel(const uint8_t* __restr
                 if (16 * g + 4 * i + 4 <= blocks32) w[i] = (uint32_t) src[4 * i] | (uint32_t) src[4 * i + 1] << 8 | (uint32_t) src[4 * i + 2] << 16 | (uint32_t) src[4 * i + 3] << 24;
         }
     }
-    const long long tile = r >> 7;
-    const int rr = (int) (r & 127), word = (rr & 31) * 4 + (rr >> 5);
+    const int word = (rr & 31) * 4 + (rr >> 5);
     for (int i = 0; i < 4; ++i) {
         const int kb = 4 * g + i;
-        if (kb < num_kb) tiles[(tile * num_kb + kb) * 128 + word] = w[i];
+        if (kb < num_kb) tiles[((tile * num_kb + kb) * parts + part) * 128 + word] = w[i];
     }
 }
 
 }  // namespace
 
-size_t scale_tiles_bytes(long long rows, long long K) { return (size_t) ((rows + 127) / 128) * (size_t) (K / 128) * 512; }
+size_t scale_tiles_bytes(long long rows, long long K, int tile_rows) {
+    return (size_t) ((rows + tile_rows - 1) / tile_rows) * (size_t) ((tile_rows + 127) / 128) * (size_t) (K / 128) * 512;
+}
 
-cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, long long K, bool beside_previous, cudaStream_t stream,
-                               int* launches) {
+cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, long long K, int tile_rows, bool beside_previous,
+                               cudaStream_t stream, int* launches) {
     const int num_kb = (int) (K / 128), groups = (num_kb + 3) / 4;
-    const long long padded = (rows + 127) / 128 * 128, total = padded * groups;
+    const long long positions = (rows + tile_rows - 1) / tile_rows * ((tile_rows + 127) / 128) * 128, total = positions * groups;
     if (K % 128 || total > 0x7fffffffLL * 256) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned) ((total + 255) / 256));
@@ -157,7 +164,7 @@ cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, 
     cfg.numAttrs = beside_previous ? 1 : 0;
     note_kernel("scale_tiles");
     ++*launches;
-    return cudaLaunchKernelEx(&cfg, scale_tiles_kernel, (const uint8_t*) scales, (uint32_t*) tiles, rows, (int) (K / 32), num_kb, padded);
+    return cudaLaunchKernelEx(&cfg, scale_tiles_kernel, (const uint8_t*) scales, (uint32_t*) tiles, rows, (int) (K / 32), num_kb, tile_rows, positions);
 }
 
 cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches) {

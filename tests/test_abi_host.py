@@ -249,7 +249,7 @@ def test_block_scaled_spec_is_validated_on_the_host(fc):
     scale tiles."""
     ch = wl.gemm_mxf8_bias_gelu_scale_clamp(256, 384, 512)
     s = fc.make_spec(ch)
-    assert fc.fc_workspace_size(s) == (2 + 3) * 4 * 512
+    assert fc.fc_workspace_size(s) == (2 + 2 * 2) * 4 * 512     # A: two 128-row tiles; B: two 240-column tiles of two 512-byte parts each
     F8, E8 = 3, 5
     ins = [_fake_tensor(fc, (256, 512), F8), _fake_tensor(fc, (384, 512), F8), _fake_tensor(fc, (256, 16), E8), _fake_tensor(fc, (384, 16), E8),
            _fake_tensor(fc, (384,), 1)]
