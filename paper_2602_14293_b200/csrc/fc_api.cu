@@ -430,25 +430,59 @@ size_t panel_counter_bytes(long long M) {
     return ((size_t) panels * 4 + 255) / 256 * 256;
 }
 
-// Column-tile width of the GEMM kernels: 256, except that a small GEMM (modes 0 and 3, 256-wide tiles on at most
-// half of the SM pairs) takes 128-wide tiles where this cost model says so.  Such a call is one round of tiles,
-// so its time is the critical tile's: main loop (of the merging slice, when tiles are cut along K) + epilogue
-// + merge.  Measured, in microseconds: a k-block 0.33 (256 wide) / 0.30 (128 wide; 24 instead of 32 KB), the
-// epilogue 6 / 3, merging a split tile 8 / 4.4.  128 x 1024 x 1024: 13.7 -> 11.2; 256 x 4096 x 4096: 23.0 -> 20.1;
-// 16 x 8192 x 8192 stays at 256 (37 against 45).  `p` has its split scratch attached already.
-int gemm_tile_width(const TcParams& p, const fc_chain_spec* s, int num_sms) {
-    if (p.mode == 1) return kSoftmaxBN;
-    if (s->N <= 128) return 128;
-    const long long tiles = ((s->M + 255) / 256) * ((s->N + 255) / 256);
-    if ((p.mode != 0 && p.mode != 3) || 2 * tiles > num_sms / 2) return 256;
-    auto cost = [&](int bn) -> double {
+// Column-tile width of the GEMM kernels (modes 0, 1, 3), and for the row softmax the choice between its two forms.
+// Small GEMMs (modes 0 and 3, 256-wide tiles on at most half of the SM pairs) take 128-wide tiles where this
+// cost model says so.  Such a call is one round of tiles, so its time is the critical tile's: main loop (of the
+// merging slice, when tiles are cut along K) + epilogue + merge.  Measured, in microseconds: a k-block 0.33
+// (256 wide) / 0.30 (128 wide; 24 instead of 32 KB), the epilogue 6 / 3, merging a split tile 8 / 4.4.
+// 128 x 1024 x 1024: 13.7 -> 11.2; 256 x 4096 x 4096: 23.0 -> 20.1; 16 x 8192 x 8192 stays at 256 (37 against 45).
+// Everything else is rounds of tiles whose main loops the tensor pipe bounds, so the time goes with
+// rounds x tile width: 240-column tiles where that product is smaller (4096 columns: 18 tiles per panel, 288
+// tiles = 4 rounds on 72 pairs x 240 against 4 rounds x 256).  `p` has its split scratch attached already.
+int gemm_tile_width(TcParams& p, const fc_chain_spec* s, int num_sms) {
+    if (p.mode == 1) {
+        // Row softmax over more tiles per panel than the pairs' accumulator buffers can hold until the panel is
+        // complete (two per pair; with a margin: 64 tiles = 16384 columns) cannot wait across tiles: a second,
+        // memory-bound kernel finishes the rows.  The same two-kernel form is also chosen where it is faster.
+        // The single pass wins where it was built for (rows of up to 4096 columns and a long contraction: 4096^3 106
+        // against 118 us); its panel-by-panel order streams B once per panel and its epilogue waits for the
+        // panel, which loses from 8192 columns on and for short contractions (8192 x 16384 x 4096: 1208
+        // against 838 us; 16384 x 16384 x 1024: 2024 against 877 us).
+        const int tiles_n = (int) ((s->N + kSoftmaxBN - 1) / kSoftmaxBN);
         TcPlan tp;
-        if (plan_gemm_tc(p, bn, num_sms, &tp) != cudaSuccess) return 1e30;
-        const bool cut = tp.split > 1;
-        const int kb = cut ? tp.num_kb - tp.split_kb * (tp.split - 1) : tp.num_kb;
-        return bn == 256 ? kb * 0.33 + 6.0 + (cut ? 8.0 : 0.0) : kb * 0.30 + 3.0 + (cut ? 4.4 : 0.0);
+        p.two_pass = false;
+        // (never more tiles per panel than SM pairs take part, whatever the device offers)
+        p.two_pass = plan_gemm_tc(p, kSoftmaxBN, num_sms, &tp) != cudaSuccess || tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs ||
+                     tiles_n > kSoftmaxOnePassBestTiles || s->K < 4096;
+        if (p.two_pass) return kSoftmaxBN;
+    } else if (p.mode != 0 && p.mode != 3) {
+        return 256;
+    } else if (s->N <= 128) {
+        return 128;
+    }
+    const long long tiles = ((s->M + 255) / 256) * ((s->N + 255) / 256);
+    if (2 * tiles <= num_sms / 2) {
+        if (p.mode == 1) return kSoftmaxBN;
+        auto cost = [&](int bn) -> double {
+            TcPlan tp;
+            if (plan_gemm_tc(p, bn, num_sms, &tp) != cudaSuccess) return 1e30;
+            const bool cut = tp.split > 1;
+            const int kb = cut ? tp.num_kb - tp.split_kb * (tp.split - 1) : tp.num_kb;
+            return bn == 256 ? kb * 0.33 + 6.0 + (cut ? 8.0 : 0.0) : kb * 0.30 + 3.0 + (cut ? 4.4 : 0.0);
+        };
+        return cost(128) < cost(256) ? 128 : 256;
+    }
+    // k-blocks on the critical path x columns per tile
+    auto rounds = [&](int bn) -> double {
+        TcPlan tp;
+        if (plan_gemm_tc(p, bn, num_sms, &tp) != cudaSuccess || tp.pairs <= 0) return 1e30;
+        if (p.mode == 1 && (s->N + bn - 1) / bn > tp.pairs) return 1e30;
+        double kb;
+        if (tp.split > 1) kb = (double) ((tp.tiles - tp.split_tiles) / tp.pairs) * tp.num_kb + (tp.num_kb - tp.split_kb * (tp.split - 1)) + 24.0;
+        else kb = (double) ((tp.tiles + tp.pairs - 1) / tp.pairs) * tp.num_kb;
+        return kb * bn;
     };
-    return cost(128) < cost(256) ? 128 : 256;
+    return rounds(240) < 0.98 * rounds(256) ? 240 : 256;
 }
 
 size_t softmax_workspace_bytes(long long M, long long N, bool per_half = false) {
@@ -670,24 +704,11 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             }
             attach_split_scratch(dev, p.mode == 1 || p.mode == 3 ? reduction_workspace_bytes(p.mode == 1, spec->M, spec->N) : 0, &p);
             if ((e = clear_counters_if_needed(dev, p, panel_bytes, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-            const int bn = gemm_tile_width(p, spec, dev->num_sms);
+            const int bn = gemm_tile_width(p, spec, dev->num_sms);   // (row softmax: also decides p.two_pass)
             CUtensorMap tmA, tmB;
             if ((st = encode_2d(&tmA, inputs[0].ptr, spec->M, spec->K, 128, spec->in_dtype))) return st;
             if ((st = encode_2d(&tmB, inputs[1].ptr, spec->N, spec->K, bn / 2, spec->in_dtype))) return st;   // each CTA of a pair loads half
-            // Row softmax over more tiles per panel than the pairs' accumulator buffers can hold until the panel is
-            // complete (two per pair; with a margin: 64 tiles = 16384 columns) cannot wait across tiles: a second,
-            // memory-bound kernel finishes the rows.  The same two-kernel form is also chosen where it is faster.
             const int tiles_n = (int) ((spec->N + bn - 1) / bn);
-            if (p.mode == 1) {
-                // (never more tiles per panel than SM pairs take part, whatever the device offers)
-                TcPlan tp;
-                if ((e = plan_gemm_tc(p, bn, dev->num_sms, &tp)) != cudaSuccess) return cuda_fail(e, "planning");
-                // The single pass wins where it was built for (rows of up to 16 tiles and a long contraction: 4096^3 106
-                // against 118 us); its panel-by-panel order streams B once per panel and its epilogue waits for the
-                // panel, which loses from 8192 columns on and for short contractions (8192 x 16384 x 4096: 1208
-                // against 838 us; 16384 x 16384 x 1024: 2024 against 877 us).
-                p.two_pass = tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs || tiles_n > kSoftmaxOnePassBestTiles || spec->K < 4096;
-            }
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             if (e == cudaSuccess && p.two_pass)
                 e = launch_softmax_rescale(p.out, p.out_dt, p.stats, spec->M, spec->N, tiles_n, bn, dev->num_sms, stream, &launches);
@@ -1024,6 +1045,7 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     } else {
         p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
         p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;
+        p.in_dt = spec->in_dtype;
         bn = 0;
         if (p.mode == 1 || p.mode == 3) red = reduction_workspace_bytes(p.mode == 1, spec->M, spec->N);
     }
@@ -1032,8 +1054,8 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     TcPlan tp;
     cudaError_t e = plan_gemm_tc(p, bn, dev->num_sms, &tp);
     if (e != cudaSuccess) return cuda_fail(e, "planning");
-    snprintf(text, capacity, "kernel=gemm_tc mode=%d bn=%d tiles=%d pairs=%d split=%d split_tiles=%d split_kb=%d", p.mode, tp.bn,
-             tp.tiles, tp.pairs, tp.split, tp.split_tiles, tp.split_kb);
+    snprintf(text, capacity, "kernel=gemm_tc mode=%d bn=%d tiles=%d pairs=%d split=%d split_tiles=%d split_kb=%d%s", p.mode, tp.bn,
+             tp.tiles, tp.pairs, tp.split, tp.split_tiles, tp.split_kb, p.mode == 1 && p.two_pass ? " two_pass=1" : "");
     return FC_OK;
 }
 

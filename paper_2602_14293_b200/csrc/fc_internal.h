@@ -108,7 +108,7 @@ struct TcParams {
     int red_kind;               // mode 3: FC_RED_ROW_LOGSUMEXP, _SUM, _MAX or _MEAN
     DevOps ops;
     // mode 1
-    float2* stats;              // [M][tiles_n] (max, sum) per tile
+    float2* stats;              // (max, sum) per row and tile: [tiles_n][M] (tile-major, so that a warp reads and writes whole sectors), or [M][tiles_n][2] in the two-kernel softmax
     unsigned int* counters;     // [panels] arrivals; zero at launch, left at zero by a launch that completes
     unsigned int* departed;     // mode 1: [panels] tiles that have left the panel wait; same rule
     // mode 2

@@ -63,6 +63,9 @@ namespace fc {
 // buffer, unused, its waits for operand stages, k-blocks issued, cycles in MMA issue + commit, producer total cycles,
 // producer waits for free stages, MMA thread total in nanoseconds (cycles / ns = the SM clock during the kernel).
 __device__ long long g_prof[160][10];
+__device__ long long g_prof_epi[160][8][8];   // per pair and tile: globaltimer at the epilogue's milestones (leader CTA, first thread)
+__device__ long long g_prof_clk[160][8][8];   // the same milestones in SM cycles
+#define EPI_MARK(i) do { if (et == 0 && leader && cluster_id < 160 && tile_iter < 8) { g_prof_epi[cluster_id][tile_iter][i] = (long long) ptx::globaltimer(); g_prof_clk[cluster_id][tile_iter][i] = clock64(); } } while (0)
 #if FC_PROF >= 2   // per-wait accounting (itself costs about a hundred cycles per k-block)
 #define PROF_T0(q) q = clock64()
 #define PROF_ADD(acc, q) acc += clock64() - q
@@ -71,6 +74,7 @@ __device__ long long g_prof[160][10];
 #define PROF_ADD(acc, q) (void) acc
 #endif
 #else
+#define EPI_MARK(i) (void) 0
 #define PROF_T0(q) (void) q
 #define PROF_ADD(acc, q) (void) acc
 #endif
@@ -92,7 +96,8 @@ struct Cfg {
     static constexpr int kVecBytes = 2 * kMaxVecSlots * BN * 4;   // double-buffered per-tile vector slices
     static constexpr int kCtrlBytes = 256;
     static constexpr int kPoolBytes = 8 * 32 * 17 * 4;   // max-pool: 32 pixels x 16 channels (+1 pad) per epilogue warp
-    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + 1024 + kPoolBytes + 1024;  // exchange, pool staging, alignment slack
+    static constexpr int kXchgBytes = 2 * BM * 8;   // a (max, sum) pair per row and column half
+    static constexpr int kSmemBytes = kStages * kStageBytes + kVecBytes + kCtrlBytes + kXchgBytes + kPoolBytes + 1024;  // + alignment slack
     // mode 6: per stage a 512-byte tile of A scales (this CTA's 128 rows) and one of B scales per 128 columns of the tile
     static constexpr int kScaleStage = 512 + 512 * ((BN + 127) / 128);
     static constexpr int kScaleBytes = kStages * kScaleStage;   // behind everything else
@@ -168,10 +173,33 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
     return v[0];
 }
 
-// One pass over this thread's half row of the accumulator in 16-column chunks, the load of chunk c + 1 in
-// flight while chunk c is processed.  f(c, r) may change r and store it back.
+// One pass over this thread's half row of the accumulator.  The loads are 32 columns wide, the next one in flight
+// while one is processed (a sweep's time is mostly the loads' latency: 16-column loads took twice as long);
+// f(c, r) sees 16-column chunks, may change r and store it back, and is called for the first `live` chunks only
+// (a 240-column tile's second half has seven: the eighth belongs to the other buffer).
 template <int kChunks, class F>
-__device__ __forceinline__ void tmem_sweep(uint32_t tacc, F&& f) {
+__device__ __forceinline__ void tmem_sweep(uint32_t tacc, int live, F&& f) {
+    static_assert(kChunks % 4 == 0, "whole pairs of 32-column loads");
+    uint32_t ra[32], rb[32];
+    auto lo = [](uint32_t (&r)[32]) -> uint32_t (&)[16] { return *reinterpret_cast<uint32_t (*)[16]>(&r[0]); };
+    auto hi = [](uint32_t (&r)[32]) -> uint32_t (&)[16] { return *reinterpret_cast<uint32_t (*)[16]>(&r[16]); };
+    ptx::tmem_ld_32x32_async(tacc, ra);
+#pragma unroll 1
+    for (int c = 0; c < kChunks; c += 4) {
+        ptx::tmem_wait_ld32(ra);
+        ptx::tmem_ld_32x32_async(tacc + (c + 2) * 16, rb);
+        f(c, lo(ra));
+        if (c + 1 < live) f(c + 1, hi(ra));
+        ptx::tmem_wait_ld32(rb);
+        if (c + 4 < kChunks) ptx::tmem_ld_32x32_async(tacc + (c + 4) * 16, ra);
+        if (c + 2 < live) f(c + 2, lo(rb));
+        if (c + 3 < live) f(c + 3, hi(rb));
+    }
+}
+
+// The same with 16-column loads (half the registers): the convolution's average pool, whose sweep is not latency-bound.
+template <int kChunks, class F>
+__device__ __forceinline__ void tmem_sweep16(uint32_t tacc, F&& f) {
     uint32_t ra[16], rb[16];
     ptx::tmem_ld_32x16_async(tacc, ra);
 #pragma unroll 1
@@ -207,9 +235,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     float* svec_all = reinterpret_cast<float*>(smem + ring_bytes);
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ring_bytes + C::kVecBytes);
     float2* xchg = reinterpret_cast<float2*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes);
-    float* pool_stage = reinterpret_cast<float*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + 1024);
+    float* pool_stage = reinterpret_cast<float*>(smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + C::kXchgBytes);
     constexpr bool kMx = MODE == 6;
-    uint8_t* scale_ring = smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + 1024 + C::kPoolBytes;   // mode 6: [stage][A tile 512 B | B tile 512 B]
+    uint8_t* scale_ring = smem + ring_bytes + C::kVecBytes + C::kCtrlBytes + C::kXchgBytes + C::kPoolBytes;   // mode 6: [stage][A tile 512 B | B tile 512 B]
     volatile int* abort_flag = &ctrl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -244,7 +272,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ptx::prefetch_tensormap(&tmSB);
         }
     }
-    constexpr int kTmemAlloc = kMx ? 512 : C::kTmemCols;   // mode 6: eight more columns for the scales (a power of two must be asked for)
+    // a power of two must be asked for: two 240-column accumulators take 512 like two of 256 (mode 6 puts its scales behind them)
+    constexpr int kTmemNeed = C::kTmemCols + (kMx ? 4 + 4 * ((BN + 127) / 128) : 0);
+    constexpr int kTmemAlloc = kTmemNeed > 256 ? 512 : 256;
+    static_assert(kTmemNeed <= kTmemAlloc, "tensor-memory allocation");
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), kTmemAlloc);
         ptx::tmem_relinquish();
@@ -477,6 +508,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;
             float* svec = svec_all + buf * (kMaxVecSlots * BN);
+            EPI_MARK(0);
             // stage this tile's slices of the per-column vectors (fp32) before the accumulator wait
             {
                 int slot = 0;
@@ -494,7 +526,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ptx::bar_sync(2, kEpiThreads);
             if (!*(volatile int*) &ctrl->epi_ok[buf]) break;
             ptx::tc_fence_after();
+            EPI_MARK(1);
             constexpr int kChunks = C::kColHalf / 16;  // 16-column chunks per thread (half a tile row; 240-column tiles: 8 and 7)
+            const int n_chunks = BN == 240 && half == 1 ? kChunks - 1 : kChunks;   // chunks of this half that belong to the tile
             const int col_half = half * C::kColHalf;
             const int n_lim = min(p.N, n_tile + BN);   // first column that is not this tile's
             const uint32_t tacc = tmem_base + buf * BN + col_half + lane_addr;
@@ -512,7 +546,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (w.nsl > 1) {
                 // Slice of a split tile.  Scratch layout per (slice, CTA): [warp 8][chunk][quad 4][lane 32] float4,
                 // so that every warp instruction moves 512 contiguous bytes.
-                constexpr size_t kSliceF4 = (size_t) BM * BN / 4;
+                constexpr size_t kSliceF4 = (size_t) BM * 2 * C::kColHalf / 4;
                 const int ws = warp - 2;
                 unsigned int* cnt = &p.split_counters[(w.v0 / w.nsl) * 2 + (int) cta_rank];
                 // a warp none of whose 32 rows exists (a short last panel: 16 rows of 256) parks and merges nothing
@@ -591,7 +625,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + acc[cc * 4 + j].z);
                             r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + acc[cc * 4 + j].w);
                         }
-                        ptx::tmem_st_32x16(tacc + (c0 + cc) * 16, r);
+                        if (c0 + cc < n_chunks) ptx::tmem_st_32x16(tacc + (c0 + cc) * 16, r);
                     }
                 }
                 ptx::tmem_wait_st();
@@ -656,7 +690,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_ld_32x16_async(tacc + c * 16, r);
                     ptx::tmem_wait_ld(r);
                     const int n0 = n_half + c * 16;
-                    if (p.out && !out_vec && n0 < p.N) {
+                    if (p.out && !out_vec && n0 < n_lim) {
                         // rows off 16-byte boundaries: every lane takes part in the store of the warp's block
                         float v[16];
 #pragma unroll
@@ -664,7 +698,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                         store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
                     }
-                    if (m < p.M && n0 < p.N) {
+                    if (m < p.M && n0 < n_lim) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
@@ -708,8 +742,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::bar_sync(1, kEpiThreads);
                 if (half == 0 && m < p.M) {
                     const float2 o = xchg[row];
-                    if (FC_DBG_IN(&p.stats[m * tiles_n + nb], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
-                        __stcg(&p.stats[m * tiles_n + nb], merge(run_m, run_s, o.x, o.y));
+                    if (FC_DBG_IN(&p.stats[(long long) nb * p.M + m], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
+                        __stcg(&p.stats[(long long) nb * p.M + m], merge(run_m, run_s, o.x, o.y));
                 }
                 __threadfence();
                 ptx::bar_sync(1, kEpiThreads);
@@ -723,7 +757,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (*(volatile int*) &ctrl->last && half == 0 && m < p.M) {
                     float2 a = make_float2(-CUDART_INF_F, 0.0f);
                     for (int j = 0; j < tiles_n; ++j) {
-                        const float2 st = __ldcg(&p.stats[m * tiles_n + j]);
+                        const float2 st = __ldcg(&p.stats[(long long) j * p.M + m]);
                         a = merge(a.x, a.y, st.x, st.y);
                     }
                     if (FC_DBG_IN(&p.red[m], 4, p.red, (long long) p.M * 4, p.status, kSiteRowResult))
@@ -735,24 +769,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // sweep A: maximum of this thread's half row of the tile (ops applied, written back in place
                 // when the list is not empty, so that the later sweeps read finished logits)
                 const bool has_ops = p.ops.n > 0;
-                float mx = -CUDART_INF_F;
-                tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                tmem_sweep<kChunks>(tacc, n_chunks, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
                     if (has_ops) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                        if (m < p.M && n0 < p.N) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                        if (m < p.M && n0 < n_lim) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
 #pragma unroll
                         for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(v[j]);
                         ptx::tmem_st_32x16(tacc + c * 16, r);
                     }
-                    if (m < p.M && n0 < p.N) {
+                    if (m < p.M && n0 + 16 <= n_lim) {
+                        // (four chains instead of one: the sweep's time was the latency of 128 dependent maxima)
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) mx = n0 + j < p.N ? fmaxf(mx, __uint_as_float(r[j])) : mx;
+                        for (int j = 0; j < 4; ++j) {
+                            mx4[0] = fmaxf(mx4[0], __uint_as_float(r[4 * j]));
+                            mx4[1] = fmaxf(mx4[1], __uint_as_float(r[4 * j + 1]));
+                            mx4[2] = fmaxf(mx4[2], __uint_as_float(r[4 * j + 2]));
+                            mx4[3] = fmaxf(mx4[3], __uint_as_float(r[4 * j + 3]));
+                        }
+                    } else if (m < p.M && n0 < n_lim) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) mx4[0] = n0 + j < p.N ? fmaxf(mx4[0], __uint_as_float(r[j])) : mx4[0];
                     }
                 });
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 if (has_ops) ptx::tmem_wait_st();
+                EPI_MARK(2);
                 if (p.two_pass) {
                     // Two-kernel form: nobody waits for the panel.  One more sweep computes the exponentials against
                     // this half row's own maximum (values in (0, 1]), sums them and stores them at once; the pair
@@ -763,9 +808,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const float2 moff = make_float2(-mbase * kLog2e, -mbase * kLog2e);
                     float2 acc2 = make_float2(0.0f, 0.0f);
                     const bool ok = *abort_flag == 0;
-                    tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                    tmem_sweep<kChunks>(tacc, n_chunks, [&](int c, uint32_t (&r)[16]) {
                         const int n0 = n_half + c * 16;
-                        if (n0 >= p.N) return;
+                        if (n0 >= n_lim) return;
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
@@ -797,9 +842,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const float mbase = mx == -CUDART_INF_F ? 0.0f : mx;
                     const float2 moff = make_float2(-mbase * kLog2e, -mbase * kLog2e);
                     float2 acc2 = make_float2(0.0f, 0.0f);
-                    tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                    tmem_sweep<kChunks>(tacc, n_chunks, [&](int c, uint32_t (&r)[16]) {
                         const int n0 = n_half + c * 16;
-                        if (m < p.M && n0 < p.N) {
+                        if (m < p.M && n0 < n_lim) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 const float2 t = __ffma2_rn(make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1])), l2e, moff);
@@ -816,16 +861,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ptx::tmem_wait_st();
                     sm = acc2.x + acc2.y;
                 }
+                EPI_MARK(3);
                 // the two column halves of a row meet in shared memory; the lower half publishes the tile's pair
                 if (half == 1) xchg[row] = make_float2(mx, sm);
                 ptx::bar_sync(1, kEpiThreads);
                 if (half == 0 && m < p.M) {
                     const float2 o = xchg[row];
                     const MaxSum a = ms_merge(MaxSum{mx, sm}, MaxSum{o.x, o.y});
-                    if (FC_DBG_IN(&p.stats[m * tiles_n + nb], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
-                        __stcg(&p.stats[m * tiles_n + nb], make_float2(a.m, a.s));
+                    if (FC_DBG_IN(&p.stats[(long long) nb * p.M + m], 8, p.stats, dbg_stats_bytes, p.status, kSiteStats))
+                        __stcg(&p.stats[(long long) nb * p.M + m], make_float2(a.m, a.s));
                 }
-                __threadfence();
+                // (no fence per thread: the barrier orders the stores above before the one release below, which is
+                // cumulative at device scope)
                 ptx::bar_sync(1, kEpiThreads);
                 // one thread announces the tile and waits (bounded) for the panel's other tiles
                 if (et == 0) {
@@ -842,31 +889,52 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             }
                         }
                     }
-                    __threadfence();
-                    // the tile that leaves the wait last puts both counters back to zero for the next launch
-                    if (*abort_flag == 0 && ptx::atom_acq_rel_gpu_add(&p.departed[mb], 1u) == (unsigned) tiles_n - 1u) {
-                        p.counters[mb] = 0u;
-                        p.departed[mb] = 0u;
-                    }
                 }
                 ptx::bar_sync(1, kEpiThreads);
+                EPI_MARK(4);
                 const bool store = *abort_flag == 0;
-                float row_m = -CUDART_INF_F, row_s = 0.0f;
+                // Departure count of the panel: asked for here, read after the last sweep, so that its round trip is off
+                // the path.  Relaxed (an acquire would hold back the loads below): this tile's last poll of the arrival
+                // counter has returned, and whoever reads tiles_n - 1 here resets the counters only after that.
+                unsigned departed_before = 0u;
+                if (et == 0 && store) departed_before = ptx::atom_relaxed_gpu_add(&p.departed[mb], 1u);
+                // The panel's pairs (max, sum) of this row: each column half of the tile merges one half of them, kBatch loads
+                // in flight (first the maximum, then the sum of the rescaled partial sums: independent exponentials
+                // instead of a chain of merges), and the two halves meet in shared memory.
+                MaxSum a = ms_identity();
                 if (m < p.M && store) {
-                    MaxSum a = ms_identity();
-                    for (int j = 0; j < tiles_n; ++j) {
-                        const float2 st = __ldcg(&p.stats[m * tiles_n + j]);
-                        a = ms_merge(a, MaxSum{st.x, st.y});
+                    constexpr int kBatch = 16;
+                    const int j_mid = (tiles_n + 1) >> 1;
+                    const int j_begin = half == 0 ? 0 : j_mid, j_end = half == 0 ? j_mid : tiles_n;
+                    const float2* scol = p.stats + m;   // tile-major: a warp's 32 rows of one tile are 256 consecutive bytes
+                    for (int j0 = j_begin; j0 < j_end; j0 += kBatch) {
+                        float2 st[kBatch];
+#pragma unroll
+                        for (int q = 0; q < kBatch; ++q) st[q] = j0 + q < j_end ? __ldcg(scol + (long long) (j0 + q) * p.M) : make_float2(-CUDART_INF_F, 0.0f);
+                        float bm = st[0].x;
+#pragma unroll
+                        for (int q = 1; q < kBatch; ++q) bm = fmaxf(bm, st[q].x);
+                        const float base = bm == -CUDART_INF_F ? 0.0f : bm;   // -inf only (an additive mask): the sums are zero
+                        float bs = 0.0f;
+#pragma unroll
+                        for (int q = 0; q < kBatch; ++q) bs = fmaf(st[q].y, exp2_fast((st[q].x - base) * kLog2e), bs);
+                        a = ms_merge(a, MaxSum{bm, bs});
                     }
-                    row_m = a.m;
-                    row_s = a.s;
                 }
+                xchg[half * BM + row] = make_float2(a.m, a.s);
+                ptx::bar_sync(1, kEpiThreads);
+                {
+                    const float2 o = xchg[(half ^ 1) * BM + row];
+                    a = ms_merge(a, MaxSum{o.x, o.y});
+                }
+                const float row_m = a.m, row_s = a.s;
+                EPI_MARK(6);
                 // last sweep: p = e * 2^((max_half - max_row) log2 e) / sum_row, one factor per thread
                 const float fac = m < p.M && store && mx != -CUDART_INF_F ? exp2_fast((mx - row_m) * kLog2e) / row_s : 0.0f;   // (a half row of -inf only holds zeros)
                 const float2 fac2 = make_float2(fac, fac);
-                tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                tmem_sweep<kChunks>(tacc, n_chunks, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
-                    if (!out_vec && n0 < p.N && __all_sync(0xffffffffu, store)) {
+                    if (!out_vec && n0 < n_lim && __all_sync(0xffffffffu, store)) {
                         // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
                         float v[16];
 #pragma unroll
@@ -876,7 +944,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             v[2 * j + 1] = t.y;
                         }
                         store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
-                    } else if (m < p.M && n0 < p.N && store && out_vec) {
+                    } else if (m < p.M && n0 < n_lim && store && out_vec) {
                         float v[16];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
@@ -887,6 +955,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                     }
                 });
+                // the tile that has left the panel wait last puts both counters back to zero for the next launch
+                // (off the path between the wait and the stores: nothing in this launch reads them again)
+                if (et == 0 && store && departed_before == (unsigned) tiles_n - 1u) {
+                    p.counters[mb] = 0u;
+                    p.departed[mb] = 0u;
+                }
             } else if (p.pool == 1) {
                 // conv + 2x2 max-pool of non-negative values (the op list ends with ReLU, the output starts at
                 // zero): every pixel that lies in a window takes part in an unsigned atomic maximum on the fp32
@@ -927,7 +1001,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float* stage = pool_stage + (warp - 2) * (32 * 17);
                 unsigned int* out_u = (unsigned int*) p.out;
                 const int ch = lane & 15;
-                tmem_sweep<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                tmem_sweep16<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
                     if (n0 >= p.N) return;
                     float v[16];
@@ -987,6 +1061,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
+            EPI_MARK(5);
             release_buf();
         }
     }
@@ -1122,22 +1197,34 @@ cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorM
         case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream, plan);
         case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream, plan);
         case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream, plan);
-        default: return p.a_packed ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan) : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
+        default:
+            // (the convolutions have no 240-column form: their widths are the channel counts, powers of two as a rule)
+            if constexpr (BN == 240) return cudaErrorInvalidValue;
+            else return p.a_packed ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan) : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
     }
+}
+
+cudaError_t launch_any(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int bn, int num_sms, cudaStream_t stream,
+                       TcPlan* plan) {
+    return bn == 256 ? launch_bn<256>(p, tmA, tmB, num_sms, stream, plan)
+         : bn == 240 ? launch_bn<240>(p, tmA, tmB, num_sms, stream, plan)
+                     : launch_bn<128>(p, tmA, tmB, num_sms, stream, plan);
 }
 
 }  // namespace
 
 #ifdef FC_PROF
 extern "C" void fc_debug_prof(long long* out) { cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 160 * 10); }
+extern "C" void fc_debug_prof_epi(long long* out) { cudaMemcpyFromSymbol(out, g_prof_epi, sizeof(long long) * 160 * 64); }
+extern "C" void fc_debug_prof_clk(long long* out) { cudaMemcpyFromSymbol(out, g_prof_clk, sizeof(long long) * 160 * 64); }
 #endif
 
-size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : Cfg<128>::kSmemBytes; }
+size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : bn == 240 ? Cfg<240>::kSmemBytes : Cfg<128>::kSmemBytes; }
 
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int num_sms,
                            cudaStream_t stream, int* launches) {
     *launches += 1;
-    return bn == 256 ? launch_bn<256>(p, &tmA, &tmB, num_sms, stream, nullptr) : launch_bn<128>(p, &tmA, &tmB, num_sms, stream, nullptr);
+    return launch_any(p, &tmA, &tmB, bn, num_sms, stream, nullptr);
 }
 
 cudaError_t launch_gemm_tc_mx(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
@@ -1148,7 +1235,7 @@ cudaError_t launch_gemm_tc_mx(const TcParams& p, const CUtensorMap& tmA, const C
 }
 
 cudaError_t plan_gemm_tc(const TcParams& p, int bn, int num_sms, TcPlan* plan) {
-    return bn == 256 ? launch_bn<256>(p, nullptr, nullptr, num_sms, nullptr, plan) : launch_bn<128>(p, nullptr, nullptr, num_sms, nullptr, plan);
+    return launch_any(p, nullptr, nullptr, bn, num_sms, nullptr, plan);
 }
 
 }  // namespace fc

@@ -369,6 +369,30 @@ def test_c3_chain_ragged(fc, orc, M, N, K):
     run_and_check(fc, orc, replace(wl.gemm_bias_gelu_scale_clamp(M, N, K, "var"), out_dtype="f32"), 4)
 
 
+@pytest.mark.parametrize("M,N,K", [(1000, 4000, 128), (1000, 3999, 72), (2048, 4096, 64), (1100, 3856, 200)])
+def test_gemm_240_column_tiles(fc, orc, M, N, K):
+    """Where rounds x tile width is smaller with 240-column tiles (two accumulators of 240 columns in tensor memory,
+    epilogue halves of 128 and 112 columns) the GEMM kernels take them: a ragged last tile, rows off 16-byte
+    boundaries, an exact multiple of 240 (3856 = 16 x 240 + 16: a last tile of one chunk), all three epilogues."""
+    ch = wl.gemm_bias_gelu_scale_clamp(M, N, K, "var")
+    run_and_check(fc, orc, ch, 21)
+    assert fc.fc_last_plan() == "gemm_tc_mode0_bn240"
+    run_and_check(fc, orc, replace(ch, out_dtype="f32"), 21)
+    run_and_check(fc, orc, wl.gemm_bias_scale_lse(M, N, K, "var", True), 22)
+    assert fc.fc_last_plan() == "gemm_tc_mode3_bn240"
+    run_and_check(fc, orc, wl.linear_row_reduce(M, N, K, "row_max", ops=(("bias_n", 2), ("relu",)), store_main=False), 22)
+    assert fc.fc_last_plan() == "gemm_tc_mode3_bn240"
+
+
+@pytest.mark.parametrize("M,N", [(520, 4000), (600, 3999), (777, 3856)])
+def test_gemm_softmax_240_column_tiles(fc, orc, M, N):
+    """The single-pass row softmax on 240-column tiles: 17 tiles per panel, the last one ragged."""
+    ch = wl.gemm_softmax(M, N, 4096)
+    run_and_check(fc, orc, ch, 23)
+    assert fc.fc_last_plan() == "gemm_tc_mode1_bn240"
+    run_and_check(fc, orc, replace(ch, out_dtype="f32"), 23)
+
+
 @pytest.mark.parametrize("M,N,K,plan", [(100, 1000, 4096, "bn128_split"), (2048, 1024, 1024, "bn128"), (250, 2304, 768, "bn128"),
                                         (16, 8192, 4096, "bn128"), (16, 4096, 8192, "bn256_split"), (1024, 1024, 8192, "bn256_split")])
 def test_gemm_few_tiles_either_tile_width(fc, orc, M, N, K, plan):
@@ -380,7 +404,7 @@ def test_gemm_few_tiles_either_tile_width(fc, orc, M, N, K, plan):
     run_and_check(fc, orc, replace(ch, out_dtype="f32"), 9)
 
 
-@pytest.mark.parametrize("M,N,K,plan", [(100, 1000, 4096, "bn128_split"), (300, 1100, 512, "bn128"), (1024, 4096, 1024, "bn256"),
+@pytest.mark.parametrize("M,N,K,plan", [(100, 1000, 4096, "bn128_split"), (300, 1100, 512, "bn128"), (1024, 4096, 1024, "bn240"),
                                         (64, 4096, 8192, "bn256_split")])
 @pytest.mark.parametrize("store_main", [False, True])
 def test_gemm_row_reduction_few_tiles_either_tile_width(fc, orc, M, N, K, plan, store_main):
@@ -499,7 +523,7 @@ def test_c4_full_size_every_element(fc, orc, variant):
     outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
     fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
     fc.fc_get_async_status()
-    assert fc.fc_last_plan() == "gemm_tc_mode1_bn256"
+    assert fc.fc_last_plan() == "gemm_tc_mode1_bn240"   # 18 tiles of 240 columns per panel: 288 tiles = 4 rounds on 72 pairs
     got = outs[0].cpu()
     for r0, r1 in _row_blocks(ch.M, 1024):
         ref = orc.run_chain(replace(ch, M=r1 - r0), [ins[0][r0:r1], ins[1]])

@@ -49,7 +49,9 @@ def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_bias_relu_f32(256, 256, 256)) == "gemm_f32"
     assert _plan(fc, wl.gemm_bias_relu_f32(1024, 1024, 64)) == "gemm_f32_mid"
     assert _plan(fc, wl.gemm_bias_relu_f32(2048, 1024, 64)) == "gemm_f32_big"
-    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(4096, 4096, 256)) == "gemm_tc_mode0_bn256"
+    # rounds of tiles: 240-column tiles where rounds x width is smaller (256 tiles = 4 rounds x 256 against 288 = 4 rounds x 240)
+    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(4096, 4096, 256)) == "gemm_tc_mode0_bn240"
+    assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(8192, 8192, 256)) == "gemm_tc_mode0_bn256"     # 14 rounds x 256 against 16 x 240
     # few tiles: 128-wide ones where the cost model prefers twice the tiles with half the epilogue each ...
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 512, 256)) == "gemm_tc_mode0_bn128"
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(128, 256, 4096)) == "gemm_tc_mode0_bn128_split"
@@ -57,12 +59,14 @@ def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(16, 8192, 8192)) == "gemm_tc_mode0_bn256_split"
     assert _plan(fc, wl.gemm_bias_gelu_scale_clamp(512, 128, 256)) == "gemm_tc_mode0_bn128"
     assert _plan(fc, wl.gemm_softmax(256, 1024, 4096)) == "gemm_tc_mode1_bn256_split"      # 4 tiles: cut along K as well
-    assert _plan(fc, wl.gemm_softmax(4096, 4096, 4096)) == "gemm_tc_mode1_bn256"
+    assert _plan(fc, wl.gemm_softmax(4096, 4096, 4096)) == "gemm_tc_mode1_bn240"
+    assert _plan(fc, wl.gemm_softmax(4096, 1024, 4096)) == "gemm_tc_mode1_bn256"      # one round of 64 tiles against two of 240-column ones
     assert _plan(fc, wl.gemm_softmax(256, 1024, 256)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"   # short contraction
     assert _plan(fc, wl.gemm_softmax(256, 8192, 4096)) == "gemm_tc_mode1_bn256_split_two_pass softmax_rescale"  # 32 tiles per panel (and few enough to be cut along K)
     assert _plan(fc, wl.gemm_softmax(64, 20000, 64)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"
     assert _plan(fc, wl.gemm_bias_scale_lse(256, 1024, 256)) == "gemm_tc_mode3_bn128"       # few tiles: as the plain GEMM
-    assert _plan(fc, wl.gemm_bias_scale_lse(2048, 4096, 256)) == "gemm_tc_mode3_bn256"
+    assert _plan(fc, wl.gemm_bias_scale_lse(2048, 4096, 256)) == "gemm_tc_mode3_bn240"
+    assert _plan(fc, wl.gemm_bias_scale_lse(4096, 8192, 256)) == "gemm_tc_mode3_bn256"
     assert _plan(fc, wl.linear_row_reduce(96, 512, 256)) == "weight_colsum colsum_finish row_dot"
     assert _plan(fc, wl.mlp(300, (64, 64, 32))) == "mlp_tc"
     conv = wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128)
