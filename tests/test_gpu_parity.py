@@ -513,6 +513,56 @@ def test_c4_softmax_dominant_logits(fc, orc):
     _check_softmax_rows(outs[0])
 
 
+@pytest.mark.parametrize("M,N", [(300, 1000), (520, 4000)])
+def test_gemm_softmax_single_pass_with_outliers(fc, orc, M, N):
+    """Single-pass form (K >= 4096) with logits far above the rest: +20 / +35 / +50 in rising order inside one half
+    row of a tile, in the second column half, in other tiles, in the last column; rows without any; then with the
+    largest one in a half row's first 16 columns and falling ones behind it.  Stresses the maximum sweep, the
+    exponentials against a half row's own maximum and the merge across halves and tiles."""
+    ch = wl.gemm_softmax(M, N, 4096, "var")
+    A, B = wl.make_inputs(ch, 2)
+    Af = rng.bf16_bits_to_f32(A).copy()
+    Bf = rng.bf16_bits_to_f32(B).copy()
+    Af[:, 0] = 8.0
+    Af[::3, 0] = 0.0                      # every third row: no outliers at all
+    Bf[:, 0] = 0.0
+    cols = {20: 2.5, 60: 4.375, 100: 6.25, 200: 6.0, 300: 6.25, 5 + 256: 3.0, N - 1: 6.25, N // 2 + 7: 5.0}
+    for c, b in cols.items():
+        Bf[c, 0] = b
+    Af[1, 0] = 8.0
+    ins = [rng.store(Af, "bf16"), rng.store(Bf, "bf16")]
+    outs, _, _ = run_and_check(fc, orc, ch, ins=ins)
+    assert fc.fc_last_plan().startswith("gemm_tc_mode1_bn") and "two_pass" not in fc.fc_last_plan()
+    _check_softmax_rows(outs[0])
+    # the largest outlier of the first half row in its first 16 columns, falling ones behind it
+    Bf[:, 0] = 0.0
+    for c, b in {3: 6.25, 40: 4.0, 90: 2.0, 130: 6.25, 140: 7.0}.items():
+        Bf[c, 0] = b
+    ins = [rng.store(Af, "bf16"), rng.store(Bf, "bf16")]
+    outs, _, _ = run_and_check(fc, orc, ch, ins=ins)
+    _check_softmax_rows(outs[0])
+
+
+def test_gemm_softmax_single_pass_with_minus_infinity_mask(fc, orc):
+    """The single-pass form behind scale + additive 0 / -inf mask: chunks, half rows and whole tiles of -inf in front
+    of, between and behind the kept columns; masked probabilities are exactly 0."""
+    M, N, K = 300, 1000, 4096
+    base = wl.gemm_softmax(M, N, K, "var")
+    rec = base.input_recipe + (("mask", "bf16", (M, N), "normal", 0.0, 1.0),)
+    ch = replace(base, ops=(("scale", 0.5), ("add_tensor", 2)), store_main=False, input_recipe=rec)
+    ins = wl.make_inputs(ch, 4)
+    keep = np.arange(N)[None, :] <= (3 * np.arange(M)[:, None] + 2)
+    keep[7] = False; keep[7, 600] = True
+    keep[9] = np.arange(N) >= 900
+    keep[11] = (np.arange(N) % 64) >= 48
+    ins[2] = rng.store(np.where(keep, 0.0, -np.inf).astype(np.float32), "bf16")
+    outs, ref, _ = run_and_check(fc, orc, ch, ins=ins)
+    assert "two_pass" not in fc.fc_last_plan()
+    got = util.to_f64(outs[0])
+    assert (got[~keep] == 0.0).all()
+    np.testing.assert_allclose(got.sum(1), 1.0, atol=2e-2)
+
+
 @pytest.mark.parametrize("variant", ["std", "var"])
 def test_c4_full_size_every_element(fc, orc, variant):
     """All 4096 x 4096 probabilities of the benchmark's GEMM + softmax chain (single-pass form, 16 tiles per row panel),
