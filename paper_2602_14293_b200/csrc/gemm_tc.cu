@@ -173,31 +173,22 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
     return v[0];
 }
 
-// One pass over this thread's half row of the accumulator.  The loads are 32 columns wide, the next one in flight
-// while one is processed (a sweep's time is mostly the loads' latency: 16-column loads took twice as long);
-// f(c, r) sees 16-column chunks, may change r and store it back, and is called for the first `live` chunks only
-// (a 240-column tile's second half has seven: the eighth belongs to the other buffer).
+// One pass over this thread's half row of the accumulator in 16-column chunks: load, wait, f(c, r), which may change r
+// and store it back; the first `live` chunks only (a 240-column tile's second half has seven: the eighth belongs to the
+// other buffer).  A plain loop on purpose: a tcgen05.ld + wait takes 30 - 60 cycles, and neither keeping the next
+// load in flight nor 32-column loads (two and four copies of f's code) measured faster than this single copy.
 template <int kChunks, class F>
 __device__ __forceinline__ void tmem_sweep(uint32_t tacc, int live, F&& f) {
-    static_assert(kChunks % 4 == 0, "whole pairs of 32-column loads");
-    uint32_t ra[32], rb[32];
-    auto lo = [](uint32_t (&r)[32]) -> uint32_t (&)[16] { return *reinterpret_cast<uint32_t (*)[16]>(&r[0]); };
-    auto hi = [](uint32_t (&r)[32]) -> uint32_t (&)[16] { return *reinterpret_cast<uint32_t (*)[16]>(&r[16]); };
-    ptx::tmem_ld_32x32_async(tacc, ra);
 #pragma unroll 1
-    for (int c = 0; c < kChunks; c += 4) {
-        ptx::tmem_wait_ld32(ra);
-        ptx::tmem_ld_32x32_async(tacc + (c + 2) * 16, rb);
-        f(c, lo(ra));
-        if (c + 1 < live) f(c + 1, hi(ra));
-        ptx::tmem_wait_ld32(rb);
-        if (c + 4 < kChunks) ptx::tmem_ld_32x32_async(tacc + (c + 4) * 16, ra);
-        if (c + 2 < live) f(c + 2, lo(rb));
-        if (c + 3 < live) f(c + 3, hi(rb));
+    for (int c = 0; c < live; ++c) {
+        uint32_t r[16];
+        ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+        ptx::tmem_wait_ld(r);
+        f(c, r);
     }
 }
 
-// The same with 16-column loads (half the registers): the convolution's average pool, whose sweep is not latency-bound.
+// Two chunks per iteration, the second load in flight while the first chunk is processed (the convolution's pooling sweeps).
 template <int kChunks, class F>
 __device__ __forceinline__ void tmem_sweep16(uint32_t tacc, F&& f) {
     uint32_t ra[16], rb[16];
@@ -632,50 +623,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
 
             if constexpr (MODE == 0 || MODE == 6) {
-                uint32_t ra[16], rb[16];
-                ptx::tmem_ld_32x16_async(tacc, ra);
+                // one chunk at a time, one copy of the code: load, wait, ops, store (keeping the next load in flight
+                // and two copies of this body was no faster; see tmem_sweep)
 #pragma unroll 1
-                for (int c = 0; c < kChunks; c += 2) {
-                    // chunk c is in flight in ra; prefetch c+1 into rb while c is processed, then swap roles
-                    ptx::tmem_wait_ld(ra);
-                    ptx::tmem_ld_32x16_async(tacc + (c + 1) * 16, rb);
-                    {
-                        const int n0 = n_half + c * 16;
-                        if (!out_vec && n0 < n_lim) {
-                            // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
-                            float v[16];
+                for (int c = 0; c < n_chunks; ++c) {
+                    const int n0 = n_half + c * 16;
+                    if (n0 >= n_lim) break;
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16_async(tacc + c * 16, r);
+                    ptx::tmem_wait_ld(r);
+                    float v[16];
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
-                            if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
-                        } else if (m < p.M && n0 < n_lim) {
-                            float v[16];
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ra[j]);
-                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                            else apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
-                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
-                        }
+                    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                    if (m < p.M) {
+                        if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+                        else apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
                     }
-                    ptx::tmem_wait_ld(rb);
-                    if (c + 2 < kChunks) ptx::tmem_ld_32x16_async(tacc + (c + 2) * 16, ra);
-                    {
-                        const int n0 = n_half + (c + 1) * 16;
-                        if (!out_vec && n0 < n_lim) {
-                            // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
-                            float v[16];
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
-                            if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
-                            store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
-                        } else if (m < p.M && n0 < n_lim) {
-                            float v[16];
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rb[j]);
-                            if (precise) apply_ops16<true>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
-                            else apply_ops16<false>(v, p.ops, svec, BN, col_half + (c + 1) * 16, m, n0, p.N, p.N);
-                            store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
-                        }
+                    if (!out_vec) {
+                        // rows off 16-byte boundaries: the warp stores its 32 x 16 block together
+                        store16_rows(p.out, p.out_dt, pool_stage + (warp - 2) * (32 * 17), v, m - lane, p.M, n0, p.N, lane, dbg_out);
+                    } else if (m < p.M) {
+                        store16(p.out, p.out_dt, out_vec, v, m, n0, p.N, dbg_out);
                     }
                 }
             } else if constexpr (MODE == 3) {
