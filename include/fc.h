@@ -222,7 +222,7 @@ fc_status fc_staging_size(const fc_chain_spec* spec, const fc_tensor* inputs, in
  * Scratch memory.  A 16-bit GEMM_NT with a row reduction needs some (per-tile partial results plus
  * per-panel arrival counters for the cross-tile merge; K + 1 doubles for the collapsed form, below), and so
  * does CONV2D_NCHW (the channels-last copies of image and weights).  The partial results are kept per row
- * and output tile; tiles are 128 or 256 columns wide, whichever the launcher expects to be faster for the
+ * and output tile; tiles are 128, 240 or 256 columns wide, whichever the launcher expects to be faster for the
  * shape, so a row reduction's value depends on the row count of the call up to fp32 summation order.
  * fc_workspace_size reports
  * the bytes a spec needs (0 for the other chains); fc_set_workspace registers a caller-owned DEVICE
@@ -257,7 +257,8 @@ fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
  * workspace registered now: "kernel=ew_rowreduce", "kernel=gemm_f32", "kernel=collapse", "kernel=mlp_tc", or
  * "kernel=gemm_tc mode=<0 store|1 softmax|2 conv+pool|3 logsumexp> bn=<tile width> tiles=<256 x bn tiles>
  * pairs=<CTA pairs launched> split=<slices per split tile, 1 = none> split_tiles=<tiles that are split>
- * split_kb=<64-wide k-blocks per parking slice>".  `text` is a caller-owned HOST buffer of `capacity`
+ * split_kb=<64-wide k-blocks per parking slice>" (a row softmax that takes its two-kernel form adds
+ * " two_pass=1").  `text` is a caller-owned HOST buffer of `capacity`
  * bytes (truncated if too small).  Launches nothing.  For logs and tests; the format may gain fields.
  */
 fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacity);
