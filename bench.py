@@ -699,6 +699,11 @@ def main():
             ent = {"ms": ms, "value": n2 / (ms * 1e-3), "unit": u2, "bound": b2}
             if b2 == "tensor":
                 ent["frac_of_burst_peak"] = ent["value"] / peaks["bf16_tflops"]
+            elif "gemm_tc_mode7" in fc.fc_last_plan():
+                # an fp32 GEMM that ran as three tf32 products per product on the tensor cores (tf32: half the bf16 rate)
+                ent["bound"] = "tensor (3 x tf32 per fp32 product; operand split kernels included in the time)"
+                ent["tensor_tflops_executed"] = 3.0 * ent["value"]
+                ent["frac_of_burst_peak_tf32"] = 3.0 * ent["value"] / (0.5 * peaks["bf16_tflops"])
             f2 = eager_fn(c2, i2)
             if f2 is not None and not args.no_eager:
                 ent["eager_ms"] = time_loop(f2, 20, 3, fl)

@@ -267,7 +267,7 @@ EXTRA = {
     "F6": lambda **kw: conv_nchw(conv_bias_relu_avgpool(**kw)),
     "F7": lambda **kw: scale_add_softmax(**kw),
     "F8": lambda **kw: gemm_softmax(**{"M": 2048, "N": 50264, "K": 4096, **kw}),   # a vocabulary-wide softmax: two kernels
-    "F9": lambda **kw: gemm_bias_relu_f32(**{"M": 2048, "N": 2048, "K": 2048, **kw}),   # C1's chain at a size the plain ALUs bound
+    "F9": lambda **kw: gemm_bias_relu_f32(**{"M": 2048, "N": 2048, "K": 2048, **kw}),   # C1's chain at a size where fp32 operands go to the tensor cores (three tf32 products per product)
     "F10": lambda **kw: gemm_mxf8_bias_gelu_scale_clamp(**kw),   # C3's chain on block-scaled 8-bit operands
 }
 ALL = {**CONFIGS, **EXTRA}

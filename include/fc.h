@@ -104,7 +104,13 @@ typedef enum {
 } fc_status;
 
 typedef enum {
-    FC_F32 = 0,
+    FC_F32 = 0,       /* as spec.in_dtype of a GEMM_NT producer: fp32 operands, fp32 output, no reduction.  Small problems
+                         (M N K < 2^29) are contracted with fp32 FMAs on the plain ALUs.  Larger ones run on the tensor
+                         cores when K is a multiple of 4, both operands are 16-byte aligned and a workspace of
+                         roundup(12 M K, 256) + 12 N K bytes is registered (fc_workspace_size reports it): every operand
+                         value x is cut into hi (the bits a tf32 multiplication reads) and lo = x - hi, and
+                         A B^T = A_hi B_hi^T + A_hi B_lo^T + A_lo B_hi^T with fp32 accumulation, which leaves out terms of
+                         2^-21 relative size per product.  Without the workspace the fp32-FMA kernels run at any size. */
     FC_BF16 = 1,
     FC_F16 = 2,       /* IEEE binary16, the storage type of the paper's kernels */
     FC_F8E4M3 = 3,    /* 8-bit float, 4 exponent bits (bias 7), 3 fraction bits, finite only (no infinities, all-ones is NaN):

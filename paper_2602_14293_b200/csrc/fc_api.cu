@@ -455,7 +455,7 @@ int gemm_tile_width(TcParams& p, const fc_chain_spec* s, int num_sms) {
         p.two_pass = plan_gemm_tc(p, kSoftmaxBN, num_sms, &tp) != cudaSuccess || tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs ||
                      tiles_n > kSoftmaxOnePassBestTiles || s->K < 4096;
         if (p.two_pass) return kSoftmaxBN;
-    } else if (p.mode != 0 && p.mode != 3) {
+    } else if (p.mode != 0 && p.mode != 3 && p.mode != 7) {
         return 256;
     } else if (s->N <= 128) {
         return 128;
@@ -484,6 +484,16 @@ int gemm_tile_width(TcParams& p, const fc_chain_spec* s, int num_sms) {
     };
     return rounds(240) < 0.98 * rounds(256) ? 240 : 256;
 }
+
+// fp32 GEMMs on the tensor cores (three tf32 products per fp32 product, see split_tf32_kernel): from this much work
+// on, where it beats the register-tiled fp32 kernels (2048^3: 454 us there); K a multiple of 4 (16-byte rows for TMA).
+// The split operands, [M, 3K] and [N, 3K] fp32, live in the workspace; without one the fp32 kernels run.
+constexpr long long kTf32MinWork = 1LL << 29;   // M * N * K
+bool tf32x3_eligible(const fc_chain_spec* s) {
+    return s->K % 4 == 0 && s->K <= 0x7fffffffLL / 3 && s->M * s->N >= (kTf32MinWork + s->K - 1) / s->K && s->N >= 64 && s->M >= 64;
+}
+size_t tf32x3_a_bytes(const fc_chain_spec* s) { return ((size_t) s->M * 3 * s->K * 4 + 255) / 256 * 256; }
+size_t tf32x3_workspace_bytes(const fc_chain_spec* s) { return tf32x3_a_bytes(s) + (size_t) s->N * 3 * s->K * 4; }
 
 size_t softmax_workspace_bytes(long long M, long long N, bool per_half = false) {
     const long long tiles_n = (N + kSoftmaxBN - 1) / kSoftmaxBN;
@@ -549,12 +559,13 @@ fc_status encode_2d(CUtensorMap* tm, const void* ptr, long long rows, long long 
     const int dev = t_device;
     const MapKey mk = {ptr, {2, rows, cols, box_rows, dt, dev, 0, 0}};
     if (g_maps.find(mk, tm)) return FC_OK;
-    const cuuint64_t esize = dt == FC_F8E4M3 ? 1 : 2;
+    const cuuint64_t esize = dt == FC_F8E4M3 ? 1 : (dt == FC_F32 ? 4 : 2);
     const cuuint64_t dims[2] = {(cuuint64_t) cols, (cuuint64_t) rows};
     const cuuint64_t strides[1] = {(cuuint64_t) cols * esize};
     const cuuint32_t box[2] = {(cuuint32_t) (128 / esize), (cuuint32_t) box_rows};   // 128-byte rows
     const cuuint32_t estr[2] = {1, 1};
     const CUtensorMapDataType tdt = dt == FC_F8E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                    : dt == FC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                     : (dt == FC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     CUresult r = g_encode_tiled(tm, tdt, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -661,6 +672,37 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             break;
         }
         case Plan::GEMM_F32: {
+            if (tf32x3_eligible(spec) && dev->workspace && dev->workspace_bytes >= tf32x3_workspace_bytes(spec) &&
+                ((reinterpret_cast<uintptr_t>(inputs[0].ptr) | reinterpret_cast<uintptr_t>(inputs[1].ptr)) & 15) == 0) {
+                {   // the split operands overwrite whatever counters a previous layout kept here
+                    std::lock_guard<std::mutex> lk(g_mu);
+                    dev->counter_layout = 0;
+                }
+                float* a3 = (float*) dev->workspace;
+                float* b3 = (float*) ((char*) dev->workspace + tf32x3_a_bytes(spec));
+                if ((e = launch_split_tf32((const float*) inputs[0].ptr, a3, spec->M, spec->K, false, false, stream, &launches)) != cudaSuccess) return cuda_fail(e, "operand split kernel launch");
+                if ((e = launch_split_tf32((const float*) inputs[1].ptr, b3, spec->N, spec->K, true, true, stream, &launches)) != cudaSuccess) return cuda_fail(e, "operand split kernel launch");
+                TcParams p;
+                memset(&p, 0, sizeof(p));
+                p.mode = 7;
+                p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) (3 * spec->K);
+                p.in_dt = FC_F32;
+                p.out = outputs[plan.main_index].ptr; p.out_dt = FC_F32;
+                p.status = dev->status;
+                p.dbg_trim = g_bounds_trip.load(std::memory_order_relaxed) ? spec->N * 4LL : 0;
+                build_ops(spec, inputs, &p.ops);
+                {
+                    const long long panel_bytes = 256LL * p.K * 4;
+                    long long g = (32LL << 20) / (panel_bytes > 0 ? panel_bytes : 1);
+                    p.group_m = (int) (g < 1 ? 1 : (g > 64 ? 64 : g));
+                }
+                const int bn = gemm_tile_width(p, spec, dev->num_sms);
+                CUtensorMap tmA, tmB;
+                if ((st = encode_2d(&tmA, a3, spec->M, p.K, 128, FC_F32))) return st;
+                if ((st = encode_2d(&tmB, b3, spec->N, p.K, bn / 2, FC_F32))) return st;   // each CTA of a pair loads half
+                e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
+                break;
+            }
             GemmF32Params p;
             p.A = (const float*) inputs[0].ptr; p.B = (const float*) inputs[1].ptr;
             p.C = (float*) outputs[plan.main_index].ptr;
@@ -1006,6 +1048,7 @@ fc_status fc_workspace_size(const fc_chain_spec* spec, size_t* bytes) {
     if ((st = validate_spec(spec, &plan))) return st;
     *bytes = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? reduction_workspace_bytes(plan.kind == Plan::TC_SOFTMAX, spec->M, spec->N)
            : plan.kind == Plan::GEMM_COLLAPSE ? collapse_workspace_bytes(spec->N, spec->K)
+           : plan.kind == Plan::GEMM_F32 ? (tf32x3_eligible(spec) ? tf32x3_workspace_bytes(spec) : 0)
            : plan.kind == Plan::TC_MX ? (spec->K % 128 ? 0 : (scale_tiles_bytes(spec->M, spec->K, 128) + 255) / 256 * 256 + scale_tiles_bytes(spec->N, spec->K, mx_tile_width(spec->N)))
            : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0;
     return FC_OK;
@@ -1029,7 +1072,13 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     if (!text || capacity == 0) return fail(FC_ERR_NULL, "text is null or has no room");
     if ((st = validate_spec(spec, &plan))) return st;
     if (plan.kind == Plan::EW) { snprintf(text, capacity, "kernel=ew_rowreduce"); return FC_OK; }
-    if (plan.kind == Plan::GEMM_F32) { snprintf(text, capacity, "kernel=gemm_f32"); return FC_OK; }
+    if (plan.kind == Plan::GEMM_F32) {
+        DeviceInfo* d2;
+        if ((st = get_device(&d2))) return st;
+        const bool tf = tf32x3_eligible(spec) && d2->workspace && d2->workspace_bytes >= tf32x3_workspace_bytes(spec);
+        snprintf(text, capacity, tf ? "kernel=gemm_tc mode=7" : "kernel=gemm_f32");
+        return FC_OK;
+    }
     if (plan.kind == Plan::GEMM_COLLAPSE) { snprintf(text, capacity, "kernel=collapse"); return FC_OK; }
     if (plan.kind == Plan::TC_MLP) { snprintf(text, capacity, "kernel=mlp_tc"); return FC_OK; }
     if (plan.kind == Plan::TC_MX) { snprintf(text, capacity, "kernel=gemm_tc mode=6 bn=%d", mx_tile_width(spec->N)); return FC_OK; }

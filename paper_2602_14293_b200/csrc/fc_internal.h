@@ -65,6 +65,9 @@ struct GemmF32Params {
     DevOps ops;
 };
 cudaError_t launch_gemm_f32(const GemmF32Params& p, cudaStream_t stream, int* launches);
+// fp32 operand [rows, K] -> [rows, 3 K] of tf32-representable pieces (see split_tf32_kernel in layout.cu)
+cudaError_t launch_split_tf32(const float* x, float* y, long long rows, long long K, bool is_b, bool beside_previous, cudaStream_t stream,
+                              int* launches);
 
 // GEMM + linear ops + row sum / mean without a main output, rewritten as out = A u + C (see collapse.cu)
 struct CollapseParams {
@@ -99,7 +102,8 @@ cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t 
 // tcgen05 GEMM family: plain epilogue (kMode 0), row softmax across tiles (1), conv + avg-pool (2)
 struct TcParams {
     int mode;                   // 0 plain store, 1 row softmax, 2 conv + pooling, 3 row reduction to one value,
-                                // 6 plain store with block-scaled E4M3 operands (scale tiles through a third and fourth tensor map)
+                                // 6 plain store with block-scaled E4M3 operands (scale tiles through a third and fourth tensor map),
+                                // 7 plain store with 32-bit operands read as tf32 (K counts their elements)
     int M, N, K;                // GEMM view (conv: M = batch*OH*OW, N = Cout, K = R*S*Cin)
     int group_m;                // mode 0 raster: 256-row panels per sweep over the column tiles
     int in_dt;                  // FC_BF16 or FC_F16: storage of both MMA operands

@@ -208,6 +208,7 @@ __device__ __forceinline__ void tmem_sweep16(uint32_t tacc, F&& f) {
 // very few channels) blocks of eight 8-channel chunks that run on across the taps (K = R*S*Cin in order).
 template <int MODE>
 __host__ __device__ __forceinline__ int count_kb(const TcParams& p) {
+    if (MODE == 7) return (p.K + BK / 2 - 1) / (BK / 2);   // 32-bit operands: 32 elements fill a 128-byte row
     if (MODE == 4) return (p.R * p.S * p.Cin + BK - 1) / BK;
     if (MODE == 2) return p.R * p.S * ((p.Cin + BK - 1) / BK);
     const int bk = p.in_dt == FC_F8E4M3 ? 2 * BK : BK;
@@ -241,7 +242,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr bool kConv = MODE == 2 || MODE == 4;   // 4: the convolution with eight filter taps per k-block (TcParams::a_packed)
     const int kb_per_tap = kConv ? (p.Cin + BK - 1) / BK : 1;
     const bool f8 = !kConv && (kMx || p.in_dt == FC_F8E4M3);
-    const int bk = f8 ? 2 * BK : BK;   // K elements per k-block: 128 bytes of a row
+    const int bk = MODE == 7 ? BK / 2 : (f8 ? 2 * BK : BK);   // K elements per k-block: 128 bytes of a row
     const int num_kb = count_kb<MODE>(p);
     const int total_units = p.split > 1 ? p.split_from + (total_tiles - p.split_from) * p.split : total_tiles;
 
@@ -290,7 +291,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int u = cluster_id; u < total_units && ok; u += num_clusters) {
                 const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 int mb2, nb;
-                tile_coords((MODE == 0 || MODE == 6 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
+                tile_coords((MODE == 0 || MODE == 6 || MODE == 7 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
                 const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
@@ -370,7 +371,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (leader && lane == 0) {
             // operand format code: bf16 = 1 and fp16 = 0 under kind::f16, E4M3 = 0 under kind::f8f6f4
-            const uint32_t idesc = ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_BF16 ? 1u : 0u);
+            const uint32_t idesc = MODE == 7 ? ptx::idesc_tf32(2 * BM, BN) : ptx::idesc_f16kind_f32(2 * BM, BN, p.in_dt == FC_BF16 ? 1u : 0u);
             uint32_t it = 0, tile_iter = 0;
             bool ok = true;
             long long pw_tempty = 0, pw_full = 0, pw_issue = 0, pt0 = clock64(), pq = 0;
@@ -422,6 +423,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int k = 1; k < 4; ++k)
                             ptx::tc_mma_mxf8_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, ptx::idesc_mxf8_e4m3(2 * BM, BN, (uint32_t) k, (uint32_t) k), t_sfa, t_sfb, 1u);
+                    } else if constexpr (MODE == 7) {
+                        const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);
+                        const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
+                        ptx::tc_mma_tf32_pair_lh(d_tmem, a_lo, b_lo, desc_hi, idesc, acc0);
+#pragma unroll
+                        for (int k = 1; k < 4; ++k)  // 8 values of 32 bits = 32 bytes per MMA along K -> +2 in 16-byte units
+                            ptx::tc_mma_tf32_pair_lh(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, idesc, 1u);
                     } else {
                         const uint32_t a_lo = desc_lo + s * (uint32_t) (C::kStageBytes >> 4);   // stage s, A tile; B follows kABytes further on
                         const uint32_t b_lo = a_lo + (uint32_t) (C::kABytes >> 4);
@@ -494,7 +502,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int u = cluster_id; u < total_units; u += num_clusters, ++tile_iter) {
             const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
             int mb2, nb;
-            tile_coords((MODE == 0 || MODE == 6 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
+            tile_coords((MODE == 0 || MODE == 6 || MODE == 7 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
             const int mb = mb2 * 2 + (int) cta_rank;    // 128-row panel of this CTA
             const uint32_t buf = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             const int n_tile = nb * BN;
@@ -622,7 +630,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::tmem_wait_st();
             }
 
-            if constexpr (MODE == 0 || MODE == 6) {
+            if constexpr (MODE == 0 || MODE == 6 || MODE == 7) {
                 // one chunk at a time, one copy of the code: load, wait, ops, store (keeping the next load in flight
                 // and two copies of this body was no faster; see tmem_sweep)
 #pragma unroll 1
@@ -1165,6 +1173,7 @@ cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorM
         case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream, plan);
         case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream, plan);
         case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream, plan);
+        case 7: return launch_one<BN, 7>(p, tmA, tmB, num_sms, stream, plan);
         default:
             // (the convolutions have no 240-column form: their widths are the channel counts, powers of two as a rule)
             if constexpr (BN == 240) return cudaErrorInvalidValue;

@@ -142,6 +142,36 @@ __global__ void __launch_bounds__(256) scale_tiles_kernel(const uint8_t* __restr
     }
 }
 
+// fp32 operands for the tensor cores.  A 32-bit value x is cut into hi (sign, exponent and the ten mantissa bits that
+// kind::tf32 reads) and lo = x - hi (exact in fp32; its own upper bits are what the tensor core reads of it).  With
+// A' = [A_lo | A_hi | A_hi] and B' = [B_hi | B_lo | B_hi] along K, A' B'^T = A_hi B_hi + A_hi B_lo + A_lo B_hi: the
+// fp32 product up to the lo x lo terms and the bits of lo beyond its own ten (2^-21 relative per product), accumulated
+// in fp32, the small terms first.  One thread per four consecutive k of a row; K is a multiple of 4.
+__global__ void __launch_bounds__(256) split_tf32_kernel(const float* __restrict__ x, float* __restrict__ y, long long rows, int K, int is_b) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int quads = K >> 2;
+    const long long idx = (long long) blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * quads) return;
+    const long long r = idx / quads;
+    const int q = (int) (idx - r * quads);
+    const float4 v = __ldg(reinterpret_cast<const float4*>(x + r * K) + q);
+    const float in[4] = {v.x, v.y, v.z, v.w};
+    float hi[4], lo[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t b = __float_as_uint(in[j]);
+        const bool finite = (b & 0x7f800000u) != 0x7f800000u;
+        hi[j] = finite ? __uint_as_float(b & 0xffffe000u) : in[j];   // (infinities and NaNs whole, nothing left over)
+        lo[j] = finite ? __uint_as_float(__float_as_uint(in[j] - hi[j]) & 0xffffe000u) : 0.0f;
+        if (!finite && (b & 0x007fffffu)) hi[j] = __uint_as_float(0x7fc00000u);   // a NaN stays one whatever bits it carried
+    }
+    const float4 h4 = make_float4(hi[0], hi[1], hi[2], hi[3]), l4 = make_float4(lo[0], lo[1], lo[2], lo[3]);
+    float4* out = reinterpret_cast<float4*>(y + r * 3 * K);
+    out[q] = is_b ? h4 : l4;
+    out[quads + q] = is_b ? l4 : h4;
+    out[2 * quads + q] = h4;
+}
+
 }  // namespace
 
 size_t scale_tiles_bytes(long long rows, long long K, int tile_rows) {
@@ -165,6 +195,24 @@ cudaError_t launch_scale_tiles(const void* scales, void* tiles, long long rows, 
     note_kernel("scale_tiles");
     ++*launches;
     return cudaLaunchKernelEx(&cfg, scale_tiles_kernel, (const uint8_t*) scales, (uint32_t*) tiles, rows, (int) (K / 32), num_kb, tile_rows, positions);
+}
+
+cudaError_t launch_split_tf32(const float* x, float* y, long long rows, long long K, bool is_b, bool beside_previous, cudaStream_t stream,
+                              int* launches) {
+    const long long total = rows * (K / 4);
+    if (K % 4 || K > 0x7fffffffLL / 3 || total > 0x7fffffffLL * 256) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned) ((total + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = beside_previous ? 1 : 0;
+    note_kernel("split_tf32");
+    ++*launches;
+    return cudaLaunchKernelEx(&cfg, split_tf32_kernel, x, y, rows, (int) K, is_b ? 1 : 0);
 }
 
 cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches) {

@@ -137,6 +137,12 @@ __host__ __device__ constexpr uint32_t idesc_f16kind_f32(int m, int n, uint32_t 
            | ((uint32_t) (m >> 4) << 24); // M / 16
 }
 
+// Instruction descriptor for kind::tf32: 32-bit operands of which the tensor core takes sign, exponent and the upper
+// ten mantissa bits (format code 2), fp32 accumulator, both operands K-major, dense.
+__host__ __device__ constexpr uint32_t idesc_tf32(int m, int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t) (n >> 3) << 17) | ((uint32_t) (m >> 4) << 24);
+}
+
 // 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread (thread i = lane base + i);
 // returns after the data has arrived.
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -234,6 +240,21 @@ __device__ __forceinline__ void tc_mma_f16_pair_lh(uint32_t d_tmem, uint32_t a_l
         "mov.b64 db, {%2, %3};\n\t"
         "setp.ne.b32 p, %5, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// the same for kind::tf32 (8 elements of 32 bits along K per instruction)
+__device__ __forceinline__ void tc_mma_tf32_pair_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                                    uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], da, db, %4, p;\n\t"
         "}"
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");

@@ -65,6 +65,40 @@ def test_gemm_f32_large_register_tiled(fc, orc, M, N, K, plan):
     assert fc.fc_last_plan() == "gemm_f32_" + plan
 
 
+@pytest.mark.parametrize("M,N,K", [(2048, 2048, 2048), (1100, 1300, 516), (700, 4003, 260), (4100, 300, 1024)])
+@pytest.mark.parametrize("variant", ["std", "var"])
+def test_gemm_f32_on_tensor_cores(fc, orc, M, N, K, variant):
+    """fp32 GEMMs of 2^29 multiply-adds and more, K a multiple of 4, with a workspace: two layout launches cut every
+    operand into the part a tf32 multiplication reads and the rest, and the tensor-core kernel contracts
+    [A_lo | A_hi | A_hi] with [B_hi | B_lo | B_hi] in fp32 accumulators.  Same fp32 tolerance as the FMA kernels; ragged
+    extents, rows of the output off 16-byte boundaries."""
+    ch = wl.gemm_bias_relu_f32(M, N, K, variant)
+    run_and_check(fc, orc, ch, 6)
+    assert fc.fc_last_plan().startswith("split_tf32 split_tf32 gemm_tc_mode7_bn")
+    assert fc.binding.fc_describe_plan(fc.make_spec(ch))["kernel"] == "gemm_tc"
+
+
+def test_gemm_f32_large_without_workspace_or_alignment_stays_on_the_alus(fc, orc):
+    """The same sizes without a registered workspace, or with K off the 16-byte grid, take the fp32-FMA kernel."""
+    ch = wl.gemm_bias_relu_f32(1100, 1300, 516, "var")
+    ins = wl.make_inputs(ch, 6)
+    ref = orc.run_chain(ch, ins)
+    spec = fc.make_spec(ch)
+    assert fc.binding.fc_workspace_size(spec) > 0
+    fc.binding.fc_set_workspace(None)
+    fc.binding._workspace.clear()
+    assert fc.binding.fc_describe_plan(spec)["kernel"] == "gemm_f32"
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.fc_run(spec, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    assert fc.fc_last_plan() == "gemm_f32_big"
+    util.check(outs[0], ref["main"], "fp32 GEMM without workspace")
+    ch2 = wl.gemm_bias_relu_f32(1100, 1300, 514, "var")
+    assert fc.binding.fc_workspace_size(fc.make_spec(ch2)) == 0
+    run_and_check(fc, orc, ch2, 6)
+    assert fc.fc_last_plan() == "gemm_f32_big"
+
+
 # ------------------------------------------------------------------ kernel (a): elementwise + logsumexp
 @pytest.mark.parametrize("M,N", [(1, 1), (3, 8), (5, 1000), (7, 4097), (33, 2048), (64, 4096), (9, 12345)])
 def test_elementwise_lse_shapes(fc, orc, M, N):
