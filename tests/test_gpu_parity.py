@@ -78,6 +78,22 @@ def test_gemm_f32_on_tensor_cores(fc, orc, M, N, K, variant):
     assert fc.binding.fc_describe_plan(fc.make_spec(ch))["kernel"] == "gemm_tc"
 
 
+@pytest.mark.parametrize("ops", [
+    (("affine_n", 2, 3), ("gelu_tanh",), ("scale", 0.5), ("clamp", -1.0, 1.0), ("add_tensor", 4)),   # the fused packed form
+    (("relu",), ("bias_n", 2), ("scale", 2.0), ("add_tensor", 4), ("clamp", -0.5, 3.0)),                # interpreted op by op
+    (),
+])
+def test_gemm_f32_on_tensor_cores_op_lists(fc, orc, ops):
+    """The tensor-core form of the fp32 GEMM shares the 16-bit GEMM's epilogue: fp32 vectors and an fp32 residual,
+    fused and interpreted op lists, an empty one; ragged extents at the smallest size that takes this path."""
+    M, N, K = 1030, 1100, 512
+    rec = (("A", "f32", (M, K), "normal", 0.0, K ** -0.25), ("B", "f32", (N, K), "normal", 0.0, K ** -0.25),
+           ("v0", "f32", (N,), "uniform", -0.1, 0.1), ("v1", "f32", (N,), "normal", 1.0, 0.1), ("t", "f32", (M, N), "normal", 0.0, 1.0))
+    ch = wl.Chain("gemm_f32_ops", "gemm_nt", "f32", "f32", M=M, N=N, K=K, ops=ops, input_recipe=rec)
+    run_and_check(fc, orc, ch, 7)
+    assert "gemm_tc_mode7" in fc.fc_last_plan()
+
+
 def test_gemm_f32_large_without_workspace_or_alignment_stays_on_the_alus(fc, orc):
     """The same sizes without a registered workspace, or with K off the 16-byte grid, take the fp32-FMA kernel."""
     ch = wl.gemm_bias_relu_f32(1100, 1300, 516, "var")

@@ -110,6 +110,19 @@ def test_softmax_of_several_rounds_is_not_split(fc, orc):
     fc.binding.fc_set_workspace(None)
 
 
+@pytest.mark.parametrize("kind", ["store", "lse"])
+def test_split_last_round_of_240_column_tiles(fc, orc, kind):
+    """84 tiles of 256 x 240 on 74 pairs: one full round and ten tiles cut along K (the second warp group of a
+    240-column tile has seven chunks: parked and merged slices must leave the eighth, the other buffer's, alone)."""
+    M, N, K = 1536, 3360, 4096
+    ch = wl.gemm_bias_gelu_scale_clamp(M, N, K, "var") if kind == "store" else wl.gemm_bias_scale_lse(M, N, K, "var", True)
+    spec = fc.make_spec(ch)
+    _register(fc, spec, True)
+    plan = fc.binding.fc_describe_plan(spec)
+    assert plan["bn"] == 240 and plan["split"] > 1 and 0 < plan["split_tiles"] < plan["tiles"], plan
+    _run_both(fc, orc, ch, 17)
+
+
 def test_split_fp16(fc, orc):
     ch = wl.gemm_bias_gelu_scale_clamp(192, 520, 4096, "var")
     ch = replace(ch, in_dtype="f16", out_dtype="f16", input_recipe=tuple((t, "f16", sh, d, a, b) for t, _, sh, d, a, b in ch.input_recipe))
