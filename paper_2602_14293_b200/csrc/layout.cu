@@ -161,9 +161,11 @@ __global__ void __launch_bounds__(256) split_tf32_kernel(const float* __restrict
     for (int j = 0; j < 4; ++j) {
         const uint32_t b = __float_as_uint(in[j]);
         const bool finite = (b & 0x7f800000u) != 0x7f800000u;
-        hi[j] = finite ? __uint_as_float(b & 0xffffe000u) : in[j];   // (infinities and NaNs whole, nothing left over)
-        lo[j] = finite ? __uint_as_float(__float_as_uint(in[j] - hi[j]) & 0xffffe000u) : 0.0f;
-        if (!finite && (b & 0x007fffffu)) hi[j] = __uint_as_float(0x7fc00000u);   // a NaN stays one whatever bits it carried
+        // An infinity or a NaN goes to lo whole and leaves hi zero: it then meets only the other operand's hi, as in
+        // the fp32 product (in hi it would also meet the other operand's lo, which is 0 for every value that tf32
+        // represents exactly: inf x 0 = NaN where fp32 gives inf).  Two non-finite values at the same k give NaN.
+        hi[j] = finite ? __uint_as_float(b & 0xffffe000u) : 0.0f;
+        lo[j] = finite ? __uint_as_float(__float_as_uint(in[j] - hi[j]) & 0xffffe000u) : ((b & 0x007fffffu) ? __uint_as_float(0x7fc00000u) : in[j]);
     }
     const float4 h4 = make_float4(hi[0], hi[1], hi[2], hi[3]), l4 = make_float4(lo[0], lo[1], lo[2], lo[3]);
     float4* out = reinterpret_cast<float4*>(y + r * 3 * K);

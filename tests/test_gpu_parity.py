@@ -94,6 +94,30 @@ def test_gemm_f32_on_tensor_cores_op_lists(fc, orc, ops):
     assert "gemm_tc_mode7" in fc.fc_last_plan()
 
 
+def test_gemm_f32_on_tensor_cores_non_finite_operands(fc, orc):
+    """Infinities and NaNs among the operands of the tensor-core fp32 GEMM: every output is an infinity of the right
+    sign, a NaN, or a finite value within tolerance exactly where the fp64 contraction says so (the non-finite values
+    sit at different k, see the split kernel)."""
+    M, N, K = 1030, 1100, 512
+    ch = wl.Chain("gemm_f32_nonfinite", "gemm_nt", "f32", "f32", M=M, N=N, K=K, ops=(),
+                  input_recipe=(("A", "f32", (M, K), "normal", 0.0, K ** -0.25), ("B", "f32", (N, K), "normal", 0.0, K ** -0.25)))
+    A, B = (np.array(t, dtype=np.float32) for t in wl.make_inputs(ch, 8))
+    A[5, 7] = np.inf; A[9, 100] = np.nan; A[700, 300] = -np.inf
+    B[11, 3] = -np.inf; B[900, 44] = np.inf; B[17, 7] = 0.25       # (exactly representable in tf32: its lo part is zero)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(A), fc.to_device(B)], outs)
+    fc.fc_get_async_status()
+    assert "gemm_tc_mode7" in fc.fc_last_plan()
+    got = outs[0].cpu().numpy().astype(np.float64)
+    with np.errstate(invalid="ignore", over="ignore"):
+        ref = A.astype(np.float64) @ B.astype(np.float64).T
+    assert (np.isnan(got) == np.isnan(ref)).all()
+    assert (np.isposinf(got) == np.isposinf(ref)).all() and (np.isneginf(got) == np.isneginf(ref)).all()
+    fin = np.isfinite(ref)
+    assert fin.sum() > 0.99 * ref.size
+    assert (np.abs(got[fin] - ref[fin]) <= 1e-4 * (1.0 + np.abs(ref[fin]))).all()
+
+
 def test_gemm_f32_large_without_workspace_or_alignment_stays_on_the_alus(fc, orc):
     """The same sizes without a registered workspace, or with K off the 16-byte grid, take the fp32-FMA kernel."""
     ch = wl.gemm_bias_relu_f32(1100, 1300, 516, "var")
