@@ -422,7 +422,9 @@ void build_ops(const fc_chain_spec* s, const fc_tensor* in, DevOps* d) {
 
 constexpr int kSoftmaxBN = 256;
 constexpr int kSoftmaxOnePassTiles = 64;       // widest row (in tiles) that the single-pass softmax can take safely
-constexpr int kSoftmaxOnePassBestTiles = 16;   // widest row for which it is also the faster form (measured)
+// where the single pass is also the faster form (measured, see gemm_tile_width): rows of up to 16 tiles at any depth
+// of the contraction, rows of up to 32 tiles from K = 2048 on
+constexpr int kSoftmaxOnePassBestTiles = 16, kSoftmaxOnePassWideTiles = 32, kSoftmaxOnePassWideMinK = 2048;
 
 // arrival counters and departure counters, one of each per 128-row panel
 size_t panel_counter_bytes(long long M) {
@@ -443,17 +445,19 @@ int gemm_tile_width(TcParams& p, const fc_chain_spec* s, int num_sms) {
     if (p.mode == 1) {
         // Row softmax over more tiles per panel than the pairs' accumulator buffers can hold until the panel is
         // complete (two per pair; with a margin: 64 tiles = 16384 columns) cannot wait across tiles: a second,
-        // memory-bound kernel finishes the rows.  The same two-kernel form is also chosen where it is faster.
-        // The single pass wins where it was built for (rows of up to 4096 columns and a long contraction: 4096^3 106
-        // against 118 us); its panel-by-panel order streams B once per panel and its epilogue waits for the
-        // panel, which loses from 8192 columns on and for short contractions (8192 x 16384 x 4096: 1208
-        // against 838 us; 16384 x 16384 x 1024: 2024 against 877 us).
+        // memory-bound kernel finishes the rows.  The same two-kernel form is also chosen where it is faster: the
+        // single pass writes every probability once, the two-kernel form writes, re-reads and re-writes it, but its
+        // tiles run in the L2-friendly order and wait for nobody.  Measured (one pass / two kernels, us): 4096 x 4096 x
+        // K: 37.8 / 40.0 at K = 64, 46.2 / 52.2 at 1024, 58.3 / 70.7 at 2048, 75.7 / 91.2 at 3072, 96 / 118 at 4096;
+        // 4096 x 6144 x 4096 142 / 157; 8192 x 7168 x 4096 329 / 343; 4096 x 8192 x 2048 101 / 110, x 4096 185 / 183;
+        // 8192 x 8192 x 512 150 / 124, x 1024 157 / 142, x 4096 376 / 371; beyond 8192 columns the two kernels win
+        // (8192 x 16384 x 4096: 1208 / 838).
         const int tiles_n = (int) ((s->N + kSoftmaxBN - 1) / kSoftmaxBN);
         TcPlan tp;
         p.two_pass = false;
         // (never more tiles per panel than SM pairs take part, whatever the device offers)
         p.two_pass = plan_gemm_tc(p, kSoftmaxBN, num_sms, &tp) != cudaSuccess || tiles_n > kSoftmaxOnePassTiles || tiles_n > tp.pairs ||
-                     tiles_n > kSoftmaxOnePassBestTiles || s->K < 4096;
+                     tiles_n > kSoftmaxOnePassWideTiles || (tiles_n > kSoftmaxOnePassBestTiles && s->K < kSoftmaxOnePassWideMinK);
         if (p.two_pass) return kSoftmaxBN;
     } else if (p.mode != 0 && p.mode != 3 && p.mode != 7) {
         return 256;

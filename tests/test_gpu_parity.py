@@ -528,13 +528,17 @@ def test_gemm_output_rows_off_16_byte_boundaries(fc, orc, M, N, K, out_dtype):
     run_and_check(fc, orc, replace(wl.gemm_bias_scale_lse(M, N, K, store_main=True), out_dtype=out_dtype), 2)
 
 
-@pytest.mark.parametrize("M,N,K,out_dtype", [(300, 20000, 72, "bf16"), (129, 16640, 136, "bf16"), (260, 16401, 64, "bf16"), (70, 16648, 64, "f32")])
+@pytest.mark.parametrize("M,N,K,out_dtype", [(300, 20000, 72, "bf16"), (129, 16640, 136, "bf16"), (260, 16401, 64, "bf16"), (70, 16648, 64, "f32"),
+                                             (130, 4400, 72, "bf16"), (257, 8190, 136, "f32"), (300, 8448, 4096, "bf16")])
 def test_gemm_softmax_rows_wider_than_one_pass_allows(fc, orc, M, N, K, out_dtype):
     """More than 64 tiles per row panel: the SM pairs cannot hold a whole panel in tensor memory until its last
     tile arrives, so every tile stores its exponentials against its own maximum and a second kernel rescales
-    the rows.  With ops and an additive -inf mask in front, aligned and unaligned rows, bf16 and fp32."""
+    the rows.  The same two-kernel form serves rows of more than 32 tiles, and of more than 16 behind a contraction
+    shorter than 2048, where it is the faster one.  With ops and an additive -inf mask in front, aligned and
+    unaligned rows, bf16 and fp32."""
     base = replace(wl.gemm_softmax(M, N, K, "var"), out_dtype=out_dtype)
     outs, _, _ = run_and_check(fc, orc, base, 5)
+    assert fc.fc_last_plan().endswith("_two_pass softmax_rescale")
     np.testing.assert_allclose(util.to_f64(outs[0]).sum(1), 1.0, atol=3e-2 if out_dtype == "bf16" else 1e-4)
     rec = base.input_recipe + (("mask", "bf16", (M, N), "normal", 0.0, 1.0),)
     ch = replace(base, ops=(("scale", 0.5), ("add_tensor", 2)), input_recipe=rec)
@@ -805,6 +809,13 @@ def test_run_host_chunk_pipeline_matches_device_path(fc, orc):
         for a, b in zip(dev_out, host_out):
             if ch.reduce == "global_avgpool":      # pooled sums are combined with atomics: order varies
                 assert torch.allclose(a.cpu(), b, rtol=1e-5, atol=1e-6)
+            elif ch.producer == "gemm_nt" and ch.reduce == "row_softmax":
+                # the same for the probabilities: a chunk of rows and the whole tensor may take tiles of different
+                # widths (256 and 240 columns), i.e. other groupings of a row's partial sums: equal up to an ulp of
+                # the 16-bit output here and there
+                af, bf = a.cpu().float(), b.float()
+                assert torch.allclose(af, bf, rtol=2 ** -7, atol=1e-9), ch.name
+                assert (af == bf).float().mean() > 0.98, ch.name
             elif ch.producer == "gemm_nt" and ch.reduce == "row_logsumexp" and a.dim() == 1:
                 # per-tile (max, sum) pairs are merged per row; the tile width depends on the row count of the
                 # launch (a chunk of rows may take 128-column tiles where the whole tensor takes 256): same

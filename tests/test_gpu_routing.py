@@ -61,8 +61,10 @@ def test_contraction_routing(fc):
     assert _plan(fc, wl.gemm_softmax(256, 1024, 4096)) == "gemm_tc_mode1_bn256_split"      # 4 tiles: cut along K as well
     assert _plan(fc, wl.gemm_softmax(4096, 4096, 4096)) == "gemm_tc_mode1_bn240"
     assert _plan(fc, wl.gemm_softmax(4096, 1024, 4096)) == "gemm_tc_mode1_bn256"      # one round of 64 tiles against two of 240-column ones
-    assert _plan(fc, wl.gemm_softmax(256, 1024, 256)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"   # short contraction
-    assert _plan(fc, wl.gemm_softmax(256, 8192, 4096)) == "gemm_tc_mode1_bn256_split_two_pass softmax_rescale"  # 32 tiles per panel (and few enough to be cut along K)
+    assert _plan(fc, wl.gemm_softmax(256, 1024, 256)) == "gemm_tc_mode1_bn256"                # rows of up to 16 tiles: one pass at any depth
+    assert _plan(fc, wl.gemm_softmax(256, 8192, 4096)) == "gemm_tc_mode1_bn256_split"         # up to 32 tiles from K = 2048 on (few enough to be cut along K)
+    assert _plan(fc, wl.gemm_softmax(256, 8192, 1024)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"         # 32 tiles behind a short contraction (too short to be cut)
+    assert _plan(fc, wl.gemm_softmax(256, 8448, 4096)) == "gemm_tc_mode1_bn256_split_two_pass softmax_rescale"   # 33 tiles per panel
     assert _plan(fc, wl.gemm_softmax(64, 20000, 64)) == "gemm_tc_mode1_bn256_two_pass softmax_rescale"
     assert _plan(fc, wl.gemm_bias_scale_lse(256, 1024, 256)) == "gemm_tc_mode3_bn128"       # few tiles: as the plain GEMM
     assert _plan(fc, wl.gemm_bias_scale_lse(2048, 4096, 256)) == "gemm_tc_mode3_bn240"
