@@ -325,6 +325,8 @@ int fc_version(void);
 #define FC_TESTING_PANEL_STALL 0
 #define FC_TESTING_SPLIT_STALL 1
 #define FC_TESTING_BOUNDS_TRIP 2   /* debug build only: value 1 shortens the checked extent of the main output by one row */
+#define FC_TESTING_TILE_WIDTH 3    /* value 128, 240 or 256: the column-tile width of every tensor-core GEMM that has a choice
+                                      (plain store, row reductions, single-pass softmax, the fp32 form); 0: the launcher's own */
 void fc_testing_set(int which, int value);
 
 #ifdef __cplusplus

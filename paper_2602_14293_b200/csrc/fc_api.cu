@@ -16,7 +16,7 @@ __device__ int g_status_word;  // written by kernels when a bounded wait expires
 namespace {
 
 // testing switches (fc_testing_set): read on every call, written by tests only
-std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0}, g_bounds_trip{0};
+std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0}, g_bounds_trip{0}, g_force_tile_width{0};
 
 thread_local int t_device = 0;   // ordinal of the current device, noted by get_device at the top of every entry point
 thread_local char t_err[512] = "";
@@ -461,9 +461,16 @@ int gemm_tile_width(TcParams& p, const fc_chain_spec* s, int num_sms) {
         if (p.two_pass) return kSoftmaxBN;
     } else if (p.mode != 0 && p.mode != 3 && p.mode != 7) {
         return 256;
-    } else if (s->N <= 128) {
-        return 128;
     }
+    // testing only (fc_testing_set): a given width for every call that could take it, so that the tests can run one
+    // shape on all three tile widths
+    const int forced = g_force_tile_width.load(std::memory_order_relaxed);
+    if (forced == 128 || forced == 240 || forced == 256) {
+        TcPlan tp;
+        const long long tn = (s->N + forced - 1) / forced;
+        if (p.mode != 1 || (plan_gemm_tc(p, forced, num_sms, &tp) == cudaSuccess && tn <= tp.pairs && tn <= kSoftmaxOnePassTiles)) return forced;
+    }
+    if (p.mode != 1 && s->N <= 128) return 128;
     const long long tiles = ((s->M + 255) / 256) * ((s->N + 255) / 256);
     if (2 * tiles <= num_sms / 2) {
         if (p.mode == 1) return kSoftmaxBN;
@@ -1174,6 +1181,7 @@ void fc_testing_set(int which, int value) {
     if (which == FC_TESTING_PANEL_STALL) g_inject_panel_stall.store(value);
     else if (which == FC_TESTING_SPLIT_STALL) g_inject_split_stall.store(value);
     else if (which == FC_TESTING_BOUNDS_TRIP) g_bounds_trip.store(value);
+    else if (which == FC_TESTING_TILE_WIDTH) g_force_tile_width.store(value);
 }
 
 }  // extern "C"

@@ -458,6 +458,32 @@ def test_gemm_240_column_tiles(fc, orc, M, N, K):
     assert fc.fc_last_plan() == "gemm_tc_mode3_bn240"
 
 
+@pytest.mark.parametrize("width", [128, 240, 256])
+def test_one_shape_on_every_tile_width(fc, orc, width):
+    """The testing switch FC_TESTING_TILE_WIDTH pins the column-tile width: the same ragged shapes through the plain
+    store (bf16 and fp32 output), the row reductions, the single-pass softmax and the fp32 form on 128-, 240- and
+    256-column tiles."""
+    b = fc.binding
+    b.fc_testing_set(b.FC_TESTING_TILE_WIDTH, width)
+    try:
+        M, N, K = 600, 1000, 264
+        ch = wl.gemm_bias_gelu_scale_clamp(M, N, K, "var")
+        run_and_check(fc, orc, ch, 31)
+        assert fc.fc_last_plan().startswith(f"gemm_tc_mode0_bn{width}")
+        run_and_check(fc, orc, replace(ch, out_dtype="f32"), 31)
+        run_and_check(fc, orc, replace(wl.gemm_bias_gelu_scale_clamp(M, 999, K, "var"), out_dtype="f32"), 31)
+        run_and_check(fc, orc, wl.gemm_bias_scale_lse(M, N, K, "var", True), 32)
+        assert fc.fc_last_plan().startswith(f"gemm_tc_mode3_bn{width}")
+        run_and_check(fc, orc, wl.linear_row_reduce(M, N, K, "row_max", ops=(("bias_n", 2), ("relu",)), store_main=False), 32)
+        outs, _, _ = run_and_check(fc, orc, wl.gemm_softmax(M, N, K, "var"), 33)
+        assert fc.fc_last_plan().startswith(f"gemm_tc_mode1_bn{width}") and "two_pass" not in fc.fc_last_plan()
+        _check_softmax_rows(outs[0])
+        run_and_check(fc, orc, wl.gemm_bias_relu_f32(1030, 1100, 512, "var"), 34)
+        assert f"gemm_tc_mode7_bn{width}" in fc.fc_last_plan()
+    finally:
+        b.fc_testing_set(b.FC_TESTING_TILE_WIDTH, 0)
+
+
 @pytest.mark.parametrize("M,N", [(520, 4000), (600, 3999), (777, 3856)])
 def test_gemm_softmax_240_column_tiles(fc, orc, M, N):
     """The single-pass row softmax on 240-column tiles: 17 tiles per panel, the last one ragged."""
