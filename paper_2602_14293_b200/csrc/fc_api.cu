@@ -432,15 +432,15 @@ size_t panel_counter_bytes(long long M) {
     return ((size_t) panels * 4 + 255) / 256 * 256;
 }
 
-// Column-tile width of the GEMM kernels (modes 0, 1, 3), and for the row softmax the choice between its two forms.
+// Column-tile width of the GEMM kernels (modes 0, 1, 3, 7), and for the row softmax the choice between its two forms.
 // Small GEMMs (modes 0 and 3, 256-wide tiles on at most half of the SM pairs) take 128-wide tiles where this
 // cost model says so.  Such a call is one round of tiles, so its time is the critical tile's: main loop (of the
 // merging slice, when tiles are cut along K) + epilogue + merge.  Measured, in microseconds: a k-block 0.33
 // (256 wide) / 0.30 (128 wide; 24 instead of 32 KB), the epilogue 6 / 3, merging a split tile 8 / 4.4.
 // 128 x 1024 x 1024: 13.7 -> 11.2; 256 x 4096 x 4096: 23.0 -> 20.1; 16 x 8192 x 8192 stays at 256 (37 against 45).
 // Everything else is rounds of tiles whose main loops the tensor pipe bounds, so the time goes with
-// rounds x tile width: 240-column tiles where that product is smaller (4096 columns: 18 tiles per panel, 288
-// tiles = 4 rounds on 72 pairs x 240 against 4 rounds x 256).  `p` has its split scratch attached already.
+// rounds x tile width: 240-column tiles where that product is smaller (4096 x 4096: 288 tiles = 4 rounds x 240
+// against 256 tiles = 4 rounds x 256 on 74 pairs).  `p` has its split scratch attached already.
 int gemm_tile_width(TcParams& p, const fc_chain_spec* s, int num_sms) {
     if (p.mode == 1) {
         // Row softmax over more tiles per panel than the pairs' accumulator buffers can hold until the panel is
