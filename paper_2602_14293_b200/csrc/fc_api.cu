@@ -859,7 +859,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             build_ops(spec, inputs, &p.ops);
             p.out = (float*) outputs[plan.red_index].ptr;
             p.post = spec->reduce == FC_RED_ROW_MEAN ? 1.0f / (float) spec->N : 1.0f;
-            e = launch_collapse(p, dev->workspace, stream, &launches);
+            e = launch_collapse(p, dev->workspace, dev->num_sms, stream, &launches);
             break;
         }
         case Plan::TC_CONV: {

@@ -79,7 +79,7 @@ struct CollapseParams {
     // carved out of the workspace by the launcher
     double* partial; double* cpart; double* cterm; float* u;
 };
-cudaError_t launch_collapse(const CollapseParams& p, void* workspace, cudaStream_t stream, int* launches);
+cudaError_t launch_collapse(const CollapseParams& p, void* workspace, int num_sms, cudaStream_t stream, int* launches);
 size_t collapse_workspace_bytes(long long N, long long K);
 
 // Appends the name of a kernel variant to this thread's record of what the current fc_run enqueues (fc_last_plan).
