@@ -29,6 +29,8 @@ def fc():
     lambda: wl.gemm_bias_gelu_scale_clamp(128, 256, 4096, "var"),          # split tiles
     lambda: wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128),
     lambda: wl.linear_row_reduce(96, 512, 256, variant="var"),             # three kernels
+    lambda: wl.gemm_bias_relu_f32(1030, 1100, 512, "var"),                 # fp32 on the tensor cores: two split launches + the GEMM
+    lambda: wl.gemm_softmax(600, 4000, 4096, "var"),                       # single-pass softmax on 240-column tiles
 ])
 def test_captured_chain_replays(fc, orc, make):
     ch = make()
