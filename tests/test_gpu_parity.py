@@ -820,7 +820,8 @@ def test_run_host_chunk_pipeline_matches_device_path(fc, orc):
              wl.conv_bias_relu_avgpool(batch=20), wl.conv_bias_relu_maxpool(batch=24, H=56, W=56, Cin=128, Cout=64, R=3, S=3, pad=1),
              wl.mlp(33000, (512, 256, 64)), wl.linear_row_reduce(20000, 1024, 1024),
              wl.scale_add_softmax(5000, 4096), wl.scale_add_softmax(300000, 64), wl.scale_add_softmax(700, 50257),
-             wl.gemm_softmax(1100, 20000, 256, "var"), wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=20))]
+             wl.gemm_softmax(1100, 20000, 256, "var"), wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=20)),
+             wl.gemm_bias_relu_f32(3000, 3000, 1024, "var")]   # (fp32 on the tensor cores: whole tensors, no chunks)
     for ch in cases:
         ins = wl.make_inputs(ch, 1)
         host_in = [fc.to_device(a, "cpu").pin_memory() for a in ins]
