@@ -606,15 +606,25 @@ fc_status encode_scale_tiles(CUtensorMap* tm, const void* ptr, long long tile_ro
 // into a k-block instead cuts a 5 x 5 filter from 25 k-blocks to 4.  The eight small copies of such a k-block
 // cost about 1.9 us against 0.35 - 0.65 us for one 64-channel copy (measured), so from 16 channels on the
 // one-tap k-blocks are as fast or faster.
-bool packed_taps(const fc_chain_spec* s) { return s->Cin == 8; }
+// Few input channels without padding: in channels-last storage the S taps of one filter row are S * Cin contiguous
+// elements per output position, so a tensor map whose "pixel" has S * Cin channels and whose pixels lie Cin
+// elements apart (they overlap) fetches a whole filter row of 128 positions in one im2col copy of 128-byte rows; what
+// the 64-element box asks for beyond S * Cin is out of range and arrives as zeros, so the weight columns that the B
+// tile holds there (the next filter row's) meet zeros.  A k-block per filter row: 5 x 5 x 8 costs 5 k-blocks of one
+// copy each instead of 4 of eight 16-byte-row copies (measured: 1.9 us per such k-block in the TMA unit).  Not with
+// padding: a position whose first tap lies left of the image would lose its whole row, not just that tap.
+bool row_taps(const fc_chain_spec* s) { return s->Cin % 8 == 0 && s->S > 1 && s->S * s->Cin <= 64 && s->pad == 0; }
+bool packed_taps(const fc_chain_spec* s) { return s->Cin == 8 && !row_taps(s); }
 
 // `packed`: copies of 8 channels x 128 pixels without swizzle (one column of 8 x 16-byte core matrices each), for
 // channel counts that do not fill 64-channel k-blocks; otherwise 64 channels x 128 pixels with 128-byte swizzle.
 fc_status encode_im2col(CUtensorMap* tm, const fc_chain_spec* s, const void* ptr, bool packed) {
     const int dev = t_device;
-    const MapKey mk = {ptr, {packed ? 5 : 4, s->batch * 65536 + dev, s->H, s->W, s->Cin, s->R * 64 + s->S, s->stride * 64 + s->pad, s->in_dtype}};
+    const bool rows = !packed && row_taps(s);
+    const MapKey mk = {ptr, {packed ? 5 : (rows ? 6 : 4), s->batch * 65536 + dev, s->H, s->W, s->Cin, s->R * 64 + s->S, s->stride * 64 + s->pad, s->in_dtype}};
     if (g_maps.find(mk, tm)) return FC_OK;
-    const cuuint64_t dims[4] = {(cuuint64_t) s->Cin, (cuuint64_t) s->W, (cuuint64_t) s->H, (cuuint64_t) s->batch};
+    // (row taps: a "pixel" of S * Cin channels; the pixel stride stays Cin elements)
+    const cuuint64_t dims[4] = {(cuuint64_t) (rows ? s->S * s->Cin : s->Cin), (cuuint64_t) s->W, (cuuint64_t) s->H, (cuuint64_t) s->batch};
     const cuuint64_t strides[3] = {(cuuint64_t) s->Cin * 2, (cuuint64_t) s->W * s->Cin * 2, (cuuint64_t) s->H * s->W * s->Cin * 2};
     // base pixels run over the output grid shifted by -pad; a filter tap adds (s, r) to every base pixel
     const int lower[2] = {(int) -s->pad, (int) -s->pad};
@@ -642,6 +652,7 @@ int conv_params(const fc_chain_spec* spec, long long out_rows, TcParams* p) {
     p->inv_hw = 1.0f / (float) (p->OH * p->OW);
     p->pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? 1 : 0;
     p->a_packed = packed_taps(spec);
+    p->a_rowtaps = row_taps(spec);
     const int bn = spec->Cout <= 128 ? 128 : 256;
     return bn;
 }

@@ -210,6 +210,7 @@ template <int MODE>
 __host__ __device__ __forceinline__ int count_kb(const TcParams& p) {
     if (MODE == 7) return (p.K + BK / 2 - 1) / (BK / 2);   // 32-bit operands: 32 elements fill a 128-byte row
     if (MODE == 4) return (p.R * p.S * p.Cin + BK - 1) / BK;
+    if (MODE == 5) return p.R;   // a k-block per filter row (TcParams::a_rowtaps)
     if (MODE == 2) return p.R * p.S * ((p.Cin + BK - 1) / BK);
     const int bk = p.in_dt == FC_F8E4M3 ? 2 * BK : BK;
     return (p.K + bk - 1) / bk;
@@ -239,7 +240,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM);   // pair-panels of 256 rows
     const int tiles_n = (p.N + BN - 1) / BN;
     const int total_tiles = tiles_m * tiles_n;
-    constexpr bool kConv = MODE == 2 || MODE == 4;   // 4: the convolution with eight filter taps per k-block (TcParams::a_packed)
+    // 4: the convolution with eight filter taps per k-block (TcParams::a_packed); 5: with a filter row per k-block
+    // (TcParams::a_rowtaps).  Instantiations of their own: as run-time branches of mode 2's producer either of them
+    // cost the ordinary convolution 2 - 10 %.
+    constexpr bool kConv = MODE == 2 || MODE == 4 || MODE == 5;
     const int kb_per_tap = kConv ? (p.Cin + BK - 1) / BK : 1;
     const bool f8 = !kConv && (kMx || p.in_dt == FC_F8E4M3);
     const int bk = MODE == 7 ? BK / 2 : (f8 ? 2 * BK : BK);   // K elements per k-block: 128 bytes of a row
@@ -310,6 +314,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tap_r = tap / p.S;
                     tap_s = tap - tap_r * p.S;
                     tap_col = tap * p.Cin;
+                } else if constexpr (MODE == 5) {
+                    // a k-block per filter row: all S taps of the row in one copy (tap offset (0, r)), the row's
+                    // S * Cin weights from column r * S * Cin on
+                    tap_r = w.kb0;
+                    tap_col = w.kb0 * p.S * p.Cin;
                 }
                 for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     const uint32_t s = hs, ph = hph;
@@ -355,6 +364,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             tap_col += p.Cin;
                             if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
                         }
+                    } else if constexpr (MODE == 5) {
+                        ptx::tma_load_im2col_4d_pair(sa, &tmA, 0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) 0, (uint16_t) tap_r, full);
+                        ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap_col, bcol0, full);
+                        tap_col += p.S * p.Cin;
+                        ++tap_r;
                     } else {
                         ptx::tma_load_2d_pair(sa, &tmA, kb * bk, row0, full);
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * bk, bcol0, full);
@@ -1156,7 +1170,8 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
     cfg.numAttrs = 2;   // cluster shape + programmatic stream serialization
     {
         char name[64];
-        snprintf(name, sizeof(name), "gemm_tc_mode%d_bn%d%s%s", MODE, BN, q.split > 1 ? "_split" : "", MODE == 1 && p.two_pass ? "_two_pass" : "");
+        snprintf(name, sizeof(name), "gemm_tc_mode%d_bn%d%s%s%s", MODE == 5 ? 2 : MODE, BN, q.split > 1 ? "_split" : "", MODE == 1 && p.two_pass ? "_two_pass" : "",
+                 MODE == 5 ? "_rowtaps" : "");
         note_kernel(name);
     }
     // (the scale-tile maps are read in mode 6 only; the other modes get the operand maps again)
@@ -1174,7 +1189,9 @@ cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorM
         default:
             // (the convolutions have no 240-column form: their widths are the channel counts, powers of two as a rule)
             if constexpr (BN == 240) return cudaErrorInvalidValue;
-            else return p.a_packed ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan) : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
+            else return p.a_packed    ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan)
+                      : p.a_rowtaps ? launch_one<BN, 5>(p, tmA, tmB, num_sms, stream, plan)
+                                    : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
     }
 }
 

@@ -748,6 +748,44 @@ def test_conv_eight_channels_packs_filter_taps(fc, orc, R, S, pad, stride, pool)
     run_and_check(fc, orc, ch, 9)
 
 
+@pytest.mark.parametrize("Cin,R,S,stride", [(8, 5, 5, 1), (8, 3, 3, 1), (16, 3, 3, 1), (8, 7, 7, 2), (32, 2, 2, 1), (16, 4, 4, 2), (24, 3, 2, 1), (8, 1, 8, 1)])
+@pytest.mark.parametrize("pool", ["avg", "max"])
+def test_conv_few_channels_without_padding_takes_filter_rows(fc, orc, Cin, R, S, stride, pool):
+    """Unpadded convolutions of few input channels (S * Cin <= 64): a k-block is one filter row, fetched as one copy
+    through a tensor map whose "pixels" are S * Cin channels wide and overlap (what the 64-element box asks for beyond
+    them is out of range and arrives as zeros).  Ragged images, strides, both poolings; the last image's last rows sit
+    at the end of the tensor."""
+    make = wl.conv_bias_relu_avgpool if pool == "avg" else wl.conv_bias_relu_maxpool
+    ch = make(batch=3, H=19, W=23, Cin=Cin, Cout=40, R=R, S=S, pad=0, stride=stride)
+    run_and_check(fc, orc, ch, 11)
+    assert fc.fc_last_plan().endswith("_rowtaps")
+    # with padding the same shapes keep the tap-by-tap traversal
+    if min(R, S) > 1:
+        run_and_check(fc, orc, make(batch=2, H=19, W=23, Cin=Cin, Cout=40, R=R, S=S, pad=1, stride=stride), 11)
+        assert "rowtaps" not in fc.fc_last_plan()
+
+
+def test_conv_filter_rows_delta_taps_bit_exact(fc):
+    """One-hot filters pin which tap and channel every column of a filter-row k-block multiplies: output channel co
+    copies input channel c shifted by (r, s), exactly (average over the image of ReLU of the shifted channel)."""
+    B, H, W, R, S = 2, 12, 14, 5, 5
+    ch = replace(wl.conv_bias_relu_maxpool(batch=B, H=H, W=W, Cin=8, Cout=32, R=R, S=S, pad=0), ops=(("relu",),))
+    ins = wl.make_inputs(ch, 4)
+    x = rng.bf16_bits_to_f32(ins[0])
+    w = np.zeros((32, R, S, 8), dtype=np.float32)
+    taps = [(co % 25 // 5, co % 25 % 5, (3 * co) % 8) for co in range(32)]
+    for co, (r, s, c) in enumerate(taps):
+        w[co, r, s, c] = 1.0
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(ins[0]), fc.to_device(rng.store(w, "bf16"))], outs)
+    fc.fc_get_async_status()
+    assert fc.fc_last_plan().endswith("_rowtaps")
+    OH, OW = H - R + 1, W - S + 1
+    want = np.stack([np.maximum(x[:, r:r + OH, s:s + OW, c], 0) for r, s, c in taps], axis=-1)
+    want = want.reshape(B, OH // 2, 2, OW // 2, 2, 32).max(axis=(2, 4))
+    assert np.array_equal(outs[0].cpu().numpy(), want)
+
+
 def test_conv_eight_channels_delta_taps_bit_exact(fc):
     """One-hot filter (tap (r, s), channel c -> output channel): the max-pooled output is the pooled ReLU of a
     shifted image channel, exactly; every tap of a 5 x 5 filter in turn lands in a different chunk of the

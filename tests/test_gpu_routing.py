@@ -74,4 +74,5 @@ def test_contraction_routing(fc):
     conv = wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128)
     assert _plan(fc, conv) == "zero_fill gemm_tc_mode2_bn128"
     assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=2)) == "zero_fill gemm_tc_mode4_bn256"
+    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=0)) == "zero_fill gemm_tc_mode2_bn256_rowtaps"
     assert _plan(fc, wl.conv_nchw(conv)) == "cfirst_to_clast cfirst_to_clast zero_fill gemm_tc_mode2_bn128"
