@@ -118,7 +118,8 @@ struct TcParams {
     // mode 2
     int batch, H, W, Cin, Cout, R, S, stride, pad, OH, OW;
     float inv_hw;
-    int pool;                   // mode 2: 0 global average pool, 1 2x2 max-pool (out pre-zeroed, values >= 0)
+    int pool;                   // mode 2: 0 global average pool; 2x2 max-pool (out pre-zeroed, values >= 0): 1 through atomics,
+                                // 2 with the windows inside a tile finished on chip (narrow outputs)
     int two_pass;               // mode 1: rows wider than the tiles the SM pairs can hold at once: no waiting across tiles; every
                                 // tile stores its exponentials against its own maximum and leaves (max, sum) in `stats`,
                                 // launch_softmax_rescale finishes the rows

@@ -1017,6 +1017,86 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     __syncwarp();
                 });
+            } else if (p.pool == 2) {
+                // conv + 2x2 max-pool of non-negative values for narrow outputs (the op list ends with ReLU, the output starts
+                // at zero; chosen by the caller where most windows lie inside one tile: OW <= 32).
+                // The 128 positions of this CTA's tile are consecutive in (image, row, column) order, and the four
+                // warps of a column half stage their values of a 16-channel chunk in one buffer, position by position.
+                // A window whose upper-left position lies at least OW + 1 positions in front of the tile's end has
+                // all four of its positions in that buffer: it is finished here and stored.  The other windows meet
+                // their second row through an unsigned atomic maximum on the fp32 bit pattern, as before (their
+                // positions sit in two tiles).  Which positions emit, what they cover and where they write does not
+                // depend on the channel chunk: listed once per tile, so that in every chunk a half-warp serves one
+                // entry with one channel per lane (16 consecutive channels per store or atomic).
+                const int hw = p.OH * p.OW, PH = p.OH >> 1, PW = p.OW >> 1;
+                const int q = lane_grp * 32 + lane;        // this thread's position in the tile
+                int win = 0;
+                bool emit = false, right = false, vert = false;
+                if (m < p.M) {
+                    const int img = (int) (m / hw);
+                    const int rem = (int) (m - (long long) img * hw);
+                    const int oh = rem / p.OW, ow = rem - oh * p.OW;
+                    if ((oh >> 1) < PH && (ow >> 1) < PW) {
+                        win = (img * PH + (oh >> 1)) * PW + (ow >> 1);      // window index, below 2^31 like the position index
+                        if ((ow & 1) == 0) {
+                            right = q < BM - 1;                             // the right neighbour (same row) is in this tile
+                            const bool top = (oh & 1) == 0;
+                            vert = top && right && q + p.OW + 1 <= BM - 1;  // and so is the row below
+                            // a lower-left position whose window the upper-left one finishes (that one is OW in front)
+                            const bool covered = !top && q >= p.OW && q <= BM - 2;
+                            emit = !covered;
+                        } else {
+                            emit = q == 0;                                  // its left neighbour sits in the tile in front
+                        }
+                    }
+                }
+                int* pool_cnt = reinterpret_cast<int*>(xchg) + half * 256;           // [4] emitters per warp, then the entries
+                int2* pool_tab = reinterpret_cast<int2*>(pool_cnt + 4);             // up to 65: (position | flags, window)
+                const unsigned emask = __ballot_sync(0xffffffffu, emit);
+                if (lane == 0) pool_cnt[lane_grp] = __popc(emask);
+                ptx::bar_sync(3 + half, 128);
+                int before = 0, n_emit = 0;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    const int cg = pool_cnt[g];
+                    before += g < lane_grp ? cg : 0;
+                    n_emit += cg;
+                }
+                if (emit) pool_tab[before + __popc(emask & ((1u << lane) - 1u))] = make_int2(q | (right ? 128 : 0) | (vert ? 256 : 0), win);
+                ptx::bar_sync(3 + half, 128);
+                float* stage = pool_stage + half * (BM * 17);     // [position][16 channels + 1]
+                unsigned int* out_u = (unsigned int*) p.out;
+                const int ch = lane & 15, hwid = q >> 4;           // channel of the chunk, half-warp 0..7 of the column half
+                const int below = p.OW * 17;
+                tmem_sweep16<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                    const int n0 = n_half + c * 16;
+                    if (n0 >= p.N) return;
+                    float v[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+                    if (m < p.M) apply_ops16<false>(v, p.ops, svec, BN, col_half + c * 16, m, n0, p.N, p.N);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (FC_DBG_IN(&stage[q * 17 + j], 4, pool_stage, (long long) C::kPoolBytes, p.status, kSitePoolStage)) stage[q * 17 + j] = v[j];
+                    ptx::bar_sync(3 + half, 128);
+                    if (n0 + ch < p.N) {
+                        for (int e = hwid; e < n_emit; e += 8) {
+                            const int2 ent = pool_tab[e];
+                            const float* sp = stage + (ent.x & 127) * 17 + ch;
+                            float x = sp[0];
+                            if (ent.x & 128) x = fmaxf(x, sp[17]);
+                            unsigned int* dst = out_u + (long long) ent.y * p.N + n0 + ch;
+                            if (!FC_DBG_IN(dst, 4, p.out, (long long) p.batch * PH * PW * p.N * 4, p.status, kSitePoolMax)) continue;
+                            if (ent.x & 256) {
+                                x = fmaxf(x, fmaxf(sp[below], sp[below + 17]));
+                                *dst = __float_as_uint(x) & 0x7fffffffu;
+                            } else {
+                                atomicMax(dst, __float_as_uint(x) & 0x7fffffffu);
+                            }
+                        }
+                    }
+                    ptx::bar_sync(3 + half, 128);
+                });
             } else {
                 // conv + global average pool: channel sums over this warp's 32 pixels
                 const int hw = p.OH * p.OW;
