@@ -656,7 +656,10 @@ int conv_params(const fc_chain_spec* spec, long long out_rows, TcParams* p) {
     p->pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? (p->OW <= 32 ? 2 : 1) : 0;
     p->a_packed = packed_taps(spec);
     p->a_rowtaps = row_taps(spec);
-    const int bn = spec->Cout <= 128 ? 128 : 256;
+    // (up to 64 output channels: 64-column tiles, so that both column halves of the epilogue warps have work: with
+    // 128-column tiles half of them idled and a 5 x 5 x 8 -> 64 layer, whose five k-blocks per tile the epilogue cannot
+    // hide behind, was bound by the other half)
+    const int bn = spec->Cout <= 64 ? 64 : (spec->Cout <= 128 ? 128 : 256);
     return bn;
 }
 

@@ -1261,17 +1261,22 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
 template <int BN>
 cudaError_t launch_bn(const TcParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB, int num_sms, cudaStream_t stream,
                       TcPlan* plan) {
-    switch (p.mode) {
-        case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream, plan);
-        case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream, plan);
-        case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream, plan);
-        case 7: return launch_one<BN, 7>(p, tmA, tmB, num_sms, stream, plan);
-        default:
-            // (the convolutions have no 240-column form: their widths are the channel counts, powers of two as a rule)
-            if constexpr (BN == 240) return cudaErrorInvalidValue;
-            else return p.a_packed    ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan)
-                      : p.a_rowtaps ? launch_one<BN, 5>(p, tmA, tmB, num_sms, stream, plan)
-                                    : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
+    if constexpr (BN != 64) {   // (64-column tiles: convolutions of at most 64 output channels only)
+        switch (p.mode) {
+            case 0: return launch_one<BN, 0>(p, tmA, tmB, num_sms, stream, plan);
+            case 1: return launch_one<BN, 1>(p, tmA, tmB, num_sms, stream, plan);
+            case 3: return launch_one<BN, 3>(p, tmA, tmB, num_sms, stream, plan);
+            case 7: return launch_one<BN, 7>(p, tmA, tmB, num_sms, stream, plan);
+            default: break;
+        }
+    }
+    // (the convolutions have no 240-column form: their widths are the channel counts, powers of two as a rule)
+    if constexpr (BN == 240) return cudaErrorInvalidValue;
+    else {
+        if (p.mode != 2) return cudaErrorInvalidValue;
+        return p.a_packed    ? launch_one<BN, 4>(p, tmA, tmB, num_sms, stream, plan)
+             : p.a_rowtaps ? launch_one<BN, 5>(p, tmA, tmB, num_sms, stream, plan)
+                           : launch_one<BN, 2>(p, tmA, tmB, num_sms, stream, plan);
     }
 }
 
@@ -1279,6 +1284,7 @@ cudaError_t launch_any(const TcParams& p, const CUtensorMap* tmA, const CUtensor
                        TcPlan* plan) {
     return bn == 256 ? launch_bn<256>(p, tmA, tmB, num_sms, stream, plan)
          : bn == 240 ? launch_bn<240>(p, tmA, tmB, num_sms, stream, plan)
+         : bn == 64  ? launch_bn<64>(p, tmA, tmB, num_sms, stream, plan)
                      : launch_bn<128>(p, tmA, tmB, num_sms, stream, plan);
 }
 
@@ -1290,7 +1296,7 @@ extern "C" void fc_debug_prof_epi(long long* out) { cudaMemcpyFromSymbol(out, g_
 extern "C" void fc_debug_prof_clk(long long* out) { cudaMemcpyFromSymbol(out, g_prof_clk, sizeof(long long) * 160 * 64); }
 #endif
 
-size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : bn == 240 ? Cfg<240>::kSmemBytes : Cfg<128>::kSmemBytes; }
+size_t gemm_tc_smem_bytes(int bn) { return bn == 256 ? Cfg<256>::kSmemBytes : bn == 240 ? Cfg<240>::kSmemBytes : bn == 64 ? Cfg<64>::kSmemBytes : Cfg<128>::kSmemBytes; }
 
 cudaError_t launch_gemm_tc(const TcParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int num_sms,
                            cudaStream_t stream, int* launches) {
