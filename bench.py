@@ -225,8 +225,9 @@ def eager_fn(ch, t):
 
 
 def network_entry(fc, binding, flush, with_eager, batch=4096):
-    """The LeNet-shaped network (conv -> ReLU -> max-pool twice, three linear layers) as five chains per step, every
-    stage reading the previous stage's output in place; the unfused eager network on the same tensors beside it."""
+    """The LeNet-shaped network (conv -> ReLU -> max-pool twice, three linear layers) as three chains per step (the
+    pooled outputs stored in bf16, the next layer's operand type), every stage reading the previous stage's output in
+    place; the unfused eager network on the same tensors beside it."""
     import torch
     import torch.nn.functional as F
     stages = wl.lenet_shaped(batch)
@@ -251,7 +252,7 @@ def network_entry(fc, binding, flush, with_eager, batch=4096):
     ent = {"ms": ms, "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "bound": "tensor", "chains_per_step": len(stages),
            "workload": f"LeNet-shaped network, batch {batch}: conv5x5 8->64 + ReLU + pool, conv5x5 64->128 + ReLU + pool, 3200->120->88->10"}
     if with_eager:
-        c1, c2, fcs = tensors[0], tensors[2], tensors[4]
+        c1, c2, fcs = tensors[0], tensors[1], tensors[2]
         x = c1[0].permute(0, 3, 1, 2)
         w1, w2 = c1[1].permute(0, 3, 1, 2), c2[1].permute(0, 3, 1, 2)
 

@@ -48,6 +48,11 @@ class Chain:
     input_recipe: Tuple[tuple, ...] = field(default=(), compare=False)
 
     @property
+    def pooled_dtype(self) -> str:
+        """Storage of a 2x2 max-pool's output: the chain's out_dtype when that is a 16-bit type, else f32."""
+        return self.out_dtype if self.out_dtype in ("bf16", "f16") else "f32"
+
+    @property
     def OH(self) -> int:
         return (self.H + 2 * self.pad - self.R) // self.stride + 1
 
@@ -214,15 +219,19 @@ def cast(M: int, N: int, in_dtype="f32", out_dtype="bf16") -> Chain:
                  store_main=True, input_recipe=(("x", in_dtype, (M, N), "normal", 0.0, 1.0),))
 
 
-def lenet_shaped(batch=64, C0=8, C1=64, C2=128, widths=(120, 88, 10)):
+def lenet_shaped(batch=64, C0=8, C1=64, C2=128, widths=(120, 88, 10), pooled="bf16"):
     """The shape of the paper's Level-3 example network (LeNet-5) as a sequence of chains, at tensor-core-sized channel counts:
     conv 5x5 -> ReLU -> 2x2 max-pool, twice (32x32 -> 28 -> 14 -> 10 -> 5), then three linear layers kept on chip.
-    The first input of every stage after the first is the previous stage's output (same bytes, reshaped)."""
+    The first input of every stage after the first is the previous stage's output (same bytes, reshaped).
+    pooled="bf16": the pooled outputs are stored in the next layer's operand type (three chains); "f32": they are
+    fp32 and a cast chain behind each re-stores them (five chains)."""
     s1 = conv_bias_relu_maxpool(batch=batch, H=32, W=32, Cin=C0, Cout=C1, R=5, S=5, pad=0)
     s2 = conv_bias_relu_maxpool(batch=batch, H=14, W=14, Cin=C1, Cout=C2, R=5, S=5, pad=0)
     flat = 5 * 5 * C2
-    return [replace(s1, name="lenet_conv1"), cast(batch, 14 * 14 * C1), replace(s2, name="lenet_conv2"), cast(batch, flat),
-            replace(mlp(batch, (flat,) + tuple(widths)), name="lenet_fc")]
+    fc3 = replace(mlp(batch, (flat,) + tuple(widths)), name="lenet_fc")
+    if pooled == "f32":
+        return [replace(s1, name="lenet_conv1"), cast(batch, 14 * 14 * C1), replace(s2, name="lenet_conv2"), cast(batch, flat), fc3]
+    return [replace(s1, name="lenet_conv1", out_dtype=pooled), replace(s2, name="lenet_conv2", out_dtype=pooled), fc3]
 
 
 def conv_nchw(base: Chain) -> Chain:
@@ -329,7 +338,7 @@ def output_shapes(chain: Chain):
     elif chain.reduce == "global_avgpool":
         outs.append(("reduce", "f32", (chain.batch, chain.Cout)))
     elif chain.reduce == "maxpool_2x2":
-        outs.append(("reduce", "f32", (chain.batch, chain.OH // 2, chain.OW // 2, chain.Cout)))
+        outs.append(("reduce", chain.pooled_dtype, (chain.batch, chain.OH // 2, chain.OW // 2, chain.Cout)))
     return outs
 
 

@@ -164,9 +164,12 @@ typedef enum {
     FC_RED_ROW_SUM = 4,         /* out[m] = sum_n v          (elementwise or GEMM producer) */
     FC_RED_ROW_MAX = 5,         /* out[m] = max_n v          (elementwise or GEMM producer) */
     FC_RED_ROW_MEAN = 6,        /* out[m] = (sum_n v) / N    (elementwise or GEMM producer) */
-    FC_RED_MAXPOOL_2X2 = 7      /* out[b][i][j][c] = max of v[b][2i..2i+1][2j..2j+1][c], fp32 [batch][OH/2][OW/2][Cout];
+    FC_RED_MAXPOOL_2X2 = 7      /* out[b][i][j][c] = max of v[b][2i..2i+1][2j..2j+1][c], [batch][OH/2][OW/2][Cout];
                                    CONV producer whose op list ends with RELU (the conv / ReLU / max-pool stage
-                                   of the paper's appendix network); a last odd row or column is dropped       */
+                                   of the paper's appendix network); a last odd row or column is dropped.
+                                   Stored as fp32, or as out_dtype when that is FC_BF16 or FC_F16 (the next
+                                   layer's operand type, the maximum rounded to nearest even): that form needs
+                                   OH even and OW <= 64, else FC_ERR_UNSUPPORTED                              */
 } fc_reduce;
 
 typedef struct {
@@ -181,7 +184,7 @@ typedef struct {
     int32_t producer;       /* fc_producer           */
     int32_t in_dtype;       /* storage of inputs[0] (and inputs[1] for GEMM / CONV) */
     int32_t acc_dtype;      /* FC_F32                */
-    int32_t out_dtype;      /* storage of the main output / softmax probabilities   */
+    int32_t out_dtype;      /* storage of the main output / softmax probabilities / a 2x2 max-pool (16-bit types) */
     int64_t M, N, K;        /* ELEMENTWISE: M rows x N cols; GEMM: M x N x K        */
     int64_t batch, H, W, Cin, Cout, R, S, stride, pad;   /* CONV only              */
     int32_t n_ops;
@@ -327,6 +330,9 @@ int fc_version(void);
 #define FC_TESTING_BOUNDS_TRIP 2   /* debug build only: value 1 shortens the checked extent of the main output by one row */
 #define FC_TESTING_TILE_WIDTH 3    /* value 128, 240 or 256: the column-tile width of every tensor-core GEMM that has a choice
                                       (plain store, row reductions, single-pass softmax, the fp32 form); 0: the launcher's own */
+#define FC_TESTING_POOL_FORM 4     /* value 1, 2 or 3: the form of the 2x2 max-pool behind a convolution (1: every window through
+                                      atomics; 2: windows inside a tile finished on chip; 3: tiles of whole row pairs, where the
+                                      shape allows them, else the launcher's own); 0: the launcher's own */
 void fc_testing_set(int which, int value);
 
 #ifdef __cplusplus

@@ -106,7 +106,7 @@ def fc_last_plan() -> str:
     return lib().fc_last_plan().decode()
 
 
-FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL, FC_TESTING_BOUNDS_TRIP, FC_TESTING_TILE_WIDTH = 0, 1, 2, 3
+FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL, FC_TESTING_BOUNDS_TRIP, FC_TESTING_TILE_WIDTH, FC_TESTING_POOL_FORM = 0, 1, 2, 3, 4
 
 
 def fc_testing_set(which: int, value: int) -> None:
@@ -314,7 +314,8 @@ def output_tensors(chain, device="cuda", pinned=False) -> List[torch.Tensor]:
     elif chain.reduce == "global_avgpool":
         outs.append(torch.empty((chain.batch, chain.Cout), dtype=torch.float32, **kw))
     elif chain.reduce == "maxpool_2x2":
-        outs.append(torch.empty((chain.batch, OH // 2, OW // 2, chain.Cout), dtype=torch.float32, **kw))
+        dt = _TORCH_DT[chain.out_dtype] if chain.out_dtype in ("bf16", "f16") else torch.float32   # (as the library stores it)
+        outs.append(torch.empty((chain.batch, OH // 2, OW // 2, chain.Cout), dtype=dt, **kw))
     return outs
 
 

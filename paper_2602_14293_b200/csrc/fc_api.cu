@@ -16,7 +16,7 @@ __device__ int g_status_word;  // written by kernels when a bounded wait expires
 namespace {
 
 // testing switches (fc_testing_set): read on every call, written by tests only
-std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0}, g_bounds_trip{0}, g_force_tile_width{0};
+std::atomic<int> g_inject_panel_stall{0}, g_inject_split_stall{0}, g_bounds_trip{0}, g_force_tile_width{0}, g_force_pool_form{0};
 
 thread_local int t_device = 0;   // ordinal of the current device, noted by get_device at the top of every entry point
 thread_local char t_err[512] = "";
@@ -136,6 +136,9 @@ fc_status check_tensor(const fc_tensor& t, const char* what, int dtype_or_any, i
     return FC_OK;
 }
 
+// MAXPOOL_2X2 stores its output as the spec's out_dtype when that is a 16-bit type (the next layer's operand type), else as fp32
+bool pooled_16bit(const fc_chain_spec* s) { return s->reduce == FC_RED_MAXPOOL_2X2 && (s->out_dtype == FC_BF16 || s->out_dtype == FC_F16); }
+
 bool is_conv(const fc_chain_spec* s) { return s->producer == FC_PROD_CONV2D_NHWC || s->producer == FC_PROD_CONV2D_NCHW; }
 
 // CONV2D_NCHW: channels-last copies of the image and of the weights at the head of the workspace
@@ -228,6 +231,9 @@ fc_status validate_spec(const fc_chain_spec* s, Plan* plan) {
                     return fail(FC_ERR_UNSUPPORTED, "MAXPOOL_2X2 needs an op list that ends with RELU");
                 const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
                 if (OH < 2 || OW < 2) return fail(FC_ERR_SHAPE, "MAXPOOL_2X2 needs a conv output of at least 2 x 2 (is %lld x %lld)", OH, OW);
+                // a 16-bit pooled output is stored, not reached through atomics: every window must lie inside one tile
+                if (pooled_16bit(s) && !(OH % 2 == 0 && 2 * OW <= 128))
+                    return fail(FC_ERR_UNSUPPORTED, "MAXPOOL_2X2 with a 16-bit out_dtype needs an even number of conv output rows and at most 64 columns (is %lld x %lld); use FC_F32", OH, OW);
             }
             if (s->stride > 8) return fail(FC_ERR_UNSUPPORTED, "conv supports stride <= 8");
             if (s->pad >= s->R || s->pad >= s->S || s->R > 16 || s->S > 16) return fail(FC_ERR_UNSUPPORTED, "conv supports pad < R,S <= 16");
@@ -366,7 +372,7 @@ fc_status validate_tensors(const fc_chain_spec* s, const Plan& plan, const fc_te
         if (s->reduce == FC_RED_MAXPOOL_2X2) {
             const long long OH = (s->H + 2 * s->pad - s->R) / s->stride + 1, OW = (s->W + 2 * s->pad - s->S) / s->stride + 1;
             const long long sh[4] = {s->batch, OH / 2, OW / 2, s->Cout};
-            if ((st = check_tensor(out[plan.red_index], "pooled output", FC_F32, 4, sh))) return st;
+            if ((st = check_tensor(out[plan.red_index], "pooled output", pooled_16bit(s) ? s->out_dtype : FC_F32, 4, sh))) return st;
         } else if (s->reduce != FC_RED_GLOBAL_AVGPOOL) {
             const long long sh[1] = {s->M};
             if ((st = check_tensor(out[plan.red_index], "row reduction output", FC_F32, 1, sh))) return st;
@@ -654,6 +660,26 @@ int conv_params(const fc_chain_spec* spec, long long out_rows, TcParams* p) {
     // positions finished on chip and stored (78 % of them at OW = 28, 92 % at 10), the others through atomics.  The
     // second form costs two 128-thread barriers per channel chunk: from OW = 56 on it measured slower (105 -> 110 us).
     p->pool = spec->reduce == FC_RED_MAXPOOL_2X2 ? (p->OW <= 32 ? 2 : 1) : 0;
+    // Tiles of whole row pairs: with an even number of output rows per image every image is a whole number of row pairs
+    // (2 * OW consecutive positions), and a CTA whose tile stands for the largest number of whole pairs that fits its
+    // 128 positions (112 of them at OW = 28 or 56, 120 at OW = 10) holds all four positions of every window it
+    // touches: the second form then finishes every window on chip, no atomics are left, and the output needs no zeros
+    // in front.  The price is the positions that a tile loads and multiplies but leaves to the next one (up to 12.5 %).
+    p->m_rows = 128;
+    p->pool_whole = 0;
+    const int forced = g_force_pool_form.load(std::memory_order_relaxed);
+    const bool whole_ok = p->pool && p->OH % 2 == 0 && 2 * p->OW <= 128;
+    const bool must = pooled_16bit(spec);     // (validated: whole_ok holds)
+    if (p->pool && forced >= 1 && forced <= 2 && !must) p->pool = forced;
+    // (fp32 outputs: only where no position of a tile is wasted, i.e. 2 * OW divides 128: 5 % faster on 64 images of
+    // 32 x 32 x 64 -> 128; with 112 or 120 of 128 positions the extra tiles cost what the atomics did.  16-bit outputs
+    // always: they cannot be reached through atomics.)
+    const bool pays = 128 % (2 * p->OW) == 0;
+    if (whole_ok && (forced == 3 || (forced == 0 && pays) || must)) {
+        p->pool = 2;
+        p->pool_whole = 1;
+        p->m_rows = 128 / (2 * p->OW) * (2 * p->OW);
+    }
     p->a_packed = packed_taps(spec);
     p->a_rowtaps = row_taps(spec);
     // (up to 64 output channels: 64-column tiles, so that both column halves of the epilogue warps have work: with
@@ -883,7 +909,7 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             TcParams p;
             memset(&p, 0, sizeof(p));
             const int bn = conv_params(spec, plan.out_rows, &p);
-            p.out = outputs[plan.red_index].ptr; p.out_dt = FC_F32;
+            p.out = outputs[plan.red_index].ptr; p.out_dt = pooled_16bit(spec) ? spec->out_dtype : FC_F32;
             p.status = dev->status;
             build_ops(spec, inputs, &p.ops);
             const size_t out_elems = p.pool ? (size_t) spec->batch * (p.OH / 2) * (p.OW / 2) * spec->Cout : (size_t) spec->batch * spec->Cout;
@@ -914,8 +940,11 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             if ((st = encode_2d(&tmB, weights, spec->Cout, p.K, bn / 2, spec->in_dtype))) return st;
             // The pooled output is cleared by a kernel directly in front of the convolution, which is launched
             // programmatically behind it: its loads and MMAs start at once, only its epilogue warps wait for the zeros.
-            if ((e = launch_zero_fill(p.out, out_elems * 4, dev->num_sms, stream, &launches)) != cudaSuccess) return cuda_fail(e, "zero-fill launch");
-            p.after_zero_fill = 1;
+            // (not for a max-pool over tiles of whole row pairs: every window is stored once, by the tile that holds it)
+            if (!p.pool_whole) {
+                if ((e = launch_zero_fill(p.out, out_elems * 4, dev->num_sms, stream, &launches)) != cudaSuccess) return cuda_fail(e, "zero-fill launch");
+                p.after_zero_fill = 1;
+            }
             e = launch_gemm_tc(p, tmA, tmB, bn, dev->num_sms, stream, &launches);
             break;
         }
@@ -1199,6 +1228,7 @@ void fc_testing_set(int which, int value) {
     else if (which == FC_TESTING_SPLIT_STALL) g_inject_split_stall.store(value);
     else if (which == FC_TESTING_BOUNDS_TRIP) g_bounds_trip.store(value);
     else if (which == FC_TESTING_TILE_WIDTH) g_force_tile_width.store(value);
+    else if (which == FC_TESTING_POOL_FORM) g_force_pool_form.store(value);
 }
 
 }  // extern "C"

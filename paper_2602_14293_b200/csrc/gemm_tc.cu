@@ -237,13 +237,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t cta_rank = ptx::cluster_ctarank();
     const bool leader = cta_rank == 0;
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
-    const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM);   // pair-panels of 256 rows
-    const int tiles_n = (p.N + BN - 1) / BN;
-    const int total_tiles = tiles_m * tiles_n;
     // 4: the convolution with eight filter taps per k-block (TcParams::a_packed); 5: with a filter row per k-block
     // (TcParams::a_rowtaps).  Instantiations of their own: as run-time branches of mode 2's producer either of them
     // cost the ordinary convolution 2 - 10 %.
     constexpr bool kConv = MODE == 2 || MODE == 4 || MODE == 5;
+    // rows of the output that a CTA's tile stands for: all 128, or (convolution + max-pool in whole row pairs,
+    // TcParams::m_rows) the first m_rows of them: the tile still loads and multiplies 128 positions, the last ones
+    // belong to the next tile and are dropped here
+    const int m_rows = kConv ? p.m_rows : BM;
+    const int tiles_m = (p.M + 2 * m_rows - 1) / (2 * m_rows);   // pair-panels of 2 * m_rows rows
+    const int tiles_n = (p.N + BN - 1) / BN;
+    const int total_tiles = tiles_m * tiles_n;
     const int kb_per_tap = kConv ? (p.Cin + BK - 1) / BK : 1;
     const bool f8 = !kConv && (kMx || p.in_dt == FC_F8E4M3);
     const int bk = MODE == 7 ? BK / 2 : (f8 ? 2 * BK : BK);   // K elements per k-block: 128 bytes of a row
@@ -296,7 +300,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
                 int mb2, nb;
                 tile_coords((MODE == 0 || MODE == 6 || MODE == 7 || MODE == 3 || (MODE == 1 && p.two_pass)) ? 0 : 1, p.group_m, w.tile, tiles_m, tiles_n, mb2, nb);   // (the two-pass softmax waits for nobody: free to use the L2-friendly order)
-                const int row0 = (mb2 * 2 + (int) cta_rank) * BM;          // this CTA's rows of A
+                const int row0 = (mb2 * 2 + (int) cta_rank) * m_rows;      // this CTA's rows of A
                 const int bcol0 = nb * BN + (int) cta_rank * (BN / 2);     // this CTA's half of the B tile
                 int img = 0, oh = 0, ow = 0;
                 if constexpr (kConv) {
@@ -545,7 +549,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int col_half = half * C::kColHalf;
             const int n_lim = min(p.N, n_tile + BN);   // first column that is not this tile's
             const uint32_t tacc = tmem_base + buf * BN + col_half + lane_addr;
-            const long long m = (long long) mb * BM + row;
+            // (rows of the tile behind m_rows: no row of the output, which `m >= M` says everywhere below)
+            const long long m = row < m_rows ? (long long) mb * m_rows + row : (long long) p.M;
             const int n_half = n_tile + col_half;
             // hands the accumulator buffer back to the leader's MMA thread
             auto release_buf = [&]() {
@@ -562,8 +567,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 constexpr size_t kSliceF4 = (size_t) BM * 2 * C::kColHalf / 4;
                 const int ws = warp - 2;
                 unsigned int* cnt = &p.split_counters[(w.v0 / w.nsl) * 2 + (int) cta_rank];
-                // a warp none of whose 32 rows exists (a short last panel: 16 rows of 256) parks and merges nothing
-                const bool live = m - lane < p.M;
+                // a warp none of whose 32 rows exists (a short last panel: 16 rows of 256; rows behind m_rows) parks and merges nothing
+                // (warp-uniform: the loops below issue warp-wide accumulator loads)
+                const bool live = lane_grp * 32 < m_rows && (long long) mb * m_rows + lane_grp * 32 < p.M;
                 if (w.slice != w.nsl - 1) {
                     float4* mine = p.split_ws + ((size_t) (w.v0 + w.slice) * 2 + cta_rank) * kSliceF4 + (size_t) ws * kChunks * 128 + lane;
 #pragma unroll 1
@@ -1068,6 +1074,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 unsigned int* out_u = (unsigned int*) p.out;
                 const int ch = lane & 15, hwid = q >> 4;           // channel of the chunk, half-warp 0..7 of the column half
                 const int below = p.OW * 17;
+                const bool out16 = p.out_dt != FC_F32;
+                // (two 16-bit channels as one word: rows of an even number of channels, the output on a 4-byte boundary)
+                const bool pair16 = (p.N & 1) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 3) == 0;
                 tmem_sweep16<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
                     if (n0 >= p.N) return;
@@ -1079,7 +1088,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int j = 0; j < 16; ++j)
                         if (FC_DBG_IN(&stage[q * 17 + j], 4, pool_stage, (long long) C::kPoolBytes, p.status, kSitePoolStage)) stage[q * 17 + j] = v[j];
                     ptx::bar_sync(3 + half, 128);
-                    if (n0 + ch < p.N) {
+                    if (out16) {
+                        // 16-bit output (tiles of whole row pairs only: every entry is a complete window): a quarter
+                        // warp per entry, two channels per lane, stored as one 32-bit word where the rows allow it.
+                        // (The same loop for fp32 outputs, two words per store, gained them 1 - 3 % and cost this form as
+                        // much, as a branch in this loop or as a second copy of it: the fp32 form keeps the loop below.)
+                        const int c2 = (lane & 7) * 2, qwid = q >> 3;
+                        if (n0 + c2 < p.N) {
+                            const bool both = pair16 || n0 + c2 + 1 < p.N;
+                            for (int e = qwid; e < n_emit; e += 16) {
+                                const int2 ent = pool_tab[e];
+                                if (!(ent.x & 256)) continue;
+                                const float* sp = stage + (ent.x & 127) * 17 + c2;
+                                const float x0 = fabsf(fmaxf(fmaxf(sp[0], sp[17]), fmaxf(sp[below], sp[below + 17])));
+                                const float x1 = fabsf(fmaxf(fmaxf(sp[1], sp[18]), fmaxf(sp[below + 1], sp[below + 18])));
+                                unsigned short* dst = (unsigned short*) p.out + (long long) ent.y * p.N + n0 + c2;
+                                if (!FC_DBG_IN(dst, both ? 4 : 2, p.out, (long long) p.batch * PH * PW * p.N * 2, p.status, kSitePoolMax)) continue;
+                                const unsigned short h0 = p.out_dt == FC_BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(x0)) : __half_as_ushort(__float2half_rn(x0));
+                                const unsigned short h1 = p.out_dt == FC_BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(x1)) : __half_as_ushort(__float2half_rn(x1));
+                                if (pair16) {
+                                    *reinterpret_cast<unsigned int*>(dst) = (unsigned int) h0 | ((unsigned int) h1 << 16);
+                                } else {
+                                    dst[0] = h0;
+                                    if (both) dst[1] = h1;
+                                }
+                            }
+                        }
+                    } else if (n0 + ch < p.N) {
                         for (int e = hwid; e < n_emit; e += 8) {
                             const int2 ent = pool_tab[e];
                             const float* sp = stage + (ent.x & 127) * 17 + ch;
@@ -1196,7 +1231,8 @@ cudaError_t launch_one(const TcParams& p, const CUtensorMap* tmA, const CUtensor
         if (known) state.max_clusters[dev].store(resident, std::memory_order_release);
     }
     const int tiles_n = (p.N + BN - 1) / BN;
-    const int tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * tiles_n;
+    const int m_rows = (MODE == 2 || MODE == 4 || MODE == 5) ? p.m_rows : BM;
+    const int tiles = ((p.M + 2 * m_rows - 1) / (2 * m_rows)) * tiles_n;
     int max_pairs = resident;
     if (max_pairs > num_sms / 2) max_pairs = num_sms / 2;
     int clusters = max_pairs < tiles ? max_pairs : tiles;

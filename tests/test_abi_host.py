@@ -179,18 +179,27 @@ def test_network_stages_fit_together_and_validate(fc):
     """The LeNet-shaped sequence: every stage's first input has exactly the bytes of the previous stage's
     output, and every stage's spec passes the library's validation (fc_workspace_size validates without a GPU)."""
     import numpy as np
-    stages = wl.lenet_shaped(batch=12)
     size = {"f32": 4, "bf16": 2, "f16": 2}
-    prev_bytes = None
-    for ch in stages:
-        spec = fc.make_spec(ch)
-        assert fc.binding.fc_workspace_size(spec) == 0
-        _, in_dt, in_shape, *_ = ch.input_recipe[0]
-        if prev_bytes is not None:
-            assert int(np.prod(in_shape)) * size[in_dt] == prev_bytes, ch.name
-        _, out_dt, out_shape = wl.output_shapes(ch)[0]
-        prev_bytes = int(np.prod(out_shape)) * size[out_dt]
-    assert wl.output_shapes(stages[-1])[0][2] == (12, 10)
+    for pooled, n_stages in (("bf16", 3), ("f32", 5)):
+        stages = wl.lenet_shaped(batch=12, pooled=pooled)
+        assert len(stages) == n_stages
+        prev_bytes = None
+        for ch in stages:
+            spec = fc.make_spec(ch)
+            assert fc.binding.fc_workspace_size(spec) == 0
+            _, in_dt, in_shape, *_ = ch.input_recipe[0]
+            if prev_bytes is not None:
+                assert int(np.prod(in_shape)) * size[in_dt] == prev_bytes, ch.name
+            _, out_dt, out_shape = wl.output_shapes(ch)[0]
+            prev_bytes = int(np.prod(out_shape)) * size[out_dt]
+        assert wl.output_shapes(stages[-1])[0][2] == (12, 10)
+    # a 16-bit pooled output is stored by the tile that holds the whole window: odd row counts and outputs wider
+    # than 64 columns are turned away with a message that names the way out
+    from dataclasses import replace
+    for H, W in ((9, 8), (8, 130)):
+        odd = replace(wl.conv_bias_relu_maxpool(batch=1, H=H, W=W, Cin=8, Cout=8, R=3, S=3, pad=1), out_dtype="bf16")
+        with pytest.raises(fc.FcError, match="16-bit out_dtype"):
+            fc.binding.fc_workspace_size(fc.make_spec(odd))
     assert fc.binding.fc_describe_plan is not None
     # an 8-channel first layer is legal; 4 channels are not (rows of the image must be multiples of 16 bytes)
     bad = wl.conv_bias_relu_maxpool(batch=1, H=8, W=8, Cin=4, Cout=8, R=3, S=3, pad=1)

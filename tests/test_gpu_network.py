@@ -36,9 +36,11 @@ def _out_name(ch):
     return wl.output_shapes(ch)[0][0]
 
 
+@pytest.mark.parametrize("pooled", ["bf16", "f32"])
 @pytest.mark.parametrize("batch", [64, 37])
-def test_lenet_shaped_network_stage_by_stage(fc, orc, batch):
-    stages = wl.lenet_shaped(batch)
+def test_lenet_shaped_network_stage_by_stage(fc, orc, batch, pooled):
+    stages = wl.lenet_shaped(batch, pooled=pooled)
+    assert len(stages) == (3 if pooled == "bf16" else 5)
     prev_gpu = None          # GPU output of the previous stage
     prev_ref = None          # oracle-only pass: stored form of the previous stage's oracle output
     launches = fc.fc_launch_count()
@@ -67,7 +69,7 @@ def test_lenet_shaped_network_stage_by_stage(fc, orc, batch):
             assert np.array_equal(_to_numpy(outs[0]), rng.f32_to_bf16_bits(ins_seen[0]))
         # oracle-only pass through the network, stored in each stage's output type
         full = orc.run_chain(ch, ins_ref)[name]
-        out_dt = "f32" if ch.reduce != "none" else ch.out_dtype
+        out_dt = wl.output_shapes(ch)[0][1]
         prev_ref = rng.store(full.astype(np.float32), out_dt)
         prev_gpu = outs[0]
     assert fc.fc_launch_count() - launches >= len(stages)

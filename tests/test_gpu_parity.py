@@ -971,6 +971,59 @@ def test_conv_relu_maxpool(fc, orc, batch, H, W, Cin, Cout, R, S, pad, stride):
         run_and_check(fc, orc, ch, seed)
 
 
+# (batch, H, W, Cin, Cout, R, S, pad): OH even and OW <= 64, so that tiles of whole row pairs exist; row pairs of 16, 20,
+# 48, 56, 112 and 128 positions (128, 120, 96, 112, 112 and 128 positions per CTA), tiles across images, a last tile
+# that ends inside its 128 positions, split last rounds (50 and 18 k-blocks), 64-, 128- and 256-column tiles
+_WHOLE_PAIRS = [(5, 8, 8, 64, 64, 3, 3, 1), (7, 12, 10, 64, 128, 3, 3, 1), (2, 28, 28, 128, 64, 5, 5, 0), (3, 30, 30, 64, 136, 3, 3, 0),
+                (2, 56, 56, 64, 256, 3, 3, 1), (3, 6, 64, 64, 72, 3, 3, 1), (9, 14, 14, 64, 128, 5, 5, 0), (4, 32, 32, 8, 64, 5, 5, 0),
+                (3, 10, 9, 64, 48, 3, 3, 1)]
+
+
+@pytest.mark.parametrize("shape", _WHOLE_PAIRS)
+def test_conv_relu_maxpool_three_forms_agree(fc, orc, shape):
+    """The 2 x 2 max-pool behind a convolution has three forms (every window through atomics; windows inside a tile
+    finished on chip; tiles of whole row pairs, no atomics and no zeros in front).  A maximum is exact: all three
+    give the same bits, and the oracle's values within the usual tolerance."""
+    batch, H, W, Cin, Cout, R, S, pad = shape
+    ch = wl.conv_bias_relu_maxpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, pad=pad)
+    got = []
+    try:
+        for form in (1, 2, 3):
+            fc.binding.fc_testing_set(fc.binding.FC_TESTING_POOL_FORM, form)
+            outs, _, _ = run_and_check(fc, orc, ch, 21)
+            assert ("zero_fill" in fc.fc_last_plan()) == (form != 3)
+            got.append(outs[0].clone())
+    finally:
+        fc.binding.fc_testing_set(fc.binding.FC_TESTING_POOL_FORM, 0)
+    assert torch.equal(got[0], got[1]) and torch.equal(got[0], got[2])
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+@pytest.mark.parametrize("shape", _WHOLE_PAIRS)
+def test_conv_relu_maxpool_stored_in_16_bits(fc, orc, shape, dt):
+    """out_dtype = bf16 / f16: the pooled output is stored in the next layer's operand type by the tile that holds the
+    whole window.  Rounding is monotonic, so the result is the fp32 form's, rounded to nearest even, bit for bit."""
+    batch, H, W, Cin, Cout, R, S, pad = shape
+    base = wl.conv_bias_relu_maxpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, pad=pad)
+    if dt == "f16":
+        base = replace(base, in_dtype="f16", input_recipe=tuple((t, "f16", sh, d, a, b) for t, _, sh, d, a, b in base.input_recipe))
+    ins = wl.make_inputs(base, 22)
+    wide, _, _ = run_and_check(fc, orc, base, ins=ins)
+    ch = replace(base, out_dtype=dt)
+    outs, _, _ = run_and_check(fc, orc, ch, ins=ins)
+    assert outs[0].dtype == (torch.bfloat16 if dt == "bf16" else torch.float16)
+    assert "zero_fill" not in fc.fc_last_plan()
+    assert torch.equal(outs[0], wide[0].to(outs[0].dtype))
+
+
+def test_conv_relu_maxpool_16_bit_output_needs_whole_row_pairs(fc):
+    for H, W in ((9, 8), (8, 130)):
+        ch = replace(wl.conv_bias_relu_maxpool(batch=1, H=H, W=W, Cin=64, Cout=64, R=3, S=3, pad=1), out_dtype="bf16")
+        ins = [fc.to_device(a) for a in wl.make_inputs(ch, 0)]
+        with pytest.raises(fc.FcError, match="16-bit out_dtype"):
+            fc.run_chain(ch, ins, fc.binding.output_tensors(ch, "cuda"))
+
+
 def test_conv_relu_maxpool_delta_kernel_is_pooled_relu_of_image(fc, orc):
     """Centre-delta weights copy the image, so the output is the 2x2 max-pool of ReLU(image): compared
     with numpy on the stored bf16 values, exactly."""
