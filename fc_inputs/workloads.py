@@ -278,6 +278,8 @@ EXTRA = {
     "F8": lambda **kw: gemm_softmax(**{"M": 2048, "N": 50264, "K": 4096, **kw}),   # a vocabulary-wide softmax: two kernels
     "F9": lambda **kw: gemm_bias_relu_f32(**{"M": 2048, "N": 2048, "K": 2048, **kw}),   # C1's chain at a size where fp32 operands go to the tensor cores (three tf32 products per product)
     "F10": lambda **kw: gemm_mxf8_bias_gelu_scale_clamp(**kw),   # C3's chain on block-scaled 8-bit operands
+    # an image layer (the network N1's first): 5 x 5 on 8 channels -> 64, ReLU, 2x2 max-pool stored in bf16 for the next layer
+    "F11": lambda **kw: replace(conv_bias_relu_maxpool(**{"batch": 4096, "H": 32, "W": 32, "Cin": 8, "Cout": 64, "R": 5, "S": 5, "pad": 0, **kw}), out_dtype="bf16"),
 }
 ALL = {**CONFIGS, **EXTRA}
 

@@ -671,10 +671,13 @@ int conv_params(const fc_chain_spec* spec, long long out_rows, TcParams* p) {
     const bool whole_ok = p->pool && p->OH % 2 == 0 && 2 * p->OW <= 128;
     const bool must = pooled_16bit(spec);     // (validated: whole_ok holds)
     if (p->pool && forced >= 1 && forced <= 2 && !must) p->pool = forced;
-    // (fp32 outputs: only where no position of a tile is wasted, i.e. 2 * OW divides 128: 5 % faster on 64 images of
-    // 32 x 32 x 64 -> 128; with 112 or 120 of 128 positions the extra tiles cost what the atomics did.  16-bit outputs
-    // always: they cannot be reached through atomics.)
-    const bool pays = 128 % (2 * p->OW) == 0;
+    // fp32 outputs: where no position of a tile is wasted (2 * OW divides 128: 33.8 against 35.9 us on 64 images of
+    // 32 x 32 x 64 -> 128), where the other choice is atomics for every window (OW > 32: F3 103.5 against 105.4 us), and
+    // where a tile's few k-blocks leave the epilogue in the open (a 5 x 5 x 8 -> 64 image layer 640 against 664 us).
+    // Elsewhere the up to 14 % more tiles cost more than the few atomics left (5 x 5 x 64 -> 128 at OW = 10: 208.9
+    // against 203.6 us).  16-bit outputs always: they cannot be reached through atomics.
+    const int kbs = row_taps(spec) ? (int) spec->R : (packed_taps(spec) ? (int) ((spec->R * spec->S * spec->Cin + 63) / 64) : (int) (spec->R * spec->S * ((spec->Cin + 63) / 64)));
+    const bool pays = 128 % (2 * p->OW) == 0 || p->OW > 32 || kbs <= 8;
     if (whole_ok && (forced == 3 || (forced == 0 && pays) || must)) {
         p->pool = 2;
         p->pool_whole = 1;

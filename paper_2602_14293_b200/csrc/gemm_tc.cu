@@ -517,6 +517,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (p.after_zero_fill) asm volatile("griddepcontrol.wait;" ::: "memory");
         }
         uint32_t tile_iter = 0;
+        int staged_nb0 = -1, staged_nb1 = -1;   // column tile whose vectors each staging buffer holds
         for (int u = cluster_id; u < total_units; u += num_clusters, ++tile_iter) {
             const Unit w = unit_decode(u, p.split_from, p.split, p.split_kb, num_kb);
             int mb2, nb;
@@ -526,8 +527,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int n_tile = nb * BN;
             float* svec = svec_all + buf * (kMaxVecSlots * BN);
             EPI_MARK(0);
-            // stage this tile's slices of the per-column vectors (fp32) before the accumulator wait
-            {
+            // stage this tile's slices of the per-column vectors (fp32) before the accumulator wait (not again when the
+            // buffer holds this column tile's already: every tile of a convolution narrower than a tile, 700 cycles of
+            // global-load latency per tile that an epilogue-bound layer cannot hide)
+            if ((buf ? staged_nb1 : staged_nb0) != nb) {
+                if (buf) staged_nb1 = nb;
+                else staged_nb0 = nb;
                 int slot = 0;
                 for (int i = 0; i < p.ops.n && slot < kMaxVecSlots; ++i) {
                     const DevOp& op = p.ops.op[i];
@@ -1036,40 +1041,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // entry with one channel per lane (16 consecutive channels per store or atomic).
                 const int hw = p.OH * p.OW, PH = p.OH >> 1, PW = p.OW >> 1;
                 const int q = lane_grp * 32 + lane;        // this thread's position in the tile
-                int win = 0;
-                bool emit = false, right = false, vert = false;
-                if (m < p.M) {
-                    const int img = (int) (m / hw);
-                    const int rem = (int) (m - (long long) img * hw);
-                    const int oh = rem / p.OW, ow = rem - oh * p.OW;
-                    if ((oh >> 1) < PH && (ow >> 1) < PW) {
-                        win = (img * PH + (oh >> 1)) * PW + (ow >> 1);      // window index, below 2^31 like the position index
-                        if ((ow & 1) == 0) {
-                            right = q < BM - 1;                             // the right neighbour (same row) is in this tile
-                            const bool top = (oh & 1) == 0;
-                            vert = top && right && q + p.OW + 1 <= BM - 1;  // and so is the row below
-                            // a lower-left position whose window the upper-left one finishes (that one is OW in front)
-                            const bool covered = !top && q >= p.OW && q <= BM - 2;
-                            emit = !covered;
-                        } else {
-                            emit = q == 0;                                  // its left neighbour sits in the tile in front
-                        }
-                    }
-                }
                 int* pool_cnt = reinterpret_cast<int*>(xchg) + half * 256;           // [4] emitters per warp, then the entries
                 int2* pool_tab = reinterpret_cast<int2*>(pool_cnt + 4);             // up to 65: (position | flags, window)
-                const unsigned emask = __ballot_sync(0xffffffffu, emit);
-                if (lane == 0) pool_cnt[lane_grp] = __popc(emask);
-                ptx::bar_sync(3 + half, 128);
-                int before = 0, n_emit = 0;
+                int n_emit = 0;
+                if (p.pool_whole) {
+                    // Tiles of whole row pairs: the tile starts on a row pair and images are whole numbers of pairs, so
+                    // the windows are the first PW column pairs of every pair of rows, numbered like the row pairs:
+                    // entry e = (pair, column pair) is written down directly, all complete (no search, no divisions
+                    // by the image size; keeping the three small quotients in registers across tiles measured slower).
+                    const int pair_len = 2 * p.OW, ppt = m_rows / pair_len;
+                    const long long pair0 = (long long) mb * ppt;
+                    const long long pairs_left = (long long) (p.M / pair_len) - pair0;
+                    n_emit = (int) (pairs_left < ppt ? (pairs_left > 0 ? pairs_left : 0) : ppt) * PW;   // at most 32
+                    if (q < n_emit) {
+                        const int pi = q / PW, j = q - pi * PW;
+                        pool_tab[q] = make_int2((pi * pair_len + 2 * j) | 128 | 256, (int) ((pair0 + pi) * PW + j));
+                    }
+                    ptx::bar_sync(3 + half, 128);
+                } else {
+                    int win = 0;
+                    bool emit = false, right = false, vert = false;
+                    if (m < p.M) {
+                        const int img = (int) (m / hw);
+                        const int rem = (int) (m - (long long) img * hw);
+                        const int oh = rem / p.OW, ow = rem - oh * p.OW;
+                        if ((oh >> 1) < PH && (ow >> 1) < PW) {
+                            win = (img * PH + (oh >> 1)) * PW + (ow >> 1);      // window index, below 2^31 like the position index
+                            if ((ow & 1) == 0) {
+                                right = q < BM - 1;                             // the right neighbour (same row) is in this tile
+                                const bool top = (oh & 1) == 0;
+                                vert = top && right && q + p.OW + 1 <= BM - 1;  // and so is the row below
+                                // a lower-left position whose window the upper-left one finishes (that one is OW in front)
+                                const bool covered = !top && q >= p.OW && q <= BM - 2;
+                                emit = !covered;
+                            } else {
+                                emit = q == 0;                                  // its left neighbour sits in the tile in front
+                            }
+                        }
+                    }
+                    const unsigned emask = __ballot_sync(0xffffffffu, emit);
+                    if (lane == 0) pool_cnt[lane_grp] = __popc(emask);
+                    ptx::bar_sync(3 + half, 128);
+                    int before = 0;
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int cg = pool_cnt[g];
-                    before += g < lane_grp ? cg : 0;
-                    n_emit += cg;
+                    for (int g = 0; g < 4; ++g) {
+                        const int cg = pool_cnt[g];
+                        before += g < lane_grp ? cg : 0;
+                        n_emit += cg;
+                    }
+                    if (emit) pool_tab[before + __popc(emask & ((1u << lane) - 1u))] = make_int2(q | (right ? 128 : 0) | (vert ? 256 : 0), win);
+                    ptx::bar_sync(3 + half, 128);
                 }
-                if (emit) pool_tab[before + __popc(emask & ((1u << lane) - 1u))] = make_int2(q | (right ? 128 : 0) | (vert ? 256 : 0), win);
-                ptx::bar_sync(3 + half, 128);
+                EPI_MARK(2);
                 float* stage = pool_stage + half * (BM * 17);     // [position][16 channels + 1]
                 unsigned int* out_u = (unsigned int*) p.out;
                 const int ch = lane & 15, hwid = q >> 4;           // channel of the chunk, half-warp 0..7 of the column half
@@ -1077,7 +1100,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const bool out16 = p.out_dt != FC_F32;
                 // (two 16-bit channels as one word: rows of an even number of channels, the output on a 4-byte boundary)
                 const bool pair16 = (p.N & 1) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 3) == 0;
-                tmem_sweep16<kChunks>(tacc, [&](int c, uint32_t (&r)[16]) {
+                auto chunk = [&](int c, uint32_t (&r)[16]) {
                     const int n0 = n_half + c * 16;
                     if (n0 >= p.N) return;
                     float v[16];
@@ -1131,7 +1154,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                     ptx::bar_sync(3 + half, 128);
-                });
+                };
+                // Two chunks per thread (64-column tiles): both loads at once and a copy of the body for each, 634 against
+                // 664 us on 4096 images of 32 x 32 x 8 -> 64.  More chunks: one copy of the body, run again and again
+                // (F3 104.4 -> 101.4 us, 64 images of 32 x 32 x 64 -> 128 36.7 -> 33.8).
+                if constexpr (kChunks <= 2) tmem_sweep16<kChunks>(tacc, chunk);
+                else tmem_sweep<kChunks>(tacc, kChunks, chunk);
             } else {
                 // conv + global average pool: channel sums over this warp's 32 pixels
                 const int hw = p.OH * p.OW;

@@ -1108,7 +1108,7 @@ def test_conv_relu_maxpool_fp16(fc, orc):
 
 
 # ------------------------------------------------------------------ the further measured workloads at full size
-@pytest.mark.parametrize("key", ["F1", "F2", "F3", "F4", "F5", "F6", "F7", "F8", "F9"])
+@pytest.mark.parametrize("key", ["F1", "F2", "F3", "F4", "F5", "F6", "F7", "F8", "F9", "F11"])
 def test_further_workloads_full_size_sampled(fc, orc, key):
     """Each workload the benchmark times beyond the five configurations, at its full size and in the launch
     configuration the benchmark uses; rows (images) are independent problems, so the oracle recomputes a sample

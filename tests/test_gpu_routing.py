@@ -73,6 +73,12 @@ def test_contraction_routing(fc):
     assert _plan(fc, wl.mlp(300, (64, 64, 32))) == "mlp_tc"
     conv = wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128)
     assert _plan(fc, conv) == "zero_fill gemm_tc_mode2_bn128"
-    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=2)) == "zero_fill gemm_tc_mode4_bn256"
-    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=0)) == "zero_fill gemm_tc_mode2_bn256_rowtaps"
+    # max-pool: tiles of whole row pairs (no zeros in front) where they pay or where the output is 16 bits wide
+    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=2)) == "gemm_tc_mode4_bn256"
+    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=0)) == "gemm_tc_mode2_bn256_rowtaps"
+    deep = wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=64, Cout=128, R=5, S=5, pad=0)          # 25 k-blocks, row pairs of 20
+    assert _plan(fc, deep) == "zero_fill gemm_tc_mode2_bn128"
+    assert _plan(fc, replace(deep, out_dtype="bf16")) == "gemm_tc_mode2_bn128"
+    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=15, W=14, Cin=8, Cout=64, R=5, S=5, pad=0)) == "zero_fill gemm_tc_mode2_bn64_rowtaps"   # 11 rows
+    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=16, W=16, Cin=64, Cout=128, R=3, S=3, pad=1)) == "gemm_tc_mode2_bn128"   # row pairs of 32
     assert _plan(fc, wl.conv_nchw(conv)) == "cfirst_to_clast cfirst_to_clast zero_fill gemm_tc_mode2_bn128"
