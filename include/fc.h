@@ -25,7 +25,8 @@
  * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
  * allocates device memory and never synchronises; it enqueues at most two memsets and one to four
  * kernels on the given stream and returns (two kernels: a convolution behind the kernel that zeroes
- * its pooled output, or a wide GEMM + ROW_SOFTMAX as the GEMM kernel and a rescaling pass; three: the
+ * its pooled output -- not launched for a 2x2 max-pool over tiles of whole row pairs, which stores every
+ * window once --, or a wide GEMM + ROW_SOFTMAX as the GEMM kernel and a rescaling pass; three: the
  * collapsed linear layer; four: CONV2D_NCHW with its two layout kernels).  Inputs are read-only;
  * outputs are fully overwritten.
  *

@@ -123,7 +123,7 @@ struct TcParams {
     int m_rows;                 // mode 2: output positions that a CTA's tile stands for: 128, or with pool_whole the largest
                                 // multiple of 2 * OW below (the tile still loads and multiplies 128 positions)
     int pool_whole;             // mode 2, pool == 2: tiles of whole row pairs (OH even): every window lies inside one tile, `out`
-                                // needs no zeros and sees no atomics
+                                // needs no zeros, sees no atomics and may be a 16-bit tensor (out_dt)
     int two_pass;               // mode 1: rows wider than the tiles the SM pairs can hold at once: no waiting across tiles; every
                                 // tile stores its exponentials against its own maximum and leaves (max, sum) in `stats`,
                                 // launch_softmax_rescale finishes the rows
