@@ -494,8 +494,9 @@ __global__ void __launch_bounds__(kThreads, SOFTMAX ? 2 : 4) ew_rows_kernel(cons
         const uint4* rr = RES ? p.res + row * chunks : nullptr;
         uint4* yr = STORE ? p.y + row * chunks : nullptr;
         float run_m = -CUDART_INF_F, run_s = 0.0f;   // log2 domain: sum of 2^(y*log2e - run_m)
-        // (softmax at 4096 columns runs one CTA per SM, its rows waiting in shared memory; twice the loads in flight
-        // per lane there gained 6 % and lost 7 % at 1024 columns: left alone)
+        // (softmax at 4096 columns, its rows waiting in shared memory: twice the loads in flight per lane gained 6 % while
+        // the kernel ran one CTA per SM and lost 7 % at 1024 columns.  With two CTAs per SM, 128 registers per thread at
+        // most, the eight chunks spill: 80 -> 121 us, as a second loop for long rows only too.  Left alone.)
         constexpr int kInFlight = kGroup;
         for (int c0 = lane; c0 < chunks; c0 += 32 * kInFlight) {
             uint4 xv[kInFlight], rv[kInFlight];
