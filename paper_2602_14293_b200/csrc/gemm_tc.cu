@@ -1044,6 +1044,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 int* pool_cnt = reinterpret_cast<int*>(xchg) + half * 256;           // [4] emitters per warp, then the entries
                 int2* pool_tab = reinterpret_cast<int2*>(pool_cnt + 4);             // up to 65: (position | flags, window)
                 int n_emit = 0;
+                int my_pos[2] = {-1, -1}, my_win[2] = {0, 0};   // 16-bit output: this quarter warp's windows (position of the upper left, -1: none)
                 if (p.pool_whole) {
                     // Tiles of whole row pairs: the tile starts on a row pair and images are whole numbers of pairs, so
                     // the windows are the first PW column pairs of every pair of rows, numbered like the row pairs:
@@ -1053,11 +1054,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const long long pair0 = (long long) mb * ppt;
                     const long long pairs_left = (long long) (p.M / pair_len) - pair0;
                     n_emit = (int) (pairs_left < ppt ? (pairs_left > 0 ? pairs_left : 0) : ppt) * PW;   // at most 32
-                    if (q < n_emit) {
-                        const int pi = q / PW, j = q - pi * PW;
-                        pool_tab[q] = make_int2((pi * pair_len + 2 * j) | 128 | 256, (int) ((pair0 + pi) * PW + j));
+                    if (p.out_dt != FC_F32) {
+                        // 16-bit output: a quarter warp serves entries e and e + 16, which it works out for itself
+                        // (no table, no barrier)
+#pragma unroll
+                        for (int t = 0; t < 2; ++t) {
+                            const int e = (q >> 3) + 16 * t;
+                            const int pi = e / PW, j = e - pi * PW;
+                            my_pos[t] = e < n_emit ? pi * pair_len + 2 * j : -1;
+                            my_win[t] = (int) ((pair0 + pi) * PW + j);
+                        }
+                    } else {
+                        if (q < n_emit) {
+                            const int pi = q / PW, j = q - pi * PW;
+                            pool_tab[q] = make_int2((pi * pair_len + 2 * j) | 128 | 256, (int) ((pair0 + pi) * PW + j));
+                        }
+                        ptx::bar_sync(3 + half, 128);
                     }
-                    ptx::bar_sync(3 + half, 128);
                 } else {
                     int win = 0;
                     bool emit = false, right = false, vert = false;
@@ -1116,16 +1129,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // warp per entry, two channels per lane, stored as one 32-bit word where the rows allow it.
                         // (The same loop for fp32 outputs, two words per store, gained them 1 - 3 % and cost this form as
                         // much, as a branch in this loop or as a second copy of it: the fp32 form keeps the loop below.)
-                        const int c2 = (lane & 7) * 2, qwid = q >> 3;
+                        const int c2 = (lane & 7) * 2;
                         if (n0 + c2 < p.N) {
                             const bool both = pair16 || n0 + c2 + 1 < p.N;
-                            for (int e = qwid; e < n_emit; e += 16) {
-                                const int2 ent = pool_tab[e];
-                                if (!(ent.x & 256)) continue;
-                                const float* sp = stage + (ent.x & 127) * 17 + c2;
+#pragma unroll
+                            for (int t = 0; t < 2; ++t) {
+                                if (my_pos[t] < 0) continue;
+                                const float* sp = stage + my_pos[t] * 17 + c2;
                                 const float x0 = fabsf(fmaxf(fmaxf(sp[0], sp[17]), fmaxf(sp[below], sp[below + 17])));
                                 const float x1 = fabsf(fmaxf(fmaxf(sp[1], sp[18]), fmaxf(sp[below + 1], sp[below + 18])));
-                                unsigned short* dst = (unsigned short*) p.out + (long long) ent.y * p.N + n0 + c2;
+                                unsigned short* dst = (unsigned short*) p.out + (long long) my_win[t] * p.N + n0 + c2;
                                 if (!FC_DBG_IN(dst, both ? 4 : 2, p.out, (long long) p.batch * PH * PW * p.N * 2, p.status, kSitePoolMax)) continue;
                                 const unsigned short h0 = p.out_dt == FC_BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(x0)) : __half_as_ushort(__float2half_rn(x0));
                                 const unsigned short h1 = p.out_dt == FC_BF16 ? __bfloat16_as_ushort(__float2bfloat16_rn(x1)) : __half_as_ushort(__float2half_rn(x1));
