@@ -1069,6 +1069,30 @@ def test_conv_channel_first_equals_channel_last_bitwise(fc):
     assert torch.equal(a[0], b[0])
 
 
+@pytest.mark.parametrize("shape", [(4, 20, 12, 72, 136, 3, 3, 1), (3, 32, 32, 8, 64, 5, 5, 0), (70, 8, 8, 64, 64, 3, 3, 1)])
+def test_conv_channel_first_pooled_in_16_bits(fc, orc, shape):
+    """Channel-first operands with the max-pool stored in bf16: the layout pre-pass in front, tiles of whole row pairs
+    behind it; the same bits as the channels-last chain on the permuted arrays, and the oracle's values."""
+    batch, H, W, Cin, Cout, R, S, pad = shape
+    base = replace(wl.conv_bias_relu_maxpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, pad=pad), out_dtype="bf16")
+    ch = wl.conv_nchw(base)
+    ins = wl.make_inputs(ch, 5)
+    a, _, _ = run_and_check(fc, orc, ch, ins=ins)
+    assert a[0].dtype == torch.bfloat16 and "zero_fill" not in fc.fc_last_plan()
+    ins_cl = [np.ascontiguousarray(ins[0].transpose(0, 2, 3, 1)), np.ascontiguousarray(ins[1].transpose(0, 2, 3, 1))] + ins[2:]
+    b = util.poison_(fc.binding.output_tensors(base, "cuda"))
+    fc.run_chain(base, [fc.to_device(x) for x in ins_cl], b)
+    fc.fc_get_async_status()
+    assert torch.equal(a[0], b[0])
+    # and through host buffers: the 16-bit pooled output comes back as it was stored
+    host_in = [fc.to_device(x, "cpu").pin_memory() for x in ins_cl]
+    outs = util.poison_(fc.binding.output_tensors(base, "cpu", pinned=True))
+    staging = torch.empty(fc.fc_staging_size(fc.make_spec(base), host_in, outs), dtype=torch.uint8, device="cuda")
+    fc.run_chain_host(base, host_in, outs, staging)
+    fc.fc_get_async_status()
+    assert torch.equal(outs[0], b[0].cpu())
+
+
 def test_conv_channel_first_f16_and_host_path(fc, orc):
     ch = _as_f16(wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=5, H=12, W=10, Cin=64, Cout=64)))
     run_and_check(fc, orc, ch, 2)
