@@ -109,3 +109,42 @@ def test_random_chain(fc, orc, seed):
             (util.check_bf16 if t.dtype == torch.bfloat16 else util.check_f16)(got / scale, want / scale, what)
         else:
             util.check_f32(got, want, what)
+
+
+def _random_maxpool_chain(r):
+    """Convolution -> random ops ending in ReLU -> 2x2 max-pool, every filter / stride / padding / channel mix of the
+    generator above; the pooled output in 16 bits wherever the library takes it (even row count, at most 64 columns)."""
+    for _ in range(100):
+        R, S = int(r.choice([1, 3, 5])), int(r.choice([1, 3, 5]))
+        pad, stride = int(r.integers(0, min(R, S))), int(r.choice([1, 1, 2]))
+        H, W = int(r.integers(max(R, 4), 40)), int(r.integers(max(S, 4), 72))
+        Cin, Cout, batch = int(r.choice([8, 16, 64, 72])), int(r.choice([8, 40, 64, 128, 136])), int(r.integers(1, 9))
+        base = wl.conv_bias_relu_maxpool(batch=batch, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, stride=stride, pad=pad)
+        if base.OH >= 2 and base.OW >= 2:
+            break
+    rec = base.input_recipe + (("v1", "bf16", (Cout,), "normal", 1.0, 0.1),)
+    ops = tuple(o for o in _random_ops(r, [2, 3], None, 3) if o[0] != "relu") + (("relu",),)
+    out_dt = "f32"
+    if base.OH % 2 == 0 and base.OW <= 64:
+        out_dt = str(r.choice(["f32", "bf16", "f16"]))
+    in_dt = "f16" if out_dt == "f16" else "bf16"
+    rec = tuple((t, in_dt if d == "bf16" else d, sh, dist, a, b) for t, d, sh, dist, a, b in rec)
+    return replace(base, ops=ops, input_recipe=rec, in_dtype=in_dt, out_dtype=out_dt)
+
+
+@pytest.mark.parametrize("seed", range(64))
+def test_random_maxpool_chain(fc, orc, seed):
+    r = np.random.default_rng(5000 + seed)
+    ch = _random_maxpool_chain(r)
+    ins = wl.make_inputs(ch, seed)
+    ref = orc.run_chain(ch, ins)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    t = outs[0]
+    assert t.dtype == {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[ch.out_dtype]
+    what = f"seed {seed}: {ch.batch}x{ch.H}x{ch.W}x{ch.Cin}->{ch.Cout} {ch.R}x{ch.S} s{ch.stride} p{ch.pad} {[o[0] for o in ch.ops]} -> {ch.out_dtype}"
+    got, want = util.to_f64(t), ref["reduce"]
+    scale = max(1.0, float(np.sqrt(np.mean(want * want))))
+    check = {"f32": util.check_f32, "bf16": util.check_bf16, "f16": util.check_f16}[ch.out_dtype]
+    check(got / scale, want / scale, what)
