@@ -90,6 +90,10 @@ void note_kernel(const char* name);
 cudaError_t launch_cfirst_to_clast(const void* src, void* dst, long long mats, int C, int P, bool beside_previous, cudaStream_t stream,
                                    int* launches);
 
+// Channels-last 16-bit image [batch][H][W][C] -> the same with a zero border of `pad` pixels (layout.cu).  C a multiple of 8.
+cudaError_t launch_pad_image(const void* src, void* dst, long long batch, int H, int W, int C, int pad, int num_sms, cudaStream_t stream,
+                             int* launches);
+
 // Second pass of a wide GEMM + row softmax: per row, merges the tiles' (max, sum) pairs and rescales the stored
 // exponentials of tile j by 2^((max_j - max_row) log2 e) / sum_row, in place.  `bn` = tile width in columns.
 cudaError_t launch_softmax_rescale(void* out, int out_dt, const float2* stats, long long M, long long N, int tiles_n, int bn,

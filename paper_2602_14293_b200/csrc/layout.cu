@@ -217,6 +217,39 @@ cudaError_t launch_split_tf32(const float* x, float* y, long long rows, long lon
     return cudaLaunchKernelEx(&cfg, split_tf32_kernel, x, y, rows, (int) K, is_b ? 1 : 0);
 }
 
+// A channels-last image with its zero border written out: [batch][H + 2 pad][W + 2 pad][C], C a multiple of 8
+// (16-byte copies).  See padded_rows in fc_api.cu.
+__global__ void __launch_bounds__(256) pad_image_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, long long batch, int H, int W,
+                                                        int c8, int pad) {
+    const int Hp = H + 2 * pad, Wp = W + 2 * pad;
+    const long long total = batch * Hp * Wp * c8;
+    const long long stride = (long long) gridDim.x * blockDim.x;
+    for (long long i = (long long) blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c = (int) (i % c8);
+        const long long px = i / c8;
+        const int w = (int) (px % Wp) - pad;
+        const long long t = px / Wp;
+        const int h = (int) (t % Hp) - pad;
+        const long long b = t / Hp;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (h >= 0 && h < H && w >= 0 && w < W) v = __ldg(src + ((b * H + h) * W + w) * c8 + c);
+        dst[i] = v;
+    }
+}
+
+cudaError_t launch_pad_image(const void* src, void* dst, long long batch, int H, int W, int C, int pad, int num_sms, cudaStream_t stream,
+                             int* launches) {
+    if ((C & 7) || (reinterpret_cast<uintptr_t>(src) & 15) || (reinterpret_cast<uintptr_t>(dst) & 15)) return cudaErrorInvalidValue;
+    const long long total = batch * (H + 2 * pad) * (W + 2 * pad) * (C / 8);
+    long long blocks = (total + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > (long long) num_sms * 8) blocks = (long long) num_sms * 8;
+    note_kernel("pad_image");
+    pad_image_kernel<<<(unsigned) blocks, 256, 0, stream>>>((const uint4*) src, (uint4*) dst, batch, H, W, C / 8, pad);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_zero_fill(void* ptr, size_t bytes, int num_sms, cudaStream_t stream, int* launches) {
     const size_t words = bytes / 4;
     size_t blocks = (words / 4 + 255) / 256;

@@ -42,6 +42,22 @@ def run_and_check(fc, orc, ch, seed=0, ins=None, tag=""):
     return outs, ref, res
 
 
+def run_without_workspace(fc, orc, ch, seed=0, ins=None):
+    """The same through fc_run with no workspace registered: the forms that need no scratch (an eight-channel image
+    with padding then takes eight filter taps per k-block instead of the bordered copy + filter rows)."""
+    if ins is None:
+        ins = wl.make_inputs(ch, seed)
+    ref = orc.run_chain(ch, ins) if orc is not None else None
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.binding.fc_set_workspace(None)
+    fc.binding.fc_run(fc.make_spec(ch), [fc.to_device(a) for a in ins], outs)
+    fc.fc_get_async_status()
+    if ref is not None:
+        for (name, _, _), t in zip(wl.output_shapes(ch), outs):
+            util.check(t, ref[name], f"{ch.name} without workspace, seed {seed}: {name}")
+    return outs
+
+
 # ------------------------------------------------------------------ C1: strict fp32 GEMM + bias + ReLU
 @pytest.mark.parametrize("seed", [0, 1, 2])
 @pytest.mark.parametrize("variant", ["std", "var"])
@@ -745,7 +761,13 @@ def test_conv_eight_channels_packs_filter_taps(fc, orc, R, S, pad, stride, pool)
     ch = make(batch=3, H=17, W=22, Cin=8, Cout=40, R=R, S=S, pad=pad, stride=stride)
     if pool == "max" and (ch.OH < 2 or ch.OW < 2):
         pytest.skip("no 2 x 2 window")
+    run_without_workspace(fc, orc, ch, 9)
+    if S == 1 or pad > 0:
+        assert "gemm_tc_mode4" in fc.fc_last_plan()
+    # with a workspace the padded shapes of more than one column run on a bordered copy of the image, a filter row per k-block
     run_and_check(fc, orc, ch, 9)
+    if S > 1 and pad > 0:
+        assert fc.fc_last_plan().startswith("pad_image ") and fc.fc_last_plan().endswith("_rowtaps")
 
 
 @pytest.mark.parametrize("Cin,R,S,stride", [(8, 5, 5, 1), (8, 3, 3, 1), (16, 3, 3, 1), (8, 7, 7, 2), (32, 2, 2, 1), (16, 4, 4, 2), (24, 3, 2, 1), (8, 1, 8, 1)])
@@ -759,10 +781,14 @@ def test_conv_few_channels_without_padding_takes_filter_rows(fc, orc, Cin, R, S,
     ch = make(batch=3, H=19, W=23, Cin=Cin, Cout=40, R=R, S=S, pad=0, stride=stride)
     run_and_check(fc, orc, ch, 11)
     assert fc.fc_last_plan().endswith("_rowtaps")
-    # with padding the same shapes keep the tap-by-tap traversal
+    # with padding the same shapes run on a bordered copy of the image (a layout pass into the workspace); without a
+    # workspace they keep the tap-by-tap traversal
     if min(R, S) > 1:
-        run_and_check(fc, orc, make(batch=2, H=19, W=23, Cin=Cin, Cout=40, R=R, S=S, pad=1, stride=stride), 11)
-        assert "rowtaps" not in fc.fc_last_plan()
+        padded = make(batch=2, H=19, W=23, Cin=Cin, Cout=40, R=R, S=S, pad=1, stride=stride)
+        run_and_check(fc, orc, padded, 11)
+        assert fc.fc_last_plan().startswith("pad_image ") and fc.fc_last_plan().endswith("_rowtaps")
+        run_without_workspace(fc, orc, padded, 11)
+        assert "rowtaps" not in fc.fc_last_plan() and "pad_image" not in fc.fc_last_plan()
 
 
 def test_conv_filter_rows_delta_taps_bit_exact(fc):
@@ -798,13 +824,18 @@ def test_conv_eight_channels_delta_taps_bit_exact(fc):
     taps = [(co % 25 // 5, co % 25 % 5, co % 8) for co in range(32)]
     for co, (r, s, c) in enumerate(taps):
         w[co, r, s, c] = 1.0
-    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
-    fc.run_chain(ch, [fc.to_device(ins[0]), fc.to_device(rng.store(w, "bf16"))], outs)
-    fc.fc_get_async_status()
     xp = np.zeros((B, H + 2 * pad, W + 2 * pad, 8), dtype=np.float32)
     xp[:, pad:pad + H, pad:pad + W] = x
     want = np.stack([np.maximum(xp[:, r:r + H, s:s + W, c], 0) for r, s, c in taps], axis=-1)
     want = want.reshape(B, H // 2, 2, W // 2, 2, 32).max(axis=(2, 4))
+    both = [ins[0], rng.store(w, "bf16")]
+    outs = run_without_workspace(fc, None, ch, ins=both)      # eight taps per k-block
+    assert "gemm_tc_mode4" in fc.fc_last_plan()
+    assert np.array_equal(outs[0].cpu().numpy(), want)
+    outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
+    fc.run_chain(ch, [fc.to_device(a) for a in both], outs)    # bordered copy + a filter row per k-block
+    fc.fc_get_async_status()
+    assert fc.fc_last_plan().startswith("pad_image ")
     assert np.array_equal(outs[0].cpu().numpy(), want)
 
 

@@ -74,7 +74,11 @@ def test_contraction_routing(fc):
     conv = wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128)
     assert _plan(fc, conv) == "zero_fill gemm_tc_mode2_bn128"
     # max-pool: tiles of whole row pairs (no zeros in front) where they pay or where the output is 16 bits wide
-    assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=2)) == "gemm_tc_mode4_bn256"
+    padded8 = wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=2)
+    assert _plan(fc, padded8) == "pad_image gemm_tc_mode2_bn256_rowtaps"           # bordered copy in the workspace, filter rows
+    fc.binding.fc_set_workspace(None)
+    fc.binding.fc_run(fc.make_spec(padded8), [fc.to_device(a) for a in wl.make_inputs(padded8, 0)], fc.binding.output_tensors(padded8, "cuda"))
+    assert fc.fc_last_plan() == "gemm_tc_mode4_bn256"                              # no workspace: eight taps per k-block
     assert _plan(fc, wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=0)) == "gemm_tc_mode2_bn256_rowtaps"
     deep = wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=64, Cout=128, R=5, S=5, pad=0)          # 25 k-blocks, row pairs of 20
     assert _plan(fc, deep) == "zero_fill gemm_tc_mode2_bn128"
