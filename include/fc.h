@@ -24,7 +24,8 @@
  *
  * Ownership.  Every tensor and the workspace are allocated and freed by the caller.  fc_run never
  * allocates device memory and never synchronises; it enqueues at most two memsets and one to four
- * kernels on the given stream and returns (two kernels: a convolution behind the kernel that zeroes
+ * kernels on the given stream (one more in front of a few-channel convolution that runs on a bordered copy
+ * of its image, see fc_workspace_size_split) and returns (two kernels: a convolution behind the kernel that zeroes
  * its pooled output -- not launched for a 2x2 max-pool over tiles of whole row pairs, which stores every
  * window once --, or a wide GEMM + ROW_SOFTMAX as the GEMM kernel and a rescaling pass; three: the
  * collapsed linear layer; four: CONV2D_NCHW with its two layout kernels).  Inputs are read-only;
@@ -259,6 +260,11 @@ fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
  * (fc_workspace_size plus a fixed region of about 20 MB; 0 for chains that never split).  A smaller
  * workspace, or none where none is required, is not an error: fc_run then never splits.  Results are
  * the same up to fp32 summation order.
+ * The size also covers one more optional use: a CONV2D_NHWC chain with padding whose filter rows are short
+ * (S > 1, S * Cin <= 64: image layers of 8 to 32 channels) runs two to three times faster on a copy of the
+ * image with its zero border written out, which fc_run makes at the head of the workspace (one more kernel
+ * in front; [batch][H + 2 pad][W + 2 pad][Cin] 16-bit elements, rounded up to 256 bytes) when the workspace
+ * has room for it.  Results are the same up to fp32 summation order.
  */
 fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
 
