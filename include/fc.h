@@ -260,11 +260,11 @@ fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
  * (fc_workspace_size plus a fixed region of about 20 MB; 0 for chains that never split).  A smaller
  * workspace, or none where none is required, is not an error: fc_run then never splits.  Results are
  * the same up to fp32 summation order.
- * The size also covers one more optional use: a CONV2D_NHWC chain with padding whose filter rows are short
+ * The size also covers one more optional use: a convolution with padding whose filter rows are short
  * (S > 1, S * Cin <= 64: image layers of 8 to 32 channels) runs two to three times faster on a copy of the
- * image with its zero border written out, which fc_run makes at the head of the workspace (one more kernel
- * in front; [batch][H + 2 pad][W + 2 pad][Cin] 16-bit elements, rounded up to 256 bytes) when the workspace
- * has room for it.  Results are the same up to fp32 summation order.
+ * image with its zero border written out, which fc_run makes in the workspace (one more kernel in front;
+ * [batch][H + 2 pad][W + 2 pad][Cin] 16-bit elements, rounded up to 256 bytes, behind the channels-last copies
+ * of CONV2D_NCHW) when the workspace has room for it.  Results are the same up to fp32 summation order.
  */
 fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
 

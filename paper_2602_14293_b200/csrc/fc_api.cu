@@ -623,15 +623,14 @@ bool row_taps(const fc_chain_spec* s) { return s->Cin % 8 == 0 && s->S > 1 && s-
 // The same shapes with padding take that form too when the caller's workspace has room for a copy of the image with its
 // zero border written out (a layout pass in front, as for channel-first operands: 85 MB for 4096 images of 32 x 32 x 8
 // with a border of 2, written in about 25 us, against 1.9 us per k-block of eight small copies in the convolution).
-// Channels-last operands only.
-bool padded_rows(const fc_chain_spec* s) {
-    return s->producer == FC_PROD_CONV2D_NHWC && s->Cin % 8 == 0 && s->S > 1 && s->S * s->Cin <= 64 && s->pad > 0;
-}
+bool padded_rows(const fc_chain_spec* s) { return s->Cin % 8 == 0 && s->S > 1 && s->S * s->Cin <= 64 && s->pad > 0; }
 size_t padded_image_bytes(const fc_chain_spec* s) {
     return ((size_t) s->batch * (s->H + 2 * s->pad) * (s->W + 2 * s->pad) * s->Cin * 2 + 255) / 256 * 256;
 }
 bool use_padded_rows(const fc_chain_spec* s, const DeviceInfo* dev) {
-    return padded_rows(s) && dev->workspace && dev->workspace_bytes >= padded_image_bytes(s);
+    // (channel-first operands: behind their channels-last copies)
+    const size_t front = s->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(s) : 0;
+    return padded_rows(s) && dev->workspace && dev->workspace_bytes >= front + padded_image_bytes(s);
 }
 // (the convolution that runs behind the border pass: the bordered image, no padding)
 fc_chain_spec bordered_spec(const fc_chain_spec* s) {
@@ -945,33 +944,35 @@ fc_status fc_run(const fc_chain_spec* spec, const fc_tensor* inputs, int n_input
             const void* image = inputs[0].ptr;
             const void* weights = inputs[1].ptr;
             size_t head = 0;   // workspace bytes in front of the split scratch
-            if (bordered) {
-                head = padded_image_bytes(user_spec);
-                {   // the copy overwrites whatever counters a previous layout kept here
-                    std::lock_guard<std::mutex> lk(g_mu);
-                    dev->counter_layout = 0;
-                }
-                if ((e = launch_pad_image(image, dev->workspace, user_spec->batch, (int) user_spec->H, (int) user_spec->W, (int) user_spec->Cin,
-                                          (int) user_spec->pad, dev->num_sms, stream, &launches)) != cudaSuccess)
-                    return cuda_fail(e, "border kernel launch");
-                image = dev->workspace;
-            }
-            if (spec->producer == FC_PROD_CONV2D_NCHW) {
-                head = nchw_workspace_bytes(spec);
+            if (user_spec->producer == FC_PROD_CONV2D_NCHW) {
+                head = nchw_workspace_bytes(user_spec);
                 if (!dev->workspace || dev->workspace_bytes < head)
                     return fail(FC_ERR_WORKSPACE, "CONV2D_NCHW needs a workspace of %zu bytes (fc_workspace_size)", head);
                 void* img_cl = dev->workspace;
-                void* w_cl = (char*) dev->workspace + nchw_image_bytes(spec);
+                void* w_cl = (char*) dev->workspace + nchw_image_bytes(user_spec);
                 {   // the copies overwrite whatever counters a previous layout kept here
                     std::lock_guard<std::mutex> lk(g_mu);
                     dev->counter_layout = 0;
                 }
-                if ((e = launch_cfirst_to_clast(weights, w_cl, spec->Cout, p.Cin, p.R * p.S, false, stream, &launches)) != cudaSuccess)
+                if ((e = launch_cfirst_to_clast(weights, w_cl, user_spec->Cout, p.Cin, p.R * p.S, false, stream, &launches)) != cudaSuccess)
                     return cuda_fail(e, "layout kernel launch");
-                if ((e = launch_cfirst_to_clast(image, img_cl, spec->batch, p.Cin, p.H * p.W, true, stream, &launches)) != cudaSuccess)
+                if ((e = launch_cfirst_to_clast(image, img_cl, user_spec->batch, p.Cin, (int) (user_spec->H * user_spec->W), true, stream, &launches)) != cudaSuccess)
                     return cuda_fail(e, "layout kernel launch");
                 image = img_cl;
                 weights = w_cl;
+            }
+            if (bordered) {
+                // (behind the channels-last copies of channel-first operands, if any)
+                void* img_b = (char*) dev->workspace + head;
+                head += padded_image_bytes(user_spec);
+                {   // the copy overwrites whatever counters a previous layout kept here
+                    std::lock_guard<std::mutex> lk(g_mu);
+                    dev->counter_layout = 0;
+                }
+                if ((e = launch_pad_image(image, img_b, user_spec->batch, (int) user_spec->H, (int) user_spec->W, (int) user_spec->Cin,
+                                          (int) user_spec->pad, dev->num_sms, stream, &launches)) != cudaSuccess)
+                    return cuda_fail(e, "border kernel launch");
+                image = img_b;
             }
             attach_split_scratch(dev, head, &p);
             if ((e = clear_counters_if_needed(dev, p, 0, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
@@ -1158,8 +1159,9 @@ fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes) {
     if ((st = validate_spec(spec, &plan))) return st;
     const bool tc = plan.kind == Plan::TC_PLAIN || plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE || plan.kind == Plan::TC_CONV;
     const size_t red = plan.kind == Plan::TC_SOFTMAX || plan.kind == Plan::TC_LSE ? reduction_workspace_bytes(plan.kind == Plan::TC_SOFTMAX, spec->M, spec->N)
-                     : spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec)
-                     : plan.kind == Plan::TC_CONV && padded_rows(spec) ? padded_image_bytes(spec) : 0;   // (the bordered copy of the image)
+                     : plan.kind == Plan::TC_CONV ? (spec->producer == FC_PROD_CONV2D_NCHW ? nchw_workspace_bytes(spec) : 0) +
+                                                     (padded_rows(spec) ? padded_image_bytes(spec) : 0)   // (the bordered copy of the image)
+                     : 0;
     *bytes = tc ? split_workspace_offset(red) + kTcSplitBytes : 0;
     return FC_OK;
 }
@@ -1188,13 +1190,13 @@ fc_status fc_describe_plan(const fc_chain_spec* spec, char* text, size_t capacit
     size_t red = 0;
     fc_chain_spec border_spec;
     if (plan.kind == Plan::TC_CONV) {
+        if (spec->producer == FC_PROD_CONV2D_NCHW) red = nchw_workspace_bytes(spec);
         if (use_padded_rows(spec, dev)) {
-            red = padded_image_bytes(spec);
+            red += padded_image_bytes(spec);
             border_spec = bordered_spec(spec);
             spec = &border_spec;
         }
         bn = conv_params(spec, plan.out_rows, &p);
-        if (spec->producer == FC_PROD_CONV2D_NCHW) red = nchw_workspace_bytes(spec);
     } else {
         p.mode = plan.kind == Plan::TC_SOFTMAX ? 1 : (plan.kind == Plan::TC_LSE ? 3 : 0);
         p.M = (int) spec->M; p.N = (int) spec->N; p.K = (int) spec->K;

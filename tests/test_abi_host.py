@@ -171,11 +171,13 @@ def test_workspace_size_of_channel_first_convolution(fc):
     spec = fc.make_spec(ch)
     assert b.fc_workspace_size(spec) == img + wts
     scratch = b.fc_workspace_size_split(fc.make_spec(wl.conv_bias_relu_avgpool(batch=3, H=7, W=9, Cin=64, Cout=24)))   # split scratch alone
-    assert b.fc_workspace_size_split(spec) == img + wts + scratch
-    assert b.fc_workspace_size(fc.make_spec(base)) == 0
-    # channels-last, few channels, padding: room (optional) for the image with its zero border written out
+    # few channels with padding: room (optional) for the image with its zero border written out, behind the channels-last copies
     bordered = (3 * 9 * 11 * 8 * 2 + 255) // 256 * 256
+    assert b.fc_workspace_size_split(spec) == img + wts + bordered + scratch
+    assert b.fc_workspace_size(fc.make_spec(base)) == 0
     assert b.fc_workspace_size_split(fc.make_spec(base)) == bordered + scratch
+    wide = wl.conv_nchw(wl.conv_bias_relu_avgpool(batch=3, H=7, W=9, Cin=64, Cout=24))
+    assert b.fc_workspace_size_split(fc.make_spec(wide)) == b.fc_workspace_size(fc.make_spec(wide)) + scratch
     assert b.fc_describe_plan is not None
 
 

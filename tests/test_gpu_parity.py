@@ -1082,6 +1082,9 @@ def test_conv_channel_first(fc, orc, batch, H, W, Cin, Cout, R, S, pad, stride, 
     if pool == "max" and (ch.OH < 2 or ch.OW < 2):
         pytest.skip("no 2 x 2 window")
     run_and_check(fc, orc, ch, 21)
+    # few channels with padding: the bordered copy of the image follows the channels-last rewrite
+    assert ("pad_image" in fc.fc_last_plan()) == (S > 1 and S * Cin <= 64 and pad > 0)
+    assert fc.fc_last_plan().startswith("cfirst_to_clast cfirst_to_clast ")
 
 
 def test_conv_channel_first_equals_channel_last_bitwise(fc):
