@@ -261,7 +261,7 @@ fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
  * workspace, or none where none is required, is not an error: fc_run then never splits.  Results are
  * the same up to fp32 summation order.
  * The size also covers one more optional use: a convolution with padding whose filter rows are short
- * (S > 1, S * Cin <= 64: image layers of 8 to 32 channels) runs two to three times faster on a copy of the
+ * (image layers of 8 to 32 channels: 5 x 5 x 8, 7 x 7 x 8, 3 x 3 x 16, 5 x 5 x 16) runs up to three times faster on a copy of the
  * image with its zero border written out, which fc_run makes in the workspace (one more kernel in front;
  * [batch][H + 2 pad][W + 2 pad][Cin] 16-bit elements, rounded up to 256 bytes, behind the channels-last copies
  * of CONV2D_NCHW) when the workspace has room for it.  Results are the same up to fp32 summation order.

@@ -619,11 +619,21 @@ fc_status encode_scale_tiles(CUtensorMap* tm, const void* ptr, long long tile_ro
 // tile holds there (the next filter row's) meet zeros.  A k-block per filter row: 5 x 5 x 8 costs 5 k-blocks of one
 // copy each instead of 4 of eight 16-byte-row copies (measured: 1.9 us per such k-block in the TMA unit).  Not with
 // padding: a position whose first tap lies left of the image would lose its whole row, not just that tap.
-bool row_taps(const fc_chain_spec* s) { return s->Cin % 8 == 0 && s->S > 1 && s->S * s->Cin <= 64 && s->pad == 0; }
+// Longer filter rows (16 channels x 5 taps, 32 x 3) go in 64-element pieces, as long as that makes fewer k-blocks than a
+// k-block per tap does (channel counts below 64 that do not divide it evenly into taps: 5 x 5 x 16 takes 10 instead of 25).
+bool short_rows(const fc_chain_spec* s) {
+    return s->Cin % 8 == 0 && s->Cin < 64 && s->S > 1 && s->S * s->Cin <= 256 && (s->S * s->Cin + 63) / 64 < s->S;
+}
+bool row_taps(const fc_chain_spec* s) { return short_rows(s) && s->pad == 0; }
 // The same shapes with padding take that form too when the caller's workspace has room for a copy of the image with its
 // zero border written out (a layout pass in front, as for channel-first operands: 85 MB for 4096 images of 32 x 32 x 8
 // with a border of 2, written in about 25 us, against 1.9 us per k-block of eight small copies in the convolution).
-bool padded_rows(const fc_chain_spec* s) { return s->Cin % 8 == 0 && s->S > 1 && s->S * s->Cin <= 64 && s->pad > 0; }
+// (the border pass is one more trip over the image: worth it against the eight small copies of an eight-channel
+// k-block, 1.9 us each, and where the pieces are at most half as many as the taps: 3 x 3 x 32 on 256 images of 56 x 56,
+// 6 k-blocks instead of 9, measured 143 against 146 us into 64 channels and 186 against 169 into 128)
+bool padded_rows(const fc_chain_spec* s) {
+    return short_rows(s) && s->pad > 0 && (s->Cin == 8 || 2 * ((s->S * s->Cin + 63) / 64) <= s->S);
+}
 size_t padded_image_bytes(const fc_chain_spec* s) {
     return ((size_t) s->batch * (s->H + 2 * s->pad) * (s->W + 2 * s->pad) * s->Cin * 2 + 255) / 256 * 256;
 }
@@ -696,7 +706,7 @@ int conv_params(const fc_chain_spec* spec, long long out_rows, TcParams* p) {
     // where a tile's few k-blocks leave the epilogue in the open (a 5 x 5 x 8 -> 64 image layer 640 against 664 us).
     // Elsewhere the up to 14 % more tiles cost more than the few atomics left (5 x 5 x 64 -> 128 at OW = 10: 208.9
     // against 203.6 us).  16-bit outputs always: they cannot be reached through atomics.
-    const int kbs = row_taps(spec) ? (int) spec->R : (packed_taps(spec) ? (int) ((spec->R * spec->S * spec->Cin + 63) / 64) : (int) (spec->R * spec->S * ((spec->Cin + 63) / 64)));
+    const int kbs = row_taps(spec) ? (int) (spec->R * ((spec->S * spec->Cin + 63) / 64)) : (packed_taps(spec) ? (int) ((spec->R * spec->S * spec->Cin + 63) / 64) : (int) (spec->R * spec->S * ((spec->Cin + 63) / 64)));
     const bool pays = 128 % (2 * p->OW) == 0 || p->OW > 32 || kbs <= 8;
     if (whole_ok && (forced == 3 || (forced == 0 && pays) || must)) {
         p->pool = 2;

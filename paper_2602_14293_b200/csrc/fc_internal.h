@@ -134,9 +134,9 @@ struct TcParams {
     int after_zero_fill;        // mode 2: launched programmatically behind the kernel that zeroes `out`; the epilogue warps wait
                                 // for that kernel before their first update of `out`, everything else starts at once
     int a_packed;               // mode 2: 1 = a k-block of A is eight 8-channel chunks, one per filter tap (Cin == 8)
-    int a_rowtaps;              // mode 2: 1 = a k-block is one filter row: the S taps x Cin channels of a row are S * Cin <= 64
-                                // contiguous elements in channels-last storage, fetched as one "pixel" of a tensor map whose
-                                // pixels overlap (see row_taps in fc_api.cu)
+    int a_rowtaps;              // mode 2: 1 = a k-block is one filter row, or a 64-element piece of one: the S taps x Cin
+                                // channels of a row are S * Cin contiguous elements in channels-last storage, fetched as
+                                // (a piece of) one "pixel" of a tensor map whose pixels overlap (see row_taps in fc_api.cu)
     int* status;                // device status word
     long long dbg_trim;         // debug build: bytes by which the checks believe the main output to be shorter (testing)
     int expect_extra;           // testing only: arrivals a wait expects beyond those that will come (mode 1: the panel

@@ -210,7 +210,7 @@ template <int MODE>
 __host__ __device__ __forceinline__ int count_kb(const TcParams& p) {
     if (MODE == 7) return (p.K + BK / 2 - 1) / (BK / 2);   // 32-bit operands: 32 elements fill a 128-byte row
     if (MODE == 4) return (p.R * p.S * p.Cin + BK - 1) / BK;
-    if (MODE == 5) return p.R;   // a k-block per filter row (TcParams::a_rowtaps)
+    if (MODE == 5) return p.R * ((p.S * p.Cin + BK - 1) / BK);   // filter rows in 64-element pieces (TcParams::a_rowtaps)
     if (MODE == 2) return p.R * p.S * ((p.Cin + BK - 1) / BK);
     const int bk = p.in_dt == FC_F8E4M3 ? 2 * BK : BK;
     return (p.K + bk - 1) / bk;
@@ -319,10 +319,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tap_s = tap - tap_r * p.S;
                     tap_col = tap * p.Cin;
                 } else if constexpr (MODE == 5) {
-                    // a k-block per filter row: all S taps of the row in one copy (tap offset (0, r)), the row's
-                    // S * Cin weights from column r * S * Cin on
-                    tap_r = w.kb0;
-                    tap_col = w.kb0 * p.S * p.Cin;
+                    // k-blocks are 64-element pieces of filter rows (one piece where S * Cin <= 64): the S taps of row
+                    // r from element c0 on in one copy (tap offset (0, r), channel c0 of the wide "pixel"), the
+                    // weights from column r * S * Cin + c0 on
+                    const int per_row = (p.S * p.Cin + BK - 1) / BK;
+                    tap_r = w.kb0 / per_row;
+                    c0 = (w.kb0 - tap_r * per_row) * BK;
+                    tap_col = tap_r * p.S * p.Cin + c0;
                 }
                 for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     const uint32_t s = hs, ph = hph;
@@ -369,10 +372,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
                         }
                     } else if constexpr (MODE == 5) {
-                        ptx::tma_load_im2col_4d_pair(sa, &tmA, 0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) 0, (uint16_t) tap_r, full);
+                        ptx::tma_load_im2col_4d_pair(sa, &tmA, c0, ow * p.stride - p.pad, oh * p.stride - p.pad, img, (uint16_t) 0, (uint16_t) tap_r, full);
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, tap_col, bcol0, full);
-                        tap_col += p.S * p.Cin;
-                        ++tap_r;
+                        c0 += BK;
+                        tap_col += BK;
+                        if (c0 >= p.S * p.Cin) {
+                            c0 = 0;
+                            ++tap_r;
+                            tap_col = tap_r * p.S * p.Cin;
+                        }
                     } else {
                         ptx::tma_load_2d_pair(sa, &tmA, kb * bk, row0, full);
                         ptx::tma_load_2d_pair(sa + C::kABytes, &tmB, kb * bk, bcol0, full);

@@ -770,10 +770,12 @@ def test_conv_eight_channels_packs_filter_taps(fc, orc, R, S, pad, stride, pool)
         assert fc.fc_last_plan().startswith("pad_image ") and fc.fc_last_plan().endswith("_rowtaps")
 
 
-@pytest.mark.parametrize("Cin,R,S,stride", [(8, 5, 5, 1), (8, 3, 3, 1), (16, 3, 3, 1), (8, 7, 7, 2), (32, 2, 2, 1), (16, 4, 4, 2), (24, 3, 2, 1), (8, 1, 8, 1)])
+@pytest.mark.parametrize("Cin,R,S,stride", [(8, 5, 5, 1), (8, 3, 3, 1), (16, 3, 3, 1), (8, 7, 7, 2), (32, 2, 2, 1), (16, 4, 4, 2), (24, 3, 2, 1), (8, 1, 8, 1),
+                                             # rows of more than 64 elements, in 64-element pieces: 80, 96, 120 (two pieces), 72, 168 (three)
+                                             (16, 5, 5, 1), (32, 3, 3, 1), (40, 3, 3, 1), (8, 3, 9, 1), (24, 2, 7, 2)])
 @pytest.mark.parametrize("pool", ["avg", "max"])
 def test_conv_few_channels_without_padding_takes_filter_rows(fc, orc, Cin, R, S, stride, pool):
-    """Unpadded convolutions of few input channels (S * Cin <= 64): a k-block is one filter row, fetched as one copy
+    """Unpadded convolutions of few input channels: a k-block is one filter row (or a 64-element piece of one), fetched as one copy
     through a tensor map whose "pixels" are S * Cin channels wide and overlap (what the 64-element box asks for beyond
     them is out of range and arrives as zeros).  Ragged images, strides, both poolings; the last image's last rows sit
     at the end of the tensor."""
@@ -786,20 +788,25 @@ def test_conv_few_channels_without_padding_takes_filter_rows(fc, orc, Cin, R, S,
     if min(R, S) > 1:
         padded = make(batch=2, H=19, W=23, Cin=Cin, Cout=40, R=R, S=S, pad=1, stride=stride)
         run_and_check(fc, orc, padded, 11)
-        assert fc.fc_last_plan().startswith("pad_image ") and fc.fc_last_plan().endswith("_rowtaps")
+        # (where the pieces are more than half as many as the taps the border pass does not pay: tap by tap)
+        pays = Cin == 8 or 2 * ((S * Cin + 63) // 64) <= S
+        assert (fc.fc_last_plan().startswith("pad_image ") and fc.fc_last_plan().endswith("_rowtaps")) == pays
         run_without_workspace(fc, orc, padded, 11)
         assert "rowtaps" not in fc.fc_last_plan() and "pad_image" not in fc.fc_last_plan()
 
 
-def test_conv_filter_rows_delta_taps_bit_exact(fc):
+@pytest.mark.parametrize("Cin,R,S", [(8, 5, 5), (16, 5, 5), (32, 3, 3), (40, 3, 3), (24, 2, 7)])
+def test_conv_filter_rows_delta_taps_bit_exact(fc, Cin, R, S):
     """One-hot filters pin which tap and channel every column of a filter-row k-block multiplies: output channel co
-    copies input channel c shifted by (r, s), exactly (average over the image of ReLU of the shifted channel)."""
-    B, H, W, R, S = 2, 12, 14, 5, 5
-    ch = replace(wl.conv_bias_relu_maxpool(batch=B, H=H, W=W, Cin=8, Cout=32, R=R, S=S, pad=0), ops=(("relu",),))
+    copies input channel c shifted by (r, s), exactly (pooled ReLU of the shifted channel).  Rows of more than 64
+    elements go in pieces: every piece of every row gets taps."""
+    B, H, W = 2, 12, 14
+    Cout = 3 * R * S + 5
+    ch = replace(wl.conv_bias_relu_maxpool(batch=B, H=H, W=W, Cin=Cin, Cout=Cout, R=R, S=S, pad=0), ops=(("relu",),))
     ins = wl.make_inputs(ch, 4)
     x = rng.bf16_bits_to_f32(ins[0])
-    w = np.zeros((32, R, S, 8), dtype=np.float32)
-    taps = [(co % 25 // 5, co % 25 % 5, (3 * co) % 8) for co in range(32)]
+    w = np.zeros((Cout, R, S, Cin), dtype=np.float32)
+    taps = [(co % (R * S) // S, co % (R * S) % S, (7 * co + co // (R * S)) % Cin) for co in range(Cout)]
     for co, (r, s, c) in enumerate(taps):
         w[co, r, s, c] = 1.0
     outs = util.poison_(fc.binding.output_tensors(ch, "cuda"))
@@ -808,7 +815,7 @@ def test_conv_filter_rows_delta_taps_bit_exact(fc):
     assert fc.fc_last_plan().endswith("_rowtaps")
     OH, OW = H - R + 1, W - S + 1
     want = np.stack([np.maximum(x[:, r:r + OH, s:s + OW, c], 0) for r, s, c in taps], axis=-1)
-    want = want.reshape(B, OH // 2, 2, OW // 2, 2, 32).max(axis=(2, 4))
+    want = want[:, :OH // 2 * 2, :OW // 2 * 2].reshape(B, OH // 2, 2, OW // 2, 2, Cout).max(axis=(2, 4))
     assert np.array_equal(outs[0].cpu().numpy(), want)
 
 
@@ -1083,7 +1090,8 @@ def test_conv_channel_first(fc, orc, batch, H, W, Cin, Cout, R, S, pad, stride, 
         pytest.skip("no 2 x 2 window")
     run_and_check(fc, orc, ch, 21)
     # few channels with padding: the bordered copy of the image follows the channels-last rewrite
-    assert ("pad_image" in fc.fc_last_plan()) == (S > 1 and S * Cin <= 64 and pad > 0)
+    short_rows = Cin < 64 and S > 1 and S * Cin <= 256 and (S * Cin + 63) // 64 < S
+    assert ("pad_image" in fc.fc_last_plan()) == (short_rows and pad > 0 and (Cin == 8 or 2 * ((S * Cin + 63) // 64) <= S))
     assert fc.fc_last_plan().startswith("cfirst_to_clast cfirst_to_clast ")
 
 
