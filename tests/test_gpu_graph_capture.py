@@ -32,6 +32,7 @@ def fc():
     lambda: wl.conv_bias_relu_avgpool(batch=2, H=14, W=14, Cin=64, Cout=128),
     lambda: wl.conv_bias_relu_maxpool(batch=3, H=15, W=14, Cin=64, Cout=128, R=3, S=3, pad=1),   # zero fill + atomics
     lambda: replace(wl.conv_bias_relu_maxpool(batch=9, H=14, W=14, Cin=8, Cout=64, R=5, S=5, pad=0), out_dtype="bf16"),   # one launch, pooled in bf16 (poisoned before every replay)
+    lambda: wl.conv_bias_relu_avgpool(batch=5, H=17, W=15, Cin=8, Cout=64, R=5, S=5, pad=2),   # border pass into the workspace + zero fill + convolution
     lambda: wl.linear_row_reduce(96, 512, 256, variant="var"),             # three kernels
     lambda: wl.gemm_bias_relu_f32(1030, 1100, 512, "var"),                 # fp32 on the tensor cores: two split launches + the GEMM
     lambda: wl.gemm_softmax(600, 4000, 4096, "var"),                       # single-pass softmax on 240-column tiles
