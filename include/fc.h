@@ -264,7 +264,7 @@ fc_status fc_set_workspace(void* dev_ptr, size_t bytes);
  * (image layers of 8 to 32 channels: 5 x 5 x 8, 7 x 7 x 8, 3 x 3 x 16, 5 x 5 x 16) runs up to three times faster on a copy of the
  * image with its zero border written out, which fc_run makes in the workspace (one more kernel in front;
  * [batch][H + 2 pad][W + 2 pad][Cin] 16-bit elements, rounded up to 256 bytes, behind the channels-last copies
- * of CONV2D_NCHW) when the workspace has room for it.  Results are the same up to fp32 summation order.
+ * of CONV2D_NCHW) when the workspace has room for it and the problem is large enough for the extra launch to pay.  Results are the same up to fp32 summation order.
  */
 fc_status fc_workspace_size_split(const fc_chain_spec* spec, size_t* bytes);
 
@@ -340,6 +340,8 @@ int fc_version(void);
 #define FC_TESTING_POOL_FORM 4     /* value 1, 2 or 3: the form of the 2x2 max-pool behind a convolution (1: every window through
                                       atomics; 2: windows inside a tile finished on chip; 3: tiles of whole row pairs, where the
                                       shape allows them, else the launcher's own); 0: the launcher's own */
+#define FC_TESTING_BORDER_PASS 5   /* value 1: a few-channel convolution with padding runs on the bordered copy of its image
+                                      whenever the workspace has room, whatever its size (0: from about eight rounds of tiles on) */
 void fc_testing_set(int which, int value);
 
 #ifdef __cplusplus

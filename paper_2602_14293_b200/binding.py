@@ -106,7 +106,7 @@ def fc_last_plan() -> str:
     return lib().fc_last_plan().decode()
 
 
-FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL, FC_TESTING_BOUNDS_TRIP, FC_TESTING_TILE_WIDTH, FC_TESTING_POOL_FORM = 0, 1, 2, 3, 4
+FC_TESTING_PANEL_STALL, FC_TESTING_SPLIT_STALL, FC_TESTING_BOUNDS_TRIP, FC_TESTING_TILE_WIDTH, FC_TESTING_POOL_FORM, FC_TESTING_BORDER_PASS = 0, 1, 2, 3, 4, 5
 
 
 def fc_testing_set(which: int, value: int) -> None:

@@ -76,6 +76,16 @@ def test_contraction_routing(fc):
     # max-pool: tiles of whole row pairs (no zeros in front) where they pay or where the output is 16 bits wide
     padded8 = wl.conv_bias_relu_maxpool(batch=2, H=14, W=14, Cin=8, Cout=264, R=5, S=5, pad=2)
     assert _plan(fc, padded8) == "pad_image gemm_tc_mode2_bn256_rowtaps"           # bordered copy in the workspace, filter rows
+    # ... by the library's own rule only from some eight rounds of tiles on (the border pass is a launch of its own)
+    fc.binding.fc_testing_set(fc.binding.FC_TESTING_BORDER_PASS, 0)
+    try:
+        assert _plan(fc, padded8) == "gemm_tc_mode4_bn256"
+        big = wl.conv_bias_relu_maxpool(batch=1024, H=32, W=32, Cin=8, Cout=32, R=3, S=3, pad=1)     # 4096 tiles
+        assert _plan(fc, big) == "pad_image gemm_tc_mode2_bn64_rowtaps"
+        small = wl.conv_bias_relu_maxpool(batch=64, H=32, W=32, Cin=8, Cout=32, R=3, S=3, pad=1)      # 256 tiles
+        assert _plan(fc, small) == "gemm_tc_mode4_bn64"
+    finally:
+        fc.binding.fc_testing_set(fc.binding.FC_TESTING_BORDER_PASS, 1)
     fc.binding.fc_set_workspace(None)
     fc.binding.fc_run(fc.make_spec(padded8), [fc.to_device(a) for a in wl.make_inputs(padded8, 0)], fc.binding.output_tensors(padded8, "cuda"))
     assert fc.fc_last_plan() == "gemm_tc_mode4_bn256"                              # no workspace: eight taps per k-block
